@@ -1,0 +1,220 @@
+"""CPU oracle for the Qift quantized linear layer -- TEST INFRASTRUCTURE ONLY.
+
+A ctypes front end to ``qift_oracle.cpp`` (plain single-threaded C++17, compiled with
+``g++ -O2 -ffp-contract=off``).  The oracle restates what the paper's layer computes; it shares no
+code with the CUDA library and must never be imported by it.  Only tests, the smoke check and the
+CPU-baseline / reference legs of the benchmark may use this package.
+
+All arrays are numpy, C-contiguous.  Level-set ids: 0 MNZ {-3,-1,+1,+3} (half-scale form of
+{+-0.5,+-1.5}), 1 PoT-MNZ {-4,-1,+1,+4}, 2 SYM-INT {-2,-1,0,+1}, 3 INT4 (-8..7).
+Scale modes: 0 given, 1 max-range, 2 MSE sweep over 80 clipping ratios.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+MNZ, POT, SYM, INT4 = 0, 1, 2, 3
+SCALE_GIVEN, SCALE_ABSMAX, SCALE_MSE = 0, 1, 2
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "qift_oracle.cpp")
+_LIB = os.path.join(_HERE, "libqift_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle shared library beside its source (no-op when up to date)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-shared", "-fPIC", _SRC, "-o", _LIB]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _p(a, t):
+    return a.ctypes.data_as(ctypes.POINTER(t))
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.orc_candidate_ratio.restype = ctypes.c_float
+        _lib.orc_row_sqerr.restype = ctypes.c_double
+        _lib.orc_row_sqerr.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_float]
+        _lib.orc_int_matmul.restype = ctypes.c_longlong
+    return _lib
+
+
+def _f32(a):
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def level_value(lv: int, code: int) -> int:
+    return int(lib().orc_level_value(int(lv), int(code)))
+
+
+def level_table(lv: int):
+    return [level_value(lv, c) for c in range(16 if lv == INT4 else 4)]
+
+
+def num_candidates() -> int:
+    return int(lib().orc_num_candidates())
+
+
+def candidate_ratio(i: int) -> float:
+    return float(lib().orc_candidate_ratio(int(i)))
+
+
+def wht_blocks(x, B: int):
+    """Unnormalised blockwise Walsh-Hadamard transform of each row (fp32 butterfly)."""
+    x = _f32(x).copy()
+    rows = x.reshape(-1, x.shape[-1])
+    K = rows.shape[1]
+    assert B >= 1 and (B & (B - 1)) == 0 and K % B == 0
+    for r in rows:
+        lib().orc_wht_blocks(r.ctypes.data_as(ctypes.c_void_p), K, B)
+    return x
+
+
+def rotate_weights(W, B: int):
+    """W Q with Q = blockdiag(H_B)/sqrt(B) along the last axis (fp32)."""
+    W = _f32(W).copy()
+    N, K = W.shape
+    assert (B & (B - 1)) == 0 and K % B == 0
+    lib().orc_rotate_weights(W.ctypes.data_as(ctypes.c_void_p), N, K, B)
+    return W
+
+
+def bf16_to_f32(u16):
+    u16 = np.ascontiguousarray(u16, dtype=np.uint16)
+    out = np.empty(u16.shape, dtype=np.float32)
+    lib().orc_bf16_to_f32(u16.ctypes.data_as(ctypes.c_void_p), out.ctypes.data_as(ctypes.c_void_p),
+                          ctypes.c_longlong(u16.size))
+    return out
+
+
+def f32_to_bf16(x):
+    x = _f32(x)
+    out = np.empty(x.shape, dtype=np.uint16)
+    lib().orc_f32_to_bf16(x.ctypes.data_as(ctypes.c_void_p), out.ctypes.data_as(ctypes.c_void_p),
+                          ctypes.c_longlong(x.size))
+    return out
+
+
+def quantize_act(X, had_block: int, clip: float = 0.9):
+    """-> (q_a int8 [M,K], s_a fp32 [M])."""
+    X = _f32(X)
+    M, K = X.shape
+    assert had_block == 0 or ((had_block & (had_block - 1)) == 0 and K % had_block == 0)
+    q = np.empty((M, K), dtype=np.int8)
+    s = np.empty((M,), dtype=np.float32)
+    scratch = np.empty((K,), dtype=np.float32)
+    lib().orc_quantize_act(X.ctypes.data_as(ctypes.c_void_p), M, K, int(had_block),
+                           ctypes.c_float(clip), q.ctypes.data_as(ctypes.c_void_p),
+                           s.ctypes.data_as(ctypes.c_void_p), scratch.ctypes.data_as(ctypes.c_void_p))
+    return q, s
+
+
+def row_sqerr(w, lv: int, s: float) -> float:
+    w = _f32(w)
+    return float(lib().orc_row_sqerr(w.ctypes.data_as(ctypes.c_void_p), w.size, int(lv),
+                                     ctypes.c_float(s)))
+
+
+def weight_scale(W, lv: int, mode: int, want_errs: bool = False):
+    """-> (s_n fp32 [N], best_idx int32 [N][, errs fp64 [N,80]])."""
+    W = _f32(W)
+    N, K = W.shape
+    s = np.empty((N,), dtype=np.float32)
+    idx = np.zeros((N,), dtype=np.int32)
+    errs = np.zeros((N, num_candidates()), dtype=np.float64) if want_errs else None
+    lib().orc_weight_scale(W.ctypes.data_as(ctypes.c_void_p), N, K, int(lv), int(mode),
+                           s.ctypes.data_as(ctypes.c_void_p), idx.ctypes.data_as(ctypes.c_void_p),
+                           errs.ctypes.data_as(ctypes.c_void_p) if want_errs else None)
+    return (s, idx, errs) if want_errs else (s, idx)
+
+
+def assign_codes(W, lv: int, s_n):
+    W = _f32(W)
+    s_n = _f32(s_n)
+    N, K = W.shape
+    codes = np.empty((N, K), dtype=np.uint8)
+    lib().orc_assign_codes(W.ctypes.data_as(ctypes.c_void_p), N, K, int(lv),
+                           s_n.ctypes.data_as(ctypes.c_void_p), codes.ctypes.data_as(ctypes.c_void_p))
+    return codes
+
+
+def codes_per_word(lv: int) -> int:
+    return 8 if lv == INT4 else 16
+
+
+def pack(codes, lv: int):
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    N, K = codes.shape
+    per = codes_per_word(lv)
+    assert K % per == 0
+    out = np.empty((N, K // per), dtype=np.uint32)
+    lib().orc_pack(codes.ctypes.data_as(ctypes.c_void_p), N, K, int(lv),
+                   out.ctypes.data_as(ctypes.c_void_p))
+    return out
+
+
+def unpack(packed, K: int, lv: int):
+    packed = np.ascontiguousarray(packed, dtype=np.uint32)
+    N = packed.shape[0]
+    out = np.empty((N, K), dtype=np.uint8)
+    lib().orc_unpack(packed.ctypes.data_as(ctypes.c_void_p), N, K, int(lv),
+                     out.ctypes.data_as(ctypes.c_void_p))
+    return out
+
+
+def int_matmul(codes, lv: int, q_a):
+    """acc int32 [M,N] = sum_k level(code[n,k]) * q_a[m,k]; asserts no int32 overflow."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    q_a = np.ascontiguousarray(q_a, dtype=np.int8)
+    N, K = codes.shape
+    M, K2 = q_a.shape
+    assert K == K2
+    acc = np.empty((M, N), dtype=np.int32)
+    bad = lib().orc_int_matmul(codes.ctypes.data_as(ctypes.c_void_p), int(lv),
+                               q_a.ctypes.data_as(ctypes.c_void_p), M, N, K,
+                               acc.ctypes.data_as(ctypes.c_void_p))
+    assert bad == 0, "int32 accumulator overflow"
+    return acc
+
+
+def epilogue(acc, s_a, s_n, bf16: bool = False):
+    """y = ((float)acc * s_a[m]) * s_n[n]; fp32, or bf16 bit patterns (uint16) by RNE."""
+    acc = np.ascontiguousarray(acc, dtype=np.int32)
+    s_a = _f32(s_a)
+    s_n = _f32(s_n)
+    M, N = acc.shape
+    if bf16:
+        y = np.empty((M, N), dtype=np.uint16)
+        fn = lib().orc_epilogue_bf16
+    else:
+        y = np.empty((M, N), dtype=np.float32)
+        fn = lib().orc_epilogue
+    fn(acc.ctypes.data_as(ctypes.c_void_p), s_a.ctypes.data_as(ctypes.c_void_p),
+       s_n.ctypes.data_as(ctypes.c_void_p), M, N, y.ctypes.data_as(ctypes.c_void_p))
+    return y
+
+
+def pack_weights(W, lv: int, mode: int, s_n=None):
+    """Whole S1 step -> (packed uint32 [N, K/per], s_n, codes)."""
+    if mode == SCALE_GIVEN:
+        s = _f32(s_n)
+    else:
+        s, _ = weight_scale(W, lv, mode)
+    codes = assign_codes(W, lv, s)
+    return pack(codes, lv), s, codes
+
+
+def linear(codes, lv: int, s_n, q_a, s_a, bf16: bool = False):
+    """S4 + S5 -> (y, acc)."""
+    acc = int_matmul(codes, lv, q_a)
+    return epilogue(acc, s_a, s_n, bf16=bf16), acc

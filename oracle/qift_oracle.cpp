@@ -1,0 +1,304 @@
+// Qift rotated W2A4 / W4A4 quantized linear layer -- CPU ORACLE.
+//
+// THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a plain, slow, single-threaded C++17
+// restatement of what the paper's quantized linear layer computes, written for checking the CUDA
+// library against.  It shares no code, header, table or constant generator with the CUDA path and
+// neither includes the other.  Only tests, the smoke check and the CPU-baseline / reference legs of
+// the benchmark may call it.  Build: g++ -O2 -std=c++17 -ffp-contract=off -shared -fPIC.
+//
+// What each function follows (paper = "Qift: Shift-Friendly No-Zero W2 Post-Training Quantization
+// for Rotated W2A4/KV4 LLM Inference"):
+//   orc_level_value      Sec. 3.3 level-set list (SYM-INT, MNZ, PoT-MNZ) and Eq. 1 with b = 4;
+//                        MNZ is held in its half-scale odd-integer form {-3,-1,+1,+3} (Sec. 3.3,
+//                        the identity {-1.5,-.5,.5,1.5} s = {-3,-1,1,3} s/2).
+//   orc_wht_blocks       Sec. 3.1 / Sec. 4.1 "default Hadamard rotation": Sylvester-Walsh matrix
+//                        in natural order applied by the textbook in-place butterfly, stages in
+//                        ascending stride, fp32.
+//   orc_rotate_weights   the same rotation with the orthonormal factor 1/sqrt(B) (offline, weights).
+//   orc_quantize_act     Eq. 1 with b = 4 on the rotated row, symmetric, clipping ratio as an
+//                        argument (Sec. 4.1 uses 0.9), one scale per token row.
+//   orc_weight_scale     Sec. 3.5 / Sec. 4.5.1: per-output-channel scale, either max-range or
+//                        "MSE-optimal by sweeping candidate clipping ratios".
+//   orc_assign_codes     Sec. 3.5 "maps weights to the nearest scaled level"; Eq. 1 for SYM-INT, INT4.
+//   orc_pack / unpack    Sec. 3.3 "four two-bit codes": 16 two-bit codes (8 nibbles) per 32-bit word.
+//   orc_int_matmul       Sec. 3.6 decoded small signed integer levels times integer activations.
+//   orc_epilogue*        Sec. 1 "the per-channel scale can be applied separately in the epilogue".
+//
+// Parity pins for every function live in the CPU test-suite (closed forms, brute force, printed
+// table values); none is "parity unpinned" except the numeric value of a forward output on the real
+// models, which the paper never prints.
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+
+namespace {
+
+enum Levels { LV_MNZ = 0, LV_POT = 1, LV_SYM = 2, LV_INT4 = 3 };
+enum ScaleMode { SC_GIVEN = 0, SC_ABSMAX = 1, SC_MSE = 2 };
+
+constexpr int kNumCandidates = 80;  // clipping ratios 1.00, 0.99, ..., 0.21
+
+// Decoded integer level of a stored code.  Two-bit sets are indexed in ascending level order.
+int level_of(int lv, int code) {
+    switch (lv) {
+        case LV_MNZ: { const int t[4] = {-3, -1, +1, +3}; return t[code & 3]; }
+        case LV_POT: { const int t[4] = {-4, -1, +1, +4}; return t[code & 3]; }
+        case LV_SYM: { const int t[4] = {-2, -1, 0, +1}; return t[code & 3]; }
+        default: {  // INT4: two's-complement nibble
+            int c = code & 15;
+            return c >= 8 ? c - 16 : c;
+        }
+    }
+}
+
+// Largest positive level: the value a row's (clipped) absolute maximum is mapped onto.
+float top_level(int lv) {
+    switch (lv) {
+        case LV_MNZ: return 3.0f;
+        case LV_POT: return 4.0f;
+        case LV_SYM: return 1.0f;
+        default: return 7.0f;
+    }
+}
+
+int clampi(int v, int lo, int hi) { return v < lo ? lo : (v > hi ? hi : v); }
+
+// Nearest-level code of one weight given its channel scale.
+int code_of(int lv, float w, float s) {
+    const float t = w / s;  // IEEE fp32 division
+    if (lv == LV_MNZ) {     // decision thresholds are the midpoints -2, 0, +2; exact ties go down
+        return (t > -2.0f) + (t > 0.0f) + (t > 2.0f);
+    }
+    if (lv == LV_POT) {     // midpoints -2.5, 0, +2.5
+        return (t > -2.5f) + (t > 0.0f) + (t > 2.5f);
+    }
+    if (lv == LV_SYM) {     // Eq. 1, b = 2: round half to even, clip to [-2, 1]
+        return clampi((int)std::rint(t), -2, 1) + 2;
+    }
+    return clampi((int)std::rint(t), -8, 7) & 15;  // Eq. 1, b = 4
+}
+
+float row_absmax(const float* w, int K) {
+    float a = 0.0f;
+    for (int k = 0; k < K; ++k) {
+        const float v = std::fabs(w[k]);
+        if (v > a) a = v;
+    }
+    return a;
+}
+
+float inv_sqrt_block(int B) { return (float)(1.0 / std::sqrt((double)B)); }
+
+uint16_t bf16_rne(float f) {
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x0040u);  // NaN stays NaN
+    const uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+}  // namespace
+
+extern "C" {
+
+int orc_level_value(int lv, int code) { return level_of(lv, code); }
+
+int orc_num_candidates() { return kNumCandidates; }
+
+// Clipping ratio of sweep candidate i.
+float orc_candidate_ratio(int i) { return (float)(100 - i) / 100.0f; }
+
+// In-place unnormalised Walsh-Hadamard transform of every contiguous block of B entries of a row
+// of length K (B a power of two dividing K).  H H^T = B I.
+void orc_wht_blocks(float* row, int K, int B) {
+    for (int base = 0; base < K; base += B) {
+        float* x = row + base;
+        for (int h = 1; h < B; h <<= 1) {
+            for (int i = 0; i < B; ++i) {
+                if ((i & h) == 0) {
+                    const float a = x[i];
+                    const float b = x[i + h];
+                    x[i] = a + b;
+                    x[i + h] = a - b;
+                }
+            }
+        }
+    }
+}
+
+// W <- W Q with Q = blockdiag(H_B) / sqrt(B), applied to each row along K (H is symmetric).
+void orc_rotate_weights(float* W, int N, int K, int B) {
+    const float r = inv_sqrt_block(B);
+    for (int n = 0; n < N; ++n) {
+        float* row = W + (size_t)n * K;
+        orc_wht_blocks(row, K, B);
+        for (int k = 0; k < K; ++k) row[k] = row[k] * r;
+    }
+}
+
+void orc_bf16_to_f32(const uint16_t* in, float* out, long long n) {
+    for (long long i = 0; i < n; ++i) {
+        const uint32_t u = (uint32_t)in[i] << 16;
+        std::memcpy(&out[i], &u, 4);
+    }
+}
+
+void orc_f32_to_bf16(const float* in, uint16_t* out, long long n) {
+    for (long long i = 0; i < n; ++i) out[i] = bf16_rne(in[i]);
+}
+
+// Rotate (B > 0) and quantize each activation row to the INT4 range.
+//   u   = H_B-blocks applied to x                      (unnormalised)
+//   s_u = (amax * clip) / 7          (1 if the row is all zero)
+//   q   = clamp(rint(u / s_u), -8, 7)
+//   s_a = s_u / sqrt(B)              (the orthonormal factor is folded into the scale)
+// `scratch` holds one row (K floats).
+void orc_quantize_act(const float* X, int M, int K, int B, float clip, int8_t* q, float* s_a,
+                      float* scratch) {
+    for (int m = 0; m < M; ++m) {
+        for (int k = 0; k < K; ++k) scratch[k] = X[(size_t)m * K + k];
+        if (B > 1) orc_wht_blocks(scratch, K, B);
+        const float amax = row_absmax(scratch, K);
+        float s_u = 1.0f;
+        if (amax != 0.0f) {
+            const float clipped = amax * clip;
+            s_u = clipped / 7.0f;
+        }
+        for (int k = 0; k < K; ++k) {
+            const float t = scratch[k] / s_u;
+            q[(size_t)m * K + k] = (int8_t)clampi((int)std::rint(t), -8, 7);
+        }
+        s_a[m] = (B > 1) ? s_u * inv_sqrt_block(B) : s_u;
+    }
+}
+
+// Sum of squared reconstruction errors of one row at scale s, fp64, ascending k.
+double orc_row_sqerr(const float* w, int K, int lv, float s) {
+    double e = 0.0;
+    for (int k = 0; k < K; ++k) {
+        const int c = code_of(lv, w[k], s);
+        const double d = (double)w[k] - (double)s * (double)level_of(lv, c);
+        e += d * d;
+    }
+    return e;
+}
+
+// Per-output-channel scale.  mode 1: amax / top level.  mode 2: sweep of 80 clipping ratios,
+// smallest squared error, first index on ties.  best_idx (may be null) receives the chosen
+// candidate (0 for ABSMAX), errs (may be null, [N*80]) every candidate's error.
+void orc_weight_scale(const float* W, int N, int K, int lv, int mode, float* s_n, int* best_idx,
+                      double* errs) {
+    const float g = top_level(lv);
+    for (int n = 0; n < N; ++n) {
+        const float* w = W + (size_t)n * K;
+        const float amax = row_absmax(w, K);
+        int best = 0;
+        float s = 1.0f;
+        if (amax != 0.0f) {
+            if (mode == SC_ABSMAX) {
+                s = amax / g;
+            } else {
+                double best_e = 0.0;
+                for (int i = 0; i < kNumCandidates; ++i) {
+                    const float p = orc_candidate_ratio(i);
+                    const float clipped = p * amax;
+                    const float si = clipped / g;
+                    const double e = orc_row_sqerr(w, K, lv, si);
+                    if (errs) errs[(size_t)n * kNumCandidates + i] = e;
+                    if (i == 0 || e < best_e) {
+                        best_e = e;
+                        best = i;
+                        s = si;
+                    }
+                }
+            }
+        } else if (errs) {
+            for (int i = 0; i < kNumCandidates; ++i) errs[(size_t)n * kNumCandidates + i] = 0.0;
+        }
+        s_n[n] = s;
+        if (best_idx) best_idx[n] = best;
+    }
+}
+
+void orc_assign_codes(const float* W, int N, int K, int lv, const float* s_n, uint8_t* codes) {
+    for (int n = 0; n < N; ++n)
+        for (int k = 0; k < K; ++k)
+            codes[(size_t)n * K + k] = (uint8_t)code_of(lv, W[(size_t)n * K + k], s_n[n]);
+}
+
+// Bit position of code k inside its word.
+//   two-bit sets: word j = k / 16, inside it k = 16 j + 4 t + b  ->  bits [8 b + 2 t + 1 : 8 b + 2 t]
+//   INT4:         word j = k / 8,  inside it k =  8 j + 4 t + b  ->  bits [8 b + 4 t + 3 : 8 b + 4 t]
+// so that (word >> (bits * t)) masked per byte yields four consecutive-k codes, one per byte.
+void orc_pack(const uint8_t* codes, int N, int K, int lv, uint32_t* packed) {
+    const int per = (lv == LV_INT4) ? 8 : 16;
+    const int bits = (lv == LV_INT4) ? 4 : 2;
+    const int words = K / per;
+    for (int n = 0; n < N; ++n) {
+        for (int j = 0; j < words; ++j) {
+            uint32_t w = 0;
+            for (int r = 0; r < per; ++r) {
+                const int t = r / 4, b = r % 4;
+                const uint32_t c = codes[(size_t)n * K + (size_t)j * per + r] & ((1u << bits) - 1u);
+                w |= c << (8 * b + bits * t);
+            }
+            packed[(size_t)n * words + j] = w;
+        }
+    }
+}
+
+void orc_unpack(const uint32_t* packed, int N, int K, int lv, uint8_t* codes) {
+    const int per = (lv == LV_INT4) ? 8 : 16;
+    const int bits = (lv == LV_INT4) ? 4 : 2;
+    const int words = K / per;
+    for (int n = 0; n < N; ++n)
+        for (int k = 0; k < K; ++k) {
+            const int j = k / per, r = k % per, t = r / 4, b = r % 4;
+            codes[(size_t)n * K + k] =
+                (uint8_t)((packed[(size_t)n * words + j] >> (8 * b + bits * t)) & ((1u << bits) - 1u));
+        }
+}
+
+// acc[m][n] = sum_k level(code[n][k]) * q_a[m][k]; plain triple loop, int32 with an int64 shadow.
+// Returns the number of entries whose int32 and int64 sums differ (0 = no overflow anywhere).
+long long orc_int_matmul(const uint8_t* codes, int lv, const int8_t* q, int M, int N, int K,
+                         int32_t* acc) {
+    long long bad = 0;
+    for (int m = 0; m < M; ++m) {
+        for (int n = 0; n < N; ++n) {
+            int32_t a32 = 0;
+            int64_t a64 = 0;
+            for (int k = 0; k < K; ++k) {
+                const int L = level_of(lv, codes[(size_t)n * K + k]);
+                const int qa = (int)q[(size_t)m * K + k];
+                a32 += L * qa;
+                a64 += (int64_t)L * (int64_t)qa;
+            }
+            if ((int64_t)a32 != a64) ++bad;
+            acc[(size_t)m * N + n] = a32;
+        }
+    }
+    return bad;
+}
+
+// y = ((float)acc * s_a[m]) * s_n[n]
+void orc_epilogue(const int32_t* acc, const float* s_a, const float* s_n, int M, int N, float* y) {
+    for (int m = 0; m < M; ++m)
+        for (int n = 0; n < N; ++n) {
+            const float t = (float)acc[(size_t)m * N + n] * s_a[m];
+            y[(size_t)m * N + n] = t * s_n[n];
+        }
+}
+
+void orc_epilogue_bf16(const int32_t* acc, const float* s_a, const float* s_n, int M, int N,
+                       uint16_t* y) {
+    for (int m = 0; m < M; ++m)
+        for (int n = 0; n < N; ++n) {
+            const float t = (float)acc[(size_t)m * N + n] * s_a[m];
+            y[(size_t)m * N + n] = bf16_rne(t * s_n[n]);
+        }
+}
+
+}  // extern "C"

@@ -1,0 +1,137 @@
+/*
+ * qift.h -- C ABI of the B200 (sm_100a) library for the rotated W2A4 / W4A4 quantized linear layer
+ * of "Qift: Shift-Friendly No-Zero W2 Post-Training Quantization for Rotated W2A4/KV4 LLM Inference".
+ *
+ *     y[m,n] = s_n[n] * ( sum_k level(code[n,k]) * q_a[m,k] ) * s_a[m]
+ *
+ * Conventions that hold for every entry point unless its comment says otherwise
+ *   - every pointer is DEVICE memory owned by the caller; the library allocates nothing and keeps no
+ *     state between calls; base pointers must be 16-byte aligned;
+ *   - all work is enqueued asynchronously on `stream` (a cudaStream_t passed as void*, NULL = the
+ *     legacy default stream); nothing synchronizes;
+ *   - matrices are row-major with the last index contiguous: W [N,K], X / q_a [M,K], Y [M,N];
+ *   - the return value is a qift_status; argument, shape and alignment errors are found on the host
+ *     before anything is launched, so a failing call has touched no buffer;
+ *   - kernels are launched with programmatic stream serialization: each waits for its predecessor
+ *     in the stream before it reads or writes any caller buffer, so ordinary stream order holds.
+ */
+#ifndef QIFT_H_
+#define QIFT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    QIFT_OK = 0,
+    QIFT_ERR_INVALID_ARG = 1,       /* null pointer, non-positive size, unknown enum value          */
+    QIFT_ERR_UNSUPPORTED_SHAPE = 2, /* K not a multiple of the codes per word, had_block invalid... */
+    QIFT_ERR_ALIGNMENT = 3,         /* a base pointer is not 16-byte aligned                        */
+    QIFT_ERR_WORKSPACE = 4,         /* workspace missing or smaller than qift_workspace_bytes()     */
+    QIFT_ERR_CUDA = 5,              /* a CUDA runtime call or a launch failed                       */
+    QIFT_ERR_TIMEOUT = 6            /* a bounded device-side wait expired (see qift_device_status)  */
+} qift_status;
+
+/* Reconstruction level sets.  Two-bit codes index the levels in ascending order (code 0 = most
+ * negative); the paper leaves the code assignment to the implementation (Sec. 3.3). */
+typedef enum {
+    QIFT_LEVELS_MNZ = 0,  /* {-3,-1,+1,+3}: half-scale form of {+-0.5,+-1.5}; s_n is s/2 (Sec. 3.3) */
+    QIFT_LEVELS_POT = 1,  /* {-4,-1,+1,+4}: power-of-two mirror no-zero set          (Sec. 3.3)     */
+    QIFT_LEVELS_SYM = 2,  /* {-2,-1, 0,+1}: standard symmetric integer W2            (Eq. 1, b = 2) */
+    QIFT_LEVELS_INT4 = 3  /* -8..7 two's-complement nibble, 8 codes per word         (Eq. 1, b = 4) */
+} qift_levels;
+
+/* How the per-output-channel scale is chosen (Sec. 3.5; Sec. 4.5.1 "sweeping candidate clipping
+ * ratios").  GIVEN reads s_n; ABSMAX writes s_n = amax / top_level; MSE sweeps the 80 ratios
+ * p = 1.00, 0.99, ..., 0.21, s = (p * amax) / top_level, and keeps the first least-squared-error one.
+ * top_level is 3 (MNZ), 4 (POT), 1 (SYM), 7 (INT4).  An all-zero row gets s_n = 1. */
+typedef enum { QIFT_SCALE_GIVEN = 0, QIFT_SCALE_ABSMAX = 1, QIFT_SCALE_MSE = 2 } qift_scale_mode;
+
+typedef enum { QIFT_F32 = 0, QIFT_BF16 = 1 } qift_dtype;
+
+/* Kernel route of qift_linear_route(): AUTO picks by M. */
+typedef enum {
+    QIFT_ROUTE_AUTO = 0,
+    QIFT_ROUTE_GENERIC = 1,  /* one warp per output channel, dp4a; any M, any K                     */
+    QIFT_ROUTE_DECODE = 2,   /* bulk-copy staged, in-register decode, mma.sync; M <= 16             */
+    QIFT_ROUTE_PREFILL = 3   /* expand to int8 scratch, TMA + tcgen05 kind::i8, TMEM accumulators   */
+} qift_route;
+
+const char* qift_status_string(int status);
+
+/* Bytes of the packed weight buffer: N*K/4 for the two-bit sets, N*K/2 for INT4.  0 on bad input. */
+size_t qift_packed_bytes(int N, int K, int levels);
+
+/* Bytes of scratch qift_w2a4_linear / qift_w4a4_linear need for this problem (0 when the decode
+ * route serves it; N*K rounded up to 1 KiB for the prefill route, which expands the codes to int8). */
+size_t qift_workspace_bytes(int M, int N, int K, int levels);
+
+/* S1 (weight quantizer + packer).  Sec. 1 Eq. 1, Sec. 3.3, Sec. 3.5.
+ *   W       in   fp32 [N,K], ALREADY rotated (this call never rotates)
+ *   s_n     in for QIFT_SCALE_GIVEN (must be > 0), out otherwise; fp32 [N]
+ *   packed  out  uint32 [N, K/16] (two-bit sets) or [N, K/8] (INT4); qift_packed_bytes() bytes
+ * Code of a weight: t = w / s_n (IEEE division).  No-zero sets: nearest level, an exact midpoint
+ * goes to the lower level, values beyond the outer levels saturate.  SYM / INT4: Eq. 1 literally,
+ * round-half-to-even then clip to [-2,1] / [-8,7]; SYM stores q+2, INT4 stores q & 15.
+ * Word layout: word j of a row holds codes k = 16j..16j+15; code k = 16j + 4t + b sits at bits
+ * [8b+2t+1 : 8b+2t] (INT4: k = 8j + 4t + b at bits [8b+4t+3 : 8b+4t]), so (word >> 2t) & 0x03030303
+ * is four consecutive-k codes, one per byte.
+ * Requires K % 16 == 0 (K % 8 == 0 for INT4) and K <= 16384. */
+int qift_pack_weights(const float* W, int N, int K, int levels, int scale_mode, float* s_n,
+                      uint32_t* packed, void* stream);
+
+/* Inverse of the word layout, for tests: codes uint8 [N,K] (INT4: the nibble 0..15). */
+int qift_unpack_codes(const uint32_t* packed, int N, int K, int levels, uint8_t* codes, void* stream);
+
+/* S0 (offline rotation, Sec. 3.1 / Sec. 4.1): Y = X Q with Q = blockdiag(H_B) / sqrt(B), H_B the
+ * Sylvester-Walsh matrix in natural order, applied to every row of X fp32 [M,K] along K.  fp32
+ * butterfly with stages in ascending stride, then one multiply by (float)(1/sqrt(B)).
+ * had_block B: a power of two >= 2 dividing K.  K <= 16384, K % 16 == 0.  In place (Y == X) is allowed. */
+int qift_rotate(const float* X, int M, int K, int had_block, float* Y, void* stream);
+
+/* S2 + S3 (online rotation + per-token symmetric INT4 quantizer; Eq. 1 with b = 4, Sec. 4.1).
+ *   X        in  [M,K] fp32 or bf16 (bf16 is widened exactly)
+ *   had_block    0 = no rotation, else a power of two >= 2 dividing K
+ *   clip_ratio   the paper uses 0.9; must be in (0, 1]
+ *   q_a      out int8 [M,K], one value of [-8,7] per byte
+ *   s_a      out fp32 [M]
+ * u = blockwise H x (unnormalised); s_u = (amax*clip)/7 (1 for a zero row);
+ * q = clamp(rint(u / s_u), -8, 7); s_a = s_u * (float)(1/sqrt(B)).   K <= 16384, K % 16 == 0. */
+int qift_quantize_act(const void* X, int x_dtype, int M, int K, int had_block, float clip_ratio,
+                      int8_t* q_a, float* s_a, void* stream);
+
+/* S4 + S5 (exact integer product + scale epilogue; Sec. 1 "per-channel scale ... in the epilogue",
+ * Sec. 3.6 decoded small signed integer levels) for the two-bit sets MNZ, POT, SYM.
+ *   packed, s_n   from qift_pack_weights
+ *   q_a, s_a      from qift_quantize_act
+ *   Y         out [M,N] fp32 or bf16 (round to nearest even): ((float)acc * s_a[m]) * s_n[n]
+ *   acc_debug out int32 [M,N] accumulators, or NULL
+ *   workspace     >= qift_workspace_bytes(M,N,K,levels) bytes, 1024-byte aligned; may be NULL when 0
+ * M <= 16 takes the decode route, larger M the prefill route. */
+int qift_w2a4_linear(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a,
+                     const float* s_a, int M, int N, int K, void* Y, int y_dtype, int32_t* acc_debug,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* Same for INT4 weights (the W4A4 layers of the layer-wise mixed-precision setting, Sec. 4.4). */
+int qift_w4a4_linear(const uint32_t* packed, const float* s_n, const int8_t* q_a, const float* s_a,
+                     int M, int N, int K, void* Y, int y_dtype, int32_t* acc_debug, void* workspace,
+                     size_t workspace_bytes, void* stream);
+
+/* The two calls above with the kernel route chosen by the caller (tests and benchmarks).
+ * QIFT_ERR_UNSUPPORTED_SHAPE when the route cannot serve the shape. */
+int qift_linear_route(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a,
+                      const float* s_a, int M, int N, int K, void* Y, int y_dtype, int32_t* acc_debug,
+                      void* workspace, size_t workspace_bytes, int route, void* stream);
+
+/* Synchronizes `stream`, then reads and clears the device status word in which a kernel records an
+ * expired bounded wait.  QIFT_OK, QIFT_ERR_TIMEOUT or QIFT_ERR_CUDA.  `detail` (host, may be NULL)
+ * receives the raw word: bits 0-7 the waiting site, the rest the block index. */
+int qift_device_status(void* stream, uint32_t* detail);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QIFT_H_ */

@@ -1,0 +1,10 @@
+"""B200-native (sm_100a) library for the rotated W2A4 / W4A4 quantized linear layer of Qift.
+
+The product is the C-ABI shared library built from csrc/ (declared in include/qift.h); this package
+is its thin Python binding.  Importing the package does not load the library; the first call does,
+and raises if it has not been built.
+"""
+from .binding import *  # noqa: F401,F403
+from .binding import (lib, status_string, QiftError, qift_packed_bytes, qift_workspace_bytes, qift_pack_weights,
+                      qift_unpack_codes, qift_rotate, qift_quantize_act, qift_w2a4_linear, qift_w4a4_linear,
+                      qift_linear_route, qift_device_status)

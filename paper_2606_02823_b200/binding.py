@@ -1,0 +1,194 @@
+"""ctypes binding of libqift.so: the same entry points as include/qift.h, taking torch CUDA tensors.
+
+Argument marshalling only -- every step of the layer runs in the library's CUDA kernels.  torch is
+used for device memory and the current stream.  There is no CPU fallback: if the shared library is
+missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libqift.so")
+
+# enums of qift.h
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
+MNZ, POT, SYM, INT4 = 0, 1, 2, 3
+SCALE_GIVEN, SCALE_ABSMAX, SCALE_MSE = 0, 1, 2
+F32, BF16 = 0, 1
+ROUTE_AUTO, ROUTE_GENERIC, ROUTE_DECODE, ROUTE_PREFILL = 0, 1, 2, 3
+
+EXPORTS = [
+    "qift_status_string", "qift_packed_bytes", "qift_workspace_bytes", "qift_pack_weights",
+    "qift_unpack_codes", "qift_rotate", "qift_quantize_act", "qift_w2a4_linear", "qift_w4a4_linear",
+    "qift_linear_route", "qift_device_status",
+]
+
+_lib = None
+
+
+class QiftError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (qift_status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libqift.so; raises if it has not been built (python -m paper_2606_02823_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2606_02823_b200.build` "
+                "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ci, cf, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+        L.qift_status_string.restype = ctypes.c_char_p
+        L.qift_status_string.argtypes = [ci]
+        L.qift_packed_bytes.restype = sz
+        L.qift_packed_bytes.argtypes = [ci, ci, ci]
+        L.qift_workspace_bytes.restype = sz
+        L.qift_workspace_bytes.argtypes = [ci, ci, ci, ci]
+        L.qift_pack_weights.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp]
+        L.qift_unpack_codes.argtypes = [vp, ci, ci, ci, vp, vp]
+        L.qift_rotate.argtypes = [vp, ci, ci, ci, vp, vp]
+        L.qift_quantize_act.argtypes = [vp, ci, ci, ci, ci, cf, vp, vp, vp]
+        L.qift_w2a4_linear.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, vp, ci, vp, vp, sz, vp]
+        L.qift_w4a4_linear.argtypes = [vp, vp, vp, vp, ci, ci, ci, vp, ci, vp, vp, sz, vp]
+        L.qift_linear_route.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, vp, ci, vp, vp, sz, ci, vp]
+        L.qift_device_status.argtypes = [vp, vp]
+        for name in EXPORTS:
+            if name not in ("qift_status_string", "qift_packed_bytes", "qift_workspace_bytes"):
+                getattr(L, name).restype = ci
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().qift_status_string(int(status)).decode()
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc: int, where: str):
+    if rc != OK:
+        raise QiftError(rc, where)
+
+
+def _dev(t, dtype=None):
+    assert t.is_cuda and t.is_contiguous(), "expected a contiguous CUDA tensor"
+    if dtype is not None:
+        assert t.dtype == dtype, f"expected {dtype}, got {t.dtype}"
+    return t
+
+
+def qift_packed_bytes(N: int, K: int, levels: int) -> int:
+    return int(lib().qift_packed_bytes(N, K, levels))
+
+
+def qift_workspace_bytes(M: int, N: int, K: int, levels: int) -> int:
+    return int(lib().qift_workspace_bytes(M, N, K, levels))
+
+
+def qift_pack_weights(W, levels: int, scale_mode: int, s_n=None, packed=None):
+    """W fp32 [N,K] (already rotated) -> (packed uint32-as-int32 [N, K/per], s_n fp32 [N])."""
+    _dev(W, torch.float32)
+    N, K = W.shape
+    per = 8 if levels == INT4 else 16
+    if s_n is None:
+        s_n = torch.empty(N, dtype=torch.float32, device=W.device)
+    if packed is None:
+        packed = torch.empty((N, max(K // per, 1)), dtype=torch.int32, device=W.device)
+    _check(lib().qift_pack_weights(_ptr(W), N, K, levels, scale_mode, _ptr(_dev(s_n, torch.float32)),
+                                   _ptr(_dev(packed)), _stream()), "qift_pack_weights")
+    return packed, s_n
+
+
+def qift_unpack_codes(packed, K: int, levels: int):
+    _dev(packed)
+    N = packed.shape[0]
+    codes = torch.empty((N, K), dtype=torch.uint8, device=packed.device)
+    _check(lib().qift_unpack_codes(_ptr(packed), N, K, levels, _ptr(codes), _stream()), "qift_unpack_codes")
+    return codes
+
+
+def qift_rotate(X, had_block: int, out=None):
+    _dev(X, torch.float32)
+    M, K = X.shape
+    if out is None:
+        out = torch.empty_like(X)
+    _check(lib().qift_rotate(_ptr(X), M, K, had_block, _ptr(_dev(out, torch.float32)), _stream()), "qift_rotate")
+    return out
+
+
+def qift_quantize_act(X, had_block: int, clip_ratio: float = 0.9, q_a=None, s_a=None):
+    """X fp32 or bf16 [M,K] -> (q_a int8 [M,K], s_a fp32 [M])."""
+    _dev(X)
+    assert X.dtype in (torch.float32, torch.bfloat16)
+    M, K = X.shape
+    if q_a is None:
+        q_a = torch.empty((M, K), dtype=torch.int8, device=X.device)
+    if s_a is None:
+        s_a = torch.empty((M,), dtype=torch.float32, device=X.device)
+    _check(lib().qift_quantize_act(_ptr(X), F32 if X.dtype == torch.float32 else BF16, M, K, had_block,
+                                   clip_ratio, _ptr(_dev(q_a, torch.int8)), _ptr(_dev(s_a, torch.float32)),
+                                   _stream()), "qift_quantize_act")
+    return q_a, s_a
+
+
+def _linear(fn_name, packed, s_n, levels, q_a, s_a, N, out_dtype, want_acc, workspace, route, out):
+    _dev(packed), _dev(s_n, torch.float32), _dev(q_a, torch.int8), _dev(s_a, torch.float32)
+    M, K = q_a.shape
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=q_a.device)
+    assert out.dtype in (torch.float32, torch.bfloat16)
+    acc = torch.empty((M, N), dtype=torch.int32, device=q_a.device) if want_acc else None
+    need = qift_workspace_bytes(max(M, 17) if route == ROUTE_PREFILL else M, N, K, levels)
+    if workspace is None and need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q_a.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    ydt = F32 if out.dtype == torch.float32 else BF16
+    L = lib()
+    if fn_name == "qift_linear_route":
+        rc = L.qift_linear_route(_ptr(packed), _ptr(s_n), levels, _ptr(q_a), _ptr(s_a), M, N, K, _ptr(out), ydt,
+                                 _ptr(acc), _ptr(workspace), ws_bytes, route, _stream())
+    elif fn_name == "qift_w4a4_linear":
+        rc = L.qift_w4a4_linear(_ptr(packed), _ptr(s_n), _ptr(q_a), _ptr(s_a), M, N, K, _ptr(out), ydt, _ptr(acc),
+                                _ptr(workspace), ws_bytes, _stream())
+    else:
+        rc = L.qift_w2a4_linear(_ptr(packed), _ptr(s_n), levels, _ptr(q_a), _ptr(s_a), M, N, K, _ptr(out), ydt,
+                                _ptr(acc), _ptr(workspace), ws_bytes, _stream())
+    _check(rc, fn_name)
+    return (out, acc) if want_acc else out
+
+
+def qift_w2a4_linear(packed, s_n, levels, q_a, s_a, out_dtype=torch.float32, want_acc=False, workspace=None, out=None):
+    return _linear("qift_w2a4_linear", packed, s_n, levels, q_a, s_a, packed.shape[0], out_dtype, want_acc,
+                   workspace, ROUTE_AUTO, out)
+
+
+def qift_w4a4_linear(packed, s_n, q_a, s_a, out_dtype=torch.float32, want_acc=False, workspace=None, out=None):
+    return _linear("qift_w4a4_linear", packed, s_n, INT4, q_a, s_a, packed.shape[0], out_dtype, want_acc,
+                   workspace, ROUTE_AUTO, out)
+
+
+def qift_linear_route(packed, s_n, levels, q_a, s_a, route, out_dtype=torch.float32, want_acc=False, workspace=None,
+                      out=None):
+    return _linear("qift_linear_route", packed, s_n, levels, q_a, s_a, packed.shape[0], out_dtype, want_acc,
+                   workspace, route, out)
+
+
+def qift_device_status():
+    """Synchronizes the current stream; returns (status, detail word)."""
+    detail = ctypes.c_uint32(0)
+    rc = lib().qift_device_status(_stream(), ctypes.byref(detail))
+    return rc, detail.value

@@ -1,0 +1,120 @@
+// Shared device helpers of the qift CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "qift.h"
+
+namespace qift {
+
+// ------------------------------------------------------------------------------------------------
+// Device status word: a kernel whose bounded wait expires records (site | block << 8) here and
+// returns normally; qift_device_status() reads and clears it.
+// ------------------------------------------------------------------------------------------------
+static __device__ unsigned int g_status_word;
+
+__device__ __forceinline__ void report_timeout(unsigned int site) {
+    atomicCAS(&g_status_word, 0u, (site & 0xffu) | (blockIdx.x << 8) | 0x80000000u);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Level sets
+// ------------------------------------------------------------------------------------------------
+__host__ __device__ constexpr int codes_per_word(int lv) { return lv == QIFT_LEVELS_INT4 ? 8 : 16; }
+__host__ __device__ constexpr float top_level(int lv) {
+    return lv == QIFT_LEVELS_MNZ ? 3.0f : lv == QIFT_LEVELS_POT ? 4.0f : lv == QIFT_LEVELS_SYM ? 1.0f : 7.0f;
+}
+
+template <int LV>
+__device__ __forceinline__ int level_from_code(int c) {
+    if constexpr (LV == QIFT_LEVELS_MNZ) return 2 * c - 3;
+    if constexpr (LV == QIFT_LEVELS_POT) return 3 * c - (c >> 1) - 4;  // 0,3,5,8 minus 4
+    if constexpr (LV == QIFT_LEVELS_SYM) return c - 2;
+    return ((c & 15) ^ 8) - 8;
+}
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// Programmatic dependent launch: let the next kernel in the stream start its prologue, and wait for
+// the previous kernel's memory before touching any caller buffer.
+__device__ __forceinline__ void pdl_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after ~2^22 polls (each poll may itself sleep for a hardware-chosen
+// interval), records the site and returns false.  Callers skip their remaining work on false.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int site) {
+    for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+    }
+    report_timeout(site);
+    return false;
+}
+
+// 1-D bulk copy global -> shared::cta (no multicast), completion counted on an mbarrier.
+// Both addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst_smem)),
+                 "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+// u8 x s8 -> s32 four-way dot product.
+__device__ __forceinline__ int dp4a_us(uint32_t a_u8x4, uint32_t b_s8x4, int c) {
+    int d;
+    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a_u8x4), "r"(b_s8x4), "r"(c));
+    return d;
+}
+
+// D(16x8,s32) += A(16x32,u8,row) * B(32x8,s8,col)
+__device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint16_t f32_to_bf16_bits(float f) {
+    return __bfloat16_as_ushort(__float2bfloat16_rn(f));
+}
+
+// y = ((float)acc * s_a) * s_n, two separately rounded multiplies.
+__device__ __forceinline__ float scale_epilogue(int acc, float s_a, float s_n) {
+    return __fmul_rn(__fmul_rn(static_cast<float>(acc), s_a), s_n);
+}
+
+}  // namespace qift

@@ -1,0 +1,351 @@
+// C-ABI entry points of the qift library: argument checks on the host, then kernel launches on the
+// caller's stream.  Single translation unit; the kernels live in the headers included below.
+#include <cmath>
+#include <cstdint>
+#include <cstdio>
+
+#include "common.cuh"
+#include "decode.cuh"
+#include "pack.cuh"
+#include "prefill.cuh"
+#include "rotate_quant.cuh"
+
+namespace qift {
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+inline bool valid_levels(int lv) { return lv >= QIFT_LEVELS_MNZ && lv <= QIFT_LEVELS_INT4; }
+
+// Launch with programmatic stream serialization: the kernel may start while its predecessor in the
+// stream drains; every kernel here executes griddepcontrol.wait before touching caller memory.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+template <typename K>
+cudaError_t allow_smem(K kernel, size_t bytes) {
+    if (bytes <= 48 * 1024) return cudaSuccess;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+}
+
+inline int cuda_status(cudaError_t e) {
+    if (e == cudaSuccess) return QIFT_OK;
+    std::fprintf(stderr, "qift: CUDA error: %s\n", cudaGetErrorString(e));
+    return QIFT_ERR_CUDA;
+}
+
+float inv_sqrt_block(int B) { return static_cast<float>(1.0 / std::sqrt(static_cast<double>(B))); }
+
+int check_rotation_shape(int K, int had_block, bool allow_none) {
+    if (K <= 0 || K % 16 != 0 || K > kMaxRowK) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (had_block == 0) return allow_none ? QIFT_OK : QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (had_block < 2 || !is_pow2(had_block) || K % had_block != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    return QIFT_OK;
+}
+
+// ---------------------------------------------------------------------------------------- decode
+template <int LV, int NT, int RT>
+int launch_decode(const DecodeParams& p, cudaStream_t st) {
+    const int words = p.K / codes_per_word(LV);
+    const int nchunks = (words + kChunkWords - 1) / kChunkWords;
+    const size_t stage = decode_stage_bytes(LV, RT, p.M);
+    int stages = static_cast<int>((80 * 1024) / stage);
+    if (stages < 2) stages = 2;
+    if (stages > nchunks) stages = nchunks;
+    DecodeParams q = p;
+    q.stages = stages;
+    const size_t smem = decode_smem_bytes(LV, RT, NT, p.M, stages);
+    auto kernel = linear_decode_kernel<LV, NT, RT>;
+    cudaError_t e = allow_smem(kernel, smem);
+    if (e != cudaSuccess) return cuda_status(e);
+    const int grid = (p.N + 16 * RT - 1) / (16 * RT);
+    return cuda_status(launch_pdl(kernel, dim3(grid), dim3(kDecThreads), smem, st, q));
+}
+
+template <int LV>
+int dispatch_decode(const DecodeParams& p, cudaStream_t st) {
+    if (p.M > 8) return launch_decode<LV, 2, 1>(p, st);
+    const int tiles = (p.N + 15) / 16;
+    if (tiles >= 4 * 148) return launch_decode<LV, 1, 2>(p, st);
+    return launch_decode<LV, 1, 1>(p, st);
+}
+
+bool decode_supports(int lv, int M, int N, int K) {
+    const int per = codes_per_word(lv);
+    return M >= 1 && M <= 16 && K % (16 * per) == 0;  // whole 16-word warp slices
+}
+
+template <int LV>
+int launch_generic(const uint32_t* packed, const float* s_n, const int8_t* q_a, const float* s_a, int M, int N, int K,
+                   void* Y, int y_bf16, int32_t* acc_debug, cudaStream_t st) {
+    const int grid = (N + kGenericWarps - 1) / kGenericWarps;
+    return cuda_status(launch_pdl(linear_generic_kernel<LV>, dim3(grid), dim3(kGenericWarps * 32), 0, st, packed, s_n, q_a,
+                                  s_a, M, N, K, Y, y_bf16, acc_debug));
+}
+
+// --------------------------------------------------------------------------------------- prefill
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// int8 [rows, K] row-major; box = 128 bytes of K x box_rows rows, 128-byte swizzle, zero fill.
+bool make_i8_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K)};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kGemmBK), static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+template <int BN>
+int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& gp, cudaStream_t st) {
+    auto kernel = gemm_i8_tcgen05_kernel<BN>;
+    const size_t smem = gemm_smem_bytes<BN>();
+    cudaError_t e = allow_smem(kernel, smem);
+    if (e != cudaSuccess) return cuda_status(e);
+    const int tiles = ((gp.M + kGemmBM - 1) / kGemmBM) * ((gp.N + BN - 1) / BN);
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    return cuda_status(launch_pdl(kernel, dim3(grid), dim3(kGemmThreads), smem, st, ma, mb, gp));
+}
+
+template <int LV>
+int launch_expand(const uint32_t* packed, int N, int K, int8_t* out, cudaStream_t st) {
+    const long long words = static_cast<long long>(N) * (K / codes_per_word(LV));
+    long long blocks = (words + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    return cuda_status(launch_pdl(expand_levels_kernel<LV>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, st, packed, words, out));
+}
+
+int run_prefill(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
+                void* Y, int y_bf16, int32_t* acc_debug, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    if (K % 16 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;  // TMA row pitch must be a multiple of 16 bytes
+    const size_t need = qift_workspace_bytes(17 > M ? 17 : M, N, K, lv);
+    if (!workspace || workspace_bytes < need) return QIFT_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 1023u) != 0) return QIFT_ERR_ALIGNMENT;
+    int8_t* wexp = static_cast<int8_t*>(workspace);
+    int rc;
+    switch (lv) {
+        case QIFT_LEVELS_MNZ: rc = launch_expand<QIFT_LEVELS_MNZ>(packed, N, K, wexp, st); break;
+        case QIFT_LEVELS_POT: rc = launch_expand<QIFT_LEVELS_POT>(packed, N, K, wexp, st); break;
+        case QIFT_LEVELS_SYM: rc = launch_expand<QIFT_LEVELS_SYM>(packed, N, K, wexp, st); break;
+        default: rc = launch_expand<QIFT_LEVELS_INT4>(packed, N, K, wexp, st); break;
+    }
+    if (rc != QIFT_OK) return rc;
+    const int m_tiles = (M + kGemmBM - 1) / kGemmBM;
+    const bool narrow = m_tiles * ((N + 255) / 256) < sm_count();
+    CUtensorMap ma, mb;
+    if (!make_i8_map(&ma, q_a, M, K, kGemmBM) || !make_i8_map(&mb, wexp, N, K, narrow ? 128 : 256)) return QIFT_ERR_CUDA;
+    GemmParams gp{s_n, s_a, Y, acc_debug, M, N, K, y_bf16};
+    return narrow ? launch_gemm<128>(ma, mb, gp, st) : launch_gemm<256>(ma, mb, gp, st);
+}
+
+int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
+                void* Y, int y_dtype, int32_t* acc_debug, void* workspace, size_t workspace_bytes, int route, void* stream) {
+    if (!packed || !s_n || !q_a || !s_a || !Y || M <= 0 || N <= 0 || K <= 0 || !valid_levels(lv)) return QIFT_ERR_INVALID_ARG;
+    if (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16) return QIFT_ERR_INVALID_ARG;
+    if (route < QIFT_ROUTE_AUTO || route > QIFT_ROUTE_PREFILL) return QIFT_ERR_INVALID_ARG;
+    if (K % codes_per_word(lv) != 0 || K % 4 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(packed) || !aligned16(s_n) || !aligned16(q_a) || !aligned16(s_a) || !aligned16(Y) ||
+        (acc_debug && !aligned16(acc_debug)))
+        return QIFT_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int y_bf16 = (y_dtype == QIFT_BF16);
+    if (route == QIFT_ROUTE_AUTO) {
+        if (M <= 16) route = decode_supports(lv, M, N, K) ? QIFT_ROUTE_DECODE : QIFT_ROUTE_GENERIC;
+        else route = (K % 16 == 0) ? QIFT_ROUTE_PREFILL : QIFT_ROUTE_GENERIC;
+    }
+    if (route == QIFT_ROUTE_DECODE) {
+        if (!decode_supports(lv, M, N, K)) return QIFT_ERR_UNSUPPORTED_SHAPE;
+        DecodeParams p{packed, s_n, q_a, s_a, Y, acc_debug, M, N, K, y_bf16, 0};
+        switch (lv) {
+            case QIFT_LEVELS_MNZ: return dispatch_decode<QIFT_LEVELS_MNZ>(p, st);
+            case QIFT_LEVELS_POT: return dispatch_decode<QIFT_LEVELS_POT>(p, st);
+            case QIFT_LEVELS_SYM: return dispatch_decode<QIFT_LEVELS_SYM>(p, st);
+            default: return dispatch_decode<QIFT_LEVELS_INT4>(p, st);
+        }
+    }
+    if (route == QIFT_ROUTE_PREFILL)
+        return run_prefill(packed, s_n, lv, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, workspace, workspace_bytes, st);
+    switch (lv) {
+        case QIFT_LEVELS_MNZ: return launch_generic<QIFT_LEVELS_MNZ>(packed, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st);
+        case QIFT_LEVELS_POT: return launch_generic<QIFT_LEVELS_POT>(packed, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st);
+        case QIFT_LEVELS_SYM: return launch_generic<QIFT_LEVELS_SYM>(packed, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st);
+        default: return launch_generic<QIFT_LEVELS_INT4>(packed, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st);
+    }
+}
+
+}  // namespace
+}  // namespace qift
+
+using namespace qift;
+
+extern "C" {
+
+const char* qift_status_string(int status) {
+    switch (status) {
+        case QIFT_OK: return "ok";
+        case QIFT_ERR_INVALID_ARG: return "invalid argument";
+        case QIFT_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case QIFT_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case QIFT_ERR_WORKSPACE: return "workspace missing or too small";
+        case QIFT_ERR_CUDA: return "CUDA error";
+        case QIFT_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+size_t qift_packed_bytes(int N, int K, int levels) {
+    if (N <= 0 || K <= 0 || !valid_levels(levels) || K % codes_per_word(levels) != 0) return 0;
+    return static_cast<size_t>(N) * (K / codes_per_word(levels)) * 4;
+}
+
+size_t qift_workspace_bytes(int M, int N, int K, int levels) {
+    if (M <= 0 || N <= 0 || K <= 0 || !valid_levels(levels)) return 0;
+    if (M <= 16) return 0;
+    const size_t b = static_cast<size_t>(N) * K;
+    return (b + 1023) & ~static_cast<size_t>(1023);
+}
+
+int qift_pack_weights(const float* W, int N, int K, int levels, int scale_mode, float* s_n, uint32_t* packed, void* stream) {
+    if (!W || !s_n || !packed || N <= 0 || K <= 0 || !valid_levels(levels)) return QIFT_ERR_INVALID_ARG;
+    if (scale_mode < QIFT_SCALE_GIVEN || scale_mode > QIFT_SCALE_MSE) return QIFT_ERR_INVALID_ARG;
+    if (K % 16 != 0 || K > kMaxRowK) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(W) || !aligned16(s_n) || !aligned16(packed)) return QIFT_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t smem = static_cast<size_t>(K) * 4;
+#define QIFT_PACK_CASE(LV)                                                                                   \
+    case LV: {                                                                                               \
+        cudaError_t e = allow_smem(pack_weights_kernel<LV>, smem);                                           \
+        if (e != cudaSuccess) return cuda_status(e);                                                         \
+        return cuda_status(launch_pdl(pack_weights_kernel<LV>, dim3(N), dim3(kPackThreads), smem, st, W, K,  \
+                                      scale_mode, s_n, packed));                                             \
+    }
+    switch (levels) {
+        QIFT_PACK_CASE(QIFT_LEVELS_MNZ)
+        QIFT_PACK_CASE(QIFT_LEVELS_POT)
+        QIFT_PACK_CASE(QIFT_LEVELS_SYM)
+        QIFT_PACK_CASE(QIFT_LEVELS_INT4)
+    }
+#undef QIFT_PACK_CASE
+    return QIFT_ERR_INVALID_ARG;
+}
+
+int qift_unpack_codes(const uint32_t* packed, int N, int K, int levels, uint8_t* codes, void* stream) {
+    if (!packed || !codes || N <= 0 || K <= 0 || !valid_levels(levels)) return QIFT_ERR_INVALID_ARG;
+    if (K % codes_per_word(levels) != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(packed) || !aligned16(codes)) return QIFT_ERR_ALIGNMENT;
+    const long long total = static_cast<long long>(N) * K;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    return cuda_status(launch_pdl(unpack_codes_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0,
+                                  static_cast<cudaStream_t>(stream), packed, total, K, codes_per_word(levels), codes));
+}
+
+int qift_rotate(const float* X, int M, int K, int had_block, float* Y, void* stream) {
+    if (!X || !Y || M <= 0 || K <= 0) return QIFT_ERR_INVALID_ARG;
+    const int rc = check_rotation_shape(K, had_block, false);
+    if (rc != QIFT_OK) return rc;
+    if (!aligned16(X) || !aligned16(Y)) return QIFT_ERR_ALIGNMENT;
+    const size_t smem = static_cast<size_t>(K) * 4;
+    cudaError_t e = allow_smem(rotate_rows_kernel, smem);
+    if (e != cudaSuccess) return cuda_status(e);
+    return cuda_status(launch_pdl(rotate_rows_kernel, dim3(M), dim3(kRowThreads), smem, static_cast<cudaStream_t>(stream), X,
+                                  K, had_block, inv_sqrt_block(had_block), Y));
+}
+
+int qift_quantize_act(const void* X, int x_dtype, int M, int K, int had_block, float clip_ratio, int8_t* q_a, float* s_a,
+                      void* stream) {
+    if (!X || !q_a || !s_a || M <= 0 || K <= 0) return QIFT_ERR_INVALID_ARG;
+    if (x_dtype != QIFT_F32 && x_dtype != QIFT_BF16) return QIFT_ERR_INVALID_ARG;
+    if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return QIFT_ERR_INVALID_ARG;
+    const int rc = check_rotation_shape(K, had_block, true);
+    if (rc != QIFT_OK) return rc;
+    if (!aligned16(X) || !aligned16(q_a) || !aligned16(s_a)) return QIFT_ERR_ALIGNMENT;
+    const size_t smem = static_cast<size_t>(K) * 4;
+    const float r = had_block > 1 ? inv_sqrt_block(had_block) : 1.0f;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (x_dtype == QIFT_BF16) {
+        cudaError_t e = allow_smem(quantize_act_kernel<true>, smem);
+        if (e != cudaSuccess) return cuda_status(e);
+        return cuda_status(launch_pdl(quantize_act_kernel<true>, dim3(M), dim3(kRowThreads), smem, st, X, K, had_block,
+                                      clip_ratio, r, q_a, s_a));
+    }
+    cudaError_t e = allow_smem(quantize_act_kernel<false>, smem);
+    if (e != cudaSuccess) return cuda_status(e);
+    return cuda_status(launch_pdl(quantize_act_kernel<false>, dim3(M), dim3(kRowThreads), smem, st, X, K, had_block,
+                                  clip_ratio, r, q_a, s_a));
+}
+
+int qift_w2a4_linear(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a, const float* s_a, int M, int N,
+                     int K, void* Y, int y_dtype, int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream) {
+    if (levels != QIFT_LEVELS_MNZ && levels != QIFT_LEVELS_POT && levels != QIFT_LEVELS_SYM) return QIFT_ERR_INVALID_ARG;
+    return linear_impl(packed, s_n, levels, q_a, s_a, M, N, K, Y, y_dtype, acc_debug, workspace, workspace_bytes,
+                       QIFT_ROUTE_AUTO, stream);
+}
+
+int qift_w4a4_linear(const uint32_t* packed, const float* s_n, const int8_t* q_a, const float* s_a, int M, int N, int K,
+                     void* Y, int y_dtype, int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream) {
+    return linear_impl(packed, s_n, QIFT_LEVELS_INT4, q_a, s_a, M, N, K, Y, y_dtype, acc_debug, workspace, workspace_bytes,
+                       QIFT_ROUTE_AUTO, stream);
+}
+
+int qift_linear_route(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a, const float* s_a, int M, int N,
+                      int K, void* Y, int y_dtype, int32_t* acc_debug, void* workspace, size_t workspace_bytes, int route,
+                      void* stream) {
+    return linear_impl(packed, s_n, levels, q_a, s_a, M, N, K, Y, y_dtype, acc_debug, workspace, workspace_bytes, route, stream);
+}
+
+int qift_device_status(void* stream, uint32_t* detail) {
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_status(e);
+    unsigned int word = 0;
+    e = cudaMemcpyFromSymbol(&word, g_status_word, sizeof(word));
+    if (e != cudaSuccess) return cuda_status(e);
+    if (detail) *detail = word;
+    if (word == 0) return QIFT_OK;
+    const unsigned int zero = 0;
+    e = cudaMemcpyToSymbol(g_status_word, &zero, sizeof(zero));
+    if (e != cudaSuccess) return cuda_status(e);
+    return QIFT_ERR_TIMEOUT;
+}
+
+}  // extern "C"

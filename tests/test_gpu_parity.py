@@ -1,0 +1,229 @@
+"""Parity of the CUDA library (through the C ABI) with the CPU oracle, element by element, on the
+same seeded inputs.  Integers (q_a, packed words, INT32 accumulators) must match bit for bit; fp32
+outputs to max relative error 1e-5; bf16 outputs to 1 bf16 ulp."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+import paper_2606_02823_b200 as qift
+
+pytestmark = pytest.mark.gpu
+
+LEVELS = {"MNZ": (qift.MNZ, oracle.MNZ), "POT": (qift.POT, oracle.POT), "SYM": (qift.SYM, oracle.SYM),
+          "INT4": (qift.INT4, oracle.INT4)}
+assert all(a == b for a, b in LEVELS.values())
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def as_u32(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def assert_status_clean():
+    rc, detail = qift.qift_device_status()
+    assert rc == qift.OK, f"device status {rc} detail {detail:#x}"
+
+
+def check_outputs(y_gpu, acc_gpu, y_ref, acc_ref, bf16):
+    assert np.array_equal(acc_gpu.cpu().numpy(), acc_ref), "INT32 accumulators differ"
+    if bf16:
+        got = y_gpu.view(torch.int16).cpu().numpy().view(np.uint16).astype(np.int64)
+        ref = y_ref.astype(np.int64)
+        # ordered-integer distance between bf16 bit patterns = ulps
+        key = lambda v: np.where(v & 0x8000, 0x8000 - (v & 0x7FFF), 0x8000 + v)
+        assert np.abs(key(got) - key(ref)).max() <= 1
+    else:
+        got = y_gpu.cpu().numpy()
+        denom = np.maximum(np.abs(y_ref), 1e-30)
+        assert (np.abs(got - y_ref) / denom).max() <= 1e-5
+        assert np.array_equal(got, y_ref)      # same two rounded multiplies in the same order
+
+
+# ---------------------------------------------------------------------------------- rotation / K2
+@pytest.mark.parametrize("M,K,B", [(1, 256, 256), (3, 4096, 4096), (5, 11008, 256), (4, 14336, 2048),
+                                   (2, 512, 0), (7, 64, 4), (2, 16384, 16384), (33, 1024, 64), (1, 16, 2)])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_quantize_act(M, K, B, bf16):
+    x, _ = synth.activations(100 + M, M, K, max(1, K // 100))
+    if bf16:
+        xb = dev(x).to(torch.bfloat16)
+        x_ref = oracle.bf16_to_f32(xb.view(torch.int16).cpu().numpy().view(np.uint16))
+        q, s = qift.qift_quantize_act(xb, B, 0.9)
+    else:
+        x_ref = x
+        q, s = qift.qift_quantize_act(dev(x), B, 0.9)
+    q_ref, s_ref = oracle.quantize_act(x_ref, B, 0.9)
+    assert np.array_equal(q.cpu().numpy(), q_ref)
+    assert np.array_equal(s.cpu().numpy(), s_ref)
+    assert_status_clean()
+
+
+def test_quantize_act_zero_and_clip():
+    x = np.zeros((2, 256), dtype=np.float32)
+    x[1, 5] = -3.0
+    for clip in (0.9, 1.0, 0.5):
+        q, s = qift.qift_quantize_act(dev(x), 256, clip)
+        q_ref, s_ref = oracle.quantize_act(x, 256, clip)
+        assert np.array_equal(q.cpu().numpy(), q_ref) and np.array_equal(s.cpu().numpy(), s_ref)
+
+
+@pytest.mark.parametrize("M,K,B", [(4, 256, 256), (3, 4096, 4096), (2, 11008, 256), (2, 14336, 2048), (5, 96, 32)])
+def test_rotate(M, K, B):
+    W = synth.student_weights(7, M, K)
+    got = qift.qift_rotate(dev(W), B).cpu().numpy()
+    assert np.array_equal(got, oracle.rotate_weights(W, B))
+    w = dev(W)
+    qift.qift_rotate(w, B, out=w)        # in place
+    assert np.array_equal(w.cpu().numpy(), got)
+
+
+# ---------------------------------------------------------------------------------- K1 packer
+@pytest.mark.parametrize("name", list(LEVELS))
+@pytest.mark.parametrize("N,K", [(256, 256), (37, 1024), (16, 11008), (3, 16)])
+def test_pack_absmax_and_given(name, N, K):
+    lv = LEVELS[name][0]
+    W = synth.gaussian_weights(0, N, K)
+    W[N // 2] = 0                                   # a zero row
+    W[0, :4] = [0.0, 1e-9, -1e-9, 0.0]
+    packed, s_n = qift.qift_pack_weights(dev(W), lv, qift.SCALE_ABSMAX)
+    p_ref, s_ref, codes_ref = oracle.pack_weights(W, lv, oracle.SCALE_ABSMAX)
+    assert np.array_equal(s_n.cpu().numpy(), s_ref)
+    assert np.array_equal(as_u32(packed), p_ref)
+    # given scales, with weights sitting exactly on decision thresholds
+    s_given = (np.abs(W).max(1) * 0.3 + 1e-3).astype(np.float32)
+    Wt = W.copy()
+    mids = np.array([-2.5, -2.0, -1.5, -0.5, 0.0, 0.5, 1.5, 2.0, 2.5, 7.5, -8.5], dtype=np.float32)
+    if K >= len(mids):
+        Wt[:, :len(mids)] = mids[None, :] * s_given[:, None]
+    packed, s_out = qift.qift_pack_weights(dev(Wt), lv, qift.SCALE_GIVEN, s_n=dev(s_given))
+    p_ref, _, _ = oracle.pack_weights(Wt, lv, oracle.SCALE_GIVEN, s_given)
+    assert np.array_equal(as_u32(packed), p_ref)
+    assert np.array_equal(s_out.cpu().numpy(), s_given)
+    codes = qift.qift_unpack_codes(packed, K, lv).cpu().numpy()
+    assert np.array_equal(codes, oracle.unpack(p_ref, K, lv))
+    assert_status_clean()
+
+
+@pytest.mark.parametrize("name", list(LEVELS))
+def test_pack_mse(name):
+    lv = LEVELS[name][0]
+    N, K = 96, 4096
+    W = oracle.rotate_weights(synth.student_weights(3, N, K), K)
+    packed, s_n = qift.qift_pack_weights(dev(W), lv, qift.SCALE_MSE)
+    s_gpu = s_n.cpu().numpy()
+    s_ref, idx_ref, errs = oracle.weight_scale(W, lv, oracle.SCALE_MSE, want_errs=True)
+    diff = np.nonzero(s_gpu != s_ref)[0]
+    for n in diff:      # the sum order differs: only a numerical tie may change the winner
+        e = np.sort(errs[n])
+        assert (e[1] - e[0]) <= 1e-12 * e[0], f"row {n}: scale differs without a tie"
+    # codes are exact given the scales the GPU chose
+    p_ref, _, _ = oracle.pack_weights(W, lv, oracle.SCALE_GIVEN, s_gpu)
+    assert np.array_equal(as_u32(packed), p_ref)
+    assert len(diff) <= 1
+
+
+# ---------------------------------------------------------------------------------- S4 + S5
+def make_problem(lv, M, N, K, seed, B=None):
+    W = synth.gaussian_weights(seed, N, K)
+    x, _ = synth.activations(seed + 1, M, K, max(1, K // 100))
+    if B is None:
+        B = synth.had_block_for(K)
+    p_ref, s_n, codes = oracle.pack_weights(W, lv, oracle.SCALE_ABSMAX)
+    q_a, s_a = oracle.quantize_act(x, B, 0.9)
+    return p_ref, s_n, codes, q_a, s_a
+
+
+def run_route(p_ref, s_n, lv, q_a, s_a, route, bf16):
+    out_dtype = torch.bfloat16 if bf16 else torch.float32
+    y, acc = qift.qift_linear_route(dev(p_ref.view(np.int32)), dev(s_n), lv, dev(q_a), dev(s_a), route,
+                                    out_dtype=out_dtype, want_acc=True)
+    assert_status_clean()
+    return y, acc
+
+
+@pytest.mark.parametrize("name", list(LEVELS))
+@pytest.mark.parametrize("route", [qift.ROUTE_GENERIC, qift.ROUTE_DECODE])
+@pytest.mark.parametrize("M,N,K", [(1, 256, 256), (1, 40, 512), (3, 100, 2304), (8, 64, 4096), (9, 48, 1024),
+                                   (16, 130, 2560), (5, 16, 11008), (2, 2400, 256)])
+def test_decode_routes(name, route, M, N, K):
+    lv = LEVELS[name][0]
+    p_ref, s_n, codes, q_a, s_a = make_problem(lv, M, N, K, seed=50 + M)
+    for bf16 in (False, True):
+        y_ref, acc_ref = oracle.linear(codes, lv, s_n, q_a, s_a, bf16=bf16)
+        y, acc = run_route(p_ref, s_n, lv, q_a, s_a, route, bf16)
+        check_outputs(y, acc, y_ref, acc_ref, bf16)
+
+
+@pytest.mark.parametrize("name", ["MNZ", "INT4"])
+def test_decode_extreme_values(name):
+    # all codes at the top level against all activations at -8 / +7: the largest accumulators
+    lv = LEVELS[name][0]
+    N, K, M = 32, 14336, 2
+    top = 15 if lv == qift.INT4 else 3
+    codes = np.full((N, K), top if lv != qift.INT4 else 7, dtype=np.uint8)
+    codes[1::2] = 0 if lv != qift.INT4 else 8                     # most negative level
+    p_ref = oracle.pack(codes, lv)
+    q_a = np.stack([np.full(K, 7, dtype=np.int8), np.full(K, -8, dtype=np.int8)])
+    s_a = np.array([0.5, 2.0], dtype=np.float32)
+    s_n = np.linspace(0.01, 0.02, N).astype(np.float32)
+    y_ref, acc_ref = oracle.linear(codes, lv, s_n, q_a, s_a)
+    assert np.abs(acc_ref).max() == K * 8 * (8 if lv == qift.INT4 else 3)
+    for route in (qift.ROUTE_GENERIC, qift.ROUTE_DECODE):
+        y, acc = run_route(p_ref, s_n, lv, q_a, s_a, route, False)
+        check_outputs(y, acc, y_ref, acc_ref, False)
+
+
+@pytest.mark.parametrize("name", list(LEVELS))
+@pytest.mark.parametrize("M,N,K", [(128, 256, 512), (200, 300, 1024), (17, 72, 256), (512, 1024, 384), (130, 520, 4096)])
+def test_prefill_route(name, M, N, K):
+    lv = LEVELS[name][0]
+    p_ref, s_n, codes, q_a, s_a = make_problem(lv, M, N, K, seed=80)
+    for bf16 in (True, False):
+        y_ref, acc_ref = oracle.linear(codes, lv, s_n, q_a, s_a, bf16=bf16)
+        y, acc = run_route(p_ref, s_n, lv, q_a, s_a, qift.ROUTE_PREFILL, bf16)
+        check_outputs(y, acc, y_ref, acc_ref, bf16)
+
+
+def test_auto_route_and_public_entry_points():
+    for M in (1, 16, 17, 140):
+        for lv in (qift.MNZ, qift.INT4):
+            p_ref, s_n, codes, q_a, s_a = make_problem(lv, M, 96, 512, seed=9)
+            y_ref, acc_ref = oracle.linear(codes, lv, s_n, q_a, s_a)
+            args = (dev(p_ref.view(np.int32)), dev(s_n))
+            if lv == qift.INT4:
+                y, acc = qift.qift_w4a4_linear(*args, dev(q_a), dev(s_a), want_acc=True)
+            else:
+                y, acc = qift.qift_w2a4_linear(*args, lv, dev(q_a), dev(s_a), want_acc=True)
+            check_outputs(y, acc, y_ref, acc_ref, False)
+    assert_status_clean()
+
+
+def test_runs_are_deterministic():
+    lv = qift.MNZ
+    p_ref, s_n, codes, q_a, s_a = make_problem(lv, 4, 512, 4096, seed=4)
+    outs = [run_route(p_ref, s_n, lv, q_a, s_a, qift.ROUTE_DECODE, False) for _ in range(3)]
+    for y, acc in outs[1:]:
+        assert torch.equal(y, outs[0][0]) and torch.equal(acc, outs[0][1])
+
+
+# ---------------------------------------------------------------------------------- whole path
+def test_whole_path_config1():
+    # config 1: N = K = 256, M = 1, N(0, 0.02^2) weights (seed 0), 4 outlier channels x20, MNZ
+    W = synth.gaussian_weights(0, 256, 256)
+    x, _ = synth.activations(1, 1, 256, 4)
+    for mode_g, mode_o in ((qift.SCALE_ABSMAX, oracle.SCALE_ABSMAX), (qift.SCALE_MSE, oracle.SCALE_MSE)):
+        packed, s_n = qift.qift_pack_weights(dev(W), qift.MNZ, mode_g)
+        q_a, s_a = qift.qift_quantize_act(dev(x), 256, 0.9)
+        y, acc = qift.qift_w2a4_linear(packed, s_n, qift.MNZ, q_a, s_a, want_acc=True)
+        p_ref, s_ref, codes = oracle.pack_weights(W, oracle.MNZ, mode_o)
+        q_ref, sa_ref = oracle.quantize_act(x, 256, 0.9)
+        y_ref, acc_ref = oracle.linear(codes, oracle.MNZ, s_ref, q_ref, sa_ref)
+        assert np.array_equal(as_u32(packed), p_ref) and np.array_equal(s_n.cpu().numpy(), s_ref)
+        assert np.array_equal(q_a.cpu().numpy(), q_ref) and np.array_equal(s_a.cpu().numpy(), sa_ref)
+        check_outputs(y, acc, y_ref, acc_ref, False)
+    assert_status_clean()

@@ -1,0 +1,447 @@
+#!/usr/bin/env python
+"""Benchmark of the Qift quantized-linear hot path on B200.
+
+Default arm: one "step" = one decode token (M = 1) through the 7 linear shapes of a LLaMA-2-7B
+layer, for 32 layers of distinct synthetic weights (224 modules, 1.63 GB of packed weights, so every
+step streams far more than the 126 MB L2).  Each module runs the whole path through the C ABI:
+rotate + INT4-quantize the activation row, then the exact W2A4 product and scale epilogue.  The
+metric is algorithmic HBM bytes per second; `roofline` times the product kernel alone over the same
+224 weight matrices; `prefill` reports the M = 2048 tcgen05 GEMM on LLaMA-3.1-8B shapes in TOPS;
+`e2e` runs the same step through the host-buffer entry point with the copies inside the timed
+region; `cpu_baseline` times the CPU oracle on a bounded sample.
+
+`--impl reference` times the CPU oracle (a deliberately plain single-threaded program) instead.
+
+Launch: python bench.py --gpus N --steps K --warmup W   (N > 1 under torch.distributed.run:
+independent replicas, one per GPU, weak scaling, no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import synth  # noqa: E402
+
+CLIP = 0.9
+N_LAYERS = 32
+
+
+# ------------------------------------------------------------------------------------------------
+# algorithmic bytes / ops (per module call)
+# ------------------------------------------------------------------------------------------------
+def product_bytes(M, N, K, bits=2, out_bytes=4):
+    """Packed codes + channel scales + int8 activations and token scales + output."""
+    return N * K * bits // 8 + 4 * N + M * (K + 4) + M * N * out_bytes
+
+
+def quant_bytes(M, K, in_bytes=4):
+    """Activation row read + int8 row and scale written."""
+    return M * K * in_bytes + M * K + 4 * M
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks sampling during the timed region
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+class Module:
+    __slots__ = ("name", "N", "K", "B", "packed", "s_n", "x", "y", "x_host", "y_host", "bits", "levels")
+
+
+def build_stack(torch, qift, shapes, n_layers, M, levels_of_layer, seed, x_dtype, y_dtype, device, gen):
+    """Synthetic stack: Student-t(5)*0.02 weights rotated by the blockwise Hadamard (our kernel),
+    MSE-scaled and packed (our kernel); Gaussian activations with 1% outlier channels x20."""
+    mods = []
+    for layer in range(n_layers):
+        lv = levels_of_layer(layer)
+        for (name, N, K) in shapes:
+            z = torch.randn((N, K), device=device, dtype=torch.float32, generator=gen)
+            chi = torch.zeros((N, K), device=device, dtype=torch.float32)
+            for _ in range(5):
+                chi += torch.randn((N, K), device=device, dtype=torch.float32, generator=gen) ** 2
+            W = 0.02 * z / torch.sqrt(chi / 5.0)
+            del z, chi
+            B = synth.had_block_for(K)
+            qift.qift_rotate(W, B, out=W)
+            m = Module()
+            m.name, m.N, m.K, m.B, m.levels = name, N, K, B, lv
+            m.bits = 4 if lv == qift.INT4 else 2
+            m.packed, m.s_n = qift.qift_pack_weights(W, lv, qift.SCALE_MSE)
+            del W
+            x = torch.randn((M, K), device=device, dtype=torch.float32, generator=gen)
+            n_out = max(1, round(0.01 * K))
+            ch = torch.randperm(K, device=device, generator=gen)[:n_out]
+            x[:, ch] *= 20.0
+            m.x = x.to(x_dtype).contiguous()
+            m.y = torch.empty((M, N), device=device, dtype=y_dtype)
+            m.x_host = m.x.cpu().pin_memory()
+            m.y_host = torch.empty((M, N), dtype=y_dtype).pin_memory()
+            mods.append(m)
+    torch.cuda.synchronize()
+    return mods
+
+
+def run_gpu(args):
+    import torch
+
+    import paper_2606_02823_b200 as qift
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the product has no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+    L = qift.lib()
+    gen = torch.Generator(device=device)
+    gen.manual_seed(2000 + rank)
+    M = 1
+    launches = [0]
+
+    mods = build_stack(torch, qift, synth.LLAMA2_7B, N_LAYERS, M, lambda l: qift.MNZ, 2000, torch.float32, torch.float32,
+                       device, gen)
+    kmax = max(m.K for m in mods)
+    q_a = torch.empty((M, kmax), dtype=torch.int8, device=device)
+    s_a = torch.empty((M,), dtype=torch.float32, device=device)
+    vp = ctypes.c_void_p
+
+    def check(rc):
+        if rc != 0:
+            raise RuntimeError(f"qift call failed: {qift.status_string(rc)}")
+
+    def step_full(stream):
+        st = vp(stream)
+        for m in mods:
+            check(L.qift_quantize_act(vp(m.x.data_ptr()), qift.F32, M, m.K, m.B, CLIP, vp(q_a.data_ptr()), vp(s_a.data_ptr()), st))
+            check(L.qift_w2a4_linear(vp(m.packed.data_ptr()), vp(m.s_n.data_ptr()), m.levels, vp(q_a.data_ptr()),
+                                     vp(s_a.data_ptr()), M, m.N, m.K, vp(m.y.data_ptr()), qift.F32, None, None, 0, st))
+        return 2 * len(mods)
+
+    def step_product_only(stream):
+        st = vp(stream)
+        for m in mods:
+            check(L.qift_w2a4_linear(vp(m.packed.data_ptr()), vp(m.s_n.data_ptr()), m.levels, vp(q_a.data_ptr()),
+                                     vp(s_a.data_ptr()), M, m.N, m.K, vp(m.y.data_ptr()), qift.F32, None, None, 0, st))
+        return len(mods)
+
+    scratch_bytes = max(qift.qift_forward_scratch_bytes(M, m.N, m.K, m.levels, qift.F32, qift.F32) for m in mods)
+    scratch = torch.empty(scratch_bytes, dtype=torch.uint8, device=device)
+
+    def step_host(stream):
+        st = vp(stream)
+        for m in mods:
+            check(L.qift_forward_host(vp(m.x_host.data_ptr()), qift.F32, M, m.K, m.B, CLIP, vp(m.packed.data_ptr()),
+                                      vp(m.s_n.data_ptr()), m.levels, m.N, vp(m.y_host.data_ptr()), qift.F32,
+                                      vp(scratch.data_ptr()), scratch_bytes, st))
+
+    def capture(fn):
+        """Capture one step into a CUDA graph (programmatic-dependent-launch edges included)."""
+        side = torch.cuda.Stream(device=device)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn(side.cuda_stream)   # warm-up outside capture: attribute calls, lazy module load
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        try:
+            with torch.cuda.graph(g, stream=side):
+                n = fn(torch.cuda.current_stream().cuda_stream)
+            return g, n
+        except Exception as e:  # noqa: BLE001
+            sys.stderr.write(f"bench: graph capture failed ({e}); timing direct launches\n")
+            return None, fn(torch.cuda.current_stream().cuda_stream)
+
+    def timed(run_once, steps, warmup):
+        for _ in range(warmup):
+            run_once()
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            run_once()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if dist:
+            t = torch.tensor([ms], device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+            dist.barrier()
+        return ms
+
+    stream = torch.cuda.current_stream()
+    g_full, n_full = capture(step_full)
+    g_prod, n_prod = capture(step_product_only)
+    run_full = (lambda: g_full.replay()) if g_full else (lambda: step_full(stream.cuda_stream))
+    run_prod = (lambda: g_prod.replay()) if g_prod else (lambda: step_product_only(stream.cuda_stream))
+
+    bytes_product = sum(product_bytes(M, m.N, m.K, m.bits) for m in mods)
+    bytes_step = bytes_product + sum(quant_bytes(M, m.K) for m in mods)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms_full = timed(run_full, args.steps, args.warmup)
+    clocks = sampler.stop()
+    ms_prod = timed(run_prod, args.steps, args.warmup)
+
+    # end to end: host buffers in, host buffers out, copies inside the timed region
+    def run_host():
+        step_host(stream.cuda_stream)
+        stream.synchronize()
+    e2e_steps = max(3, min(args.steps, 20))
+    ms_host = timed(run_host, e2e_steps, 3)
+    rc, detail = qift.qift_device_status()
+    if rc != 0:
+        raise RuntimeError(f"device status {rc} detail {detail:#x}")
+
+    pk = peaks()
+    step_ms = ms_full / args.steps
+    value = world * bytes_step / (step_ms * 1e-3) / 1e9
+    prod_ms = ms_prod / args.steps
+    launch_us = prod_ms * 1e3 / n_prod
+    achieved = (bytes_product / n_prod) / (launch_us * 1e-6) / 1e9
+    host_ms = ms_host / e2e_steps
+    out = {
+        "metric": "w2a4_decode_hbm_gbs", "value": round(value, 2), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(step_ms, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": "config 2: LLaMA-2-7B-shaped decode, M=1, 7 linear shapes x 32 layers of distinct weights, "
+                               "MNZ {+-1,+-3}, Hadamard + INT4 act quant + W2A4 product per module",
+                   "tokens_per_step": M, "modules_per_step": len(mods), "packed_weight_bytes": sum(m.packed.numel() * 4 for m in mods),
+                   "l2": "inputs larger than L2: each step streams 1.63 GB of distinct packed weights",
+                   "cuda_graph": g_full is not None, "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+        "tokens_per_s": round(world * M / (step_ms * 1e-3), 1),
+        "pct_of_8TBs": round(100 * value / world / 8000.0, 2),
+        "roofline": {"bound": "hbm", "kernel": "linear_decode_kernel", "achieved": round(achieved, 1), "peak": pk["hbm_gbs"],
+                     "unit": "GB/s", "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": None,
+                     "peak_source": pk["source"], "avg_launch_us": round(launch_us, 3),
+                     "algorithmic_bytes_per_launch": round(bytes_product / n_prod)},
+        "e2e": {"value": round(world * bytes_step / (host_ms * 1e-3) / 1e9, 2), "unit": "GB/s",
+                "h2d_bytes_per_step": sum(M * m.K * 4 for m in mods), "d2h_bytes_per_step": sum(M * m.N * 4 for m in mods),
+                "ms_per_step": round(host_ms, 4), "api": "qift_forward_host"},
+        "gpu_launches": n_full * args.steps,
+        "clocks": clocks,
+    }
+    if rank == 0 and world == 1 and not args.no_prefill:
+        out["prefill"] = run_prefill(torch, qift, L, device, gen, pk)
+    if rank == 0 and world == 1 and not args.no_cpu:
+        out["cpu_baseline"] = cpu_baseline(budget_s=12.0)
+    if rank == 0:
+        print(json.dumps(out))
+    if dist:
+        dist.destroy_process_group()
+
+
+def run_prefill(torch, qift, L, device, gen, pk):
+    """Config 4: LLaMA-3.1-8B shapes, M = 2048 tokens, bf16 in, bf16 out, MNZ."""
+    M = 2048
+    mods = build_stack(torch, qift, synth.LLAMA31_8B, 1, M, lambda l: qift.MNZ, 4000, torch.bfloat16, torch.bfloat16, device, gen)
+    kmax = max(m.K for m in mods)
+    q_a = torch.empty((M, kmax), dtype=torch.int8, device=device)
+    s_a = torch.empty((M,), dtype=torch.float32, device=device)
+    ws_bytes = max(qift.qift_workspace_bytes(M, m.N, m.K, m.levels) for m in mods)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
+    vp = ctypes.c_void_p
+    st = vp(torch.cuda.current_stream().cuda_stream)
+
+    def layer(with_quant=True):
+        for m in mods:
+            if with_quant:
+                rc = L.qift_quantize_act(vp(m.x.data_ptr()), qift.BF16, M, m.K, m.B, CLIP, vp(q_a.data_ptr()), vp(s_a.data_ptr()), st)
+                assert rc == 0, rc
+            rc = L.qift_w2a4_linear(vp(m.packed.data_ptr()), vp(m.s_n.data_ptr()), m.levels, vp(q_a.data_ptr()), vp(s_a.data_ptr()),
+                                    M, m.N, m.K, vp(m.y.data_ptr()), qift.BF16, None, vp(ws.data_ptr()), ws_bytes, st)
+            assert rc == 0, rc
+
+    res = {}
+    for key, wq in (("layer_with_act_quant", True), ("product_only", False)):
+        for _ in range(3):
+            layer(wq)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        iters = 10
+        e0.record()
+        for _ in range(iters):
+            layer(wq)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / iters
+        ops = sum(2.0 * M * m.N * m.K for m in mods)
+        res[key] = {"ms_per_layer": round(ms, 4), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
+    tops = res["product_only"]["tops"]
+    int8_peak = 2.0 * pk["bf16_tflops"]    # dense int8 is nominally 2x bf16; scaled from the measured bf16 burst
+    res.update({"workload": "config 4: LLaMA-3.1-8B shapes, M=2048, 7 modules, MNZ, bf16 out", "unit": "TOPS",
+                "pct_of_nominal_4500": round(100 * tops / 4500.0, 2),
+                "roofline": {"bound": "tensor", "kernel": "gemm_i8_tcgen05_kernel (+ expand_levels_kernel)", "achieved": tops,
+                             "peak": int8_peak, "unit": "TOP/s", "frac": round(tops / int8_peak, 4),
+                             "peak_source": f"2 x {pk['source']} bf16 burst"},
+                "tokens_per_s": round(M / (res["layer_with_act_quant"]["ms_per_layer"] * 1e-3), 1)})
+    return res
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle timing (baseline / reference arm)
+# ------------------------------------------------------------------------------------------------
+def oracle_layer_inputs():
+    import oracle
+    mods = []
+    for i, (name, N, K) in enumerate(synth.LLAMA2_7B):
+        rng = np.random.default_rng(2000 + i)
+        codes = rng.integers(0, 4, (N, K), dtype=np.uint8)      # timing only: any codes cost the same
+        s_n = np.full((N,), 0.01, dtype=np.float32)
+        x, _ = synth.activations(synth.config_seed(2, i, 1), 1, K, max(1, round(0.01 * K)))
+        mods.append((name, N, K, codes, s_n, x))
+    return oracle, mods
+
+
+def oracle_layer_once(oracle, mods):
+    for (_, N, K, codes, s_n, x) in mods:
+        q_a, s_a = oracle.quantize_act(x, synth.had_block_for(K), CLIP)
+        oracle.linear(codes, oracle.MNZ, s_n, q_a, s_a)
+
+
+def layer_bytes():
+    return sum(product_bytes(1, N, K) + quant_bytes(1, K) for _, N, K in synth.LLAMA2_7B)
+
+
+def cpu_baseline(budget_s=12.0):
+    oracle, mods = oracle_layer_inputs()
+    oracle_layer_once(oracle, mods)
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        oracle_layer_once(oracle, mods)
+        reps += 1
+        if time.perf_counter() - t0 > budget_s or reps >= N_LAYERS:
+            break
+    dt = time.perf_counter() - t0
+    return {"value": round(reps * layer_bytes() / dt / 1e9, 4), "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "sample": f"{reps} of 32 layers (7 modules each, M=1) of the same workload, single thread, {dt:.1f} s",
+            "host": f"{os.cpu_count()} logical cores"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    oracle, mods = oracle_layer_inputs()
+    for _ in range(max(1, min(args.warmup, 2))):
+        oracle_layer_once(oracle, mods)
+    steps = max(1, min(args.steps, 20))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_layer_once(oracle, mods)
+    dt = time.perf_counter() - t0
+    # one reference "step" is a bounded sample: 1 of the 32 layers; scale to the full step
+    step_s = dt / steps * N_LAYERS
+    value = N_LAYERS * layer_bytes() / step_s / 1e9
+    sample = f"each step = 1 of 32 layers (7 modules, M=1), {steps} steps, single thread; ms_per_step scaled x32"
+    print(json.dumps({
+        "impl": "reference", "metric": "w2a4_decode_hbm_gbs", "value": round(value, 4), "unit": "GB/s",
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": steps, "warmup": args.warmup,
+        "ms_per_step": round(step_s * 1e3, 2), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32", "data": "synthetic",
+        "config": {"workload": "config 2: LLaMA-2-7B-shaped decode, M=1, 7 linear shapes x 32 layers, MNZ; CPU oracle"},
+        "cpu_baseline": {"value": round(value, 4), "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-prefill", action="store_true", help="skip the M=2048 prefill measurement")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -109,7 +109,7 @@ int qift_quantize_act(const void* X, int x_dtype, int M, int K, int had_block, f
  *   q_a, s_a      from qift_quantize_act
  *   Y         out [M,N] fp32 or bf16 (round to nearest even): ((float)acc * s_a[m]) * s_n[n]
  *   acc_debug out int32 [M,N] accumulators, or NULL
- *   workspace     >= qift_workspace_bytes(M,N,K,levels) bytes, 1024-byte aligned; may be NULL when 0
+ *   workspace     >= qift_workspace_bytes(M,N,K,levels) bytes, 256-byte aligned; may be NULL when 0
  * M <= 16 takes the decode route, larger M the prefill route. */
 int qift_w2a4_linear(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a,
                      const float* s_a, int M, int N, int K, void* Y, int y_dtype, int32_t* acc_debug,
@@ -125,6 +125,22 @@ int qift_w4a4_linear(const uint32_t* packed, const float* s_n, const int8_t* q_a
 int qift_linear_route(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a,
                       const float* s_a, int M, int N, int K, void* Y, int y_dtype, int32_t* acc_debug,
                       void* workspace, size_t workspace_bytes, int route, void* stream);
+
+/* Whole layer in one call, S2..S5: qift_quantize_act followed by the product, X and Y on the device.
+ *   scratch  >= qift_forward_scratch_bytes(...) bytes of device memory, 256-byte aligned; holds
+ *            q_a, s_a and (for M > 16) the prefill workspace.  Contents are undefined afterwards. */
+size_t qift_forward_scratch_bytes(int M, int N, int K, int levels, int x_dtype, int y_dtype);
+int qift_forward(const void* X, int x_dtype, int M, int K, int had_block, float clip_ratio,
+                 const uint32_t* packed, const float* s_n, int levels, int N, void* Y, int y_dtype,
+                 void* scratch, size_t scratch_bytes, void* stream);
+
+/* The same with X and Y in HOST memory (pinned memory makes the copies asynchronous): the call
+ * enqueues the host-to-device copy of X, the layer, and the device-to-host copy of Y on `stream`;
+ * Y_host is valid once the stream has been synchronized.  The scratch additionally holds the
+ * device copies of X and Y (qift_forward_scratch_bytes already counts them). */
+int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_block, float clip_ratio,
+                      const uint32_t* packed, const float* s_n, int levels, int N, void* Y_host,
+                      int y_dtype, void* scratch, size_t scratch_bytes, void* stream);
 
 /* Synchronizes `stream`, then reads and clears the device status word in which a kernel records an
  * expired bounded wait.  QIFT_OK, QIFT_ERR_TIMEOUT or QIFT_ERR_CUDA.  `detail` (host, may be NULL)

@@ -24,7 +24,7 @@ ROUTE_AUTO, ROUTE_GENERIC, ROUTE_DECODE, ROUTE_PREFILL = 0, 1, 2, 3
 EXPORTS = [
     "qift_status_string", "qift_packed_bytes", "qift_workspace_bytes", "qift_pack_weights",
     "qift_unpack_codes", "qift_rotate", "qift_quantize_act", "qift_w2a4_linear", "qift_w4a4_linear",
-    "qift_linear_route", "qift_device_status",
+    "qift_linear_route", "qift_device_status", "qift_forward_scratch_bytes", "qift_forward", "qift_forward_host",
 ]
 
 _lib = None
@@ -60,8 +60,14 @@ def lib() -> ctypes.CDLL:
         L.qift_w4a4_linear.argtypes = [vp, vp, vp, vp, ci, ci, ci, vp, ci, vp, vp, sz, vp]
         L.qift_linear_route.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, vp, ci, vp, vp, sz, ci, vp]
         L.qift_device_status.argtypes = [vp, vp]
+        L.qift_forward_scratch_bytes.restype = sz
+        L.qift_forward_scratch_bytes.argtypes = [ci, ci, ci, ci, ci, ci]
+        fwd = [vp, ci, ci, ci, ci, cf, vp, vp, ci, ci, vp, ci, vp, sz, vp]
+        L.qift_forward.argtypes = fwd
+        L.qift_forward_host.argtypes = fwd
         for name in EXPORTS:
-            if name not in ("qift_status_string", "qift_packed_bytes", "qift_workspace_bytes"):
+            if name not in ("qift_status_string", "qift_packed_bytes", "qift_workspace_bytes",
+                            "qift_forward_scratch_bytes"):
                 getattr(L, name).restype = ci
         _lib = L
     return _lib
@@ -192,3 +198,38 @@ def qift_device_status():
     detail = ctypes.c_uint32(0)
     rc = lib().qift_device_status(_stream(), ctypes.byref(detail))
     return rc, detail.value
+
+
+def _dt(t):
+    assert t.dtype in (torch.float32, torch.bfloat16)
+    return F32 if t.dtype == torch.float32 else BF16
+
+
+def qift_forward_scratch_bytes(M: int, N: int, K: int, levels: int, x_dtype: int = F32, y_dtype: int = F32) -> int:
+    return int(lib().qift_forward_scratch_bytes(M, N, K, levels, x_dtype, y_dtype))
+
+
+def _forward(fn, X, had_block, clip_ratio, packed, s_n, levels, out, scratch):
+    M, K = X.shape
+    N = packed.shape[0]
+    need = qift_forward_scratch_bytes(M, N, K, levels, _dt(X), _dt(out))
+    if scratch is None:
+        scratch = torch.empty(need, dtype=torch.uint8, device=packed.device)
+    _check(fn(_ptr(X), _dt(X), M, K, had_block, clip_ratio, _ptr(_dev(packed)), _ptr(_dev(s_n, torch.float32)), levels, N,
+              _ptr(out), _dt(out), _ptr(_dev(scratch)), scratch.numel(), _stream()), "qift_forward")
+    return out
+
+
+def qift_forward(X, had_block, packed, s_n, levels, clip_ratio: float = 0.9, out_dtype=torch.float32, out=None,
+                 scratch=None):
+    """Whole layer on device tensors: rotate + quantize X [M,K], multiply, scale -> Y [M,N]."""
+    _dev(X)
+    if out is None:
+        out = torch.empty((X.shape[0], packed.shape[0]), dtype=out_dtype, device=X.device)
+    return _forward(lib().qift_forward, X, had_block, clip_ratio, packed, s_n, levels, out, scratch)
+
+
+def qift_forward_host(X_host, had_block, packed, s_n, levels, out_host, clip_ratio: float = 0.9, scratch=None):
+    """Whole layer with X and Y in (pinned) host tensors; Y is valid after the stream is synchronized."""
+    assert not X_host.is_cuda and not out_host.is_cuda and X_host.is_contiguous() and out_host.is_contiguous()
+    return _forward(lib().qift_forward_host, X_host, had_block, clip_ratio, packed, s_n, levels, out_host, scratch)

@@ -34,10 +34,27 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Opt a kernel in to more than 48 KiB of dynamic shared memory; remembered per kernel so that the
+// steady state (and any stream capture after a warm-up call) makes no attribute call.
 template <typename K>
 cudaError_t allow_smem(K kernel, size_t bytes) {
-    if (bytes <= 48 * 1024) return cudaSuccess;
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+    if (bytes <= 32 * 1024) return cudaSuccess;  // static shared memory counts against the 48 KiB default too
+    struct Entry {
+        const void* fn;
+        size_t bytes;
+    };
+    static Entry table[64];
+    static int used = 0;
+    const void* key = reinterpret_cast<const void*>(kernel);
+    Entry* slot = nullptr;
+    for (int i = 0; i < used; ++i)
+        if (table[i].fn == key) slot = &table[i];
+    if (slot && bytes <= slot->bytes) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+    if (e != cudaSuccess) return e;
+    if (!slot && used < 64) slot = &table[used++], slot->fn = key;
+    if (slot) slot->bytes = bytes;
+    return e;
 }
 
 inline int cuda_status(cudaError_t e) {
@@ -160,7 +177,7 @@ int run_prefill(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
     if (K % 16 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;  // TMA row pitch must be a multiple of 16 bytes
     const size_t need = qift_workspace_bytes(17 > M ? 17 : M, N, K, lv);
     if (!workspace || workspace_bytes < need) return QIFT_ERR_WORKSPACE;
-    if ((reinterpret_cast<uintptr_t>(workspace) & 1023u) != 0) return QIFT_ERR_ALIGNMENT;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
     int8_t* wexp = static_cast<int8_t*>(workspace);
     int rc;
     switch (lv) {
@@ -332,6 +349,82 @@ int qift_linear_route(const uint32_t* packed, const float* s_n, int levels, cons
                       int K, void* Y, int y_dtype, int32_t* acc_debug, void* workspace, size_t workspace_bytes, int route,
                       void* stream) {
     return linear_impl(packed, s_n, levels, q_a, s_a, M, N, K, Y, y_dtype, acc_debug, workspace, workspace_bytes, route, stream);
+}
+
+namespace {
+struct ForwardLayout {
+    size_t x_off, q_off, sa_off, y_off, ws_off, total;
+};
+inline size_t up1k(size_t v) { return (v + 1023) & ~static_cast<size_t>(1023); }
+ForwardLayout forward_layout(int M, int N, int K, int levels, int x_dtype, int y_dtype) {
+    ForwardLayout L;
+    size_t o = 0;
+    L.x_off = o, o += up1k(static_cast<size_t>(M) * K * (x_dtype == QIFT_BF16 ? 2 : 4));
+    L.q_off = o, o += up1k(static_cast<size_t>(M) * K);
+    L.sa_off = o, o += up1k(static_cast<size_t>(M) * 4);
+    L.y_off = o, o += up1k(static_cast<size_t>(M) * N * (y_dtype == QIFT_BF16 ? 2 : 4));
+    L.ws_off = o, o += qift_workspace_bytes(M, N, K, levels);
+    L.total = o;
+    return L;
+}
+}  // namespace
+
+size_t qift_forward_scratch_bytes(int M, int N, int K, int levels, int x_dtype, int y_dtype) {
+    if (M <= 0 || N <= 0 || K <= 0 || !valid_levels(levels)) return 0;
+    return forward_layout(M, N, K, levels, x_dtype, y_dtype).total;
+}
+
+static int forward_impl(const void* X, bool host, int x_dtype, int M, int K, int had_block, float clip_ratio,
+                        const uint32_t* packed, const float* s_n, int levels, int N, void* Y, int y_dtype, void* scratch,
+                        size_t scratch_bytes, void* stream) {
+    if (!X || !Y || !packed || !s_n || M <= 0 || N <= 0 || K <= 0 || !valid_levels(levels)) return QIFT_ERR_INVALID_ARG;
+    if ((x_dtype != QIFT_F32 && x_dtype != QIFT_BF16) || (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16))
+        return QIFT_ERR_INVALID_ARG;
+    if (K % codes_per_word(levels) != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    const int rs = check_rotation_shape(K, had_block, true);
+    if (rs != QIFT_OK) return rs;
+    const ForwardLayout L = forward_layout(M, N, K, levels, x_dtype, y_dtype);
+    if (!scratch || scratch_bytes < L.total) return QIFT_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(scratch) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* base = static_cast<unsigned char*>(scratch);
+    const void* x_dev = X;
+    void* y_dev = Y;
+    if (host) {
+        x_dev = base + L.x_off;
+        y_dev = base + L.y_off;
+        cudaError_t e = cudaMemcpyAsync(base + L.x_off, X, static_cast<size_t>(M) * K * (x_dtype == QIFT_BF16 ? 2 : 4),
+                                        cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return cuda_status(e);
+    }
+    int8_t* q_a = reinterpret_cast<int8_t*>(base + L.q_off);
+    float* s_a = reinterpret_cast<float*>(base + L.sa_off);
+    int rc = qift_quantize_act(x_dev, x_dtype, M, K, had_block, clip_ratio, q_a, s_a, stream);
+    if (rc != QIFT_OK) return rc;
+    rc = linear_impl(packed, s_n, levels, q_a, s_a, M, N, K, y_dev, y_dtype, nullptr, base + L.ws_off, L.total - L.ws_off,
+                     QIFT_ROUTE_AUTO, stream);
+    if (rc != QIFT_OK) return rc;
+    if (host) {
+        cudaError_t e = cudaMemcpyAsync(Y, y_dev, static_cast<size_t>(M) * N * (y_dtype == QIFT_BF16 ? 2 : 4),
+                                        cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return cuda_status(e);
+    }
+    return QIFT_OK;
+}
+
+int qift_forward(const void* X, int x_dtype, int M, int K, int had_block, float clip_ratio, const uint32_t* packed,
+                 const float* s_n, int levels, int N, void* Y, int y_dtype, void* scratch, size_t scratch_bytes, void* stream) {
+    if (X && !aligned16(X)) return QIFT_ERR_ALIGNMENT;
+    if (Y && !aligned16(Y)) return QIFT_ERR_ALIGNMENT;
+    return forward_impl(X, false, x_dtype, M, K, had_block, clip_ratio, packed, s_n, levels, N, Y, y_dtype, scratch,
+                        scratch_bytes, stream);
+}
+
+int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_block, float clip_ratio, const uint32_t* packed,
+                      const float* s_n, int levels, int N, void* Y_host, int y_dtype, void* scratch, size_t scratch_bytes,
+                      void* stream) {
+    return forward_impl(X_host, true, x_dtype, M, K, had_block, clip_ratio, packed, s_n, levels, N, Y_host, y_dtype, scratch,
+                        scratch_bytes, stream);
 }
 
 int qift_device_status(void* stream, uint32_t* detail) {

@@ -176,7 +176,7 @@ def run_gpu(args):
     M = 1
     launches = [0]
 
-    mods = build_stack(torch, qift, synth.LLAMA2_7B, N_LAYERS, M, lambda l: qift.MNZ, 2000, torch.float32, torch.float32,
+    mods = build_stack(torch, qift, synth.LLAMA2_7B, args.layers, M, lambda l: qift.MNZ, 2000, torch.float32, torch.float32,
                        device, gen)
     kmax = max(m.K for m in mods)
     q_a = torch.empty((M, kmax), dtype=torch.int8, device=device)
@@ -286,9 +286,10 @@ def run_gpu(args):
         "warmup": args.warmup, "ms_per_step": round(step_ms, 5), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int32", "data": "synthetic",
         "config": {"workload": "config 2: LLaMA-2-7B-shaped decode, M=1, 7 linear shapes x 32 layers of distinct weights, "
-                               "MNZ {+-1,+-3}, Hadamard + INT4 act quant + W2A4 product per module",
+                               "MNZ {+-1,+-3}, Hadamard + INT4 act quant + W2A4 product per module" +
+                               ("" if args.layers == N_LAYERS else f" [REDUCED to {args.layers} layers: not a bench number]"),
                    "tokens_per_step": M, "modules_per_step": len(mods), "packed_weight_bytes": sum(m.packed.numel() * 4 for m in mods),
-                   "l2": "inputs larger than L2: each step streams 1.63 GB of distinct packed weights",
+                   "l2": f"inputs larger than L2: each step streams {sum(m.packed.numel() * 4 for m in mods) / 1e9:.2f} GB of distinct packed weights",
                    "cuda_graph": g_full is not None, "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
         "tokens_per_s": round(world * M / (step_ms * 1e-3), 1),
         "pct_of_8TBs": round(100 * value / world / 8000.0, 2),
@@ -433,6 +434,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=N_LAYERS, help="layers of distinct weights per step (32 = the full workload)")
     ap.add_argument("--no-prefill", action="store_true", help="skip the M=2048 prefill measurement")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     args = ap.parse_args()

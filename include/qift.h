@@ -62,7 +62,8 @@ typedef enum {
 
 const char* qift_status_string(int status);
 
-/* Bytes of the packed weight buffer: N*K/4 for the two-bit sets, N*K/2 for INT4.  0 on bad input. */
+/* Bytes of the packed weight buffer: N*K/4 for the two-bit sets, N*K/2 for INT4, after padding N and
+ * the words per row to multiples of 16.  0 on bad input. */
 size_t qift_packed_bytes(int N, int K, int levels);
 
 /* Bytes of scratch qift_w2a4_linear / qift_w4a4_linear need for this problem (0 when the decode
@@ -72,18 +73,24 @@ size_t qift_workspace_bytes(int M, int N, int K, int levels);
 /* S1 (weight quantizer + packer).  Sec. 1 Eq. 1, Sec. 3.3, Sec. 3.5.
  *   W       in   fp32 [N,K], ALREADY rotated (this call never rotates)
  *   s_n     in for QIFT_SCALE_GIVEN (must be > 0), out otherwise; fp32 [N]
- *   packed  out  uint32 [N, K/16] (two-bit sets) or [N, K/8] (INT4); qift_packed_bytes() bytes
+ *   packed  out  qift_packed_bytes(N,K,levels) bytes of uint32 words in the tiled order below
  * Code of a weight: t = w / s_n (IEEE division).  No-zero sets: nearest level, an exact midpoint
  * goes to the lower level, values beyond the outer levels saturate.  SYM / INT4: Eq. 1 literally,
  * round-half-to-even then clip to [-2,1] / [-8,7]; SYM stores q+2, INT4 stores q & 15.
- * Word layout: word j of a row holds codes k = 16j..16j+15; code k = 16j + 4t + b sits at bits
+ * Bits in a word: word j of a row holds codes k = 16j..16j+15; code k = 16j + 4t + b sits at bits
  * [8b+2t+1 : 8b+2t] (INT4: k = 8j + 4t + b at bits [8b+4t+3 : 8b+4t]), so (word >> 2t) & 0x03030303
  * is four consecutive-k codes, one per byte.
+ * Order of the words in memory: tiles of 16 rows x 128 words (the last tile of a row block may be
+ * narrower), row blocks outermost, then ascending k.  Inside a tile, 16-byte groups of four
+ * consecutive words of one row, group index ((slice*2 + half)*32 + (row%8)*4 + quad) with
+ * slice = (j%128)/16, half = (row%16)/8, quad = (j%16)/4.  Rows and words per row are padded to
+ * multiples of 16 with zero words (no padding for any LLaMA shape).  A tile is one 8 KB contiguous
+ * block, and the 32 groups a warp needs for one mma step are 512 contiguous bytes.
  * Requires K % 16 == 0 (K % 8 == 0 for INT4) and K <= 16384. */
 int qift_pack_weights(const float* W, int N, int K, int levels, int scale_mode, float* s_n,
                       uint32_t* packed, void* stream);
 
-/* Inverse of the word layout, for tests: codes uint8 [N,K] (INT4: the nibble 0..15). */
+/* Inverse of the packed layout, for tests: codes uint8 [N,K] (INT4: the nibble 0..15). */
 int qift_unpack_codes(const uint32_t* packed, int N, int K, int levels, uint8_t* codes, void* stream);
 
 /* S0 (offline rotation, Sec. 3.1 / Sec. 4.1): Y = X Q with Q = blockdiag(H_B) / sqrt(B), H_B the
@@ -141,6 +148,42 @@ int qift_forward(const void* X, int x_dtype, int M, int K, int had_block, float 
 int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_block, float clip_ratio,
                       const uint32_t* packed, const float* s_n, int levels, int N, void* Y_host,
                       int y_dtype, void* scratch, size_t scratch_bytes, void* stream);
+
+/* ---- Grouped decode path -----------------------------------------------------------------------
+ * One persistent launch serves a list of independent layer problems that share M (<= 16 token rows),
+ * the level set, the dtypes and the clip ratio -- e.g. all linear modules of one decode step.  A W2
+ * matrix is only 1-15 MB, far too little for one launch to reach an HBM steady state; the grouped
+ * kernel streams the whole list back to back.  (No counterpart in the paper: it describes no kernels.)
+ *
+ * qift_group_plan validates the list and writes a plan into caller memory: `plan_host` (host) and
+ * `plan_dev` (device), each qift_group_plan_bytes(count) bytes; the device copy is enqueued on
+ * `stream`.  The plan holds the caller's pointers, so it stays valid while those buffers live;
+ * plan_host must stay alive and unchanged while the plan is used.  The run calls enqueue
+ *   qift_group_quantize_act : S2+S3 for every problem (one launch)  X -> q_a, s_a
+ *   qift_group_linear       : S4+S5 for every problem (one launch)  q_a, s_a -> Y
+ *   qift_group_forward      : both.
+ * Problems must not alias each other's q_a / s_a / Y.  K % 256 == 0 (two-bit sets) or K % 128 == 0
+ * (INT4), K <= 16384. */
+typedef struct qift_group_problem {
+    const void* X;          /* dev [M,K] fp32 or bf16                         */
+    const uint32_t* packed; /* dev, from qift_pack_weights                    */
+    const float* s_n;       /* dev [N]                                        */
+    int8_t* q_a;            /* dev [M,K] scratch: quantized activations       */
+    float* s_a;             /* dev [M]   scratch: token scales                */
+    void* Y;                /* dev [M,N] output                               */
+    int32_t* acc_debug;     /* dev [M,N] INT32 accumulators, or NULL          */
+    int N, K;
+    int had_block;          /* 0 = no rotation, else power of two dividing K  */
+    int reserved;
+} qift_group_problem;
+
+size_t qift_group_plan_bytes(int count);
+int qift_group_plan(const qift_group_problem* problems /*host*/, int count, int M, int levels, int x_dtype,
+                    int y_dtype, float clip_ratio, void* plan_host, void* plan_dev, size_t plan_bytes,
+                    void* stream);
+int qift_group_quantize_act(const void* plan_host, const void* plan_dev, void* stream);
+int qift_group_linear(const void* plan_host, const void* plan_dev, void* stream);
+int qift_group_forward(const void* plan_host, const void* plan_dev, void* stream);
 
 /* Synchronizes `stream`, then reads and clears the device status word in which a kernel records an
  * expired bounded wait.  QIFT_OK, QIFT_ERR_TIMEOUT or QIFT_ERR_CUDA.  `detail` (host, may be NULL)

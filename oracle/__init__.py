@@ -46,6 +46,7 @@ def lib():
         _lib.orc_row_sqerr.restype = ctypes.c_double
         _lib.orc_row_sqerr.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_float]
         _lib.orc_int_matmul.restype = ctypes.c_longlong
+        _lib.orc_packed_words.restype = ctypes.c_longlong
     return _lib
 
 
@@ -152,20 +153,26 @@ def codes_per_word(lv: int) -> int:
     return 8 if lv == INT4 else 16
 
 
+def packed_words(N: int, K: int, lv: int) -> int:
+    """Words of the packed buffer: rows padded to a multiple of 16."""
+    return int(lib().orc_packed_words(N, K, int(lv)))
+
+
 def pack(codes, lv: int):
+    """codes uint8 [N,K] -> flat uint32 buffer in the tiled layout."""
     codes = np.ascontiguousarray(codes, dtype=np.uint8)
     N, K = codes.shape
     per = codes_per_word(lv)
     assert K % per == 0
-    out = np.empty((N, K // per), dtype=np.uint32)
+    out = np.empty((packed_words(N, K, lv),), dtype=np.uint32)
     lib().orc_pack(codes.ctypes.data_as(ctypes.c_void_p), N, K, int(lv),
                    out.ctypes.data_as(ctypes.c_void_p))
     return out
 
 
-def unpack(packed, K: int, lv: int):
+def unpack(packed, N: int, K: int, lv: int):
     packed = np.ascontiguousarray(packed, dtype=np.uint32)
-    N = packed.shape[0]
+    assert packed.size == packed_words(N, K, lv)
     out = np.empty((N, K), dtype=np.uint8)
     lib().orc_unpack(packed.ctypes.data_as(ctypes.c_void_p), N, K, int(lv),
                      out.ctypes.data_as(ctypes.c_void_p))
@@ -205,7 +212,7 @@ def epilogue(acc, s_a, s_n, bf16: bool = False):
 
 
 def pack_weights(W, lv: int, mode: int, s_n=None):
-    """Whole S1 step -> (packed uint32 [N, K/per], s_n, codes)."""
+    """Whole S1 step -> (packed uint32 flat (tiled layout), s_n, codes)."""
     if mode == SCALE_GIVEN:
         s = _f32(s_n)
     else:

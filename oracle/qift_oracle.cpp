@@ -20,7 +20,8 @@
 //   orc_weight_scale     Sec. 3.5 / Sec. 4.5.1: per-output-channel scale, either max-range or
 //                        "MSE-optimal by sweeping candidate clipping ratios".
 //   orc_assign_codes     Sec. 3.5 "maps weights to the nearest scaled level"; Eq. 1 for SYM-INT, INT4.
-//   orc_pack / unpack    Sec. 3.3 "four two-bit codes": 16 two-bit codes (8 nibbles) per 32-bit word.
+//   orc_pack / unpack    Sec. 3.3 "four two-bit codes": 16 two-bit codes (8 nibbles) per 32-bit word,
+//                        words stored in 16-row x 128-word tiles (layout comment at orc_pack).
 //   orc_int_matmul       Sec. 3.6 decoded small signed integer levels times integer activations.
 //   orc_epilogue*        Sec. 1 "the per-channel scale can be applied separately in the epilogue".
 //
@@ -228,14 +229,39 @@ void orc_assign_codes(const float* W, int N, int K, int lv, const float* s_n, ui
             codes[(size_t)n * K + k] = (uint8_t)code_of(lv, W[(size_t)n * K + k], s_n[n]);
 }
 
-// Bit position of code k inside its word.
-//   two-bit sets: word j = k / 16, inside it k = 16 j + 4 t + b  ->  bits [8 b + 2 t + 1 : 8 b + 2 t]
-//   INT4:         word j = k / 8,  inside it k =  8 j + 4 t + b  ->  bits [8 b + 4 t + 3 : 8 b + 4 t]
+// Packed layout.
+// Bits inside a word: word j of row n holds codes k = per*j .. per*j + per-1;
+//   two-bit sets: k = 16 j + 4 t + b  ->  bits [8 b + 2 t + 1 : 8 b + 2 t]
+//   INT4:         k =  8 j + 4 t + b  ->  bits [8 b + 4 t + 3 : 8 b + 4 t]
 // so that (word >> (bits * t)) masked per byte yields four consecutive-k codes, one per byte.
+// Order of the words in memory: tiles of 16 rows x 128 words (the last tile of a row block may be
+// narrower), row blocks outermost, tiles of one row block in ascending k.  Inside a tile the words
+// go in groups of four (16 bytes): group index ((slice * 2 + half) * 32 + (row % 8) * 4 + quad),
+// where slice = (j % 128) / 16, quad = (j % 16) / 4, half = (row % 16) / 8; word j % 4 inside the
+// group.  Rows are padded to a multiple of 16 and the words of a row to a multiple of 16, with zero
+// words.
+static inline int pad16(int N) { return (N + 15) / 16 * 16; }
+
+static size_t word_address(int n, int j, int words_per_row) {
+    const int pitch = pad16(words_per_row);
+    const int rb = n / 16, r = n % 16, half = r / 8, g = r % 8;
+    const int c = j / 128, jj = j % 128;
+    const size_t tile = (size_t)rb * 16 * pitch + (size_t)c * 16 * 128;
+    const int slice = jj / 16, quad = (jj % 16) / 4, e = jj % 4;
+    return tile + (size_t)(((slice * 2 + half) * 32 + g * 4 + quad) * 4 + e);
+}
+
+long long orc_packed_words(int N, int K, int lv) {
+    const int per = (lv == LV_INT4) ? 8 : 16;
+    return (long long)pad16(N) * pad16(K / per);
+}
+
 void orc_pack(const uint8_t* codes, int N, int K, int lv, uint32_t* packed) {
     const int per = (lv == LV_INT4) ? 8 : 16;
     const int bits = (lv == LV_INT4) ? 4 : 2;
     const int words = K / per;
+    const long long total = orc_packed_words(N, K, lv);
+    for (long long i = 0; i < total; ++i) packed[i] = 0;
     for (int n = 0; n < N; ++n) {
         for (int j = 0; j < words; ++j) {
             uint32_t w = 0;
@@ -244,7 +270,7 @@ void orc_pack(const uint8_t* codes, int N, int K, int lv, uint32_t* packed) {
                 const uint32_t c = codes[(size_t)n * K + (size_t)j * per + r] & ((1u << bits) - 1u);
                 w |= c << (8 * b + bits * t);
             }
-            packed[(size_t)n * words + j] = w;
+            packed[word_address(n, j, words)] = w;
         }
     }
 }
@@ -257,7 +283,7 @@ void orc_unpack(const uint32_t* packed, int N, int K, int lv, uint8_t* codes) {
         for (int k = 0; k < K; ++k) {
             const int j = k / per, r = k % per, t = r / 4, b = r % 4;
             codes[(size_t)n * K + k] =
-                (uint8_t)((packed[(size_t)n * words + j] >> (8 * b + bits * t)) & ((1u << bits) - 1u));
+                (uint8_t)((packed[word_address(n, j, words)] >> (8 * b + bits * t)) & ((1u << bits) - 1u));
         }
 }
 

@@ -25,6 +25,7 @@ EXPORTS = [
     "qift_status_string", "qift_packed_bytes", "qift_workspace_bytes", "qift_pack_weights",
     "qift_unpack_codes", "qift_rotate", "qift_quantize_act", "qift_w2a4_linear", "qift_w4a4_linear",
     "qift_linear_route", "qift_device_status", "qift_forward_scratch_bytes", "qift_forward", "qift_forward_host",
+    "qift_group_plan_bytes", "qift_group_plan", "qift_group_quantize_act", "qift_group_linear", "qift_group_forward",
 ]
 
 _lib = None
@@ -65,9 +66,14 @@ def lib() -> ctypes.CDLL:
         fwd = [vp, ci, ci, ci, ci, cf, vp, vp, ci, ci, vp, ci, vp, sz, vp]
         L.qift_forward.argtypes = fwd
         L.qift_forward_host.argtypes = fwd
+        L.qift_group_plan_bytes.restype = sz
+        L.qift_group_plan_bytes.argtypes = [ci]
+        L.qift_group_plan.argtypes = [vp, ci, ci, ci, ci, ci, cf, vp, vp, sz, vp]
+        for name in ("qift_group_quantize_act", "qift_group_linear", "qift_group_forward"):
+            getattr(L, name).argtypes = [vp, vp, vp]
         for name in EXPORTS:
             if name not in ("qift_status_string", "qift_packed_bytes", "qift_workspace_bytes",
-                            "qift_forward_scratch_bytes"):
+                            "qift_forward_scratch_bytes", "qift_group_plan_bytes"):
                 getattr(L, name).restype = ci
         _lib = L
     return _lib
@@ -106,22 +112,21 @@ def qift_workspace_bytes(M: int, N: int, K: int, levels: int) -> int:
 
 
 def qift_pack_weights(W, levels: int, scale_mode: int, s_n=None, packed=None):
-    """W fp32 [N,K] (already rotated) -> (packed uint32-as-int32 [N, K/per], s_n fp32 [N])."""
+    """W fp32 [N,K] (already rotated) -> (packed: flat int32 buffer of qift_packed_bytes(N,K) bytes in
+    the tiled storage order, s_n fp32 [N])."""
     _dev(W, torch.float32)
     N, K = W.shape
-    per = 8 if levels == INT4 else 16
     if s_n is None:
         s_n = torch.empty(N, dtype=torch.float32, device=W.device)
     if packed is None:
-        packed = torch.empty((N, max(K // per, 1)), dtype=torch.int32, device=W.device)
+        packed = torch.empty((max(qift_packed_bytes(N, K, levels) // 4, 1),), dtype=torch.int32, device=W.device)
     _check(lib().qift_pack_weights(_ptr(W), N, K, levels, scale_mode, _ptr(_dev(s_n, torch.float32)),
                                    _ptr(_dev(packed)), _stream()), "qift_pack_weights")
     return packed, s_n
 
 
-def qift_unpack_codes(packed, K: int, levels: int):
+def qift_unpack_codes(packed, N: int, K: int, levels: int):
     _dev(packed)
-    N = packed.shape[0]
     codes = torch.empty((N, K), dtype=torch.uint8, device=packed.device)
     _check(lib().qift_unpack_codes(_ptr(packed), N, K, levels, _ptr(codes), _stream()), "qift_unpack_codes")
     return codes
@@ -178,18 +183,19 @@ def _linear(fn_name, packed, s_n, levels, q_a, s_a, N, out_dtype, want_acc, work
 
 
 def qift_w2a4_linear(packed, s_n, levels, q_a, s_a, out_dtype=torch.float32, want_acc=False, workspace=None, out=None):
-    return _linear("qift_w2a4_linear", packed, s_n, levels, q_a, s_a, packed.shape[0], out_dtype, want_acc,
+    """N is the length of s_n."""
+    return _linear("qift_w2a4_linear", packed, s_n, levels, q_a, s_a, s_n.shape[0], out_dtype, want_acc,
                    workspace, ROUTE_AUTO, out)
 
 
 def qift_w4a4_linear(packed, s_n, q_a, s_a, out_dtype=torch.float32, want_acc=False, workspace=None, out=None):
-    return _linear("qift_w4a4_linear", packed, s_n, INT4, q_a, s_a, packed.shape[0], out_dtype, want_acc,
+    return _linear("qift_w4a4_linear", packed, s_n, INT4, q_a, s_a, s_n.shape[0], out_dtype, want_acc,
                    workspace, ROUTE_AUTO, out)
 
 
 def qift_linear_route(packed, s_n, levels, q_a, s_a, route, out_dtype=torch.float32, want_acc=False, workspace=None,
                       out=None):
-    return _linear("qift_linear_route", packed, s_n, levels, q_a, s_a, packed.shape[0], out_dtype, want_acc,
+    return _linear("qift_linear_route", packed, s_n, levels, q_a, s_a, s_n.shape[0], out_dtype, want_acc,
                    workspace, route, out)
 
 
@@ -211,7 +217,7 @@ def qift_forward_scratch_bytes(M: int, N: int, K: int, levels: int, x_dtype: int
 
 def _forward(fn, X, had_block, clip_ratio, packed, s_n, levels, out, scratch):
     M, K = X.shape
-    N = packed.shape[0]
+    N = s_n.shape[0]
     need = qift_forward_scratch_bytes(M, N, K, levels, _dt(X), _dt(out))
     if scratch is None:
         scratch = torch.empty(need, dtype=torch.uint8, device=packed.device)
@@ -225,7 +231,7 @@ def qift_forward(X, had_block, packed, s_n, levels, clip_ratio: float = 0.9, out
     """Whole layer on device tensors: rotate + quantize X [M,K], multiply, scale -> Y [M,N]."""
     _dev(X)
     if out is None:
-        out = torch.empty((X.shape[0], packed.shape[0]), dtype=out_dtype, device=X.device)
+        out = torch.empty((X.shape[0], s_n.shape[0]), dtype=out_dtype, device=X.device)
     return _forward(lib().qift_forward, X, had_block, clip_ratio, packed, s_n, levels, out, scratch)
 
 
@@ -233,3 +239,66 @@ def qift_forward_host(X_host, had_block, packed, s_n, levels, out_host, clip_rat
     """Whole layer with X and Y in (pinned) host tensors; Y is valid after the stream is synchronized."""
     assert not X_host.is_cuda and not out_host.is_cuda and X_host.is_contiguous() and out_host.is_contiguous()
     return _forward(lib().qift_forward_host, X_host, had_block, clip_ratio, packed, s_n, levels, out_host, scratch)
+
+
+class GroupProblem(ctypes.Structure):
+    """Mirror of qift_group_problem."""
+    _fields_ = [("X", ctypes.c_void_p), ("packed", ctypes.c_void_p), ("s_n", ctypes.c_void_p), ("q_a", ctypes.c_void_p),
+                ("s_a", ctypes.c_void_p), ("Y", ctypes.c_void_p), ("acc_debug", ctypes.c_void_p), ("N", ctypes.c_int),
+                ("K", ctypes.c_int), ("had_block", ctypes.c_int), ("reserved", ctypes.c_int)]
+
+
+class GroupPlan:
+    """A validated problem list: host and device copies of the plan plus references that keep every
+    tensor named in it alive."""
+
+    def __init__(self, host, dev, keep, outputs, accs):
+        self.host, self.dev, self.keep, self.outputs, self.accs = host, dev, keep, outputs, accs
+
+
+def qift_group_plan_bytes(count: int) -> int:
+    return int(lib().qift_group_plan_bytes(count))
+
+
+def qift_group_plan(problems, levels: int, clip_ratio: float = 0.9, out_dtype=torch.float32, want_acc: bool = False):
+    """problems: list of (X [M,K], packed, s_n, had_block) sharing M and the dtype of X.  Allocates
+    q_a / s_a / Y (and the accumulators when asked) and returns a GroupPlan."""
+    assert problems
+    M = problems[0][0].shape[0]
+    xdt = _dt(problems[0][0])
+    device = problems[0][0].device
+    arr = (GroupProblem * len(problems))()
+    keep, outs, accs = [], [], []
+    for i, (X, packed, s_n, had_block) in enumerate(problems):
+        _dev(X), _dev(packed), _dev(s_n, torch.float32)
+        assert X.shape[0] == M and _dt(X) == xdt
+        K, N = X.shape[1], s_n.shape[0]
+        q_a = torch.empty((M, K), dtype=torch.int8, device=device)
+        s_a = torch.empty((max(M, 4),), dtype=torch.float32, device=device)
+        Y = torch.empty((M, N), dtype=out_dtype, device=device)
+        acc = torch.empty((M, N), dtype=torch.int32, device=device) if want_acc else None
+        arr[i] = GroupProblem(X.data_ptr(), packed.data_ptr(), s_n.data_ptr(), q_a.data_ptr(), s_a.data_ptr(), Y.data_ptr(),
+                              acc.data_ptr() if want_acc else None, N, K, had_block, 0)
+        keep += [X, packed, s_n, q_a, s_a]
+        outs.append(Y)
+        accs.append(acc)
+    nbytes = qift_group_plan_bytes(len(problems))
+    host = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    dev = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    ydt = F32 if out_dtype == torch.float32 else BF16
+    _check(lib().qift_group_plan(ctypes.addressof(arr), len(problems), M, levels, xdt, ydt, clip_ratio, host.data_ptr(),
+                                 dev.data_ptr(), nbytes, _stream()), "qift_group_plan")
+    return GroupPlan(host, dev, keep, outs, accs)
+
+
+def qift_group_quantize_act(plan: GroupPlan):
+    _check(lib().qift_group_quantize_act(plan.host.data_ptr(), plan.dev.data_ptr(), _stream()), "qift_group_quantize_act")
+
+
+def qift_group_linear(plan: GroupPlan):
+    _check(lib().qift_group_linear(plan.host.data_ptr(), plan.dev.data_ptr(), _stream()), "qift_group_linear")
+
+
+def qift_group_forward(plan: GroupPlan):
+    _check(lib().qift_group_forward(plan.host.data_ptr(), plan.dev.data_ptr(), _stream()), "qift_group_forward")
+    return plan.outputs

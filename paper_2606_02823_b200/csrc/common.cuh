@@ -27,6 +27,28 @@ __host__ __device__ constexpr float top_level(int lv) {
     return lv == QIFT_LEVELS_MNZ ? 3.0f : lv == QIFT_LEVELS_POT ? 4.0f : lv == QIFT_LEVELS_SYM ? 1.0f : 7.0f;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Packed-weight storage order.  Words live in tiles of 16 rows x 128 words (the last tile of a row
+// block may be narrower), row blocks outermost.  Inside a tile, 16-byte groups of four consecutive
+// words of one row are ordered (slice = word/16, half = row/8, row%8, quad = word/4 % 4): the 32
+// groups a warp needs for one mma step (8 rows x 4 quads) are 512 contiguous bytes, so a tile is
+// one bulk copy and every shared-memory read of it is a conflict-free 128-bit access.  Rows and
+// words per row are padded to multiples of 16 with zero words.
+// ------------------------------------------------------------------------------------------------
+constexpr int kTileRows = 16;
+constexpr int kChunkWords = 128;                               // words per row in a full tile
+constexpr int kTileBytes = kTileRows * kChunkWords * 4;        // 8192
+
+__host__ __device__ constexpr int round_up16(int v) { return (v + 15) & ~15; }
+__host__ __device__ inline int packed_pitch(int K, int lv) { return round_up16(K / codes_per_word(lv)); }
+__host__ __device__ inline size_t packed_word_address(int n, int j, int pitch) {
+    const int rb = n >> 4, half = (n >> 3) & 1, g = n & 7;
+    const int c = j >> 7, jj = j & 127;
+    const int slice = jj >> 4, quad = (jj >> 2) & 3, e = jj & 3;
+    return static_cast<size_t>(rb) * 16 * pitch + static_cast<size_t>(c) * (kTileRows * kChunkWords) +
+           static_cast<size_t>((((slice * 2 + half) * 32 + g * 4 + quad) << 2) + e);
+}
+
 template <int LV>
 __device__ __forceinline__ int level_from_code(int c) {
     if constexpr (LV == QIFT_LEVELS_MNZ) return 2 * c - 3;

@@ -2,9 +2,9 @@
 // registers, accumulate exactly in INT32, apply the scales in the epilogue.
 //
 //  * linear_generic_kernel: one warp per output channel, dp4a.  Any M, any K; the slow, simple route.
-//  * linear_decode_kernel:  the bandwidth route.  A producer warp stages [16*RT rows] x [128 words]
-//    slabs of packed weights, and the matching slice of q_a, into a shared-memory ring with
-//    cp.async.bulk + mbarriers.  The weight copies are issued BEFORE the programmatic-dependent-launch
+//  * linear_decode_kernel:  the bandwidth route.  A producer warp stages 16-row x 128-word tiles of
+//    packed weights (8 KB each, contiguous in memory: one cp.async.bulk per tile), and the matching
+//    slice of q_a, into a shared-memory ring guarded by mbarriers.  The weight copies are issued BEFORE the programmatic-dependent-launch
 //    wait, so in a stream of such launches the next layer's weights are in flight while the previous
 //    layer finishes.  Eight consumer warps split each slab along K; a lane turns a packed word into
 //    four u8 operand registers with one LOP3 each (w & (0x03030303 << 2t) = code * 4^t, which the
@@ -48,13 +48,13 @@ linear_generic_kernel(const uint32_t* __restrict__ packed, const float* __restri
     const int n = blockIdx.x * kGenericWarps + (threadIdx.x >> 5);
     if (n >= N) return;
     const int words = K / PER;
-    const uint32_t* wrow = packed + static_cast<size_t>(n) * words;
+    const int pitch = round_up16(words);
     const uint32_t* q32 = reinterpret_cast<const uint32_t*>(q_a);
     const size_t qpitch = K / 4;
     for (int m0 = 0; m0 < M; m0 += kGenericTokens) {
         int S[kGenericTokens] = {}, Sb[kGenericTokens] = {}, Sq[kGenericTokens] = {};
         for (int j = lane; j < words; j += 32) {
-            const uint32_t w = wrow[j];
+            const uint32_t w = packed[packed_word_address(n, j, pitch)];
 #pragma unroll
             for (int t = 0; t < NPL; ++t) {
                 uint32_t a, hb = 0;
@@ -102,8 +102,6 @@ linear_generic_kernel(const uint32_t* __restrict__ packed, const float* __restri
 constexpr int kDecWarps = 8;                       // consumer warps
 constexpr int kDecConsumers = kDecWarps * 32;      // 256
 constexpr int kDecThreads = kDecConsumers + 32;    // + producer warp
-constexpr int kChunkWords = 128;                   // packed words per row per stage (512 B)
-constexpr int kWStride = kChunkWords * 4 + 64;     // row pitch inside a stage: 64 B pad = conflict-free LDS.128
 constexpr int kQPad = 64;
 
 template <int LV>
@@ -131,7 +129,7 @@ struct DecodeParams {
 __host__ __device__ inline size_t decode_stage_bytes(int lv, int rt, int M) {
     const int per = codes_per_word(lv);
     const int nqp = (lv == QIFT_LEVELS_POT) ? 2 : 1;
-    return static_cast<size_t>(rt) * 16 * kWStride + static_cast<size_t>(nqp) * M * (kChunkWords * per + kQPad);
+    return static_cast<size_t>(rt) * kTileBytes + static_cast<size_t>(nqp) * M * (kChunkWords * per + kQPad);
 }
 __host__ __device__ inline size_t decode_smem_bytes(int lv, int rt, int nt, int M, int stages) {
     return stages * decode_stage_bytes(lv, rt, M) + static_cast<size_t>(kDecWarps) * rt * nt * 128 * 4  // reduce
@@ -187,25 +185,27 @@ linear_decode_kernel(const DecodeParams p) {
 
     if (warp == kDecWarps) {
         // ---------------------------------------------------------------- producer warp
+        const int pitch = round_up16(words_per_row);
         const unsigned char* wbase = reinterpret_cast<const unsigned char*>(p.packed) +
-                                     static_cast<size_t>(n0) * words_per_row * 4;
-        const size_t wpitch = static_cast<size_t>(words_per_row) * 4;
+                                     static_cast<size_t>(n0) * pitch * 4;  // first tile of the first row block
+        const size_t rb_bytes = static_cast<size_t>(16) * pitch * 4;
+        const int tiles_valid = (rows_valid + 15) / 16;
         auto chunk_words = [&](int c) { return min(kChunkWords, words_per_row - c * kChunkWords); };
-        auto issue_w = [&](int c, int s) {
-            const uint32_t seg = chunk_words(c) * 4;
+        auto issue_w = [&](int c, int s) {  // one bulk copy per 16-row tile
+            const uint32_t bytes = chunk_words(c) * 16 * 4;
             unsigned char* dst = ring + s * stage_bytes;
-            for (int r = lane; r < rows_valid; r += 32)
-                bulk_g2s(dst + r * kWStride, wbase + r * wpitch + static_cast<size_t>(c) * kChunkWords * 4, seg, &full[s]);
+            if (lane < tiles_valid)
+                bulk_g2s(dst + lane * kTileBytes, wbase + lane * rb_bytes + static_cast<size_t>(c) * kTileBytes, bytes, &full[s]);
         };
         auto issue_q = [&](int c, int s) {
             const uint32_t seg = chunk_words(c) * T::PER;
-            unsigned char* dst = ring + s * stage_bytes + ROWS * kWStride;
+            unsigned char* dst = ring + s * stage_bytes + RT * kTileBytes;
             for (int m = lane; m < M; m += 32)
                 bulk_g2s(dst + m * T::QSTRIDE, p.q_a + static_cast<size_t>(m) * p.K + static_cast<size_t>(c) * T::QBYTES, seg,
                          &full[s]);
         };
         auto expect = [&](int c, int s) {
-            if (lane == 0) mbar_expect_tx(&full[s], chunk_words(c) * (4 * rows_valid + T::PER * M));
+            if (lane == 0) mbar_expect_tx(&full[s], chunk_words(c) * (64 * tiles_valid + T::PER * M));
             __syncwarp();
         };
         const int npre = min(stages, nchunks);
@@ -250,7 +250,7 @@ linear_decode_kernel(const DecodeParams p) {
         }
         const int cw = min(kChunkWords, words_per_row - c * kChunkWords);
         unsigned char* wst = ring + s * stage_bytes;
-        unsigned char* qst = wst + ROWS * kWStride;
+        unsigned char* qst = wst + RT * kTileBytes;
 
         // sum of q per token (and the 5q / 6q planes of POT): every consumer thread owns BPT bytes
         {
@@ -300,8 +300,9 @@ linear_decode_kernel(const DecodeParams p) {
             }
 #pragma unroll
             for (int rt = 0; rt < RT; ++rt) {
-                const uint4 wa = *reinterpret_cast<const uint4*>(wst + (rt * 16 + g) * kWStride + (16 * warp + 4 * cq) * 4);
-                const uint4 wb = *reinterpret_cast<const uint4*>(wst + (rt * 16 + g + 8) * kWStride + (16 * warp + 4 * cq) * 4);
+                // tile order: group ((slice*2 + half)*32 + lane); slice = this warp, half = rows g / g+8
+                const uint4 wa = *reinterpret_cast<const uint4*>(wst + rt * kTileBytes + ((2 * warp) * 32 + lane) * 16);
+                const uint4 wb = *reinterpret_cast<const uint4*>(wst + rt * kTileBytes + ((2 * warp + 1) * 32 + lane) * 16);
                 const uint32_t a_lo[4] = {wa.x, wa.y, wa.z, wa.w};
                 const uint32_t a_hi[4] = {wb.x, wb.y, wb.z, wb.w};
 #pragma unroll

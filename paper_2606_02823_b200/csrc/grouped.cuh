@@ -1,0 +1,405 @@
+// Grouped decode path: ONE persistent launch serves a whole list of independent layer problems
+// (all of one level set and one token count M <= 16), e.g. every linear module of a decode step.
+//
+// A single W2 matrix is 1-15 MB, i.e. 0.15-2 us of HBM time: no per-matrix launch can reach a
+// bandwidth steady state.  Here the work list (problem, 16*RT-row block) is dealt round-robin to a
+// grid of resident CTAs; in each CTA a producer warp streams 8 KB tiles of packed codes (one
+// cp.async.bulk each, plus the matching q_a slices) through a ring of shared-memory stages guarded
+// by mbarriers and keeps running ahead across item boundaries, so HBM requests never drain between
+// matrices; eight consumer warps do the same in-register decode + mma.sync as the per-call kernel.
+#pragma once
+
+#include "common.cuh"
+#include "decode.cuh"
+#include "rotate_quant.cuh"
+
+namespace qift {
+
+struct GroupHeader {
+    uint32_t magic;
+    int count;          // problems
+    int M;              // token rows of every problem
+    int levels;
+    int y_bf16;
+    int x_bf16;
+    float clip;
+    int total_items;    // row blocks over all problems
+    int rows_per_item;  // 16 * RT
+    int max_k;
+    int reserved[6];
+};
+static_assert(sizeof(GroupHeader) == 64, "header is one 64-byte record");
+
+struct GroupProblemDev {
+    const void* X;          // [M,K] activations (fp32 or bf16), input of the quantizer
+    const uint32_t* packed;
+    const float* s_n;
+    int8_t* q_a;            // [M,K] written by the grouped quantizer, read by the product
+    float* s_a;             // [M]
+    void* Y;                // [M,N]
+    int32_t* acc_debug;     // [M,N] or null
+    int N, K, had_block;
+    int item_begin;         // first work item of this problem
+    float inv_sqrt_b;
+    int pad[5];
+};
+static_assert(sizeof(GroupProblemDev) == 96, "problem record is 96 bytes");
+
+constexpr uint32_t kGroupMagic = 0x51494654u;
+
+// ------------------------------------------------------------------------------------------------
+// grouped quantizer: one CTA per (problem, token row)
+// ------------------------------------------------------------------------------------------------
+template <bool BF16_IN>
+__global__ void __launch_bounds__(kRowThreads)
+quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int M, float clip) {
+    extern __shared__ __align__(16) float row[];
+    __shared__ float red[kRowThreads / 32];
+    pdl_launch_dependents();
+    pdl_wait();
+    const GroupProblemDev P = problems[blockIdx.x / M];
+    const size_t m = blockIdx.x % M;
+    const int K = P.K, B = P.had_block;
+    load_and_transform<BF16_IN>(P.X, m, K, B, row);
+    const int groups = K / 16;
+    float amax = 0.0f;
+    for (int q = threadIdx.x; q < groups; q += blockDim.x) {
+        const float4* src = reinterpret_cast<const float4*>(row) + 4 * q;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 f = src[i];
+            amax = fmaxf(amax, fmaxf(fmaxf(fabsf(f.x), fabsf(f.y)), fmaxf(fabsf(f.z), fabsf(f.w))));
+        }
+    }
+    amax = block_max(amax, red);
+    float s_u = 1.0f;
+    if (amax != 0.0f) s_u = __fdiv_rn(__fmul_rn(amax, clip), 7.0f);
+    if (threadIdx.x == 0) P.s_a[m] = (B > 1) ? __fmul_rn(s_u, P.inv_sqrt_b) : s_u;
+    for (int q = threadIdx.x; q < groups; q += blockDim.x) {
+        const float4* src = reinterpret_cast<const float4*>(row) + 4 * q;
+        uint32_t out[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 f = src[i];
+            const float e[4] = {f.x, f.y, f.z, f.w};
+            uint32_t w = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                int v = __float2int_rn(__fdiv_rn(e[j], s_u));
+                v = max(-8, min(7, v));
+                w |= (static_cast<uint32_t>(v) & 0xffu) << (8 * j);
+            }
+            out[i] = w;
+        }
+        reinterpret_cast<uint4*>(P.q_a + m * K)[q] = make_uint4(out[0], out[1], out[2], out[3]);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// grouped product
+// ------------------------------------------------------------------------------------------------
+// Walks this CTA's share of the work list chunk by chunk; producer and consumers run one each and
+// see the same sequence.
+struct GroupCursor {
+    const GroupProblemDev* problems;
+    int count, total_items, rows_per_item, per;
+    int item, p;
+    // current item
+    const unsigned char* wbase;   // first tile of the item's first row block
+    const int8_t* q_a;
+    size_t rb_bytes;              // bytes between consecutive row blocks
+    int N, K, n0, tiles_valid, words_per_row, nchunks;
+    int chunk;
+
+    __device__ __forceinline__ void init(const GroupProblemDev* pr, int cnt, int total, int rpi, int per_) {
+        problems = pr, count = cnt, total_items = total, rows_per_item = rpi, per = per_;
+        item = blockIdx.x, p = 0, chunk = 0;
+        load_item();
+    }
+    __device__ __forceinline__ bool valid() const { return item < total_items; }
+    __device__ __forceinline__ void load_item() {
+        if (item >= total_items) return;
+        while (p + 1 < count && item >= problems[p + 1].item_begin) ++p;
+        const GroupProblemDev& P = problems[p];
+        N = P.N, K = P.K;
+        words_per_row = K / per;
+        nchunks = (words_per_row + kChunkWords - 1) / kChunkWords;
+        n0 = (item - P.item_begin) * rows_per_item;
+        tiles_valid = (min(rows_per_item, N - n0) + 15) / 16;
+        const int pitch = round_up16(words_per_row);
+        rb_bytes = static_cast<size_t>(16) * pitch * 4;
+        wbase = reinterpret_cast<const unsigned char*>(P.packed) + static_cast<size_t>(n0) * pitch * 4;
+        q_a = P.q_a;
+    }
+    __device__ __forceinline__ int chunk_words() const { return min(kChunkWords, words_per_row - chunk * kChunkWords); }
+    __device__ __forceinline__ bool last_chunk() const { return chunk + 1 == nchunks; }
+    __device__ __forceinline__ void next() {
+        if (++chunk == nchunks) {
+            chunk = 0;
+            item += gridDim.x;
+            load_item();
+        }
+    }
+};
+
+__host__ __device__ inline size_t grouped_smem_bytes(int lv, int rt, int nt, int M, int stages) {
+    return stages * decode_stage_bytes(lv, rt, M) + static_cast<size_t>(kDecWarps) * rt * nt * 128 * 4 + 2 * stages * 8 +
+           32 * 4 + 16;
+}
+
+struct GroupParams {
+    const GroupProblemDev* problems;
+    int count, total_items, M, y_bf16, stages;
+};
+
+template <int LV, int NT, int RT>
+__global__ void __launch_bounds__(kDecThreads)
+linear_grouped_kernel(const GroupParams gp) {
+    using T = DecodeTraits<LV>;
+    constexpr int ROWS = 16 * RT;
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int M = gp.M;
+    const size_t stage_bytes = decode_stage_bytes(LV, RT, M);
+    const int stages = gp.stages;
+    unsigned char* ring = smem;
+    int* red = reinterpret_cast<int*>(smem + stages * stage_bytes);
+    uint64_t* full = reinterpret_cast<uint64_t*>(red + kDecWarps * RT * NT * 128);
+    uint64_t* empty = full + stages;
+    int* sumq_all = reinterpret_cast<int*>(empty + stages);  // two buffers of 16, alternating per item
+    volatile int* fail = sumq_all + 32;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    pdl_launch_dependents();
+    if (tid == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], kDecWarps);
+        }
+        mbar_fence_init();
+    }
+    if (tid < 32) sumq_all[tid] = 0;
+    if (tid == 32) *fail = 0;
+    __syncthreads();
+
+    if (warp == kDecWarps) {
+        // ---------------------------------------------------------------- producer warp
+        auto expect = [&](const GroupCursor& c, int s) {
+            if (lane == 0) mbar_expect_tx(&full[s], c.chunk_words() * (64 * c.tiles_valid + T::PER * M));
+            __syncwarp();
+        };
+        auto issue_w = [&](const GroupCursor& c, int s) {  // one bulk copy per 16-row tile
+            const uint32_t bytes = c.chunk_words() * 16 * 4;
+            unsigned char* dst = ring + s * stage_bytes;
+            if (lane < c.tiles_valid)
+                bulk_g2s(dst + lane * kTileBytes, c.wbase + lane * c.rb_bytes + static_cast<size_t>(c.chunk) * kTileBytes, bytes,
+                         &full[s]);
+        };
+        auto issue_q = [&](const GroupCursor& c, int s) {
+            const uint32_t seg = c.chunk_words() * T::PER;
+            unsigned char* dst = ring + s * stage_bytes + RT * kTileBytes;
+            for (int m = lane; m < M; m += 32)
+                bulk_g2s(dst + m * T::QSTRIDE, c.q_a + static_cast<size_t>(m) * c.K + static_cast<size_t>(c.chunk) * T::QBYTES, seg,
+                         &full[s]);
+        };
+        // the packed weights never depend on the previous kernel: fill the ring with them first
+        GroupCursor a;
+        a.init(gp.problems, gp.count, gp.total_items, ROWS, T::PER);
+        int pre = 0;
+        for (; pre < stages && a.valid(); ++pre, a.next()) {
+            expect(a, pre);
+            issue_w(a, pre);
+        }
+        pdl_wait();
+        GroupCursor b;
+        b.init(gp.problems, gp.count, gp.total_items, ROWS, T::PER);
+        for (int i = 0; i < pre; ++i, b.next()) issue_q(b, i);
+        for (uint32_t it = pre; b.valid(); ++it, b.next()) {
+            const int s = it % stages;
+            if (!mbar_wait(&empty[s], ((it / stages) - 1) & 1, 3)) break;
+            expect(b, s);
+            issue_w(b, s);
+            issue_q(b, s);
+        }
+        return;
+    }
+
+    // -------------------------------------------------------------------- consumer warps
+    pdl_wait();
+    const int g = lane >> 2, cq = lane & 3;
+    GroupCursor cur;
+    cur.init(gp.problems, gp.count, gp.total_items, ROWS, T::PER);
+    bool ok = true;
+    uint32_t it = 0, item_no = 0;
+    constexpr int SH = (LV == QIFT_LEVELS_INT4) ? 4 : 2;
+
+    for (; cur.valid() && ok; ++item_no) {
+        int* sumq = sumq_all + 16 * (item_no & 1);
+        int acc[RT][NT][T::NPL][4];
+#pragma unroll
+        for (int a = 0; a < RT; ++a)
+#pragma unroll
+            for (int b = 0; b < NT; ++b)
+#pragma unroll
+                for (int t = 0; t < T::NPL; ++t)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[a][b][t][i] = 0;
+        int sq[8 * NT];
+#pragma unroll
+        for (int i = 0; i < 8 * NT; ++i) sq[i] = 0;
+        const int p_item = cur.p, n0 = cur.n0, N = cur.N;
+
+        for (;;) {
+            const int s = it % stages;
+            if (!mbar_wait(&full[s], (it / stages) & 1, 4)) {
+                ok = false;
+                break;
+            }
+            const int cw = cur.chunk_words();
+            unsigned char* wst = ring + s * stage_bytes;
+            unsigned char* qst = wst + RT * kTileBytes;
+            {
+                const int off = tid * T::BPT;
+                if (off < cw * T::PER) {
+#pragma unroll
+                    for (int m = 0; m < 8 * NT; ++m) {
+                        if (m < M) {
+                            uint32_t* qp = reinterpret_cast<uint32_t*>(qst + m * T::QSTRIDE + off);
+#pragma unroll
+                            for (int i = 0; i < T::BPT / 4; ++i) {
+                                const uint32_t v = qp[i];
+                                sq[m] = dp4a_us(0x01010101u, v, sq[m]);
+                                if constexpr (LV == QIFT_LEVELS_POT) {
+                                    qp[i] = scale_s8x4(v, 5);
+                                    reinterpret_cast<uint32_t*>(qst + (M + m) * T::QSTRIDE + off)[i] = scale_s8x4(v, 6);
+                                }
+                            }
+                        }
+                    }
+                }
+                if constexpr (LV == QIFT_LEVELS_POT) consumer_bar_sync();
+            }
+            if (16 * warp < cw) {
+                uint32_t qb[NT][T::NQP][4 * T::NPL];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int m = nt * 8 + g;
+#pragma unroll
+                    for (int pl = 0; pl < T::NQP; ++pl) {
+                        if (m < M) {
+                            const uint4* src = reinterpret_cast<const uint4*>(qst + (pl * M + m) * T::QSTRIDE +
+                                                                              (16 * warp + 4 * cq) * T::PER);
+#pragma unroll
+                            for (int i = 0; i < T::NPL; ++i) {
+                                const uint4 v = src[i];
+                                qb[nt][pl][4 * i] = v.x, qb[nt][pl][4 * i + 1] = v.y;
+                                qb[nt][pl][4 * i + 2] = v.z, qb[nt][pl][4 * i + 3] = v.w;
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 4 * T::NPL; ++i) qb[nt][pl][i] = 0;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int rt = 0; rt < RT; ++rt) {
+                    const uint4 wa = *reinterpret_cast<const uint4*>(wst + rt * kTileBytes + ((2 * warp) * 32 + lane) * 16);
+                    const uint4 wb = *reinterpret_cast<const uint4*>(wst + rt * kTileBytes + ((2 * warp + 1) * 32 + lane) * 16);
+                    const uint32_t a_lo[4] = {wa.x, wa.y, wa.z, wa.w};
+                    const uint32_t a_hi[4] = {wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+                    for (int pr = 0; pr < 2; ++pr) {
+                        const int i0 = 2 * pr, i1 = 2 * pr + 1;
+#pragma unroll
+                        for (int t = 0; t < T::NPL; ++t) {
+                            if constexpr (LV == QIFT_LEVELS_INT4) {
+                                const uint32_t msk = 0x0f0f0f0fu << (4 * t), flip = 0x08080808u << (4 * t);
+#pragma unroll
+                                for (int nt = 0; nt < NT; ++nt)
+                                    mma_u8s8(acc[rt][nt][t], (a_lo[i0] & msk) ^ flip, (a_hi[i0] & msk) ^ flip,
+                                             (a_lo[i1] & msk) ^ flip, (a_hi[i1] & msk) ^ flip,
+                                             qb[nt][0][i0 * T::NPL + t], qb[nt][0][i1 * T::NPL + t]);
+                            } else if constexpr (LV == QIFT_LEVELS_POT) {
+                                const uint32_t m1 = 0x02020202u << (2 * t), m0 = 0x01010101u << (2 * t);
+#pragma unroll
+                                for (int nt = 0; nt < NT; ++nt) {
+                                    mma_u8s8(acc[rt][nt][t], a_lo[i0] & m1, a_hi[i0] & m1, a_lo[i1] & m1, a_hi[i1] & m1,
+                                             qb[nt][0][i0 * T::NPL + t], qb[nt][0][i1 * T::NPL + t]);
+                                    mma_u8s8(acc[rt][nt][t], a_lo[i0] & m0, a_hi[i0] & m0, a_lo[i1] & m0, a_hi[i1] & m0,
+                                             qb[nt][1][i0 * T::NPL + t], qb[nt][1][i1 * T::NPL + t]);
+                                }
+                            } else {
+                                const uint32_t msk = 0x03030303u << (2 * t);
+#pragma unroll
+                                for (int nt = 0; nt < NT; ++nt)
+                                    mma_u8s8(acc[rt][nt][t], a_lo[i0] & msk, a_hi[i0] & msk, a_lo[i1] & msk, a_hi[i1] & msk,
+                                             qb[nt][0][i0 * T::NPL + t], qb[nt][0][i1 * T::NPL + t]);
+                            }
+                        }
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[s]);
+            ++it;
+            const bool last = cur.last_chunk();
+            cur.next();
+            if (last) break;
+        }
+        if (!ok) break;
+
+        // item epilogue
+#pragma unroll
+        for (int rt = 0; rt < RT; ++rt)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                int* dst = red + ((warp * RT + rt) * NT + nt) * 128;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    int v = 0;
+#pragma unroll
+                    for (int t = 0; t < T::NPL; ++t) v += acc[rt][nt][t][i] >> (SH * t);
+                    dst[(g + ((i & 2) ? 8 : 0)) * 8 + 2 * cq + (i & 1)] = v;
+                }
+            }
+#pragma unroll
+        for (int m = 0; m < 8 * NT; ++m) {
+            if (m < M) {
+                int v = sq[m];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if (lane == 0) atomicAdd(&sumq[m], v);
+            }
+        }
+        consumer_bar_sync();
+        const GroupProblemDev& P = gp.problems[p_item];
+        const float* s_n = P.s_n;
+        const float* s_a = P.s_a;
+        for (int o = tid; o < ROWS * M; o += kDecConsumers) {
+            const int row = o % ROWS, m = o / ROWS;
+            const int n = n0 + row;
+            if (n >= N) continue;
+            const int rt = row / 16, r = row % 16, nt = m / 8, tk = m % 8;
+            int S = 0;
+#pragma unroll
+            for (int w = 0; w < kDecWarps; ++w) S += red[((w * RT + rt) * NT + nt) * 128 + r * 8 + tk];
+            const int Sq = sumq[m];
+            int acc_v;
+            if constexpr (LV == QIFT_LEVELS_MNZ) acc_v = 2 * S - 3 * Sq;
+            else if constexpr (LV == QIFT_LEVELS_SYM) acc_v = S - 2 * Sq;
+            else if constexpr (LV == QIFT_LEVELS_POT) acc_v = (S >> 1) - 4 * Sq;
+            else acc_v = S - 8 * Sq;
+            const size_t idx = static_cast<size_t>(m) * N + n;
+            if (P.acc_debug) P.acc_debug[idx] = acc_v;
+            const float y = scale_epilogue(acc_v, s_a[m], s_n[n]);
+            if (gp.y_bf16) static_cast<uint16_t*>(P.Y)[idx] = f32_to_bf16_bits(y);
+            else static_cast<float*>(P.Y)[idx] = y;
+        }
+        consumer_bar_sync();
+        // this buffer is next used two items from now, after the next item's barriers
+        if (tid < 16) sumq[tid] = 0;
+    }
+    if (!ok) *fail = 1;
+}
+
+}  // namespace qift

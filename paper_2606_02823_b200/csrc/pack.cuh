@@ -19,7 +19,7 @@ __device__ __forceinline__ int nearest_code(float w, float s) {
 
 template <int LV>
 __global__ void __launch_bounds__(kPackThreads)
-pack_weights_kernel(const float* __restrict__ W, int K, int mode, float* __restrict__ s_n,
+pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* __restrict__ s_n,
                     uint32_t* __restrict__ packed) {
     extern __shared__ __align__(16) float row[];
     __shared__ float red[kPackThreads / 32];
@@ -29,6 +29,12 @@ pack_weights_kernel(const float* __restrict__ W, int K, int mode, float* __restr
     pdl_wait();
     const size_t n = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int pitch = packed_pitch(K, LV);
+    if (n >= static_cast<size_t>(N)) {  // padding row of the last row block: zero words
+        for (int u = tid; u < pitch / 4; u += blockDim.x)
+            *reinterpret_cast<uint4*>(packed + packed_word_address(static_cast<int>(n), 4 * u, pitch)) = make_uint4(0, 0, 0, 0);
+        return;
+    }
 
     float amax = 0.0f;
     for (int i = tid; i < K / 4; i += blockDim.x) {
@@ -102,14 +108,23 @@ pack_weights_kernel(const float* __restrict__ W, int K, int mode, float* __restr
     constexpr int PER = codes_per_word(LV);
     constexpr int BITS = 32 / PER;
     const int words = K / PER;
-    for (int j = tid; j < words; j += blockDim.x) {
-        uint32_t w = 0;
+    for (int u = tid; u < pitch / 4; u += blockDim.x) {  // one 16-byte group of four words per thread
+        uint32_t out[4];
 #pragma unroll
-        for (int r = 0; r < PER; ++r) {
-            const int t = r / 4, b = r % 4;
-            w |= static_cast<uint32_t>(nearest_code<LV>(row[j * PER + r], s)) << (8 * b + BITS * t);
+        for (int e = 0; e < 4; ++e) {
+            const int j = 4 * u + e;
+            uint32_t w = 0;
+            if (j < words) {
+#pragma unroll
+                for (int r = 0; r < PER; ++r) {
+                    const int t = r / 4, b = r % 4;
+                    w |= static_cast<uint32_t>(nearest_code<LV>(row[j * PER + r], s)) << (8 * b + BITS * t);
+                }
+            }
+            out[e] = w;
         }
-        packed[n * words + j] = w;
+        *reinterpret_cast<uint4*>(packed + packed_word_address(static_cast<int>(n), 4 * u, pitch)) =
+            make_uint4(out[0], out[1], out[2], out[3]);
     }
 }
 
@@ -123,7 +138,8 @@ __global__ void unpack_codes_kernel(const uint32_t* __restrict__ packed, long lo
         const long long n = i / K;
         const int k = static_cast<int>(i % K);
         const int j = k / per, r = k % per, t = r / 4, b = r % 4;
-        codes[i] = static_cast<uint8_t>((packed[n * (K / per) + j] >> (8 * b + bits * t)) & ((1u << bits) - 1u));
+        const uint32_t w = packed[packed_word_address(static_cast<int>(n), j, round_up16(K / per))];
+        codes[i] = static_cast<uint8_t>((w >> (8 * b + bits * t)) & ((1u << bits) - 1u));
     }
 }
 

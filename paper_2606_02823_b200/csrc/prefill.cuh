@@ -25,13 +25,15 @@ namespace qift {
 // ------------------------------------------------------------------------------------------------
 template <int LV>
 __global__ void __launch_bounds__(256)
-expand_levels_kernel(const uint32_t* __restrict__ packed, long long total_words, int8_t* __restrict__ out) {
+expand_levels_kernel(const uint32_t* __restrict__ packed, long long total_words, int words_per_row,
+                     int8_t* __restrict__ out) {
     constexpr int PER = codes_per_word(LV);
     pdl_launch_dependents();
     pdl_wait();
+    const int pitch = round_up16(words_per_row);
     for (long long j = blockIdx.x * (long long)blockDim.x + threadIdx.x; j < total_words;
          j += (long long)gridDim.x * blockDim.x) {
-        const uint32_t w = packed[j];
+        const uint32_t w = packed[packed_word_address(static_cast<int>(j / words_per_row), static_cast<int>(j % words_per_row), pitch)];
         uint32_t o[PER / 4];
 #pragma unroll
         for (int t = 0; t < PER / 4; ++t) {

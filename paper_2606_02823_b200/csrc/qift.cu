@@ -6,6 +6,7 @@
 
 #include "common.cuh"
 #include "decode.cuh"
+#include "grouped.cuh"
 #include "pack.cuh"
 #include "prefill.cuh"
 #include "rotate_quant.cuh"
@@ -169,7 +170,8 @@ int launch_expand(const uint32_t* packed, int N, int K, int8_t* out, cudaStream_
     const long long words = static_cast<long long>(N) * (K / codes_per_word(LV));
     long long blocks = (words + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    return cuda_status(launch_pdl(expand_levels_kernel<LV>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, st, packed, words, out));
+    return cuda_status(launch_pdl(expand_levels_kernel<LV>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, st, packed, words,
+                                  K / codes_per_word(LV), out));
 }
 
 int run_prefill(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
@@ -252,7 +254,7 @@ const char* qift_status_string(int status) {
 
 size_t qift_packed_bytes(int N, int K, int levels) {
     if (N <= 0 || K <= 0 || !valid_levels(levels) || K % codes_per_word(levels) != 0) return 0;
-    return static_cast<size_t>(N) * (K / codes_per_word(levels)) * 4;
+    return static_cast<size_t>(round_up16(N)) * packed_pitch(K, levels) * 4;
 }
 
 size_t qift_workspace_bytes(int M, int N, int K, int levels) {
@@ -273,8 +275,8 @@ int qift_pack_weights(const float* W, int N, int K, int levels, int scale_mode, 
     case LV: {                                                                                               \
         cudaError_t e = allow_smem(pack_weights_kernel<LV>, smem);                                           \
         if (e != cudaSuccess) return cuda_status(e);                                                         \
-        return cuda_status(launch_pdl(pack_weights_kernel<LV>, dim3(N), dim3(kPackThreads), smem, st, W, K,  \
-                                      scale_mode, s_n, packed));                                             \
+        return cuda_status(launch_pdl(pack_weights_kernel<LV>, dim3(round_up16(N)), dim3(kPackThreads), smem, st, W, \
+                                      N, K, scale_mode, s_n, packed));                                       \
     }
     switch (levels) {
         QIFT_PACK_CASE(QIFT_LEVELS_MNZ)
@@ -425,6 +427,122 @@ int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_blo
                       void* stream) {
     return forward_impl(X_host, true, x_dtype, M, K, had_block, clip_ratio, packed, s_n, levels, N, Y_host, y_dtype, scratch,
                         scratch_bytes, stream);
+}
+
+// ------------------------------------------------------------------------------------------- grouped
+size_t qift_group_plan_bytes(int count) {
+    if (count <= 0) return 0;
+    return sizeof(GroupHeader) + static_cast<size_t>(count) * sizeof(GroupProblemDev);
+}
+
+int qift_group_plan(const qift_group_problem* problems, int count, int M, int levels, int x_dtype, int y_dtype, float clip_ratio,
+                    void* plan_host, void* plan_dev, size_t plan_bytes, void* stream) {
+    if (!problems || !plan_host || !plan_dev || count <= 0 || M <= 0 || !valid_levels(levels)) return QIFT_ERR_INVALID_ARG;
+    if ((x_dtype != QIFT_F32 && x_dtype != QIFT_BF16) || (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16))
+        return QIFT_ERR_INVALID_ARG;
+    if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return QIFT_ERR_INVALID_ARG;
+    if (M > 16) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (plan_bytes < qift_group_plan_bytes(count)) return QIFT_ERR_WORKSPACE;
+    if (!aligned16(plan_dev) || !aligned16(plan_host)) return QIFT_ERR_ALIGNMENT;
+    const int rows_per_item = (M > 8) ? 16 : 32;
+    GroupHeader* h = static_cast<GroupHeader*>(plan_host);
+    GroupProblemDev* d = reinterpret_cast<GroupProblemDev*>(h + 1);
+    int items = 0, max_k = 0;
+    for (int i = 0; i < count; ++i) {
+        const qift_group_problem& q = problems[i];
+        if (!q.X || !q.packed || !q.s_n || !q.q_a || !q.s_a || !q.Y || q.N <= 0 || q.K <= 0) return QIFT_ERR_INVALID_ARG;
+        if (!decode_supports(levels, M, q.N, q.K)) return QIFT_ERR_UNSUPPORTED_SHAPE;
+        const int rs = check_rotation_shape(q.K, q.had_block, true);
+        if (rs != QIFT_OK) return rs;
+        if (!aligned16(q.X) || !aligned16(q.packed) || !aligned16(q.s_n) || !aligned16(q.q_a) || !aligned16(q.s_a) ||
+            !aligned16(q.Y) || (q.acc_debug && !aligned16(q.acc_debug)))
+            return QIFT_ERR_ALIGNMENT;
+        GroupProblemDev& o = d[i];
+        o.X = q.X, o.packed = q.packed, o.s_n = q.s_n, o.q_a = q.q_a, o.s_a = q.s_a, o.Y = q.Y, o.acc_debug = q.acc_debug;
+        o.N = q.N, o.K = q.K, o.had_block = q.had_block;
+        o.item_begin = items;
+        o.inv_sqrt_b = q.had_block > 1 ? inv_sqrt_block(q.had_block) : 1.0f;
+        for (int j = 0; j < 5; ++j) o.pad[j] = 0;
+        items += (q.N + rows_per_item - 1) / rows_per_item;
+        if (q.K > max_k) max_k = q.K;
+    }
+    *h = GroupHeader{};
+    h->magic = kGroupMagic, h->count = count, h->M = M, h->levels = levels, h->y_bf16 = (y_dtype == QIFT_BF16);
+    h->x_bf16 = (x_dtype == QIFT_BF16), h->clip = clip_ratio, h->total_items = items, h->rows_per_item = rows_per_item;
+    h->max_k = max_k;
+    return cuda_status(cudaMemcpyAsync(plan_dev, plan_host, qift_group_plan_bytes(count), cudaMemcpyHostToDevice,
+                                       static_cast<cudaStream_t>(stream)));
+}
+
+}  // extern "C"
+
+namespace {
+const GroupHeader* plan_header(const void* plan_host, const void* plan_dev) {
+    if (!plan_host || !plan_dev) return nullptr;
+    const GroupHeader* h = static_cast<const GroupHeader*>(plan_host);
+    return h->magic == kGroupMagic ? h : nullptr;
+}
+
+template <int LV, int NT, int RT>
+int launch_grouped(const GroupHeader* h, const GroupProblemDev* dev, cudaStream_t st) {
+    const size_t stage = decode_stage_bytes(LV, RT, h->M);
+    const size_t fixed = grouped_smem_bytes(LV, RT, NT, h->M, 0);
+    int stages = static_cast<int>((110 * 1024 - fixed) / (stage + 16));
+    if (stages < 2) stages = 2;
+    if (stages > 12) stages = 12;
+    const size_t smem = grouped_smem_bytes(LV, RT, NT, h->M, stages);
+    auto kernel = linear_grouped_kernel<LV, NT, RT>;
+    cudaError_t e = allow_smem(kernel, smem);
+    if (e != cudaSuccess) return cuda_status(e);
+    int grid = 2 * sm_count();
+    if (grid > h->total_items) grid = h->total_items;
+    GroupParams gp{dev, h->count, h->total_items, h->M, h->y_bf16, stages};
+    return cuda_status(launch_pdl(kernel, dim3(grid), dim3(kDecThreads), smem, st, gp));
+}
+
+template <int LV>
+int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* dev, cudaStream_t st) {
+    if (h->M > 8) return launch_grouped<LV, 2, 1>(h, dev, st);
+    return launch_grouped<LV, 1, 2>(h, dev, st);
+}
+}  // namespace
+
+extern "C" {
+
+int qift_group_quantize_act(const void* plan_host, const void* plan_dev, void* stream) {
+    const GroupHeader* h = plan_header(plan_host, plan_dev);
+    if (!h) return QIFT_ERR_INVALID_ARG;
+    const GroupProblemDev* dev = reinterpret_cast<const GroupProblemDev*>(static_cast<const GroupHeader*>(plan_dev) + 1);
+    const size_t smem = static_cast<size_t>(h->max_k) * 4;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const dim3 grid(static_cast<unsigned>(h->count) * h->M);
+    if (h->x_bf16) {
+        cudaError_t e = allow_smem(quantize_act_grouped_kernel<true>, smem);
+        if (e != cudaSuccess) return cuda_status(e);
+        return cuda_status(launch_pdl(quantize_act_grouped_kernel<true>, grid, dim3(kRowThreads), smem, st, dev, h->M, h->clip));
+    }
+    cudaError_t e = allow_smem(quantize_act_grouped_kernel<false>, smem);
+    if (e != cudaSuccess) return cuda_status(e);
+    return cuda_status(launch_pdl(quantize_act_grouped_kernel<false>, grid, dim3(kRowThreads), smem, st, dev, h->M, h->clip));
+}
+
+int qift_group_linear(const void* plan_host, const void* plan_dev, void* stream) {
+    const GroupHeader* h = plan_header(plan_host, plan_dev);
+    if (!h) return QIFT_ERR_INVALID_ARG;
+    const GroupProblemDev* dev = reinterpret_cast<const GroupProblemDev*>(static_cast<const GroupHeader*>(plan_dev) + 1);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    switch (h->levels) {
+        case QIFT_LEVELS_MNZ: return dispatch_grouped<QIFT_LEVELS_MNZ>(h, dev, st);
+        case QIFT_LEVELS_POT: return dispatch_grouped<QIFT_LEVELS_POT>(h, dev, st);
+        case QIFT_LEVELS_SYM: return dispatch_grouped<QIFT_LEVELS_SYM>(h, dev, st);
+        default: return dispatch_grouped<QIFT_LEVELS_INT4>(h, dev, st);
+    }
+}
+
+int qift_group_forward(const void* plan_host, const void* plan_dev, void* stream) {
+    const int rc = qift_group_quantize_act(plan_host, plan_dev, stream);
+    if (rc != QIFT_OK) return rc;
+    return qift_group_linear(plan_host, plan_dev, stream);
 }
 
 int qift_device_status(void* stream, uint32_t* detail) {

@@ -251,31 +251,70 @@ def test_lloyd_max_levels_are_a_fixed_point():
 
 
 # ----------------------------------------------------------------------------- packing (P8)
+def tiled_address(n, j, words):
+    """The storage order, written out independently of the oracle: 16-row x 128-word tiles, row
+    blocks outermost; inside a tile 16-byte groups ordered (slice, half, row % 8, quad)."""
+    pitch = -(-words // 16) * 16
+    rb, r = divmod(n, 16)
+    half, g = divmod(r, 8)
+    c, jj = divmod(j, 128)
+    sl, rem = divmod(jj, 16)
+    quad, e = divmod(rem, 4)
+    return rb * 16 * pitch + c * 2048 + (((sl * 2 + half) * 32 + g * 4 + quad) * 4 + e)
+
+
 @pytest.mark.parametrize("lv", [oracle.MNZ, oracle.POT, oracle.SYM, oracle.INT4])
-def test_pack_layout_and_roundtrip(lv):
+@pytest.mark.parametrize("N,words", [(5, 8), (16, 16), (37, 144), (33, 688)])
+def test_pack_layout_and_roundtrip(lv, N, words):
     per, bits = (8, 4) if lv == oracle.INT4 else (16, 2)
-    N, K = 5, 8 * per
+    K = words * per
     rng = np.random.default_rng(3)
     pats = [rng.integers(0, 1 << bits, (N, K)), np.zeros((N, K)), np.full((N, K), (1 << bits) - 1),
             np.tile(np.arange(K) % (1 << bits), (N, 1))]
+    n_pad, pitch = -(-N // 16) * 16, -(-words // 16) * 16
+    # the address map is a bijection from (row, word) onto distinct slots of the padded buffer
+    addr = np.array([[tiled_address(n, j, words) for j in range(words)] for n in range(N)])
+    assert len(np.unique(addr)) == N * words and addr.max() < n_pad * pitch
+    if words % 16 == 0 and N % 16 == 0:
+        assert addr.max() == n_pad * pitch - 1
     for codes in pats:
         codes = codes.astype(np.uint8)
         p = oracle.pack(codes, lv)
-        assert p.shape == (N, K // per) and p.dtype == np.uint32 and p.nbytes == N * K * bits // 8
-        assert np.array_equal(oracle.unpack(p, K, lv), codes)
-        # the layout formula, written out independently: k = per*j + 4t + b -> bit 8b + bits*t
-        ref = np.zeros((N, K // per), dtype=np.uint64)
+        assert p.shape == (n_pad * pitch,) and p.dtype == np.uint32
+        assert oracle.packed_words(N, K, lv) == n_pad * pitch
+        assert np.array_equal(oracle.unpack(p, N, K, lv), codes)
+        # bits inside a word: k = per*j + 4t + b -> bit 8b + bits*t
+        ref = np.zeros((N, words), dtype=np.uint64)
         for k in range(K):
             j, r = divmod(k, per)
             t, b = divmod(r, 4)
             ref[:, j] |= codes[:, k].astype(np.uint64) << np.uint64(8 * b + bits * t)
-        assert np.array_equal(p, ref.astype(np.uint32))
+        assert np.array_equal(p[addr], ref.astype(np.uint32))
+        # padding slots are zero
+        mask = np.ones(p.shape, dtype=bool)
+        mask[addr.ravel()] = False
+        assert not p[mask].any()
         # byte-lane property: (word >> bits*t) & mask gives four consecutive-k codes
-        mask = 0x03030303 if bits == 2 else 0x0F0F0F0F
+        w = p[addr]
+        m = 0x03030303 if bits == 2 else 0x0F0F0F0F
         for t in range(per // 4):
-            lanes = ((p >> np.uint32(bits * t)) & np.uint32(mask)).view(np.uint8).reshape(N, K // per, 4)
-            want = codes.reshape(N, K // per, per // 4, 4)[:, :, t, :]
+            lanes = ((w >> np.uint32(bits * t)) & np.uint32(m)).view(np.uint8).reshape(N, words, 4)
+            want = codes.reshape(N, words, per // 4, 4)[:, :, t, :]
             assert np.array_equal(lanes, want)
+    # a 16-byte group holds four consecutive words of one row; a warp's 32 groups are contiguous
+    if words >= 16 and N >= 16:
+        base = tiled_address(0, 0, words)
+        for g in range(8):
+            for quad in range(4):
+                assert tiled_address(g, 4 * quad, words) == base + (g * 4 + quad) * 4
+        assert tiled_address(8, 0, words) == base + 128          # rows 8..15: the next 512 bytes
+
+
+def test_packed_bytes_of_llama_shapes():
+    # no padding on the paper's shapes: exactly 2 (or 4) bits per weight
+    for _, N, K in synth.LLAMA2_7B + synth.LLAMA31_8B:
+        assert oracle.packed_words(N, K, oracle.MNZ) * 4 == N * K // 4
+        assert oracle.packed_words(N, K, oracle.INT4) * 4 == N * K // 2
 
 
 def test_mixed_stack_is_three_bits_per_weight():
@@ -351,7 +390,7 @@ def test_whole_layer_on_config1_matches_the_dequantized_definition():
     x, _ = synth.activations(1, 1, 256, 4)
     packed, s_n, codes = oracle.pack_weights(W, oracle.MNZ, oracle.SCALE_MSE)
     q_a, s_a = oracle.quantize_act(x, 256, 0.9)
-    y, acc = oracle.linear(oracle.unpack(packed, 256, oracle.MNZ), oracle.MNZ, s_n, q_a, s_a)
+    y, acc = oracle.linear(oracle.unpack(packed, 256, 256, oracle.MNZ), oracle.MNZ, s_n, q_a, s_a)
     table = np.array(paper_levels()["MNZ_INT"])
     w_hat = table[codes] * s_n[:, None].astype(np.float64)
     a_hat = q_a.astype(np.float64) * s_a[:, None].astype(np.float64)

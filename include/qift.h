@@ -32,7 +32,8 @@ typedef enum {
     QIFT_ERR_ALIGNMENT = 3,         /* a base pointer is not 16-byte aligned                        */
     QIFT_ERR_WORKSPACE = 4,         /* workspace missing or smaller than qift_workspace_bytes()     */
     QIFT_ERR_CUDA = 5,              /* a CUDA runtime call or a launch failed                       */
-    QIFT_ERR_TIMEOUT = 6            /* a bounded device-side wait expired (see qift_device_status)  */
+    QIFT_ERR_TIMEOUT = 6,           /* a bounded device-side wait expired (see qift_device_status)  */
+    QIFT_ERR_TOO_LARGE = 7          /* N*K exceeds the built-in scratch of qift_w2a4_linear_static  */
 } qift_status;
 
 /* Reconstruction level sets.  Two-bit codes index the levels in ascending order (code 0 = most
@@ -184,6 +185,33 @@ int qift_group_plan(const qift_group_problem* problems /*host*/, int count, int 
 int qift_group_quantize_act(const void* plan_host, const void* plan_dev, void* stream);
 int qift_group_linear(const void* plan_host, const void* plan_dev, void* stream);
 int qift_group_forward(const void* plan_host, const void* plan_dev, void* stream);
+
+/* ---- Product without any allocation by anyone ------------------------------------------------
+ * (No counterpart in the paper: this is a packaging variant of qift_w2a4_linear's prefill route.)
+ *
+ * Some callers cannot allocate device memory at the moment they need the layer: code running inside
+ * a region where cudaMalloc is forbidden or would synchronize the device (a latency-critical serving
+ * loop, a plugin whose host hands it fixed buffers and no allocator, a stream that is being
+ * captured), or a process whose memory pool is owned by another framework and already fully
+ * committed.  The prefill route needs N*K bytes of scratch for the decoded int8 levels; this entry
+ * point takes that scratch from an array that is compiled into the library instead of from the
+ * caller.  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ *   qift_static_scratch_bytes()   capacity of the built-in array (16 MiB): problems need N*K <= it.
+ *   qift_w2a4_linear_static(...)  same arguments and results as qift_w2a4_linear (any M >= 1, the
+ *                                 two-bit level sets), minus the workspace; always takes the
+ *                                 prefill route.  QIFT_ERR_TOO_LARGE when N*K exceeds the capacity.
+ *
+ * The array lives in every GPU context that loads the library, until the process exits.  The first
+ * call on each device looks up the array's device address (one cudaGetSymbolAddress, with that device
+ * current); make that first call before starting any stream capture.  All calls on a device share
+ * the one array and it keeps the previous call's bytes: every byte the product reads is rewritten by
+ * the call itself, so nothing needs clearing, but two calls that can overlap on the GPU (different
+ * streams without an ordering between them) race on it -- serialize them. */
+size_t qift_static_scratch_bytes(void);
+int qift_w2a4_linear_static(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a,
+                            const float* s_a, int M, int N, int K, void* Y, int y_dtype,
+                            int32_t* acc_debug, void* stream);
 
 /* Synchronizes `stream`, then reads and clears the device status word in which a kernel records an
  * expired bounded wait.  QIFT_OK, QIFT_ERR_TIMEOUT or QIFT_ERR_CUDA.  `detail` (host, may be NULL)

@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libqift.so")
 
 # enums of qift.h
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = range(8)
 MNZ, POT, SYM, INT4 = 0, 1, 2, 3
 SCALE_GIVEN, SCALE_ABSMAX, SCALE_MSE = 0, 1, 2
 F32, BF16 = 0, 1
@@ -26,6 +26,7 @@ EXPORTS = [
     "qift_unpack_codes", "qift_rotate", "qift_quantize_act", "qift_w2a4_linear", "qift_w4a4_linear",
     "qift_linear_route", "qift_device_status", "qift_forward_scratch_bytes", "qift_forward", "qift_forward_host",
     "qift_group_plan_bytes", "qift_group_plan", "qift_group_quantize_act", "qift_group_linear", "qift_group_forward",
+    "qift_static_scratch_bytes", "qift_w2a4_linear_static",
 ]
 
 _lib = None
@@ -71,9 +72,12 @@ def lib() -> ctypes.CDLL:
         L.qift_group_plan.argtypes = [vp, ci, ci, ci, ci, ci, cf, vp, vp, sz, vp]
         for name in ("qift_group_quantize_act", "qift_group_linear", "qift_group_forward"):
             getattr(L, name).argtypes = [vp, vp, vp]
+        L.qift_static_scratch_bytes.restype = sz
+        L.qift_static_scratch_bytes.argtypes = []
+        L.qift_w2a4_linear_static.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, vp, ci, vp, vp]
         for name in EXPORTS:
             if name not in ("qift_status_string", "qift_packed_bytes", "qift_workspace_bytes",
-                            "qift_forward_scratch_bytes", "qift_group_plan_bytes"):
+                            "qift_forward_scratch_bytes", "qift_group_plan_bytes", "qift_static_scratch_bytes"):
                 getattr(L, name).restype = ci
         _lib = L
     return _lib
@@ -302,3 +306,22 @@ def qift_group_linear(plan: GroupPlan):
 def qift_group_forward(plan: GroupPlan):
     _check(lib().qift_group_forward(plan.host.data_ptr(), plan.dev.data_ptr(), _stream()), "qift_group_forward")
     return plan.outputs
+
+
+def qift_static_scratch_bytes() -> int:
+    return int(lib().qift_static_scratch_bytes())
+
+
+def qift_w2a4_linear_static(packed, s_n, levels, q_a, s_a, out, acc=None):
+    """The W2A4 product for callers that cannot allocate: the int8 scratch of the prefill route comes
+    from an array built into the library, and the caller passes every output buffer (`out` [M,N]
+    fp32 or bf16, optionally `acc` int32 [M,N]).  This wrapper allocates nothing either.  Calls that
+    may overlap on the GPU share the scratch and must be serialized; make the first call on a device
+    outside stream capture."""
+    _dev(packed), _dev(s_n, torch.float32), _dev(q_a, torch.int8), _dev(s_a, torch.float32), _dev(out)
+    M, K = q_a.shape
+    N = s_n.shape[0]
+    assert tuple(out.shape) == (M, N)
+    _check(lib().qift_w2a4_linear_static(_ptr(packed), _ptr(s_n), levels, _ptr(q_a), _ptr(s_a), M, N, K, _ptr(out),
+                                         _dt(out), _ptr(acc), _stream()), "qift_w2a4_linear_static")
+    return out

@@ -248,6 +248,7 @@ const char* qift_status_string(int status) {
         case QIFT_ERR_WORKSPACE: return "workspace missing or too small";
         case QIFT_ERR_CUDA: return "CUDA error";
         case QIFT_ERR_TIMEOUT: return "device-side wait timed out";
+        case QIFT_ERR_TOO_LARGE: return "N*K exceeds the built-in static scratch";
         default: return "unknown status";
     }
 }
@@ -543,6 +544,56 @@ int qift_group_forward(const void* plan_host, const void* plan_dev, void* stream
     const int rc = qift_group_quantize_act(plan_host, plan_dev, stream);
     if (rc != QIFT_OK) return rc;
     return qift_group_linear(plan_host, plan_dev, stream);
+}
+
+// ------------------------------------------------------------------------- allocation-free product
+}  // extern "C"
+
+namespace {
+// Scratch for the decoded int8 levels of qift_w2a4_linear_static.  In host code this name is only a
+// handle for the runtime's symbol lookup, never a device address: kernels get the address that
+// cudaGetSymbolAddress returns.
+constexpr size_t kStaticScratchBytes = size_t(16) << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};
+
+// Device address of the array on the current device; looked up once per device.
+cudaError_t static_scratch_address(void** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!g_static_scratch_addr[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_scratch_addr[dev] = ptr;
+    }
+    *out = g_static_scratch_addr[dev];
+    return cudaSuccess;
+}
+}  // namespace
+
+extern "C" {
+
+size_t qift_static_scratch_bytes(void) { return kStaticScratchBytes; }
+
+int qift_w2a4_linear_static(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a, const float* s_a, int M,
+                            int N, int K, void* Y, int y_dtype, int32_t* acc_debug, void* stream) {
+    if (levels != QIFT_LEVELS_MNZ && levels != QIFT_LEVELS_POT && levels != QIFT_LEVELS_SYM) return QIFT_ERR_INVALID_ARG;
+    if (!packed || !s_n || !q_a || !s_a || !Y || M <= 0 || N <= 0 || K <= 0) return QIFT_ERR_INVALID_ARG;
+    if (static_cast<size_t>(N) * static_cast<size_t>(K) > kStaticScratchBytes) {
+        std::fprintf(stderr, "qift_w2a4_linear_static: N*K = %zu bytes of scratch needed, the built-in array holds %zu\n",
+                     static_cast<size_t>(N) * static_cast<size_t>(K), kStaticScratchBytes);
+        return QIFT_ERR_TOO_LARGE;
+    }
+    void* scratch = nullptr;
+    const cudaError_t e = static_scratch_address(&scratch);
+    if (e != cudaSuccess) return cuda_status(e);
+    return linear_impl(packed, s_n, levels, q_a, s_a, M, N, K, Y, y_dtype, acc_debug, scratch, kStaticScratchBytes,
+                       QIFT_ROUTE_PREFILL, stream);
 }
 
 int qift_device_status(void* stream, uint32_t* detail) {

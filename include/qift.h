@@ -161,7 +161,9 @@ int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_blo
  * `stream`.  The plan holds the caller's pointers, so it stays valid while those buffers live;
  * plan_host must stay alive and unchanged while the plan is used.  The run calls enqueue
  *   qift_group_quantize_act : S2+S3 for every problem (one launch)  X -> q_a, s_a
- *   qift_group_linear       : S4+S5 for every problem (one launch)  q_a, s_a -> Y
+ *   qift_group_linear       : S4+S5 for every problem (one launch per 256 problems)  q_a, s_a -> Y;
+ *                             needs the q_a, s_a and token sums that qift_group_quantize_act left
+ *                             in the problems' buffers and in plan_dev
  *   qift_group_forward      : both.
  * Problems must not alias each other's q_a / s_a / Y.  K % 256 == 0 (two-bit sets) or K % 128 == 0
  * (INT4), K <= 16384. */

@@ -48,16 +48,18 @@ static_assert(sizeof(GroupProblemDev) == 96, "problem record is 96 bytes");
 constexpr uint32_t kGroupMagic = 0x51494654u;
 
 // ------------------------------------------------------------------------------------------------
-// grouped quantizer: one CTA per (problem, token row)
+// grouped quantizer: one CTA per (problem, token row); also leaves sum_k q_a for the product kernel
 // ------------------------------------------------------------------------------------------------
 template <bool BF16_IN>
 __global__ void __launch_bounds__(kRowThreads)
-quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int M, float clip) {
+quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* __restrict__ sumq, int M, float clip) {
     extern __shared__ __align__(16) float row[];
     __shared__ float red[kRowThreads / 32];
+    __shared__ int redi[kRowThreads / 32];
     pdl_launch_dependents();
     pdl_wait();
-    const GroupProblemDev P = problems[blockIdx.x / M];
+    const int p = blockIdx.x / M;
+    const GroupProblemDev P = problems[p];
     const size_t m = blockIdx.x % M;
     const int K = P.K, B = P.had_block;
     load_and_transform<BF16_IN>(P.X, m, K, B, row);
@@ -75,6 +77,7 @@ quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int M,
     float s_u = 1.0f;
     if (amax != 0.0f) s_u = __fdiv_rn(__fmul_rn(amax, clip), 7.0f);
     if (threadIdx.x == 0) P.s_a[m] = (B > 1) ? __fmul_rn(s_u, P.inv_sqrt_b) : s_u;
+    int total = 0;
     for (int q = threadIdx.x; q < groups; q += blockDim.x) {
         const float4* src = reinterpret_cast<const float4*>(row) + 4 * q;
         uint32_t out[4];
@@ -87,40 +90,64 @@ quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int M,
             for (int j = 0; j < 4; ++j) {
                 int v = __float2int_rn(__fdiv_rn(e[j], s_u));
                 v = max(-8, min(7, v));
+                total += v;
                 w |= (static_cast<uint32_t>(v) & 0xffu) << (8 * j);
             }
             out[i] = w;
         }
         reinterpret_cast<uint4*>(P.q_a + m * K)[q] = make_uint4(out[0], out[1], out[2], out[3]);
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    if ((threadIdx.x & 31) == 0) redi[threadIdx.x >> 5] = total;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 0;
+        for (int w = 0; w < kRowThreads / 32; ++w) t += redi[w];
+        sumq[p * 16 + m] = t;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
 // grouped product
 // ------------------------------------------------------------------------------------------------
-// Walks this CTA's share of the work list chunk by chunk; producer and consumers run one each and
-// see the same sequence.
+struct SmemProblem {  // what the product kernel needs of a problem, 64 bytes, in shared memory
+    const unsigned char* packed;
+    const int8_t* q_a;
+    const float* s_n;
+    const float* s_a;
+    void* Y;
+    int32_t* acc_debug;
+    int N, K;
+    int item_begin;
+    int index;  // position in the whole plan (row of the sum-q table)
+};
+static_assert(sizeof(SmemProblem) == 64, "shared-memory problem record is 64 bytes");
+
+constexpr int kGroupSlice = 256;  // problems per launch (their table lives in shared memory)
+
+// Walks this CTA's share of the work list chunk by chunk; the producer and the consumers each run
+// one and see the same sequence.
 struct GroupCursor {
-    const GroupProblemDev* problems;
-    int count, total_items, rows_per_item, per;
+    const SmemProblem* table;
+    int count, item_end, rows_per_item, per;
     int item, p;
-    // current item
     const unsigned char* wbase;   // first tile of the item's first row block
     const int8_t* q_a;
     size_t rb_bytes;              // bytes between consecutive row blocks
     int N, K, n0, tiles_valid, words_per_row, nchunks;
     int chunk;
 
-    __device__ __forceinline__ void init(const GroupProblemDev* pr, int cnt, int total, int rpi, int per_) {
-        problems = pr, count = cnt, total_items = total, rows_per_item = rpi, per = per_;
-        item = blockIdx.x, p = 0, chunk = 0;
+    __device__ __forceinline__ void init(const SmemProblem* t, int cnt, int item_first, int item_last, int rpi, int per_) {
+        table = t, count = cnt, item_end = item_last, rows_per_item = rpi, per = per_;
+        item = item_first + blockIdx.x, p = 0, chunk = 0;
         load_item();
     }
-    __device__ __forceinline__ bool valid() const { return item < total_items; }
+    __device__ __forceinline__ bool valid() const { return item < item_end; }
     __device__ __forceinline__ void load_item() {
-        if (item >= total_items) return;
-        while (p + 1 < count && item >= problems[p + 1].item_begin) ++p;
-        const GroupProblemDev& P = problems[p];
+        if (item >= item_end) return;
+        while (p + 1 < count && item >= table[p + 1].item_begin) ++p;
+        const SmemProblem& P = table[p];
         N = P.N, K = P.K;
         words_per_row = K / per;
         nchunks = (words_per_row + kChunkWords - 1) / kChunkWords;
@@ -128,7 +155,7 @@ struct GroupCursor {
         tiles_valid = (min(rows_per_item, N - n0) + 15) / 16;
         const int pitch = round_up16(words_per_row);
         rb_bytes = static_cast<size_t>(16) * pitch * 4;
-        wbase = reinterpret_cast<const unsigned char*>(P.packed) + static_cast<size_t>(n0) * pitch * 4;
+        wbase = P.packed + static_cast<size_t>(n0) * pitch * 4;
         q_a = P.q_a;
     }
     __device__ __forceinline__ int chunk_words() const { return min(kChunkWords, words_per_row - chunk * kChunkWords); }
@@ -142,14 +169,20 @@ struct GroupCursor {
     }
 };
 
-__host__ __device__ inline size_t grouped_smem_bytes(int lv, int rt, int nt, int M, int stages) {
-    return stages * decode_stage_bytes(lv, rt, M) + static_cast<size_t>(kDecWarps) * rt * nt * 128 * 4 + 2 * stages * 8 +
-           32 * 4 + 16;
+__host__ __device__ inline size_t grouped_fixed_smem(int rt, int nt, int count) {
+    return static_cast<size_t>(count) * sizeof(SmemProblem) + 2 * static_cast<size_t>(kDecWarps) * rt * nt * 128 * 4 + 16;
+}
+__host__ __device__ inline size_t grouped_smem_bytes(int lv, int rt, int nt, int M, int stages, int count) {
+    return grouped_fixed_smem(rt, nt, count) + stages * (decode_stage_bytes(lv, rt, M) + 16);
 }
 
 struct GroupParams {
-    const GroupProblemDev* problems;
-    int count, total_items, M, y_bf16, stages;
+    const GroupProblemDev* problems;  // first problem of this launch's slice
+    const int* sumq;                  // [plan count][16]
+    int first_index;                  // plan index of problems[0]
+    int count;                        // problems in the slice (<= kGroupSlice)
+    int item_first, item_end;         // work items of the slice
+    int M, y_bf16, stages;
 };
 
 template <int LV, int NT, int RT>
@@ -157,16 +190,17 @@ __global__ void __launch_bounds__(kDecThreads)
 linear_grouped_kernel(const GroupParams gp) {
     using T = DecodeTraits<LV>;
     constexpr int ROWS = 16 * RT;
+    constexpr int RED = kDecWarps * RT * NT * 128;  // ints per reduction buffer
     extern __shared__ __align__(128) unsigned char smem[];
     const int M = gp.M;
     const size_t stage_bytes = decode_stage_bytes(LV, RT, M);
     const int stages = gp.stages;
     unsigned char* ring = smem;
-    int* red = reinterpret_cast<int*>(smem + stages * stage_bytes);
-    uint64_t* full = reinterpret_cast<uint64_t*>(red + kDecWarps * RT * NT * 128);
+    int* red_all = reinterpret_cast<int*>(smem + stages * stage_bytes);
+    SmemProblem* table = reinterpret_cast<SmemProblem*>(red_all + 2 * RED);
+    uint64_t* full = reinterpret_cast<uint64_t*>(table + gp.count);
     uint64_t* empty = full + stages;
-    int* sumq_all = reinterpret_cast<int*>(empty + stages);  // two buffers of 16, alternating per item
-    volatile int* fail = sumq_all + 32;
+    volatile int* fail = reinterpret_cast<volatile int*>(empty + stages);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -177,9 +211,17 @@ linear_grouped_kernel(const GroupParams gp) {
             mbar_init(&empty[s], kDecWarps);
         }
         mbar_fence_init();
+        *fail = 0;
     }
-    if (tid < 32) sumq_all[tid] = 0;
-    if (tid == 32) *fail = 0;
+    // the plan was uploaded by a copy that completed before any kernel of this stream segment began
+    for (int i = tid; i < gp.count; i += kDecThreads) {
+        const GroupProblemDev& P = gp.problems[i];
+        SmemProblem e;
+        e.packed = reinterpret_cast<const unsigned char*>(P.packed);
+        e.q_a = P.q_a, e.s_n = P.s_n, e.s_a = P.s_a, e.Y = P.Y, e.acc_debug = P.acc_debug;
+        e.N = P.N, e.K = P.K, e.item_begin = P.item_begin, e.index = gp.first_index + i;
+        table[i] = e;
+    }
     __syncthreads();
 
     if (warp == kDecWarps) {
@@ -204,7 +246,7 @@ linear_grouped_kernel(const GroupParams gp) {
         };
         // the packed weights never depend on the previous kernel: fill the ring with them first
         GroupCursor a;
-        a.init(gp.problems, gp.count, gp.total_items, ROWS, T::PER);
+        a.init(table, gp.count, gp.item_first, gp.item_end, ROWS, T::PER);
         int pre = 0;
         for (; pre < stages && a.valid(); ++pre, a.next()) {
             expect(a, pre);
@@ -212,7 +254,7 @@ linear_grouped_kernel(const GroupParams gp) {
         }
         pdl_wait();
         GroupCursor b;
-        b.init(gp.problems, gp.count, gp.total_items, ROWS, T::PER);
+        b.init(table, gp.count, gp.item_first, gp.item_end, ROWS, T::PER);
         for (int i = 0; i < pre; ++i, b.next()) issue_q(b, i);
         for (uint32_t it = pre; b.valid(); ++it, b.next()) {
             const int s = it % stages;
@@ -228,13 +270,15 @@ linear_grouped_kernel(const GroupParams gp) {
     pdl_wait();
     const int g = lane >> 2, cq = lane & 3;
     GroupCursor cur;
-    cur.init(gp.problems, gp.count, gp.total_items, ROWS, T::PER);
+    cur.init(table, gp.count, gp.item_first, gp.item_end, ROWS, T::PER);
     bool ok = true;
     uint32_t it = 0, item_no = 0;
     constexpr int SH = (LV == QIFT_LEVELS_INT4) ? 4 : 2;
+    // epilogue role of this thread: output (row, token) = (tid % ROWS, tid / ROWS); ROWS * M <= 256
+    const int e_row = tid % ROWS, e_m = tid / ROWS;
 
     for (; cur.valid() && ok; ++item_no) {
-        int* sumq = sumq_all + 16 * (item_no & 1);
+        int* red = red_all + RED * (item_no & 1);
         int acc[RT][NT][T::NPL][4];
 #pragma unroll
         for (int a = 0; a < RT; ++a)
@@ -244,10 +288,18 @@ linear_grouped_kernel(const GroupParams gp) {
                 for (int t = 0; t < T::NPL; ++t)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) acc[a][b][t][i] = 0;
-        int sq[8 * NT];
-#pragma unroll
-        for (int i = 0; i < 8 * NT; ++i) sq[i] = 0;
-        const int p_item = cur.p, n0 = cur.n0, N = cur.N;
+        const SmemProblem P = table[cur.p];
+        const int n0 = cur.n0;
+        const int e_n = n0 + e_row;
+        const bool e_on = (e_m < M) && (e_n < P.N);
+        // fetch what the epilogue needs now; the loads complete under the chunk loop
+        float e_sn = 0.0f, e_sa = 0.0f;
+        int e_sq = 0;
+        if (e_on) {
+            e_sn = __ldg(P.s_n + e_n);
+            e_sa = P.s_a[e_m];
+            e_sq = gp.sumq[P.index * 16 + e_m];
+        }
 
         for (;;) {
             const int s = it % stages;
@@ -258,7 +310,7 @@ linear_grouped_kernel(const GroupParams gp) {
             const int cw = cur.chunk_words();
             unsigned char* wst = ring + s * stage_bytes;
             unsigned char* qst = wst + RT * kTileBytes;
-            {
+            if constexpr (LV == QIFT_LEVELS_POT) {  // build the 5q and 6q planes
                 const int off = tid * T::BPT;
                 if (off < cw * T::PER) {
 #pragma unroll
@@ -268,16 +320,13 @@ linear_grouped_kernel(const GroupParams gp) {
 #pragma unroll
                             for (int i = 0; i < T::BPT / 4; ++i) {
                                 const uint32_t v = qp[i];
-                                sq[m] = dp4a_us(0x01010101u, v, sq[m]);
-                                if constexpr (LV == QIFT_LEVELS_POT) {
-                                    qp[i] = scale_s8x4(v, 5);
-                                    reinterpret_cast<uint32_t*>(qst + (M + m) * T::QSTRIDE + off)[i] = scale_s8x4(v, 6);
-                                }
+                                qp[i] = scale_s8x4(v, 5);
+                                reinterpret_cast<uint32_t*>(qst + (M + m) * T::QSTRIDE + off)[i] = scale_s8x4(v, 6);
                             }
                         }
                     }
                 }
-                if constexpr (LV == QIFT_LEVELS_POT) consumer_bar_sync();
+                consumer_bar_sync();
             }
             if (16 * warp < cw) {
                 uint32_t qb[NT][T::NQP][4 * T::NPL];
@@ -348,7 +397,7 @@ linear_grouped_kernel(const GroupParams gp) {
         }
         if (!ok) break;
 
-        // item epilogue
+        // item epilogue: one barrier; the other reduction buffer belongs to the next item
 #pragma unroll
         for (int rt = 0; rt < RT; ++rt)
 #pragma unroll
@@ -362,42 +411,23 @@ linear_grouped_kernel(const GroupParams gp) {
                     dst[(g + ((i & 2) ? 8 : 0)) * 8 + 2 * cq + (i & 1)] = v;
                 }
             }
-#pragma unroll
-        for (int m = 0; m < 8 * NT; ++m) {
-            if (m < M) {
-                int v = sq[m];
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                if (lane == 0) atomicAdd(&sumq[m], v);
-            }
-        }
         consumer_bar_sync();
-        const GroupProblemDev& P = gp.problems[p_item];
-        const float* s_n = P.s_n;
-        const float* s_a = P.s_a;
-        for (int o = tid; o < ROWS * M; o += kDecConsumers) {
-            const int row = o % ROWS, m = o / ROWS;
-            const int n = n0 + row;
-            if (n >= N) continue;
-            const int rt = row / 16, r = row % 16, nt = m / 8, tk = m % 8;
+        if (e_on) {
+            const int rt = e_row / 16, r = e_row % 16, nt = e_m / 8, tk = e_m % 8;
             int S = 0;
 #pragma unroll
             for (int w = 0; w < kDecWarps; ++w) S += red[((w * RT + rt) * NT + nt) * 128 + r * 8 + tk];
-            const int Sq = sumq[m];
             int acc_v;
-            if constexpr (LV == QIFT_LEVELS_MNZ) acc_v = 2 * S - 3 * Sq;
-            else if constexpr (LV == QIFT_LEVELS_SYM) acc_v = S - 2 * Sq;
-            else if constexpr (LV == QIFT_LEVELS_POT) acc_v = (S >> 1) - 4 * Sq;
-            else acc_v = S - 8 * Sq;
-            const size_t idx = static_cast<size_t>(m) * N + n;
+            if constexpr (LV == QIFT_LEVELS_MNZ) acc_v = 2 * S - 3 * e_sq;
+            else if constexpr (LV == QIFT_LEVELS_SYM) acc_v = S - 2 * e_sq;
+            else if constexpr (LV == QIFT_LEVELS_POT) acc_v = (S >> 1) - 4 * e_sq;
+            else acc_v = S - 8 * e_sq;
+            const size_t idx = static_cast<size_t>(e_m) * P.N + e_n;
             if (P.acc_debug) P.acc_debug[idx] = acc_v;
-            const float y = scale_epilogue(acc_v, s_a[m], s_n[n]);
+            const float y = scale_epilogue(acc_v, e_sa, e_sn);
             if (gp.y_bf16) static_cast<uint16_t*>(P.Y)[idx] = f32_to_bf16_bits(y);
             else static_cast<float*>(P.Y)[idx] = y;
         }
-        consumer_bar_sync();
-        // this buffer is next used two items from now, after the next item's barriers
-        if (tid < 16) sumq[tid] = 0;
     }
     if (!ok) *fail = 1;
 }

@@ -433,7 +433,7 @@ int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_blo
 // ------------------------------------------------------------------------------------------- grouped
 size_t qift_group_plan_bytes(int count) {
     if (count <= 0) return 0;
-    return sizeof(GroupHeader) + static_cast<size_t>(count) * sizeof(GroupProblemDev);
+    return sizeof(GroupHeader) + static_cast<size_t>(count) * (sizeof(GroupProblemDev) + 16 * sizeof(int));
 }
 
 int qift_group_plan(const qift_group_problem* problems, int count, int M, int levels, int x_dtype, int y_dtype, float clip_ratio,
@@ -471,8 +471,8 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     h->magic = kGroupMagic, h->count = count, h->M = M, h->levels = levels, h->y_bf16 = (y_dtype == QIFT_BF16);
     h->x_bf16 = (x_dtype == QIFT_BF16), h->clip = clip_ratio, h->total_items = items, h->rows_per_item = rows_per_item;
     h->max_k = max_k;
-    return cuda_status(cudaMemcpyAsync(plan_dev, plan_host, qift_group_plan_bytes(count), cudaMemcpyHostToDevice,
-                                       static_cast<cudaStream_t>(stream)));
+    return cuda_status(cudaMemcpyAsync(plan_dev, plan_host, sizeof(GroupHeader) + static_cast<size_t>(count) * sizeof(GroupProblemDev),
+                                       cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));
 }
 
 }  // extern "C"
@@ -484,27 +484,41 @@ const GroupHeader* plan_header(const void* plan_host, const void* plan_dev) {
     return h->magic == kGroupMagic ? h : nullptr;
 }
 
+inline const int* plan_sumq(const void* plan_dev, int count) {
+    return reinterpret_cast<const int*>(reinterpret_cast<const GroupProblemDev*>(static_cast<const GroupHeader*>(plan_dev) + 1) +
+                                        count);
+}
+
 template <int LV, int NT, int RT>
-int launch_grouped(const GroupHeader* h, const GroupProblemDev* dev, cudaStream_t st) {
-    const size_t stage = decode_stage_bytes(LV, RT, h->M);
-    const size_t fixed = grouped_smem_bytes(LV, RT, NT, h->M, 0);
-    int stages = static_cast<int>((110 * 1024 - fixed) / (stage + 16));
-    if (stages < 2) stages = 2;
-    if (stages > 12) stages = 12;
-    const size_t smem = grouped_smem_bytes(LV, RT, NT, h->M, stages);
+int launch_grouped(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
+                   cudaStream_t st) {
     auto kernel = linear_grouped_kernel<LV, NT, RT>;
-    cudaError_t e = allow_smem(kernel, smem);
-    if (e != cudaSuccess) return cuda_status(e);
-    int grid = 2 * sm_count();
-    if (grid > h->total_items) grid = h->total_items;
-    GroupParams gp{dev, h->count, h->total_items, h->M, h->y_bf16, stages};
-    return cuda_status(launch_pdl(kernel, dim3(grid), dim3(kDecThreads), smem, st, gp));
+    const size_t stage = decode_stage_bytes(LV, RT, h->M) + 16;
+    for (int first = 0; first < h->count; first += kGroupSlice) {  // the problem table of a launch lives in shared memory
+        const int count = (h->count - first < kGroupSlice) ? h->count - first : kGroupSlice;
+        const int item_first = host[first].item_begin;
+        const int item_end = (first + count < h->count) ? host[first + count].item_begin : h->total_items;
+        const size_t fixed = grouped_fixed_smem(RT, NT, count);
+        int stages = static_cast<int>((111 * 1024 - fixed) / stage);
+        if (stages < 2) stages = 2;
+        if (stages > 12) stages = 12;
+        const size_t smem = grouped_smem_bytes(LV, RT, NT, h->M, stages, count);
+        cudaError_t e = allow_smem(kernel, smem);
+        if (e != cudaSuccess) return cuda_status(e);
+        int grid = 2 * sm_count();
+        if (grid > item_end - item_first) grid = item_end - item_first;
+        GroupParams gp{dev + first, sumq, first, count, item_first, item_end, h->M, h->y_bf16, stages};
+        const int rc = cuda_status(launch_pdl(kernel, dim3(grid), dim3(kDecThreads), smem, st, gp));
+        if (rc != QIFT_OK) return rc;
+    }
+    return QIFT_OK;
 }
 
 template <int LV>
-int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* dev, cudaStream_t st) {
-    if (h->M > 8) return launch_grouped<LV, 2, 1>(h, dev, st);
-    return launch_grouped<LV, 1, 2>(h, dev, st);
+int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
+                     cudaStream_t st) {
+    if (h->M > 8) return launch_grouped<LV, 2, 1>(h, host, dev, sumq, st);
+    return launch_grouped<LV, 1, 2>(h, host, dev, sumq, st);
 }
 }  // namespace
 
@@ -516,27 +530,30 @@ int qift_group_quantize_act(const void* plan_host, const void* plan_dev, void* s
     const GroupProblemDev* dev = reinterpret_cast<const GroupProblemDev*>(static_cast<const GroupHeader*>(plan_dev) + 1);
     const size_t smem = static_cast<size_t>(h->max_k) * 4;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int* sumq = const_cast<int*>(plan_sumq(plan_dev, h->count));
     const dim3 grid(static_cast<unsigned>(h->count) * h->M);
     if (h->x_bf16) {
         cudaError_t e = allow_smem(quantize_act_grouped_kernel<true>, smem);
         if (e != cudaSuccess) return cuda_status(e);
-        return cuda_status(launch_pdl(quantize_act_grouped_kernel<true>, grid, dim3(kRowThreads), smem, st, dev, h->M, h->clip));
+        return cuda_status(launch_pdl(quantize_act_grouped_kernel<true>, grid, dim3(kRowThreads), smem, st, dev, sumq, h->M, h->clip));
     }
     cudaError_t e = allow_smem(quantize_act_grouped_kernel<false>, smem);
     if (e != cudaSuccess) return cuda_status(e);
-    return cuda_status(launch_pdl(quantize_act_grouped_kernel<false>, grid, dim3(kRowThreads), smem, st, dev, h->M, h->clip));
+    return cuda_status(launch_pdl(quantize_act_grouped_kernel<false>, grid, dim3(kRowThreads), smem, st, dev, sumq, h->M, h->clip));
 }
 
 int qift_group_linear(const void* plan_host, const void* plan_dev, void* stream) {
     const GroupHeader* h = plan_header(plan_host, plan_dev);
     if (!h) return QIFT_ERR_INVALID_ARG;
     const GroupProblemDev* dev = reinterpret_cast<const GroupProblemDev*>(static_cast<const GroupHeader*>(plan_dev) + 1);
+    const GroupProblemDev* host = reinterpret_cast<const GroupProblemDev*>(h + 1);
+    const int* sumq = plan_sumq(plan_dev, h->count);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     switch (h->levels) {
-        case QIFT_LEVELS_MNZ: return dispatch_grouped<QIFT_LEVELS_MNZ>(h, dev, st);
-        case QIFT_LEVELS_POT: return dispatch_grouped<QIFT_LEVELS_POT>(h, dev, st);
-        case QIFT_LEVELS_SYM: return dispatch_grouped<QIFT_LEVELS_SYM>(h, dev, st);
-        default: return dispatch_grouped<QIFT_LEVELS_INT4>(h, dev, st);
+        case QIFT_LEVELS_MNZ: return dispatch_grouped<QIFT_LEVELS_MNZ>(h, host, dev, sumq, st);
+        case QIFT_LEVELS_POT: return dispatch_grouped<QIFT_LEVELS_POT>(h, host, dev, sumq, st);
+        case QIFT_LEVELS_SYM: return dispatch_grouped<QIFT_LEVELS_SYM>(h, host, dev, sumq, st);
+        default: return dispatch_grouped<QIFT_LEVELS_INT4>(h, host, dev, sumq, st);
     }
 }
 

@@ -84,22 +84,22 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint = 0x989680u) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(hint)  // time hint: the hardware may park the thread while it waits
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after ~2^22 polls (each poll may itself sleep for a hardware-chosen
-// interval), records the site and returns false.  Callers skip their remaining work on false.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int site) {
-    for (uint32_t i = 0; i < (1u << 22); ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
+// Bounded wait: gives up after 2^20 polls (each poll may itself be suspended by the hardware for up
+// to its time hint), records the site and returns false.  Callers skip their remaining work on false.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int site, uint32_t hint = 0x989680u) {
+    for (uint32_t i = 0; i < (1u << 20); ++i) {
+        if (mbar_try_wait(bar, parity, hint)) return true;
     }
     report_timeout(site);
     return false;
@@ -128,6 +128,22 @@ __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, 
         "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// The same with the A operand formed inside the instruction sequence: a_i = (w_i & mask) ^ flip.
+// Keeping the logic ops and the mma in one block lets the assembler write the masked words straight
+// into the operand registers.
+__device__ __forceinline__ void mma_u8s8_masked(int (&d)[4], uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3,
+                                                uint32_t mask, uint32_t flip, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "{\n\t.reg .b32 a0, a1, a2, a3;\n\t"
+        "lop3.b32 a0, %4, %8, %9, 0x6a;\n\t"
+        "lop3.b32 a1, %5, %8, %9, 0x6a;\n\t"
+        "lop3.b32 a2, %6, %8, %9, 0x6a;\n\t"
+        "lop3.b32 a3, %7, %8, %9, 0x6a;\n\t"
+        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {a0,a1,a2,a3}, {%10,%11}, {%0,%1,%2,%3};\n\t}"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+        : "r"(w0), "r"(w1), "r"(w2), "r"(w3), "r"(mask), "r"(flip), "r"(b0), "r"(b1));
 }
 
 __device__ __forceinline__ uint16_t f32_to_bf16_bits(float f) {

@@ -7,9 +7,9 @@
 //    slice of q_a, into a shared-memory ring guarded by mbarriers.  The weight copies are issued BEFORE the programmatic-dependent-launch
 //    wait, so in a stream of such launches the next layer's weights are in flight while the previous
 //    layer finishes.  Eight consumer warps split each slab along K; a lane turns a packed word into
-//    four u8 operand registers with one LOP3 each (w & (0x03030303 << 2t) = code * 4^t, which the
+//    u8 operand registers with one logic op each (w & (0x03030303 << 2t) = code * 4^t, which the
 //    integer tensor-core instruction mma.sync.m16n8k32.u8.s8 multiplies against q_a directly) and keeps
-//    one accumulator set per t; the exact division by 4^t, the affine level map
+//    one accumulator set per place value; the exact division by the place value, the affine level map
 //    (level = alpha*code + gamma  =>  acc = alpha * sum code*q + gamma * sum q) and the scales come last.
 #pragma once
 
@@ -104,15 +104,95 @@ constexpr int kDecConsumers = kDecWarps * 32;      // 256
 constexpr int kDecThreads = kDecConsumers + 32;    // + producer warp
 constexpr int kQPad = 64;
 
+// How one packed word becomes tensor-core operands.  An m16n8k32 instruction has two k-halves of
+// 16; a lane supplies 4 bytes of each.  Both halves are fed from the SAME word: half 0 takes code
+// plane tt (w & mask), half 1 takes plane tt+1, so that the matching activations are two adjacent
+// 32-bit words of q_a -- an aligned register pair, no register shuffling.  The two planes differ by
+// a factor 4 (INT4: 16) in place value; either the odd plane is shifted down first (plain q_a), or
+// q_a arrives with its even-plane bytes already multiplied by that factor (PRESCALED, the grouped
+// path), in which case a single logic op per operand register remains.
+//   accumulator sets: MNZ/SYM 2 (planes 0-1, 2-3), POT 4 (two code bits x two plane pairs), INT4 1
 template <int LV>
 struct DecodeTraits {
     static constexpr int PER = codes_per_word(LV);
-    static constexpr int NPL = PER / 4;                     // operand registers per packed word
+    static constexpr int NPL = PER / 4;                     // 32-bit q words per packed word
     static constexpr int QBYTES = kChunkWords * PER;        // q_a bytes per token per stage
     static constexpr int QSTRIDE = QBYTES + kQPad;
-    static constexpr int NQP = (LV == QIFT_LEVELS_POT) ? 2 : 1;  // q planes (POT: 5q and 6q)
     static constexpr int BPT = QBYTES / kDecConsumers;      // q bytes per consumer thread per token
+    static constexpr int NACC = (LV == QIFT_LEVELS_INT4) ? 1 : (LV == QIFT_LEVELS_POT) ? 4 : 2;
 };
+
+// Place value of accumulator set `a` (a power of two; the set holds scale * sum code*q exactly).
+template <int LV, bool PRESCALED>
+__host__ __device__ constexpr int acc_shift(int a) {
+    if (LV == QIFT_LEVELS_INT4) return PRESCALED ? 4 : 0;
+    if (LV == QIFT_LEVELS_POT) {  // sets: 0,1 = code bit 1 (planes 0-1, 2-3); 2,3 = code bit 0
+        const int bit1 = (a < 2) ? 1 : 0;
+        return bit1 + 4 * (a & 1) + (PRESCALED ? 2 : 0);
+    }
+    return 4 * a + (PRESCALED ? 2 : 0);
+}
+
+// Exact level sum from the accumulator sets and sum_k q:  acc = sum_k level(code_k) * q_k.
+template <int LV, bool PRESCALED, int NACC>
+__device__ __forceinline__ int level_sum(const int (&v)[NACC], int Sq) {
+    if constexpr (LV == QIFT_LEVELS_INT4) {
+        return (v[0] >> acc_shift<LV, PRESCALED>(0)) - 8 * Sq;  // code' = nibble ^ 8 = level + 8
+    } else if constexpr (LV == QIFT_LEVELS_POT) {                // level = 5*b1 + 3*b0 - 4
+        const int b1 = (v[0] >> acc_shift<LV, PRESCALED>(0)) + (v[1] >> acc_shift<LV, PRESCALED>(1));
+        const int b0 = (v[2] >> acc_shift<LV, PRESCALED>(2)) + (v[3] >> acc_shift<LV, PRESCALED>(3));
+        return 5 * b1 + 3 * b0 - 4 * Sq;
+    } else {
+        const int S = (v[0] >> acc_shift<LV, PRESCALED>(0)) + (v[1] >> acc_shift<LV, PRESCALED>(1));
+        return (LV == QIFT_LEVELS_MNZ) ? 2 * S - 3 * Sq : S - 2 * Sq;  // level = 2c - 3  /  c - 2
+    }
+}
+
+// One mma step of a warp: its four words of rows g (wa) and g+8 (wb) against the q words in qb
+// (qb[NPL*i + t] = q word of plane t of word i).
+template <int LV, int NT, bool PRESCALED>
+__device__ __forceinline__ void mma_tile_step(int (&acc)[NT][DecodeTraits<LV>::NACC][4], const uint4 wa, const uint4 wb,
+                                              const uint32_t (&qb)[NT][4 * DecodeTraits<LV>::NPL]) {
+    constexpr int NPL = DecodeTraits<LV>::NPL;
+    const uint32_t lo[4] = {wa.x, wa.y, wa.z, wa.w};
+    const uint32_t hi[4] = {wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if constexpr (LV == QIFT_LEVELS_INT4) {
+            const uint32_t lo1 = PRESCALED ? lo[i] : (lo[i] >> 4), hi1 = PRESCALED ? hi[i] : (hi[i] >> 4);
+            constexpr uint32_t m1 = PRESCALED ? 0xf0f0f0f0u : 0x0f0f0f0fu, f1 = PRESCALED ? 0x80808080u : 0x08080808u;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+                mma_u8s8(acc[nt][0], (lo[i] & 0x0f0f0f0fu) ^ 0x08080808u, (hi[i] & 0x0f0f0f0fu) ^ 0x08080808u, (lo1 & m1) ^ f1,
+                         (hi1 & m1) ^ f1, qb[nt][NPL * i], qb[nt][NPL * i + 1]);
+        } else {
+            const uint32_t lo2 = lo[i] >> 2, hi2 = hi[i] >> 2;  // unused when PRESCALED
+#pragma unroll
+            for (int tt = 0; tt < 4; tt += 2) {
+                if constexpr (LV == QIFT_LEVELS_POT) {
+#pragma unroll
+                    for (int bit = 1; bit >= 0; --bit) {
+                        const uint32_t m0 = (bit ? 0x02020202u : 0x01010101u) << (2 * tt);
+                        const uint32_t m1 = PRESCALED ? (m0 << 2) : m0;
+                        const uint32_t l1 = PRESCALED ? lo[i] : lo2, h1 = PRESCALED ? hi[i] : hi2;
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt)
+                            mma_u8s8(acc[nt][(bit ? 0 : 2) + tt / 2], lo[i] & m0, hi[i] & m0, l1 & m1, h1 & m1, qb[nt][NPL * i + tt],
+                                     qb[nt][NPL * i + tt + 1]);
+                    }
+                } else {
+                    const uint32_t m0 = 0x03030303u << (2 * tt);
+                    const uint32_t m1 = PRESCALED ? (m0 << 2) : m0;
+                    const uint32_t l1 = PRESCALED ? lo[i] : lo2, h1 = PRESCALED ? hi[i] : hi2;
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+                        mma_u8s8(acc[nt][tt / 2], lo[i] & m0, hi[i] & m0, l1 & m1, h1 & m1, qb[nt][NPL * i + tt],
+                                 qb[nt][NPL * i + tt + 1]);
+                }
+            }
+        }
+    }
+}
 
 struct DecodeParams {
     const uint32_t* packed;
@@ -127,24 +207,12 @@ struct DecodeParams {
 };
 
 __host__ __device__ inline size_t decode_stage_bytes(int lv, int rt, int M) {
-    const int per = codes_per_word(lv);
-    const int nqp = (lv == QIFT_LEVELS_POT) ? 2 : 1;
-    return static_cast<size_t>(rt) * kTileBytes + static_cast<size_t>(nqp) * M * (kChunkWords * per + kQPad);
+    return static_cast<size_t>(rt) * kTileBytes + static_cast<size_t>(M) * (kChunkWords * codes_per_word(lv) + kQPad);
 }
 __host__ __device__ inline size_t decode_smem_bytes(int lv, int rt, int nt, int M, int stages) {
-    return stages * decode_stage_bytes(lv, rt, M) + static_cast<size_t>(kDecWarps) * rt * nt * 128 * 4  // reduce
+    const int nacc = (lv == QIFT_LEVELS_INT4) ? 1 : (lv == QIFT_LEVELS_POT) ? 4 : 2;
+    return stages * decode_stage_bytes(lv, rt, M) + static_cast<size_t>(kDecWarps) * rt * nt * nacc * 128 * 4  // reduce
            + 2 * stages * 8 + 16 * 4 + 16;  // barriers, sum-q, flag
-}
-
-// Per-byte k*q on four packed s8 values (|k*q| < 128).
-__device__ __forceinline__ uint32_t scale_s8x4(uint32_t q, int k) {
-    uint32_t r = 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int v = static_cast<int>(static_cast<int8_t>(q >> (8 * i))) * k;
-        r |= (static_cast<uint32_t>(v) & 0xffu) << (8 * i);
-    }
-    return r;
 }
 
 __device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers) : "memory"); }
@@ -154,15 +222,16 @@ __global__ void __launch_bounds__(kDecThreads)
 linear_decode_kernel(const DecodeParams p) {
     using T = DecodeTraits<LV>;
     constexpr int ROWS = 16 * RT;
+    constexpr int FR = RT * NT * T::NACC;  // accumulator fragments per warp
     extern __shared__ __align__(128) unsigned char smem[];
     const int M = p.M;
     const size_t stage_bytes = decode_stage_bytes(LV, RT, M);
     const int stages = p.stages;
     unsigned char* ring = smem;
-    int* red = reinterpret_cast<int*>(smem + stages * stage_bytes);                 // [warp][RT*NT][16][8]
-    uint64_t* full = reinterpret_cast<uint64_t*>(red + kDecWarps * RT * NT * 128);  // [stages]
-    uint64_t* empty = full + stages;                                                // [stages]
-    int* sumq = reinterpret_cast<int*>(empty + stages);                             // [16]
+    int* red = reinterpret_cast<int*>(smem + stages * stage_bytes);   // [warp][RT][NT][NACC][16][8]
+    uint64_t* full = reinterpret_cast<uint64_t*>(red + kDecWarps * FR * 128);  // [stages]
+    uint64_t* empty = full + stages;                                           // [stages]
+    int* sumq = reinterpret_cast<int*>(empty + stages);                        // [16]
     volatile int* fail = sumq + 16;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -228,13 +297,13 @@ linear_decode_kernel(const DecodeParams p) {
     // -------------------------------------------------------------------- consumer warps
     pdl_wait();
     const int g = lane >> 2, cq = lane & 3;
-    int acc[RT][NT][T::NPL][4];
+    int acc[RT][NT][T::NACC][4];
 #pragma unroll
     for (int a = 0; a < RT; ++a)
 #pragma unroll
         for (int b = 0; b < NT; ++b)
 #pragma unroll
-            for (int t = 0; t < T::NPL; ++t)
+            for (int t = 0; t < T::NACC; ++t)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[a][b][t][i] = 0;
     int sq[8 * NT];
@@ -252,50 +321,37 @@ linear_decode_kernel(const DecodeParams p) {
         unsigned char* wst = ring + s * stage_bytes;
         unsigned char* qst = wst + RT * kTileBytes;
 
-        // sum of q per token (and the 5q / 6q planes of POT): every consumer thread owns BPT bytes
+        // sum of q per token: every consumer thread owns BPT bytes of each token's slice
         {
             const int off = tid * T::BPT;
             if (off < cw * T::PER) {
 #pragma unroll
                 for (int m = 0; m < 8 * NT; ++m) {
                     if (m < M) {
-                        uint32_t* qp = reinterpret_cast<uint32_t*>(qst + m * T::QSTRIDE + off);
+                        const uint32_t* qp = reinterpret_cast<const uint32_t*>(qst + m * T::QSTRIDE + off);
 #pragma unroll
-                        for (int i = 0; i < T::BPT / 4; ++i) {
-                            const uint32_t v = qp[i];
-                            sq[m] = dp4a_us(0x01010101u, v, sq[m]);
-                            if constexpr (LV == QIFT_LEVELS_POT) {
-                                qp[i] = scale_s8x4(v, 5);
-                                reinterpret_cast<uint32_t*>(qst + (M + m) * T::QSTRIDE + off)[i] = scale_s8x4(v, 6);
-                            }
-                        }
+                        for (int i = 0; i < T::BPT / 4; ++i) sq[m] = dp4a_us(0x01010101u, qp[i], sq[m]);
                     }
                 }
             }
-            if constexpr (LV == QIFT_LEVELS_POT) consumer_bar_sync();
         }
 
         if (16 * warp < cw) {
             // B operands: the lane's four words cover 4*PER consecutive q bytes of token g (+8)
-            uint32_t qb[NT][T::NQP][4 * T::NPL];
+            uint32_t qb[NT][4 * T::NPL];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 const int m = nt * 8 + g;
+                if (m < M) {
+                    const uint4* src = reinterpret_cast<const uint4*>(qst + m * T::QSTRIDE + (16 * warp + 4 * cq) * T::PER);
 #pragma unroll
-                for (int pl = 0; pl < T::NQP; ++pl) {
-                    if (m < M) {
-                        const uint4* src = reinterpret_cast<const uint4*>(qst + (pl * M + m) * T::QSTRIDE +
-                                                                          (16 * warp + 4 * cq) * T::PER);
-#pragma unroll
-                        for (int i = 0; i < T::NPL; ++i) {
-                            const uint4 v = src[i];
-                            qb[nt][pl][4 * i] = v.x, qb[nt][pl][4 * i + 1] = v.y;
-                            qb[nt][pl][4 * i + 2] = v.z, qb[nt][pl][4 * i + 3] = v.w;
-                        }
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 4 * T::NPL; ++i) qb[nt][pl][i] = 0;
+                    for (int i = 0; i < T::NPL; ++i) {
+                        const uint4 v = src[i];
+                        qb[nt][4 * i] = v.x, qb[nt][4 * i + 1] = v.y, qb[nt][4 * i + 2] = v.z, qb[nt][4 * i + 3] = v.w;
                     }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4 * T::NPL; ++i) qb[nt][i] = 0;
                 }
             }
 #pragma unroll
@@ -303,39 +359,7 @@ linear_decode_kernel(const DecodeParams p) {
                 // tile order: group ((slice*2 + half)*32 + lane); slice = this warp, half = rows g / g+8
                 const uint4 wa = *reinterpret_cast<const uint4*>(wst + rt * kTileBytes + ((2 * warp) * 32 + lane) * 16);
                 const uint4 wb = *reinterpret_cast<const uint4*>(wst + rt * kTileBytes + ((2 * warp + 1) * 32 + lane) * 16);
-                const uint32_t a_lo[4] = {wa.x, wa.y, wa.z, wa.w};
-                const uint32_t a_hi[4] = {wb.x, wb.y, wb.z, wb.w};
-#pragma unroll
-                for (int pr = 0; pr < 2; ++pr) {
-                    const int i0 = 2 * pr, i1 = 2 * pr + 1;
-#pragma unroll
-                    for (int t = 0; t < T::NPL; ++t) {
-                        if constexpr (LV == QIFT_LEVELS_INT4) {
-                            const uint32_t msk = 0x0f0f0f0fu << (4 * t), flip = 0x08080808u << (4 * t);
-#pragma unroll
-                            for (int nt = 0; nt < NT; ++nt)
-                                mma_u8s8(acc[rt][nt][t], (a_lo[i0] & msk) ^ flip, (a_hi[i0] & msk) ^ flip,
-                                         (a_lo[i1] & msk) ^ flip, (a_hi[i1] & msk) ^ flip,
-                                         qb[nt][0][i0 * T::NPL + t], qb[nt][0][i1 * T::NPL + t]);
-                        } else if constexpr (LV == QIFT_LEVELS_POT) {
-                            // 10*b1 + 6*b0 = 2*(level + 4): bit 1 against the 5q plane, bit 0 against 6q
-                            const uint32_t m1 = 0x02020202u << (2 * t), m0 = 0x01010101u << (2 * t);
-#pragma unroll
-                            for (int nt = 0; nt < NT; ++nt) {
-                                mma_u8s8(acc[rt][nt][t], a_lo[i0] & m1, a_hi[i0] & m1, a_lo[i1] & m1, a_hi[i1] & m1,
-                                         qb[nt][0][i0 * T::NPL + t], qb[nt][0][i1 * T::NPL + t]);
-                                mma_u8s8(acc[rt][nt][t], a_lo[i0] & m0, a_hi[i0] & m0, a_lo[i1] & m0, a_hi[i1] & m0,
-                                         qb[nt][1][i0 * T::NPL + t], qb[nt][1][i1 * T::NPL + t]);
-                            }
-                        } else {
-                            const uint32_t msk = 0x03030303u << (2 * t);
-#pragma unroll
-                            for (int nt = 0; nt < NT; ++nt)
-                                mma_u8s8(acc[rt][nt][t], a_lo[i0] & msk, a_hi[i0] & msk, a_lo[i1] & msk, a_hi[i1] & msk,
-                                         qb[nt][0][i0 * T::NPL + t], qb[nt][0][i1 * T::NPL + t]);
-                        }
-                    }
-                }
+                mma_tile_step<LV, NT, false>(acc[rt], wa, wb, qb);
             }
         }
         if (nchunks > stages) {
@@ -345,22 +369,17 @@ linear_decode_kernel(const DecodeParams p) {
     }
     if (!ok) *fail = 1;
 
-    // per-warp partials: divide the t-planes out (exact) and park them for the cross-warp sum
-    constexpr int SH = (LV == QIFT_LEVELS_INT4) ? 4 : 2;
+    // per-warp partials, parked for the cross-warp sum
 #pragma unroll
     for (int rt = 0; rt < RT; ++rt)
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            int* dst = red + ((warp * RT + rt) * NT + nt) * 128;
+        for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                int v = 0;
+            for (int a = 0; a < T::NACC; ++a) {
+                int* dst = red + (((warp * RT + rt) * NT + nt) * T::NACC + a) * 128;
 #pragma unroll
-                for (int t = 0; t < T::NPL; ++t) v += acc[rt][nt][t][i] >> (SH * t);
-                const int row = g + ((i & 2) ? 8 : 0), tok = 2 * cq + (i & 1);
-                dst[row * 8 + tok] = v;
+                for (int i = 0; i < 4; ++i) dst[(g + ((i & 2) ? 8 : 0)) * 8 + 2 * cq + (i & 1)] = acc[rt][nt][a][i];
             }
-        }
 #pragma unroll
     for (int m = 0; m < 8 * NT; ++m) {
         if (m < M) {
@@ -378,15 +397,15 @@ linear_decode_kernel(const DecodeParams p) {
         const int n = n0 + row;
         if (n >= p.N) continue;
         const int rt = row / 16, r = row % 16, nt = m / 8, tk = m % 8;
-        int S = 0;
+        int v[T::NACC];
 #pragma unroll
-        for (int w = 0; w < kDecWarps; ++w) S += red[((w * RT + rt) * NT + nt) * 128 + r * 8 + tk];
-        const int Sq = sumq[m];
-        int acc_v;
-        if constexpr (LV == QIFT_LEVELS_MNZ) acc_v = 2 * S - 3 * Sq;
-        else if constexpr (LV == QIFT_LEVELS_SYM) acc_v = S - 2 * Sq;
-        else if constexpr (LV == QIFT_LEVELS_POT) acc_v = (S >> 1) - 4 * Sq;
-        else acc_v = S - 8 * Sq;
+        for (int a = 0; a < T::NACC; ++a) {
+            int S = 0;
+#pragma unroll
+            for (int w = 0; w < kDecWarps; ++w) S += red[(((w * RT + rt) * NT + nt) * T::NACC + a) * 128 + r * 8 + tk];
+            v[a] = S;
+        }
+        const int acc_v = level_sum<LV, false, T::NACC>(v, sumq[m]);
         const size_t idx = static_cast<size_t>(m) * p.N + n;
         if (p.acc_debug) p.acc_debug[idx] = acc_v;
         const float y = scale_epilogue(acc_v, p.s_a[m], p.s_n[n]);

@@ -50,9 +50,13 @@ constexpr uint32_t kGroupMagic = 0x51494654u;
 // ------------------------------------------------------------------------------------------------
 // grouped quantizer: one CTA per (problem, token row); also leaves sum_k q_a for the product kernel
 // ------------------------------------------------------------------------------------------------
+// q_a is written PRESCALED for the product kernel (see mma_tile_step): with two-bit weights the
+// bytes of the even code planes (k % 16 in 0..3 or 8..11) hold 4*q, with INT4 weights the bytes of
+// plane 0 (k % 8 in 0..3) hold 16*q; sumq holds the plain sum of q.
 template <bool BF16_IN>
 __global__ void __launch_bounds__(kRowThreads)
-quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* __restrict__ sumq, int M, float clip) {
+quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* __restrict__ sumq, int M, float clip,
+                            int int4_weights) {
     extern __shared__ __align__(16) float row[];
     __shared__ float red[kRowThreads / 32];
     __shared__ int redi[kRowThreads / 32];
@@ -91,7 +95,9 @@ quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* _
                 int v = __float2int_rn(__fdiv_rn(e[j], s_u));
                 v = max(-8, min(7, v));
                 total += v;
-                w |= (static_cast<uint32_t>(v) & 0xffu) << (8 * j);
+                // i = 32-bit word of this 16-byte group = code plane (two-bit: i; INT4: i & 1)
+                const int mult = int4_weights ? ((i & 1) ? 1 : 16) : ((i & 1) ? 1 : 4);
+                w |= (static_cast<uint32_t>(v * mult) & 0xffu) << (8 * j);
             }
             out[i] = w;
         }
@@ -127,10 +133,11 @@ static_assert(sizeof(SmemProblem) == 64, "shared-memory problem record is 64 byt
 constexpr int kGroupSlice = 256;  // problems per launch (their table lives in shared memory)
 
 // Walks this CTA's share of the work list chunk by chunk; the producer and the consumers each run
-// one and see the same sequence.
+// one and see the same sequence.  PER = codes per packed word.
+template <int PER>
 struct GroupCursor {
     const SmemProblem* table;
-    int count, item_end, rows_per_item, per;
+    int count, item_end, rows_per_item;
     int item, p;
     const unsigned char* wbase;   // first tile of the item's first row block
     const int8_t* q_a;
@@ -138,8 +145,8 @@ struct GroupCursor {
     int N, K, n0, tiles_valid, words_per_row, nchunks;
     int chunk;
 
-    __device__ __forceinline__ void init(const SmemProblem* t, int cnt, int item_first, int item_last, int rpi, int per_) {
-        table = t, count = cnt, item_end = item_last, rows_per_item = rpi, per = per_;
+    __device__ __forceinline__ void init(const SmemProblem* t, int cnt, int item_first, int item_last, int rpi) {
+        table = t, count = cnt, item_end = item_last, rows_per_item = rpi;
         item = item_first + blockIdx.x, p = 0, chunk = 0;
         load_item();
     }
@@ -149,10 +156,10 @@ struct GroupCursor {
         while (p + 1 < count && item >= table[p + 1].item_begin) ++p;
         const SmemProblem& P = table[p];
         N = P.N, K = P.K;
-        words_per_row = K / per;
+        words_per_row = K / PER;
         nchunks = (words_per_row + kChunkWords - 1) / kChunkWords;
         n0 = (item - P.item_begin) * rows_per_item;
-        tiles_valid = (min(rows_per_item, N - n0) + 15) / 16;
+        tiles_valid = (min(rows_per_item, N - n0) + 15) >> 4;
         const int pitch = round_up16(words_per_row);
         rb_bytes = static_cast<size_t>(16) * pitch * 4;
         wbase = P.packed + static_cast<size_t>(n0) * pitch * 4;
@@ -169,11 +176,16 @@ struct GroupCursor {
     }
 };
 
-__host__ __device__ inline size_t grouped_fixed_smem(int rt, int nt, int count) {
-    return static_cast<size_t>(count) * sizeof(SmemProblem) + 2 * static_cast<size_t>(kDecWarps) * rt * nt * 128 * 4 + 16;
+// Cross-warp reduction buffer: [warp][row tile][accumulator set][token][row], only the M live columns.
+__host__ __device__ inline int grouped_red_ints(int lv, int rt, int M) {
+    const int nacc = (lv == QIFT_LEVELS_INT4) ? 1 : (lv == QIFT_LEVELS_POT) ? 4 : 2;
+    return kDecWarps * rt * nacc * 16 * M;
 }
-__host__ __device__ inline size_t grouped_smem_bytes(int lv, int rt, int nt, int M, int stages, int count) {
-    return grouped_fixed_smem(rt, nt, count) + stages * (decode_stage_bytes(lv, rt, M) + 16);
+__host__ __device__ inline size_t grouped_fixed_smem(int lv, int rt, int M, int count) {
+    return static_cast<size_t>(count) * sizeof(SmemProblem) + 2 * static_cast<size_t>(grouped_red_ints(lv, rt, M)) * 4 + 16;
+}
+__host__ __device__ inline size_t grouped_smem_bytes(int lv, int rt, int M, int stages, int count) {
+    return grouped_fixed_smem(lv, rt, M, count) + stages * (decode_stage_bytes(lv, rt, M) + 16);
 }
 
 struct GroupParams {
@@ -185,15 +197,16 @@ struct GroupParams {
     int M, y_bf16, stages;
 };
 
-template <int LV, int NT, int RT>
+// M1: the single-token specialisation (only accumulator column 0 is live).
+template <int LV, int NT, int RT, bool M1>
 __global__ void __launch_bounds__(kDecThreads)
 linear_grouped_kernel(const GroupParams gp) {
     using T = DecodeTraits<LV>;
     constexpr int ROWS = 16 * RT;
-    constexpr int RED = kDecWarps * RT * NT * 128;  // ints per reduction buffer
     extern __shared__ __align__(128) unsigned char smem[];
-    const int M = gp.M;
-    const size_t stage_bytes = decode_stage_bytes(LV, RT, M);
+    const int M = M1 ? 1 : gp.M;
+    const int RED = grouped_red_ints(LV, RT, M);  // ints per reduction buffer
+    const uint32_t stage_bytes = static_cast<uint32_t>(decode_stage_bytes(LV, RT, M));
     const int stages = gp.stages;
     unsigned char* ring = smem;
     int* red_all = reinterpret_cast<int*>(smem + stages * stage_bytes);
@@ -226,18 +239,19 @@ linear_grouped_kernel(const GroupParams gp) {
 
     if (warp == kDecWarps) {
         // ---------------------------------------------------------------- producer warp
-        auto expect = [&](const GroupCursor& c, int s) {
+        using Cursor = GroupCursor<T::PER>;
+        auto expect = [&](const Cursor& c, int s) {
             if (lane == 0) mbar_expect_tx(&full[s], c.chunk_words() * (64 * c.tiles_valid + T::PER * M));
             __syncwarp();
         };
-        auto issue_w = [&](const GroupCursor& c, int s) {  // one bulk copy per 16-row tile
+        auto issue_w = [&](const Cursor& c, int s) {  // one bulk copy per 16-row tile
             const uint32_t bytes = c.chunk_words() * 16 * 4;
             unsigned char* dst = ring + s * stage_bytes;
             if (lane < c.tiles_valid)
                 bulk_g2s(dst + lane * kTileBytes, c.wbase + lane * c.rb_bytes + static_cast<size_t>(c.chunk) * kTileBytes, bytes,
                          &full[s]);
         };
-        auto issue_q = [&](const GroupCursor& c, int s) {
+        auto issue_q = [&](const Cursor& c, int s) {
             const uint32_t seg = c.chunk_words() * T::PER;
             unsigned char* dst = ring + s * stage_bytes + RT * kTileBytes;
             for (int m = lane; m < M; m += 32)
@@ -245,23 +259,25 @@ linear_grouped_kernel(const GroupParams gp) {
                          &full[s]);
         };
         // the packed weights never depend on the previous kernel: fill the ring with them first
-        GroupCursor a;
-        a.init(table, gp.count, gp.item_first, gp.item_end, ROWS, T::PER);
+        Cursor a;
+        a.init(table, gp.count, gp.item_first, gp.item_end, ROWS);
         int pre = 0;
         for (; pre < stages && a.valid(); ++pre, a.next()) {
             expect(a, pre);
             issue_w(a, pre);
         }
         pdl_wait();
-        GroupCursor b;
-        b.init(table, gp.count, gp.item_first, gp.item_end, ROWS, T::PER);
+        Cursor b;
+        b.init(table, gp.count, gp.item_first, gp.item_end, ROWS);
         for (int i = 0; i < pre; ++i, b.next()) issue_q(b, i);
-        for (uint32_t it = pre; b.valid(); ++it, b.next()) {
-            const int s = it % stages;
-            if (!mbar_wait(&empty[s], ((it / stages) - 1) & 1, 3)) break;
+        int s = 0;
+        uint32_t ph = 0;  // parity of the consumers' release this slot is waiting for
+        for (; b.valid(); b.next()) {
+            if (!mbar_wait(&empty[s], ph, 3)) break;
             expect(b, s);
             issue_w(b, s);
             issue_q(b, s);
+            if (++s == stages) s = 0, ph ^= 1;
         }
         return;
     }
@@ -269,128 +285,75 @@ linear_grouped_kernel(const GroupParams gp) {
     // -------------------------------------------------------------------- consumer warps
     pdl_wait();
     const int g = lane >> 2, cq = lane & 3;
-    GroupCursor cur;
-    cur.init(table, gp.count, gp.item_first, gp.item_end, ROWS, T::PER);
+    GroupCursor<T::PER> cur;
+    cur.init(table, gp.count, gp.item_first, gp.item_end, ROWS);
     bool ok = true;
-    uint32_t it = 0, item_no = 0;
-    constexpr int SH = (LV == QIFT_LEVELS_INT4) ? 4 : 2;
+    int s = 0;
+    uint32_t ph = 0, item_no = 0;
     // epilogue role of this thread: output (row, token) = (tid % ROWS, tid / ROWS); ROWS * M <= 256
     const int e_row = tid % ROWS, e_m = tid / ROWS;
+    const uint32_t a_off = (2 * warp * 32 + lane) * 16;           // this lane's group inside a tile (rows g), +512 for g+8
+    const uint32_t q_off = (16 * warp + 4 * cq) * T::PER;         // this lane's q bytes inside a token's slice
 
     for (; cur.valid() && ok; ++item_no) {
         int* red = red_all + RED * (item_no & 1);
-        int acc[RT][NT][T::NPL][4];
+        int acc[RT][NT][T::NACC][4];
 #pragma unroll
         for (int a = 0; a < RT; ++a)
 #pragma unroll
             for (int b = 0; b < NT; ++b)
 #pragma unroll
-                for (int t = 0; t < T::NPL; ++t)
+                for (int t = 0; t < T::NACC; ++t)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) acc[a][b][t][i] = 0;
-        const SmemProblem P = table[cur.p];
+        const SmemProblem* P = &table[cur.p];
         const int n0 = cur.n0;
         const int e_n = n0 + e_row;
-        const bool e_on = (e_m < M) && (e_n < P.N);
+        const bool e_on = (e_m < M) && (e_n < cur.N);
         // fetch what the epilogue needs now; the loads complete under the chunk loop
         float e_sn = 0.0f, e_sa = 0.0f;
         int e_sq = 0;
         if (e_on) {
-            e_sn = __ldg(P.s_n + e_n);
-            e_sa = P.s_a[e_m];
-            e_sq = gp.sumq[P.index * 16 + e_m];
+            e_sn = __ldg(P->s_n + e_n);
+            e_sa = P->s_a[e_m];
+            e_sq = gp.sumq[P->index * 16 + e_m];
         }
 
         for (;;) {
-            const int s = it % stages;
-            if (!mbar_wait(&full[s], (it / stages) & 1, 4)) {
+            if (!mbar_wait(&full[s], ph, 4)) {
                 ok = false;
                 break;
             }
             const int cw = cur.chunk_words();
             unsigned char* wst = ring + s * stage_bytes;
             unsigned char* qst = wst + RT * kTileBytes;
-            if constexpr (LV == QIFT_LEVELS_POT) {  // build the 5q and 6q planes
-                const int off = tid * T::BPT;
-                if (off < cw * T::PER) {
-#pragma unroll
-                    for (int m = 0; m < 8 * NT; ++m) {
-                        if (m < M) {
-                            uint32_t* qp = reinterpret_cast<uint32_t*>(qst + m * T::QSTRIDE + off);
-#pragma unroll
-                            for (int i = 0; i < T::BPT / 4; ++i) {
-                                const uint32_t v = qp[i];
-                                qp[i] = scale_s8x4(v, 5);
-                                reinterpret_cast<uint32_t*>(qst + (M + m) * T::QSTRIDE + off)[i] = scale_s8x4(v, 6);
-                            }
-                        }
-                    }
-                }
-                consumer_bar_sync();
-            }
             if (16 * warp < cw) {
-                uint32_t qb[NT][T::NQP][4 * T::NPL];
+                uint32_t qb[NT][4 * T::NPL];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     const int m = nt * 8 + g;
+                    if (M1 ? (g == 0) : (m < M)) {
+                        const uint4* src = reinterpret_cast<const uint4*>(qst + m * T::QSTRIDE + q_off);
 #pragma unroll
-                    for (int pl = 0; pl < T::NQP; ++pl) {
-                        if (m < M) {
-                            const uint4* src = reinterpret_cast<const uint4*>(qst + (pl * M + m) * T::QSTRIDE +
-                                                                              (16 * warp + 4 * cq) * T::PER);
-#pragma unroll
-                            for (int i = 0; i < T::NPL; ++i) {
-                                const uint4 v = src[i];
-                                qb[nt][pl][4 * i] = v.x, qb[nt][pl][4 * i + 1] = v.y;
-                                qb[nt][pl][4 * i + 2] = v.z, qb[nt][pl][4 * i + 3] = v.w;
-                            }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 4 * T::NPL; ++i) qb[nt][pl][i] = 0;
+                        for (int i = 0; i < T::NPL; ++i) {
+                            const uint4 v = src[i];
+                            qb[nt][4 * i] = v.x, qb[nt][4 * i + 1] = v.y, qb[nt][4 * i + 2] = v.z, qb[nt][4 * i + 3] = v.w;
                         }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 4 * T::NPL; ++i) qb[nt][i] = 0;
                     }
                 }
 #pragma unroll
                 for (int rt = 0; rt < RT; ++rt) {
-                    const uint4 wa = *reinterpret_cast<const uint4*>(wst + rt * kTileBytes + ((2 * warp) * 32 + lane) * 16);
-                    const uint4 wb = *reinterpret_cast<const uint4*>(wst + rt * kTileBytes + ((2 * warp + 1) * 32 + lane) * 16);
-                    const uint32_t a_lo[4] = {wa.x, wa.y, wa.z, wa.w};
-                    const uint32_t a_hi[4] = {wb.x, wb.y, wb.z, wb.w};
-#pragma unroll
-                    for (int pr = 0; pr < 2; ++pr) {
-                        const int i0 = 2 * pr, i1 = 2 * pr + 1;
-#pragma unroll
-                        for (int t = 0; t < T::NPL; ++t) {
-                            if constexpr (LV == QIFT_LEVELS_INT4) {
-                                const uint32_t msk = 0x0f0f0f0fu << (4 * t), flip = 0x08080808u << (4 * t);
-#pragma unroll
-                                for (int nt = 0; nt < NT; ++nt)
-                                    mma_u8s8(acc[rt][nt][t], (a_lo[i0] & msk) ^ flip, (a_hi[i0] & msk) ^ flip,
-                                             (a_lo[i1] & msk) ^ flip, (a_hi[i1] & msk) ^ flip,
-                                             qb[nt][0][i0 * T::NPL + t], qb[nt][0][i1 * T::NPL + t]);
-                            } else if constexpr (LV == QIFT_LEVELS_POT) {
-                                const uint32_t m1 = 0x02020202u << (2 * t), m0 = 0x01010101u << (2 * t);
-#pragma unroll
-                                for (int nt = 0; nt < NT; ++nt) {
-                                    mma_u8s8(acc[rt][nt][t], a_lo[i0] & m1, a_hi[i0] & m1, a_lo[i1] & m1, a_hi[i1] & m1,
-                                             qb[nt][0][i0 * T::NPL + t], qb[nt][0][i1 * T::NPL + t]);
-                                    mma_u8s8(acc[rt][nt][t], a_lo[i0] & m0, a_hi[i0] & m0, a_lo[i1] & m0, a_hi[i1] & m0,
-                                             qb[nt][1][i0 * T::NPL + t], qb[nt][1][i1 * T::NPL + t]);
-                                }
-                            } else {
-                                const uint32_t msk = 0x03030303u << (2 * t);
-#pragma unroll
-                                for (int nt = 0; nt < NT; ++nt)
-                                    mma_u8s8(acc[rt][nt][t], a_lo[i0] & msk, a_hi[i0] & msk, a_lo[i1] & msk, a_hi[i1] & msk,
-                                             qb[nt][0][i0 * T::NPL + t], qb[nt][0][i1 * T::NPL + t]);
-                            }
-                        }
-                    }
+                    const uint4 wa = *reinterpret_cast<const uint4*>(wst + rt * kTileBytes + a_off);
+                    const uint4 wb = *reinterpret_cast<const uint4*>(wst + rt * kTileBytes + a_off + 512);
+                    mma_tile_step<LV, NT, true>(acc[rt], wa, wb, qb);
                 }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[s]);
-            ++it;
+            if (++s == stages) s = 0, ph ^= 1;
             const bool last = cur.last_chunk();
             cur.next();
             if (last) break;
@@ -401,32 +364,34 @@ linear_grouped_kernel(const GroupParams gp) {
 #pragma unroll
         for (int rt = 0; rt < RT; ++rt)
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                int* dst = red + ((warp * RT + rt) * NT + nt) * 128;
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    int v = 0;
+                for (int a = 0; a < T::NACC; ++a) {
+                    int* dst = red + ((warp * RT + rt) * T::NACC + a) * 16 * M;
 #pragma unroll
-                    for (int t = 0; t < T::NPL; ++t) v += acc[rt][nt][t][i] >> (SH * t);
-                    dst[(g + ((i & 2) ? 8 : 0)) * 8 + 2 * cq + (i & 1)] = v;
+                    for (int i = 0; i < 4; ++i) {
+                        if (M1 && (i & 1)) continue;  // token 1 does not exist
+                        const int tok = nt * 8 + 2 * cq + (i & 1);
+                        if (tok < M) dst[tok * 16 + g + ((i & 2) ? 8 : 0)] = acc[rt][nt][a][i];
+                    }
                 }
-            }
         consumer_bar_sync();
         if (e_on) {
-            const int rt = e_row / 16, r = e_row % 16, nt = e_m / 8, tk = e_m % 8;
-            int S = 0;
+            const int rt = e_row / 16, r = e_row % 16;
+            int v[T::NACC];
 #pragma unroll
-            for (int w = 0; w < kDecWarps; ++w) S += red[((w * RT + rt) * NT + nt) * 128 + r * 8 + tk];
-            int acc_v;
-            if constexpr (LV == QIFT_LEVELS_MNZ) acc_v = 2 * S - 3 * e_sq;
-            else if constexpr (LV == QIFT_LEVELS_SYM) acc_v = S - 2 * e_sq;
-            else if constexpr (LV == QIFT_LEVELS_POT) acc_v = (S >> 1) - 4 * e_sq;
-            else acc_v = S - 8 * e_sq;
-            const size_t idx = static_cast<size_t>(e_m) * P.N + e_n;
-            if (P.acc_debug) P.acc_debug[idx] = acc_v;
+            for (int a = 0; a < T::NACC; ++a) {
+                int S = 0;
+#pragma unroll
+                for (int w = 0; w < kDecWarps; ++w) S += red[(((w * RT + rt) * T::NACC + a) * M + e_m) * 16 + r];
+                v[a] = S;
+            }
+            const int acc_v = level_sum<LV, true, T::NACC>(v, e_sq);
+            const size_t idx = static_cast<size_t>(e_m) * P->N + e_n;
+            if (P->acc_debug) P->acc_debug[idx] = acc_v;
             const float y = scale_epilogue(acc_v, e_sa, e_sn);
-            if (gp.y_bf16) static_cast<uint16_t*>(P.Y)[idx] = f32_to_bf16_bits(y);
-            else static_cast<float*>(P.Y)[idx] = y;
+            if (gp.y_bf16) static_cast<uint16_t*>(P->Y)[idx] = f32_to_bf16_bits(y);
+            else static_cast<float*>(P->Y)[idx] = y;
         }
     }
     if (!ok) *fail = 1;

@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstdio>
+#include <cstdlib>
 
 #include "common.cuh"
 #include "decode.cuh"
@@ -489,20 +490,22 @@ inline const int* plan_sumq(const void* plan_dev, int count) {
                                         count);
 }
 
-template <int LV, int NT, int RT>
+template <int LV, int NT, int RT, bool M1>
 int launch_grouped(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
                    cudaStream_t st) {
-    auto kernel = linear_grouped_kernel<LV, NT, RT>;
+    auto kernel = linear_grouped_kernel<LV, NT, RT, M1>;
     const size_t stage = decode_stage_bytes(LV, RT, h->M) + 16;
+    const char* e_stages = std::getenv("QIFT_G_STAGES");
     for (int first = 0; first < h->count; first += kGroupSlice) {  // the problem table of a launch lives in shared memory
         const int count = (h->count - first < kGroupSlice) ? h->count - first : kGroupSlice;
         const int item_first = host[first].item_begin;
         const int item_end = (first + count < h->count) ? host[first + count].item_begin : h->total_items;
-        const size_t fixed = grouped_fixed_smem(RT, NT, count);
-        int stages = static_cast<int>((111 * 1024 - fixed) / stage);
+        const size_t fixed = grouped_fixed_smem(LV, RT, h->M, count);
+        int stages = static_cast<int>((113 * 1024 - fixed) / stage);  // two CTAs per SM
         if (stages < 2) stages = 2;
         if (stages > 12) stages = 12;
-        const size_t smem = grouped_smem_bytes(LV, RT, NT, h->M, stages, count);
+        if (e_stages) stages = std::atoi(e_stages);
+        const size_t smem = grouped_smem_bytes(LV, RT, h->M, stages, count);
         cudaError_t e = allow_smem(kernel, smem);
         if (e != cudaSuccess) return cuda_status(e);
         int grid = 2 * sm_count();
@@ -517,8 +520,9 @@ int launch_grouped(const GroupHeader* h, const GroupProblemDev* host, const Grou
 template <int LV>
 int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
                      cudaStream_t st) {
-    if (h->M > 8) return launch_grouped<LV, 2, 1>(h, host, dev, sumq, st);
-    return launch_grouped<LV, 1, 2>(h, host, dev, sumq, st);
+    if (h->M > 8) return launch_grouped<LV, 2, 1, false>(h, host, dev, sumq, st);
+    if (h->M == 1) return launch_grouped<LV, 1, 2, true>(h, host, dev, sumq, st);
+    return launch_grouped<LV, 1, 2, false>(h, host, dev, sumq, st);
 }
 }  // namespace
 
@@ -535,11 +539,13 @@ int qift_group_quantize_act(const void* plan_host, const void* plan_dev, void* s
     if (h->x_bf16) {
         cudaError_t e = allow_smem(quantize_act_grouped_kernel<true>, smem);
         if (e != cudaSuccess) return cuda_status(e);
-        return cuda_status(launch_pdl(quantize_act_grouped_kernel<true>, grid, dim3(kRowThreads), smem, st, dev, sumq, h->M, h->clip));
+        return cuda_status(launch_pdl(quantize_act_grouped_kernel<true>, grid, dim3(kRowThreads), smem, st, dev, sumq, h->M, h->clip,
+                                      h->levels == QIFT_LEVELS_INT4 ? 1 : 0));
     }
     cudaError_t e = allow_smem(quantize_act_grouped_kernel<false>, smem);
     if (e != cudaSuccess) return cuda_status(e);
-    return cuda_status(launch_pdl(quantize_act_grouped_kernel<false>, grid, dim3(kRowThreads), smem, st, dev, sumq, h->M, h->clip));
+    return cuda_status(launch_pdl(quantize_act_grouped_kernel<false>, grid, dim3(kRowThreads), smem, st, dev, sumq, h->M, h->clip,
+                                  h->levels == QIFT_LEVELS_INT4 ? 1 : 0));
 }
 
 int qift_group_linear(const void* plan_host, const void* plan_dev, void* stream) {

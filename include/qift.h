@@ -188,6 +188,14 @@ int qift_group_quantize_act(const void* plan_host, const void* plan_dev, void* s
 int qift_group_linear(const void* plan_host, const void* plan_dev, void* stream);
 int qift_group_forward(const void* plan_host, const void* plan_dev, void* stream);
 
+/* qift_group_forward with the activations and the results in HOST memory.  The caller lays all X of
+ * the plan out in one device arena and all Y in another (the plan's X / Y pointers point into them)
+ * and keeps host mirrors of both (pinned memory makes the copies asynchronous).  The call enqueues
+ * one host-to-device copy of the X arena, the two grouped launches, and one device-to-host copy of
+ * the Y arena; y_host is valid once `stream` has been synchronized. */
+int qift_group_forward_host(const void* plan_host, const void* plan_dev, const void* x_host, void* x_dev,
+                            size_t x_bytes, const void* y_dev, void* y_host, size_t y_bytes, void* stream);
+
 /* ---- Product without any allocation by anyone ------------------------------------------------
  * (No counterpart in the paper: this is a packaging variant of qift_w2a4_linear's prefill route.)
  *

@@ -26,7 +26,7 @@ EXPORTS = [
     "qift_unpack_codes", "qift_rotate", "qift_quantize_act", "qift_w2a4_linear", "qift_w4a4_linear",
     "qift_linear_route", "qift_device_status", "qift_forward_scratch_bytes", "qift_forward", "qift_forward_host",
     "qift_group_plan_bytes", "qift_group_plan", "qift_group_quantize_act", "qift_group_linear", "qift_group_forward",
-    "qift_static_scratch_bytes", "qift_w2a4_linear_static",
+    "qift_group_forward_host", "qift_static_scratch_bytes", "qift_w2a4_linear_static",
 ]
 
 _lib = None
@@ -72,6 +72,7 @@ def lib() -> ctypes.CDLL:
         L.qift_group_plan.argtypes = [vp, ci, ci, ci, ci, ci, cf, vp, vp, sz, vp]
         for name in ("qift_group_quantize_act", "qift_group_linear", "qift_group_forward"):
             getattr(L, name).argtypes = [vp, vp, vp]
+        L.qift_group_forward_host.argtypes = [vp, vp, vp, vp, sz, vp, vp, sz, vp]
         L.qift_static_scratch_bytes.restype = sz
         L.qift_static_scratch_bytes.argtypes = []
         L.qift_w2a4_linear_static.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, vp, ci, vp, vp]
@@ -254,36 +255,64 @@ class GroupProblem(ctypes.Structure):
 
 class GroupPlan:
     """A validated problem list: host and device copies of the plan plus references that keep every
-    tensor named in it alive."""
+    tensor named in it alive.  `outputs[i]` / `accs[i]` are the results of problem i; `inputs[i]` is
+    its activation tensor (a view into the X arena when the plan owns the inputs)."""
 
-    def __init__(self, host, dev, keep, outputs, accs):
-        self.host, self.dev, self.keep, self.outputs, self.accs = host, dev, keep, outputs, accs
+    def __init__(self, host, dev, keep, inputs, outputs, accs, x_arena=None, y_arena=None):
+        self.host, self.dev, self.keep, self.inputs, self.outputs, self.accs = host, dev, keep, inputs, outputs, accs
+        self.x_arena, self.y_arena = x_arena, y_arena
+        self.x_host = self.y_host = None
 
 
 def qift_group_plan_bytes(count: int) -> int:
     return int(lib().qift_group_plan_bytes(count))
 
 
-def qift_group_plan(problems, levels: int, clip_ratio: float = 0.9, out_dtype=torch.float32, want_acc: bool = False):
+def _align(n, a=256):
+    return (n + a - 1) // a * a
+
+
+def qift_group_plan(problems, levels: int, clip_ratio: float = 0.9, out_dtype=torch.float32, want_acc: bool = False,
+                    arenas: bool = False):
     """problems: list of (X [M,K], packed, s_n, had_block) sharing M and the dtype of X.  Allocates
-    q_a / s_a / Y (and the accumulators when asked) and returns a GroupPlan."""
+    q_a / s_a / Y (and the accumulators when asked) and returns a GroupPlan.  With arenas=True the
+    activations are copied into one contiguous device arena and the outputs live in another, each
+    with a pinned host mirror (plan.x_host / plan.y_host), for qift_group_forward_host."""
     assert problems
     M = problems[0][0].shape[0]
     xdt = _dt(problems[0][0])
     device = problems[0][0].device
     arr = (GroupProblem * len(problems))()
-    keep, outs, accs = [], [], []
+    keep, ins, outs, accs = [], [], [], []
+    x_arena = y_arena = None
+    if arenas:
+        xe = problems[0][0].element_size()
+        ye = torch.empty(0, dtype=out_dtype).element_size()
+        xo, yo, x_off, y_off = 0, 0, [], []
+        for (X, packed, s_n, had_block) in problems:
+            x_off.append(xo), y_off.append(yo)
+            xo += _align(M * X.shape[1] * xe)
+            yo += _align(M * s_n.shape[0] * ye)
+        x_arena = torch.zeros(xo, dtype=torch.uint8, device=device)
+        y_arena = torch.zeros(yo, dtype=torch.uint8, device=device)
     for i, (X, packed, s_n, had_block) in enumerate(problems):
         _dev(X), _dev(packed), _dev(s_n, torch.float32)
         assert X.shape[0] == M and _dt(X) == xdt
         K, N = X.shape[1], s_n.shape[0]
+        if arenas:
+            xv = x_arena[x_off[i]:x_off[i] + M * K * xe].view(X.dtype).view(M, K)
+            xv.copy_(X)
+            X = xv
+            Y = y_arena[y_off[i]:y_off[i] + M * N * ye].view(out_dtype).view(M, N)
+        else:
+            Y = torch.empty((M, N), dtype=out_dtype, device=device)
         q_a = torch.empty((M, K), dtype=torch.int8, device=device)
         s_a = torch.empty((max(M, 4),), dtype=torch.float32, device=device)
-        Y = torch.empty((M, N), dtype=out_dtype, device=device)
         acc = torch.empty((M, N), dtype=torch.int32, device=device) if want_acc else None
         arr[i] = GroupProblem(X.data_ptr(), packed.data_ptr(), s_n.data_ptr(), q_a.data_ptr(), s_a.data_ptr(), Y.data_ptr(),
                               acc.data_ptr() if want_acc else None, N, K, had_block, 0)
         keep += [X, packed, s_n, q_a, s_a]
+        ins.append(X)
         outs.append(Y)
         accs.append(acc)
     nbytes = qift_group_plan_bytes(len(problems))
@@ -292,7 +321,11 @@ def qift_group_plan(problems, levels: int, clip_ratio: float = 0.9, out_dtype=to
     ydt = F32 if out_dtype == torch.float32 else BF16
     _check(lib().qift_group_plan(ctypes.addressof(arr), len(problems), M, levels, xdt, ydt, clip_ratio, host.data_ptr(),
                                  dev.data_ptr(), nbytes, _stream()), "qift_group_plan")
-    return GroupPlan(host, dev, keep, outs, accs)
+    plan = GroupPlan(host, dev, keep, ins, outs, accs, x_arena, y_arena)
+    if arenas:
+        plan.x_host = x_arena.cpu().pin_memory()
+        plan.y_host = torch.empty(y_arena.shape, dtype=torch.uint8).pin_memory()
+    return plan
 
 
 def qift_group_quantize_act(plan: GroupPlan):
@@ -325,3 +358,13 @@ def qift_w2a4_linear_static(packed, s_n, levels, q_a, s_a, out, acc=None):
     _check(lib().qift_w2a4_linear_static(_ptr(packed), _ptr(s_n), levels, _ptr(q_a), _ptr(s_a), M, N, K, _ptr(out),
                                          _dt(out), _ptr(acc), _stream()), "qift_w2a4_linear_static")
     return out
+
+
+def qift_group_forward_host(plan: GroupPlan):
+    """The grouped layer with activations read from plan.x_host and results written to plan.y_host
+    (pinned host arenas laid out like the device arenas); valid after the stream is synchronized."""
+    assert plan.x_arena is not None, "build the plan with arenas=True"
+    _check(lib().qift_group_forward_host(plan.host.data_ptr(), plan.dev.data_ptr(), plan.x_host.data_ptr(),
+                                         plan.x_arena.data_ptr(), plan.x_arena.numel(), plan.y_arena.data_ptr(),
+                                         plan.y_host.data_ptr(), plan.y_arena.numel(), _stream()), "qift_group_forward_host")
+    return plan.y_host

@@ -195,6 +195,7 @@ struct GroupParams {
     int count;                        // problems in the slice (<= kGroupSlice)
     int item_first, item_end;         // work items of the slice
     int M, y_bf16, stages;
+    int dbg;
 };
 
 // M1: the single-token specialisation (only accumulator column 0 is live).
@@ -327,13 +328,15 @@ linear_grouped_kernel(const GroupParams gp) {
             const int cw = cur.chunk_words();
             unsigned char* wst = ring + s * stage_bytes;
             unsigned char* qst = wst + RT * kTileBytes;
-            if (16 * warp < cw) {
+            if (16 * warp < cw && !(gp.dbg & 1)) {
                 uint32_t qb[NT][4 * T::NPL];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     const int m = nt * 8 + g;
-                    if (M1 ? (g == 0) : (m < M)) {
-                        const uint4* src = reinterpret_cast<const uint4*>(qst + m * T::QSTRIDE + q_off);
+                    // single token: every lane reads token 0 (a broadcast); accumulator columns 1..7 then
+                    // hold copies that are never read, and no lane needs predication or zero fill
+                    if (M1 || m < M) {
+                        const uint4* src = reinterpret_cast<const uint4*>(qst + (M1 ? 0 : m) * T::QSTRIDE + q_off);
 #pragma unroll
                         for (int i = 0; i < T::NPL; ++i) {
                             const uint4 v = src[i];
@@ -361,6 +364,7 @@ linear_grouped_kernel(const GroupParams gp) {
         if (!ok) break;
 
         // item epilogue: one barrier; the other reduction buffer belongs to the next item
+        if (gp.dbg & 2) continue;
 #pragma unroll
         for (int rt = 0; rt < RT; ++rt)
 #pragma unroll

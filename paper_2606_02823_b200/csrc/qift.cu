@@ -446,7 +446,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     if (M > 16) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (plan_bytes < qift_group_plan_bytes(count)) return QIFT_ERR_WORKSPACE;
     if (!aligned16(plan_dev) || !aligned16(plan_host)) return QIFT_ERR_ALIGNMENT;
-    const int rows_per_item = (M > 8) ? 16 : 32;
+    const int rows_per_item = (M > 8) ? 16 : (M == 1) ? 64 : 32;  // must match dispatch_grouped's row tiles
     GroupHeader* h = static_cast<GroupHeader*>(plan_host);
     GroupProblemDev* d = reinterpret_cast<GroupProblemDev*>(h + 1);
     int items = 0, max_k = 0;
@@ -501,16 +501,19 @@ int launch_grouped(const GroupHeader* h, const GroupProblemDev* host, const Grou
         const int item_first = host[first].item_begin;
         const int item_end = (first + count < h->count) ? host[first + count].item_begin : h->total_items;
         const size_t fixed = grouped_fixed_smem(LV, RT, h->M, count);
-        int stages = static_cast<int>((113 * 1024 - fixed) / stage);  // two CTAs per SM
+        const char* e_cps = std::getenv("QIFT_G_CPS");
+        const int cps = e_cps ? std::atoi(e_cps) : 2;
+        int stages = static_cast<int>(((cps == 3 ? 75 : cps == 4 ? 56 : 113) * 1024 - fixed) / stage);  // CTAs per SM
         if (stages < 2) stages = 2;
         if (stages > 12) stages = 12;
         if (e_stages) stages = std::atoi(e_stages);
         const size_t smem = grouped_smem_bytes(LV, RT, h->M, stages, count);
         cudaError_t e = allow_smem(kernel, smem);
         if (e != cudaSuccess) return cuda_status(e);
-        int grid = 2 * sm_count();
+        int grid = cps * sm_count();
         if (grid > item_end - item_first) grid = item_end - item_first;
-        GroupParams gp{dev + first, sumq, first, count, item_first, item_end, h->M, h->y_bf16, stages};
+        const char* e_dbg = std::getenv("QIFT_G_DBG");
+        GroupParams gp{dev + first, sumq, first, count, item_first, item_end, h->M, h->y_bf16, stages, e_dbg ? std::atoi(e_dbg) : 0};
         const int rc = cuda_status(launch_pdl(kernel, dim3(grid), dim3(kDecThreads), smem, st, gp));
         if (rc != QIFT_OK) return rc;
     }
@@ -521,7 +524,7 @@ template <int LV>
 int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
                      cudaStream_t st) {
     if (h->M > 8) return launch_grouped<LV, 2, 1, false>(h, host, dev, sumq, st);
-    if (h->M == 1) return launch_grouped<LV, 1, 2, true>(h, host, dev, sumq, st);
+    if (h->M == 1) return launch_grouped<LV, 1, 4, true>(h, host, dev, sumq, st);
     return launch_grouped<LV, 1, 2, false>(h, host, dev, sumq, st);
 }
 }  // namespace
@@ -567,6 +570,18 @@ int qift_group_forward(const void* plan_host, const void* plan_dev, void* stream
     const int rc = qift_group_quantize_act(plan_host, plan_dev, stream);
     if (rc != QIFT_OK) return rc;
     return qift_group_linear(plan_host, plan_dev, stream);
+}
+
+int qift_group_forward_host(const void* plan_host, const void* plan_dev, const void* x_host, void* x_dev, size_t x_bytes,
+                            const void* y_dev, void* y_host, size_t y_bytes, void* stream) {
+    if (!x_host || !x_dev || !y_dev || !y_host || x_bytes == 0 || y_bytes == 0) return QIFT_ERR_INVALID_ARG;
+    if (!plan_header(plan_host, plan_dev)) return QIFT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_status(e);
+    const int rc = qift_group_forward(plan_host, plan_dev, stream);
+    if (rc != QIFT_OK) return rc;
+    return cuda_status(cudaMemcpyAsync(y_host, y_dev, y_bytes, cudaMemcpyDeviceToHost, st));
 }
 
 // ------------------------------------------------------------------------- allocation-free product

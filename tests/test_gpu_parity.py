@@ -276,3 +276,28 @@ def test_grouped_rejects_bad_plans():
     assert e.value.status == qift.ERR_UNSUPPORTED_SHAPE
     L = qift.lib()
     assert L.qift_group_forward(None, None, None) == qift.ERR_INVALID_ARG
+
+
+def test_grouped_forward_host_arenas():
+    lv = qift.MNZ
+    probs, refs = [], []
+    for i, (N, K) in enumerate([(256, 256), (96, 512), (40, 1024)]):
+        W = synth.gaussian_weights(500 + i, N, K)
+        x, _ = synth.activations(600 + i, 2, K, 3)
+        p_ref, s_n, codes = oracle.pack_weights(W, lv, oracle.SCALE_ABSMAX)
+        q_ref, sa_ref = oracle.quantize_act(x, synth.had_block_for(K), 0.9)
+        refs.append(oracle.linear(codes, lv, s_n, q_ref, sa_ref)[0])
+        probs.append((dev(x), dev(p_ref.view(np.int32)), dev(s_n), synth.had_block_for(K)))
+    plan = qift.qift_group_plan(probs, lv, 0.9, arenas=True)
+    plan.x_arena.zero_()                       # the device copy must come from the host arena
+    y_host = qift.qift_group_forward_host(plan)
+    torch.cuda.synchronize()
+    assert_status_clean()
+    for ref, y in zip(refs, plan.outputs):
+        assert np.array_equal(y.cpu().numpy(), ref)
+    off = 0
+    for ref in refs:                           # and the host arena holds the same bytes
+        n = ref.size * 4
+        got = y_host[off:off + n].view(torch.float32).numpy().reshape(ref.shape)
+        assert np.array_equal(got, ref)
+        off += (n + 255) // 256 * 256

@@ -51,6 +51,21 @@ def quant_bytes(M, K, in_bytes=4):
     return M * K * in_bytes + M * K + 4 * M
 
 
+def reduce_max_ms(dist, ms, device):
+    """Step time of the job = the slowest rank's (device-measured) time."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(world, bytes_per_rank, ms_per_step):
+    """Whole-job GB/s: every replica moves bytes_per_rank per step, in ms_per_step."""
+    return world * bytes_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -258,11 +273,8 @@ def run_gpu(args):
             run_once()
         e1.record()
         torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
+        ms = reduce_max_ms(dist, e0.elapsed_time(e1), device)
         if dist:
-            t = torch.tensor([ms], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
             dist.barrier()
         return ms
 
@@ -309,7 +321,7 @@ def run_gpu(args):
 
     pk = peaks()
     step_ms = ms_grp / args.steps
-    value = world * bytes_step / (step_ms * 1e-3) / 1e9
+    value = aggregate_throughput(world, bytes_step, step_ms)
     launch_us = ms_grp_prod / args.steps * 1e3          # one persistent launch per step
     achieved = bytes_product / (launch_us * 1e-6) / 1e9
     percall_ms = ms_full / pc_steps

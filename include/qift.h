@@ -14,6 +14,11 @@
  *     before anything is launched, so a failing call has touched no buffer;
  *   - kernels are launched with programmatic stream serialization: each waits for its predecessor
  *     in the stream before it reads or writes any caller buffer, so ordinary stream order holds.
+ *     One exception: the product kernels start fetching the PACKED WEIGHTS before that wait (this is
+ *     what lets consecutive layers overlap).  It is safe whenever the weights were written by
+ *     qift_pack_weights, by a copy, or by any kernel that does not itself use programmatic early
+ *     launch -- i.e. always, unless a caller's own kernel both writes packed weights and calls
+ *     cudaTriggerProgrammaticLaunchCompletion before finishing them.
  */
 #ifndef QIFT_H_
 #define QIFT_H_
@@ -58,7 +63,9 @@ typedef enum {
     QIFT_ROUTE_AUTO = 0,
     QIFT_ROUTE_GENERIC = 1,  /* one warp per output channel, dp4a; any M, any K                     */
     QIFT_ROUTE_DECODE = 2,   /* bulk-copy staged, in-register decode, mma.sync; M <= 16             */
-    QIFT_ROUTE_PREFILL = 3   /* expand to int8 scratch, TMA + tcgen05 kind::i8, TMEM accumulators   */
+    QIFT_ROUTE_PREFILL = 3,  /* tcgen05 kind::i8 GEMM, codes expanded in the kernel; scratch 4*M    */
+    QIFT_ROUTE_PREFILL_SCRATCH = 4 /* codes expanded to an int8 [N,K] scratch first, then a TMA-fed
+                                      tcgen05 GEMM; scratch N*K bytes                              */
 } qift_route;
 
 const char* qift_status_string(int status);
@@ -67,9 +74,12 @@ const char* qift_status_string(int status);
  * the words per row to multiples of 16.  0 on bad input. */
 size_t qift_packed_bytes(int N, int K, int levels);
 
-/* Bytes of scratch qift_w2a4_linear / qift_w4a4_linear need for this problem (0 when the decode
- * route serves it; N*K rounded up to 1 KiB for the prefill route, which expands the codes to int8). */
+/* Bytes of scratch qift_w2a4_linear / qift_w4a4_linear need for this problem: 0 when the decode
+ * route serves it (M <= 16); 4*M rounded up to 1 KiB for 16 < M <= 768 (QIFT_ROUTE_PREFILL: the
+ * per-token sums of q_a); N*K rounded up to 1 KiB for M > 768 (QIFT_ROUTE_PREFILL_SCRATCH: the codes
+ * decoded to int8 once per call).  qift_workspace_bytes_route gives the figure for an explicit route. */
 size_t qift_workspace_bytes(int M, int N, int K, int levels);
+size_t qift_workspace_bytes_route(int M, int N, int K, int levels, int route);
 
 /* S1 (weight quantizer + packer).  Sec. 1 Eq. 1, Sec. 3.3, Sec. 3.5.
  *   W       in   fp32 [N,K], ALREADY rotated (this call never rotates)
@@ -118,7 +128,7 @@ int qift_quantize_act(const void* X, int x_dtype, int M, int K, int had_block, f
  *   Y         out [M,N] fp32 or bf16 (round to nearest even): ((float)acc * s_a[m]) * s_n[n]
  *   acc_debug out int32 [M,N] accumulators, or NULL
  *   workspace     >= qift_workspace_bytes(M,N,K,levels) bytes, 256-byte aligned; may be NULL when 0
- * M <= 16 takes the decode route, larger M the prefill route. */
+ * M <= 16 takes the decode route, 16 < M <= 768 the fused prefill route, larger M the scratch prefill route. */
 int qift_w2a4_linear(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a,
                      const float* s_a, int M, int N, int K, void* Y, int y_dtype, int32_t* acc_debug,
                      void* workspace, size_t workspace_bytes, void* stream);

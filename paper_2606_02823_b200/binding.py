@@ -19,10 +19,10 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CU
 MNZ, POT, SYM, INT4 = 0, 1, 2, 3
 SCALE_GIVEN, SCALE_ABSMAX, SCALE_MSE = 0, 1, 2
 F32, BF16 = 0, 1
-ROUTE_AUTO, ROUTE_GENERIC, ROUTE_DECODE, ROUTE_PREFILL = 0, 1, 2, 3
+ROUTE_AUTO, ROUTE_GENERIC, ROUTE_DECODE, ROUTE_PREFILL, ROUTE_PREFILL_SCRATCH = 0, 1, 2, 3, 4
 
 EXPORTS = [
-    "qift_status_string", "qift_packed_bytes", "qift_workspace_bytes", "qift_pack_weights",
+    "qift_status_string", "qift_packed_bytes", "qift_workspace_bytes", "qift_workspace_bytes_route", "qift_pack_weights",
     "qift_unpack_codes", "qift_rotate", "qift_quantize_act", "qift_w2a4_linear", "qift_w4a4_linear",
     "qift_linear_route", "qift_device_status", "qift_forward_scratch_bytes", "qift_forward", "qift_forward_host",
     "qift_group_plan_bytes", "qift_group_plan", "qift_group_quantize_act", "qift_group_linear", "qift_group_forward",
@@ -54,6 +54,8 @@ def lib() -> ctypes.CDLL:
         L.qift_packed_bytes.argtypes = [ci, ci, ci]
         L.qift_workspace_bytes.restype = sz
         L.qift_workspace_bytes.argtypes = [ci, ci, ci, ci]
+        L.qift_workspace_bytes_route.restype = sz
+        L.qift_workspace_bytes_route.argtypes = [ci, ci, ci, ci, ci]
         L.qift_pack_weights.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp]
         L.qift_unpack_codes.argtypes = [vp, ci, ci, ci, vp, vp]
         L.qift_rotate.argtypes = [vp, ci, ci, ci, vp, vp]
@@ -78,7 +80,8 @@ def lib() -> ctypes.CDLL:
         L.qift_w2a4_linear_static.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, vp, ci, vp, vp]
         for name in EXPORTS:
             if name not in ("qift_status_string", "qift_packed_bytes", "qift_workspace_bytes",
-                            "qift_forward_scratch_bytes", "qift_group_plan_bytes", "qift_static_scratch_bytes"):
+                            "qift_forward_scratch_bytes", "qift_group_plan_bytes", "qift_static_scratch_bytes",
+                            "qift_workspace_bytes_route"):
                 getattr(L, name).restype = ci
         _lib = L
     return _lib
@@ -112,8 +115,8 @@ def qift_packed_bytes(N: int, K: int, levels: int) -> int:
     return int(lib().qift_packed_bytes(N, K, levels))
 
 
-def qift_workspace_bytes(M: int, N: int, K: int, levels: int) -> int:
-    return int(lib().qift_workspace_bytes(M, N, K, levels))
+def qift_workspace_bytes(M: int, N: int, K: int, levels: int, route: int = ROUTE_AUTO) -> int:
+    return int(lib().qift_workspace_bytes_route(M, N, K, levels, route))
 
 
 def qift_pack_weights(W, levels: int, scale_mode: int, s_n=None, packed=None):
@@ -168,7 +171,7 @@ def _linear(fn_name, packed, s_n, levels, q_a, s_a, N, out_dtype, want_acc, work
         out = torch.empty((M, N), dtype=out_dtype, device=q_a.device)
     assert out.dtype in (torch.float32, torch.bfloat16)
     acc = torch.empty((M, N), dtype=torch.int32, device=q_a.device) if want_acc else None
-    need = qift_workspace_bytes(max(M, 17) if route == ROUTE_PREFILL else M, N, K, levels)
+    need = qift_workspace_bytes(M, N, K, levels, route)
     if workspace is None and need:
         workspace = torch.empty(need, dtype=torch.uint8, device=q_a.device)
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()

@@ -25,7 +25,8 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
     __shared__ float red[kPackThreads / 32];
     __shared__ double err[kNumCandidates][kPackThreads / 32];
     __shared__ float s_shared;
-    pdl_launch_dependents();
+    // No early launch of dependents here: the product kernels prefetch packed weights before their
+    // own dependency wait, which is only safe if whoever writes those weights has fully completed.
     pdl_wait();
     const size_t n = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;

@@ -10,10 +10,15 @@
 #include "grouped.cuh"
 #include "pack.cuh"
 #include "prefill.cuh"
+#include "prefill_fused.cuh"
 #include "rotate_quant.cuh"
 
 namespace qift {
 namespace {
+
+// Up to this many token rows the prefill route expands the codes inside the GEMM (one expansion per
+// 128-token tile); beyond it, expanding once into an int8 scratch and re-reading it wins.
+constexpr int kFusedMaxM = 768;
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
@@ -178,7 +183,7 @@ int launch_expand(const uint32_t* packed, int N, int K, int8_t* out, cudaStream_
 int run_prefill(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
                 void* Y, int y_bf16, int32_t* acc_debug, void* workspace, size_t workspace_bytes, cudaStream_t st) {
     if (K % 16 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;  // TMA row pitch must be a multiple of 16 bytes
-    const size_t need = qift_workspace_bytes(17 > M ? 17 : M, N, K, lv);
+    const size_t need = (static_cast<size_t>(N) * K + 1023) & ~static_cast<size_t>(1023);
     if (!workspace || workspace_bytes < need) return QIFT_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
     int8_t* wexp = static_cast<int8_t*>(workspace);
@@ -198,11 +203,50 @@ int run_prefill(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
     return narrow ? launch_gemm<128>(ma, mb, gp, st) : launch_gemm<256>(ma, mb, gp, st);
 }
 
+template <int LV, int BN>
+int launch_fused(const CUtensorMap& ma, const FusedParams& fp, cudaStream_t st) {
+    auto kernel = gemm_fused_kernel<LV, BN>;
+    const size_t smem = fused_smem_bytes<BN>();
+    cudaError_t e = allow_smem(kernel, smem);
+    if (e != cudaSuccess) return cuda_status(e);
+    const int tiles = ((fp.M + kGemmBM - 1) / kGemmBM) * ((fp.N + BN - 1) / BN);
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    return cuda_status(launch_pdl(kernel, dim3(grid), dim3(kFusedThreads), smem, st, ma, fp));
+}
+
+template <int LV>
+int dispatch_fused(const CUtensorMap& ma, const FusedParams& fp, cudaStream_t st) {
+    const int m_tiles = (fp.M + kGemmBM - 1) / kGemmBM;
+    const bool narrow = m_tiles * ((fp.N + 255) / 256) < sm_count();
+    return narrow ? launch_fused<LV, 128>(ma, fp, st) : launch_fused<LV, 256>(ma, fp, st);
+}
+
+// Prefill route with the expansion fused into the GEMM; workspace = per-token sums of q_a.
+int run_prefill_fused(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N,
+                      int K, void* Y, int y_bf16, int32_t* acc_debug, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    if (K % 16 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;  // TMA row pitch must be a multiple of 16 bytes
+    const size_t need = (static_cast<size_t>(M) * 4 + 1023) & ~static_cast<size_t>(1023);
+    if (!workspace || workspace_bytes < need) return QIFT_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
+    int* sumq = static_cast<int*>(workspace);
+    int rc = cuda_status(launch_pdl(rowsum_q_kernel, dim3((M + 7) / 8), dim3(256), 0, st, q_a, M, K, sumq));
+    if (rc != QIFT_OK) return rc;
+    CUtensorMap ma;
+    if (!make_i8_map(&ma, q_a, M, K, kGemmBM)) return QIFT_ERR_CUDA;
+    FusedParams fp{packed, s_n, s_a, sumq, Y, acc_debug, M, N, K, y_bf16};
+    switch (lv) {
+        case QIFT_LEVELS_MNZ: return dispatch_fused<QIFT_LEVELS_MNZ>(ma, fp, st);
+        case QIFT_LEVELS_POT: return dispatch_fused<QIFT_LEVELS_POT>(ma, fp, st);
+        case QIFT_LEVELS_SYM: return dispatch_fused<QIFT_LEVELS_SYM>(ma, fp, st);
+        default: return dispatch_fused<QIFT_LEVELS_INT4>(ma, fp, st);
+    }
+}
+
 int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
                 void* Y, int y_dtype, int32_t* acc_debug, void* workspace, size_t workspace_bytes, int route, void* stream) {
     if (!packed || !s_n || !q_a || !s_a || !Y || M <= 0 || N <= 0 || K <= 0 || !valid_levels(lv)) return QIFT_ERR_INVALID_ARG;
     if (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16) return QIFT_ERR_INVALID_ARG;
-    if (route < QIFT_ROUTE_AUTO || route > QIFT_ROUTE_PREFILL) return QIFT_ERR_INVALID_ARG;
+    if (route < QIFT_ROUTE_AUTO || route > QIFT_ROUTE_PREFILL_SCRATCH) return QIFT_ERR_INVALID_ARG;
     if (K % codes_per_word(lv) != 0 || K % 4 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(packed) || !aligned16(s_n) || !aligned16(q_a) || !aligned16(s_a) || !aligned16(Y) ||
         (acc_debug && !aligned16(acc_debug)))
@@ -211,7 +255,7 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
     const int y_bf16 = (y_dtype == QIFT_BF16);
     if (route == QIFT_ROUTE_AUTO) {
         if (M <= 16) route = decode_supports(lv, M, N, K) ? QIFT_ROUTE_DECODE : QIFT_ROUTE_GENERIC;
-        else route = (K % 16 == 0) ? QIFT_ROUTE_PREFILL : QIFT_ROUTE_GENERIC;
+        else route = (K % 16 != 0) ? QIFT_ROUTE_GENERIC : (M <= kFusedMaxM) ? QIFT_ROUTE_PREFILL : QIFT_ROUTE_PREFILL_SCRATCH;
     }
     if (route == QIFT_ROUTE_DECODE) {
         if (!decode_supports(lv, M, N, K)) return QIFT_ERR_UNSUPPORTED_SHAPE;
@@ -224,6 +268,8 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
         }
     }
     if (route == QIFT_ROUTE_PREFILL)
+        return run_prefill_fused(packed, s_n, lv, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, workspace, workspace_bytes, st);
+    if (route == QIFT_ROUTE_PREFILL_SCRATCH)
         return run_prefill(packed, s_n, lv, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, workspace, workspace_bytes, st);
     switch (lv) {
         case QIFT_LEVELS_MNZ: return launch_generic<QIFT_LEVELS_MNZ>(packed, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st);
@@ -259,11 +305,18 @@ size_t qift_packed_bytes(int N, int K, int levels) {
     return static_cast<size_t>(round_up16(N)) * packed_pitch(K, levels) * 4;
 }
 
-size_t qift_workspace_bytes(int M, int N, int K, int levels) {
+size_t qift_workspace_bytes_route(int M, int N, int K, int levels, int route) {
     if (M <= 0 || N <= 0 || K <= 0 || !valid_levels(levels)) return 0;
-    if (M <= 16) return 0;
-    const size_t b = static_cast<size_t>(N) * K;
+    if (route == QIFT_ROUTE_AUTO)
+        route = (M <= 16) ? QIFT_ROUTE_DECODE : (M <= kFusedMaxM) ? QIFT_ROUTE_PREFILL : QIFT_ROUTE_PREFILL_SCRATCH;
+    size_t b = 0;
+    if (route == QIFT_ROUTE_PREFILL) b = static_cast<size_t>(M) * 4;
+    if (route == QIFT_ROUTE_PREFILL_SCRATCH) b = static_cast<size_t>(N) * K;
     return (b + 1023) & ~static_cast<size_t>(1023);
+}
+
+size_t qift_workspace_bytes(int M, int N, int K, int levels) {
+    return qift_workspace_bytes_route(M, N, K, levels, QIFT_ROUTE_AUTO);
 }
 
 int qift_pack_weights(const float* W, int N, int K, int levels, int scale_mode, float* s_n, uint32_t* packed, void* stream) {
@@ -631,7 +684,7 @@ int qift_w2a4_linear_static(const uint32_t* packed, const float* s_n, int levels
     const cudaError_t e = static_scratch_address(&scratch);
     if (e != cudaSuccess) return cuda_status(e);
     return linear_impl(packed, s_n, levels, q_a, s_a, M, N, K, Y, y_dtype, acc_debug, scratch, kStaticScratchBytes,
-                       QIFT_ROUTE_PREFILL, stream);
+                       QIFT_ROUTE_PREFILL_SCRATCH, stream);
 }
 
 int qift_device_status(void* stream, uint32_t* detail) {

@@ -36,8 +36,12 @@ def test_sizes(L):
     assert qift.qift_packed_bytes(0, 16, qift.MNZ) == 0
     assert qift.qift_workspace_bytes(1, 4096, 4096, qift.MNZ) == 0
     assert qift.qift_workspace_bytes(16, 4096, 4096, qift.POT) == 0
-    assert qift.qift_workspace_bytes(2048, 4096, 4096, qift.MNZ) == 4096 * 4096
-    assert qift.qift_workspace_bytes(17, 3, 16, qift.SYM) == 1024  # rounded up to 1 KiB
+    assert qift.qift_workspace_bytes(512, 4096, 4096, qift.MNZ) == 512 * 4            # per-token sums only
+    assert qift.qift_workspace_bytes(2048, 4096, 4096, qift.MNZ) == 4096 * 4096       # int8 scratch
+    assert qift.qift_workspace_bytes(17, 3, 16, qift.SYM) == 1024                      # rounded up to 1 KiB
+    assert qift.qift_workspace_bytes(2048, 4096, 4096, qift.MNZ, qift.ROUTE_PREFILL_SCRATCH) == 4096 * 4096
+    assert qift.qift_workspace_bytes(8, 4096, 4096, qift.MNZ, qift.ROUTE_PREFILL_SCRATCH) == 4096 * 4096
+    assert qift.qift_workspace_bytes(8, 4096, 4096, qift.MNZ, qift.ROUTE_GENERIC) == 0
     # the L = 16 mixed stack stores exactly 3 bits per weight
     import synth
     w4 = sum(qift.qift_packed_bytes(n, k, qift.INT4) for _, n, k in synth.LLAMA2_7B)

@@ -181,13 +181,15 @@ def test_decode_extreme_values(name):
 
 
 @pytest.mark.parametrize("name", list(LEVELS))
-@pytest.mark.parametrize("M,N,K", [(128, 256, 512), (200, 300, 1024), (17, 72, 256), (512, 1024, 384), (130, 520, 4096)])
-def test_prefill_route(name, M, N, K):
+@pytest.mark.parametrize("route", [qift.ROUTE_PREFILL, qift.ROUTE_PREFILL_SCRATCH])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 512), (200, 300, 1024), (17, 72, 256), (512, 1024, 384), (130, 520, 4096),
+                                   (300, 2000, 2320), (1, 40, 48)])
+def test_prefill_route(name, route, M, N, K):
     lv = LEVELS[name][0]
     p_ref, s_n, codes, q_a, s_a = make_problem(lv, M, N, K, seed=80)
     for bf16 in (True, False):
         y_ref, acc_ref = oracle.linear(codes, lv, s_n, q_a, s_a, bf16=bf16)
-        y, acc = run_route(p_ref, s_n, lv, q_a, s_a, qift.ROUTE_PREFILL, bf16)
+        y, acc = run_route(p_ref, s_n, lv, q_a, s_a, route, bf16)
         check_outputs(y, acc, y_ref, acc_ref, bf16)
 
 

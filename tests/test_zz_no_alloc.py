@@ -39,8 +39,7 @@ def test_static_scratch_matches_the_workspace_entry_point_twice_in_a_row():
     for rounds in range(2):
         for lv, M, N, K, seed, dt in cases:
             packed, s_n, q_a, s_a = problem(lv, M, N, K, seed)
-            want, want_acc = qift.qift_linear_route(packed, s_n, lv, q_a, s_a, qift.ROUTE_PREFILL, out_dtype=dt,
-                                                    want_acc=True)
+            want, want_acc = qift.qift_w2a4_linear(packed, s_n, lv, q_a, s_a, out_dtype=dt, want_acc=True)
             out = torch.empty((M, N), dtype=dt, device="cuda")
             acc = torch.empty((M, N), dtype=torch.int32, device="cuda")
             torch.cuda.synchronize()

@@ -36,6 +36,10 @@ import synth  # noqa: E402
 
 CLIP = 0.9
 N_LAYERS = 32
+# dram__bytes_read.sum + dram__bytes_write.sum of one linear_grouped_kernel launch in the ncu capture of
+# the 4-layer case (profiles/linear_grouped_kernel_llama2_m1_4layers.md): 203 236 864 + 4 653 056 bytes
+# for 203 877 488 algorithmic bytes.  Every packed word is read once, so traffic scales with the layers.
+NCU_TRAFFIC_BYTES_4_LAYERS = 203_236_864 + 4_653_056
 
 
 # ------------------------------------------------------------------------------------------------
@@ -340,7 +344,9 @@ def run_gpu(args):
         "tokens_per_s": round(world * M / (step_ms * 1e-3), 1),
         "pct_of_8TBs": round(100 * value / world / 8000.0, 2),
         "roofline": {"bound": "hbm", "kernel": "linear_grouped_kernel", "achieved": round(achieved, 1), "peak": pk["hbm_gbs"],
-                     "unit": "GB/s", "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": None,
+                     "unit": "GB/s", "frac": round(achieved / pk["hbm_gbs"], 4),
+                     "traffic": round(NCU_TRAFFIC_BYTES_4_LAYERS * args.layers / 4),
+                     "traffic_source": "ncu capture of the 4-layer case, scaled by layers",
                      "peak_source": pk["source"], "avg_launch_us": round(launch_us, 3),
                      "algorithmic_bytes_per_launch": bytes_product},
         "per_call": {"what": "same step as 224 x (qift_quantize_act + qift_w2a4_linear) in one CUDA graph with "

@@ -173,11 +173,12 @@ int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& 
 
 template <int LV>
 int launch_expand(const uint32_t* packed, int N, int K, int8_t* out, cudaStream_t st) {
-    const long long words = static_cast<long long>(N) * (K / codes_per_word(LV));
-    long long blocks = (words + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
-    return cuda_status(launch_pdl(expand_levels_kernel<LV>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, st, packed, words,
-                                  K / codes_per_word(LV), out));
+    const int row_blocks = (N + 15) / 16;
+    const int nchunks = (packed_pitch(K, LV) + kChunkWords - 1) / kChunkWords;
+    int split = (8 * sm_count() + row_blocks - 1) / row_blocks;  // enough CTAs to fill the machine a few times over
+    if (split > nchunks) split = nchunks;
+    if (split < 1) split = 1;
+    return cuda_status(launch_pdl(expand_levels_kernel<LV>, dim3(row_blocks, split), dim3(256), 0, st, packed, N, K, out));
 }
 
 int run_prefill(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,

@@ -19,7 +19,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CU
 MNZ, POT, SYM, INT4 = 0, 1, 2, 3
 SCALE_GIVEN, SCALE_ABSMAX, SCALE_MSE = 0, 1, 2
 F32, BF16 = 0, 1
-ROUTE_AUTO, ROUTE_GENERIC, ROUTE_DECODE, ROUTE_PREFILL, ROUTE_PREFILL_SCRATCH = 0, 1, 2, 3, 4
+ROUTE_AUTO, ROUTE_GENERIC, ROUTE_DECODE, ROUTE_PREFILL, ROUTE_PREFILL_SCRATCH, ROUTE_PREFILL_PAIR = 0, 1, 2, 3, 4, 5
 
 EXPORTS = [
     "qift_status_string", "qift_packed_bytes", "qift_workspace_bytes", "qift_workspace_bytes_route", "qift_pack_weights",

@@ -84,22 +84,32 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint = 0x989680u) {
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity), "r"(hint)  // time hint: the hardware may park the thread while it waits
+        : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)  // time hint: the hardware may park the thread while it waits
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after 2^20 polls (each poll may itself be suspended by the hardware for up
-// to its time hint), records the site and returns false.  Callers skip their remaining work on false.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int site, uint32_t hint = 0x989680u) {
-    for (uint32_t i = 0; i < (1u << 20); ++i) {
-        if (mbar_try_wait(bar, parity, hint)) return true;
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: polls (each poll may be parked by the hardware for up to its time hint) until the
+// phase completes or two seconds of wall time have passed; then records the site and returns false.
+// Callers skip their remaining work on false.
+constexpr uint64_t kWaitLimitNs = 2000000000ull;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int site) {
+    if (mbar_try_wait(bar, parity, 100000u)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (;;) {
+        if (mbar_try_wait(bar, parity, 1000000u)) return true;
+        if (global_timer_ns() - t0 > kWaitLimitNs) break;
     }
     report_timeout(site);
     return false;

@@ -23,51 +23,30 @@ namespace qift {
 // ------------------------------------------------------------------------------------------------
 // expansion: packed codes -> int8 levels, K contiguous
 // ------------------------------------------------------------------------------------------------
-// Walks the packed buffer in storage order: a thread takes one 16-byte group (four consecutive words
-// of one row = 64 or 32 codes), so a warp reads 512 contiguous bytes and writes, per row, 256 (128)
-// contiguous bytes of levels.  grid.x = row blocks of 16 channels, grid.y splits the k-tiles.
 template <int LV>
 __global__ void __launch_bounds__(256)
-expand_levels_kernel(const uint32_t* __restrict__ packed, int N, int K, int8_t* __restrict__ out) {
+expand_levels_kernel(const uint32_t* __restrict__ packed, long long total_words, int words_per_row,
+                     int8_t* __restrict__ out) {
     constexpr int PER = codes_per_word(LV);
-    constexpr int BITS = 32 / PER;
     pdl_launch_dependents();
     pdl_wait();
-    const int words_per_row = K / PER;
     const int pitch = round_up16(words_per_row);
-    const int nchunks = (pitch + kChunkWords - 1) / kChunkWords;
-    const int rb = blockIdx.x;
-    const uint4* tile_row = reinterpret_cast<const uint4*>(packed + static_cast<size_t>(rb) * 16 * pitch);
-    for (int c = blockIdx.y; c < nchunks; c += gridDim.y) {
-        const int cw = min(kChunkWords, pitch - c * kChunkWords);  // words per row in this tile (multiple of 16)
-        const int groups = 4 * cw;                                 // 16 rows * cw / 4
-        const uint4* tile = tile_row + static_cast<size_t>(c) * (kTileRows * kChunkWords / 4);
-        for (int gi = threadIdx.x; gi < groups; gi += blockDim.x) {
-            const int slice = gi >> 6, half = (gi >> 5) & 1, g = (gi >> 2) & 7, quad = gi & 3;
-            const int n = rb * 16 + half * 8 + g;
-            const int j = c * kChunkWords + slice * 16 + quad * 4;  // first word of the group
-            if (n >= N || j >= words_per_row) continue;
-            const uint4 v = tile[gi];
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-            int8_t* dst = out + static_cast<size_t>(n) * K + static_cast<size_t>(j) * PER;
+    for (long long j = blockIdx.x * (long long)blockDim.x + threadIdx.x; j < total_words;
+         j += (long long)gridDim.x * blockDim.x) {
+        const uint32_t w = packed[packed_word_address(static_cast<int>(j / words_per_row), static_cast<int>(j % words_per_row), pitch)];
+        uint32_t o[PER / 4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                if (j + e >= words_per_row) break;
-                uint32_t o[PER / 4];
+        for (int t = 0; t < PER / 4; ++t) {
+            uint32_t r = 0;
 #pragma unroll
-                for (int t = 0; t < PER / 4; ++t) {
-                    uint32_t r = 0;
-#pragma unroll
-                    for (int b = 0; b < 4; ++b) {
-                        const int code = (w[e] >> (8 * b + BITS * t)) & ((1u << BITS) - 1u);
-                        r |= (static_cast<uint32_t>(level_from_code<LV>(code)) & 0xffu) << (8 * b);
-                    }
-                    o[t] = r;
-                }
-                if constexpr (PER == 16) reinterpret_cast<uint4*>(dst)[e] = make_uint4(o[0], o[1], o[2], o[3]);
-                else reinterpret_cast<uint2*>(dst)[e] = make_uint2(o[0], o[1]);
+            for (int b = 0; b < 4; ++b) {
+                const int code = (w >> (8 * b + (32 / PER) * t)) & ((1u << (32 / PER)) - 1u);
+                r |= (static_cast<uint32_t>(level_from_code<LV>(code)) & 0xffu) << (8 * b);
             }
+            o[t] = r;
         }
+        if constexpr (PER == 16) reinterpret_cast<uint4*>(out)[j] = make_uint4(o[0], o[1], o[2], o[3]);
+        else reinterpret_cast<uint2*>(out)[j] = make_uint2(o[0], o[1]);
     }
 }
 

@@ -10,6 +10,7 @@
 #include "grouped.cuh"
 #include "pack.cuh"
 #include "prefill.cuh"
+#include "prefill_2cta.cuh"
 #include "prefill_fused.cuh"
 #include "rotate_quant.cuh"
 
@@ -43,6 +44,26 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 
 // Opt a kernel in to more than 48 KiB of dynamic shared memory; remembered per kernel so that the
 // steady state (and any stream capture after a warm-up call) makes no attribute call.
+// The same for a kernel that runs as clusters of two CTAs along x.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl_pairs(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 template <typename K>
 cudaError_t allow_smem(K kernel, size_t bytes) {
     if (bytes <= 32 * 1024) return cudaSuccess;  // static shared memory counts against the 48 KiB default too
@@ -173,16 +194,28 @@ int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& 
 
 template <int LV>
 int launch_expand(const uint32_t* packed, int N, int K, int8_t* out, cudaStream_t st) {
-    const int row_blocks = (N + 15) / 16;
-    const int nchunks = (packed_pitch(K, LV) + kChunkWords - 1) / kChunkWords;
-    int split = (8 * sm_count() + row_blocks - 1) / row_blocks;  // enough CTAs to fill the machine a few times over
-    if (split > nchunks) split = nchunks;
-    if (split < 1) split = 1;
-    return cuda_status(launch_pdl(expand_levels_kernel<LV>, dim3(row_blocks, split), dim3(256), 0, st, packed, N, K, out));
+    const long long words = static_cast<long long>(N) * (K / codes_per_word(LV));
+    long long blocks = (words + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    return cuda_status(launch_pdl(expand_levels_kernel<LV>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, st, packed, words,
+                                  K / codes_per_word(LV), out));
+}
+
+template <int BN>
+int launch_gemm_pairs(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& gp, cudaStream_t st) {
+    auto kernel = gemm_i8_pair_kernel<BN>;
+    const size_t smem = pair_smem_bytes<BN>();
+    cudaError_t e = allow_smem(kernel, smem);
+    if (e != cudaSuccess) return cuda_status(e);
+    const int tiles = ((gp.M + 2 * kGemmBM - 1) / (2 * kGemmBM)) * ((gp.N + BN - 1) / BN);
+    int pairs = sm_count() / 2;
+    if (pairs > tiles) pairs = tiles;
+    return cuda_status(launch_pdl_pairs(kernel, dim3(2 * pairs), dim3(kPairThreads), smem, st, ma, mb, gp));
 }
 
 int run_prefill(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
-                void* Y, int y_bf16, int32_t* acc_debug, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+                void* Y, int y_bf16, int32_t* acc_debug, void* workspace, size_t workspace_bytes, cudaStream_t st,
+                bool pairs = false) {
     if (K % 16 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;  // TMA row pitch must be a multiple of 16 bytes
     const size_t need = (static_cast<size_t>(N) * K + 1023) & ~static_cast<size_t>(1023);
     if (!workspace || workspace_bytes < need) return QIFT_ERR_WORKSPACE;
@@ -199,8 +232,12 @@ int run_prefill(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
     const int m_tiles = (M + kGemmBM - 1) / kGemmBM;
     const bool narrow = m_tiles * ((N + 255) / 256) < sm_count();
     CUtensorMap ma, mb;
-    if (!make_i8_map(&ma, q_a, M, K, kGemmBM) || !make_i8_map(&mb, wexp, N, K, narrow ? 128 : 256)) return QIFT_ERR_CUDA;
     GemmParams gp{s_n, s_a, Y, acc_debug, M, N, K, y_bf16};
+    if (pairs) {  // each CTA of a pair loads its own 128 tokens and half of the tile's channels
+        if (!make_i8_map(&ma, q_a, M, K, kGemmBM) || !make_i8_map(&mb, wexp, N, K, narrow ? 64 : 128)) return QIFT_ERR_CUDA;
+        return narrow ? launch_gemm_pairs<128>(ma, mb, gp, st) : launch_gemm_pairs<256>(ma, mb, gp, st);
+    }
+    if (!make_i8_map(&ma, q_a, M, K, kGemmBM) || !make_i8_map(&mb, wexp, N, K, narrow ? 128 : 256)) return QIFT_ERR_CUDA;
     return narrow ? launch_gemm<128>(ma, mb, gp, st) : launch_gemm<256>(ma, mb, gp, st);
 }
 
@@ -247,7 +284,7 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
                 void* Y, int y_dtype, int32_t* acc_debug, void* workspace, size_t workspace_bytes, int route, void* stream) {
     if (!packed || !s_n || !q_a || !s_a || !Y || M <= 0 || N <= 0 || K <= 0 || !valid_levels(lv)) return QIFT_ERR_INVALID_ARG;
     if (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16) return QIFT_ERR_INVALID_ARG;
-    if (route < QIFT_ROUTE_AUTO || route > QIFT_ROUTE_PREFILL_SCRATCH) return QIFT_ERR_INVALID_ARG;
+    if (route < QIFT_ROUTE_AUTO || route > QIFT_ROUTE_PREFILL_PAIR) return QIFT_ERR_INVALID_ARG;
     if (K % codes_per_word(lv) != 0 || K % 4 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(packed) || !aligned16(s_n) || !aligned16(q_a) || !aligned16(s_a) || !aligned16(Y) ||
         (acc_debug && !aligned16(acc_debug)))
@@ -256,7 +293,7 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
     const int y_bf16 = (y_dtype == QIFT_BF16);
     if (route == QIFT_ROUTE_AUTO) {
         if (M <= 16) route = decode_supports(lv, M, N, K) ? QIFT_ROUTE_DECODE : QIFT_ROUTE_GENERIC;
-        else route = (K % 16 != 0) ? QIFT_ROUTE_GENERIC : (M <= kFusedMaxM) ? QIFT_ROUTE_PREFILL : QIFT_ROUTE_PREFILL_SCRATCH;
+        else route = (K % 16 != 0) ? QIFT_ROUTE_GENERIC : (M <= kFusedMaxM) ? QIFT_ROUTE_PREFILL : QIFT_ROUTE_PREFILL_PAIR;
     }
     if (route == QIFT_ROUTE_DECODE) {
         if (!decode_supports(lv, M, N, K)) return QIFT_ERR_UNSUPPORTED_SHAPE;
@@ -270,8 +307,9 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
     }
     if (route == QIFT_ROUTE_PREFILL)
         return run_prefill_fused(packed, s_n, lv, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, workspace, workspace_bytes, st);
-    if (route == QIFT_ROUTE_PREFILL_SCRATCH)
-        return run_prefill(packed, s_n, lv, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, workspace, workspace_bytes, st);
+    if (route == QIFT_ROUTE_PREFILL_SCRATCH || route == QIFT_ROUTE_PREFILL_PAIR)
+        return run_prefill(packed, s_n, lv, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, workspace, workspace_bytes, st,
+                           route == QIFT_ROUTE_PREFILL_PAIR);
     switch (lv) {
         case QIFT_LEVELS_MNZ: return launch_generic<QIFT_LEVELS_MNZ>(packed, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st);
         case QIFT_LEVELS_POT: return launch_generic<QIFT_LEVELS_POT>(packed, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st);
@@ -309,10 +347,10 @@ size_t qift_packed_bytes(int N, int K, int levels) {
 size_t qift_workspace_bytes_route(int M, int N, int K, int levels, int route) {
     if (M <= 0 || N <= 0 || K <= 0 || !valid_levels(levels)) return 0;
     if (route == QIFT_ROUTE_AUTO)
-        route = (M <= 16) ? QIFT_ROUTE_DECODE : (M <= kFusedMaxM) ? QIFT_ROUTE_PREFILL : QIFT_ROUTE_PREFILL_SCRATCH;
+        route = (M <= 16) ? QIFT_ROUTE_DECODE : (M <= kFusedMaxM) ? QIFT_ROUTE_PREFILL : QIFT_ROUTE_PREFILL_PAIR;
     size_t b = 0;
     if (route == QIFT_ROUTE_PREFILL) b = static_cast<size_t>(M) * 4;
-    if (route == QIFT_ROUTE_PREFILL_SCRATCH) b = static_cast<size_t>(N) * K;
+    if (route == QIFT_ROUTE_PREFILL_SCRATCH || route == QIFT_ROUTE_PREFILL_PAIR) b = static_cast<size_t>(N) * K;
     return (b + 1023) & ~static_cast<size_t>(1023);
 }
 

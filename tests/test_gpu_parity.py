@@ -181,7 +181,7 @@ def test_decode_extreme_values(name):
 
 
 @pytest.mark.parametrize("name", list(LEVELS))
-@pytest.mark.parametrize("route", [qift.ROUTE_PREFILL, qift.ROUTE_PREFILL_SCRATCH])
+@pytest.mark.parametrize("route", [qift.ROUTE_PREFILL, qift.ROUTE_PREFILL_SCRATCH, qift.ROUTE_PREFILL_PAIR])
 @pytest.mark.parametrize("M,N,K", [(128, 256, 512), (200, 300, 1024), (17, 72, 256), (512, 1024, 384), (130, 520, 4096),
                                    (300, 2000, 2320), (1, 40, 48)])
 def test_prefill_route(name, route, M, N, K):

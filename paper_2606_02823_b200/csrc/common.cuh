@@ -105,11 +105,12 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // Callers skip their remaining work on false.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int site) {
-    if (mbar_try_wait(bar, parity, 100000u)) return true;
-    const uint64_t t0 = global_timer_ns();
+    uint64_t t0 = 0;
     for (;;) {
         if (mbar_try_wait(bar, parity, 1000000u)) return true;
-        if (global_timer_ns() - t0 > kWaitLimitNs) break;
+        const uint64_t t = global_timer_ns();
+        if (t0 == 0) t0 = t;
+        else if (t - t0 > kWaitLimitNs) break;
     }
     report_timeout(site);
     return false;
@@ -138,22 +139,6 @@ __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, 
         "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-// The same with the A operand formed inside the instruction sequence: a_i = (w_i & mask) ^ flip.
-// Keeping the logic ops and the mma in one block lets the assembler write the masked words straight
-// into the operand registers.
-__device__ __forceinline__ void mma_u8s8_masked(int (&d)[4], uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3,
-                                                uint32_t mask, uint32_t flip, uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "{\n\t.reg .b32 a0, a1, a2, a3;\n\t"
-        "lop3.b32 a0, %4, %8, %9, 0x6a;\n\t"
-        "lop3.b32 a1, %5, %8, %9, 0x6a;\n\t"
-        "lop3.b32 a2, %6, %8, %9, 0x6a;\n\t"
-        "lop3.b32 a3, %7, %8, %9, 0x6a;\n\t"
-        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {a0,a1,a2,a3}, {%10,%11}, {%0,%1,%2,%3};\n\t}"
-        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
-        : "r"(w0), "r"(w1), "r"(w2), "r"(w3), "r"(mask), "r"(flip), "r"(b0), "r"(b1));
 }
 
 __device__ __forceinline__ uint16_t f32_to_bf16_bits(float f) {

@@ -195,12 +195,19 @@ struct GroupParams {
     int count;                        // problems in the slice (<= kGroupSlice)
     int item_first, item_end;         // work items of the slice
     int M, y_bf16, stages;
-    int dbg;
 };
+
+// CTAs per SM the kernel is compiled and launched for.  Nine warps per CTA and registers handed out
+// to four warps at a time leave room for two CTAs only up to 96 registers per thread; the PoT
+// variants (four accumulator sets) would spill at that size and run one CTA per SM instead.
+template <int LV>
+constexpr int grouped_ctas_per_sm() {
+    return (LV == QIFT_LEVELS_POT) ? 1 : 2;
+}
 
 // M1: the single-token specialisation (only accumulator column 0 is live).
 template <int LV, int NT, int RT, bool M1>
-__global__ void __launch_bounds__(kDecThreads)
+__global__ void __launch_bounds__(kDecThreads, grouped_ctas_per_sm<LV>())
 linear_grouped_kernel(const GroupParams gp) {
     using T = DecodeTraits<LV>;
     constexpr int ROWS = 16 * RT;
@@ -328,7 +335,7 @@ linear_grouped_kernel(const GroupParams gp) {
             const int cw = cur.chunk_words();
             unsigned char* wst = ring + s * stage_bytes;
             unsigned char* qst = wst + RT * kTileBytes;
-            if (16 * warp < cw && !(gp.dbg & 1)) {
+            if (16 * warp < cw) {
                 uint32_t qb[NT][4 * T::NPL];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
@@ -364,7 +371,6 @@ linear_grouped_kernel(const GroupParams gp) {
         if (!ok) break;
 
         // item epilogue: one barrier; the other reduction buffer belongs to the next item
-        if (gp.dbg & 2) continue;
 #pragma unroll
         for (int rt = 0; rt < RT; ++rt)
 #pragma unroll

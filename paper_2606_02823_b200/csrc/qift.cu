@@ -587,25 +587,21 @@ int launch_grouped(const GroupHeader* h, const GroupProblemDev* host, const Grou
                    cudaStream_t st) {
     auto kernel = linear_grouped_kernel<LV, NT, RT, M1>;
     const size_t stage = decode_stage_bytes(LV, RT, h->M) + 16;
-    const char* e_stages = std::getenv("QIFT_G_STAGES");
     for (int first = 0; first < h->count; first += kGroupSlice) {  // the problem table of a launch lives in shared memory
         const int count = (h->count - first < kGroupSlice) ? h->count - first : kGroupSlice;
         const int item_first = host[first].item_begin;
         const int item_end = (first + count < h->count) ? host[first + count].item_begin : h->total_items;
         const size_t fixed = grouped_fixed_smem(LV, RT, h->M, count);
-        const char* e_cps = std::getenv("QIFT_G_CPS");
-        const int cps = e_cps ? std::atoi(e_cps) : 2;
-        int stages = static_cast<int>(((cps == 3 ? 75 : cps == 4 ? 56 : 113) * 1024 - fixed) / stage);  // CTAs per SM
+        constexpr int cps = grouped_ctas_per_sm<LV>();  // each CTA gets its share of the SM's shared memory
+        int stages = static_cast<int>(((cps == 2 ? 113 : 226) * 1024 - fixed) / stage);
         if (stages < 2) stages = 2;
         if (stages > 12) stages = 12;
-        if (e_stages) stages = std::atoi(e_stages);
         const size_t smem = grouped_smem_bytes(LV, RT, h->M, stages, count);
         cudaError_t e = allow_smem(kernel, smem);
         if (e != cudaSuccess) return cuda_status(e);
         int grid = cps * sm_count();
         if (grid > item_end - item_first) grid = item_end - item_first;
-        const char* e_dbg = std::getenv("QIFT_G_DBG");
-        GroupParams gp{dev + first, sumq, first, count, item_first, item_end, h->M, h->y_bf16, stages, e_dbg ? std::atoi(e_dbg) : 0};
+        GroupParams gp{dev + first, sumq, first, count, item_first, item_end, h->M, h->y_bf16, stages};
         const int rc = cuda_status(launch_pdl(kernel, dim3(grid), dim3(kDecThreads), smem, st, gp));
         if (rc != QIFT_OK) return rc;
     }

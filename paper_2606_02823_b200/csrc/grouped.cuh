@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(kRowThreads)
 quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* __restrict__ sumq, int M, float clip,
                             int int4_weights) {
     extern __shared__ __align__(16) float row[];
-    __shared__ float red[kRowThreads / 32];
+    __shared__ float red[kRowThreads / 32 + 2];
     __shared__ int redi[kRowThreads / 32];
     pdl_launch_dependents();
     pdl_wait();
@@ -66,43 +66,10 @@ quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* _
     const GroupProblemDev P = problems[p];
     const size_t m = blockIdx.x % M;
     const int K = P.K, B = P.had_block;
-    load_and_transform<BF16_IN>(P.X, m, K, B, row);
-    const int groups = K / 16;
-    float amax = 0.0f;
-    for (int q = threadIdx.x; q < groups; q += blockDim.x) {
-        const float4* src = reinterpret_cast<const float4*>(row) + 4 * q;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float4 f = src[i];
-            amax = fmaxf(amax, fmaxf(fmaxf(fabsf(f.x), fabsf(f.y)), fmaxf(fabsf(f.z), fabsf(f.w))));
-        }
-    }
-    amax = block_max(amax, red);
-    float s_u = 1.0f;
-    if (amax != 0.0f) s_u = __fdiv_rn(__fmul_rn(amax, clip), 7.0f);
-    if (threadIdx.x == 0) P.s_a[m] = (B > 1) ? __fmul_rn(s_u, P.inv_sqrt_b) : s_u;
-    int total = 0;
-    for (int q = threadIdx.x; q < groups; q += blockDim.x) {
-        const float4* src = reinterpret_cast<const float4*>(row) + 4 * q;
-        uint32_t out[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float4 f = src[i];
-            const float e[4] = {f.x, f.y, f.z, f.w};
-            uint32_t w = 0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                int v = __float2int_rn(__fdiv_rn(e[j], s_u));
-                v = max(-8, min(7, v));
-                total += v;
-                // i = 32-bit word of this 16-byte group = code plane (two-bit: i; INT4: i & 1)
-                const int mult = int4_weights ? ((i & 1) ? 1 : 16) : ((i & 1) ? 1 : 4);
-                w |= (static_cast<uint32_t>(v * mult) & 0xffu) << (8 * j);
-            }
-            out[i] = w;
-        }
-        reinterpret_cast<uint4*>(P.q_a + m * K)[q] = make_uint4(out[0], out[1], out[2], out[3]);
-    }
+    const RowScale sc = block_row_scale(load_and_transform<BF16_IN>(P.X, m, K, B, row), clip, red);
+    if (threadIdx.x == 0) P.s_a[m] = (B > 1) ? __fmul_rn(sc.s_u, P.inv_sqrt_b) : sc.s_u;
+    // 32-bit word i of a 16-byte group = code plane (two-bit: i; INT4: i & 1); even planes are prescaled
+    int total = quantize_row<true>(row, K, sc, P.q_a + m * K, int4_weights ? 16.0f : 4.0f, 1.0f);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
     if ((threadIdx.x & 31) == 0) redi[threadIdx.x >> 5] = total;

@@ -364,7 +364,7 @@ int qift_pack_weights(const float* W, int N, int K, int levels, int scale_mode, 
     if (K % 16 != 0 || K > kMaxRowK) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(W) || !aligned16(s_n) || !aligned16(packed)) return QIFT_ERR_ALIGNMENT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t smem = static_cast<size_t>(K) * 4;
+    const size_t smem = padded_row_bytes(K);
 #define QIFT_PACK_CASE(LV)                                                                                   \
     case LV: {                                                                                               \
         cudaError_t e = allow_smem(pack_weights_kernel<LV>, smem);                                           \
@@ -398,10 +398,10 @@ int qift_rotate(const float* X, int M, int K, int had_block, float* Y, void* str
     const int rc = check_rotation_shape(K, had_block, false);
     if (rc != QIFT_OK) return rc;
     if (!aligned16(X) || !aligned16(Y)) return QIFT_ERR_ALIGNMENT;
-    const size_t smem = static_cast<size_t>(K) * 4;
+    const size_t smem = padded_row_bytes(K);
     cudaError_t e = allow_smem(rotate_rows_kernel, smem);
     if (e != cudaSuccess) return cuda_status(e);
-    return cuda_status(launch_pdl(rotate_rows_kernel, dim3(M), dim3(kRowThreads), smem, static_cast<cudaStream_t>(stream), X,
+    return cuda_status(launch_pdl(rotate_rows_kernel, dim3(M), dim3(row_threads(K)), smem, static_cast<cudaStream_t>(stream), X,
                                   K, had_block, inv_sqrt_block(had_block), Y));
 }
 
@@ -413,18 +413,18 @@ int qift_quantize_act(const void* X, int x_dtype, int M, int K, int had_block, f
     const int rc = check_rotation_shape(K, had_block, true);
     if (rc != QIFT_OK) return rc;
     if (!aligned16(X) || !aligned16(q_a) || !aligned16(s_a)) return QIFT_ERR_ALIGNMENT;
-    const size_t smem = static_cast<size_t>(K) * 4;
+    const size_t smem = padded_row_bytes(K);
     const float r = had_block > 1 ? inv_sqrt_block(had_block) : 1.0f;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (x_dtype == QIFT_BF16) {
         cudaError_t e = allow_smem(quantize_act_kernel<true>, smem);
         if (e != cudaSuccess) return cuda_status(e);
-        return cuda_status(launch_pdl(quantize_act_kernel<true>, dim3(M), dim3(kRowThreads), smem, st, X, K, had_block,
+        return cuda_status(launch_pdl(quantize_act_kernel<true>, dim3(M), dim3(row_threads(K)), smem, st, X, K, had_block,
                                       clip_ratio, r, q_a, s_a));
     }
     cudaError_t e = allow_smem(quantize_act_kernel<false>, smem);
     if (e != cudaSuccess) return cuda_status(e);
-    return cuda_status(launch_pdl(quantize_act_kernel<false>, dim3(M), dim3(kRowThreads), smem, st, X, K, had_block,
+    return cuda_status(launch_pdl(quantize_act_kernel<false>, dim3(M), dim3(row_threads(K)), smem, st, X, K, had_block,
                                   clip_ratio, r, q_a, s_a));
 }
 
@@ -623,7 +623,7 @@ int qift_group_quantize_act(const void* plan_host, const void* plan_dev, void* s
     const GroupHeader* h = plan_header(plan_host, plan_dev);
     if (!h) return QIFT_ERR_INVALID_ARG;
     const GroupProblemDev* dev = reinterpret_cast<const GroupProblemDev*>(static_cast<const GroupHeader*>(plan_dev) + 1);
-    const size_t smem = static_cast<size_t>(h->max_k) * 4;
+    const size_t smem = padded_row_bytes(h->max_k);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int* sumq = const_cast<int*>(plan_sumq(plan_dev, h->count));
     const dim3 grid(static_cast<unsigned>(h->count) * h->M);

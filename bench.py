@@ -362,6 +362,7 @@ def run_gpu(args):
         "clocks": clocks,
     }
     if rank == 0 and world == 1 and not args.no_prefill:
+        out["mixed_stack"] = run_mixed_stack(torch, qift, L, device, gen, args)
         out["prefill"] = run_prefill(torch, qift, L, device, gen, pk)
     if rank == 0 and world == 1 and not args.no_cpu:
         out["cpu_baseline"] = cpu_baseline(budget_s=12.0)
@@ -369,6 +370,67 @@ def run_gpu(args):
         print(json.dumps(out))
     if dist:
         dist.destroy_process_group()
+
+
+def run_mixed_stack(torch, qift, L, device, gen, args):
+    """Config 5: layer-wise mixed precision on LLaMA-2-7B shapes at M = 1: layers 0..15 INT4 weights (W4A4),
+    layers 16..31 MNZ (W2A4), 3 bits per weight on average.  Two grouped plans (a plan holds one level set):
+    four launches per token-step.  Modules run on their own staged inputs, as in the headline."""
+    n4 = args.layers // 2
+    n2 = args.layers - n4
+    vp = ctypes.c_void_p
+    plans, algo = [], 0
+    for lv, n in ((qift.INT4, n4), (qift.MNZ, n2)):
+        mods = build_stack(torch, qift, synth.LLAMA2_7B, n, 1, lambda l, lv=lv: lv, 5000 + lv, torch.float32, torch.float32,
+                           device, gen)
+        plans.append((qift.qift_group_plan([(m.x, m.packed, m.s_n, m.B) for m in mods], lv, CLIP), mods))
+        algo += sum(product_bytes(1, m.N, m.K, m.bits) + quant_bytes(1, m.K) for m in mods)
+    st = vp(torch.cuda.current_stream().cuda_stream)
+
+    def step():
+        for plan, _ in plans:
+            rc = L.qift_group_forward(vp(plan.host.data_ptr()), vp(plan.dev.data_ptr()), st)
+            assert rc == 0, rc
+
+    for _ in range(5):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    steps = max(3, min(args.steps, 100))
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return {"workload": f"config 5: {n4} W4A4 layers + {n2} W2A4 (MNZ) layers, LLaMA-2-7B shapes, M=1, grouped API (4 launches per step)",
+            "ms_per_step": round(ms, 5), "tokens_per_s": round(1.0 / (ms * 1e-3), 1),
+            "value": round(algo / (ms * 1e-3) / 1e9, 2), "unit": "GB/s", "algorithmic_bytes_per_step": algo,
+            "pct_of_8TBs": round(100 * algo / (ms * 1e-3) / 8e12, 2)}
+
+
+def int8_library_point(torch, M, shapes, device):
+    """cuBLASLt int8 GEMM (torch._int_mm) on the same shapes: a library reference for the tensor-core rate."""
+    try:
+        ops, ms_total = 0.0, 0.0
+        for (_, N, K) in shapes:
+            a = torch.randint(-8, 8, (M, K), dtype=torch.int8, device=device)
+            b = torch.randint(-3, 4, (N, K), dtype=torch.int8, device=device).t()
+            for _ in range(3):
+                torch._int_mm(a, b)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                torch._int_mm(a, b)
+            e1.record()
+            torch.cuda.synchronize()
+            ms_total += e0.elapsed_time(e1) / 10
+            ops += 2.0 * M * N * K
+        return {"api": "torch._int_mm (int8 x int8 -> int32, no scales, no decode)", "ms_per_layer": round(ms_total, 4),
+                "tops": round(ops / (ms_total * 1e-3) / 1e12, 1)}
+    except Exception as e:  # noqa: BLE001
+        return {"api": "torch._int_mm", "unavailable": str(e)[:120]}
 
 
 def run_prefill(torch, qift, L, device, gen, pk):
@@ -411,10 +473,11 @@ def run_prefill(torch, qift, L, device, gen, pk):
     int8_peak = 2.0 * pk["bf16_tflops"]    # dense int8 is nominally 2x bf16; scaled from the measured bf16 burst
     res.update({"workload": "config 4: LLaMA-3.1-8B shapes, M=2048, 7 modules, MNZ, bf16 out", "unit": "TOPS",
                 "pct_of_nominal_4500": round(100 * tops / 4500.0, 2),
-                "roofline": {"bound": "tensor", "kernel": "gemm_i8_tcgen05_kernel (+ expand_levels_kernel)", "achieved": tops,
+                "roofline": {"bound": "tensor", "kernel": "gemm_i8_pair_kernel (+ expand_levels_kernel)", "achieved": tops,
                              "peak": int8_peak, "unit": "TOP/s", "frac": round(tops / int8_peak, 4),
                              "peak_source": f"2 x {pk['source']} bf16 burst"},
                 "tokens_per_s": round(M / (res["layer_with_act_quant"]["ms_per_layer"] * 1e-3), 1)})
+    res["library_int8"] = int8_library_point(torch, M, synth.LLAMA31_8B, device)
     return res
 
 

@@ -193,6 +193,18 @@ def test_prefill_route(name, route, M, N, K):
         check_outputs(y, acc, y_ref, acc_ref, bf16)
 
 
+def test_prefill_pair_route_224_wide_tiles():
+    # 3 token-tile pairs x 3100 channels: one round of 224-wide tiles (42 of them) beats one round of
+    # 256-wide and two rounds of 128-wide ones in the launcher's cost model, so this exercises the third
+    # tile width, ragged in both directions (600 = 2*256 + 88 tokens, 3100 = 13*224 + 188 channels)
+    lv = qift.MNZ
+    p_ref, s_n, codes, q_a, s_a = make_problem(lv, 600, 3100, 256, seed=81)
+    y_ref, acc_ref = oracle.linear(codes, lv, s_n, q_a, s_a, bf16=True)
+    y, acc = run_route(p_ref, s_n, lv, q_a, s_a, qift.ROUTE_PREFILL_PAIR, True)
+    check_outputs(y, acc, y_ref, acc_ref, True)
+    assert_status_clean()
+
+
 def test_auto_route_and_public_entry_points():
     for M in (1, 16, 17, 140):
         for lv in (qift.MNZ, qift.INT4):

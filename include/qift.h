@@ -66,8 +66,10 @@ typedef enum {
     QIFT_ROUTE_PREFILL = 3,  /* tcgen05 kind::i8 GEMM, codes expanded in the kernel; scratch 4*M    */
     QIFT_ROUTE_PREFILL_SCRATCH = 4, /* codes expanded to an int8 [N,K] scratch first, then a TMA-fed
                                       tcgen05 GEMM, one CTA per tile; scratch N*K bytes            */
-    QIFT_ROUTE_PREFILL_PAIR = 5    /* the same with CTA pairs (tcgen05 cta_group::2, 256-token tiles);
+    QIFT_ROUTE_PREFILL_PAIR = 5,   /* the same with CTA pairs (tcgen05 cta_group::2, 256-token tiles);
                                       scratch N*K bytes                                            */
+    QIFT_ROUTE_PREFILL_FUSED_PAIR = 6 /* CTA pairs with the codes expanded in the kernel (each CTA
+                                      expands half of the tile's channels); scratch 4*M            */
 } qift_route;
 
 const char* qift_status_string(int status);
@@ -77,9 +79,9 @@ const char* qift_status_string(int status);
 size_t qift_packed_bytes(int N, int K, int levels);
 
 /* Bytes of scratch qift_w2a4_linear / qift_w4a4_linear need for this problem: 0 when the decode
- * route serves it (M <= 16); 4*M rounded up to 1 KiB for 16 < M <= 768 (QIFT_ROUTE_PREFILL: the
- * per-token sums of q_a); N*K rounded up to 1 KiB for M > 768 (QIFT_ROUTE_PREFILL_PAIR: the codes
- * decoded to int8 once per call).  qift_workspace_bytes_route gives the figure for an explicit route. */
+ * route serves it (M <= 16); 4*M rounded up to 1 KiB for 16 < M <= 512 (QIFT_ROUTE_PREFILL up to 128
+ * rows, QIFT_ROUTE_PREFILL_FUSED_PAIR above: the per-token sums of q_a); N*K rounded up to 1 KiB for
+ * M > 512 (QIFT_ROUTE_PREFILL_PAIR: the codes decoded to int8 once per call).  qift_workspace_bytes_route gives the figure for an explicit route. */
 size_t qift_workspace_bytes(int M, int N, int K, int levels);
 size_t qift_workspace_bytes_route(int M, int N, int K, int levels, int route);
 
@@ -130,7 +132,7 @@ int qift_quantize_act(const void* X, int x_dtype, int M, int K, int had_block, f
  *   Y         out [M,N] fp32 or bf16 (round to nearest even): ((float)acc * s_a[m]) * s_n[n]
  *   acc_debug out int32 [M,N] accumulators, or NULL
  *   workspace     >= qift_workspace_bytes(M,N,K,levels) bytes, 256-byte aligned; may be NULL when 0
- * M <= 16 takes the decode route, 16 < M <= 768 the fused prefill route, larger M the CTA-pair scratch route. */
+ * M <= 16 takes the decode route, 16 < M <= 512 the fused prefill routes, larger M the CTA-pair scratch route. */
 int qift_w2a4_linear(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a,
                      const float* s_a, int M, int N, int K, void* Y, int y_dtype, int32_t* acc_debug,
                      void* workspace, size_t workspace_bytes, void* stream);

@@ -12,14 +12,20 @@
 #include "prefill.cuh"
 #include "prefill_2cta.cuh"
 #include "prefill_fused.cuh"
+#include "prefill_fused_pair.cuh"
 #include "rotate_quant.cuh"
 
 namespace qift {
 namespace {
 
-// Up to this many token rows the prefill route expands the codes inside the GEMM (one expansion per
-// 128-token tile); beyond it, expanding once into an int8 scratch and re-reading it wins.
-constexpr int kFusedMaxM = 768;
+// Prefill routes by token count (measured on a LLaMA-3.1-8B layer): up to 128 rows one CTA per tile
+// expanding the codes in the kernel; up to 512 rows CTA pairs expanding in the kernel (one expansion
+// per 256-token tile); beyond that, expanding once into an int8 scratch and re-reading it wins.
+constexpr int kFusedMaxM = 128;
+constexpr int kFusedPairMaxM = 512;
+inline int auto_prefill_route(int M) {
+    return (M <= kFusedMaxM) ? QIFT_ROUTE_PREFILL : (M <= kFusedPairMaxM) ? QIFT_ROUTE_PREFILL_FUSED_PAIR : QIFT_ROUTE_PREFILL_PAIR;
+}
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
@@ -201,6 +207,24 @@ int launch_expand(const uint32_t* packed, int N, int K, int8_t* out, cudaStream_
                                   K / codes_per_word(LV), out));
 }
 
+// Tile width of the CTA-pair kernels: the one whose rounds over the SM pairs cost least.  Measured at
+// M = 2048, K = 4096 a round of 128 / 224 / 256-wide tiles takes 10.3 / 13.0 / 13.5 us (the activation
+// tile is re-read from L2 for every channel tile, so narrow tiles are not proportionally cheaper):
+// cost ~ width + 284.  14336 channels then run 7 full rounds of 224-wide tiles instead of the
+// 6.05 -> 7 rounds of 256-wide ones; 1024 channels one round of 128-wide tiles.
+int pair_tile_width(int M, int N) {
+    const int widths[3] = {256, 224, 128};
+    const int pair_count = sm_count() / 2, m_pairs = (M + 2 * kGemmBM - 1) / (2 * kGemmBM);
+    int bn = 256;
+    long best = -1;
+    for (int w : widths) {
+        const long tiles = static_cast<long>(m_pairs) * ((N + w - 1) / w);
+        const long cost = ((tiles + pair_count - 1) / pair_count) * (w + 284);
+        if (best < 0 || cost < best) best = cost, bn = w;
+    }
+    return bn;
+}
+
 template <int BN>
 int launch_gemm_pairs(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& gp, cudaStream_t st) {
     auto kernel = gemm_i8_pair_kernel<BN>;
@@ -234,20 +258,7 @@ int run_prefill(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
     CUtensorMap ma, mb;
     GemmParams gp{s_n, s_a, Y, acc_debug, M, N, K, y_bf16};
     if (pairs) {  // each CTA of a pair loads its own 128 tokens and half of the tile's channels
-        // Tile width: the one whose rounds over the SM pairs cost least.  Measured at M = 2048, K = 4096
-        // a round of 128 / 224 / 256-wide tiles takes 10.3 / 13.0 / 13.5 us (the activation tile is
-        // re-read from L2 for every channel tile, so narrow tiles are not proportionally cheaper):
-        // cost ~ width + 284.  14336 channels then run 7 full rounds of 224-wide tiles instead of the
-        // 6.05 -> 7 rounds of 256-wide ones; 1024 channels one round of 128-wide tiles.
-        const int widths[3] = {256, 224, 128};
-        const int pair_count = sm_count() / 2, m_pairs = (M + 2 * kGemmBM - 1) / (2 * kGemmBM);
-        int bn = 256;
-        long best = -1;
-        for (int w : widths) {
-            const long tiles = static_cast<long>(m_pairs) * ((N + w - 1) / w);
-            const long cost = ((tiles + pair_count - 1) / pair_count) * (w + 284);
-            if (best < 0 || cost < best) best = cost, bn = w;
-        }
+        const int bn = pair_tile_width(M, N);
         if (!make_i8_map(&ma, q_a, M, K, kGemmBM) || !make_i8_map(&mb, wexp, N, K, bn / 2)) return QIFT_ERR_CUDA;
         switch (bn) {
             case 256: return launch_gemm_pairs<256>(ma, mb, gp, st);
@@ -277,9 +288,31 @@ int dispatch_fused(const CUtensorMap& ma, const FusedParams& fp, cudaStream_t st
     return narrow ? launch_fused<LV, 128>(ma, fp, st) : launch_fused<LV, 256>(ma, fp, st);
 }
 
+template <int LV, int BN>
+int launch_fused_pairs(const CUtensorMap& ma, const FusedParams& fp, cudaStream_t st) {
+    auto kernel = gemm_fused_pair_kernel<LV, BN>;
+    const size_t smem = fused_pair_smem_bytes<BN>();
+    cudaError_t e = allow_smem(kernel, smem);
+    if (e != cudaSuccess) return cuda_status(e);
+    const int tiles = ((fp.M + 2 * kGemmBM - 1) / (2 * kGemmBM)) * ((fp.N + BN - 1) / BN);
+    int pairs = sm_count() / 2;
+    if (pairs > tiles) pairs = tiles;
+    return cuda_status(launch_pdl_pairs(kernel, dim3(2 * pairs), dim3(kFusedThreads), smem, st, ma, fp));
+}
+
+template <int LV>
+int dispatch_fused_pairs(const CUtensorMap& ma, const FusedParams& fp, cudaStream_t st) {
+    switch (pair_tile_width(fp.M, fp.N)) {
+        case 256: return launch_fused_pairs<LV, 256>(ma, fp, st);
+        case 224: return launch_fused_pairs<LV, 224>(ma, fp, st);
+        default: return launch_fused_pairs<LV, 128>(ma, fp, st);
+    }
+}
+
 // Prefill route with the expansion fused into the GEMM; workspace = per-token sums of q_a.
 int run_prefill_fused(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N,
-                      int K, void* Y, int y_bf16, int32_t* acc_debug, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+                      int K, void* Y, int y_bf16, int32_t* acc_debug, void* workspace, size_t workspace_bytes, cudaStream_t st,
+                      bool pairs = false) {
     if (K % 16 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;  // TMA row pitch must be a multiple of 16 bytes
     const size_t need = (static_cast<size_t>(M) * 4 + 1023) & ~static_cast<size_t>(1023);
     if (!workspace || workspace_bytes < need) return QIFT_ERR_WORKSPACE;
@@ -290,6 +323,14 @@ int run_prefill_fused(const uint32_t* packed, const float* s_n, int lv, const in
     CUtensorMap ma;
     if (!make_i8_map(&ma, q_a, M, K, kGemmBM)) return QIFT_ERR_CUDA;
     FusedParams fp{packed, s_n, s_a, sumq, Y, acc_debug, M, N, K, y_bf16};
+    if (pairs) {
+        switch (lv) {
+            case QIFT_LEVELS_MNZ: return dispatch_fused_pairs<QIFT_LEVELS_MNZ>(ma, fp, st);
+            case QIFT_LEVELS_POT: return dispatch_fused_pairs<QIFT_LEVELS_POT>(ma, fp, st);
+            case QIFT_LEVELS_SYM: return dispatch_fused_pairs<QIFT_LEVELS_SYM>(ma, fp, st);
+            default: return dispatch_fused_pairs<QIFT_LEVELS_INT4>(ma, fp, st);
+        }
+    }
     switch (lv) {
         case QIFT_LEVELS_MNZ: return dispatch_fused<QIFT_LEVELS_MNZ>(ma, fp, st);
         case QIFT_LEVELS_POT: return dispatch_fused<QIFT_LEVELS_POT>(ma, fp, st);
@@ -302,7 +343,7 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
                 void* Y, int y_dtype, int32_t* acc_debug, void* workspace, size_t workspace_bytes, int route, void* stream) {
     if (!packed || !s_n || !q_a || !s_a || !Y || M <= 0 || N <= 0 || K <= 0 || !valid_levels(lv)) return QIFT_ERR_INVALID_ARG;
     if (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16) return QIFT_ERR_INVALID_ARG;
-    if (route < QIFT_ROUTE_AUTO || route > QIFT_ROUTE_PREFILL_PAIR) return QIFT_ERR_INVALID_ARG;
+    if (route < QIFT_ROUTE_AUTO || route > QIFT_ROUTE_PREFILL_FUSED_PAIR) return QIFT_ERR_INVALID_ARG;
     if (K % codes_per_word(lv) != 0 || K % 4 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(packed) || !aligned16(s_n) || !aligned16(q_a) || !aligned16(s_a) || !aligned16(Y) ||
         (acc_debug && !aligned16(acc_debug)))
@@ -311,7 +352,7 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
     const int y_bf16 = (y_dtype == QIFT_BF16);
     if (route == QIFT_ROUTE_AUTO) {
         if (M <= 16) route = decode_supports(lv, M, N, K) ? QIFT_ROUTE_DECODE : QIFT_ROUTE_GENERIC;
-        else route = (K % 16 != 0) ? QIFT_ROUTE_GENERIC : (M <= kFusedMaxM) ? QIFT_ROUTE_PREFILL : QIFT_ROUTE_PREFILL_PAIR;
+        else route = (K % 16 != 0) ? QIFT_ROUTE_GENERIC : auto_prefill_route(M);
     }
     if (route == QIFT_ROUTE_DECODE) {
         if (!decode_supports(lv, M, N, K)) return QIFT_ERR_UNSUPPORTED_SHAPE;
@@ -323,8 +364,9 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
             default: return dispatch_decode<QIFT_LEVELS_INT4>(p, st);
         }
     }
-    if (route == QIFT_ROUTE_PREFILL)
-        return run_prefill_fused(packed, s_n, lv, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, workspace, workspace_bytes, st);
+    if (route == QIFT_ROUTE_PREFILL || route == QIFT_ROUTE_PREFILL_FUSED_PAIR)
+        return run_prefill_fused(packed, s_n, lv, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, workspace, workspace_bytes, st,
+                                 route == QIFT_ROUTE_PREFILL_FUSED_PAIR);
     if (route == QIFT_ROUTE_PREFILL_SCRATCH || route == QIFT_ROUTE_PREFILL_PAIR)
         return run_prefill(packed, s_n, lv, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, workspace, workspace_bytes, st,
                            route == QIFT_ROUTE_PREFILL_PAIR);
@@ -365,9 +407,9 @@ size_t qift_packed_bytes(int N, int K, int levels) {
 size_t qift_workspace_bytes_route(int M, int N, int K, int levels, int route) {
     if (M <= 0 || N <= 0 || K <= 0 || !valid_levels(levels)) return 0;
     if (route == QIFT_ROUTE_AUTO)
-        route = (M <= 16) ? QIFT_ROUTE_DECODE : (M <= kFusedMaxM) ? QIFT_ROUTE_PREFILL : QIFT_ROUTE_PREFILL_PAIR;
+        route = (M <= 16) ? QIFT_ROUTE_DECODE : auto_prefill_route(M);
     size_t b = 0;
-    if (route == QIFT_ROUTE_PREFILL) b = static_cast<size_t>(M) * 4;
+    if (route == QIFT_ROUTE_PREFILL || route == QIFT_ROUTE_PREFILL_FUSED_PAIR) b = static_cast<size_t>(M) * 4;
     if (route == QIFT_ROUTE_PREFILL_SCRATCH || route == QIFT_ROUTE_PREFILL_PAIR) b = static_cast<size_t>(N) * K;
     return (b + 1023) & ~static_cast<size_t>(1023);
 }

@@ -181,7 +181,8 @@ def test_decode_extreme_values(name):
 
 
 @pytest.mark.parametrize("name", list(LEVELS))
-@pytest.mark.parametrize("route", [qift.ROUTE_PREFILL, qift.ROUTE_PREFILL_SCRATCH, qift.ROUTE_PREFILL_PAIR])
+@pytest.mark.parametrize("route", [qift.ROUTE_PREFILL, qift.ROUTE_PREFILL_SCRATCH, qift.ROUTE_PREFILL_PAIR,
+                                   qift.ROUTE_PREFILL_FUSED_PAIR])
 @pytest.mark.parametrize("M,N,K", [(128, 256, 512), (200, 300, 1024), (17, 72, 256), (512, 1024, 384), (130, 520, 4096),
                                    (300, 2000, 2320), (1, 40, 48)])
 def test_prefill_route(name, route, M, N, K):
@@ -200,8 +201,9 @@ def test_prefill_pair_route_224_wide_tiles():
     lv = qift.MNZ
     p_ref, s_n, codes, q_a, s_a = make_problem(lv, 600, 3100, 256, seed=81)
     y_ref, acc_ref = oracle.linear(codes, lv, s_n, q_a, s_a, bf16=True)
-    y, acc = run_route(p_ref, s_n, lv, q_a, s_a, qift.ROUTE_PREFILL_PAIR, True)
-    check_outputs(y, acc, y_ref, acc_ref, True)
+    for route in (qift.ROUTE_PREFILL_PAIR, qift.ROUTE_PREFILL_FUSED_PAIR):
+        y, acc = run_route(p_ref, s_n, lv, q_a, s_a, route, True)
+        check_outputs(y, acc, y_ref, acc_ref, True)
     assert_status_clean()
 
 

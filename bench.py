@@ -39,7 +39,7 @@ N_LAYERS = 32
 # dram__bytes_read.sum + dram__bytes_write.sum of one linear_grouped_kernel launch in the ncu capture of
 # the 4-layer case (profiles/linear_grouped_kernel_llama2_m1_4layers.md): 203 236 864 + 4 653 056 bytes
 # for 203 877 488 algorithmic bytes.  Every packed word is read once, so traffic scales with the layers.
-NCU_TRAFFIC_BYTES_4_LAYERS = 203_236_864 + 4_653_056
+NCU_TRAFFIC_BYTES_4_LAYERS = 207318528   # dram__bytes_read.sum + dram__bytes_write.sum of linear_grouped_kernel, 4-layer capture (profiles/)
 
 
 # ------------------------------------------------------------------------------------------------

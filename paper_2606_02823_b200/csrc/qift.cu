@@ -598,7 +598,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     if (M > 16) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (plan_bytes < qift_group_plan_bytes(count)) return QIFT_ERR_WORKSPACE;
     if (!aligned16(plan_dev) || !aligned16(plan_host)) return QIFT_ERR_ALIGNMENT;
-    const int rows_per_item = (M > 8) ? 16 : (M == 1) ? 64 : 32;  // must match dispatch_grouped's row tiles
+    const int rows_per_item = (M > 8) ? kWideRows : (M == 1) ? 64 : 32;  // must match dispatch_grouped's row tiles
     GroupHeader* h = static_cast<GroupHeader*>(plan_host);
     GroupProblemDev* d = reinterpret_cast<GroupProblemDev*>(h + 1);
     int items = 0, max_k = 0;
@@ -668,10 +668,35 @@ int launch_grouped(const GroupHeader* h, const GroupProblemDev* host, const Grou
     return QIFT_OK;
 }
 
+// 9..16 token rows: 128-row items split by rows over the warps, one CTA per SM.
+template <int LV>
+int launch_grouped_wide(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
+                        cudaStream_t st) {
+    auto kernel = linear_grouped_wide_kernel<LV>;
+    const size_t stage = wide_stage_bytes(LV, h->M) + 16;
+    for (int first = 0; first < h->count; first += kGroupSlice) {
+        const int count = (h->count - first < kGroupSlice) ? h->count - first : kGroupSlice;
+        const int item_first = host[first].item_begin;
+        const int item_end = (first + count < h->count) ? host[first + count].item_begin : h->total_items;
+        int stages = static_cast<int>((226 * 1024 - static_cast<size_t>(count) * sizeof(SmemProblem) - 64) / stage);
+        if (stages < 2) stages = 2;
+        if (stages > 8) stages = 8;
+        const size_t smem = wide_smem_bytes(LV, h->M, stages, count);
+        cudaError_t e = allow_smem(kernel, smem);
+        if (e != cudaSuccess) return cuda_status(e);
+        int grid = sm_count();
+        if (grid > item_end - item_first) grid = item_end - item_first;
+        GroupParams gp{dev + first, sumq, first, count, item_first, item_end, h->M, h->y_bf16, stages};
+        const int rc = cuda_status(launch_pdl(kernel, dim3(grid), dim3(kDecThreads), smem, st, gp));
+        if (rc != QIFT_OK) return rc;
+    }
+    return QIFT_OK;
+}
+
 template <int LV>
 int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
                      cudaStream_t st) {
-    if (h->M > 8) return launch_grouped<LV, 2, 1, false>(h, host, dev, sumq, st);
+    if (h->M > 8) return launch_grouped_wide<LV>(h, host, dev, sumq, st);
     if (h->M == 1) return launch_grouped<LV, 1, 4, true>(h, host, dev, sumq, st);
     return launch_grouped<LV, 1, 2, false>(h, host, dev, sumq, st);
 }

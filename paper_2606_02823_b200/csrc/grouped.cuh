@@ -101,7 +101,7 @@ constexpr int kGroupSlice = 256;  // problems per launch (their table lives in s
 
 // Walks this CTA's share of the work list chunk by chunk; the producer and the consumers each run
 // one and see the same sequence.  PER = codes per packed word.
-template <int PER>
+template <int PER, int CW = kChunkWords>
 struct GroupCursor {
     const SmemProblem* table;
     int count, item_end, rows_per_item;
@@ -124,7 +124,7 @@ struct GroupCursor {
         const SmemProblem& P = table[p];
         N = P.N, K = P.K;
         words_per_row = K / PER;
-        nchunks = (words_per_row + kChunkWords - 1) / kChunkWords;
+        nchunks = (words_per_row + CW - 1) / CW;
         n0 = (item - P.item_begin) * rows_per_item;
         tiles_valid = (min(rows_per_item, N - n0) + 15) >> 4;
         const int pitch = round_up16(words_per_row);
@@ -132,7 +132,7 @@ struct GroupCursor {
         wbase = P.packed + static_cast<size_t>(n0) * pitch * 4;
         q_a = P.q_a;
     }
-    __device__ __forceinline__ int chunk_words() const { return min(kChunkWords, words_per_row - chunk * kChunkWords); }
+    __device__ __forceinline__ int chunk_words() const { return min(CW, words_per_row - chunk * CW); }
     __device__ __forceinline__ bool last_chunk() const { return chunk + 1 == nchunks; }
     __device__ __forceinline__ void next() {
         if (++chunk == nchunks) {
@@ -369,6 +369,204 @@ linear_grouped_kernel(const GroupParams gp) {
             const float y = scale_epilogue(acc_v, e_sa, e_sn);
             if (gp.y_bf16) static_cast<uint16_t*>(P->Y)[idx] = f32_to_bf16_bits(y);
             else static_cast<float*>(P->Y)[idx] = y;
+        }
+    }
+    if (!ok) *fail = 1;
+}
+
+// ------------------------------------------------------------------------------------------------
+// grouped product for 9..16 token rows
+// ------------------------------------------------------------------------------------------------
+// With more than eight tokens the split of a stage along K over the eight consumer warps stops paying:
+// every item then ends in a cross-warp reduction of rows x tokens x 8 partial sums, as much work as
+// the product itself, and its buffers leave room for two small stages only.  Here an item is 128
+// rows and the warps split it by ROWS: warp w owns the 16-row tile w of the item for the whole K
+// loop, accumulates all 16 tokens in registers and writes its outputs itself -- no reduction, no CTA
+// barrier.  The price is that every warp reads the whole activation slice of a stage, so stages are
+// half tiles (64 words per row: 32 KB of weights + 17 KB of activations at 16 tokens), four deep.
+constexpr int kWideChunkWords = 64;
+constexpr int kWideQPad = 16;                    // token stride = 16 bytes mod 128: see the consumer's loads
+constexpr int kWideTiles = kDecWarps;            // row tiles per item, one per consumer warp
+constexpr int kWideRows = 16 * kWideTiles;       // 128
+
+__host__ __device__ inline size_t wide_stage_bytes(int lv, int M) {
+    return static_cast<size_t>(kWideTiles) * (kTileBytes / 2) + static_cast<size_t>(M) * (kWideChunkWords * codes_per_word(lv) + kWideQPad);
+}
+__host__ __device__ inline size_t wide_smem_bytes(int lv, int M, int stages, int count) {
+    return static_cast<size_t>(count) * sizeof(SmemProblem) + stages * (wide_stage_bytes(lv, M) + 16) + 16;
+}
+
+template <int LV>
+__global__ void __launch_bounds__(kDecThreads, 1)
+linear_grouped_wide_kernel(const GroupParams gp) {
+    using T = DecodeTraits<LV>;
+    constexpr int QSTRIDE = kWideChunkWords * T::PER + kWideQPad;
+    using Cursor = GroupCursor<T::PER, kWideChunkWords>;
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int M = gp.M;
+    const uint32_t stage_bytes = static_cast<uint32_t>(wide_stage_bytes(LV, M));
+    const int stages = gp.stages;
+    unsigned char* ring = smem;
+    SmemProblem* table = reinterpret_cast<SmemProblem*>(smem + stages * stage_bytes);
+    uint64_t* full = reinterpret_cast<uint64_t*>(table + gp.count);
+    uint64_t* empty = full + stages;
+    volatile int* fail = reinterpret_cast<volatile int*>(empty + stages);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    pdl_launch_dependents();
+    if (tid == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], kDecWarps);
+        }
+        mbar_fence_init();
+        *fail = 0;
+    }
+    for (int i = tid; i < gp.count; i += kDecThreads) {
+        const GroupProblemDev& P = gp.problems[i];
+        SmemProblem e;
+        e.packed = reinterpret_cast<const unsigned char*>(P.packed);
+        e.q_a = P.q_a, e.s_n = P.s_n, e.s_a = P.s_a, e.Y = P.Y, e.acc_debug = P.acc_debug;
+        e.N = P.N, e.K = P.K, e.item_begin = P.item_begin, e.index = gp.first_index + i;
+        table[i] = e;
+    }
+    __syncthreads();
+
+    if (warp == kDecWarps) {
+        // ---------------------------------------------------------------- producer warp
+        auto expect = [&](const Cursor& c, int s) {
+            if (lane == 0) mbar_expect_tx(&full[s], c.chunk_words() * (64 * c.tiles_valid + T::PER * M));
+            __syncwarp();
+        };
+        auto issue_w = [&](const Cursor& c, int s) {  // one bulk copy per 16-row tile: the chunk's slices are contiguous in it
+            const uint32_t bytes = c.chunk_words() * 16 * 4;
+            unsigned char* dst = ring + s * stage_bytes;
+            if (lane < c.tiles_valid)
+                bulk_g2s(dst + lane * (kTileBytes / 2), c.wbase + lane * c.rb_bytes + static_cast<size_t>(c.chunk) * (kTileBytes / 2),
+                         bytes, &full[s]);
+        };
+        auto issue_q = [&](const Cursor& c, int s) {
+            const uint32_t seg = c.chunk_words() * T::PER;
+            unsigned char* dst = ring + s * stage_bytes + kWideTiles * (kTileBytes / 2);
+            for (int m = lane; m < M; m += 32)
+                bulk_g2s(dst + m * QSTRIDE, c.q_a + static_cast<size_t>(m) * c.K + static_cast<size_t>(c.chunk) * (kWideChunkWords * T::PER),
+                         seg, &full[s]);
+        };
+        Cursor a;
+        a.init(table, gp.count, gp.item_first, gp.item_end, kWideRows);
+        int pre = 0;
+        for (; pre < stages && a.valid(); ++pre, a.next()) {  // weights do not depend on the previous kernel
+            expect(a, pre);
+            issue_w(a, pre);
+        }
+        pdl_wait();
+        Cursor b;
+        b.init(table, gp.count, gp.item_first, gp.item_end, kWideRows);
+        for (int i = 0; i < pre; ++i, b.next()) issue_q(b, i);
+        int s = 0;
+        uint32_t ph = 0;
+        for (; b.valid(); b.next()) {
+            if (!mbar_wait(&empty[s], ph, 5)) break;
+            expect(b, s);
+            issue_w(b, s);
+            issue_q(b, s);
+            if (++s == stages) s = 0, ph ^= 1;
+        }
+        return;
+    }
+
+    // -------------------------------------------------------------------- consumer warps
+    pdl_wait();
+    const int g = lane >> 2, cq = lane & 3;
+    Cursor cur;
+    cur.init(table, gp.count, gp.item_first, gp.item_end, kWideRows);
+    bool ok = true;
+    int s = 0;
+    uint32_t ph = 0;
+    while (cur.valid() && ok) {
+        int acc[2][T::NACC][4];
+#pragma unroll
+        for (int b = 0; b < 2; ++b)
+#pragma unroll
+            for (int t = 0; t < T::NACC; ++t)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[b][t][i] = 0;
+        const SmemProblem* P = &table[cur.p];
+        const int row0 = cur.n0 + 16 * warp;          // this warp's tile
+        const bool tile_on = warp < cur.tiles_valid;
+
+        for (;;) {
+            if (!mbar_wait(&full[s], ph, 6)) {
+                ok = false;
+                break;
+            }
+            const int cw = cur.chunk_words();
+            const unsigned char* wst = ring + s * stage_bytes + warp * (kTileBytes / 2);
+            const unsigned char* qst = ring + s * stage_bytes + kWideTiles * (kTileBytes / 2);
+            if (tile_on) {
+                // A lane needs 64 contiguous activation bytes per token and slice (its four packed words x 16
+                // codes), lanes of a quad 64 bytes apart: read straight, lanes cq and cq+2 would hit the same
+                // banks.  Lanes with cq >= 2 therefore take their four words in the order 2,3,0,1 (the sums do
+                // not depend on the order) -- with a token stride of 16 bytes mod 128 every quarter-warp then
+                // covers all eight 16-byte bank groups.
+                // (INT4 weights: 32 bytes per lane, already conflict-free without the rotation.)
+                const int rot = (T::PER == 16) ? (cq & 2) : 0;
+                for (int sl = 0; 16 * sl < cw; ++sl) {   // 16-word slices of the chunk
+                    uint32_t qb[2][4 * T::NPL];
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt) {
+                        const int m = nt * 8 + g;
+                        if (m < M) {
+                            const unsigned char* src = qst + m * QSTRIDE + (16 * sl + 4 * cq) * T::PER;
+#pragma unroll
+                            for (int i = 0; i < T::NPL; ++i) {
+                                // NPL 16-byte pieces hold the lane's four words in order; piece i holds word 4i/NPL
+                                const uint4 v = *reinterpret_cast<const uint4*>(src + ((i + rot * T::NPL / 4) % T::NPL) * 16);
+                                qb[nt][4 * i] = v.x, qb[nt][4 * i + 1] = v.y, qb[nt][4 * i + 2] = v.z, qb[nt][4 * i + 3] = v.w;
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 4 * T::NPL; ++i) qb[nt][i] = 0;
+                        }
+                    }
+                    const unsigned char* wsrc = wst + (2 * sl * 32 + lane) * 16;
+                    const uint2 a_lo = *reinterpret_cast<const uint2*>(wsrc + 4 * rot), a_hi = *reinterpret_cast<const uint2*>(wsrc + 8 - 4 * rot);
+                    const uint2 b_lo = *reinterpret_cast<const uint2*>(wsrc + 512 + 4 * rot), b_hi = *reinterpret_cast<const uint2*>(wsrc + 520 - 4 * rot);
+                    const uint4 wa = make_uint4(a_lo.x, a_lo.y, a_hi.x, a_hi.y);
+                    const uint4 wb = make_uint4(b_lo.x, b_lo.y, b_hi.x, b_hi.y);
+                    mma_tile_step<LV, 2, true>(acc, wa, wb, qb);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[s]);
+            if (++s == stages) s = 0, ph ^= 1;
+            const bool last = cur.last_chunk();
+            cur.next();
+            if (last) break;
+        }
+        if (!ok) break;
+
+        // epilogue from registers: rows g and g+8 of the tile, tokens nt*8 + 2cq + {0,1}
+        if (tile_on) {
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int tok = nt * 8 + 2 * cq + (i & 1);
+                    const int n = row0 + g + ((i & 2) ? 8 : 0);
+                    if (tok < M && n < P->N) {
+                        int v[T::NACC];
+#pragma unroll
+                        for (int a = 0; a < T::NACC; ++a) v[a] = acc[nt][a][i];
+                        const int acc_v = level_sum<LV, true, T::NACC>(v, gp.sumq[P->index * 16 + tok]);
+                        const size_t idx = static_cast<size_t>(tok) * P->N + n;
+                        if (P->acc_debug) P->acc_debug[idx] = acc_v;
+                        const float y = scale_epilogue(acc_v, P->s_a[tok], __ldg(P->s_n + n));
+                        if (gp.y_bf16) static_cast<uint16_t*>(P->Y)[idx] = f32_to_bf16_bits(y);
+                        else static_cast<float*>(P->Y)[idx] = y;
+                    }
+                }
         }
     }
     if (!ok) *fail = 1;

@@ -396,7 +396,7 @@ __host__ __device__ inline size_t wide_smem_bytes(int lv, int M, int stages, int
     return static_cast<size_t>(count) * sizeof(SmemProblem) + stages * (wide_stage_bytes(lv, M) + 16) + 16;
 }
 
-template <int LV>
+template <int LV, int NT>
 __global__ void __launch_bounds__(kDecThreads, 1)
 linear_grouped_wide_kernel(const GroupParams gp) {
     using T = DecodeTraits<LV>;
@@ -485,9 +485,9 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     int s = 0;
     uint32_t ph = 0;
     while (cur.valid() && ok) {
-        int acc[2][T::NACC][4];
+        int acc[NT][T::NACC][4];
 #pragma unroll
-        for (int b = 0; b < 2; ++b)
+        for (int b = 0; b < NT; ++b)
 #pragma unroll
             for (int t = 0; t < T::NACC; ++t)
 #pragma unroll
@@ -513,9 +513,9 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                 // (INT4 weights: 32 bytes per lane, already conflict-free without the rotation.)
                 const int rot = (T::PER == 16) ? (cq & 2) : 0;
                 for (int sl = 0; 16 * sl < cw; ++sl) {   // 16-word slices of the chunk
-                    uint32_t qb[2][4 * T::NPL];
+                    uint32_t qb[NT][4 * T::NPL];
 #pragma unroll
-                    for (int nt = 0; nt < 2; ++nt) {
+                    for (int nt = 0; nt < NT; ++nt) {
                         const int m = nt * 8 + g;
                         if (m < M) {
                             const unsigned char* src = qst + m * QSTRIDE + (16 * sl + 4 * cq) * T::PER;
@@ -535,7 +535,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                     const uint2 b_lo = *reinterpret_cast<const uint2*>(wsrc + 512 + 4 * rot), b_hi = *reinterpret_cast<const uint2*>(wsrc + 520 - 4 * rot);
                     const uint4 wa = make_uint4(a_lo.x, a_lo.y, a_hi.x, a_hi.y);
                     const uint4 wb = make_uint4(b_lo.x, b_lo.y, b_hi.x, b_hi.y);
-                    mma_tile_step<LV, 2, true>(acc, wa, wb, qb);
+                    mma_tile_step<LV, NT, true>(acc, wa, wb, qb);
                 }
             }
             __syncwarp();
@@ -550,7 +550,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
         // epilogue from registers: rows g and g+8 of the tile, tokens nt*8 + 2cq + {0,1}
         if (tile_on) {
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt)
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int tok = nt * 8 + 2 * cq + (i & 1);

@@ -21,6 +21,10 @@ namespace {
 // Prefill routes by token count (measured on a LLaMA-3.1-8B layer): up to 128 rows one CTA per tile
 // expanding the codes in the kernel; up to 512 rows CTA pairs expanding in the kernel (one expansion
 // per 256-token tile); beyond that, expanding once into an int8 scratch and re-reading it wins.
+// Grouped decode: from this many token rows on the row-split kernel (128-row items) is the faster one
+// (measured on 32 LLaMA-2-7B layers: MNZ 369 us flat against 348 / 385 us at 5 / 6 rows for the K-split
+// kernel; PoT 510 against 561 at 2 rows; INT4 641 against 604 at 8 rows).
+inline int wide_min_m(int lv) { return lv == QIFT_LEVELS_POT ? 2 : lv == QIFT_LEVELS_INT4 ? 9 : 6; }
 constexpr int kFusedMaxM = 128;
 constexpr int kFusedPairMaxM = 512;
 inline int auto_prefill_route(int M) {
@@ -598,7 +602,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     if (M > 16) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (plan_bytes < qift_group_plan_bytes(count)) return QIFT_ERR_WORKSPACE;
     if (!aligned16(plan_dev) || !aligned16(plan_host)) return QIFT_ERR_ALIGNMENT;
-    const int rows_per_item = (M > 8) ? kWideRows : (M == 1) ? 64 : 32;  // must match dispatch_grouped's row tiles
+    const int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : (M == 1) ? 64 : 32;  // must match dispatch_grouped's row tiles
     GroupHeader* h = static_cast<GroupHeader*>(plan_host);
     GroupProblemDev* d = reinterpret_cast<GroupProblemDev*>(h + 1);
     int items = 0, max_k = 0;
@@ -668,11 +672,11 @@ int launch_grouped(const GroupHeader* h, const GroupProblemDev* host, const Grou
     return QIFT_OK;
 }
 
-// 9..16 token rows: 128-row items split by rows over the warps, one CTA per SM.
-template <int LV>
+// From this many token rows on: 128-row items split by rows over the warps, one CTA per SM.
+template <int LV, int NT>
 int launch_grouped_wide(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
                         cudaStream_t st) {
-    auto kernel = linear_grouped_wide_kernel<LV>;
+    auto kernel = linear_grouped_wide_kernel<LV, NT>;
     const size_t stage = wide_stage_bytes(LV, h->M) + 16;
     for (int first = 0; first < h->count; first += kGroupSlice) {
         const int count = (h->count - first < kGroupSlice) ? h->count - first : kGroupSlice;
@@ -696,7 +700,8 @@ int launch_grouped_wide(const GroupHeader* h, const GroupProblemDev* host, const
 template <int LV>
 int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
                      cudaStream_t st) {
-    if (h->M > 8) return launch_grouped_wide<LV>(h, host, dev, sumq, st);
+    if (h->M > 8) return launch_grouped_wide<LV, 2>(h, host, dev, sumq, st);
+    if (h->M >= wide_min_m(LV)) return launch_grouped_wide<LV, 1>(h, host, dev, sumq, st);
     if (h->M == 1) return launch_grouped<LV, 1, 4, true>(h, host, dev, sumq, st);
     return launch_grouped<LV, 1, 2, false>(h, host, dev, sumq, st);
 }

@@ -249,7 +249,7 @@ def test_whole_path_config1():
 
 # ---------------------------------------------------------------------------------- grouped path
 @pytest.mark.parametrize("name", list(LEVELS))
-@pytest.mark.parametrize("M", [1, 5, 8, 9, 13, 16])
+@pytest.mark.parametrize("M", [1, 2, 5, 6, 8, 9, 13, 16])
 def test_grouped_forward(name, M):
     # a ragged list: different N (incl. not a multiple of the row block), different K (incl. a
     # partial last chunk), more items than CTAs

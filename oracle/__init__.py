@@ -225,3 +225,56 @@ def linear(codes, lv: int, s_n, q_a, s_a, bf16: bool = False):
     """S4 + S5 -> (y, acc)."""
     acc = int_matmul(codes, lv, q_a)
     return epilogue(acc, s_a, s_n, bf16=bf16), acc
+
+
+# ---------------------------------------------------------------------------------------- KV4
+def kv4_quantize(X, had_block: int = 0, clip: float = 0.95):
+    """X fp32 [rows, D] -> (codes uint8 [rows, D] in 0..15, scale fp32 [rows], zero fp32 [rows])."""
+    X = _f32(X)
+    rows, D = X.shape
+    assert had_block == 0 or ((had_block & (had_block - 1)) == 0 and D % had_block == 0)
+    codes = np.empty((rows, D), dtype=np.uint8)
+    scale = np.empty((rows,), dtype=np.float32)
+    zero = np.empty((rows,), dtype=np.float32)
+    scratch = np.empty((D,), dtype=np.float32)
+    vp = ctypes.c_void_p
+    lib().orc_kv4_quantize(X.ctypes.data_as(vp), ctypes.c_longlong(rows), D, int(had_block), ctypes.c_float(clip),
+                           codes.ctypes.data_as(vp), scale.ctypes.data_as(vp), zero.ctypes.data_as(vp),
+                           scratch.ctypes.data_as(vp))
+    return codes, scale, zero
+
+
+def kv4_pack(codes):
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    rows, D = codes.reshape(-1, codes.shape[-1]).shape
+    out = np.empty((rows, D // 2), dtype=np.uint8)
+    vp = ctypes.c_void_p
+    lib().orc_kv4_pack(codes.ctypes.data_as(vp), ctypes.c_longlong(rows), D, out.ctypes.data_as(vp))
+    return out.reshape(codes.shape[:-1] + (D // 2,))
+
+
+def kv4_unpack(packed):
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    rows, half = packed.reshape(-1, packed.shape[-1]).shape
+    out = np.empty((rows, 2 * half), dtype=np.uint8)
+    vp = ctypes.c_void_p
+    lib().orc_kv4_unpack(packed.ctypes.data_as(vp), ctypes.c_longlong(rows), 2 * half, out.ctypes.data_as(vp))
+    return out.reshape(packed.shape[:-1] + (2 * half,))
+
+
+def kv4_attention(q, kc, ks, kz, vc, vs, vz):
+    """q fp32 [Hq, D]; codes uint8 [Hkv, T, D]; scales / zero-points fp32 [Hkv, T] -> out fp64 [Hq, D]."""
+    q = _f32(q)
+    Hq, D = q.shape
+    kc = np.ascontiguousarray(kc, dtype=np.uint8)
+    vc = np.ascontiguousarray(vc, dtype=np.uint8)
+    Hkv, T, D2 = kc.shape
+    assert D2 == D and vc.shape == kc.shape and Hq % Hkv == 0
+    ks, kz, vs, vz = (_f32(a) for a in (ks, kz, vs, vz))
+    out = np.empty((Hq, D), dtype=np.float64)
+    scratch = np.empty((T,), dtype=np.float64)
+    vp = ctypes.c_void_p
+    lib().orc_kv4_attention(q.ctypes.data_as(vp), kc.ctypes.data_as(vp), ks.ctypes.data_as(vp), kz.ctypes.data_as(vp),
+                            vc.ctypes.data_as(vp), vs.ctypes.data_as(vp), vz.ctypes.data_as(vp), T, Hq, Hkv, D,
+                            out.ctypes.data_as(vp), scratch.ctypes.data_as(vp))
+    return out

@@ -24,6 +24,14 @@
 //                        words stored in 16-row x 128-word tiles (layout comment at orc_pack).
 //   orc_int_matmul       Sec. 3.6 decoded small signed integer levels times integer activations.
 //   orc_epilogue*        Sec. 1 "the per-channel scale can be applied separately in the epilogue".
+//   orc_kv4_quantize     Sec. 4.1: the KV cache is quantized to four bits asymmetrically with a
+//                        clipping ratio (0.95 there), keys and values alike; the paper gives no
+//                        more, so the rest is the usual asymmetric integer quantizer: one
+//                        (scale, zero-point) pair per token and head over the head dimension, the
+//                        range [min(x,0), max(x,0)] shrunk by the clipping ratio, 16 levels.
+//   orc_kv4_pack/unpack  two 4-bit codes per byte, even dimension in the low nibble.
+//   orc_kv4_attention    single-query scaled dot-product attention over the dequantized cache (the
+//                        decode step whose memory traffic Sec. 1 calls the bottleneck), in fp64.
 //
 // Parity pins for every function live in the CPU test-suite (closed forms, brute force, printed
 // table values); none is "parity unpinned" except the numeric value of a forward output on the real
@@ -325,6 +333,96 @@ void orc_epilogue_bf16(const int32_t* acc, const float* s_a, const float* s_n, i
             const float t = (float)acc[(size_t)m * N + n] * s_a[m];
             y[(size_t)m * N + n] = bf16_rne(t * s_n[n]);
         }
+}
+
+// ------------------------------------------------------------------------------------------------
+// KV4: asymmetric 4-bit key / value cache
+// ------------------------------------------------------------------------------------------------
+// Quantize `rows` vectors of length D (one per token and head).  With B > 1 the vector is first
+// rotated by the ORTHONORMAL blockwise Hadamard (butterfly, then one multiply by 1/sqrt(B)): queries
+// carry no per-vector scale into which the factor could be folded.
+//   lo = clip * min(0, min_d u),  hi = clip * max(0, max_d u)       (zero always inside the range)
+//   s  = (hi - lo) / 15            (s = 1, z = 0 if hi == lo)
+//   z  = rint(-lo / s)             (integer zero-point, 0..15, stored as a float)
+//   c  = clamp(rint(u / s) + z, 0, 15),   dequantized value  s * (c - z)
+// All in fp32 with IEEE division and round-half-even.  codes: one per byte.  scratch: D floats.
+void orc_kv4_quantize(const float* X, long long rows, int D, int B, float clip, uint8_t* codes, float* scale,
+                      float* zero, float* scratch) {
+    for (long long r = 0; r < rows; ++r) {
+        for (int d = 0; d < D; ++d) scratch[d] = X[(size_t)r * D + d];
+        if (B > 1) {
+            orc_wht_blocks(scratch, D, B);
+            const float f = inv_sqrt_block(B);
+            for (int d = 0; d < D; ++d) scratch[d] = scratch[d] * f;
+        }
+        float mn = 0.0f, mx = 0.0f;
+        for (int d = 0; d < D; ++d) {
+            if (scratch[d] < mn) mn = scratch[d];
+            if (scratch[d] > mx) mx = scratch[d];
+        }
+        const float lo = mn * clip, hi = mx * clip;
+        float s = 1.0f, z = 0.0f;
+        if (hi != lo) {
+            const float range = hi - lo;
+            s = range / 15.0f;
+            const float nlo = -lo;
+            z = (float)std::rint(nlo / s);
+        }
+        for (int d = 0; d < D; ++d) {
+            const float t = scratch[d] / s;
+            const int c = (int)std::rint(t) + (int)z;
+            codes[(size_t)r * D + d] = (uint8_t)clampi(c, 0, 15);
+        }
+        scale[r] = s;
+        zero[r] = z;
+    }
+}
+
+void orc_kv4_pack(const uint8_t* codes, long long rows, int D, uint8_t* bytes) {
+    for (long long r = 0; r < rows; ++r)
+        for (int i = 0; i < D / 2; ++i)
+            bytes[(size_t)r * (D / 2) + i] =
+                (uint8_t)(codes[(size_t)r * D + 2 * i] | (codes[(size_t)r * D + 2 * i + 1] << 4));
+}
+
+void orc_kv4_unpack(const uint8_t* bytes, long long rows, int D, uint8_t* codes) {
+    for (long long r = 0; r < rows; ++r)
+        for (int i = 0; i < D / 2; ++i) {
+            const uint8_t b = bytes[(size_t)r * (D / 2) + i];
+            codes[(size_t)r * D + 2 * i] = b & 15;
+            codes[(size_t)r * D + 2 * i + 1] = b >> 4;
+        }
+}
+
+// out[h][:] = sum_t softmax_t( q[h] . Khat[kv(h)][t] / sqrt(D) ) * Vhat[kv(h)][t][:],  kv(h) = h / (Hq / Hkv),
+// Khat = ks * (kc - kz), Vhat likewise, everything in fp64.  Codes: one per byte, [Hkv][T][D];
+// scales and zero-points [Hkv][T].  scratch: T doubles.
+void orc_kv4_attention(const float* q, const uint8_t* kc, const float* ks, const float* kz, const uint8_t* vc,
+                       const float* vs, const float* vz, int T, int Hq, int Hkv, int D, double* out, double* scratch) {
+    const int group = Hq / Hkv;
+    const double inv = 1.0 / std::sqrt((double)D);
+    for (int h = 0; h < Hq; ++h) {
+        const int kv = h / group;
+        double m = -INFINITY;
+        for (int t = 0; t < T; ++t) {
+            const size_t row = (size_t)kv * T + t;
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d)
+                dot += (double)q[(size_t)h * D + d] * ((double)ks[row] * ((double)kc[row * D + d] - (double)kz[row]));
+            scratch[t] = dot * inv;
+            if (scratch[t] > m) m = scratch[t];
+        }
+        double den = 0.0;
+        for (int d = 0; d < D; ++d) out[(size_t)h * D + d] = 0.0;
+        for (int t = 0; t < T; ++t) {
+            const size_t row = (size_t)kv * T + t;
+            const double p = std::exp(scratch[t] - m);
+            den += p;
+            for (int d = 0; d < D; ++d)
+                out[(size_t)h * D + d] += p * ((double)vs[row] * ((double)vc[row * D + d] - (double)vz[row]));
+        }
+        for (int d = 0; d < D; ++d) out[(size_t)h * D + d] /= den;
+    }
 }
 
 }  // extern "C"

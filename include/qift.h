@@ -237,6 +237,41 @@ int qift_w2a4_linear_static(const uint32_t* packed, const float* s_n, int levels
                             const float* s_a, int M, int N, int K, void* Y, int y_dtype,
                             int32_t* acc_debug, void* stream);
 
+/* ---------------------------------------------------------------------------------------------------
+ * KV4: the 4-bit key / value cache of the paper's W2A4/KV4 setting (Sec. 4.1: "asymmetric key and value
+ * quantization with clipping ratios of 0.95") and the single-query decode attention that reads it.
+ *
+ * Cache layout (device memory, owned by the caller), head-major:
+ *   codes uint8 [H][T_cap][D/2]   two 4-bit codes per byte, even dimension in the low nibble
+ *   scale fp32  [H][T_cap]        step s of the (token, head) vector
+ *   zero  fp32  [H][T_cap]        its integer zero-point z (0..15) as a float; value = s * (code - z)
+ * D must be 128.
+ *
+ * qift_kv4_quantize: quantizes T new tokens and writes them to cache slots t0 .. t0+T-1.
+ *   X        in  [T][H][D] fp32 or bf16 (the layout a projection produces), 16-byte aligned
+ *   had_block    0 / 1: no rotation; else a power of two <= D: orthonormal blockwise Hadamard first
+ *                (keys: rotate the query the same way, e.g. with qift_rotate)
+ *   clip         clipping ratio in (0, 1]; the paper uses 0.95
+ *   per vector: lo = clip * min(0, min x), hi = clip * max(0, max x), s = (hi - lo) / 15 (1 if hi == lo),
+ *   z = rint(-lo / s), code = clamp(rint(x / s) + z, 0, 15); fp32, IEEE division, round half to even.
+ *
+ * qift_kv4_attention_decode: out[h] = sum_t softmax_t(q[h] . K[t] / sqrt(D)) V[t] over tokens 0 .. T-1 of
+ * KV head h / (Hq / Hkv), K and V dequantized on the fly; fp32 arithmetic.
+ *   q        in  [Hq][D] fp32, in the basis the keys were quantized in
+ *   out      out [Hq][D] fp32
+ *   Hq / Hkv     1, 2, 4 or 8
+ *   workspace    >= qift_kv4_attention_workspace_bytes(T, Hq, Hkv) bytes, 16-byte aligned: partial results
+ *                of the token splits (two launches: partial attention per split, then the merge)
+ * Errors: INVALID_ARG (null pointer, T <= 0, T > T_cap, clip outside (0,1]), UNSUPPORTED_SHAPE (D != 128,
+ * head ratio, had_block), ALIGNMENT, WORKSPACE, CUDA. */
+int qift_kv4_quantize(const void* X, int x_dtype, int T, int H, int D, int had_block, float clip_ratio, int t0,
+                      int T_cap, uint8_t* codes, float* scale, float* zero, void* stream);
+size_t qift_kv4_attention_workspace_bytes(int T, int Hq, int Hkv);
+int qift_kv4_attention_decode(const float* q, const uint8_t* k_codes, const float* k_scale, const float* k_zero,
+                              const uint8_t* v_codes, const float* v_scale, const float* v_zero, int T, int T_cap,
+                              int Hq, int Hkv, int D, float* out, void* workspace, size_t workspace_bytes,
+                              void* stream);
+
 /* Synchronizes `stream`, then reads and clears the device status word in which a kernel records an
  * expired bounded wait.  QIFT_OK, QIFT_ERR_TIMEOUT or QIFT_ERR_CUDA.  `detail` (host, may be NULL)
  * receives the raw word: bits 0-7 the waiting site, the rest the block index. */

@@ -28,6 +28,7 @@ EXPORTS = [
     "qift_linear_route", "qift_device_status", "qift_forward_scratch_bytes", "qift_forward", "qift_forward_host",
     "qift_group_plan_bytes", "qift_group_plan", "qift_group_quantize_act", "qift_group_linear", "qift_group_forward",
     "qift_group_forward_host", "qift_static_scratch_bytes", "qift_w2a4_linear_static",
+    "qift_kv4_quantize", "qift_kv4_attention_workspace_bytes", "qift_kv4_attention_decode",
 ]
 
 _lib = None
@@ -79,10 +80,14 @@ def lib() -> ctypes.CDLL:
         L.qift_static_scratch_bytes.restype = sz
         L.qift_static_scratch_bytes.argtypes = []
         L.qift_w2a4_linear_static.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, vp, ci, vp, vp]
+        L.qift_kv4_quantize.argtypes = [vp, ci, ci, ci, ci, ci, cf, ci, ci, vp, vp, vp, vp]
+        L.qift_kv4_attention_workspace_bytes.restype = sz
+        L.qift_kv4_attention_workspace_bytes.argtypes = [ci, ci, ci]
+        L.qift_kv4_attention_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, vp, vp, sz, vp]
         for name in EXPORTS:
             if name not in ("qift_status_string", "qift_packed_bytes", "qift_workspace_bytes",
                             "qift_forward_scratch_bytes", "qift_group_plan_bytes", "qift_static_scratch_bytes",
-                            "qift_workspace_bytes_route"):
+                            "qift_workspace_bytes_route", "qift_kv4_attention_workspace_bytes"):
                 getattr(L, name).restype = ci
         _lib = L
     return _lib
@@ -372,3 +377,44 @@ def qift_group_forward_host(plan: GroupPlan):
                                          plan.x_arena.data_ptr(), plan.x_arena.numel(), plan.y_arena.data_ptr(),
                                          plan.y_host.data_ptr(), plan.y_arena.numel(), _stream()), "qift_group_forward_host")
     return plan.y_host
+
+
+# ---------------------------------------------------------------------------------------- KV4
+class Kv4Cache:
+    """Device buffers of a 4-bit cache for one of K or V: codes uint8 [H, T_cap, D/2], scale / zero fp32 [H, T_cap]."""
+
+    def __init__(self, H: int, T_cap: int, D: int = 128, device="cuda"):
+        self.H, self.T_cap, self.D = H, T_cap, D
+        self.codes = torch.zeros((H, T_cap, D // 2), dtype=torch.uint8, device=device)
+        self.scale = torch.zeros((H, T_cap), dtype=torch.float32, device=device)
+        self.zero = torch.zeros((H, T_cap), dtype=torch.float32, device=device)
+
+
+def qift_kv4_quantize(X, cache: Kv4Cache, t0: int = 0, had_block: int = 0, clip_ratio: float = 0.95):
+    """X fp32 or bf16 [T, H, D] -> written into cache slots t0 .. t0+T-1."""
+    _dev(X)
+    assert X.dtype in (torch.float32, torch.bfloat16)
+    T, H, D = X.shape
+    _check(lib().qift_kv4_quantize(_ptr(X), F32 if X.dtype == torch.float32 else BF16, T, H, D, had_block, clip_ratio, t0,
+                                   cache.T_cap, _ptr(cache.codes), _ptr(cache.scale), _ptr(cache.zero), _stream()),
+           "qift_kv4_quantize")
+    return cache
+
+
+def qift_kv4_attention_workspace_bytes(T: int, Hq: int, Hkv: int) -> int:
+    return int(lib().qift_kv4_attention_workspace_bytes(T, Hq, Hkv))
+
+
+def qift_kv4_attention_decode(q, K: Kv4Cache, V: Kv4Cache, T: int, out=None, workspace=None):
+    """q fp32 [Hq, D] -> out fp32 [Hq, D]: softmax(q K^T / sqrt(D)) V over the first T cached tokens."""
+    _dev(q, torch.float32)
+    Hq, D = q.shape
+    if out is None:
+        out = torch.empty((Hq, D), dtype=torch.float32, device=q.device)
+    need = qift_kv4_attention_workspace_bytes(T, Hq, K.H)
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)
+    _check(lib().qift_kv4_attention_decode(_ptr(q), _ptr(K.codes), _ptr(K.scale), _ptr(K.zero), _ptr(V.codes), _ptr(V.scale),
+                                           _ptr(V.zero), T, K.T_cap, Hq, K.H, D, _ptr(_dev(out, torch.float32)),
+                                           _ptr(workspace), workspace.numel(), _stream()), "qift_kv4_attention_decode")
+    return out

@@ -364,6 +364,7 @@ def run_gpu(args):
     if rank == 0 and world == 1 and not args.no_prefill:
         out["mixed_stack"] = run_mixed_stack(torch, qift, L, device, gen, args)
         out["prefill"] = run_prefill(torch, qift, L, device, gen, pk)
+        out["kv4"] = run_kv4(torch, qift, L, pk)
     if rank == 0 and world == 1 and not args.no_cpu:
         out["cpu_baseline"] = cpu_baseline(budget_s=12.0)
     if rank == 0:
@@ -407,6 +408,67 @@ def run_mixed_stack(torch, qift, L, device, gen, args):
             "ms_per_step": round(ms, 5), "tokens_per_s": round(1.0 / (ms * 1e-3), 1),
             "value": round(algo / (ms * 1e-3) / 1e9, 2), "unit": "GB/s", "algorithmic_bytes_per_step": algo,
             "pct_of_8TBs": round(100 * algo / (ms * 1e-3) / 8e12, 2)}
+
+
+def run_kv4(torch, qift, L, pk):
+    """KV4 cache path: decode attention over a 4-bit cache (LLaMA-3.1-8B heads: 32 query / 8 KV heads of 128, 32768
+    cached tokens, 32 layers of distinct caches = 1.2 GB) and the cache quantizer.  Bytes = codes + scales + zero-points."""
+    vp = ctypes.c_void_p
+    T, Hq, Hkv, D, layers = 32768, 32, 8, 128, 32
+    caches = []
+    for _ in range(layers):
+        K, V = qift.Kv4Cache(Hkv, T), qift.Kv4Cache(Hkv, T)
+        for c in (K, V):
+            c.codes.random_(0, 256)
+            c.scale.uniform_(0.05, 0.2)
+            c.zero.random_(0, 16)
+        caches.append((K, V))
+    q = torch.randn(Hq, D, device="cuda")
+    o = torch.empty(Hq, D, device="cuda")
+    ws = torch.empty(qift.qift_kv4_attention_workspace_bytes(T, Hq, Hkv), dtype=torch.uint8, device="cuda")
+    st = vp(torch.cuda.current_stream().cuda_stream)
+
+    def step():
+        for K, V in caches:
+            rc = L.qift_kv4_attention_decode(vp(q.data_ptr()), vp(K.codes.data_ptr()), vp(K.scale.data_ptr()), vp(K.zero.data_ptr()),
+                                             vp(V.codes.data_ptr()), vp(V.scale.data_ptr()), vp(V.zero.data_ptr()), T, T, Hq, Hkv, D,
+                                             vp(o.data_ptr()), vp(ws.data_ptr()), ws.numel(), st)
+            assert rc == 0, rc
+
+    def timed(fn, n):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    ms = timed(step, 5)
+    cache_bytes = layers * 2 * Hkv * T * (D // 2 + 8)
+    gbs = cache_bytes / (ms * 1e-3) / 1e9
+    # quantizer: 8192 new tokens of all 8 KV heads (bf16 in), with the head-dimension rotation
+    x = torch.randn(8192, Hkv, D, device="cuda", dtype=torch.bfloat16)
+    Kq = qift.Kv4Cache(Hkv, 8192)
+
+    def quant():
+        rc = L.qift_kv4_quantize(vp(x.data_ptr()), qift.BF16, 8192, Hkv, D, D, ctypes.c_float(0.95), 0, 8192,
+                                 vp(Kq.codes.data_ptr()), vp(Kq.scale.data_ptr()), vp(Kq.zero.data_ptr()), st)
+        assert rc == 0, rc
+
+    msq = timed(quant, 20)
+    qbytes = 8192 * Hkv * (2 * D + D // 2 + 8)
+    return {"workload": f"decode attention over a KV4 cache: {Hq} query / {Hkv} KV heads x {D}, {T} cached tokens, {layers} layers of "
+                        "distinct caches (two launches per layer)", "us_per_layer": round(ms * 1e3 / layers, 2),
+            "value": round(gbs, 1), "unit": "GB/s", "algorithmic_bytes_per_layer": cache_bytes // layers,
+            "roofline": {"bound": "alu", "kernel": "kv4_attention_partial_kernel", "achieved": round(gbs, 1), "peak": pk["hbm_gbs"],
+                         "unit": "GB/s", "frac": round(gbs / pk["hbm_gbs"], 4),
+                         "note": "fp32 SIMT dequantize-and-accumulate: instruction-issue bound, reported against the HBM peak it would have to reach"},
+            "quantizer": {"workload": "8192 tokens x 8 heads x 128, bf16 in, Hadamard over the head dimension", "us": round(msq * 1e3, 2),
+                          "value": round(qbytes / (msq * 1e-3) / 1e9, 1), "unit": "GB/s"}}
 
 
 def int8_library_point(torch, M, shapes, device):

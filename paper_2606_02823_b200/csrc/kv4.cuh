@@ -98,8 +98,10 @@ kv4_quantize_kernel(const void* __restrict__ X, long long rows, int H, int had_b
 // out[h] = sum_t softmax_t(q[h] . Khat[t] / sqrt(D)) Vhat[t],  Khat = ks (kc - kz),  Vhat = vs (vc - vz),
 // for the G = Hq / Hkv query heads that share a KV head.  fp32 throughout.
 //
-// Grid (splits, Hkv): a CTA takes a contiguous range of tokens of one KV head; eight warps take
-// tiles of four tokens in turn.  A lane is (token j of the tile, 16-dimension chunk c): it loads the 8
+// Grid (head groups, splits, Hkv): a CTA takes a contiguous range of tokens of one KV head for G of the
+// query heads that share it (G <= 2: more accumulators per thread would leave one CTA per SM; the head
+// groups of a split run side by side and the second finds the codes in L2); eight warps take runs of
+// four-token tiles in turn.  A lane is (token j of the tile, 16-dimension chunk c): it loads the 8
 // bytes of codes of its chunk (a warp reads 256 contiguous bytes), turns them into floats ONCE and
 // uses them for all G heads.  The zero-points never touch the per-element path:
 //   q . Khat = ks (sum_d c_d q_d - kz sum_d q_d),     sum_t w_t Vhat_t = sum_t w_t vs_t c_t - (sum_t w_t vs_t vz_t).
@@ -116,10 +118,12 @@ struct Kv4Params {
     float* partial;  // [Hq][splits][D + 2]: numerator, running max, denominator
     float* out;      // [Hq][D]
     int T, T_cap, Hq, Hkv, splits, tokens_per_split;
+    int heads_per_kv;  // Hq / Hkv
     float inv_sqrt_d;
 };
 
 constexpr int kKvWarps = 8;
+constexpr int kKvUnroll = 2;  // four-token tiles a warp loads ahead (more costs the second CTA per SM)
 constexpr int kKvPartial = kKvD + 2;
 
 // Eight codes of a 32-bit word as floats: 2^23 + c has the code in its low mantissa bits.
@@ -144,12 +148,13 @@ kv4_attention_partial_kernel(const Kv4Params p) {
     __shared__ float red[kKvWarps][G][kKvPartial];
     pdl_launch_dependents();
     pdl_wait();
-    const int kv = blockIdx.y, split = blockIdx.x;
+    const int kv = blockIdx.z, split = blockIdx.y;
+    const int head0 = kv * p.heads_per_kv + blockIdx.x * G;  // first query head of this CTA
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int j = lane >> 3, c = lane & 7;
 
     for (int i = threadIdx.x; i < G * kKvD; i += blockDim.x)
-        qs[i / kKvD][i % kKvD] = __fmul_rn(p.q[static_cast<size_t>(kv * G) * kKvD + i], p.inv_sqrt_d);
+        qs[i / kKvD][i % kKvD] = __fmul_rn(p.q[static_cast<size_t>(head0) * kKvD + i], p.inv_sqrt_d);
     __syncthreads();
     if (threadIdx.x < G * 8) {
         const int g = threadIdx.x >> 3, cc = threadIdx.x & 7;
@@ -171,53 +176,65 @@ kv4_attention_partial_kernel(const Kv4Params p) {
         for (int i = 0; i < 16; ++i) acc[g][i] = 0.0f;
     }
 
-    for (int t0 = t_begin + 4 * warp; t0 < t_end; t0 += 4 * kKvWarps) {
-        const int t = t0 + j;
-        const bool valid = t < t_end;
-        const size_t row = head_row + (valid ? t : t_begin);
-        const uint2 kw = *reinterpret_cast<const uint2*>(p.k_codes + row * kKvRowBytes + 8 * c);
-        const uint2 vw = *reinterpret_cast<const uint2*>(p.v_codes + row * kKvRowBytes + 8 * c);
-        const float ks = p.k_scale[row], kz = p.k_zero[row], vs = p.v_scale[row], vz = p.v_zero[row];
-        float kd[16], vd[16];
-        {
-            float a[8], b[8];
-            nibbles_to_floats(kw.x, a), nibbles_to_floats(kw.y, b);
+    // kKvUnroll tiles per trip, all their loads issued before the first is used (a warp otherwise waits
+    // out the full memory latency once per tile)
+    for (int tb = t_begin + 4 * kKvUnroll * warp; tb < t_end; tb += 4 * kKvUnroll * kKvWarps) {
+        uint2 kw[kKvUnroll], vw[kKvUnroll];
+        float ks[kKvUnroll], kz[kKvUnroll], vs[kKvUnroll], vz[kKvUnroll];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) kd[i] = a[i], kd[8 + i] = b[i];
-            nibbles_to_floats(vw.x, a), nibbles_to_floats(vw.y, b);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) vd[i] = a[i], vd[8 + i] = b[i];
+        for (int u = 0; u < kKvUnroll; ++u) {
+            const int t = tb + 4 * u + j;
+            const size_t row = head_row + (t < t_end ? t : t_begin);
+            kw[u] = *reinterpret_cast<const uint2*>(p.k_codes + row * kKvRowBytes + 8 * c);
+            vw[u] = *reinterpret_cast<const uint2*>(p.v_codes + row * kKvRowBytes + 8 * c);
+            ks[u] = p.k_scale[row], kz[u] = p.k_zero[row], vs[u] = p.v_scale[row], vz[u] = p.v_zero[row];
         }
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const float4* qv = reinterpret_cast<const float4*>(&qs[g][16 * c]);
-            float part = 0.0f;
+        for (int u = 0; u < kKvUnroll; ++u) {
+            if (tb + 4 * u >= t_end) break;  // warp-uniform: no token of this tile exists
+            const bool valid = tb + 4 * u + j < t_end;
+            float kd[16], vd[16];
+            {
+                float a[8], b[8];
+                nibbles_to_floats(kw[u].x, a), nibbles_to_floats(kw[u].y, b);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float4 f = qv[i];
-                part = fmaf(kd[4 * i], f.x, part), part = fmaf(kd[4 * i + 1], f.y, part);
-                part = fmaf(kd[4 * i + 2], f.z, part), part = fmaf(kd[4 * i + 3], f.w, part);
+                for (int i = 0; i < 8; ++i) kd[i] = a[i], kd[8 + i] = b[i];
+                nibbles_to_floats(vw[u].x, a), nibbles_to_floats(vw[u].y, b);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) vd[i] = a[i], vd[8 + i] = b[i];
             }
-            part = fmaf(-kz, qsum[g][c], part);
-            part += __shfl_xor_sync(0xffffffffu, part, 1);
-            part += __shfl_xor_sync(0xffffffffu, part, 2);
-            part += __shfl_xor_sync(0xffffffffu, part, 4);
-            const float score = valid ? ks * part : -INFINITY;
-            float tmax = fmaxf(score, __shfl_xor_sync(0xffffffffu, score, 8));
-            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 16));
-            if (tmax > m[g]) {  // warp-uniform: rescale what has been accumulated so far
-                const float corr = expf(m[g] - tmax);  // exp(-inf) = 0 on the first tile
-                l[g] *= corr, zacc[g] *= corr;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) acc[g][i] *= corr;
-                m[g] = tmax;
+            for (int g = 0; g < G; ++g) {
+                const float4* qv = reinterpret_cast<const float4*>(&qs[g][16 * c]);
+                float p0 = 0.0f, p1 = 0.0f, p2 = 0.0f, p3 = 0.0f;  // four independent chains
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float4 f = qv[i];
+                    p0 = fmaf(kd[4 * i], f.x, p0), p1 = fmaf(kd[4 * i + 1], f.y, p1);
+                    p2 = fmaf(kd[4 * i + 2], f.z, p2), p3 = fmaf(kd[4 * i + 3], f.w, p3);
+                }
+                float part = (p0 + p1) + (p2 + p3);
+                part = fmaf(-kz[u], qsum[g][c], part);
+                part += __shfl_xor_sync(0xffffffffu, part, 1);
+                part += __shfl_xor_sync(0xffffffffu, part, 2);
+                part += __shfl_xor_sync(0xffffffffu, part, 4);
+                const float score = valid ? ks[u] * part : -INFINITY;
+                float tmax = fmaxf(score, __shfl_xor_sync(0xffffffffu, score, 8));
+                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 16));
+                if (tmax > m[g]) {  // warp-uniform: rescale what has been accumulated so far
+                    const float corr = expf(m[g] - tmax);  // exp(-inf) = 0 on the first tile
+                    l[g] *= corr, zacc[g] *= corr;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) acc[g][i] *= corr;
+                    m[g] = tmax;
+                }
+                const float pr = valid ? expf(score - m[g]) : 0.0f;
+                const float w = pr * vs[u];
+                l[g] += pr;
+                zacc[g] = fmaf(w, vz[u], zacc[g]);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[g][i] = fmaf(w, vd[i], acc[g][i]);
             }
-            const float pr = valid ? expf(score - m[g]) : 0.0f;
-            const float w = pr * vs;
-            l[g] += pr;
-            zacc[g] = fmaf(w, vz, zacc[g]);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) acc[g][i] = fmaf(w, vd[i], acc[g][i]);
         }
     }
 
@@ -252,7 +269,7 @@ kv4_attention_partial_kernel(const Kv4Params p) {
                 if (mw > -INFINITY) val = fmaf(red[w][g][d], expf(mw - mm), val);
             }
         }
-        p.partial[(static_cast<size_t>(kv * G + g) * p.splits + split) * kKvPartial + d] = val;
+        p.partial[(static_cast<size_t>(head0 + g) * p.splits + split) * kKvPartial + d] = val;
     }
 }
 

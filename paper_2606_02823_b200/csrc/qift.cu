@@ -833,18 +833,19 @@ namespace {
 // Token splits of the decode attention: enough CTAs for a few per SM, whole 32-token rounds of the
 // eight warps per split.
 void kv4_splits(int T, int Hkv, int* splits, int* tokens_per_split) {
-    int want = (4 * sm_count() + Hkv - 1) / Hkv;
+    int want = (2 * sm_count() + Hkv - 1) / Hkv;
     if (want < 1) want = 1;
     int tps = (T + want - 1) / want;
-    tps = ((tps + 31) / 32) * 32;
-    if (tps < 128) tps = 128;
+    const int round = 4 * kKvUnroll * kKvWarps;  // tokens the eight warps take per trip
+    tps = ((tps + round - 1) / round) * round;
     *tokens_per_split = tps;
     *splits = (T + tps - 1) / tps;
 }
 
-template <int G>
+template <int G>  // query heads per CTA
 int launch_kv4_attention(const Kv4Params& p, cudaStream_t st) {
-    int rc = cuda_status(launch_pdl(kv4_attention_partial_kernel<G>, dim3(p.splits, p.Hkv), dim3(32 * kKvWarps), 0, st, p));
+    int rc = cuda_status(launch_pdl(kv4_attention_partial_kernel<G>, dim3(p.heads_per_kv / G, p.splits, p.Hkv),
+                                    dim3(32 * kKvWarps), 0, st, p));
     if (rc != QIFT_OK) return rc;
     return cuda_status(launch_pdl(kv4_attention_combine_kernel, dim3(p.Hq), dim3(kKvD), 0, st, p));
 }
@@ -898,12 +899,8 @@ int qift_kv4_attention_decode(const float* q, const uint8_t* k_codes, const floa
     p.T = T, p.T_cap = T_cap, p.Hq = Hq, p.Hkv = Hkv;
     p.inv_sqrt_d = static_cast<float>(1.0 / std::sqrt(static_cast<double>(D)));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    switch (G) {
-        case 1: return launch_kv4_attention<1>(p, st);
-        case 2: return launch_kv4_attention<2>(p, st);
-        case 4: return launch_kv4_attention<4>(p, st);
-        default: return launch_kv4_attention<8>(p, st);
-    }
+    p.heads_per_kv = G;
+    return (G == 1) ? launch_kv4_attention<1>(p, st) : launch_kv4_attention<2>(p, st);
 }
 
 }  // extern "C"

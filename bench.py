@@ -377,8 +377,8 @@ def run_mixed_stack(torch, qift, L, device, gen, args):
     """Config 5: layer-wise mixed precision on LLaMA-2-7B shapes at M = 1: layers 0..15 INT4 weights (W4A4),
     layers 16..31 MNZ (W2A4), 3 bits per weight on average.  Two grouped plans (a plan holds one level set):
     four launches per token-step.  Modules run on their own staged inputs, as in the headline."""
-    n4 = args.layers // 2
-    n2 = args.layers - n4
+    n4 = max(1, args.layers // 2)
+    n2 = max(1, args.layers - n4)
     vp = ctypes.c_void_p
     plans, algo = [], 0
     for lv, n in ((qift.INT4, n4), (qift.MNZ, n2)):

@@ -440,7 +440,7 @@ def run_kv4(torch, qift, L, pk):
     T, Hq, Hkv, D, layers = 32768, 32, 8, 128, 32
     caches = []
     for _ in range(layers):
-        K, V = qift.Kv4Cache(Hkv, T), qift.Kv4Cache(Hkv, T)
+        K, V = qift.Kv4Cache(Hkv, T), qift.Kv4Cache(Hkv, T, qift.KV_VALUES)
         for c in (K, V):
             c.codes.random_(0, 256)
             c.scale.uniform_(0.05, 0.2)
@@ -478,7 +478,7 @@ def run_kv4(torch, qift, L, pk):
     Kq = qift.Kv4Cache(Hkv, 8192)
 
     def quant():
-        rc = L.qift_kv4_quantize(vp(x.data_ptr()), qift.BF16, 8192, Hkv, D, D, ctypes.c_float(0.95), 0, 8192,
+        rc = L.qift_kv4_quantize(vp(x.data_ptr()), qift.BF16, 8192, Hkv, D, D, ctypes.c_float(0.95), 0, 8192, qift.KV_KEYS,
                                  vp(Kq.codes.data_ptr()), vp(Kq.scale.data_ptr()), vp(Kq.zero.data_ptr()), st)
         assert rc == 0, rc
 
@@ -487,9 +487,10 @@ def run_kv4(torch, qift, L, pk):
     return {"workload": f"decode attention over a KV4 cache: {Hq} query / {Hkv} KV heads x {D}, {T} cached tokens, {layers} layers of "
                         "distinct caches (two launches per layer)", "us_per_layer": round(ms * 1e3 / layers, 2),
             "value": round(gbs, 1), "unit": "GB/s", "algorithmic_bytes_per_layer": cache_bytes // layers,
-            "roofline": {"bound": "alu", "kernel": "kv4_attention_partial_kernel", "achieved": round(gbs, 1), "peak": pk["hbm_gbs"],
+            "roofline": {"bound": "hbm", "kernel": "kv4_attention_partial_kernel", "achieved": round(gbs, 1), "peak": pk["hbm_gbs"],
                          "unit": "GB/s", "frac": round(gbs / pk["hbm_gbs"], 4),
-                         "note": "fp32 SIMT dequantize-and-accumulate: instruction-issue bound, reported against the HBM peak it would have to reach"},
+                         "note": "both products on mma.sync fp16 with fp32 accumulators; the unpacking of the codes into operand "
+                                 "registers keeps it instruction-bound above its memory time"},
             "quantizer": {"workload": "8192 tokens x 8 heads x 128, bf16 in, Hadamard over the head dimension", "us": round(msq * 1e3, 2),
                           "value": round(qbytes / (msq * 1e-3) / 1e9, 1), "unit": "GB/s"}}
 

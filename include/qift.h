@@ -241,13 +241,15 @@ int qift_w2a4_linear_static(const uint32_t* packed, const float* s_n, int levels
  * KV4: the 4-bit key / value cache of the paper's W2A4/KV4 setting (Sec. 4.1: "asymmetric key and value
  * quantization with clipping ratios of 0.95") and the single-query decode attention that reads it.
  *
- * Cache layout (device memory, owned by the caller), head-major:
- *   codes uint8 [H][T_cap][D/2]   two 4-bit codes per byte, even dimension in the low nibble
- *   scale fp32  [H][T_cap]        step s of the (token, head) vector
- *   zero  fp32  [H][T_cap]        its integer zero-point z (0..15) as a float; value = s * (code - z)
- * D must be 128.
+ * Cache layout (device memory, owned by the caller), head-major, T_cap even:
+ *   key codes   uint8 [H][T_cap][D/2]   two neighbouring dimensions of a token per byte (even one low)
+ *   value codes uint8 [H][T_cap/2][D]   two consecutive tokens of a dimension per byte (even one low)
+ *   scale fp32  [H][T_cap]              step s of the (token, head) vector
+ *   zero  fp32  [H][T_cap]              its integer zero-point z (0..15) as a float; value = s * (code - z)
+ * (a byte is then one tensor-core operand register of the product it feeds).  D must be 128.
  *
- * qift_kv4_quantize: quantizes T new tokens and writes them to cache slots t0 .. t0+T-1.
+ * qift_kv4_quantize: quantizes T new tokens and writes them to cache slots t0 .. t0+T-1 of a key cache
+ * (layout = QIFT_KV_KEYS) or a value cache (QIFT_KV_VALUES; a slot's partner nibble is preserved).
  *   X        in  [T][H][D] fp32 or bf16 (the layout a projection produces), 16-byte aligned
  *   had_block    0 / 1: no rotation; else a power of two <= D: orthonormal blockwise Hadamard first
  *                (keys: rotate the query the same way, e.g. with qift_rotate)
@@ -259,13 +261,14 @@ int qift_w2a4_linear_static(const uint32_t* packed, const float* s_n, int levels
  * KV head h / (Hq / Hkv), K and V dequantized on the fly; fp32 arithmetic.
  *   q        in  [Hq][D] fp32, in the basis the keys were quantized in
  *   out      out [Hq][D] fp32
- *   Hq / Hkv     1, 2, 4 or 8
+ *   Hq / Hkv     1 .. 8
  *   workspace    >= qift_kv4_attention_workspace_bytes(T, Hq, Hkv) bytes, 16-byte aligned: partial results
  *                of the token splits (two launches: partial attention per split, then the merge)
- * Errors: INVALID_ARG (null pointer, T <= 0, T > T_cap, clip outside (0,1]), UNSUPPORTED_SHAPE (D != 128,
- * head ratio, had_block), ALIGNMENT, WORKSPACE, CUDA. */
+ * Errors: INVALID_ARG (null pointer, T <= 0, T > T_cap, clip outside (0,1], layout), UNSUPPORTED_SHAPE
+ * (D != 128, odd T_cap, more than 8 query heads per KV head, had_block), ALIGNMENT, WORKSPACE, CUDA. */
+enum { QIFT_KV_KEYS = 0, QIFT_KV_VALUES = 1 };
 int qift_kv4_quantize(const void* X, int x_dtype, int T, int H, int D, int had_block, float clip_ratio, int t0,
-                      int T_cap, uint8_t* codes, float* scale, float* zero, void* stream);
+                      int T_cap, int layout, uint8_t* codes, float* scale, float* zero, void* stream);
 size_t qift_kv4_attention_workspace_bytes(int T, int Hq, int Hkv);
 int qift_kv4_attention_decode(const float* q, const uint8_t* k_codes, const float* k_scale, const float* k_zero,
                               const uint8_t* v_codes, const float* v_scale, const float* v_zero, int T, int T_cap,

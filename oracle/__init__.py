@@ -253,6 +253,18 @@ def kv4_pack(codes):
     return out.reshape(codes.shape[:-1] + (D // 2,))
 
 
+def kv4_pack_token_pairs(codes):
+    """codes uint8 [H, T, D] (T even) -> bytes uint8 [H, T/2, D]: tokens 2i (low nibble) and 2i+1 of a dimension per byte."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    H, T, D = codes.shape
+    assert T % 2 == 0
+    out = np.empty((H, T // 2, D), dtype=np.uint8)
+    vp = ctypes.c_void_p
+    for h in range(H):
+        lib().orc_kv4_pack_token_pairs(codes[h].ctypes.data_as(vp), ctypes.c_longlong(T), D, out[h].ctypes.data_as(vp))
+    return out
+
+
 def kv4_unpack(packed):
     packed = np.ascontiguousarray(packed, dtype=np.uint8)
     rows, half = packed.reshape(-1, packed.shape[-1]).shape

@@ -29,7 +29,8 @@
 //                        more, so the rest is the usual asymmetric integer quantizer: one
 //                        (scale, zero-point) pair per token and head over the head dimension, the
 //                        range [min(x,0), max(x,0)] shrunk by the clipping ratio, 16 levels.
-//   orc_kv4_pack/unpack  two 4-bit codes per byte, even dimension in the low nibble.
+//   orc_kv4_pack/unpack  two 4-bit codes per byte, even dimension in the low nibble (keys);
+//   orc_kv4_pack_token_pairs  values: two consecutive tokens of a dimension per byte (layout is the build's).
 //   orc_kv4_attention    single-query scaled dot-product attention over the dequantized cache (the
 //                        decode step whose memory traffic Sec. 1 calls the bottleneck), in fp64.
 //
@@ -383,6 +384,14 @@ void orc_kv4_pack(const uint8_t* codes, long long rows, int D, uint8_t* bytes) {
         for (int i = 0; i < D / 2; ++i)
             bytes[(size_t)r * (D / 2) + i] =
                 (uint8_t)(codes[(size_t)r * D + 2 * i] | (codes[(size_t)r * D + 2 * i + 1] << 4));
+}
+
+// Value-cache byte order: the codes of two CONSECUTIVE TOKENS of one head at the same dimension share a
+// byte (even token in the low nibble).  codes: [T][D] of one head, T even; bytes: [T/2][D].
+void orc_kv4_pack_token_pairs(const uint8_t* codes, long long T, int D, uint8_t* bytes) {
+    for (long long i = 0; i < T / 2; ++i)
+        for (int d = 0; d < D; ++d)
+            bytes[(size_t)i * D + d] = (uint8_t)(codes[(size_t)(2 * i) * D + d] | (codes[(size_t)(2 * i + 1) * D + d] << 4));
 }
 
 void orc_kv4_unpack(const uint8_t* bytes, long long rows, int D, uint8_t* codes) {

@@ -80,7 +80,7 @@ def lib() -> ctypes.CDLL:
         L.qift_static_scratch_bytes.restype = sz
         L.qift_static_scratch_bytes.argtypes = []
         L.qift_w2a4_linear_static.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, vp, ci, vp, vp]
-        L.qift_kv4_quantize.argtypes = [vp, ci, ci, ci, ci, ci, cf, ci, ci, vp, vp, vp, vp]
+        L.qift_kv4_quantize.argtypes = [vp, ci, ci, ci, ci, ci, cf, ci, ci, ci, vp, vp, vp, vp]
         L.qift_kv4_attention_workspace_bytes.restype = sz
         L.qift_kv4_attention_workspace_bytes.argtypes = [ci, ci, ci]
         L.qift_kv4_attention_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, vp, vp, sz, vp]
@@ -380,12 +380,18 @@ def qift_group_forward_host(plan: GroupPlan):
 
 
 # ---------------------------------------------------------------------------------------- KV4
-class Kv4Cache:
-    """Device buffers of a 4-bit cache for one of K or V: codes uint8 [H, T_cap, D/2], scale / zero fp32 [H, T_cap]."""
+KV_KEYS, KV_VALUES = 0, 1
 
-    def __init__(self, H: int, T_cap: int, D: int = 128, device="cuda"):
-        self.H, self.T_cap, self.D = H, T_cap, D
-        self.codes = torch.zeros((H, T_cap, D // 2), dtype=torch.uint8, device=device)
+
+class Kv4Cache:
+    """Device buffers of a 4-bit cache for keys (codes uint8 [H, T_cap, D/2], two dimensions per byte) or values
+    (codes uint8 [H, T_cap/2, D], two tokens per byte); scale / zero fp32 [H, T_cap].  T_cap even."""
+
+    def __init__(self, H: int, T_cap: int, layout: int = KV_KEYS, D: int = 128, device="cuda"):
+        assert T_cap % 2 == 0
+        self.H, self.T_cap, self.D, self.layout = H, T_cap, D, layout
+        shape = (H, T_cap, D // 2) if layout == KV_KEYS else (H, T_cap // 2, D)
+        self.codes = torch.zeros(shape, dtype=torch.uint8, device=device)
         self.scale = torch.zeros((H, T_cap), dtype=torch.float32, device=device)
         self.zero = torch.zeros((H, T_cap), dtype=torch.float32, device=device)
 
@@ -396,7 +402,7 @@ def qift_kv4_quantize(X, cache: Kv4Cache, t0: int = 0, had_block: int = 0, clip_
     assert X.dtype in (torch.float32, torch.bfloat16)
     T, H, D = X.shape
     _check(lib().qift_kv4_quantize(_ptr(X), F32 if X.dtype == torch.float32 else BF16, T, H, D, had_block, clip_ratio, t0,
-                                   cache.T_cap, _ptr(cache.codes), _ptr(cache.scale), _ptr(cache.zero), _stream()),
+                                   cache.T_cap, cache.layout, _ptr(cache.codes), _ptr(cache.scale), _ptr(cache.zero), _stream()),
            "qift_kv4_quantize")
     return cache
 

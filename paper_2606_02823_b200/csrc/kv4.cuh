@@ -2,10 +2,14 @@
 // clipping ratios of 0.95") and the single-query decode attention that reads it.
 //
 // Cache layout (device memory, owned by the caller), head-major so that the tokens of one KV head are
-// contiguous:  codes uint8 [Hkv][T_cap][D/2] (two codes per byte, even dimension in the low nibble),
-// scale fp32 [Hkv][T_cap], zero fp32 [Hkv][T_cap] (the integer zero-point 0..15 as a float).
+// contiguous.  Keys: codes uint8 [Hkv][T_cap][D/2], two neighbouring dimensions of a token per byte
+// (even dimension in the low nibble).  Values: codes uint8 [Hkv][T_cap/2][D], two consecutive tokens
+// of a dimension per byte (even token in the low nibble).  Both: scale fp32 [Hkv][T_cap], zero fp32
+// [Hkv][T_cap] (the integer zero-point 0..15 as a float).  T_cap is even.
 // D = 128 (the head dimension of the LLaMA models the paper evaluates).
 #pragma once
+
+#include <cuda_fp16.h>
 
 #include "common.cuh"
 
@@ -22,27 +26,14 @@ constexpr int kKvRowBytes = kKvD / 2;
 // element of a pair takes a + b, the upper a - b, exactly the operands of the in-place butterfly, so
 // the result is bit-identical to it.  Then one multiply by 1/sqrt(B) (orthonormal: queries carry no
 // per-vector scale the factor could be folded into).
-template <bool BF16_IN>
-__global__ void __launch_bounds__(256)
-kv4_quantize_kernel(const void* __restrict__ X, long long rows, int H, int had_block, float inv_sqrt_b, float clip, int t0,
-                    int T_cap, uint8_t* __restrict__ codes, float* __restrict__ scale, float* __restrict__ zero) {
-    pdl_launch_dependents();
-    pdl_wait();
-    const int lane = threadIdx.x & 31;
-    const long long r = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);  // input row = token * H + head
-    if (r >= rows) return;
-    float v[4];
-    if constexpr (BF16_IN) {
-        const uint2 w = reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(X) + r * kKvD)[lane];
-        v[0] = __uint_as_float(w.x << 16), v[1] = __uint_as_float(w.x & 0xffff0000u);
-        v[2] = __uint_as_float(w.y << 16), v[3] = __uint_as_float(w.y & 0xffff0000u);
-    } else {
-        const float4 f = reinterpret_cast<const float4*>(static_cast<const float*>(X) + r * kKvD)[lane];
-        v[0] = f.x, v[1] = f.y, v[2] = f.z, v[3] = f.w;
-    }
+// Quantizes the vector whose four elements per lane are in v (rotating it first when had_block > 1);
+// returns the lane's four codes in the low 16 bits (element e at bits 4e) and the vector's scale and
+// zero-point.
+__device__ __forceinline__ uint32_t kv4_quantize_vector(float (&v)[4], int lane, int had_block, float inv_sqrt_b, float clip, float& s,
+                                                        float& z) {
     if (had_block > 1) {
         // element index = 4 * lane + e; strides below had_block only
-        if (had_block > 1) {
+        {
             const float a0 = v[0], a1 = v[1], a2 = v[2], a3 = v[3];
             v[0] = __fadd_rn(a0, a1), v[1] = __fsub_rn(a0, a1), v[2] = __fadd_rn(a2, a3), v[3] = __fsub_rn(a2, a3);
         }
@@ -70,7 +61,7 @@ kv4_quantize_kernel(const void* __restrict__ X, long long rows, int H, int had_b
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     }
     const float lo = __fmul_rn(mn, clip), hi = __fmul_rn(mx, clip);
-    float s = 1.0f, z = 0.0f;
+    s = 1.0f, z = 0.0f;
     if (hi != lo) {
         s = __fdiv_rn(__fsub_rn(hi, lo), 15.0f);
         z = rintf(__fdiv_rn(-lo, s));
@@ -82,6 +73,34 @@ kv4_quantize_kernel(const void* __restrict__ X, long long rows, int H, int had_b
         const int c = max(0, min(15, __float2int_rn(__fdiv_rn(v[e], s)) + zi));
         packed |= static_cast<uint32_t>(c) << (4 * e);
     }
+    return packed;
+}
+
+template <bool BF16_IN>
+__device__ __forceinline__ void kv4_load_vector(const void* X, long long r, int lane, float (&v)[4]) {
+    if constexpr (BF16_IN) {
+        const uint2 w = reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(X) + r * kKvD)[lane];
+        v[0] = __uint_as_float(w.x << 16), v[1] = __uint_as_float(w.x & 0xffff0000u);
+        v[2] = __uint_as_float(w.y << 16), v[3] = __uint_as_float(w.y & 0xffff0000u);
+    } else {
+        const float4 f = reinterpret_cast<const float4*>(static_cast<const float*>(X) + r * kKvD)[lane];
+        v[0] = f.x, v[1] = f.y, v[2] = f.z, v[3] = f.w;
+    }
+}
+
+// Keys: one warp per (token, head); byte = two neighbouring dimensions.
+template <bool BF16_IN>
+__global__ void __launch_bounds__(256)
+kv4_quantize_kernel(const void* __restrict__ X, long long rows, int H, int had_block, float inv_sqrt_b, float clip, int t0,
+                    int T_cap, uint8_t* __restrict__ codes, float* __restrict__ scale, float* __restrict__ zero) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const long long r = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);  // input row = token * H + head
+    if (r >= rows) return;
+    float v[4], s, z;
+    kv4_load_vector<BF16_IN>(X, r, lane, v);
+    const uint32_t packed = kv4_quantize_vector(v, lane, had_block, inv_sqrt_b, clip, s, z);
     const long long t = r / H;
     const int h = static_cast<int>(r - t * H);
     const size_t slot = static_cast<size_t>(h) * T_cap + t0 + t;
@@ -92,21 +111,74 @@ kv4_quantize_kernel(const void* __restrict__ X, long long rows, int H, int had_b
     }
 }
 
+// Values: one warp per (pair of consecutive cache slots, head); byte = the two tokens of the pair at one
+// dimension (even slot in the low nibble), bytes [H][T_cap / 2][D].  A slot of the pair that is not
+// among the T new tokens keeps its nibble (no other warp of the launch touches the pair).
+template <bool BF16_IN>
+__global__ void __launch_bounds__(256)
+kv4_quantize_pairs_kernel(const void* __restrict__ X, int T, int H, int had_block, float inv_sqrt_b, float clip, int t0, int T_cap,
+                          uint8_t* __restrict__ codes, float* __restrict__ scale, float* __restrict__ zero) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const int first_pair = t0 >> 1, n_pairs = ((t0 + T + 1) >> 1) - first_pair;
+    const long long w = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);  // (pair, head)
+    if (w >= static_cast<long long>(n_pairs) * H) return;
+    const int pair = first_pair + static_cast<int>(w / H), h = static_cast<int>(w % H);
+    uint32_t nib[2] = {0, 0};
+    bool have[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const int slot = 2 * pair + k;
+        have[k] = slot >= t0 && slot < t0 + T;
+        if (have[k]) {  // warp-uniform
+            float v[4], s, z;
+            kv4_load_vector<BF16_IN>(X, static_cast<long long>(slot - t0) * H + h, lane, v);
+            nib[k] = kv4_quantize_vector(v, lane, had_block, inv_sqrt_b, clip, s, z);
+            if (lane == 0) {
+                scale[static_cast<size_t>(h) * T_cap + slot] = s;
+                zero[static_cast<size_t>(h) * T_cap + slot] = z;
+            }
+        }
+    }
+    uint32_t* dst = reinterpret_cast<uint32_t*>(codes + (static_cast<size_t>(h) * (T_cap >> 1) + pair) * kKvD) + lane;
+    // spread the four codes of each token over four bytes: token k's code e -> byte e, nibble k
+    uint32_t lo = (nib[0] & 0xf) | ((nib[0] & 0xf0) << 4) | ((nib[0] & 0xf00) << 8) | ((nib[0] & 0xf000) << 12);
+    uint32_t hi = (nib[1] & 0xf) | ((nib[1] & 0xf0) << 4) | ((nib[1] & 0xf00) << 8) | ((nib[1] & 0xf000) << 12);
+    uint32_t bytes = lo | (hi << 4);
+    if (!(have[0] && have[1])) {
+        const uint32_t old = *dst;
+        bytes = have[0] ? (bytes & 0x0f0f0f0fu) | (old & 0xf0f0f0f0u) : (bytes & 0xf0f0f0f0u) | (old & 0x0f0f0f0fu);
+    }
+    *dst = bytes;
+}
+
 // ------------------------------------------------------------------------------------------------
-// decode attention over the 4-bit cache
+// decode attention over the 4-bit cache (tensor cores)
 // ------------------------------------------------------------------------------------------------
 // out[h] = sum_t softmax_t(q[h] . Khat[t] / sqrt(D)) Vhat[t],  Khat = ks (kc - kz),  Vhat = vs (vc - vz),
-// for the G = Hq / Hkv query heads that share a KV head.  fp32 throughout.
+// for the G = Hq / Hkv <= 8 query heads that share a KV head.
 //
-// Grid (head groups, splits, Hkv): a CTA takes a contiguous range of tokens of one KV head for G of the
-// query heads that share it (G <= 2: more accumulators per thread would leave one CTA per SM; the head
-// groups of a split run side by side and the second finds the codes in L2); eight warps take runs of
-// four-token tiles in turn.  A lane is (token j of the tile, 16-dimension chunk c): it loads the 8
-// bytes of codes of its chunk (a warp reads 256 contiguous bytes), turns them into floats ONCE and
-// uses them for all G heads.  The zero-points never touch the per-element path:
-//   q . Khat = ks (sum_d c_d q_d - kz sum_d q_d),     sum_t w_t Vhat_t = sum_t w_t vs_t c_t - (sum_t w_t vs_t vz_t).
-// Softmax is the usual running-max form; partial (max, denominator, numerator) triples are merged
-// across lanes, warps and finally splits (kv4_attention_combine_kernel).
+// Both products run on mma.sync.m16n8k16 (fp16 operands, fp32 accumulators) with the query heads as
+// the 16 rows (rows G..15 are zero):
+//   S[head][token] = sum_d q[head][d] * kc[token][d]          A = q,           B = key codes
+//   O[head][d]    += sum_t w[head][t] * vc[t][d]              A = w = p * vs,  B = value codes
+// The 4-bit codes are exact in fp16.  The fp32 operands q and w are each split into a high and a low
+// fp16 part (two instructions per product), which keeps the result at fp32 accuracy: the residual of
+// the split is 2^-22 of the value.  Scales and zero-points stay out of the element path:
+//   score = ks[t] * (S - kz[t] * sum_d q[d]),     O_final = O - sum_t w[t] * vz[t].
+// A byte of the cache is exactly one operand register: two neighbouring dimensions of a token for the
+// keys (the k index of the first product), two neighbouring tokens of a dimension for the values (the
+// k index of the second), low nibble = lower index.  Which dimension sits at which k (or n) position
+// of an instruction is free as long as both operands agree, and is chosen so that a lane reads 16
+// contiguous bytes per cache row:
+//   keys:   lane (g, cq) holds bytes [16cq, 16cq+16) of token g's row; k-step ks uses bytes 2ks, 2ks+1,
+//           i.e. k positions 2cq, 2cq+1 <-> dimensions 32cq + 4ks, +1 and 2cq+8, 2cq+9 <-> 32cq + 4ks + 2, +3;
+//   values: lane (g, cq) holds bytes [16g, 16g+16) of pair rows cq and cq+4; n-tile nt uses byte nt,
+//           i.e. column g of n-tile nt <-> dimension 16g + nt.
+// Grid (splits, Hkv): a CTA takes a contiguous range of tokens of one KV head, its four warps take
+// 16-token tiles in turn, each with its own running max / denominator / numerator (merged through
+// shared memory at the end, and across splits by kv4_attention_combine_kernel).
 struct Kv4Params {
     const float* q;  // [Hq][D]
     const uint8_t* k_codes;
@@ -122,154 +194,175 @@ struct Kv4Params {
     float inv_sqrt_d;
 };
 
-constexpr int kKvWarps = 8;
-constexpr int kKvUnroll = 2;  // four-token tiles a warp loads ahead (more costs the second CTA per SM)
+constexpr int kKvWarps = 4;
+constexpr int kKvTile = 16;          // tokens per warp tile
 constexpr int kKvPartial = kKvD + 2;
 
-// Eight codes of a 32-bit word as floats: 2^23 + c has the code in its low mantissa bits.
-__device__ __forceinline__ void nibbles_to_floats(uint32_t w, float (&f)[8]) {
-    const uint32_t lo = w & 0x0f0f0f0fu, hi = (w >> 4) & 0x0f0f0f0fu;
-    constexpr uint32_t magic = 0x4b000000u;  // 2^23
-    f[0] = __uint_as_float(__byte_perm(lo, magic, 0x7440)) - 8388608.0f;
-    f[1] = __uint_as_float(__byte_perm(hi, magic, 0x7440)) - 8388608.0f;
-    f[2] = __uint_as_float(__byte_perm(lo, magic, 0x7441)) - 8388608.0f;
-    f[3] = __uint_as_float(__byte_perm(hi, magic, 0x7441)) - 8388608.0f;
-    f[4] = __uint_as_float(__byte_perm(lo, magic, 0x7442)) - 8388608.0f;
-    f[5] = __uint_as_float(__byte_perm(hi, magic, 0x7442)) - 8388608.0f;
-    f[6] = __uint_as_float(__byte_perm(lo, magic, 0x7443)) - 8388608.0f;
-    f[7] = __uint_as_float(__byte_perm(hi, magic, 0x7443)) - 8388608.0f;
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-template <int G>
+// Byte `pos` of a word -> two fp16 codes (low nibble in the low half): 0x6400 | c is 1024 + c.
+__device__ __forceinline__ uint32_t byte_to_half2(uint32_t word, int pos) {
+    const uint32_t x = (word >> (8 * pos)) & 0xffu;
+    const uint32_t h = ((x * 4097u) & 0x000f000fu) | 0x64006400u;
+    uint32_t r;
+    asm("sub.f16x2 %0, %1, %2;" : "=r"(r) : "r"(h), "r"(0x64006400u));
+    return r;
+}
+
+// fp32 pair -> high fp16 parts and low fp16 parts (the residuals).
+__device__ __forceinline__ void split_half2(float x, float y, uint32_t& hi, uint32_t& lo) {
+    const __half2 h = __floats2half2_rn(x, y);
+    const float2 back = __half22float2(h);
+    const __half2 l = __floats2half2_rn(x - back.x, y - back.y);
+    hi = *reinterpret_cast<const uint32_t*>(&h);
+    lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+
 __global__ void __launch_bounds__(32 * kKvWarps)
 kv4_attention_partial_kernel(const Kv4Params p) {
-    __shared__ __align__(16) float qs[G][kKvD];       // q / sqrt(D)
-    __shared__ float qsum[G][8];                       // its chunk sums
-    __shared__ float red[kKvWarps][G][kKvPartial];
+    __shared__ float red[kKvWarps][8][kKvPartial];
     pdl_launch_dependents();
     pdl_wait();
-    const int kv = blockIdx.z, split = blockIdx.y;
-    const int head0 = kv * p.heads_per_kv + blockIdx.x * G;  // first query head of this CTA
+    const int kv = blockIdx.y, split = blockIdx.x, G = p.heads_per_kv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int j = lane >> 3, c = lane & 7;
+    const int g = lane >> 2, cq = lane & 3;
 
-    for (int i = threadIdx.x; i < G * kKvD; i += blockDim.x)
-        qs[i / kKvD][i % kKvD] = __fmul_rn(p.q[static_cast<size_t>(head0) * kKvD + i], p.inv_sqrt_d);
-    __syncthreads();
-    if (threadIdx.x < G * 8) {
-        const int g = threadIdx.x >> 3, cc = threadIdx.x & 7;
-        float s = 0.0f;
-        for (int i = 0; i < 16; ++i) s += qs[g][16 * cc + i];
-        qsum[g][cc] = s;
+    // query fragments: row g (head kv*G + g, zero beyond G), scaled by 1/sqrt(D), split in two fp16 parts
+    uint32_t qh[8][2], ql[8][2];
+    float qsum = 0.0f;  // sum over all dimensions of (high + low) parts of head g
+    {
+        const float* qrow = p.q + static_cast<size_t>(kv * G + (g < G ? g : 0)) * kKvD;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            float4 f = *reinterpret_cast<const float4*>(qrow + 32 * cq + 4 * ks);
+            if (g >= G) f = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            f.x = __fmul_rn(f.x, p.inv_sqrt_d), f.y = __fmul_rn(f.y, p.inv_sqrt_d);
+            f.z = __fmul_rn(f.z, p.inv_sqrt_d), f.w = __fmul_rn(f.w, p.inv_sqrt_d);
+            split_half2(f.x, f.y, qh[ks][0], ql[ks][0]);
+            split_half2(f.z, f.w, qh[ks][1], ql[ks][1]);
+            qsum += (f.x + f.y) + (f.z + f.w);
+        }
+        qsum += __shfl_xor_sync(0xffffffffu, qsum, 1);
+        qsum += __shfl_xor_sync(0xffffffffu, qsum, 2);
     }
-    __syncthreads();
 
     const int t_begin = split * p.tokens_per_split;
     const int t_end = min(p.T, t_begin + p.tokens_per_split);
     const size_t head_row = static_cast<size_t>(kv) * p.T_cap;
+    const uint8_t* vbase = p.v_codes + static_cast<size_t>(kv) * (p.T_cap >> 1) * kKvD;
+    const int last_row = p.T_cap - 1, last_pair = (p.T_cap >> 1) - 1;
 
-    float m[G], l[G], zacc[G], acc[G][16];
+    float o[16][4];
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-        m[g] = -INFINITY, l[g] = 0.0f, zacc[g] = 0.0f;
+    for (int nt = 0; nt < 16; ++nt)
 #pragma unroll
-        for (int i = 0; i < 16; ++i) acc[g][i] = 0.0f;
-    }
+        for (int i = 0; i < 4; ++i) o[nt][i] = 0.0f;
+    float m_run = -INFINITY, l_run = 0.0f, z_run = 0.0f;  // of head g (l and z: this lane's tokens only)
 
-    // kKvUnroll tiles per trip, all their loads issued before the first is used (a warp otherwise waits
-    // out the full memory latency once per tile)
-    for (int tb = t_begin + 4 * kKvUnroll * warp; tb < t_end; tb += 4 * kKvUnroll * kKvWarps) {
-        uint2 kw[kKvUnroll], vw[kKvUnroll];
-        float ks[kKvUnroll], kz[kKvUnroll], vs[kKvUnroll], vz[kKvUnroll];
+    for (int tb = t_begin + kKvTile * warp; tb < t_end; tb += kKvTile * kKvWarps) {
+        // ---- loads of the tile: key rows of tokens tb+g and tb+8+g, value pair rows tb/2+cq and tb/2+4+cq,
+        //      scales and zero-points of this lane's four tokens tb + 8n + 2cq + {0,1}
+        uint4 kraw[2], vraw[2];
+        float2 ksc[2], kzp[2], vsc[2], vzp[2];
 #pragma unroll
-        for (int u = 0; u < kKvUnroll; ++u) {
-            const int t = tb + 4 * u + j;
-            const size_t row = head_row + (t < t_end ? t : t_begin);
-            kw[u] = *reinterpret_cast<const uint2*>(p.k_codes + row * kKvRowBytes + 8 * c);
-            vw[u] = *reinterpret_cast<const uint2*>(p.v_codes + row * kKvRowBytes + 8 * c);
-            ks[u] = p.k_scale[row], kz[u] = p.k_zero[row], vs[u] = p.v_scale[row], vz[u] = p.v_zero[row];
+        for (int n = 0; n < 2; ++n) {
+            const int krow = min(tb + 8 * n + g, last_row);
+            kraw[n] = *reinterpret_cast<const uint4*>(p.k_codes + (head_row + krow) * kKvRowBytes + 16 * cq);
+            const int vrow = min((tb >> 1) + 4 * n + cq, last_pair);
+            vraw[n] = *reinterpret_cast<const uint4*>(vbase + static_cast<size_t>(vrow) * kKvD + 16 * g);
+            const int t = min(tb + 8 * n + 2 * cq, last_row - 1);   // even: the pair t, t+1 is inside the arrays
+            ksc[n] = *reinterpret_cast<const float2*>(p.k_scale + head_row + t);
+            kzp[n] = *reinterpret_cast<const float2*>(p.k_zero + head_row + t);
+            vsc[n] = *reinterpret_cast<const float2*>(p.v_scale + head_row + t);
+            vzp[n] = *reinterpret_cast<const float2*>(p.v_zero + head_row + t);
         }
+        // ---- S = q . codes for the two 8-token n-tiles
+        float sc[2][4];
 #pragma unroll
-        for (int u = 0; u < kKvUnroll; ++u) {
-            if (tb + 4 * u >= t_end) break;  // warp-uniform: no token of this tile exists
-            const bool valid = tb + 4 * u + j < t_end;
-            float kd[16], vd[16];
-            {
-                float a[8], b[8];
-                nibbles_to_floats(kw[u].x, a), nibbles_to_floats(kw[u].y, b);
+        for (int n = 0; n < 2; ++n) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) kd[i] = a[i], kd[8 + i] = b[i];
-                nibbles_to_floats(vw[u].x, a), nibbles_to_floats(vw[u].y, b);
+            for (int i = 0; i < 4; ++i) sc[n][i] = 0.0f;
+            const uint32_t w[4] = {kraw[n].x, kraw[n].y, kraw[n].z, kraw[n].w};
 #pragma unroll
-                for (int i = 0; i < 8; ++i) vd[i] = a[i], vd[8 + i] = b[i];
-            }
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                const float4* qv = reinterpret_cast<const float4*>(&qs[g][16 * c]);
-                float p0 = 0.0f, p1 = 0.0f, p2 = 0.0f, p3 = 0.0f;  // four independent chains
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float4 f = qv[i];
-                    p0 = fmaf(kd[4 * i], f.x, p0), p1 = fmaf(kd[4 * i + 1], f.y, p1);
-                    p2 = fmaf(kd[4 * i + 2], f.z, p2), p3 = fmaf(kd[4 * i + 3], f.w, p3);
-                }
-                float part = (p0 + p1) + (p2 + p3);
-                part = fmaf(-kz[u], qsum[g][c], part);
-                part += __shfl_xor_sync(0xffffffffu, part, 1);
-                part += __shfl_xor_sync(0xffffffffu, part, 2);
-                part += __shfl_xor_sync(0xffffffffu, part, 4);
-                const float score = valid ? ks[u] * part : -INFINITY;
-                float tmax = fmaxf(score, __shfl_xor_sync(0xffffffffu, score, 8));
-                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 16));
-                if (tmax > m[g]) {  // warp-uniform: rescale what has been accumulated so far
-                    const float corr = expf(m[g] - tmax);  // exp(-inf) = 0 on the first tile
-                    l[g] *= corr, zacc[g] *= corr;
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) acc[g][i] *= corr;
-                    m[g] = tmax;
-                }
-                const float pr = valid ? expf(score - m[g]) : 0.0f;
-                const float w = pr * vs[u];
-                l[g] += pr;
-                zacc[g] = fmaf(w, vz[u], zacc[g]);
-#pragma unroll
-                for (int i = 0; i < 16; ++i) acc[g][i] = fmaf(w, vd[i], acc[g][i]);
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t b0 = byte_to_half2(w[ks >> 1], 2 * (ks & 1)), b1 = byte_to_half2(w[ks >> 1], 2 * (ks & 1) + 1);
+                mma_f16(sc[n], qh[ks][0], 0u, qh[ks][1], 0u, b0, b1);
+                mma_f16(sc[n], ql[ks][0], 0u, ql[ks][1], 0u, b0, b1);
             }
         }
+        // ---- scores of head g for this lane's four tokens, running max, weights
+        float s4[4];
+        float tmax = -INFINITY;
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+            const int t = tb + 8 * n + 2 * cq;
+            s4[2 * n] = (t < t_end) ? ksc[n].x * fmaf(-kzp[n].x, qsum, sc[n][0]) : -INFINITY;
+            s4[2 * n + 1] = (t + 1 < t_end) ? ksc[n].y * fmaf(-kzp[n].y, qsum, sc[n][1]) : -INFINITY;
+            tmax = fmaxf(tmax, fmaxf(s4[2 * n], s4[2 * n + 1]));
+        }
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+        const bool grew = tmax > m_run;
+        if (__any_sync(0xffffffffu, grew)) {  // rescale what the rows that found a new max have accumulated
+            const float corr = grew ? expf(m_run - tmax) : 1.0f;  // exp(-inf) = 0 on a row's first tile
+            l_run *= corr, z_run *= corr;
+#pragma unroll
+            for (int nt = 0; nt < 16; ++nt) o[nt][0] *= corr, o[nt][1] *= corr;
+            if (grew) m_run = tmax;
+        }
+        float w4[4];
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+            const float p0 = (s4[2 * n] > -INFINITY) ? expf(s4[2 * n] - m_run) : 0.0f;
+            const float p1 = (s4[2 * n + 1] > -INFINITY) ? expf(s4[2 * n + 1] - m_run) : 0.0f;
+            l_run += p0 + p1;
+            w4[2 * n] = p0 * vsc[n].x, w4[2 * n + 1] = p1 * vsc[n].y;
+            z_run = fmaf(w4[2 * n], vzp[n].x, fmaf(w4[2 * n + 1], vzp[n].y, z_run));
+        }
+        // ---- O += w . value codes: k = the tile's 16 tokens, A rows = heads
+        uint32_t wh[2], wl[2];
+        split_half2(w4[0], w4[1], wh[0], wl[0]);
+        split_half2(w4[2], w4[3], wh[1], wl[1]);
+        const uint32_t va[4] = {vraw[0].x, vraw[0].y, vraw[0].z, vraw[0].w};
+        const uint32_t vb[4] = {vraw[1].x, vraw[1].y, vraw[1].z, vraw[1].w};
+#pragma unroll
+        for (int nt = 0; nt < 16; ++nt) {
+            const uint32_t b0 = byte_to_half2(va[nt >> 2], nt & 3), b1 = byte_to_half2(vb[nt >> 2], nt & 3);
+            mma_f16(o[nt], wh[0], 0u, wh[1], 0u, b0, b1);
+            mma_f16(o[nt], wl[0], 0u, wl[1], 0u, b0, b1);
+        }
     }
 
-    // merge the four token lanes of the warp (same running max), then the warps through shared memory
+    // ---- merge: the four lanes of a row, then the warps through shared memory
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1), l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    z_run += __shfl_xor_sync(0xffffffffu, z_run, 1), z_run += __shfl_xor_sync(0xffffffffu, z_run, 2);
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-#pragma unroll
-        for (int o = 8; o <= 16; o <<= 1) {
-            l[g] += __shfl_xor_sync(0xffffffffu, l[g], o);
-            zacc[g] += __shfl_xor_sync(0xffffffffu, zacc[g], o);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) acc[g][i] += __shfl_xor_sync(0xffffffffu, acc[g][i], o);
-        }
-        if (j == 0) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) red[warp][g][16 * c + i] = acc[g][i] - zacc[g];  // zero-point term folded in
-            if (c == 0) red[warp][g][kKvD] = m[g], red[warp][g][kKvD + 1] = l[g];
-        }
+    for (int nt = 0; nt < 16; ++nt) {  // column 2cq + e of n-tile nt is dimension 16 (2cq + e) + nt
+        red[warp][g][16 * (2 * cq) + nt] = o[nt][0] - z_run;
+        red[warp][g][16 * (2 * cq + 1) + nt] = o[nt][1] - z_run;
     }
+    if (cq == 0) red[warp][g][kKvD] = m_run, red[warp][g][kKvD + 1] = l_run;
     __syncthreads();
     for (int i = threadIdx.x; i < G * kKvPartial; i += blockDim.x) {
-        const int g = i / kKvPartial, d = i % kKvPartial;
+        const int h = i / kKvPartial, d = i % kKvPartial;
         float mm = -INFINITY;
-        for (int w = 0; w < kKvWarps; ++w) mm = fmaxf(mm, red[w][g][kKvD]);
+        for (int w = 0; w < kKvWarps; ++w) mm = fmaxf(mm, red[w][h][kKvD]);
         float val;
         if (d == kKvD) {
             val = mm;
         } else {
             val = 0.0f;
             for (int w = 0; w < kKvWarps; ++w) {
-                const float mw = red[w][g][kKvD];
-                if (mw > -INFINITY) val = fmaf(red[w][g][d], expf(mw - mm), val);
+                const float mw = red[w][h][kKvD];
+                if (mw > -INFINITY) val = fmaf(red[w][h][d], expf(mw - mm), val);
             }
         }
-        p.partial[(static_cast<size_t>(head0 + g) * p.splits + split) * kKvPartial + d] = val;
+        p.partial[(static_cast<size_t>(kv * G + h) * p.splits + split) * kKvPartial + d] = val;
     }
 }
 

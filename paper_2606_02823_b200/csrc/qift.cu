@@ -830,42 +830,44 @@ int qift_device_status(void* stream, uint32_t* detail) {
 }  // extern "C"
 
 namespace {
-// Token splits of the decode attention: enough CTAs for a few per SM, whole 32-token rounds of the
-// eight warps per split.
+// Token splits of the decode attention: enough CTAs for a few per SM, whole 64-token rounds of the
+// four warps per split.
 void kv4_splits(int T, int Hkv, int* splits, int* tokens_per_split) {
-    int want = (2 * sm_count() + Hkv - 1) / Hkv;
+    int want = (4 * sm_count() + Hkv - 1) / Hkv;
     if (want < 1) want = 1;
     int tps = (T + want - 1) / want;
-    const int round = 4 * kKvUnroll * kKvWarps;  // tokens the eight warps take per trip
+    const int round = kKvTile * kKvWarps;  // tokens the warps of a CTA take per trip
     tps = ((tps + round - 1) / round) * round;
     *tokens_per_split = tps;
     *splits = (T + tps - 1) / tps;
-}
-
-template <int G>  // query heads per CTA
-int launch_kv4_attention(const Kv4Params& p, cudaStream_t st) {
-    int rc = cuda_status(launch_pdl(kv4_attention_partial_kernel<G>, dim3(p.heads_per_kv / G, p.splits, p.Hkv),
-                                    dim3(32 * kKvWarps), 0, st, p));
-    if (rc != QIFT_OK) return rc;
-    return cuda_status(launch_pdl(kv4_attention_combine_kernel, dim3(p.Hq), dim3(kKvD), 0, st, p));
 }
 }  // namespace
 
 extern "C" {
 
 int qift_kv4_quantize(const void* X, int x_dtype, int T, int H, int D, int had_block, float clip_ratio, int t0, int T_cap,
-                      uint8_t* codes, float* scale, float* zero, void* stream) {
+                      int layout, uint8_t* codes, float* scale, float* zero, void* stream) {
     if (!X || !codes || !scale || !zero || T <= 0 || H <= 0 || t0 < 0 || T_cap <= 0) return QIFT_ERR_INVALID_ARG;
     if (static_cast<long long>(t0) + T > T_cap) return QIFT_ERR_INVALID_ARG;
     if (x_dtype != QIFT_F32 && x_dtype != QIFT_BF16) return QIFT_ERR_INVALID_ARG;
+    if (layout != QIFT_KV_KEYS && layout != QIFT_KV_VALUES) return QIFT_ERR_INVALID_ARG;
     if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return QIFT_ERR_INVALID_ARG;
-    if (D != kKvD) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (D != kKvD || (T_cap & 1)) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (had_block < 0 || (had_block > 1 && (!is_pow2(had_block) || had_block > D))) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(X) || !aligned16(codes) || !aligned16(scale) || !aligned16(zero)) return QIFT_ERR_ALIGNMENT;
-    const long long rows = static_cast<long long>(T) * H;
     const float r = had_block > 1 ? inv_sqrt_block(had_block) : 1.0f;
-    const dim3 grid(static_cast<unsigned>((rows + 7) / 8));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (layout == QIFT_KV_VALUES) {
+        const long long warps = static_cast<long long>(((t0 + T + 1) >> 1) - (t0 >> 1)) * H;
+        const dim3 grid(static_cast<unsigned>((warps + 7) / 8));
+        if (x_dtype == QIFT_BF16)
+            return cuda_status(launch_pdl(kv4_quantize_pairs_kernel<true>, grid, dim3(256), 0, st, X, T, H, had_block, r, clip_ratio,
+                                          t0, T_cap, codes, scale, zero));
+        return cuda_status(launch_pdl(kv4_quantize_pairs_kernel<false>, grid, dim3(256), 0, st, X, T, H, had_block, r, clip_ratio, t0,
+                                      T_cap, codes, scale, zero));
+    }
+    const long long rows = static_cast<long long>(T) * H;
+    const dim3 grid(static_cast<unsigned>((rows + 7) / 8));
     if (x_dtype == QIFT_BF16)
         return cuda_status(launch_pdl(kv4_quantize_kernel<true>, grid, dim3(256), 0, st, X, rows, H, had_block, r, clip_ratio, t0,
                                       T_cap, codes, scale, zero));
@@ -887,7 +889,7 @@ int qift_kv4_attention_decode(const float* q, const uint8_t* k_codes, const floa
     if (T <= 0 || T > T_cap || Hq <= 0 || Hkv <= 0) return QIFT_ERR_INVALID_ARG;
     if (D != kKvD || Hq % Hkv != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
     const int G = Hq / Hkv;
-    if (G != 1 && G != 2 && G != 4 && G != 8) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (G > 8 || (T_cap & 1)) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(q) || !aligned16(k_codes) || !aligned16(v_codes) || !aligned16(k_scale) || !aligned16(k_zero) ||
         !aligned16(v_scale) || !aligned16(v_zero) || !aligned16(out) || !aligned16(workspace))
         return QIFT_ERR_ALIGNMENT;
@@ -896,11 +898,12 @@ int qift_kv4_attention_decode(const float* q, const uint8_t* k_codes, const floa
     if (!workspace || workspace_bytes < static_cast<size_t>(Hq) * p.splits * kKvPartial * sizeof(float)) return QIFT_ERR_WORKSPACE;
     p.q = q, p.k_codes = k_codes, p.k_scale = k_scale, p.k_zero = k_zero, p.v_codes = v_codes, p.v_scale = v_scale;
     p.v_zero = v_zero, p.partial = static_cast<float*>(workspace), p.out = out;
-    p.T = T, p.T_cap = T_cap, p.Hq = Hq, p.Hkv = Hkv;
+    p.T = T, p.T_cap = T_cap, p.Hq = Hq, p.Hkv = Hkv, p.heads_per_kv = G;
     p.inv_sqrt_d = static_cast<float>(1.0 / std::sqrt(static_cast<double>(D)));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    p.heads_per_kv = G;
-    return (G == 1) ? launch_kv4_attention<1>(p, st) : launch_kv4_attention<2>(p, st);
+    const int rc = cuda_status(launch_pdl(kv4_attention_partial_kernel, dim3(p.splits, p.Hkv), dim3(32 * kKvWarps), 0, st, p));
+    if (rc != QIFT_OK) return rc;
+    return cuda_status(launch_pdl(kv4_attention_combine_kernel, dim3(p.Hq), dim3(kKvD), 0, st, p));
 }
 
 }  // extern "C"

@@ -30,7 +30,7 @@ def vectors(seed, T, H, shift, outlier=None):
 
 @pytest.mark.parametrize("had_block", [0, 128, 16])
 @pytest.mark.parametrize("bf16", [False, True])
-def test_kv4_quantize_matches_oracle(had_block, bf16):
+def test_kv4_quantize_keys_matches_oracle(had_block, bf16):
     T, H = 37, 5
     x = vectors(40, T, H, 0.2, outlier=9)
     xd = dev(x)
@@ -49,6 +49,28 @@ def test_kv4_quantize_matches_oracle(had_block, bf16):
     assert rc == qift.OK
 
 
+@pytest.mark.parametrize("t0,T", [(0, 36), (3, 37), (4, 1), (5, 1), (7, 2)])
+def test_kv4_quantize_values_token_pairs(t0, T):
+    # the value cache holds two consecutive tokens per byte: appends of any parity must keep the partner nibble
+    H, T_cap = 3, 64
+    cache = qift.Kv4Cache(H, T_cap, qift.KV_VALUES)
+    ref_codes = np.zeros((H, T_cap, D), np.uint8)
+    ref_s = np.zeros((H, T_cap), np.float32)
+    ref_z = np.zeros((H, T_cap), np.float32)
+    pos = 0
+    for step, (a, n) in enumerate([(0, t0), (t0, T)]):                            # fill [0, t0) first, then append T tokens
+        if n == 0:
+            continue
+        x = vectors(41 + step, n, H, -0.3)
+        qift.qift_kv4_quantize(dev(x), cache, t0=a, had_block=0, clip_ratio=0.95)
+        codes, s, z = oracle.kv4_quantize(x.reshape(n * H, D), 0, 0.95)
+        ref_codes[:, a:a + n] = codes.reshape(n, H, D).transpose(1, 0, 2)
+        ref_s[:, a:a + n] = s.reshape(n, H).T
+        ref_z[:, a:a + n] = z.reshape(n, H).T
+    assert np.array_equal(cache.codes.cpu().numpy(), oracle.kv4_pack_token_pairs(ref_codes))
+    assert np.array_equal(cache.scale.cpu().numpy(), ref_s) and np.array_equal(cache.zero.cpu().numpy(), ref_z)
+
+
 def test_kv4_quantize_degenerate_rows():
     x = np.zeros((4, 2, D), np.float32)
     x[1] = 3.0                      # constant positive: range [0, 3]
@@ -65,16 +87,19 @@ def test_kv4_quantize_degenerate_rows():
 def build_cache(seed, T, Hkv, T_cap):
     k = vectors(seed, T, Hkv, 0.1, outlier=5)
     v = vectors(seed + 1, T, Hkv, -0.1)
-    K, V = qift.Kv4Cache(Hkv, T_cap), qift.Kv4Cache(Hkv, T_cap)
+    T_cap += T_cap & 1
+    K, V = qift.Kv4Cache(Hkv, T_cap), qift.Kv4Cache(Hkv, T_cap, qift.KV_VALUES)
     qift.qift_kv4_quantize(dev(k), K, had_block=128)
     qift.qift_kv4_quantize(dev(v), V, had_block=0)
-    unpack = lambda c: oracle.kv4_unpack(c.codes.cpu().numpy()[:, :T])
-    return K, V, (unpack(K), K.scale.cpu().numpy()[:, :T], K.zero.cpu().numpy()[:, :T],
-                  unpack(V), V.scale.cpu().numpy()[:, :T], V.zero.cpu().numpy()[:, :T])
+    kc = oracle.kv4_unpack(K.codes.cpu().numpy()[:, :T])
+    vb = V.codes.cpu().numpy()                                                    # [Hkv, T_cap/2, D]: tokens 2i | 2i+1 << 4
+    vc = np.stack([vb & 15, vb >> 4], axis=2).reshape(Hkv, T_cap, D)[:, :T]
+    return K, V, (kc, K.scale.cpu().numpy()[:, :T], K.zero.cpu().numpy()[:, :T],
+                  vc, V.scale.cpu().numpy()[:, :T], V.zero.cpu().numpy()[:, :T])
 
 
-@pytest.mark.parametrize("T,Hq,Hkv", [(1, 4, 4), (5, 8, 2), (130, 8, 8), (1000, 32, 8), (4133, 32, 8), (3000, 16, 2),
-                                      (20000, 8, 8)])
+@pytest.mark.parametrize("T,Hq,Hkv", [(1, 4, 4), (5, 8, 2), (16, 6, 2), (130, 8, 8), (1000, 32, 8), (4133, 32, 8),
+                                      (3000, 16, 2), (999, 14, 2), (20000, 8, 8)])
 def test_kv4_attention_matches_oracle(T, Hq, Hkv):
     K, V, ref_args = build_cache(50 + T, T, Hkv, T + 11)
     q = (synth.normal(60, 4, (Hq, D)) * 1.5).astype(np.float32)
@@ -102,6 +127,8 @@ def test_kv4_attention_peaked_and_uniform_scores():
 
 def test_kv4_rejects_bad_arguments():
     L = qift.lib()
+    with pytest.raises(AssertionError):
+        qift.Kv4Cache(2, 15)                                                      # odd capacity
     K = qift.Kv4Cache(2, 16)
     x = torch.zeros((4, 2, 64), device="cuda")
     with pytest.raises(qift.QiftError) as e:
@@ -111,9 +138,9 @@ def test_kv4_rejects_bad_arguments():
     with pytest.raises(qift.QiftError) as e:
         qift.qift_kv4_quantize(x, K)                                              # more tokens than slots
     assert e.value.status == qift.ERR_INVALID_ARG
-    q = torch.zeros((6, D), device="cuda")
+    q = torch.zeros((18, D), device="cuda")
     with pytest.raises(qift.QiftError) as e:
-        qift.qift_kv4_attention_decode(q, K, K, 4)                                # 3 query heads per KV head
+        qift.qift_kv4_attention_decode(q, K, K, 4)                                # 9 query heads per KV head
     assert e.value.status == qift.ERR_UNSUPPORTED_SHAPE
     q = torch.zeros((4, D), device="cuda")
     with pytest.raises(qift.QiftError) as e:

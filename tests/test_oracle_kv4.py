@@ -89,6 +89,13 @@ def test_pack_roundtrip_and_nibble_order():
     assert packed[0, 0, 0] == (codes[0, 0, 0] | (codes[0, 0, 1] << 4))           # even dimension in the low nibble
 
 
+def test_token_pair_packing_of_values():
+    codes = ((np.arange(2 * 6 * 64).reshape(2, 6, 64) * 7) % 16).astype(np.uint8)
+    packed = oracle.kv4_pack_token_pairs(codes)
+    assert packed.shape == (2, 3, 64)
+    assert np.array_equal(packed & 15, codes[:, 0::2]) and np.array_equal(packed >> 4, codes[:, 1::2])
+
+
 def make_cache(seed, Hkv, T, D):
     K = rows(seed, Hkv * T, D, shift=0.1)
     V = rows(seed + 1, Hkv * T, D, shift=-0.1)

@@ -160,12 +160,13 @@ kv4_quantize_pairs_kernel(const void* __restrict__ X, int T, int H, int had_bloc
 // for the G = Hq / Hkv <= 8 query heads that share a KV head.
 //
 // Both products run on mma.sync.m16n8k16 (fp16 operands, fp32 accumulators) with the query heads as
-// the 16 rows (rows G..15 are zero):
+// rows (rows g < 8: the high fp16 part of head g's operand, rows g + 8: its low part; heads beyond G are zero):
 //   S[head][token] = sum_d q[head][d] * kc[token][d]          A = q,           B = key codes
 //   O[head][d]    += sum_t w[head][t] * vc[t][d]              A = w = p * vs,  B = value codes
 // The 4-bit codes are exact in fp16.  The fp32 operands q and w are each split into a high and a low
-// fp16 part (two instructions per product), which keeps the result at fp32 accuracy: the residual of
-// the split is 2^-22 of the value.  Scales and zero-points stay out of the element path:
+// fp16 part, which keeps the result at fp32 accuracy (the residual of the split is 2^-22 of the
+// value); the two parts occupy rows g and g + 8 of the same instruction and their accumulators are
+// added at the end, so the sixteen rows of the tile are all used.  Scales and zero-points stay out of the element path:
 //   score = ks[t] * (S - kz[t] * sum_d q[d]),     O_final = O - sum_t w[t] * vz[t].
 // A byte of the cache is exactly one operand register: two neighbouring dimensions of a token for the
 // keys (the k index of the first product), two neighbouring tokens of a dimension for the values (the
@@ -205,12 +206,15 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1,
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Byte `pos` of a word -> two fp16 codes (low nibble in the low half): 0x6400 | c is 1024 + c.
+// Byte `pos` of a word -> two fp16 codes (low nibble in the low half), three instructions: the byte is
+// copied into both halves, its low nibble kept in the low half and its high nibble (in place, i.e.
+// times 16) in the high half, each under the exponent of 1024: the halves read 1024 + c_lo and
+// 1024 + 16 c_hi; one fused multiply-add by (1, 1/16) plus (-1024, -64) leaves (c_lo, c_hi), exactly.
 __device__ __forceinline__ uint32_t byte_to_half2(uint32_t word, int pos) {
-    const uint32_t x = (word >> (8 * pos)) & 0xffu;
-    const uint32_t h = ((x * 4097u) & 0x000f000fu) | 0x64006400u;
+    const uint32_t x2 = __byte_perm(word, 0u, 0x4040u | static_cast<uint32_t>(pos) | (static_cast<uint32_t>(pos) << 8));
+    const uint32_t h = (x2 & 0x00f0000fu) | 0x64006400u;
     uint32_t r;
-    asm("sub.f16x2 %0, %1, %2;" : "=r"(r) : "r"(h), "r"(0x64006400u));
+    asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(h), "r"(0x2c003c00u), "r"(0xd400e400u));
     return r;
 }
 
@@ -223,7 +227,7 @@ __device__ __forceinline__ void split_half2(float x, float y, uint32_t& hi, uint
     lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
-__global__ void __launch_bounds__(32 * kKvWarps)
+__global__ void __launch_bounds__(32 * kKvWarps, 2)
 kv4_attention_partial_kernel(const Kv4Params p) {
     __shared__ float red[kKvWarps][8][kKvPartial];
     pdl_launch_dependents();
@@ -264,23 +268,37 @@ kv4_attention_partial_kernel(const Kv4Params p) {
         for (int i = 0; i < 4; ++i) o[nt][i] = 0.0f;
     float m_run = -INFINITY, l_run = 0.0f, z_run = 0.0f;  // of head g (l and z: this lane's tokens only)
 
-    for (int tb = t_begin + kKvTile * warp; tb < t_end; tb += kKvTile * kKvWarps) {
-        // ---- loads of the tile: key rows of tokens tb+g and tb+8+g, value pair rows tb/2+cq and tb/2+4+cq,
-        //      scales and zero-points of this lane's four tokens tb + 8n + 2cq + {0,1}
+    // loads of a tile: key rows of tokens tb+g and tb+8+g, value pair rows tb/2+cq and tb/2+4+cq, scales and
+    // zero-points of this lane's four tokens tb + 8n + 2cq + {0,1}; issued one tile ahead of their use
+    struct Tile {
         uint4 kraw[2], vraw[2];
         float2 ksc[2], kzp[2], vsc[2], vzp[2];
+    };
+    auto load_tile = [&](Tile& x, int tb) {
 #pragma unroll
         for (int n = 0; n < 2; ++n) {
             const int krow = min(tb + 8 * n + g, last_row);
-            kraw[n] = *reinterpret_cast<const uint4*>(p.k_codes + (head_row + krow) * kKvRowBytes + 16 * cq);
+            x.kraw[n] = *reinterpret_cast<const uint4*>(p.k_codes + (head_row + krow) * kKvRowBytes + 16 * cq);
             const int vrow = min((tb >> 1) + 4 * n + cq, last_pair);
-            vraw[n] = *reinterpret_cast<const uint4*>(vbase + static_cast<size_t>(vrow) * kKvD + 16 * g);
+            x.vraw[n] = *reinterpret_cast<const uint4*>(vbase + static_cast<size_t>(vrow) * kKvD + 16 * g);
             const int t = min(tb + 8 * n + 2 * cq, last_row - 1);   // even: the pair t, t+1 is inside the arrays
-            ksc[n] = *reinterpret_cast<const float2*>(p.k_scale + head_row + t);
-            kzp[n] = *reinterpret_cast<const float2*>(p.k_zero + head_row + t);
-            vsc[n] = *reinterpret_cast<const float2*>(p.v_scale + head_row + t);
-            vzp[n] = *reinterpret_cast<const float2*>(p.v_zero + head_row + t);
+            x.ksc[n] = *reinterpret_cast<const float2*>(p.k_scale + head_row + t);
+            x.kzp[n] = *reinterpret_cast<const float2*>(p.k_zero + head_row + t);
+            x.vsc[n] = *reinterpret_cast<const float2*>(p.v_scale + head_row + t);
+            x.vzp[n] = *reinterpret_cast<const float2*>(p.v_zero + head_row + t);
         }
+    };
+    Tile cur;
+    if (t_begin + kKvTile * warp < t_end) load_tile(cur, t_begin + kKvTile * warp);
+    for (int tb = t_begin + kKvTile * warp; tb < t_end; tb += kKvTile * kKvWarps) {
+        Tile nxt = cur;
+        if (tb + kKvTile * kKvWarps < t_end) load_tile(nxt, tb + kKvTile * kKvWarps);
+        const uint4(&kraw)[2] = cur.kraw;
+        const uint4(&vraw)[2] = cur.vraw;
+        const float2(&ksc)[2] = cur.ksc;
+        const float2(&kzp)[2] = cur.kzp;
+        const float2(&vsc)[2] = cur.vsc;
+        const float2(&vzp)[2] = cur.vzp;
         // ---- S = q . codes for the two 8-token n-tiles
         float sc[2][4];
 #pragma unroll
@@ -291,8 +309,7 @@ kv4_attention_partial_kernel(const Kv4Params p) {
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
                 const uint32_t b0 = byte_to_half2(w[ks >> 1], 2 * (ks & 1)), b1 = byte_to_half2(w[ks >> 1], 2 * (ks & 1) + 1);
-                mma_f16(sc[n], qh[ks][0], 0u, qh[ks][1], 0u, b0, b1);
-                mma_f16(sc[n], ql[ks][0], 0u, ql[ks][1], 0u, b0, b1);
+                mma_f16(sc[n], qh[ks][0], ql[ks][0], qh[ks][1], ql[ks][1], b0, b1);  // rows g: high parts, rows g+8: low parts
             }
         }
         // ---- scores of head g for this lane's four tokens, running max, weights
@@ -301,8 +318,8 @@ kv4_attention_partial_kernel(const Kv4Params p) {
 #pragma unroll
         for (int n = 0; n < 2; ++n) {
             const int t = tb + 8 * n + 2 * cq;
-            s4[2 * n] = (t < t_end) ? ksc[n].x * fmaf(-kzp[n].x, qsum, sc[n][0]) : -INFINITY;
-            s4[2 * n + 1] = (t + 1 < t_end) ? ksc[n].y * fmaf(-kzp[n].y, qsum, sc[n][1]) : -INFINITY;
+            s4[2 * n] = (t < t_end) ? ksc[n].x * fmaf(-kzp[n].x, qsum, sc[n][0] + sc[n][2]) : -INFINITY;
+            s4[2 * n + 1] = (t + 1 < t_end) ? ksc[n].y * fmaf(-kzp[n].y, qsum, sc[n][1] + sc[n][3]) : -INFINITY;
             tmax = fmaxf(tmax, fmaxf(s4[2 * n], s4[2 * n + 1]));
         }
         tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
@@ -312,7 +329,7 @@ kv4_attention_partial_kernel(const Kv4Params p) {
             const float corr = grew ? expf(m_run - tmax) : 1.0f;  // exp(-inf) = 0 on a row's first tile
             l_run *= corr, z_run *= corr;
 #pragma unroll
-            for (int nt = 0; nt < 16; ++nt) o[nt][0] *= corr, o[nt][1] *= corr;
+            for (int nt = 0; nt < 16; ++nt) o[nt][0] *= corr, o[nt][1] *= corr, o[nt][2] *= corr, o[nt][3] *= corr;
             if (grew) m_run = tmax;
         }
         float w4[4];
@@ -333,9 +350,9 @@ kv4_attention_partial_kernel(const Kv4Params p) {
 #pragma unroll
         for (int nt = 0; nt < 16; ++nt) {
             const uint32_t b0 = byte_to_half2(va[nt >> 2], nt & 3), b1 = byte_to_half2(vb[nt >> 2], nt & 3);
-            mma_f16(o[nt], wh[0], 0u, wh[1], 0u, b0, b1);
-            mma_f16(o[nt], wl[0], 0u, wl[1], 0u, b0, b1);
+            mma_f16(o[nt], wh[0], wl[0], wh[1], wl[1], b0, b1);
         }
+        cur = nxt;
     }
 
     // ---- merge: the four lanes of a row, then the warps through shared memory
@@ -343,8 +360,8 @@ kv4_attention_partial_kernel(const Kv4Params p) {
     z_run += __shfl_xor_sync(0xffffffffu, z_run, 1), z_run += __shfl_xor_sync(0xffffffffu, z_run, 2);
 #pragma unroll
     for (int nt = 0; nt < 16; ++nt) {  // column 2cq + e of n-tile nt is dimension 16 (2cq + e) + nt
-        red[warp][g][16 * (2 * cq) + nt] = o[nt][0] - z_run;
-        red[warp][g][16 * (2 * cq + 1) + nt] = o[nt][1] - z_run;
+        red[warp][g][16 * (2 * cq) + nt] = (o[nt][0] + o[nt][2]) - z_run;
+        red[warp][g][16 * (2 * cq + 1) + nt] = (o[nt][1] + o[nt][3]) - z_run;
     }
     if (cq == 0) red[warp][g][kKvD] = m_run, red[warp][g][kKvD + 1] = l_run;
     __syncthreads();

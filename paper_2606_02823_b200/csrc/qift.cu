@@ -830,10 +830,10 @@ int qift_device_status(void* stream, uint32_t* detail) {
 }  // extern "C"
 
 namespace {
-// Token splits of the decode attention: enough CTAs for a few per SM, whole 64-token rounds of the
-// four warps per split.
+// Token splits of the decode attention: one resident wave of CTAs, whole 64-token rounds of the four
+// warps per split.
 void kv4_splits(int T, int Hkv, int* splits, int* tokens_per_split) {
-    int want = (4 * sm_count() + Hkv - 1) / Hkv;
+    int want = (2 * sm_count()) / Hkv;  // two CTAs fit an SM: one resident wave (measured best of 1..4)
     if (want < 1) want = 1;
     int tps = (T + want - 1) / want;
     const int round = kKvTile * kKvWarps;  // tokens the warps of a CTA take per trip

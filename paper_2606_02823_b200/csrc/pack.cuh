@@ -17,6 +17,51 @@ __device__ __forceinline__ int nearest_code(float w, float s) {
     return max(-8, min(7, __float2int_rn(t))) & 15;
 }
 
+// Division-free nearest level for one scale, bit-identical to nearest_code().
+//   No-zero sets: the decision t > theta with t = fl(w / s) equals |w| > fl(theta * s) unless |w| lies
+//   within 2^-20 (relative) of that product -- roundings of the product and of the quotient move either
+//   side by at most 2^-23 -- and t > 0 equals w > 0 unless the quotient underflows; in those (rare)
+//   cases the division decides.
+//   Integer sets: t = w * (1/s) differs from the quotient by < 2^-19 for |t| <= 8, so both round to the
+//   same integer unless t lies within 2^-17 of a tie; clamp before rounding = clamp after.
+template <int LV>
+struct LevelCoder {
+    float s, thr, band, tiny, inv;
+    __device__ __forceinline__ void init(float scale) {
+        s = scale;
+        constexpr float theta = (LV == QIFT_LEVELS_POT) ? 2.5f : 2.0f;
+        thr = __fmul_rn(theta, scale);
+        band = __fmul_rn(thr, 9.5367431640625e-07f);  // 2^-20
+        tiny = __fmul_rn(scale, 7.888609052210118e-31f);  // 2^-100
+        inv = (scale >= 1e-30f && scale <= 1e30f) ? __fdiv_rn(1.0f, scale) : 0.0f;
+    }
+    // Branch-free part: code of w and, in `mag`, |level| for the no-zero sets / the signed level for the
+    // integer sets; `unsure` is set when the division has to decide (then use exact()).
+    __device__ __forceinline__ int fast(float w, float& mag, bool& unsure) const {
+        if constexpr (LV == QIFT_LEVELS_MNZ || LV == QIFT_LEVELS_POT) {
+            const float a = fabsf(w);
+            unsure = unsure || fabsf(__fsub_rn(a, thr)) <= band || (a != 0.0f && a < tiny);
+            const bool outer = a > thr;
+            mag = outer ? top_level(LV) : 1.0f;
+            return (w > 0.0f) ? 2 + static_cast<int>(outer) : 1 - static_cast<int>(outer);
+        } else {
+            constexpr float lo = (LV == QIFT_LEVELS_SYM) ? -2.0f : -8.0f, hi = (LV == QIFT_LEVELS_SYM) ? 1.0f : 7.0f;
+            const float t = fminf(fmaxf(__fmul_rn(w, inv), lo), hi);
+            const float r = __fsub_rn(__fadd_rn(t, 12582912.0f), 12582912.0f);
+            unsure = unsure || inv == 0.0f || fabsf(__fsub_rn(t, r)) > 0.49999237f;
+            mag = r;
+            const int q = static_cast<int>(r);
+            return (LV == QIFT_LEVELS_SYM) ? q + 2 : (q & 15);
+        }
+    }
+    __device__ __forceinline__ int exact(float w, float& mag) const {
+        const int c = nearest_code<LV>(w, s);
+        const float lv = static_cast<float>(level_from_code<LV>(c));
+        mag = (LV == QIFT_LEVELS_MNZ || LV == QIFT_LEVELS_POT) ? fabsf(lv) : lv;
+        return c;
+    }
+};
+
 template <int LV>
 __global__ void __launch_bounds__(kPackThreads)
 pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* __restrict__ s_n,
@@ -24,6 +69,8 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
     extern __shared__ __align__(16) float row[];
     __shared__ float red[kPackThreads / 32];
     __shared__ double err[kNumCandidates][kPackThreads / 32];
+    __shared__ int cnt[kNumCandidates][kPackThreads / 32];
+    __shared__ double mom[2][kPackThreads / 32];
     __shared__ float s_shared;
     // No early launch of dependents here: the product kernels prefetch packed weights before their
     // own dependency wait, which is only safe if whoever writes those weights has fully completed.
@@ -58,25 +105,119 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
         if (mode == QIFT_SCALE_ABSMAX) {
             s = __fdiv_rn(amax, g);
         } else {
-            // Squared error of every candidate scale; per-element terms are formed exactly as
-            // d = w - s*level, d*d in fp64 without contraction, partial sums per thread in
-            // ascending k, then a fixed-order tree.
+            constexpr bool kNoZero = (LV == QIFT_LEVELS_MNZ || LV == QIFT_LEVELS_POT);
+            if constexpr (kNoZero) {
+                // No-zero sets {+-1, +-top}: a weight's level has its sign and magnitude 1 (inner) or top
+                // (outer, |w| / s > theta), so with a = |w| the squared error of a candidate scale s is
+                //   E(s) = sum a^2 - 2 s (sum a + (top-1) sum_outer a) + s^2 (K + (top^2-1) n_outer):
+                // per candidate only the sum and the count of the outer weights are needed -- one fp64 add
+                // per weight and candidate instead of a subtract, a multiply and an add (the sweep is
+                // bound by the fp64 pipe).  The regrouping changes E by ~1e-15 relative, far inside the
+                // 1e-12 within which two candidates count as tied.  All sums: per thread in ascending k,
+                // then fixed-order trees.
+                constexpr double top = top_level(LV);
+                double a2 = 0.0, a1 = 0.0;
+                for (int k = tid; k < K; k += blockDim.x) {
+                    const double ad = static_cast<double>(fabsf(row[k]));
+                    a2 = __dadd_rn(a2, __dmul_rn(ad, ad));
+                    a1 = __dadd_rn(a1, ad);
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    a2 = __dadd_rn(a2, __shfl_xor_sync(0xffffffffu, a2, o));
+                    a1 = __dadd_rn(a1, __shfl_xor_sync(0xffffffffu, a1, o));
+                }
+                if (lane == 0) mom[0][warp] = a2, mom[1][warp] = a1;
+                for (int c0 = 0; c0 < kNumCandidates; c0 += 8) {
+                    LevelCoder<LV> coder[8];
+                    double so[8];
+                    int no[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float p = __fdiv_rn(static_cast<float>(100 - (c0 + j)), 100.0f);
+                        coder[j].init(__fdiv_rn(__fmul_rn(p, amax), g));
+                        so[j] = 0.0, no[j] = 0;
+                    }
+                    for (int k = tid; k < K; k += blockDim.x) {
+                        const float w = row[k];
+                        const float a = fabsf(w);
+                        const double ad = static_cast<double>(a);
+                        bool unsure = false;
+                        bool outer[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            outer[j] = a > coder[j].thr;
+                            unsure = unsure || fabsf(__fsub_rn(a, coder[j].thr)) <= coder[j].band;
+                        }
+                        if (unsure) {  // rare: too close to a threshold to call without the division
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                float mag;
+                                coder[j].exact(w, mag);
+                                outer[j] = mag != 1.0f;
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            if (outer[j]) so[j] = __dadd_rn(so[j], ad), no[j] += 1;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        double v = so[j];
+                        int c = no[j];
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            v = __dadd_rn(v, __shfl_xor_sync(0xffffffffu, v, o));
+                            c += __shfl_xor_sync(0xffffffffu, c, o);
+                        }
+                        if (lane == 0) err[c0 + j][warp] = v, cnt[c0 + j][warp] = c;
+                    }
+                }
+                __syncthreads();
+                if (tid < kNumCandidates) {  // E of candidate tid, left in err[tid][0]
+                    double A = 0.0, S = 0.0, So = 0.0;
+                    int n_out = 0;
+                    for (int w = 0; w < kPackThreads / 32; ++w) {
+                        A = __dadd_rn(A, mom[0][w]), S = __dadd_rn(S, mom[1][w]);
+                        So = __dadd_rn(So, err[tid][w]), n_out += cnt[tid][w];
+                    }
+                    const float p = __fdiv_rn(static_cast<float>(100 - tid), 100.0f);
+                    const double sj = static_cast<double>(__fdiv_rn(__fmul_rn(p, amax), g));
+                    const double lin = S + (top - 1.0) * So;
+                    const double quad = static_cast<double>(K) + (top * top - 1.0) * static_cast<double>(n_out);
+                    const double E = A - 2.0 * sj * lin + sj * sj * quad;
+                    err[tid][0] = E;  // each thread touches its own row of err only
+#pragma unroll
+                    for (int w = 1; w < kPackThreads / 32; ++w) err[tid][w] = 0.0;
+                }
+            } else {
+            // Integer sets: squared error of every candidate scale; per-element terms are formed exactly as
+            // d = w - s*level, d*d in fp64 without contraction, partial sums per thread in ascending k,
+            // then a fixed-order tree.
             for (int c0 = 0; c0 < kNumCandidates; c0 += 8) {
-                float sc[8];
-                double e[8];
+                LevelCoder<LV> coder[8];
+                double sd[8], e[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const float p = __fdiv_rn(static_cast<float>(100 - (c0 + j)), 100.0f);
-                    sc[j] = __fdiv_rn(__fmul_rn(p, amax), g);
+                    coder[j].init(__fdiv_rn(__fmul_rn(p, amax), g));
+                    sd[j] = static_cast<double>(coder[j].s);
                     e[j] = 0.0;
                 }
                 for (int k = tid; k < K; k += blockDim.x) {
                     const float w = row[k];
+                    const double wd = static_cast<double>(w);
+                    float mag[8];
+                    bool unsure = false;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) coder[j].fast(w, mag[j], unsure);
+                    if (unsure) {  // rare: some candidate's decision is too close to call without the division
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) coder[j].exact(w, mag[j]);
+                    }
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
-                        const int code = nearest_code<LV>(w, sc[j]);
-                        const double rec = __dmul_rn(static_cast<double>(sc[j]), static_cast<double>(level_from_code<LV>(code)));
-                        const double d = __dsub_rn(static_cast<double>(w), rec);
+                        const double d = __dsub_rn(wd, __dmul_rn(sd[j], static_cast<double>(mag[j])));
                         e[j] = __dadd_rn(e[j], __dmul_rn(d, d));
                     }
                 }
@@ -87,6 +228,7 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
                     for (int o = 16; o > 0; o >>= 1) v = __dadd_rn(v, __shfl_xor_sync(0xffffffffu, v, o));
                     if (lane == 0) err[c0 + j][warp] = v;
                 }
+            }
             }
             __syncthreads();
             if (tid == 0) {
@@ -106,26 +248,40 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
     }
     if (tid == 0 && mode != QIFT_SCALE_GIVEN) s_n[n] = s;
 
+    // Codes: first one byte per weight into shared memory (threads stride over k: conflict-free), then
+    // one packed word per thread from 16 consecutive code bytes -- with the bit layout of the packed
+    // word four code bytes (k = 4t .. 4t+3) shifted left by 2t (4t for INT4) ARE plane t of the word --
+    // and the four words of a 16-byte group are gathered in its first lane for one 128-bit store.
     constexpr int PER = codes_per_word(LV);
-    constexpr int BITS = 32 / PER;
     const int words = K / PER;
-    for (int u = tid; u < pitch / 4; u += blockDim.x) {  // one 16-byte group of four words per thread
-        uint32_t out[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int j = 4 * u + e;
-            uint32_t w = 0;
-            if (j < words) {
-#pragma unroll
-                for (int r = 0; r < PER; ++r) {
-                    const int t = r / 4, b = r % 4;
-                    w |= static_cast<uint32_t>(nearest_code<LV>(row[j * PER + r], s)) << (8 * b + BITS * t);
-                }
+    unsigned char* code_bytes = reinterpret_cast<unsigned char*>(row + K);
+    LevelCoder<LV> final_coder;
+    final_coder.init(s);
+    __syncthreads();
+    for (int k = tid; k < K; k += blockDim.x) {
+        float mag;
+        bool unsure = false;
+        int c = final_coder.fast(row[k], mag, unsure);
+        if (unsure) c = final_coder.exact(row[k], mag);
+        code_bytes[k] = static_cast<unsigned char>(c);
+    }
+    __syncthreads();
+    for (int j0 = 0; j0 < pitch; j0 += blockDim.x) {  // pitch is a multiple of 16, blockDim of 32: whole groups per warp
+        const int j = j0 + tid;
+        uint32_t w = 0;
+        if (j < words) {
+            if constexpr (PER == 16) {
+                const uint4 c = *reinterpret_cast<const uint4*>(code_bytes + 16 * j);
+                w = c.x | (c.y << 2) | (c.z << 4) | (c.w << 6);
+            } else {
+                const uint2 c = *reinterpret_cast<const uint2*>(code_bytes + 8 * j);
+                w = c.x | (c.y << 4);
             }
-            out[e] = w;
         }
-        *reinterpret_cast<uint4*>(packed + packed_word_address(static_cast<int>(n), 4 * u, pitch)) =
-            make_uint4(out[0], out[1], out[2], out[3]);
+        const uint32_t w1 = __shfl_down_sync(0xffffffffu, w, 1), w2 = __shfl_down_sync(0xffffffffu, w, 2),
+                       w3 = __shfl_down_sync(0xffffffffu, w, 3);
+        if ((tid & 3) == 0 && j < pitch)
+            *reinterpret_cast<uint4*>(packed + packed_word_address(static_cast<int>(n), j, pitch)) = make_uint4(w, w1, w2, w3);
     }
 }
 

@@ -429,7 +429,7 @@ int qift_pack_weights(const float* W, int N, int K, int levels, int scale_mode, 
     if (K % 16 != 0 || K > kMaxRowK) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(W) || !aligned16(s_n) || !aligned16(packed)) return QIFT_ERR_ALIGNMENT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t smem = padded_row_bytes(K);
+    const size_t smem = static_cast<size_t>(K) * 5;  // the fp32 row and one code byte per weight
 #define QIFT_PACK_CASE(LV)                                                                                   \
     case LV: {                                                                                               \
         cudaError_t e = allow_smem(pack_weights_kernel<LV>, smem);                                           \

@@ -69,8 +69,10 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
     extern __shared__ __align__(16) float row[];
     __shared__ float red[kPackThreads / 32];
     __shared__ double err[kNumCandidates][kPackThreads / 32];
-    __shared__ int cnt[kNumCandidates][kPackThreads / 32];
     __shared__ double mom[2][kPackThreads / 32];
+    __shared__ float cand[kNumCandidates];
+    __shared__ unsigned long long bin_sum[kNumCandidates];
+    __shared__ int bin_cnt[kNumCandidates];
     __shared__ float s_shared;
     // No early launch of dependents here: the product kernels prefetch packed weights before their
     // own dependency wait, which is only safe if whoever writes those weights has fully completed.
@@ -109,18 +111,67 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
             if constexpr (kNoZero) {
                 // No-zero sets {+-1, +-top}: a weight's level has its sign and magnitude 1 (inner) or top
                 // (outer, |w| / s > theta), so with a = |w| the squared error of a candidate scale s is
-                //   E(s) = sum a^2 - 2 s (sum a + (top-1) sum_outer a) + s^2 (K + (top^2-1) n_outer):
-                // per candidate only the sum and the count of the outer weights are needed -- one fp64 add
-                // per weight and candidate instead of a subtract, a multiply and an add (the sweep is
-                // bound by the fp64 pipe).  The regrouping changes E by ~1e-15 relative, far inside the
-                // 1e-12 within which two candidates count as tied.  All sums: per thread in ascending k,
-                // then fixed-order trees.
+                //   E(s) = sum a^2 - 2 s (sum a + (top-1) sum_outer a) + s^2 (K + (top^2-1) n_outer),
+                // and because the candidate scales decrease, a weight that is outer for candidate j is outer
+                // for every later one.  So each weight is looked at ONCE: its switch index b (the first
+                // candidate for which it is outer) is found from the table of thresholds (a first guess
+                // from the ratio, corrected by comparisons; decided by the division where |w| is within
+                // 2^-20 of a threshold), and its magnitude and a count go into bin b.  Outer sums and
+                // counts of all 80 candidates are prefix sums over the bins.  The magnitudes are added as
+                // 64-bit fixed-point integers scaled by the row's maximum (outer weights are >= 0.14 max, so
+                // they are represented exactly and the shared-memory atomics give the same sum in any
+                // order); sum a and sum a^2 are fp64, per thread in ascending k, then fixed-order trees.
+                // The regrouping changes E by ~1e-15 relative, far inside the 1e-12 within which two
+                // candidates count as tied.
                 constexpr double top = top_level(LV);
+                float* thr = cand;  // [kNumCandidates] thresholds theta * s_j, decreasing in j
+                for (int j = tid; j < kNumCandidates; j += blockDim.x) {
+                    LevelCoder<LV> c;
+                    c.init(__fdiv_rn(__fmul_rn(__fdiv_rn(static_cast<float>(100 - j), 100.0f), amax), g));
+                    thr[j] = c.thr;
+                    bin_sum[j] = 0ull, bin_cnt[j] = 0;
+                }
+                __syncthreads();
+                int ex;
+                frexpf(amax, &ex);                              // amax < 2^ex
+                const double to_fixed = ldexp(1.0, 48 - ex);    // a * to_fixed < 2^48, exact for a >= amax * 2^-24
+                const float ratio = __fdiv_rn(g, __fmul_rn((LV == QIFT_LEVELS_POT) ? 2.5f : 2.0f, amax));
                 double a2 = 0.0, a1 = 0.0;
                 for (int k = tid; k < K; k += blockDim.x) {
-                    const double ad = static_cast<double>(fabsf(row[k]));
+                    const float w = row[k];
+                    const float a = fabsf(w);
+                    const double ad = static_cast<double>(a);
                     a2 = __dadd_rn(a2, __dmul_rn(ad, ad));
                     a1 = __dadd_rn(a1, ad);
+                    // first guess: a > theta p_j amax / g  <=>  (100 - j) / 100 < a g / (theta amax)
+                    int bsw = min(kNumCandidates, max(0, 101 - static_cast<int>(100.0f * a * ratio)));
+                    while (bsw > 0 && a > thr[bsw - 1]) --bsw;
+                    while (bsw < kNumCandidates && !(a > thr[bsw])) ++bsw;
+                    // |w| within 2^-20 of a neighbouring threshold: the division decides (monotone in j)
+                    if (bsw > 0 && __fsub_rn(thr[bsw - 1], a) <= thr[bsw - 1] * 9.5367431640625e-07f) {
+                        while (bsw > 0) {
+                            float mag;
+                            LevelCoder<LV> c;
+                            c.init(__fdiv_rn(__fmul_rn(__fdiv_rn(static_cast<float>(100 - (bsw - 1)), 100.0f), amax), g));
+                            c.exact(w, mag);
+                            if (mag == 1.0f) break;
+                            --bsw;
+                        }
+                    }
+                    if (bsw < kNumCandidates && __fsub_rn(a, thr[bsw]) <= thr[bsw] * 9.5367431640625e-07f) {
+                        while (bsw < kNumCandidates) {
+                            float mag;
+                            LevelCoder<LV> c;
+                            c.init(__fdiv_rn(__fmul_rn(__fdiv_rn(static_cast<float>(100 - bsw), 100.0f), amax), g));
+                            c.exact(w, mag);
+                            if (mag != 1.0f) break;
+                            ++bsw;
+                        }
+                    }
+                    if (bsw < kNumCandidates) {
+                        atomicAdd(&bin_sum[bsw], static_cast<unsigned long long>(__dmul_rn(ad, to_fixed)));
+                        atomicAdd(&bin_cnt[bsw], 1);
+                    }
                 }
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) {
@@ -128,65 +179,19 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
                     a1 = __dadd_rn(a1, __shfl_xor_sync(0xffffffffu, a1, o));
                 }
                 if (lane == 0) mom[0][warp] = a2, mom[1][warp] = a1;
-                for (int c0 = 0; c0 < kNumCandidates; c0 += 8) {
-                    LevelCoder<LV> coder[8];
-                    double so[8];
-                    int no[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const float p = __fdiv_rn(static_cast<float>(100 - (c0 + j)), 100.0f);
-                        coder[j].init(__fdiv_rn(__fmul_rn(p, amax), g));
-                        so[j] = 0.0, no[j] = 0;
-                    }
-                    for (int k = tid; k < K; k += blockDim.x) {
-                        const float w = row[k];
-                        const float a = fabsf(w);
-                        const double ad = static_cast<double>(a);
-                        bool unsure = false;
-                        bool outer[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            outer[j] = a > coder[j].thr;
-                            unsure = unsure || fabsf(__fsub_rn(a, coder[j].thr)) <= coder[j].band;
-                        }
-                        if (unsure) {  // rare: too close to a threshold to call without the division
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                float mag;
-                                coder[j].exact(w, mag);
-                                outer[j] = mag != 1.0f;
-                            }
-                        }
-#pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            if (outer[j]) so[j] = __dadd_rn(so[j], ad), no[j] += 1;
-                    }
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        double v = so[j];
-                        int c = no[j];
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) {
-                            v = __dadd_rn(v, __shfl_xor_sync(0xffffffffu, v, o));
-                            c += __shfl_xor_sync(0xffffffffu, c, o);
-                        }
-                        if (lane == 0) err[c0 + j][warp] = v, cnt[c0 + j][warp] = c;
-                    }
-                }
                 __syncthreads();
                 if (tid < kNumCandidates) {  // E of candidate tid, left in err[tid][0]
-                    double A = 0.0, S = 0.0, So = 0.0;
+                    double A = 0.0, S = 0.0;
+                    for (int w = 0; w < kPackThreads / 32; ++w) A = __dadd_rn(A, mom[0][w]), S = __dadd_rn(S, mom[1][w]);
+                    unsigned long long so = 0;
                     int n_out = 0;
-                    for (int w = 0; w < kPackThreads / 32; ++w) {
-                        A = __dadd_rn(A, mom[0][w]), S = __dadd_rn(S, mom[1][w]);
-                        So = __dadd_rn(So, err[tid][w]), n_out += cnt[tid][w];
-                    }
+                    for (int b = 0; b <= tid; ++b) so += bin_sum[b], n_out += bin_cnt[b];
+                    const double So = ldexp(static_cast<double>(so), ex - 48);
                     const float p = __fdiv_rn(static_cast<float>(100 - tid), 100.0f);
                     const double sj = static_cast<double>(__fdiv_rn(__fmul_rn(p, amax), g));
                     const double lin = S + (top - 1.0) * So;
                     const double quad = static_cast<double>(K) + (top * top - 1.0) * static_cast<double>(n_out);
-                    const double E = A - 2.0 * sj * lin + sj * sj * quad;
-                    err[tid][0] = E;  // each thread touches its own row of err only
+                    err[tid][0] = A - 2.0 * sj * lin + sj * sj * quad;  // each thread touches its own row of err only
 #pragma unroll
                     for (int w = 1; w < kPackThreads / 32; ++w) err[tid][w] = 0.0;
                 }

@@ -198,6 +198,7 @@ struct Kv4Params {
 constexpr int kKvWarps = 4;
 constexpr int kKvTile = 16;          // tokens per warp tile
 constexpr int kKvPartial = kKvD + 2;
+constexpr float kKvSlack = 8.0f;     // weights stay below e^8 relative to the reference point
 
 __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -288,11 +289,7 @@ kv4_attention_partial_kernel(const Kv4Params p) {
             x.vzp[n] = *reinterpret_cast<const float2*>(p.v_zero + head_row + t);
         }
     };
-    Tile cur;
-    if (t_begin + kKvTile * warp < t_end) load_tile(cur, t_begin + kKvTile * warp);
-    for (int tb = t_begin + kKvTile * warp; tb < t_end; tb += kKvTile * kKvWarps) {
-        Tile nxt = cur;
-        if (tb + kKvTile * kKvWarps < t_end) load_tile(nxt, tb + kKvTile * kKvWarps);
+    auto process_tile = [&](const Tile& cur, int tb) {
         const uint4(&kraw)[2] = cur.kraw;
         const uint4(&vraw)[2] = cur.vraw;
         const float2(&ksc)[2] = cur.ksc;
@@ -324,8 +321,10 @@ kv4_attention_partial_kernel(const Kv4Params p) {
         }
         tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
         tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
-        const bool grew = tmax > m_run;
-        if (__any_sync(0xffffffffu, grew)) {  // rescale what the rows that found a new max have accumulated
+        // The reference point of the exponentials only has to keep them in range: it is moved (and the
+        // accumulators rescaled) when a row's scores exceed it by more than kKvSlack, not at every new max.
+        const bool grew = tmax > m_run + kKvSlack;
+        if (__any_sync(0xffffffffu, grew)) {
             const float corr = grew ? expf(m_run - tmax) : 1.0f;  // exp(-inf) = 0 on a row's first tile
             l_run *= corr, z_run *= corr;
 #pragma unroll
@@ -352,7 +351,22 @@ kv4_attention_partial_kernel(const Kv4Params p) {
             const uint32_t b0 = byte_to_half2(va[nt >> 2], nt & 3), b1 = byte_to_half2(vb[nt >> 2], nt & 3);
             mma_f16(o[nt], wh[0], wl[0], wh[1], wl[1], b0, b1);
         }
-        cur = nxt;
+    };
+    // two tile buffers used alternately, each loaded one tile ahead of its use
+    {
+        constexpr int stride = kKvTile * kKvWarps;
+        Tile ta, tb2;
+        int tb = t_begin + kKvTile * warp;
+        if (tb < t_end) load_tile(ta, tb);
+        while (tb < t_end) {
+            if (tb + stride < t_end) load_tile(tb2, tb + stride);
+            process_tile(ta, tb);
+            tb += stride;
+            if (tb >= t_end) break;
+            if (tb + stride < t_end) load_tile(ta, tb + stride);
+            process_tile(tb2, tb);
+            tb += stride;
+        }
     }
 
     // ---- merge: the four lanes of a row, then the warps through shared memory

@@ -196,44 +196,93 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
                     for (int w = 1; w < kPackThreads / 32; ++w) err[tid][w] = 0.0;
                 }
             } else {
-            // Integer sets: squared error of every candidate scale; per-element terms are formed exactly as
-            // d = w - s*level, d*d in fp64 without contraction, partial sums per thread in ascending k,
-            // then a fixed-order tree.
-            for (int c0 = 0; c0 < kNumCandidates; c0 += 8) {
-                LevelCoder<LV> coder[8];
-                double sd[8], e[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float p = __fdiv_rn(static_cast<float>(100 - (c0 + j)), 100.0f);
-                    coder[j].init(__fdiv_rn(__fmul_rn(p, amax), g));
-                    sd[j] = static_cast<double>(coder[j].s);
-                    e[j] = 0.0;
+                // Integer sets (Eq. 1): level q = clamp(rint(w / s)).  |q| is the number of boundaries
+                // m + 1/2 (m = 0, 1, ...) that |w| / s has crossed, up to 7 (1) on the positive and 8 (2)
+                // on the negative side for INT4 (the standard W2 set), and w q = |w| |q|, q^2 = sum over
+                // the crossed boundaries of 2m + 1.  So
+                //   E(s) = sum w^2 - 2 s sum_{crossings} |w| + s^2 sum_{crossings} (2m + 1),
+                // and as for the no-zero sets a crossing, once made, stays for every later (smaller)
+                // candidate scale: each (weight, boundary) pair is binned once at its switch index and the
+                // two sums of every candidate are prefix sums over the bins.  Decisions within 2^-20 of a
+                // boundary (where round-half-even and the rounding of the quotient matter) are taken with
+                // the division.  |w| enters as an exact 64-bit fixed-point integer (crossing weights are
+                // >= 0.015 max); pairs that have switched at the first candidate already -- the majority --
+                // are summed per thread first.
+                constexpr int kLimPos = (LV == QIFT_LEVELS_SYM) ? 1 : 7, kLimNeg = (LV == QIFT_LEVELS_SYM) ? 2 : 8;
+                float* sj = cand;  // [kNumCandidates] candidate scales, decreasing in j
+                for (int j = tid; j < kNumCandidates; j += blockDim.x) {
+                    sj[j] = __fdiv_rn(__fmul_rn(__fdiv_rn(static_cast<float>(100 - j), 100.0f), amax), g);
+                    bin_sum[j] = 0ull, bin_cnt[j] = 0;
                 }
+                __syncthreads();
+                int ex;
+                frexpf(amax, &ex);                              // amax < 2^ex
+                const double to_fixed = ldexp(1.0, 44 - ex);    // |w| * to_fixed < 2^44
+                const float guess = __fdiv_rn(100.0f * g, amax);
+                const float s_last = sj[kNumCandidates - 1];
+                double a2 = 0.0;
+                unsigned long long first_sum = 0;
+                int first_cnt = 0;
+                auto crossed = [&](float w, int j, int m) {  // exact: has |q| reached m + 1 at candidate j
+                    const int lv = level_from_code<LV>(nearest_code<LV>(w, sj[j]));
+                    return abs(lv) >= m + 1;
+                };
                 for (int k = tid; k < K; k += blockDim.x) {
                     const float w = row[k];
-                    const double wd = static_cast<double>(w);
-                    float mag[8];
-                    bool unsure = false;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) coder[j].fast(w, mag[j], unsure);
-                    if (unsure) {  // rare: some candidate's decision is too close to call without the division
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) coder[j].exact(w, mag[j]);
-                    }
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const double d = __dsub_rn(wd, __dmul_rn(sd[j], static_cast<double>(mag[j])));
-                        e[j] = __dadd_rn(e[j], __dmul_rn(d, d));
+                    const float a = fabsf(w);
+                    const double ad = static_cast<double>(a);
+                    a2 = __dadd_rn(a2, __dmul_rn(ad, ad));
+                    const unsigned long long fx = static_cast<unsigned long long>(__dmul_rn(ad, to_fixed));
+                    const int lim = (w < 0.0f) ? kLimNeg : kLimPos;
+                    for (int m = 0; m < lim; ++m) {
+                        const float h = static_cast<float>(m) + 0.5f;
+                        if (a < __fmul_rn(__fmul_rn(h, s_last), 0.999999f)) break;  // never crossed, nor the later ones
+                        // first guess: a > h p_j amax / g  <=>  (100 - j) < 100 a g / (h amax)
+                        int bsw = min(kNumCandidates, max(0, 101 - static_cast<int>(__fdiv_rn(a * guess, h))));
+                        while (bsw > 0 && a > __fmul_rn(h, sj[bsw - 1])) --bsw;
+                        while (bsw < kNumCandidates && !(a > __fmul_rn(h, sj[bsw]))) ++bsw;
+                        if (bsw > 0) {
+                            const float t = __fmul_rn(h, sj[bsw - 1]);
+                            if (__fsub_rn(t, a) <= t * 9.5367431640625e-07f)
+                                while (bsw > 0 && crossed(w, bsw - 1, m)) --bsw;
+                        }
+                        if (bsw < kNumCandidates) {
+                            const float t = __fmul_rn(h, sj[bsw]);
+                            if (__fsub_rn(a, t) <= t * 9.5367431640625e-07f)
+                                while (bsw < kNumCandidates && !crossed(w, bsw, m)) ++bsw;
+                        }
+                        if (bsw == 0) {
+                            first_sum += fx, first_cnt += 2 * m + 1;
+                        } else if (bsw < kNumCandidates) {
+                            atomicAdd(&bin_sum[bsw], fx);
+                            atomicAdd(&bin_cnt[bsw], 2 * m + 1);
+                        }
                     }
                 }
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    double v = e[j];
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) v = __dadd_rn(v, __shfl_xor_sync(0xffffffffu, v, o));
-                    if (lane == 0) err[c0 + j][warp] = v;
+                for (int o = 16; o > 0; o >>= 1) {
+                    a2 = __dadd_rn(a2, __shfl_xor_sync(0xffffffffu, a2, o));
+                    first_sum += __shfl_xor_sync(0xffffffffu, first_sum, o);
+                    first_cnt += __shfl_xor_sync(0xffffffffu, first_cnt, o);
                 }
-            }
+                if (lane == 0) {
+                    mom[0][warp] = a2;
+                    atomicAdd(&bin_sum[0], first_sum);
+                    atomicAdd(&bin_cnt[0], first_cnt);
+                }
+                __syncthreads();
+                if (tid < kNumCandidates) {  // E of candidate tid, left in err[tid][0]
+                    double A = 0.0;
+                    for (int w = 0; w < kPackThreads / 32; ++w) A = __dadd_rn(A, mom[0][w]);
+                    unsigned long long ps = 0;
+                    long long pq = 0;
+                    for (int bb = 0; bb <= tid; ++bb) ps += bin_sum[bb], pq += bin_cnt[bb];
+                    const double P = ldexp(static_cast<double>(ps), ex - 44);
+                    const double sd = static_cast<double>(sj[tid]);
+                    err[tid][0] = A - 2.0 * sd * P + sd * sd * static_cast<double>(pq);  // each thread touches its own row of err only
+#pragma unroll
+                    for (int w = 1; w < kPackThreads / 32; ++w) err[tid][w] = 0.0;
+                }
             }
             __syncthreads();
             if (tid == 0) {

@@ -397,23 +397,35 @@ kv4_attention_partial_kernel(const Kv4Params p) {
     }
 }
 
-// Merge the splits of each query head: one CTA per head, one thread per dimension.
+// Merge the splits of each query head: one CTA per head.  Thread s first turns split s's running max
+// into its weight exp(m_s - max) (one exponential per split, not per element), then thread d sums
+// dimension d over the splits.
+constexpr int kKvMaxSplits = 1024;
 __global__ void __launch_bounds__(kKvD)
 kv4_attention_combine_kernel(const Kv4Params p) {
+    __shared__ float weight[kKvMaxSplits];
+    __shared__ float wmax[kKvD / 32];
     pdl_launch_dependents();
     pdl_wait();
     const int h = blockIdx.x, d = threadIdx.x;
     const float* base = p.partial + static_cast<size_t>(h) * p.splits * kKvPartial;
     float mm = -INFINITY;
-    for (int s = 0; s < p.splits; ++s) mm = fmaxf(mm, base[s * kKvPartial + kKvD]);
+    for (int s = d; s < p.splits; s += kKvD) mm = fmaxf(mm, base[s * kKvPartial + kKvD]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
+    if ((d & 31) == 0) wmax[d >> 5] = mm;
+    __syncthreads();
+    mm = fmaxf(fmaxf(wmax[0], wmax[1]), fmaxf(wmax[2], wmax[3]));
+    for (int s = d; s < p.splits; s += kKvD) {
+        const float ms = base[s * kKvPartial + kKvD];
+        weight[s] = (ms > -INFINITY) ? expf(ms - mm) : 0.0f;
+    }
+    __syncthreads();
     float num = 0.0f, den = 0.0f;
     for (int s = 0; s < p.splits; ++s) {
-        const float ms = base[s * kKvPartial + kKvD];
-        if (ms > -INFINITY) {
-            const float f = expf(ms - mm);
-            num = fmaf(base[s * kKvPartial + d], f, num);
-            den = fmaf(base[s * kKvPartial + kKvD + 1], f, den);
-        }
+        const float f = weight[s];
+        num = fmaf(base[s * kKvPartial + d], f, num);
+        den = fmaf(base[s * kKvPartial + kKvD + 1], f, den);
     }
     p.out[static_cast<size_t>(h) * kKvD + d] = num / den;
 }

@@ -839,7 +839,7 @@ void kv4_splits(int T, int Hkv, int* splits, int* tokens_per_split) {
     const int round = kKvTile * kKvWarps;  // tokens the warps of a CTA take per trip
     tps = ((tps + round - 1) / round) * round;
     *tokens_per_split = tps;
-    *splits = (T + tps - 1) / tps;
+    *splits = (T + tps - 1) / tps;  // <= 2 * SMs / Hkv, far below kKvMaxSplits
 }
 }  // namespace
 
@@ -895,6 +895,7 @@ int qift_kv4_attention_decode(const float* q, const uint8_t* k_codes, const floa
         return QIFT_ERR_ALIGNMENT;
     Kv4Params p{};
     kv4_splits(T, Hkv, &p.splits, &p.tokens_per_split);
+    if (p.splits > kKvMaxSplits) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!workspace || workspace_bytes < static_cast<size_t>(Hq) * p.splits * kKvPartial * sizeof(float)) return QIFT_ERR_WORKSPACE;
     p.q = q, p.k_codes = k_codes, p.k_scale = k_scale, p.k_zero = k_zero, p.v_codes = v_codes, p.v_scale = v_scale;
     p.v_zero = v_zero, p.partial = static_cast<float*>(workspace), p.out = out;

@@ -237,6 +237,20 @@ int qift_w2a4_linear_static(const uint32_t* packed, const float* s_n, int levels
                             const float* s_a, int M, int N, int K, void* Y, int y_dtype,
                             int32_t* acc_debug, void* stream);
 
+/* Prefill with RESIDENT decoded weights.  The prefill product is compute-bound and a B200 has room to
+ * keep, beside the packed codes that the decode path streams, the same weights decoded to one int8 level
+ * per byte (4x the packed size for the two-bit sets): qift_expand_weights writes them once,
+ * qift_expanded_linear is then the tensor-core product alone (S4 + S5 on CTA pairs), with no
+ * per-call decoding pass and no scratch.
+ *   levels_out / levels_in  dev int8 [N][K] row-major, 256-byte aligned, N*K bytes; level(code[n][k])
+ *                           (MNZ in its odd-integer form -3..3, s_n being the half-scale)
+ *   other arguments as for qift_w2a4_linear; any M >= 1 (meant for M of a few hundred and more)
+ * The paper has no counterpart (it keeps no second copy of the weights); results are bit-identical to
+ * qift_w2a4_linear / qift_w4a4_linear. */
+int qift_expand_weights(const uint32_t* packed, int N, int K, int levels, int8_t* levels_out, void* stream);
+int qift_expanded_linear(const int8_t* levels_in, const float* s_n, const int8_t* q_a, const float* s_a, int M, int N,
+                         int K, void* Y, int y_dtype, int32_t* acc_debug, void* stream);
+
 /* ---------------------------------------------------------------------------------------------------
  * KV4: the 4-bit key / value cache of the paper's W2A4/KV4 setting (Sec. 4.1: "asymmetric key and value
  * quantization with clipping ratios of 0.95") and the single-query decode attention that reads it.

@@ -29,6 +29,7 @@ EXPORTS = [
     "qift_group_plan_bytes", "qift_group_plan", "qift_group_quantize_act", "qift_group_linear", "qift_group_forward",
     "qift_group_forward_host", "qift_static_scratch_bytes", "qift_w2a4_linear_static",
     "qift_kv4_quantize", "qift_kv4_attention_workspace_bytes", "qift_kv4_attention_decode",
+    "qift_expand_weights", "qift_expanded_linear",
 ]
 
 _lib = None
@@ -80,6 +81,8 @@ def lib() -> ctypes.CDLL:
         L.qift_static_scratch_bytes.restype = sz
         L.qift_static_scratch_bytes.argtypes = []
         L.qift_w2a4_linear_static.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, vp, ci, vp, vp]
+        L.qift_expand_weights.argtypes = [vp, ci, ci, ci, vp, vp]
+        L.qift_expanded_linear.argtypes = [vp, vp, vp, vp, ci, ci, ci, vp, ci, vp, vp]
         L.qift_kv4_quantize.argtypes = [vp, ci, ci, ci, ci, ci, cf, ci, ci, ci, vp, vp, vp, vp]
         L.qift_kv4_attention_workspace_bytes.restype = sz
         L.qift_kv4_attention_workspace_bytes.argtypes = [ci, ci, ci]
@@ -424,3 +427,26 @@ def qift_kv4_attention_decode(q, K: Kv4Cache, V: Kv4Cache, T: int, out=None, wor
                                            _ptr(V.zero), T, K.T_cap, Hq, K.H, D, _ptr(_dev(out, torch.float32)),
                                            _ptr(workspace), workspace.numel(), _stream()), "qift_kv4_attention_decode")
     return out
+
+
+# ---------------------------------------------------------------------------------------- resident decoded weights
+def qift_expand_weights(packed, N: int, K: int, levels: int, out=None):
+    """packed codes -> int8 levels [N, K] (kept resident for the prefill product)."""
+    _dev(packed)
+    if out is None:
+        out = torch.empty((N, K), dtype=torch.int8, device=packed.device)
+    _check(lib().qift_expand_weights(_ptr(packed), N, K, levels, _ptr(_dev(out, torch.int8)), _stream()), "qift_expand_weights")
+    return out
+
+
+def qift_expanded_linear(levels_i8, s_n, q_a, s_a, out_dtype=torch.float32, want_acc: bool = False, out=None):
+    """The prefill product on resident decoded weights -> (Y [M, N], acc int32 [M, N] or None)."""
+    _dev(levels_i8, torch.int8), _dev(s_n, torch.float32), _dev(q_a, torch.int8), _dev(s_a, torch.float32)
+    N, K = levels_i8.shape
+    M = q_a.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=q_a.device)
+    acc = torch.empty((M, N), dtype=torch.int32, device=q_a.device) if want_acc else None
+    _check(lib().qift_expanded_linear(_ptr(levels_i8), _ptr(s_n), _ptr(q_a), _ptr(s_a), M, N, K, _ptr(out),
+                                      F32 if out.dtype == torch.float32 else BF16, _ptr(acc), _stream()), "qift_expanded_linear")
+    return out, acc

@@ -242,6 +242,18 @@ int launch_gemm_pairs(const CUtensorMap& ma, const CUtensorMap& mb, const GemmPa
     return cuda_status(launch_pdl_pairs(kernel, dim3(2 * pairs), dim3(kPairThreads), smem, st, ma, mb, gp));
 }
 
+int run_expand(const uint32_t* packed, int lv, int N, int K, int8_t* wexp, cudaStream_t st) {
+    switch (lv) {
+        case QIFT_LEVELS_MNZ: return launch_expand<QIFT_LEVELS_MNZ>(packed, N, K, wexp, st);
+        case QIFT_LEVELS_POT: return launch_expand<QIFT_LEVELS_POT>(packed, N, K, wexp, st);
+        case QIFT_LEVELS_SYM: return launch_expand<QIFT_LEVELS_SYM>(packed, N, K, wexp, st);
+        default: return launch_expand<QIFT_LEVELS_INT4>(packed, N, K, wexp, st);
+    }
+}
+
+int run_i8_gemm(const int8_t* wexp, const float* s_n, const int8_t* q_a, const float* s_a, int M, int N, int K, void* Y,
+                int y_bf16, int32_t* acc_debug, cudaStream_t st, bool pairs);
+
 int run_prefill(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
                 void* Y, int y_bf16, int32_t* acc_debug, void* workspace, size_t workspace_bytes, cudaStream_t st,
                 bool pairs = false) {
@@ -250,14 +262,13 @@ int run_prefill(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
     if (!workspace || workspace_bytes < need) return QIFT_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
     int8_t* wexp = static_cast<int8_t*>(workspace);
-    int rc;
-    switch (lv) {
-        case QIFT_LEVELS_MNZ: rc = launch_expand<QIFT_LEVELS_MNZ>(packed, N, K, wexp, st); break;
-        case QIFT_LEVELS_POT: rc = launch_expand<QIFT_LEVELS_POT>(packed, N, K, wexp, st); break;
-        case QIFT_LEVELS_SYM: rc = launch_expand<QIFT_LEVELS_SYM>(packed, N, K, wexp, st); break;
-        default: rc = launch_expand<QIFT_LEVELS_INT4>(packed, N, K, wexp, st); break;
-    }
+    const int rc = run_expand(packed, lv, N, K, wexp, st);
     if (rc != QIFT_OK) return rc;
+    return run_i8_gemm(wexp, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st, pairs);
+}
+
+int run_i8_gemm(const int8_t* wexp, const float* s_n, const int8_t* q_a, const float* s_a, int M, int N, int K, void* Y,
+                int y_bf16, int32_t* acc_debug, cudaStream_t st, bool pairs) {
     const int m_tiles = (M + kGemmBM - 1) / kGemmBM;
     const bool narrow = m_tiles * ((N + 255) / 256) < sm_count();
     CUtensorMap ma, mb;
@@ -873,6 +884,25 @@ int qift_kv4_quantize(const void* X, int x_dtype, int T, int H, int D, int had_b
                                       T_cap, codes, scale, zero));
     return cuda_status(launch_pdl(kv4_quantize_kernel<false>, grid, dim3(256), 0, st, X, rows, H, had_block, r, clip_ratio, t0,
                                   T_cap, codes, scale, zero));
+}
+
+int qift_expand_weights(const uint32_t* packed, int N, int K, int levels, int8_t* levels_out, void* stream) {
+    if (!packed || !levels_out || N <= 0 || K <= 0 || !valid_levels(levels)) return QIFT_ERR_INVALID_ARG;
+    if (K % 16 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(packed) || (reinterpret_cast<uintptr_t>(levels_out) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
+    return run_expand(packed, levels, N, K, levels_out, static_cast<cudaStream_t>(stream));
+}
+
+int qift_expanded_linear(const int8_t* levels_in, const float* s_n, const int8_t* q_a, const float* s_a, int M, int N, int K,
+                         void* Y, int y_dtype, int32_t* acc_debug, void* stream) {
+    if (!levels_in || !s_n || !q_a || !s_a || !Y || M <= 0 || N <= 0 || K <= 0) return QIFT_ERR_INVALID_ARG;
+    if (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16) return QIFT_ERR_INVALID_ARG;
+    if (K % 16 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(levels_in) & 255u) != 0 || !aligned16(s_n) || !aligned16(q_a) || !aligned16(s_a) ||
+        !aligned16(Y) || (acc_debug && !aligned16(acc_debug)))
+        return QIFT_ERR_ALIGNMENT;
+    return run_i8_gemm(levels_in, s_n, q_a, s_a, M, N, K, Y, y_dtype == QIFT_BF16, acc_debug, static_cast<cudaStream_t>(stream),
+                       true);
 }
 
 size_t qift_kv4_attention_workspace_bytes(int T, int Hq, int Hkv) {

@@ -207,6 +207,23 @@ def test_prefill_pair_route_224_wide_tiles():
     assert_status_clean()
 
 
+@pytest.mark.parametrize("name", list(LEVELS))
+def test_resident_decoded_weights(name):
+    # decode once to int8 levels, then the product alone: levels and outputs against the oracle
+    lv = LEVELS[name][0]
+    M, N, K = 300, 520, 1040
+    p_ref, s_n, codes, q_a, s_a = make_problem(lv, M, N, K, seed=82)
+    lev = qift.qift_expand_weights(dev(p_ref.view(np.int32)), N, K, lv)
+    want = np.vectorize(lambda c: oracle.level_value(lv, int(c)))(codes).astype(np.int8)
+    assert np.array_equal(lev.cpu().numpy(), want)
+    for bf16 in (True, False):
+        y_ref, acc_ref = oracle.linear(codes, lv, s_n, q_a, s_a, bf16=bf16)
+        y, acc = qift.qift_expanded_linear(lev, dev(s_n), dev(q_a), dev(s_a),
+                                           out_dtype=torch.bfloat16 if bf16 else torch.float32, want_acc=True)
+        check_outputs(y, acc, y_ref, acc_ref, bf16)
+    assert_status_clean()
+
+
 def test_auto_route_and_public_entry_points():
     for M in (1, 16, 17, 140):
         for lv in (qift.MNZ, qift.INT4):

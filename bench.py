@@ -553,9 +553,20 @@ def run_prefill(torch, qift, L, device, gen, pk):
                                         M, m.N, m.K, vp(m.y.data_ptr()), qift.BF16, None, st)
             assert rc == 0, rc
 
+    def layer_resident_shared(_=True):
+        # a transformer layer quantizes four inputs, not seven: q / k / v share one, gate / up share one
+        for i, m in enumerate(mods):
+            if m.name in ("q", "o", "gate", "down"):
+                rc = L.qift_quantize_act(vp(m.x.data_ptr()), qift.BF16, M, m.K, m.B, CLIP, vp(q_a.data_ptr()), vp(s_a.data_ptr()), st)
+                assert rc == 0, rc
+            rc = L.qift_expanded_linear(vp(m.levels_i8.data_ptr()), vp(m.s_n.data_ptr()), vp(q_a.data_ptr()), vp(s_a.data_ptr()),
+                                        M, m.N, m.K, vp(m.y.data_ptr()), qift.BF16, None, st)
+            assert rc == 0, rc
+
     res = {}
     for key, fn, wq in (("layer_with_act_quant", layer, True), ("product_only", layer, False),
-                        ("resident_with_act_quant", layer_resident, True), ("resident_product_only", layer_resident, False)):
+                        ("resident_with_act_quant", layer_resident, True), ("resident_product_only", layer_resident, False),
+                        ("resident_shared_act_quant", layer_resident_shared, True)):
         for _ in range(3):
             fn(wq)
         torch.cuda.synchronize()
@@ -570,7 +581,9 @@ def run_prefill(torch, qift, L, device, gen, pk):
         ops = sum(2.0 * M * m.N * m.K for m in mods)
         res[key] = {"ms_per_layer": round(ms, 4), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
     res["resident_note"] = ("resident_*: the same layer through qift_expanded_linear on int8 levels decoded once "
-                            "(4x the packed size, kept beside the packed codes); product_only decodes on every call")
+                            "(4x the packed size, kept beside the packed codes); product_only decodes on every call; "
+                            "resident_shared_act_quant quantizes the four distinct inputs of a layer (q/k/v and gate/up share "
+                            "theirs) instead of one per module")
     tops = res["product_only"]["tops"]
     gemm_tops = res["resident_product_only"]["tops"]      # the GEMM kernel alone (no decoding pass in the timed region)
     int8_peak = 2.0 * pk["bf16_tflops"]    # dense int8 is nominally 2x bf16; scaled from the measured bf16 burst

@@ -57,7 +57,8 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 // steady state (and any stream capture after a warm-up call) makes no attribute call.
 // The same for a kernel that runs as clusters of two CTAs along x.
 template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl_pairs(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), unsigned cluster_x, dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                               Args&&... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -67,12 +68,16 @@ cudaError_t launch_pdl_pairs(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.x = cluster_x;
     attr[1].val.clusterDim.y = 1;
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl_pairs(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    return launch_pdl_cluster(kernel, 2u, grid, block, smem, st, std::forward<Args>(args)...);
 }
 
 template <typename K>
@@ -489,9 +494,9 @@ int qift_quantize_act(const void* X, int x_dtype, int M, int K, int had_block, f
     const int rc = check_rotation_shape(K, had_block, true);
     if (rc != QIFT_OK) return rc;
     if (!aligned16(X) || !aligned16(q_a) || !aligned16(s_a)) return QIFT_ERR_ALIGNMENT;
-    const size_t smem = padded_row_bytes(K);
     const float r = had_block > 1 ? inv_sqrt_block(had_block) : 1.0f;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t smem = padded_row_bytes(K);
     if (x_dtype == QIFT_BF16) {
         cudaError_t e = allow_smem(quantize_act_kernel<true>, smem);
         if (e != cudaSuccess) return cuda_status(e);

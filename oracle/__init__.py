@@ -81,11 +81,23 @@ def wht_blocks(x, B: int):
     return x
 
 
+def is_kron28(K: int, B: int) -> bool:
+    """B == K == 28 * 2^p selects the full-dimension rotation H_28 (x) H_{2^p}."""
+    P = K // 28
+    return B == K and K % 28 == 0 and P >= 1 and (P & (P - 1)) == 0
+
+
+def hadamard28():
+    H = np.empty((28, 28), dtype=np.int8)
+    lib().orc_hadamard28(H.ctypes.data_as(ctypes.c_void_p))
+    return H
+
+
 def rotate_weights(W, B: int):
-    """W Q with Q = blockdiag(H_B)/sqrt(B) along the last axis (fp32)."""
+    """W Q with Q = blockdiag(H_B)/sqrt(B) along the last axis (fp32); B = K = 28 * 2^p: full-dimension rotation."""
     W = _f32(W).copy()
     N, K = W.shape
-    assert (B & (B - 1)) == 0 and K % B == 0
+    assert ((B & (B - 1)) == 0 and K % B == 0) or is_kron28(K, B)
     lib().orc_rotate_weights(W.ctypes.data_as(ctypes.c_void_p), N, K, B)
     return W
 
@@ -110,7 +122,7 @@ def quantize_act(X, had_block: int, clip: float = 0.9):
     """-> (q_a int8 [M,K], s_a fp32 [M])."""
     X = _f32(X)
     M, K = X.shape
-    assert had_block == 0 or ((had_block & (had_block - 1)) == 0 and K % had_block == 0)
+    assert had_block == 0 or ((had_block & (had_block - 1)) == 0 and K % had_block == 0) or is_kron28(K, had_block)
     q = np.empty((M, K), dtype=np.int8)
     s = np.empty((M,), dtype=np.float32)
     scratch = np.empty((K,), dtype=np.float32)

@@ -15,6 +15,8 @@
 //                        in natural order applied by the textbook in-place butterfly, stages in
 //                        ascending stride, fp32.
 //   orc_rotate_weights   the same rotation with the orthonormal factor 1/sqrt(B) (offline, weights).
+//   orc_hadamard28, orc_wht_kron28   full-dimension rotation for K = 28 * 2^p (14336 = 28 * 512), which
+//                        has no Sylvester matrix: H_28 (Paley's second construction, q = 13) Kronecker H_{2^p}.
 //   orc_quantize_act     Eq. 1 with b = 4 on the rotated row, symmetric, clipping ratio as an
 //                        argument (Sec. 4.1 uses 0.9), one scale per token row.
 //   orc_weight_scale     Sec. 3.5 / Sec. 4.5.1: per-output-channel scale, either max-range or
@@ -138,12 +140,66 @@ void orc_wht_blocks(float* row, int K, int B) {
     }
 }
 
+// Hadamard matrix of order 28 by Paley's second construction with q = 13 (13 = 1 mod 4): with chi the
+// quadratic character mod 13 and C the symmetric conference matrix of order 14
+//   C = [0 1^T; 1 Q],  Q[i][j] = chi(i - j),   C C^T = 13 I,
+// H = [C + I, C - I; C - I, -C - I] has entries +-1, is symmetric and satisfies H H^T = 28 I.
+// H: 28 x 28, row-major, entries +1 / -1.
+void orc_hadamard28(int8_t* H) {
+    int chi[13];
+    for (int a = 0; a < 13; ++a) chi[a] = (a == 0) ? 0 : -1;
+    for (int x = 1; x < 13; ++x) chi[(x * x) % 13] = 1;
+    int C[14][14];
+    for (int i = 0; i < 14; ++i)
+        for (int j = 0; j < 14; ++j) {
+            if (i == 0 || j == 0) C[i][j] = (i == j) ? 0 : 1;
+            else C[i][j] = chi[((i - j) % 13 + 13) % 13];
+        }
+    for (int i = 0; i < 14; ++i)
+        for (int j = 0; j < 14; ++j) {
+            const int d = (i == j) ? 1 : 0;
+            H[i * 28 + j] = (int8_t)(C[i][j] + d);
+            H[i * 28 + j + 14] = (int8_t)(C[i][j] - d);
+            H[(i + 14) * 28 + j] = (int8_t)(C[i][j] - d);
+            H[(i + 14) * 28 + j + 14] = (int8_t)(-C[i][j] - d);
+        }
+}
+
+// Full-dimension rotation of a row of length K = 28 * P (P a power of two), unnormalised: the Kronecker
+// product H_28 (x) H_P, i.e. the Sylvester butterfly on every contiguous block of P entries, then H_28
+// across the 28 blocks at every position i < P.  Each output of the second step is the signed sum of its
+// 28 inputs taken in ascending block order in fp32 (first term +-x_0, then one add or subtract per
+// block).  (H_28 (x) H_P)(H_28 (x) H_P)^T = K I, and the matrix is symmetric.
+void orc_wht_kron28(float* row, int K) {
+    const int P = K / 28;
+    orc_wht_blocks(row, K, P);
+    int8_t H[28 * 28];
+    orc_hadamard28(H);
+    float x[28], y[28];
+    for (int i = 0; i < P; ++i) {
+        for (int j = 0; j < 28; ++j) x[j] = row[(size_t)j * P + i];
+        for (int r = 0; r < 28; ++r) {
+            float acc = (H[r * 28] > 0) ? x[0] : -x[0];
+            for (int j = 1; j < 28; ++j) acc = (H[r * 28 + j] > 0) ? acc + x[j] : acc - x[j];
+            y[r] = acc;
+        }
+        for (int r = 0; r < 28; ++r) row[(size_t)r * P + i] = y[r];
+    }
+}
+
+// The rotation selected by `B`: a power of two dividing K -> block-diagonal Sylvester blocks of B;
+// B = K = 28 * 2^p -> the full-dimension Kronecker rotation above.
+static void wht_select(float* row, int K, int B) {
+    if ((B & (B - 1)) == 0) orc_wht_blocks(row, K, B);
+    else orc_wht_kron28(row, K);
+}
+
 // W <- W Q with Q = blockdiag(H_B) / sqrt(B), applied to each row along K (H is symmetric).
 void orc_rotate_weights(float* W, int N, int K, int B) {
     const float r = inv_sqrt_block(B);
     for (int n = 0; n < N; ++n) {
         float* row = W + (size_t)n * K;
-        orc_wht_blocks(row, K, B);
+        wht_select(row, K, B);
         for (int k = 0; k < K; ++k) row[k] = row[k] * r;
     }
 }
@@ -169,7 +225,7 @@ void orc_quantize_act(const float* X, int M, int K, int B, float clip, int8_t* q
                       float* scratch) {
     for (int m = 0; m < M; ++m) {
         for (int k = 0; k < K; ++k) scratch[k] = X[(size_t)m * K + k];
-        if (B > 1) orc_wht_blocks(scratch, K, B);
+        if (B > 1) wht_select(scratch, K, B);
         const float amax = row_absmax(scratch, K);
         float s_u = 1.0f;
         if (amax != 0.0f) {

@@ -175,3 +175,43 @@ def test_bf16_roundtrip_helpers():
     assert np.array_equal(got, man)
     back = oracle.bf16_to_f32(got)
     assert np.array_equal(back.view(np.uint32), got.astype(np.uint32) << 16)
+
+
+# ------------------------------------------------------------------------------- full-dimension rotation, K = 28 * 2^p
+def sylvester(P):
+    return np.array([[(-1) ** bin(i & j).count("1") for j in range(P)] for i in range(P)], dtype=np.int64)
+
+
+def test_hadamard28_is_a_symmetric_hadamard_matrix():
+    H = oracle.hadamard28().astype(np.int64)
+    assert set(np.unique(H)) == {-1, 1}
+    assert np.array_equal(H @ H.T, 28 * np.eye(28, dtype=np.int64))     # closed form of a Hadamard matrix
+    assert np.array_equal(H, H.T)                                        # Paley II with q = 1 mod 4 is symmetric
+    # the conference core: first row / column of the top-left block C + I are all ones
+    assert np.all(H[0, :14] == 1) and np.all(H[:14, 0] == 1)
+
+
+@pytest.mark.parametrize("P", [1, 4, 16])
+def test_kron28_rotation_against_the_dense_kronecker_product(P):
+    K = 28 * P
+    H = np.kron(oracle.hadamard28().astype(np.int64), sylvester(P))      # block index outer, position inner
+    assert np.array_equal(H @ H.T, K * np.eye(K, dtype=np.int64))
+    x = synth.normal(77, 1, (3, K)).astype(np.float32)
+    got = oracle.rotate_weights(x, K).astype(np.float64) * np.sqrt(K)    # undo the orthonormal factor
+    want = x.astype(np.float64) @ H.T
+    assert np.allclose(got, want, rtol=0, atol=K * 2.0 ** -22 * np.abs(x).max())
+    # orthonormal and symmetric: applying it twice gives the input back
+    back = oracle.rotate_weights(oracle.rotate_weights(x, K), K)
+    assert np.allclose(back, x, atol=1e-5)
+
+
+def test_kron28_quantizer_uses_the_full_dimension_scale():
+    K = 28 * 16
+    x = synth.normal(78, 1, (2, K)).astype(np.float32)
+    x[:, 5] += 50.0                                                      # one outlier channel: spread over all K
+    q, s = oracle.quantize_act(x, K, 0.9)
+    qb, sb = oracle.quantize_act(x, 16, 0.9)                             # block-diagonal alternative
+    assert q.min() >= -8 and q.max() <= 7
+    u = oracle.rotate_weights(x, K).astype(np.float64)                   # orthonormal rotation of the row
+    assert np.allclose(s.astype(np.float64) * 7 / 0.9, np.abs(u).max(axis=1), rtol=1e-5)
+    assert np.all(s < 0.5 * sb)                                          # the outlier is diffused much further

@@ -111,12 +111,16 @@ int qift_unpack_codes(const uint32_t* packed, int N, int K, int levels, uint8_t*
 /* S0 (offline rotation, Sec. 3.1 / Sec. 4.1): Y = X Q with Q = blockdiag(H_B) / sqrt(B), H_B the
  * Sylvester-Walsh matrix in natural order, applied to every row of X fp32 [M,K] along K.  fp32
  * butterfly with stages in ascending stride, then one multiply by (float)(1/sqrt(B)).
- * had_block B: a power of two >= 2 dividing K.  K <= 16384, K % 16 == 0.  In place (Y == X) is allowed. */
+ * had_block B: a power of two >= 2 dividing K (block-diagonal Sylvester blocks), or B = K when K = 28 * 2^p
+ * (p >= 4; e.g. 14336 = 28 * 512): the full-dimension rotation H_28 (x) H_{2^p} / sqrt(K), H_28 by Paley's
+ * second construction (q = 13), the sum over the 28 blocks taken in ascending block order in fp32 -- there is
+ * no Sylvester matrix of such an order and the block-diagonal form rotates only inside blocks of 2^p.
+ * K <= 16384, K % 16 == 0.  In place (Y == X) is allowed. */
 int qift_rotate(const float* X, int M, int K, int had_block, float* Y, void* stream);
 
 /* S2 + S3 (online rotation + per-token symmetric INT4 quantizer; Eq. 1 with b = 4, Sec. 4.1).
  *   X        in  [M,K] fp32 or bf16 (bf16 is widened exactly)
- *   had_block    0 = no rotation, else a power of two >= 2 dividing K
+ *   had_block    0 = no rotation, else as for qift_rotate (a power of two >= 2 dividing K, or K = 28 * 2^p)
  *   clip_ratio   the paper uses 0.9; must be in (0, 1]
  *   q_a      out int8 [M,K], one value of [-8,7] per byte
  *   s_a      out fp32 [M]
@@ -190,7 +194,7 @@ typedef struct qift_group_problem {
     void* Y;                /* dev [M,N] output                               */
     int32_t* acc_debug;     /* dev [M,N] INT32 accumulators, or NULL          */
     int N, K;
-    int had_block;          /* 0 = no rotation, else power of two dividing K  */
+    int had_block;          /* 0 = no rotation, else as for qift_rotate       */
     int reserved;
 } qift_group_problem;
 

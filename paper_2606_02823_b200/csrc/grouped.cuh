@@ -26,7 +26,8 @@ struct GroupHeader {
     int total_items;    // row blocks over all problems
     int rows_per_item;  // 16 * RT
     int max_k;
-    int reserved[6];
+    int any_kron;       // some problem's had_block selects the full-dimension rotation (K = 28 * 2^p)
+    int reserved[5];
 };
 static_assert(sizeof(GroupHeader) == 64, "header is one 64-byte record");
 
@@ -53,7 +54,7 @@ constexpr uint32_t kGroupMagic = 0x51494654u;
 // q_a is written PRESCALED for the product kernel (see mma_tile_step): with two-bit weights the
 // bytes of the even code planes (k % 16 in 0..3 or 8..11) hold 4*q, with INT4 weights the bytes of
 // plane 0 (k % 8 in 0..3) hold 16*q; sumq holds the plain sum of q.
-template <bool BF16_IN>
+template <bool BF16_IN, bool KRON = false>
 __global__ void __launch_bounds__(kRowThreads)
 quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* __restrict__ sumq, int M, float clip,
                             int int4_weights) {
@@ -66,7 +67,7 @@ quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* _
     const GroupProblemDev P = problems[p];
     const size_t m = blockIdx.x % M;
     const int K = P.K, B = P.had_block;
-    const RowScale sc = block_row_scale(load_and_transform<BF16_IN>(P.X, m, K, B, row), clip, red);
+    const RowScale sc = block_row_scale(load_and_transform<BF16_IN, KRON>(P.X, m, K, B, row), clip, red);
     if (threadIdx.x == 0) P.s_a[m] = (B > 1) ? __fmul_rn(sc.s_u, P.inv_sqrt_b) : sc.s_u;
     // 32-bit word i of a 16-byte group = code plane (two-bit: i; INT4: i & 1); even planes are prescaled
     int total = quantize_row<true>(row, K, sc, P.q_a + m * K, int4_weights ? 16.0f : 4.0f, 1.0f);

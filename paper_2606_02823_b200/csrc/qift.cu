@@ -112,6 +112,7 @@ float inv_sqrt_block(int B) { return static_cast<float>(1.0 / std::sqrt(static_c
 int check_rotation_shape(int K, int had_block, bool allow_none) {
     if (K <= 0 || K % 16 != 0 || K > kMaxRowK) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (had_block == 0) return allow_none ? QIFT_OK : QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (had_block == K && K % 28 == 0 && is_pow2(K / 28) && K / 28 >= 16) return QIFT_OK;  // H_28 (x) H_{K/28}
     if (had_block < 2 || !is_pow2(had_block) || K % had_block != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
     return QIFT_OK;
 }
@@ -480,10 +481,11 @@ int qift_rotate(const float* X, int M, int K, int had_block, float* Y, void* str
     if (rc != QIFT_OK) return rc;
     if (!aligned16(X) || !aligned16(Y)) return QIFT_ERR_ALIGNMENT;
     const size_t smem = padded_row_bytes(K);
-    cudaError_t e = allow_smem(rotate_rows_kernel, smem);
+    auto kernel = is_pow2(had_block) ? rotate_rows_kernel<false> : rotate_rows_kernel<true>;
+    cudaError_t e = allow_smem(kernel, smem);
     if (e != cudaSuccess) return cuda_status(e);
-    return cuda_status(launch_pdl(rotate_rows_kernel, dim3(M), dim3(row_threads(K)), smem, static_cast<cudaStream_t>(stream), X,
-                                  K, had_block, inv_sqrt_block(had_block), Y));
+    return cuda_status(launch_pdl(kernel, dim3(M), dim3(row_threads(K)), smem, static_cast<cudaStream_t>(stream), X, K, had_block,
+                                  inv_sqrt_block(had_block), Y));
 }
 
 int qift_quantize_act(const void* X, int x_dtype, int M, int K, int had_block, float clip_ratio, int8_t* q_a, float* s_a,
@@ -497,16 +499,12 @@ int qift_quantize_act(const void* X, int x_dtype, int M, int K, int had_block, f
     const float r = had_block > 1 ? inv_sqrt_block(had_block) : 1.0f;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t smem = padded_row_bytes(K);
-    if (x_dtype == QIFT_BF16) {
-        cudaError_t e = allow_smem(quantize_act_kernel<true>, smem);
-        if (e != cudaSuccess) return cuda_status(e);
-        return cuda_status(launch_pdl(quantize_act_kernel<true>, dim3(M), dim3(row_threads(K)), smem, st, X, K, had_block,
-                                      clip_ratio, r, q_a, s_a));
-    }
-    cudaError_t e = allow_smem(quantize_act_kernel<false>, smem);
+    const bool kron = had_block > 1 && !is_pow2(had_block);
+    auto kernel = (x_dtype == QIFT_BF16) ? (kron ? quantize_act_kernel<true, true> : quantize_act_kernel<true, false>)
+                                         : (kron ? quantize_act_kernel<false, true> : quantize_act_kernel<false, false>);
+    cudaError_t e = allow_smem(kernel, smem);
     if (e != cudaSuccess) return cuda_status(e);
-    return cuda_status(launch_pdl(quantize_act_kernel<false>, dim3(M), dim3(row_threads(K)), smem, st, X, K, had_block,
-                                  clip_ratio, r, q_a, s_a));
+    return cuda_status(launch_pdl(kernel, dim3(M), dim3(row_threads(K)), smem, st, X, K, had_block, clip_ratio, r, q_a, s_a));
 }
 
 int qift_w2a4_linear(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a, const float* s_a, int M, int N,
@@ -622,7 +620,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     const int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : (M == 1) ? 64 : 32;  // must match dispatch_grouped's row tiles
     GroupHeader* h = static_cast<GroupHeader*>(plan_host);
     GroupProblemDev* d = reinterpret_cast<GroupProblemDev*>(h + 1);
-    int items = 0, max_k = 0;
+    int items = 0, max_k = 0, any_kron = 0;
     for (int i = 0; i < count; ++i) {
         const qift_group_problem& q = problems[i];
         if (!q.X || !q.packed || !q.s_n || !q.q_a || !q.s_a || !q.Y || q.N <= 0 || q.K <= 0) return QIFT_ERR_INVALID_ARG;
@@ -640,11 +638,13 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
         for (int j = 0; j < 5; ++j) o.pad[j] = 0;
         items += (q.N + rows_per_item - 1) / rows_per_item;
         if (q.K > max_k) max_k = q.K;
+        if (q.had_block > 1 && !is_pow2(q.had_block)) any_kron = 1;
     }
     *h = GroupHeader{};
     h->magic = kGroupMagic, h->count = count, h->M = M, h->levels = levels, h->y_bf16 = (y_dtype == QIFT_BF16);
     h->x_bf16 = (x_dtype == QIFT_BF16), h->clip = clip_ratio, h->total_items = items, h->rows_per_item = rows_per_item;
     h->max_k = max_k;
+    h->any_kron = any_kron;
     return cuda_status(cudaMemcpyAsync(plan_dev, plan_host, sizeof(GroupHeader) + static_cast<size_t>(count) * sizeof(GroupProblemDev),
                                        cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));
 }
@@ -734,15 +734,12 @@ int qift_group_quantize_act(const void* plan_host, const void* plan_dev, void* s
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int* sumq = const_cast<int*>(plan_sumq(plan_dev, h->count));
     const dim3 grid(static_cast<unsigned>(h->count) * h->M);
-    if (h->x_bf16) {
-        cudaError_t e = allow_smem(quantize_act_grouped_kernel<true>, smem);
-        if (e != cudaSuccess) return cuda_status(e);
-        return cuda_status(launch_pdl(quantize_act_grouped_kernel<true>, grid, dim3(kRowThreads), smem, st, dev, sumq, h->M, h->clip,
-                                      h->levels == QIFT_LEVELS_INT4 ? 1 : 0));
-    }
-    cudaError_t e = allow_smem(quantize_act_grouped_kernel<false>, smem);
+    const bool kron = h->any_kron != 0;  // some problem uses the full-dimension rotation: the variant with the 28-point pass
+    auto kernel = h->x_bf16 ? (kron ? quantize_act_grouped_kernel<true, true> : quantize_act_grouped_kernel<true, false>)
+                            : (kron ? quantize_act_grouped_kernel<false, true> : quantize_act_grouped_kernel<false, false>);
+    cudaError_t e = allow_smem(kernel, smem);
     if (e != cudaSuccess) return cuda_status(e);
-    return cuda_status(launch_pdl(quantize_act_grouped_kernel<false>, grid, dim3(kRowThreads), smem, st, dev, sumq, h->M, h->clip,
+    return cuda_status(launch_pdl(kernel, grid, dim3(kRowThreads), smem, st, dev, sumq, h->M, h->clip,
                                   h->levels == QIFT_LEVELS_INT4 ? 1 : 0));
 }
 

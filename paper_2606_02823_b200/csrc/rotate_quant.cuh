@@ -137,11 +137,82 @@ __device__ __forceinline__ float wht_pass_smem(float* row, int K, int B) {
     return amax;
 }
 
+// Hadamard matrix of order 28 (there is no Sylvester matrix of that order): Paley's second construction
+// with q = 13.  chi = quadratic character mod 13; conference matrix C = [0 1; 1 Q] with Q[i][j] =
+// chi(i - j); H = [C + I, C - I; C - I, -C - I].  Built at compile time, so that the fully unrolled
+// 28-point transform below turns every entry into the sign of an add.
+struct Hadamard28 {
+    signed char v[28][28];
+};
+constexpr Hadamard28 make_hadamard28() {
+    Hadamard28 t{};
+    int chi[13] = {};
+    for (int a = 1; a < 13; ++a) chi[a] = -1;
+    for (int x = 1; x < 13; ++x) chi[(x * x) % 13] = 1;
+    for (int i = 0; i < 14; ++i)
+        for (int j = 0; j < 14; ++j) {
+            const int c = (i == 0 || j == 0) ? ((i == j) ? 0 : 1) : chi[((i - j) % 13 + 13) % 13];
+            const int d = (i == j) ? 1 : 0;
+            t.v[i][j] = static_cast<signed char>(c + d);
+            t.v[i][j + 14] = static_cast<signed char>(c - d);
+            t.v[i + 14][j] = static_cast<signed char>(c - d);
+            t.v[i + 14][j + 14] = static_cast<signed char>(-c - d);
+        }
+    return t;
+}
+constexpr Hadamard28 kH28 = make_hadamard28();
+
+template <int R, int J>
+__device__ __forceinline__ float h28_acc(const float (&x)[28], float acc) {  // terms J..27 of row R, in order
+    if constexpr (J < 28) {
+        constexpr bool plus = kH28.v[R][J] > 0;
+        return h28_acc<R, J + 1>(x, plus ? __fadd_rn(acc, x[J]) : __fsub_rn(acc, x[J]));
+    } else {
+        return acc;
+    }
+}
+template <int R>
+__device__ __forceinline__ float h28_row(const float (&x)[28]) {  // signed sum in ascending order, first term +-x[0]
+    constexpr bool plus0 = kH28.v[R][0] > 0;
+    return h28_acc<R, 1>(x, plus0 ? x[0] : -x[0]);
+}
+template <int R>
+__device__ __forceinline__ void h28_rows(const float (&x)[28], float (&y)[28]) {
+    if constexpr (R < 28) {
+        y[R] = h28_row<R>(x);
+        h28_rows<R + 1>(x, y);
+    }
+}
+
+// Second factor of the full-dimension rotation H_28 (x) H_P of a row of K = 28 P entries (the first, the
+// Sylvester transform of every block of P, has been done): H_28 across the 28 blocks at every position.
+// Returns the thread's max |value| written.
+__device__ __forceinline__ float kron28_pass_smem(float* row, int P) {
+    float amax = 0.0f;
+    for (int i = threadIdx.x; i < P; i += blockDim.x) {
+        float x[28], y[28];
+#pragma unroll
+        for (int j = 0; j < 28; ++j) x[j] = row[pad_index(j * P + i)];
+        h28_rows<0>(x, y);
+#pragma unroll
+        for (int j = 0; j < 28; ++j) {
+            row[pad_index(j * P + i)] = y[j];
+            amax = fmaxf(amax, fabsf(y[j]));
+        }
+    }
+    return amax;
+}
+
 // Loads the row (fp32 or bf16), runs the strides 1..8 in registers, leaves the row in shared memory
 // (padded layout), then finishes the transform there.  B <= 1 means no rotation.  Returns the
 // thread's partial max |value| of the transformed row (taken in whichever pass ran last).
-template <bool BF16_IN>
-__device__ __forceinline__ float load_and_transform(const void* X, size_t row_index, int K, int B, float* row) {
+// KRON: compiled with the 28-point pass (56 more registers); kernels without it reject nothing -- the host
+// picks the variant from had_block.
+template <bool BF16_IN, bool KRON = false>
+__device__ __forceinline__ float load_and_transform(const void* X, size_t row_index, int K, int had_block, float* row) {
+    // had_block: a power of two = block-diagonal Sylvester blocks; K = 28 * 2^p = the full-dimension rotation
+    const bool kron = KRON && (had_block & (had_block - 1)) != 0;
+    const int B = kron ? K / 28 : had_block;
     const int groups = K / 16;
     const int stages0 = (B > 1) ? min(4, 31 - __clz(B)) : 0;
     float amax = 0.0f;
@@ -196,6 +267,12 @@ __device__ __forceinline__ float load_and_transform(const void* X, size_t row_in
     if (B > 4096) {
         amax = wht_pass_smem<4096, true>(row, K, B);
         __syncthreads();
+    }
+    if constexpr (KRON) {
+        if (kron) {
+            amax = kron28_pass_smem(row, B);
+            __syncthreads();
+        }
     }
     return amax;
 }
@@ -302,7 +379,7 @@ __device__ __forceinline__ int quantize_row(const float* row, int K, RowScale sc
 }
 
 // K2: rotate + quantize one token row per CTA.
-template <bool BF16_IN>
+template <bool BF16_IN, bool KRON = false>
 __global__ void __launch_bounds__(kRowThreads)
 quantize_act_kernel(const void* __restrict__ X, int K, int B, float clip, float inv_sqrt_b,
                     int8_t* __restrict__ q_a, float* __restrict__ s_a) {
@@ -311,19 +388,20 @@ quantize_act_kernel(const void* __restrict__ X, int K, int B, float clip, float 
     pdl_launch_dependents();
     pdl_wait();
     const size_t m = blockIdx.x;
-    const RowScale sc = block_row_scale(load_and_transform<BF16_IN>(X, m, K, B, row), clip, red);
+    const RowScale sc = block_row_scale(load_and_transform<BF16_IN, KRON>(X, m, K, B, row), clip, red);
     if (threadIdx.x == 0) s_a[m] = (B > 1) ? __fmul_rn(sc.s_u, inv_sqrt_b) : sc.s_u;
     quantize_row<false>(row, K, sc, q_a + m * K, 1.0f, 1.0f);
 }
 
 // S0: orthonormal blockwise rotation of fp32 rows.
+template <bool KRON>
 __global__ void __launch_bounds__(kRowThreads)
 rotate_rows_kernel(const float* __restrict__ X, int K, int B, float inv_sqrt_b, float* __restrict__ Y) {
     extern __shared__ __align__(16) float row[];
     pdl_launch_dependents();
     pdl_wait();
     const size_t m = blockIdx.x;
-    load_and_transform<false>(X, m, K, B, row);
+    load_and_transform<false, KRON>(X, m, K, B, row);
     for (int i = threadIdx.x; i < K / 4; i += blockDim.x) {
         float4 f = *reinterpret_cast<const float4*>(row + pad_index(4 * i));
         f.x = __fmul_rn(f.x, inv_sqrt_b), f.y = __fmul_rn(f.y, inv_sqrt_b);

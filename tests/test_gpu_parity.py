@@ -64,6 +64,46 @@ def test_quantize_act(M, K, B, bf16):
     assert_status_clean()
 
 
+@pytest.mark.parametrize("M,K", [(3, 14336), (2, 448), (5, 7168)])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_quantize_act_full_dimension_rotation(M, K, bf16):
+    # K = 28 * 2^p with had_block = K: H_28 (x) H_{2^p}, bit-exact with the oracle (same summation order)
+    x, _ = synth.activations(110 + M, M, K, max(1, K // 100))
+    xd = dev(x)
+    if bf16:
+        xd = xd.to(torch.bfloat16)
+        x = oracle.bf16_to_f32(xd.view(torch.int16).cpu().numpy().view(np.uint16))
+    q, s = qift.qift_quantize_act(xd, K, 0.9)
+    q_ref, s_ref = oracle.quantize_act(x, K, 0.9)
+    assert np.array_equal(q.cpu().numpy(), q_ref) and np.array_equal(s.cpu().numpy(), s_ref)
+    if not bf16:
+        W = synth.student_weights(8, M, K)
+        assert np.array_equal(qift.qift_rotate(dev(W), K).cpu().numpy(), oracle.rotate_weights(W, K))
+    assert_status_clean()
+
+
+def test_full_dimension_rotation_grouped_and_rejections():
+    # a plan that mixes a full-dimension problem with a block-diagonal one
+    lv, M = qift.MNZ, 2
+    probs, refs = [], []
+    for i, (N, K, B) in enumerate([(64, 14336, 14336), (48, 4096, 4096)]):
+        W = synth.gaussian_weights(700 + i, N, K)
+        x, _ = synth.activations(710 + i, M, K, 8)
+        p_ref, s_n, codes = oracle.pack_weights(W, lv, oracle.SCALE_ABSMAX)
+        q_ref, sa_ref = oracle.quantize_act(x, B, 0.9)
+        refs.append(oracle.linear(codes, lv, s_n, q_ref, sa_ref))
+        probs.append((dev(x), dev(p_ref.view(np.int32)), dev(s_n), B))
+    plan = qift.qift_group_plan(probs, lv, 0.9, want_acc=True)
+    outs = qift.qift_group_forward(plan)
+    for (y_ref, acc_ref), y, acc in zip(refs, outs, plan.accs):
+        check_outputs(y, acc, y_ref, acc_ref, False)
+    x = torch.zeros((1, 11008), device="cuda")
+    with pytest.raises(qift.QiftError) as e:
+        qift.qift_quantize_act(x, 11008, 0.9)                    # 11008 = 43 * 256: no construction for order 43 * 2^p here
+    assert e.value.status == qift.ERR_UNSUPPORTED_SHAPE
+    assert_status_clean()
+
+
 def test_quantize_act_zero_and_clip():
     x = np.zeros((2, 256), dtype=np.float32)
     x[1, 5] = -3.0

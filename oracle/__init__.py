@@ -302,3 +302,64 @@ def kv4_attention(q, kc, ks, kz, vc, vs, vz):
                             vc.ctypes.data_as(vp), vs.ctypes.data_as(vp), vz.ctypes.data_as(vp), T, Hq, Hkv, D,
                             out.ctypes.data_as(vp), scratch.ctypes.data_as(vp))
     return out
+
+
+# ------------------------------------------------------------------ quantizer diagnostics (Sec. 4.5)
+def _grid(g):
+    g = _f32(g).reshape(-1)
+    assert g.size == 4 and np.all(np.diff(g) > 0) and g[3] > 0
+    return g
+
+
+def grid_scale(W, grid, mode: int, want_errs: bool = False):
+    """Per-row scale of a four-level float grid -> (s_n fp32 [N], best_idx int32 [N][, errs fp64 [N,80]])."""
+    W = _f32(W)
+    g = _grid(grid)
+    N, K = W.shape
+    s = np.empty((N,), dtype=np.float32)
+    idx = np.zeros((N,), dtype=np.int32)
+    errs = np.zeros((N, num_candidates()), dtype=np.float64) if want_errs else None
+    vp = ctypes.c_void_p
+    lib().orc_grid_scale(W.ctypes.data_as(vp), N, K, g.ctypes.data_as(vp), int(mode), s.ctypes.data_as(vp),
+                         idx.ctypes.data_as(vp), errs.ctypes.data_as(vp) if want_errs else None)
+    return (s, idx, errs) if want_errs else (s, idx)
+
+
+def grid_codes(W, grid, s_n):
+    W = _f32(W)
+    g = _grid(grid)
+    s_n = _f32(s_n)
+    N, K = W.shape
+    codes = np.empty((N, K), dtype=np.uint8)
+    vp = ctypes.c_void_p
+    lib().orc_grid_codes(W.ctypes.data_as(vp), N, K, g.ctypes.data_as(vp), s_n.ctypes.data_as(vp),
+                         codes.ctypes.data_as(vp))
+    return codes
+
+
+def bucket_stats(W, codes, s_n, values):
+    """-> (count int64 [L], sqerr fp64 [L]) of the weights assigned to each of the L levels."""
+    W = _f32(W)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    s_n = _f32(s_n)
+    v = _f32(values).reshape(-1)
+    N, K = W.shape
+    assert codes.shape == W.shape and int(codes.max(initial=0)) < v.size
+    count = np.zeros((v.size,), dtype=np.int64)
+    sqerr = np.zeros((v.size,), dtype=np.float64)
+    vp = ctypes.c_void_p
+    lib().orc_bucket_stats(W.ctypes.data_as(vp), codes.ctypes.data_as(vp), N, K, s_n.ctypes.data_as(vp),
+                           v.ctypes.data_as(vp), v.size, count.ctypes.data_as(vp), sqerr.ctypes.data_as(vp))
+    return count, sqerr
+
+
+def ratio_scan(x, ratios):
+    """-> (beta fp64 [R], nmse fp64 [R]): best global scale and its NMSE for each grid {-1,-r,+r,+1}."""
+    x = _f32(x).reshape(-1)
+    r = np.ascontiguousarray(ratios, dtype=np.float64).reshape(-1)
+    beta = np.empty_like(r)
+    nmse = np.empty_like(r)
+    vp = ctypes.c_void_p
+    lib().orc_ratio_scan(x.ctypes.data_as(vp), ctypes.c_longlong(x.size), r.ctypes.data_as(vp), r.size,
+                         beta.ctypes.data_as(vp), nmse.ctypes.data_as(vp))
+    return beta, nmse

@@ -35,14 +35,21 @@
 //   orc_kv4_pack_token_pairs  values: two consecutive tokens of a dimension per byte (layout is the build's).
 //   orc_kv4_attention    single-query scaled dot-product attention over the dequantized cache (the
 //                        decode step whose memory traffic Sec. 1 calls the bottleneck), in fp64.
+//   orc_grid_*           Sec. 3.3 grid list: the same nearest-level quantizer for any four float levels
+//                        (Lloyd-Max, NF2, Far-MNZ next to the deployable sets), scale as in orc_weight_scale.
+//   orc_bucket_stats     Sec. 4.5.1: per assigned level, the share of weights and of squared error.
+//   orc_ratio_scan       Sec. 4.5.2: NMSE(r) = min over a global scale beta of the error of
+//                        beta * {-1,-r,+r,+1} on pooled samples, relative to their power.
 //
 // Parity pins for every function live in the CPU test-suite (closed forms, brute force, printed
 // table values); none is "parity unpinned" except the numeric value of a forward output on the real
 // models, which the paper never prints.
 
+#include <algorithm>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <vector>
 
 namespace {
 
@@ -487,6 +494,121 @@ void orc_kv4_attention(const float* q, const uint8_t* kc, const float* ks, const
                 out[(size_t)h * D + d] += p * ((double)vs[row] * ((double)vc[row * D + d] - (double)vz[row]));
         }
         for (int d = 0; d < D; ++d) out[(size_t)h * D + d] /= den;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Quantizer diagnostics (Sec. 4.5.1, 4.5.2) on four-level float grids (Sec. 3.3).
+// A grid is four ascending float levels g[0] < g[1] < g[2] < g[3], g[3] > 0.
+
+// Nearest level of w / s: the number of midpoints (g[i] + g[i+1]) / 2 below t; a tie goes to the
+// lower level.  The division and the midpoints are fp32.
+int orc_grid_code(const float* g, float w, float s) {
+    const float t = w / s;
+    int c = 0;
+    for (int i = 0; i < 3; ++i) c += (t > (g[i] + g[i + 1]) * 0.5f);
+    return c;
+}
+
+void orc_grid_codes(const float* W, int N, int K, const float* g, const float* s_n, uint8_t* codes) {
+    for (int n = 0; n < N; ++n)
+        for (int k = 0; k < K; ++k)
+            codes[(size_t)n * K + k] = (uint8_t)orc_grid_code(g, W[(size_t)n * K + k], s_n[n]);
+}
+
+double orc_grid_row_sqerr(const float* w, int K, const float* g, float s) {
+    double e = 0.0;
+    for (int k = 0; k < K; ++k) {
+        const double d = (double)w[k] - (double)s * (double)g[orc_grid_code(g, w[k], s)];
+        e += d * d;
+    }
+    return e;
+}
+
+// Per-row scale of a float grid: the row's absolute maximum (times a clipping ratio) lands on the
+// largest level g[3]; mode as in orc_weight_scale (1: ratio 1, 2: sweep of the same 80 ratios).
+void orc_grid_scale(const float* W, int N, int K, const float* g, int mode, float* s_n, int* best_idx,
+                    double* errs) {
+    for (int n = 0; n < N; ++n) {
+        const float* w = W + (size_t)n * K;
+        const float amax = row_absmax(w, K);
+        int best = 0;
+        float s = 1.0f;
+        double best_e = 0.0;
+        if (amax != 0.0f) {
+            const int cands = mode == SC_ABSMAX ? 1 : kNumCandidates;
+            for (int i = 0; i < cands; ++i) {
+                const float si = (orc_candidate_ratio(i) * amax) / g[3];
+                const double e = orc_grid_row_sqerr(w, K, g, si);
+                if (errs) errs[(size_t)n * kNumCandidates + i] = e;
+                if (i == 0 || e < best_e) {
+                    best_e = e;
+                    best = i;
+                    s = si;
+                }
+            }
+        }
+        s_n[n] = s;
+        if (best_idx) best_idx[n] = best;
+    }
+}
+
+// Bucket diagnostic: for each level index c < L, how many weights carry code c and the sum of
+// their squared reconstruction errors (w - s_n * value[c])^2 in fp64.  Shares are these divided
+// by their totals.
+void orc_bucket_stats(const float* W, const uint8_t* codes, int N, int K, const float* s_n, const float* value,
+                      int L, long long* count, double* sqerr) {
+    for (int c = 0; c < L; ++c) {
+        count[c] = 0;
+        sqerr[c] = 0.0;
+    }
+    for (int n = 0; n < N; ++n)
+        for (int k = 0; k < K; ++k) {
+            const int c = codes[(size_t)n * K + k];
+            const double d = (double)W[(size_t)n * K + k] - (double)s_n[n] * (double)value[c];
+            count[c] += 1;
+            sqerr[c] += d * d;
+        }
+}
+
+// Ratio scan.  For each ratio r the exact minimum over beta > 0 of
+//     f(beta) = sum_i (x_i - Q(x_i))^2,   Q = nearest of beta * {-1, -r, +r, +1},
+// divided by sum_i x_i^2.  With a = |x| sorted ascending, the j smallest samples go to the inner
+// level exactly when the decision threshold beta (1 + r) / 2 lies in [a_(j-1), a_j]; on that
+// interval f is the parabola  S2 - 2 beta (r A_j + B_j) + beta^2 (r^2 j + n - j)  with A_j the sum
+// of the j smallest a and B_j the sum of the others, so its minimum there is at the vertex clamped
+// to the interval; the answer is the least of these n + 1 minima.  fp64 throughout.
+void orc_ratio_scan(const float* x, long long n, const double* r, int R, double* beta, double* nmse) {
+    std::vector<double> a((size_t)n);
+    double S1 = 0.0, S2 = 0.0;
+    for (long long i = 0; i < n; ++i) a[(size_t)i] = std::fabs((double)x[i]);
+    std::sort(a.begin(), a.end());
+    for (long long i = 0; i < n; ++i) {
+        S1 += a[(size_t)i];
+        S2 += a[(size_t)i] * a[(size_t)i];
+    }
+    for (int q = 0; q < R; ++q) {
+        const double rr = r[q];
+        double best_f = S2, best_b = 0.0, A = 0.0;
+        for (long long j = 0; j <= n; ++j) {
+            const double lin = rr * A + (S1 - A);
+            const double quad = rr * rr * (double)j + (double)(n - j);
+            const double lo = (j == 0 ? 0.0 : a[(size_t)j - 1]) * 2.0 / (1.0 + rr);
+            double b = lin / quad;
+            if (b < lo) b = lo;
+            if (j < n) {
+                const double hi = a[(size_t)j] * 2.0 / (1.0 + rr);
+                if (b > hi) b = hi;
+            }
+            const double f = S2 - 2.0 * b * lin + b * b * quad;
+            if (f < best_f) {
+                best_f = f;
+                best_b = b;
+            }
+            if (j < n) A += a[(size_t)j];
+        }
+        beta[q] = best_b;
+        nmse[q] = S2 > 0.0 ? best_f / S2 : 0.0;
     }
 }
 

@@ -293,6 +293,46 @@ int qift_kv4_attention_decode(const float* q, const uint8_t* k_codes, const floa
                               int Hq, int Hkv, int D, float* out, void* workspace, size_t workspace_bytes,
                               void* stream);
 
+/* Quantizer diagnostics (not on the inference path).  Sec. 3.3 (list of evaluated grids), Sec. 4.5.1
+ * (bucket diagnostic), Sec. 4.5.2 (scale-invariant ratio scan).
+ *
+ * qift_diag_grid_quantize: nearest-level quantization of rotated weights onto s_n * grid for ANY four
+ * float levels (Lloyd-Max, NF2, Far-MNZ, or a deployable set written as floats).
+ *   W      in   fp32 [N,K] device, 16-byte aligned; K <= 16384
+ *   grid   in   HOST, four ascending levels, grid[3] > 0
+ *   s_n    in for QIFT_SCALE_GIVEN, out otherwise; fp32 [N] device.  ABSMAX: the row's absolute maximum
+ *               lands on grid[3]; MSE: the packer's sweep of 80 clipping ratios 1.00 .. 0.21, least
+ *               fp64 squared error, first index on ties (an all-zero row gets 1)
+ *   codes  out  uint8 [N,K] device, one code 0..3 per weight (index into grid); may be NULL
+ * Code of a weight: t = w / s_n (IEEE fp32 division); the number of fp32 midpoints
+ * (grid[i] + grid[i+1]) / 2 that t exceeds, so an exact midpoint goes to the lower level.  For the
+ * no-zero sets this is the rule of qift_pack_weights.
+ *
+ * qift_diag_bucket_stats: per level c < L, count[c] = weights with code c and sqerr[c] = the sum of
+ * (w - s_n * values[c])^2 over them in fp64; the shares of Sec. 4.5.1 are these over their totals.
+ *   codes  in   uint8 [N,K] device (qift_unpack_codes or qift_diag_grid_quantize), 4-byte aligned
+ *   values in   HOST, L level values (the level table of the set, or the float grid); L = 4 or 16
+ *   count  out  uint64 [L] device;  sqerr out fp64 [L] device (both overwritten)
+ * K % 4 == 0.  The order of the fp64 additions is not fixed: sums repeat to about 1e-15 relative.
+ *
+ * qift_diag_ratio_scan: for each ratio r, NMSE(r) = min over beta > 0 of
+ * sum_i (x_i - Q(x_i))^2 / sum_i x_i^2 with Q the nearest of beta * {-1, -r, +r, +1}, and the beta
+ * that attains it.  The minimum is exact: the magnitudes are sorted, and for every split of the sorted
+ * samples into inner and outer level the error is a parabola in beta whose constrained minimum is
+ * closed-form; the least over all n + 1 splits is the answer (fp64).
+ *   x      in   fp32 [n] device (pooled, normalized weights); 1 <= n <= 2^28
+ *   ratios in   HOST, R values in (0, 1]; 1 <= R <= 65535
+ *   beta, nmse  out fp64 [R] device
+ *   workspace   >= qift_diag_ratio_scan_workspace_bytes(n, R) bytes, device, 256-byte aligned
+ * Errors: INVALID_ARG, UNSUPPORTED_SHAPE (sizes outside the ranges above), ALIGNMENT, WORKSPACE, CUDA. */
+int qift_diag_grid_quantize(const float* W, int N, int K, const float* grid, int scale_mode, float* s_n,
+                            uint8_t* codes, void* stream);
+int qift_diag_bucket_stats(const float* W, const uint8_t* codes, int N, int K, const float* s_n,
+                           const float* values, int L, unsigned long long* count, double* sqerr, void* stream);
+size_t qift_diag_ratio_scan_workspace_bytes(long long n, int R);
+int qift_diag_ratio_scan(const float* x, long long n, const double* ratios, int R, double* beta, double* nmse,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronizes `stream`, then reads and clears the device status word in which a kernel records an
  * expired bounded wait.  QIFT_OK, QIFT_ERR_TIMEOUT or QIFT_ERR_CUDA.  `detail` (host, may be NULL)
  * receives the raw word: bits 0-7 the waiting site, the rest the block index. */

@@ -11,4 +11,5 @@ from .binding import (lib, status_string, QiftError, qift_packed_bytes, qift_wor
                       qift_forward_host, qift_group_plan_bytes, qift_group_plan, qift_group_quantize_act,
                       qift_group_linear, qift_group_forward, qift_group_forward_host, GroupPlan, qift_static_scratch_bytes,
                       qift_w2a4_linear_static, Kv4Cache, KV_KEYS, KV_VALUES, qift_kv4_quantize, qift_kv4_attention_workspace_bytes,
-                      qift_kv4_attention_decode, qift_expand_weights, qift_expanded_linear)
+                      qift_kv4_attention_decode, qift_expand_weights, qift_expanded_linear, qift_diag_grid_quantize,
+                      qift_diag_bucket_stats, qift_diag_ratio_scan_workspace_bytes, qift_diag_ratio_scan)

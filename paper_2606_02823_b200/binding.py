@@ -30,6 +30,7 @@ EXPORTS = [
     "qift_group_forward_host", "qift_static_scratch_bytes", "qift_w2a4_linear_static",
     "qift_kv4_quantize", "qift_kv4_attention_workspace_bytes", "qift_kv4_attention_decode",
     "qift_expand_weights", "qift_expanded_linear",
+    "qift_diag_grid_quantize", "qift_diag_bucket_stats", "qift_diag_ratio_scan_workspace_bytes", "qift_diag_ratio_scan",
 ]
 
 _lib = None
@@ -87,8 +88,13 @@ def lib() -> ctypes.CDLL:
         L.qift_kv4_attention_workspace_bytes.restype = sz
         L.qift_kv4_attention_workspace_bytes.argtypes = [ci, ci, ci]
         L.qift_kv4_attention_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, vp, vp, sz, vp]
+        L.qift_diag_grid_quantize.argtypes = [vp, ci, ci, vp, ci, vp, vp, vp]
+        L.qift_diag_bucket_stats.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, vp, vp]
+        L.qift_diag_ratio_scan_workspace_bytes.restype = sz
+        L.qift_diag_ratio_scan_workspace_bytes.argtypes = [ctypes.c_longlong, ci]
+        L.qift_diag_ratio_scan.argtypes = [vp, ctypes.c_longlong, vp, ci, vp, vp, vp, sz, vp]
         for name in EXPORTS:
-            if name not in ("qift_status_string", "qift_packed_bytes", "qift_workspace_bytes",
+            if name not in ("qift_diag_ratio_scan_workspace_bytes", "qift_status_string", "qift_packed_bytes", "qift_workspace_bytes",
                             "qift_forward_scratch_bytes", "qift_group_plan_bytes", "qift_static_scratch_bytes",
                             "qift_workspace_bytes_route", "qift_kv4_attention_workspace_bytes"):
                 getattr(L, name).restype = ci
@@ -450,3 +456,57 @@ def qift_expanded_linear(levels_i8, s_n, q_a, s_a, out_dtype=torch.float32, want
     _check(lib().qift_expanded_linear(_ptr(levels_i8), _ptr(s_n), _ptr(q_a), _ptr(s_a), M, N, K, _ptr(out),
                                       F32 if out.dtype == torch.float32 else BF16, _ptr(acc), _stream()), "qift_expanded_linear")
     return out, acc
+
+
+# ------------------------------------------------------------------------------------------ quantizer diagnostics
+def _host_array(values, ctype):
+    values = [float(v) for v in values]
+    return (ctype * len(values))(*values), len(values)
+
+
+def qift_diag_grid_quantize(W, grid, scale_mode: int, s_n=None, want_codes: bool = True):
+    """Nearest-level quantization onto four float levels -> (s_n fp32 [N], codes uint8 [N, K] or None)."""
+    _dev(W, torch.float32)
+    N, K = W.shape
+    g, n = _host_array(grid, ctypes.c_float)
+    if n != 4:
+        raise ValueError("a grid has four levels")
+    if s_n is None:
+        if scale_mode == SCALE_GIVEN:
+            raise ValueError("SCALE_GIVEN needs s_n")
+        s_n = torch.empty((N,), dtype=torch.float32, device=W.device)
+    codes = torch.empty((N, K), dtype=torch.uint8, device=W.device) if want_codes else None
+    _check(lib().qift_diag_grid_quantize(_ptr(W), N, K, g, scale_mode, _ptr(_dev(s_n, torch.float32)), _ptr(codes), _stream()),
+           "qift_diag_grid_quantize")
+    return s_n, codes
+
+
+def qift_diag_bucket_stats(W, codes, s_n, values):
+    """-> (count int64 [L], sqerr fp64 [L]): weights and squared error per assigned level."""
+    _dev(W, torch.float32), _dev(codes, torch.uint8), _dev(s_n, torch.float32)
+    N, K = W.shape
+    v, L = _host_array(values, ctypes.c_float)
+    count = torch.empty((L,), dtype=torch.int64, device=W.device)
+    sqerr = torch.empty((L,), dtype=torch.float64, device=W.device)
+    _check(lib().qift_diag_bucket_stats(_ptr(W), _ptr(codes), N, K, _ptr(s_n), v, L, _ptr(count), _ptr(sqerr), _stream()),
+           "qift_diag_bucket_stats")
+    return count, sqerr
+
+
+def qift_diag_ratio_scan_workspace_bytes(n: int, R: int) -> int:
+    return int(lib().qift_diag_ratio_scan_workspace_bytes(int(n), int(R)))
+
+
+def qift_diag_ratio_scan(x, ratios, workspace=None):
+    """x fp32 [n] -> (beta fp64 [R], nmse fp64 [R]) for the grids {-1, -r, +r, +1}."""
+    _dev(x, torch.float32)
+    n = x.numel()
+    r, R = _host_array(ratios, ctypes.c_double)
+    need = qift_diag_ratio_scan_workspace_bytes(n, R)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=x.device)
+    beta = torch.empty((R,), dtype=torch.float64, device=x.device)
+    nmse = torch.empty((R,), dtype=torch.float64, device=x.device)
+    _check(lib().qift_diag_ratio_scan(_ptr(x), n, r, R, _ptr(beta), _ptr(nmse), _ptr(workspace), workspace.numel(), _stream()),
+           "qift_diag_ratio_scan")
+    return beta, nmse

@@ -1,0 +1,513 @@
+// Quantizer diagnostics on the GPU (Sec. 4.5.1 bucket diagnostic, Sec. 4.5.2 ratio scan) and the
+// nearest-level quantizer for any four float levels (Sec. 3.3 grid list: Lloyd-Max, NF2, Far-MNZ
+// next to the deployable sets).  None of this is on the inference path; everything that decides an
+// integer (a code, a sort position) is exact, the error sums are fp64.
+#pragma once
+
+#include <cstdint>
+
+#include "common.cuh"
+
+namespace qift {
+
+constexpr int kDiagCandidates = 80;  // clipping ratios 1.00, 0.99, ..., 0.21 (the packer's sweep)
+constexpr int kDiagThreads = 256;
+constexpr int kDiagWarps = kDiagThreads / 32;
+
+struct Grid4 {
+    float g[4];  // ascending levels
+    float m[3];  // fp32 midpoints (g[i] + g[i+1]) / 2
+};
+
+// Code and level of t = w / s: the number of midpoints below t (a tie goes to the lower level).
+__device__ __forceinline__ int grid_code(const Grid4& G, float t, float& level) {
+    const bool a = t > G.m[0], b = t > G.m[1], c = t > G.m[2];
+    level = b ? (c ? G.g[3] : G.g[2]) : (a ? G.g[1] : G.g[0]);
+    return static_cast<int>(a) + static_cast<int>(b) + static_cast<int>(c);
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// One CTA per weight row: absolute maximum, scale (given / maximum on the top level / the sweep of
+// 80 clipping ratios with the least fp64 squared error, first index on ties), then the codes, one
+// per byte.  Each warp evaluates every eighth candidate over the whole row, so a candidate's error is
+// one warp reduction and the block meets once.
+__global__ void __launch_bounds__(kDiagThreads) grid_quantize_kernel(const float* __restrict__ W, int K, Grid4 G, int mode,
+                                                                     float* __restrict__ s_n, uint8_t* __restrict__ codes) {
+    extern __shared__ float row[];
+    __shared__ float red[kDiagWarps];
+    __shared__ double err[kDiagCandidates];
+    __shared__ float s_sh;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const size_t base = static_cast<size_t>(blockIdx.x) * K;
+    float amax = 0.0f;
+    for (int k = tid; k < K; k += kDiagThreads) {
+        const float w = W[base + k];
+        row[k] = w;
+        amax = fmaxf(amax, fabsf(w));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if (lane == 0) red[warp] = amax;
+    __syncthreads();
+    amax = red[0];
+#pragma unroll
+    for (int w = 1; w < kDiagWarps; ++w) amax = fmaxf(amax, red[w]);
+
+    auto candidate = [&](int i) {
+        return __fdiv_rn(__fmul_rn(__fdiv_rn(static_cast<float>(100 - i), 100.0f), amax), G.g[3]);
+    };
+    if (mode == 2 && amax != 0.0f) {
+        for (int i = warp; i < kDiagCandidates; i += kDiagWarps) {
+            const float s = candidate(i);
+            const double sd = static_cast<double>(s);
+            double e = 0.0;
+            for (int k = lane; k < K; k += 32) {
+                const float w = row[k];
+                float level;
+                grid_code(G, __fdiv_rn(w, s), level);
+                const double d = static_cast<double>(w) - sd * static_cast<double>(level);
+                e = fma(d, d, e);
+            }
+            e = warp_sum(e);
+            if (lane == 0) err[i] = e;
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        float s = 1.0f;
+        if (mode == 0) {
+            s = s_n[blockIdx.x];
+        } else if (amax != 0.0f) {
+            int best = 0;
+            if (mode == 2)
+                for (int i = 1; i < kDiagCandidates; ++i)
+                    if (err[i] < err[best]) best = i;
+            s = candidate(best);
+        }
+        if (mode != 0) s_n[blockIdx.x] = s;
+        s_sh = s;
+    }
+    __syncthreads();
+    if (codes) {
+        const float s = s_sh;
+        for (int k = tid; k < K; k += kDiagThreads) {
+            float level;
+            codes[base + k] = static_cast<uint8_t>(grid_code(G, __fdiv_rn(row[k], s), level));
+        }
+    }
+}
+
+// Bucket diagnostic: count and fp64 squared error per assigned level.  Four weights and four code
+// bytes per thread and trip; per-thread accumulators for every level (selected by predicates, no
+// indexed registers), one block reduction, one atomic per level and block.
+struct BucketValues {
+    float v[16];
+};
+
+template <int L>
+__global__ void __launch_bounds__(kDiagThreads) bucket_stats_kernel(const float* __restrict__ W, const uint8_t* __restrict__ codes,
+                                                                    long long total4, int K, const float* __restrict__ s_n,
+                                                                    BucketValues values, unsigned long long* __restrict__ count,
+                                                                    double* __restrict__ sqerr) {
+    double e[L];
+    unsigned n[L];
+#pragma unroll
+    for (int c = 0; c < L; ++c) {
+        e[c] = 0.0;
+        n[c] = 0u;
+    }
+    __shared__ double e_sh[kDiagWarps][L];
+    __shared__ unsigned long long n_sh[kDiagWarps][L];
+    const long long stride = static_cast<long long>(gridDim.x) * kDiagThreads;
+    for (long long v = static_cast<long long>(blockIdx.x) * kDiagThreads + threadIdx.x; v < total4; v += stride) {
+        const float4 w4 = reinterpret_cast<const float4*>(W)[v];
+        const uint32_t c4 = reinterpret_cast<const uint32_t*>(codes)[v];
+        const double s = static_cast<double>(s_n[(v * 4) / K]);
+        const float w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int code = (c4 >> (8 * i)) & 0xff;
+            float level = 0.0f;
+#pragma unroll
+            for (int c = 0; c < L; ++c) level = code == c ? values.v[c] : level;
+            const double d = static_cast<double>(w[i]) - s * static_cast<double>(level);
+            const double d2 = d * d;
+#pragma unroll
+            for (int c = 0; c < L; ++c) {
+                e[c] += code == c ? d2 : 0.0;
+                n[c] += code == c ? 1u : 0u;
+            }
+        }
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int c = 0; c < L; ++c) {
+        const double es = warp_sum(e[c]);
+        unsigned long long ns = n[c];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ns += __shfl_xor_sync(0xffffffffu, ns, o);
+        if (lane == 0) {
+            e_sh[warp][c] = es;
+            n_sh[warp][c] = ns;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < L) {
+        double es = 0.0;
+        unsigned long long ns = 0ull;
+#pragma unroll
+        for (int w = 0; w < kDiagWarps; ++w) {
+            es += e_sh[w][threadIdx.x];
+            ns += n_sh[w][threadIdx.x];
+        }
+        if (ns) {
+            atomicAdd(&sqerr[threadIdx.x], es);
+            atomicAdd(&count[threadIdx.x], ns);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------ ratio scan
+// Step 1: the magnitudes as sortable keys (the bit pattern of a non-negative float orders like the value).
+__global__ void __launch_bounds__(kDiagThreads) abs_keys_kernel(const float* __restrict__ x, long long n, uint32_t* __restrict__ keys) {
+    const long long stride = static_cast<long long>(gridDim.x) * kDiagThreads;
+    for (long long i = static_cast<long long>(blockIdx.x) * kDiagThreads + threadIdx.x; i < n; i += stride)
+        keys[i] = __float_as_uint(x[i]) & 0x7fffffffu;
+}
+
+// Step 2: least-significant-digit radix sort, 8 bits per pass.  The keys are cut into V contiguous
+// segments, one warp per segment.  Per pass: (a) each warp counts the digits of its segment into
+// hist[digit][segment]; (b) one CTA per digit turns its row of hist into exclusive prefix sums and
+// leaves the row total; (c) each warp walks its segment in order, 32 keys at a time, and places every
+// key at (keys with a smaller digit) + (same digit in earlier segments) + (same digit earlier in this
+// segment), the last term from a warp match, which keeps equal digits in order (a stable pass).
+__device__ __forceinline__ uint32_t lanemask_lt() {
+    uint32_t m;
+    asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+    return m;
+}
+
+__global__ void __launch_bounds__(kDiagThreads) radix_hist_kernel(const uint32_t* __restrict__ keys, long long n, int seg, int V, int shift,
+                                                                  uint32_t* __restrict__ hist) {
+    __shared__ uint32_t ctr[kDiagWarps][256];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int v = blockIdx.x * kDiagWarps + warp;
+    for (int d = lane; d < 256; d += 32) ctr[warp][d] = 0u;
+    __syncwarp();
+    if (v < V) {
+        const long long lo = static_cast<long long>(v) * seg;
+        const long long hi = lo + seg < n ? lo + seg : n;
+        for (long long i0 = lo; i0 < hi; i0 += 32) {
+            const long long i = i0 + lane;
+            const bool valid = i < hi;
+            const uint32_t d = valid ? (keys[i] >> shift) & 255u : 256u + lane;
+            const uint32_t peers = __match_any_sync(0xffffffffu, d);
+            if (valid && (peers & lanemask_lt()) == 0u) ctr[warp][d] += __popc(peers);
+            __syncwarp();
+        }
+        for (int d = lane; d < 256; d += 32) hist[static_cast<size_t>(d) * V + v] = ctr[warp][d];
+    }
+}
+
+// One CTA of 1024 threads per digit; V <= 4096 entries, four per thread.
+__global__ void __launch_bounds__(1024) radix_rowscan_kernel(uint32_t* __restrict__ hist, int V, uint32_t* __restrict__ totals) {
+    __shared__ uint32_t wsum[32];
+    uint32_t* rowp = hist + static_cast<size_t>(blockIdx.x) * V;
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    uint32_t a[4];
+    uint32_t s = 0u;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int idx = t * 4 + i;
+        a[i] = idx < V ? rowp[idx] : 0u;
+        s += a[i];
+    }
+    uint32_t inc = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += y;
+    }
+    if (lane == 31) wsum[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = wsum[lane];
+        uint32_t winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += y;
+        }
+        wsum[lane] = winc - w;  // exclusive over warps
+        if (lane == 31) totals[blockIdx.x] = winc;
+    }
+    __syncthreads();
+    uint32_t run = wsum[warp] + inc - s;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int idx = t * 4 + i;
+        if (idx < V) rowp[idx] = run;
+        run += a[i];
+    }
+}
+
+__global__ void __launch_bounds__(kDiagThreads) radix_scatter_kernel(const uint32_t* __restrict__ in, long long n, int seg, int V, int shift,
+                                                                     const uint32_t* __restrict__ hist, const uint32_t* __restrict__ totals,
+                                                                     uint32_t* __restrict__ out) {
+    __shared__ uint32_t ctr[kDiagWarps][256];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int v = blockIdx.x * kDiagWarps + warp;
+    if (v >= V) return;
+    {   // digits 8 lane .. 8 lane + 7: keys with a smaller digit + the same digit in earlier segments
+        uint32_t t[8];
+        uint32_t s = 0u;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            t[i] = totals[lane * 8 + i];
+            s += t[i];
+        }
+        uint32_t inc = s;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += y;
+        }
+        uint32_t run = inc - s;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int d = lane * 8 + i;
+            ctr[warp][d] = run + hist[static_cast<size_t>(d) * V + v];
+            run += t[i];
+        }
+    }
+    __syncwarp();
+    const long long lo = static_cast<long long>(v) * seg;
+    const long long hi = lo + seg < n ? lo + seg : n;
+    for (long long i0 = lo; i0 < hi; i0 += 32) {
+        const long long i = i0 + lane;
+        const bool valid = i < hi;
+        const uint32_t key = valid ? in[i] : 0u;
+        const uint32_t d = valid ? (key >> shift) & 255u : 256u + lane;
+        const uint32_t peers = __match_any_sync(0xffffffffu, d);
+        const uint32_t rank = __popc(peers & lanemask_lt());
+        uint32_t pos = 0u;
+        if (valid) pos = ctr[warp][d] + rank;
+        __syncwarp();
+        if (valid && rank == 0u) ctr[warp][d] += __popc(peers);
+        __syncwarp();
+        if (valid) out[pos] = key;
+    }
+}
+
+// Step 3: P[j] = sum of the j smallest magnitudes (exclusive prefix sums, fp64) and the totals
+// S1 = sum a, S2 = sum a^2.  Blocks of 4096 keys: block sums, a one-CTA scan of the block sums, and
+// the prefix sums inside each block on top of its base.
+constexpr int kScanPerThread = 16;
+constexpr int kScanBlock = kDiagThreads * kScanPerThread;
+
+__device__ __forceinline__ double block_exclusive_scan(double v, double* warp_sh, double& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    double inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double y = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += y;
+    }
+    if (lane == 31) warp_sh[warp] = inc;
+    __syncthreads();
+    double base = 0.0, tot = 0.0;
+#pragma unroll
+    for (int w = 0; w < kDiagWarps; ++w) {
+        if (w < warp) base += warp_sh[w];
+        tot += warp_sh[w];
+    }
+    total = tot;
+    __syncthreads();
+    return base + inc - v;
+}
+
+__global__ void __launch_bounds__(kDiagThreads) scan_block_sums_kernel(const uint32_t* __restrict__ keys, long long n,
+                                                                       double* __restrict__ block_s1, double* __restrict__ block_s2) {
+    __shared__ double sh[2][kDiagWarps];
+    const long long lo = static_cast<long long>(blockIdx.x) * kScanBlock + static_cast<long long>(threadIdx.x) * kScanPerThread;
+    double s1 = 0.0, s2 = 0.0;
+#pragma unroll
+    for (int i = 0; i < kScanPerThread; ++i) {
+        if (lo + i < n) {
+            const double a = static_cast<double>(__uint_as_float(keys[lo + i]));
+            s1 += a;
+            s2 = fma(a, a, s2);
+        }
+    }
+    s1 = warp_sum(s1);
+    s2 = warp_sum(s2);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) {
+        sh[0][warp] = s1;
+        sh[1][warp] = s2;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double a = 0.0, b = 0.0;
+#pragma unroll
+        for (int w = 0; w < kDiagWarps; ++w) {
+            a += sh[0][w];
+            b += sh[1][w];
+        }
+        block_s1[blockIdx.x] = a;
+        block_s2[blockIdx.x] = b;
+    }
+}
+
+// One CTA: exclusive scan of block_s1 in place, totals[0] = S1, totals[1] = S2.
+__global__ void __launch_bounds__(kDiagThreads) scan_bases_kernel(double* __restrict__ block_s1, const double* __restrict__ block_s2,
+                                                                  int blocks, double* __restrict__ totals) {
+    __shared__ double warp_sh[kDiagWarps];
+    double carry = 0.0, s2 = 0.0;
+    for (int b0 = 0; b0 < blocks; b0 += kDiagThreads) {
+        const int b = b0 + threadIdx.x;
+        const double v = b < blocks ? block_s1[b] : 0.0;
+        s2 += b < blocks ? block_s2[b] : 0.0;
+        double total;
+        const double ex = block_exclusive_scan(v, warp_sh, total);
+        if (b < blocks) block_s1[b] = carry + ex;
+        carry += total;
+    }
+    s2 = warp_sum(s2);
+    if ((threadIdx.x & 31) == 0) warp_sh[threadIdx.x >> 5] = s2;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+#pragma unroll
+        for (int w = 0; w < kDiagWarps; ++w) t += warp_sh[w];
+        totals[0] = carry;
+        totals[1] = t;
+    }
+}
+
+__global__ void __launch_bounds__(kDiagThreads) scan_write_kernel(const uint32_t* __restrict__ keys, long long n,
+                                                                  const double* __restrict__ bases, double* __restrict__ P) {
+    __shared__ double warp_sh[kDiagWarps];
+    const long long lo = static_cast<long long>(blockIdx.x) * kScanBlock + static_cast<long long>(threadIdx.x) * kScanPerThread;
+    double a[kScanPerThread];
+    double s = 0.0;
+#pragma unroll
+    for (int i = 0; i < kScanPerThread; ++i) {
+        a[i] = lo + i < n ? static_cast<double>(__uint_as_float(keys[lo + i])) : 0.0;
+        s += a[i];
+    }
+    double total;
+    double run = bases[blockIdx.x] + block_exclusive_scan(s, warp_sh, total);
+#pragma unroll
+    for (int i = 0; i < kScanPerThread; ++i) {
+        if (lo + i < n) P[lo + i] = run;
+        run += a[i];
+    }
+}
+
+// Step 4 (Sec. 4.5.2): for ratio r and every split j (the j smallest magnitudes on the inner level),
+// the least value on [a_(j-1), a_j] * 2 / (1 + r) of the parabola
+//     f(beta) = S2 - 2 beta (r A_j + B_j) + beta^2 (r^2 j + n - j),   A_j = P[j], B_j = S1 - A_j.
+// grid = (chunks of j, ratios); each CTA leaves its best (f, beta); the lowest j wins exact ties.
+struct ScanBest {
+    double f;
+    double beta;
+    long long j;
+};
+
+__device__ __forceinline__ bool better(const ScanBest& a, const ScanBest& b) {  // a before b
+    return a.f < b.f || (a.f == b.f && a.j < b.j);
+}
+
+__device__ __forceinline__ ScanBest warp_best(ScanBest v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        ScanBest y;
+        y.f = __shfl_xor_sync(0xffffffffu, v.f, o);
+        y.beta = __shfl_xor_sync(0xffffffffu, v.beta, o);
+        y.j = __shfl_xor_sync(0xffffffffu, v.j, o);
+        if (better(y, v)) v = y;
+    }
+    return v;
+}
+
+constexpr int kEvalPerThread = 8;
+constexpr int kEvalBlock = kDiagThreads * kEvalPerThread;
+
+__global__ void __launch_bounds__(kDiagThreads) ratio_eval_kernel(const uint32_t* __restrict__ keys, const double* __restrict__ P,
+                                                                  long long n, const double* __restrict__ totals,
+                                                                  const double* __restrict__ ratios, ScanBest* __restrict__ partial) {
+    __shared__ ScanBest sh[kDiagWarps];
+    const double r = ratios[blockIdx.y];
+    const double S1 = totals[0], S2 = totals[1];
+    const double to_beta = 2.0 / (1.0 + r);
+    ScanBest best;
+    best.f = S2;  // beta = 0 (everything reconstructed as zero) is the value to beat
+    best.beta = 0.0;
+    best.j = -1;
+    const long long j0 = static_cast<long long>(blockIdx.x) * kEvalBlock + threadIdx.x;
+#pragma unroll
+    for (int i = 0; i < kEvalPerThread; ++i) {
+        const long long j = j0 + static_cast<long long>(i) * kDiagThreads;
+        if (j <= n) {
+            const double A = j < n ? P[j] : S1;
+            const double lin = r * A + (S1 - A);
+            const double quad = r * r * static_cast<double>(j) + static_cast<double>(n - j);
+            const double lo = (j == 0 ? 0.0 : static_cast<double>(__uint_as_float(keys[j - 1]))) * to_beta;
+            double b = lin / quad;
+            if (b < lo) b = lo;
+            if (j < n) {
+                const double hi = static_cast<double>(__uint_as_float(keys[j])) * to_beta;
+                if (b > hi) b = hi;
+            }
+            ScanBest c;
+            c.f = S2 - 2.0 * b * lin + b * b * quad;
+            c.beta = b;
+            c.j = j;
+            if (better(c, best)) best = c;
+        }
+    }
+    best = warp_best(best);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) sh[warp] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 1; w < kDiagWarps; ++w)
+            if (better(sh[w], best)) best = sh[w];
+        partial[static_cast<size_t>(blockIdx.y) * gridDim.x + blockIdx.x] = best;
+    }
+}
+
+// One CTA per ratio: the best of its partial results; NMSE = f / S2 (0 for an all-zero input).
+__global__ void __launch_bounds__(kDiagThreads) ratio_final_kernel(const ScanBest* __restrict__ partial, int chunks,
+                                                                   const double* __restrict__ totals, double* __restrict__ beta,
+                                                                   double* __restrict__ nmse) {
+    __shared__ ScanBest sh[kDiagWarps];
+    ScanBest best;
+    best.f = totals[1];
+    best.beta = 0.0;
+    best.j = -1;
+    for (int c = threadIdx.x; c < chunks; c += kDiagThreads) {
+        const ScanBest p = partial[static_cast<size_t>(blockIdx.x) * chunks + c];
+        if (better(p, best)) best = p;
+    }
+    best = warp_best(best);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) sh[warp] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 1; w < kDiagWarps; ++w)
+            if (better(sh[w], best)) best = sh[w];
+        beta[blockIdx.x] = best.beta;
+        nmse[blockIdx.x] = totals[1] > 0.0 ? best.f / totals[1] : 0.0;
+    }
+}
+
+}  // namespace qift

@@ -7,6 +7,7 @@
 
 #include "common.cuh"
 #include "decode.cuh"
+#include "diag.cuh"
 #include "grouped.cuh"
 #include "kv4.cuh"
 #include "pack.cuh"
@@ -824,6 +825,140 @@ int qift_w2a4_linear_static(const uint32_t* packed, const float* s_n, int levels
     if (e != cudaSuccess) return cuda_status(e);
     return linear_impl(packed, s_n, levels, q_a, s_a, M, N, K, Y, y_dtype, acc_debug, scratch, kStaticScratchBytes,
                        QIFT_ROUTE_PREFILL_SCRATCH, stream);
+}
+
+// --------------------------------------------------------------------------------- diagnostics
+namespace {
+
+struct RatioScanLayout {
+    int seg, V, scan_blocks, chunks;
+    size_t P, keys_a, keys_b, hist, digit_totals, block_s1, block_s2, totals, ratios, partial, bytes;
+};
+
+bool ratio_scan_layout(long long n, int R, RatioScanLayout& l) {
+    if (n < 1 || n > (1ll << 28) || R < 1 || R > 65535) return false;
+    long long seg = (n + 4095) / 4096;
+    seg = (seg + 31) / 32 * 32;
+    if (seg < 1024) seg = 1024;
+    l.seg = static_cast<int>(seg);
+    l.V = static_cast<int>((n + seg - 1) / seg);
+    l.scan_blocks = static_cast<int>((n + kScanBlock - 1) / kScanBlock);
+    l.chunks = static_cast<int>((n + 1 + kEvalBlock - 1) / kEvalBlock);
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t at = off;
+        off += (bytes + 255) / 256 * 256;
+        return at;
+    };
+    l.P = take(sizeof(double) * n);
+    l.keys_a = take(sizeof(uint32_t) * n);
+    l.keys_b = take(sizeof(uint32_t) * n);
+    l.hist = take(sizeof(uint32_t) * 256 * l.V);
+    l.digit_totals = take(sizeof(uint32_t) * 256);
+    l.block_s1 = take(sizeof(double) * l.scan_blocks);
+    l.block_s2 = take(sizeof(double) * l.scan_blocks);
+    l.totals = take(sizeof(double) * 2);
+    l.ratios = take(sizeof(double) * R);
+    l.partial = take(sizeof(ScanBest) * static_cast<size_t>(R) * l.chunks);
+    l.bytes = off;
+    return true;
+}
+
+int stream_blocks(long long items) {
+    long long blocks = (items + kDiagThreads - 1) / kDiagThreads;
+    const long long cap = static_cast<long long>(sm_count()) * 8;
+    return static_cast<int>(blocks < cap ? (blocks < 1 ? 1 : blocks) : cap);
+}
+
+}  // namespace
+
+int qift_diag_grid_quantize(const float* W, int N, int K, const float* grid, int scale_mode, float* s_n, uint8_t* codes,
+                            void* stream) {
+    if (!W || !grid || !s_n || N <= 0 || K <= 0) return QIFT_ERR_INVALID_ARG;
+    if (scale_mode != QIFT_SCALE_GIVEN && scale_mode != QIFT_SCALE_ABSMAX && scale_mode != QIFT_SCALE_MSE) return QIFT_ERR_INVALID_ARG;
+    if (!(grid[0] < grid[1] && grid[1] < grid[2] && grid[2] < grid[3] && grid[3] > 0.0f)) return QIFT_ERR_INVALID_ARG;
+    if (K > 16384) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(W)) return QIFT_ERR_ALIGNMENT;
+    Grid4 G;
+    for (int i = 0; i < 4; ++i) G.g[i] = grid[i];
+    for (int i = 0; i < 3; ++i) G.m[i] = (grid[i] + grid[i + 1]) * 0.5f;
+    const size_t smem = sizeof(float) * K;
+    cudaError_t e = allow_smem(grid_quantize_kernel, smem);
+    if (e != cudaSuccess) return cuda_status(e);
+    grid_quantize_kernel<<<N, kDiagThreads, smem, static_cast<cudaStream_t>(stream)>>>(W, K, G, scale_mode, s_n, codes);
+    return cuda_status(cudaGetLastError());
+}
+
+int qift_diag_bucket_stats(const float* W, const uint8_t* codes, int N, int K, const float* s_n, const float* values, int L,
+                           unsigned long long* count, double* sqerr, void* stream) {
+    if (!W || !codes || !s_n || !values || !count || !sqerr || N <= 0 || K <= 0) return QIFT_ERR_INVALID_ARG;
+    if (L != 4 && L != 16) return QIFT_ERR_INVALID_ARG;
+    if (K % 4 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(W) || (reinterpret_cast<uintptr_t>(codes) & 3u) || (reinterpret_cast<uintptr_t>(count) & 7u) ||
+        (reinterpret_cast<uintptr_t>(sqerr) & 7u))
+        return QIFT_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(count, 0, sizeof(unsigned long long) * L, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(sqerr, 0, sizeof(double) * L, st);
+    if (e != cudaSuccess) return cuda_status(e);
+    BucketValues v = {};
+    for (int i = 0; i < L; ++i) v.v[i] = values[i];
+    const long long total4 = static_cast<long long>(N) * K / 4;
+    const int blocks = stream_blocks(total4);
+    if (L == 4)
+        bucket_stats_kernel<4><<<blocks, kDiagThreads, 0, st>>>(W, codes, total4, K, s_n, v, count, sqerr);
+    else
+        bucket_stats_kernel<16><<<blocks, kDiagThreads, 0, st>>>(W, codes, total4, K, s_n, v, count, sqerr);
+    return cuda_status(cudaGetLastError());
+}
+
+size_t qift_diag_ratio_scan_workspace_bytes(long long n, int R) {
+    RatioScanLayout l;
+    return ratio_scan_layout(n, R, l) ? l.bytes : 0;
+}
+
+int qift_diag_ratio_scan(const float* x, long long n, const double* ratios, int R, double* beta, double* nmse, void* workspace,
+                         size_t workspace_bytes, void* stream) {
+    if (!x || !ratios || !beta || !nmse || n <= 0 || R <= 0) return QIFT_ERR_INVALID_ARG;
+    for (int i = 0; i < R && i < 65536; ++i)
+        if (!(ratios[i] > 0.0 && ratios[i] <= 1.0)) return QIFT_ERR_INVALID_ARG;
+    RatioScanLayout l;
+    if (!ratio_scan_layout(n, R, l)) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!workspace || workspace_bytes < l.bytes) return QIFT_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return QIFT_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    double* P = reinterpret_cast<double*>(ws + l.P);
+    uint32_t* keys_a = reinterpret_cast<uint32_t*>(ws + l.keys_a);
+    uint32_t* keys_b = reinterpret_cast<uint32_t*>(ws + l.keys_b);
+    uint32_t* hist = reinterpret_cast<uint32_t*>(ws + l.hist);
+    uint32_t* digit_totals = reinterpret_cast<uint32_t*>(ws + l.digit_totals);
+    double* block_s1 = reinterpret_cast<double*>(ws + l.block_s1);
+    double* block_s2 = reinterpret_cast<double*>(ws + l.block_s2);
+    double* totals = reinterpret_cast<double*>(ws + l.totals);
+    double* d_ratios = reinterpret_cast<double*>(ws + l.ratios);
+    ScanBest* partial = reinterpret_cast<ScanBest*>(ws + l.partial);
+
+    cudaError_t e = cudaMemcpyAsync(d_ratios, ratios, sizeof(double) * R, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_status(e);
+    abs_keys_kernel<<<stream_blocks(n), kDiagThreads, 0, st>>>(x, n, keys_a);
+    const int seg_blocks = (l.V + kDiagWarps - 1) / kDiagWarps;
+    uint32_t* in = keys_a;
+    uint32_t* out = keys_b;
+    for (int shift = 0; shift < 32; shift += 8) {  // four stable passes: the sorted keys end in keys_a
+        radix_hist_kernel<<<seg_blocks, kDiagThreads, 0, st>>>(in, n, l.seg, l.V, shift, hist);
+        radix_rowscan_kernel<<<256, 1024, 0, st>>>(hist, l.V, digit_totals);
+        radix_scatter_kernel<<<seg_blocks, kDiagThreads, 0, st>>>(in, n, l.seg, l.V, shift, hist, digit_totals, out);
+        uint32_t* t = in;
+        in = out;
+        out = t;
+    }
+    scan_block_sums_kernel<<<l.scan_blocks, kDiagThreads, 0, st>>>(keys_a, n, block_s1, block_s2);
+    scan_bases_kernel<<<1, kDiagThreads, 0, st>>>(block_s1, block_s2, l.scan_blocks, totals);
+    scan_write_kernel<<<l.scan_blocks, kDiagThreads, 0, st>>>(keys_a, n, block_s1, P);
+    ratio_eval_kernel<<<dim3(l.chunks, R), kDiagThreads, 0, st>>>(keys_a, P, n, totals, d_ratios, partial);
+    ratio_final_kernel<<<R, kDiagThreads, 0, st>>>(partial, l.chunks, totals, beta, nmse);
+    return cuda_status(cudaGetLastError());
 }
 
 int qift_device_status(void* stream, uint32_t* detail) {

@@ -388,6 +388,7 @@ def run_gpu(args):
         out["mixed_stack"] = run_mixed_stack(torch, qift, L, device, gen, args)
         out["prefill"] = run_prefill(torch, qift, L, device, gen, pk)
         out["kv4"] = run_kv4(torch, qift, L, pk)
+        out["diagnostics"] = run_diagnostics(torch, qift, pk)
     if rank == 0 and world == 1 and not args.no_cpu:
         out["cpu_baseline"] = cpu_baseline(budget_s=12.0)
     if rank == 0:
@@ -493,6 +494,44 @@ def run_kv4(torch, qift, L, pk):
                                  "registers keeps it instruction-bound above its memory time"},
             "quantizer": {"workload": "8192 tokens x 8 heads x 128, bf16 in, Hadamard over the head dimension", "us": round(msq * 1e3, 2),
                           "value": round(qbytes / (msq * 1e-3) / 1e9, 1), "unit": "GB/s"}}
+
+
+def run_diagnostics(torch, qift, pk):
+    """Quantizer diagnostics (Sec. 4.5): bucket statistics of one LLaMA-2 gate matrix (11008 x 4096 synthetic rotated
+    weights, 225 MB of weights + codes), the float-grid quantizer with its 80-candidate sweep on the same matrix, and the
+    ratio scan at the paper's size (100 000 pooled samples, the 0.005 grid of 199 ratios)."""
+    N, K = 11008, 4096
+    W = torch.randn(N, K, device="cuda") * 0.02
+    lloyd = [-1.5104, -0.4528, 0.4528, 1.5104]
+    s, codes = qift.qift_diag_grid_quantize(W, lloyd, qift.SCALE_MSE)
+
+    def timed(fn, n):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    ms_q = timed(lambda: qift.qift_diag_grid_quantize(W, lloyd, qift.SCALE_MSE, s_n=s), 3)
+    ms_b = timed(lambda: qift.qift_diag_bucket_stats(W, codes, s, lloyd), 10)
+    n, ratios = 100_000, [0.005 * i for i in range(1, 200)]
+    x = torch.randn(n, device="cuda")
+    ws = torch.empty(qift.qift_diag_ratio_scan_workspace_bytes(n, len(ratios)), dtype=torch.uint8, device="cuda")
+    ms_r = timed(lambda: qift.qift_diag_ratio_scan(x, ratios, workspace=ws), 10)
+    _, nmse = qift.qift_diag_ratio_scan(x, ratios, workspace=ws)
+    gbs = N * K * 5 / (ms_b * 1e-3) / 1e9
+    return {"workload": "Sec. 4.5 diagnostics on synthetic Gaussian weights",
+            "bucket_stats": {"shape": [N, K], "us": round(ms_b * 1e3, 1), "value": round(gbs, 1), "unit": "GB/s",
+                             "frac_of_hbm_peak": round(gbs / pk["hbm_gbs"], 3)},
+            "grid_quantize_mse_sweep": {"shape": [N, K], "grid": "Lloyd-Max", "us": round(ms_q * 1e3, 1),
+                                        "candidate_evaluations_per_s": round(N * K * 80 / (ms_q * 1e-3), 0)},
+            "ratio_scan": {"samples": n, "ratios": len(ratios), "us": round(ms_r * 1e3, 1),
+                           "best_ratio": round(ratios[int(nmse.argmin())], 3), "best_nmse": round(float(nmse.min()), 6)}}
 
 
 def int8_library_point(torch, M, shapes, device):

@@ -124,10 +124,13 @@ __global__ void __launch_bounds__(kDiagThreads) bucket_stats_kernel(const float*
     __shared__ double e_sh[kDiagWarps][L];
     __shared__ unsigned long long n_sh[kDiagWarps][L];
     const long long stride = static_cast<long long>(gridDim.x) * kDiagThreads;
+    const uint32_t K4 = static_cast<uint32_t>(K) / 4u;  // vectors per row
+    const bool narrow = total4 <= 0xffffffffll;           // a 32-bit division finds the row
     for (long long v = static_cast<long long>(blockIdx.x) * kDiagThreads + threadIdx.x; v < total4; v += stride) {
         const float4 w4 = reinterpret_cast<const float4*>(W)[v];
         const uint32_t c4 = reinterpret_cast<const uint32_t*>(codes)[v];
-        const double s = static_cast<double>(s_n[(v * 4) / K]);
+        const long long r = narrow ? static_cast<long long>(static_cast<uint32_t>(v) / K4) : v / K4;
+        const double s = static_cast<double>(s_n[r]);
         const float w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {

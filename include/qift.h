@@ -183,7 +183,9 @@ int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_blo
  *                             needs the q_a, s_a and token sums that qift_group_quantize_act left
  *                             in the problems' buffers and in plan_dev
  *   qift_group_forward      : both.
- * Problems must not alias each other's q_a / s_a / Y.  K % 256 == 0 (two-bit sets) or K % 128 == 0
+ * Problems must not alias each other's Y, nor each other's q_a / s_a with one exception: modules that
+ * read the SAME activation (q/k/v; gate/up) may name the same X, q_a, s_a (same K and had_block); the
+ * plan then quantizes that activation once and every such product reads it.  K % 256 == 0 (two-bit sets) or K % 128 == 0
  * (INT4), K <= 16384. */
 typedef struct qift_group_problem {
     const void* X;          /* dev [M,K] fp32 or bf16                         */

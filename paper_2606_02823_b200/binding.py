@@ -291,9 +291,10 @@ def _align(n, a=256):
 
 
 def qift_group_plan(problems, levels: int, clip_ratio: float = 0.9, out_dtype=torch.float32, want_acc: bool = False,
-                    arenas: bool = False):
+                    arenas: bool = False, share: bool = True):
     """problems: list of (X [M,K], packed, s_n, had_block) sharing M and the dtype of X.  Allocates
-    q_a / s_a / Y (and the accumulators when asked) and returns a GroupPlan.  With arenas=True the
+    q_a / s_a / Y (and the accumulators when asked) and returns a GroupPlan.  Problems that name the same X tensor
+    (and rotation) get the same q_a / s_a, which the library then quantizes once (share=False: one each).  With arenas=True the
     activations are copied into one contiguous device arena and the outputs live in another, each
     with a pinned host mirror (plan.x_host / plan.y_host), for qift_group_forward_host."""
     assert problems
@@ -302,6 +303,7 @@ def qift_group_plan(problems, levels: int, clip_ratio: float = 0.9, out_dtype=to
     device = problems[0][0].device
     arr = (GroupProblem * len(problems))()
     keep, ins, outs, accs = [], [], [], []
+    shared = {}
     x_arena = y_arena = None
     if arenas:
         xe = problems[0][0].element_size()
@@ -324,8 +326,13 @@ def qift_group_plan(problems, levels: int, clip_ratio: float = 0.9, out_dtype=to
             Y = y_arena[y_off[i]:y_off[i] + M * N * ye].view(out_dtype).view(M, N)
         else:
             Y = torch.empty((M, N), dtype=out_dtype, device=device)
-        q_a = torch.empty((M, K), dtype=torch.int8, device=device)
-        s_a = torch.empty((max(M, 4),), dtype=torch.float32, device=device)
+        key = (X.data_ptr(), K, had_block)
+        if share and not arenas and key in shared:      # modules reading one activation share its quantization
+            q_a, s_a = shared[key]
+        else:
+            q_a = torch.empty((M, K), dtype=torch.int8, device=device)
+            s_a = torch.empty((max(M, 4),), dtype=torch.float32, device=device)
+            shared[key] = (q_a, s_a)
         acc = torch.empty((M, N), dtype=torch.int32, device=device) if want_acc else None
         arr[i] = GroupProblem(X.data_ptr(), packed.data_ptr(), s_n.data_ptr(), q_a.data_ptr(), s_a.data_ptr(), Y.data_ptr(),
                               acc.data_ptr() if want_acc else None, N, K, had_block, 0)

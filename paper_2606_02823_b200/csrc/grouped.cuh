@@ -42,7 +42,9 @@ struct GroupProblemDev {
     int N, K, had_block;
     int item_begin;         // first work item of this problem
     float inv_sqrt_b;
-    int pad[5];
+    int quant_src;          // problem whose quantized activation (q_a, s_a, sum of q) this one uses: itself, or an earlier one
+                            // with the same X, q_a, s_a, K and rotation (q/k/v, gate/up: one quantization for all)
+    int pad[4];
 };
 static_assert(sizeof(GroupProblemDev) == 96, "problem record is 96 bytes");
 
@@ -65,6 +67,7 @@ quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* _
     pdl_wait();
     const int p = blockIdx.x / M;
     const GroupProblemDev P = problems[p];
+    if (P.quant_src != p) return;  // an earlier problem quantizes this activation
     const size_t m = blockIdx.x % M;
     const int K = P.K, B = P.had_block;
     const RowScale sc = block_row_scale(load_and_transform<BF16_IN, KRON>(P.X, m, K, B, row), clip, red);
@@ -94,7 +97,7 @@ struct SmemProblem {  // what the product kernel needs of a problem, 64 bytes, i
     int32_t* acc_debug;
     int N, K;
     int item_begin;
-    int index;  // position in the whole plan (row of the sum-q table)
+    int index;  // row of the sum-q table: the plan position of the problem that quantized the activation
 };
 static_assert(sizeof(SmemProblem) == 64, "shared-memory problem record is 64 bytes");
 
@@ -208,7 +211,7 @@ linear_grouped_kernel(const GroupParams gp) {
         SmemProblem e;
         e.packed = reinterpret_cast<const unsigned char*>(P.packed);
         e.q_a = P.q_a, e.s_n = P.s_n, e.s_a = P.s_a, e.Y = P.Y, e.acc_debug = P.acc_debug;
-        e.N = P.N, e.K = P.K, e.item_begin = P.item_begin, e.index = gp.first_index + i;
+        e.N = P.N, e.K = P.K, e.item_begin = P.item_begin, e.index = P.quant_src;
         table[i] = e;
     }
     __syncthreads();
@@ -429,7 +432,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
         SmemProblem e;
         e.packed = reinterpret_cast<const unsigned char*>(P.packed);
         e.q_a = P.q_a, e.s_n = P.s_n, e.s_a = P.s_a, e.Y = P.Y, e.acc_debug = P.acc_debug;
-        e.N = P.N, e.K = P.K, e.item_begin = P.item_begin, e.index = gp.first_index + i;
+        e.N = P.N, e.K = P.K, e.item_begin = P.item_begin, e.index = P.quant_src;
         table[i] = e;
     }
     __syncthreads();

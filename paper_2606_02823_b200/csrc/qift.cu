@@ -636,7 +636,13 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
         o.N = q.N, o.K = q.K, o.had_block = q.had_block;
         o.item_begin = items;
         o.inv_sqrt_b = q.had_block > 1 ? inv_sqrt_block(q.had_block) : 1.0f;
-        for (int j = 0; j < 5; ++j) o.pad[j] = 0;
+        o.quant_src = i;
+        for (int j = 0; j < i; ++j)
+            if (d[j].X == q.X && d[j].q_a == q.q_a && d[j].s_a == q.s_a && d[j].K == q.K && d[j].had_block == q.had_block) {
+                o.quant_src = d[j].quant_src;
+                break;
+            }
+        for (int j = 0; j < 4; ++j) o.pad[j] = 0;
         items += (q.N + rows_per_item - 1) / rows_per_item;
         if (q.K > max_k) max_k = q.K;
         if (q.had_block > 1 && !is_pow2(q.had_block)) any_kron = 1;

@@ -337,6 +337,41 @@ def test_grouped_forward(name, M):
     check_outputs(plan.outputs[2], plan.accs[2], refs[2][2], refs[2][3], False)
 
 
+@pytest.mark.parametrize("M", [1, 7])
+def test_grouped_shared_activation(M):
+    # q/k/v-style and gate/up-style modules read one activation: the plan quantizes it once (the buffers of the
+    # sharing problems are the same) and every product still matches the oracle
+    lv = oracle.MNZ
+    K = 1024
+    x1, _ = synth.activations(700, M, K, 8)
+    x2, _ = synth.activations(701, M, K, 8)
+    X1, X2 = dev(x1), dev(x2)
+    probs, refs = [], []
+    for i, (X, x, N) in enumerate([(X1, x1, 256), (X1, x1, 64), (X2, x2, 512), (X1, x1, 96), (X2, x2, 48)]):
+        W = synth.gaussian_weights(710 + i, N, K)
+        p_ref, s_n, codes = oracle.pack_weights(W, lv, oracle.SCALE_ABSMAX)
+        q_ref, sa_ref = oracle.quantize_act(x, 256, 0.9)
+        refs.append(oracle.linear(codes, lv, s_n, q_ref, sa_ref))
+        probs.append((X, dev(p_ref.view(np.int32)), dev(s_n), 256))
+    for share in (True, False):
+        plan = qift.qift_group_plan(probs, lv, 0.9, want_acc=True, share=share)
+        q_ptrs = {plan.keep[5 * i + 3].data_ptr() for i in range(5)}
+        assert len(q_ptrs) == (2 if share else 5)
+        outs = qift.qift_group_forward(plan)
+        assert_status_clean()
+        for (y_ref, acc_ref), y, acc in zip(refs, outs, plan.accs):
+            check_outputs(y, acc, y_ref, acc_ref, False)
+    # same X with a different rotation does not share
+    plan = qift.qift_group_plan([probs[0], (X1, probs[1][1], probs[1][2], 128)], lv, 0.9, want_acc=True)
+    assert plan.keep[3].data_ptr() != plan.keep[8].data_ptr()
+    qift.qift_group_forward(plan)
+    q128, sa128 = oracle.quantize_act(x1, 128, 0.9)
+    W = synth.gaussian_weights(711, 64, K)
+    _, s_n, codes = oracle.pack_weights(W, lv, oracle.SCALE_ABSMAX)
+    y_ref, acc_ref = oracle.linear(codes, lv, s_n, q128, sa128)
+    check_outputs(plan.outputs[1], plan.accs[1], y_ref, acc_ref, False)
+
+
 def test_grouped_rejects_bad_plans():
     x = torch.zeros((1, 256), device="cuda")
     packed = torch.zeros((16, 16), dtype=torch.int32, device="cuda")

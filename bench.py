@@ -398,40 +398,48 @@ def run_gpu(args):
 
 
 def run_mixed_stack(torch, qift, L, device, gen, args):
-    """Config 5: layer-wise mixed precision on LLaMA-2-7B shapes at M = 1: layers 0..15 INT4 weights (W4A4),
-    layers 16..31 MNZ (W2A4), 3 bits per weight on average.  Two grouped plans (a plan holds one level set):
-    four launches per token-step.  Modules run on their own staged inputs, as in the headline."""
-    n4 = max(1, args.layers // 2)
-    n2 = max(1, args.layers - n4)
+    """Config 5: layer-wise mixed precision on LLaMA-2-7B shapes at M = 1: the first L layers INT4 weights (W4A4), the
+    rest MNZ (W2A4), b_avg = 2 + L/16 bits per weight for 32 layers (Sec. 3.7).  Config 5 itself is L = 16 (3 bits on
+    average); the sweep adds L = 4, 8, 12.  Two grouped plans (a plan holds one level set): four launches per
+    token-step.  Modules run on their own staged inputs, as in the headline."""
     vp = ctypes.c_void_p
-    plans, algo = [], 0
-    for lv, n in ((qift.INT4, n4), (qift.MNZ, n2)):
-        mods = build_stack(torch, qift, synth.LLAMA2_7B, n, 1, lambda l, lv=lv: lv, 5000 + lv, torch.float32, torch.float32,
-                           device, gen)
-        plans.append((qift.qift_group_plan([(m.x, m.packed, m.s_n, m.B) for m in mods], lv, CLIP), mods))
-        algo += sum(product_bytes(1, m.N, m.K, m.bits) + quant_bytes(1, m.K) for m in mods)
     st = vp(torch.cuda.current_stream().cuda_stream)
 
-    def step():
-        for plan, _ in plans:
-            rc = L.qift_group_forward(vp(plan.host.data_ptr()), vp(plan.dev.data_ptr()), st)
-            assert rc == 0, rc
+    def point(n4, n2):
+        plans, algo = [], 0
+        for lv, n in ((qift.INT4, n4), (qift.MNZ, n2)):
+            mods = build_stack(torch, qift, synth.LLAMA2_7B, n, 1, lambda l, lv=lv: lv, 5000 + lv, torch.float32, torch.float32,
+                               device, gen)
+            plans.append((qift.qift_group_plan([(m.x, m.packed, m.s_n, m.B) for m in mods], lv, CLIP), mods))
+            algo += sum(product_bytes(1, m.N, m.K, m.bits) + quant_bytes(1, m.K) for m in mods)
 
-    for _ in range(5):
-        step()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    steps = max(3, min(args.steps, 100))
-    e0.record()
-    for _ in range(steps):
-        step()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / steps
-    return {"workload": f"config 5: {n4} W4A4 layers + {n2} W2A4 (MNZ) layers, LLaMA-2-7B shapes, M=1, grouped API (4 launches per step)",
-            "ms_per_step": round(ms, 5), "tokens_per_s": round(1.0 / (ms * 1e-3), 1),
-            "value": round(algo / (ms * 1e-3) / 1e9, 2), "unit": "GB/s", "algorithmic_bytes_per_step": algo,
-            "pct_of_8TBs": round(100 * algo / (ms * 1e-3) / 8e12, 2)}
+        def step():
+            for plan, _ in plans:
+                rc = L.qift_group_forward(vp(plan.host.data_ptr()), vp(plan.dev.data_ptr()), st)
+                assert rc == 0, rc
+
+        for _ in range(5):
+            step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        steps = max(3, min(args.steps, 100))
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        return {"w4_layers": n4, "w2_layers": n2, "bits_per_weight": round(2 + 2 * n4 / (n4 + n2), 3), "ms_per_step": round(ms, 5),
+                "tokens_per_s": round(1.0 / (ms * 1e-3), 1), "value": round(algo / (ms * 1e-3) / 1e9, 2), "unit": "GB/s",
+                "algorithmic_bytes_per_step": algo, "pct_of_8TBs": round(100 * algo / (ms * 1e-3) / 8e12, 2)}
+
+    n4 = max(1, args.layers // 2)
+    out = point(n4, max(1, args.layers - n4))
+    out["workload"] = (f"config 5: {out['w4_layers']} W4A4 layers + {out['w2_layers']} W2A4 (MNZ) layers, LLaMA-2-7B shapes, M=1, "
+                       "grouped API (4 launches per step)")
+    if args.layers >= 16:
+        out["l_sweep"] = [point(args.layers * l // 32, args.layers - args.layers * l // 32) for l in (4, 8, 12)]
+    return out
 
 
 def run_kv4(torch, qift, L, pk):

@@ -483,6 +483,14 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     // -------------------------------------------------------------------- consumer warps
     pdl_wait();
     const int g = lane >> 2, cq = lane & 3;
+    // per-lane byte offsets inside a stage, fixed for the whole kernel
+    const int rot = (T::PER == 16) ? (cq & 2) : 0;
+    int q_off[NT], piece_off[T::NPL];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) q_off[nt] = min(nt * 8 + g, M - 1) * QSTRIDE + 4 * cq * T::PER;
+#pragma unroll
+    for (int i = 0; i < T::NPL; ++i) piece_off[i] = ((i + rot * T::NPL / 4) % T::NPL) * 16;
+    const int w_off = lane * 16 + 4 * rot, w_hi = 8 - 8 * rot;  // second pair of words: +8, or -8 after the rotation
     Cursor cur;
     cur.init(table, gp.count, gp.item_first, gp.item_end, kWideRows);
     bool ok = true;
@@ -515,31 +523,32 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                 // not depend on the order) -- with a token stride of 16 bytes mod 128 every quarter-warp then
                 // covers all eight 16-byte bank groups.
                 // (INT4 weights: 32 bytes per lane, already conflict-free without the rotation.)
-                const int rot = (T::PER == 16) ? (cq & 2) : 0;
-                for (int sl = 0; 16 * sl < cw; ++sl) {   // 16-word slices of the chunk
+                // Token columns beyond M read the last token's bytes instead of zeros: a column of the
+                // product depends on its own activations only, and those columns are never written.
+                auto slice = [&](int sl) {
                     uint32_t qb[NT][4 * T::NPL];
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
-                        const int m = nt * 8 + g;
-                        if (m < M) {
-                            const unsigned char* src = qst + m * QSTRIDE + (16 * sl + 4 * cq) * T::PER;
+                        const unsigned char* src = qst + q_off[nt] + sl * (16 * T::PER);
 #pragma unroll
-                            for (int i = 0; i < T::NPL; ++i) {
-                                // NPL 16-byte pieces hold the lane's four words in order; piece i holds word 4i/NPL
-                                const uint4 v = *reinterpret_cast<const uint4*>(src + ((i + rot * T::NPL / 4) % T::NPL) * 16);
-                                qb[nt][4 * i] = v.x, qb[nt][4 * i + 1] = v.y, qb[nt][4 * i + 2] = v.z, qb[nt][4 * i + 3] = v.w;
-                            }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 4 * T::NPL; ++i) qb[nt][i] = 0;
+                        for (int i = 0; i < T::NPL; ++i) {
+                            // NPL 16-byte pieces hold the lane's four words in order; piece i holds word 4i/NPL
+                            const uint4 v = *reinterpret_cast<const uint4*>(src + piece_off[i]);
+                            qb[nt][4 * i] = v.x, qb[nt][4 * i + 1] = v.y, qb[nt][4 * i + 2] = v.z, qb[nt][4 * i + 3] = v.w;
                         }
                     }
-                    const unsigned char* wsrc = wst + (2 * sl * 32 + lane) * 16;
-                    const uint2 a_lo = *reinterpret_cast<const uint2*>(wsrc + 4 * rot), a_hi = *reinterpret_cast<const uint2*>(wsrc + 8 - 4 * rot);
-                    const uint2 b_lo = *reinterpret_cast<const uint2*>(wsrc + 512 + 4 * rot), b_hi = *reinterpret_cast<const uint2*>(wsrc + 520 - 4 * rot);
+                    const unsigned char* wsrc = wst + w_off + sl * 1024;
+                    const uint2 a_lo = *reinterpret_cast<const uint2*>(wsrc), a_hi = *reinterpret_cast<const uint2*>(wsrc + w_hi);
+                    const uint2 b_lo = *reinterpret_cast<const uint2*>(wsrc + 512), b_hi = *reinterpret_cast<const uint2*>(wsrc + 512 + w_hi);
                     const uint4 wa = make_uint4(a_lo.x, a_lo.y, a_hi.x, a_hi.y);
                     const uint4 wb = make_uint4(b_lo.x, b_lo.y, b_hi.x, b_hi.y);
                     mma_tile_step<LV, NT, true>(acc, wa, wb, qb);
+                };
+                if (cw == kWideChunkWords) {
+#pragma unroll
+                    for (int sl = 0; sl < kWideChunkWords / 16; ++sl) slice(sl);
+                } else {
+                    for (int sl = 0; 16 * sl < cw; ++sl) slice(sl);   // 16-word slices of a short last chunk
                 }
             }
             __syncwarp();

@@ -388,27 +388,36 @@ linear_grouped_kernel(const GroupParams gp) {
 // loop, accumulates all 16 tokens in registers and writes its outputs itself -- no reduction, no CTA
 // barrier.  The price is that every warp reads the whole activation slice of a stage, so stages are
 // half tiles (64 words per row: 32 KB of weights + 17 KB of activations at 16 tokens), four deep.
-constexpr int kWideChunkWords = 64;
 constexpr int kWideQPad = 16;                    // token stride = 16 bytes mod 128: see the consumer's loads
-constexpr int kWideTiles = kDecWarps;            // row tiles per item, one per consumer warp
-constexpr int kWideRows = 16 * kWideTiles;       // 128
+constexpr int kWideRows = 16 * kDecWarps;        // 128 rows per item with one tile per warp
 
-__host__ __device__ inline size_t wide_stage_bytes(int lv, int M) {
-    return static_cast<size_t>(kWideTiles) * (kTileBytes / 2) + static_cast<size_t>(M) * (kWideChunkWords * codes_per_word(lv) + kWideQPad);
+// CWARPS consumer warps with RT row tiles each: an item is 16 * CWARPS * RT rows.  256-row items come either as
+// sixteen warps (twice the warps to hide the latencies of the load -> logic -> product chains) or as two tiles per
+// warp (the activation registers of a slice feed both tiles); their stages are a quarter tile of K (32 words) so
+// that as many stages fit as with 128 rows.
+__host__ __device__ constexpr int wide_chunk_words(int tiles) { return tiles > 8 ? 32 : 64; }
+
+__host__ __device__ inline size_t wide_stage_bytes(int lv, int M, int tiles) {
+    const int cw = wide_chunk_words(tiles);
+    return static_cast<size_t>(tiles) * (cw * 64) + static_cast<size_t>(M) * (cw * codes_per_word(lv) + kWideQPad);
 }
-__host__ __device__ inline size_t wide_smem_bytes(int lv, int M, int stages, int count) {
-    return static_cast<size_t>(count) * sizeof(SmemProblem) + stages * (wide_stage_bytes(lv, M) + 16) + 16;
+__host__ __device__ inline size_t wide_smem_bytes(int lv, int M, int tiles, int stages, int count) {
+    return static_cast<size_t>(count) * sizeof(SmemProblem) + stages * (wide_stage_bytes(lv, M, tiles) + 16) + 16;
 }
 
-template <int LV, int NT>
-__global__ void __launch_bounds__(kDecThreads, 1)
+template <int LV, int NT, int RT, int CWARPS>
+__global__ void __launch_bounds__((CWARPS + 1) * 32, 1)
 linear_grouped_wide_kernel(const GroupParams gp) {
     using T = DecodeTraits<LV>;
-    constexpr int QSTRIDE = kWideChunkWords * T::PER + kWideQPad;
-    using Cursor = GroupCursor<T::PER, kWideChunkWords>;
+    constexpr int TILES = CWARPS * RT;           // row tiles per item
+    constexpr int CW = wide_chunk_words(TILES);
+    constexpr int THREADS = (CWARPS + 1) * 32;
+    constexpr int TILE_STAGE = CW * 64;          // bytes of one tile in a stage: CW words x 16 rows, contiguous in the packed order
+    constexpr int QSTRIDE = CW * T::PER + kWideQPad;
+    using Cursor = GroupCursor<T::PER, CW>;
     extern __shared__ __align__(128) unsigned char smem[];
     const int M = gp.M;
-    const uint32_t stage_bytes = static_cast<uint32_t>(wide_stage_bytes(LV, M));
+    const uint32_t stage_bytes = static_cast<uint32_t>(wide_stage_bytes(LV, M, TILES));
     const int stages = gp.stages;
     unsigned char* ring = smem;
     SmemProblem* table = reinterpret_cast<SmemProblem*>(smem + stages * stage_bytes);
@@ -422,12 +431,12 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(&full[s], 1);
-            mbar_init(&empty[s], kDecWarps);
+            mbar_init(&empty[s], CWARPS);
         }
         mbar_fence_init();
         *fail = 0;
     }
-    for (int i = tid; i < gp.count; i += kDecThreads) {
+    for (int i = tid; i < gp.count; i += THREADS) {
         const GroupProblemDev& P = gp.problems[i];
         SmemProblem e;
         e.packed = reinterpret_cast<const unsigned char*>(P.packed);
@@ -437,7 +446,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     }
     __syncthreads();
 
-    if (warp == kDecWarps) {
+    if (warp == CWARPS) {
         // ---------------------------------------------------------------- producer warp
         auto expect = [&](const Cursor& c, int s) {
             if (lane == 0) mbar_expect_tx(&full[s], c.chunk_words() * (64 * c.tiles_valid + T::PER * M));
@@ -447,18 +456,16 @@ linear_grouped_wide_kernel(const GroupParams gp) {
             const uint32_t bytes = c.chunk_words() * 16 * 4;
             unsigned char* dst = ring + s * stage_bytes;
             if (lane < c.tiles_valid)
-                bulk_g2s(dst + lane * (kTileBytes / 2), c.wbase + lane * c.rb_bytes + static_cast<size_t>(c.chunk) * (kTileBytes / 2),
-                         bytes, &full[s]);
+                bulk_g2s(dst + lane * TILE_STAGE, c.wbase + lane * c.rb_bytes + static_cast<size_t>(c.chunk) * TILE_STAGE, bytes, &full[s]);
         };
         auto issue_q = [&](const Cursor& c, int s) {
             const uint32_t seg = c.chunk_words() * T::PER;
-            unsigned char* dst = ring + s * stage_bytes + kWideTiles * (kTileBytes / 2);
+            unsigned char* dst = ring + s * stage_bytes + TILES * TILE_STAGE;
             for (int m = lane; m < M; m += 32)
-                bulk_g2s(dst + m * QSTRIDE, c.q_a + static_cast<size_t>(m) * c.K + static_cast<size_t>(c.chunk) * (kWideChunkWords * T::PER),
-                         seg, &full[s]);
+                bulk_g2s(dst + m * QSTRIDE, c.q_a + static_cast<size_t>(m) * c.K + static_cast<size_t>(c.chunk) * (CW * T::PER), seg, &full[s]);
         };
         Cursor a;
-        a.init(table, gp.count, gp.item_first, gp.item_end, kWideRows);
+        a.init(table, gp.count, gp.item_first, gp.item_end, 16 * TILES);
         int pre = 0;
         for (; pre < stages && a.valid(); ++pre, a.next()) {  // weights do not depend on the previous kernel
             expect(a, pre);
@@ -466,7 +473,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
         }
         pdl_wait();
         Cursor b;
-        b.init(table, gp.count, gp.item_first, gp.item_end, kWideRows);
+        b.init(table, gp.count, gp.item_first, gp.item_end, 16 * TILES);
         for (int i = 0; i < pre; ++i, b.next()) issue_q(b, i);
         int s = 0;
         uint32_t ph = 0;
@@ -485,28 +492,56 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     const int g = lane >> 2, cq = lane & 3;
     // per-lane byte offsets inside a stage, fixed for the whole kernel
     const int rot = (T::PER == 16) ? (cq & 2) : 0;
-    int q_off[NT], piece_off[T::NPL];
+    // Activation pieces: NPL 16-byte pieces per token hold the lane's four words in order; a lane visits them
+    // starting at piece `rot` (order 2,3,0,1 for cq >= 2).  Two byte offsets per token tile cover that with constant
+    // displacements: the first half of the visit starts at q_lo, the second at q_hi.
+    uint32_t q_lo[NT], q_hi[NT];
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) q_off[nt] = min(nt * 8 + g, M - 1) * QSTRIDE + 4 * cq * T::PER;
-#pragma unroll
-    for (int i = 0; i < T::NPL; ++i) piece_off[i] = ((i + rot * T::NPL / 4) % T::NPL) * 16;
-    const int w_off = lane * 16 + 4 * rot, w_hi = 8 - 8 * rot;  // second pair of words: +8, or -8 after the rotation
+    for (int nt = 0; nt < NT; ++nt) {
+        const uint32_t tok = static_cast<uint32_t>(min(nt * 8 + g, M - 1) * QSTRIDE + 4 * cq * T::PER);
+        q_lo[nt] = tok + rot * (T::NPL * 4);                                   // pieces rot .. rot + NPL/2 - 1
+        q_hi[nt] = tok + ((rot ? 0 : T::NPL / 2) * 16);                        // the other half
+    }
+    const uint32_t w_lo = lane * 16 + 4 * rot, w_hi = w_lo + 8 - 8 * rot;      // the two word pairs of a lane's four words
+    const uint32_t ring_addr = smem_u32(ring);
     Cursor cur;
-    cur.init(table, gp.count, gp.item_first, gp.item_end, kWideRows);
+    cur.init(table, gp.count, gp.item_first, gp.item_end, 16 * TILES);
     bool ok = true;
     int s = 0;
     uint32_t ph = 0;
     while (cur.valid() && ok) {
-        int acc[NT][T::NACC][4];
+        int acc[RT][NT][T::NACC][4];
 #pragma unroll
-        for (int b = 0; b < NT; ++b)
+        for (int r = 0; r < RT; ++r)
 #pragma unroll
-            for (int t = 0; t < T::NACC; ++t)
+            for (int b = 0; b < NT; ++b)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[b][t][i] = 0;
+                for (int t = 0; t < T::NACC; ++t)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[r][b][t][i] = 0;
         const SmemProblem* P = &table[cur.p];
-        const int row0 = cur.n0 + 16 * warp;          // this warp's tile
-        const bool tile_on = warp < cur.tiles_valid;
+        const int cur_n0 = cur.n0;
+        const int tile0 = warp * RT;                       // this warp's tiles: tile0 .. tile0 + RT - 1
+        const int tiles_on = min(RT, cur.tiles_valid - tile0);   // <= 0: nothing to do in this item
+        // what the epilogue needs besides the accumulators, fetched now so that the latency of these loads is
+        // hidden behind the K loop instead of standing between two items
+        int e_sq[NT][2];
+        float e_sa[NT][2], e_sn[RT][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int tok = min(nt * 8 + 2 * cq + j, M - 1);
+                e_sq[nt][j] = gp.sumq[P->index * 16 + tok];
+                e_sa[nt][j] = P->s_a[tok];
+            }
+#pragma unroll
+        for (int r = 0; r < RT; ++r)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int n = cur_n0 + 16 * (tile0 + r) + g + 8 * j;
+                e_sn[r][j] = (n < P->N) ? __ldg(P->s_n + n) : 0.0f;
+            }
 
         for (;;) {
             if (!mbar_wait(&full[s], ph, 6)) {
@@ -514,9 +549,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                 break;
             }
             const int cw = cur.chunk_words();
-            const unsigned char* wst = ring + s * stage_bytes + warp * (kTileBytes / 2);
-            const unsigned char* qst = ring + s * stage_bytes + kWideTiles * (kTileBytes / 2);
-            if (tile_on) {
+            if (tiles_on > 0) {
                 // A lane needs 64 contiguous activation bytes per token and slice (its four packed words x 16
                 // codes), lanes of a quad 64 bytes apart: read straight, lanes cq and cq+2 would hit the same
                 // banks.  Lanes with cq >= 2 therefore take their four words in the order 2,3,0,1 (the sums do
@@ -525,28 +558,38 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                 // (INT4 weights: 32 bytes per lane, already conflict-free without the rotation.)
                 // Token columns beyond M read the last token's bytes instead of zeros: a column of the
                 // product depends on its own activations only, and those columns are never written.
+                // A warp whose second tile lies beyond the matrix computes it on stale bytes of the stage
+                // (the copy skipped it) and drops the result in the epilogue.
+                const uint32_t qs = ring_addr + s * stage_bytes + TILES * TILE_STAGE;
+                const uint32_t ws = ring_addr + s * stage_bytes + tile0 * TILE_STAGE;
+                uint32_t qa_lo[NT], qa_hi[NT];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) qa_lo[nt] = qs + q_lo[nt], qa_hi[nt] = qs + q_hi[nt];
+                const uint32_t wa_lo = ws + w_lo, wa_hi = ws + w_hi;
                 auto slice = [&](int sl) {
                     uint32_t qb[NT][4 * T::NPL];
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
-                        const unsigned char* src = qst + q_off[nt] + sl * (16 * T::PER);
 #pragma unroll
                         for (int i = 0; i < T::NPL; ++i) {
-                            // NPL 16-byte pieces hold the lane's four words in order; piece i holds word 4i/NPL
-                            const uint4 v = *reinterpret_cast<const uint4*>(src + piece_off[i]);
+                            const uint32_t a = (i < T::NPL / 2 ? qa_lo[nt] + i * 16 : qa_hi[nt] + (i - T::NPL / 2) * 16) + sl * (16 * T::PER);
+                            const uint4 v = lds128(a);
                             qb[nt][4 * i] = v.x, qb[nt][4 * i + 1] = v.y, qb[nt][4 * i + 2] = v.z, qb[nt][4 * i + 3] = v.w;
                         }
                     }
-                    const unsigned char* wsrc = wst + w_off + sl * 1024;
-                    const uint2 a_lo = *reinterpret_cast<const uint2*>(wsrc), a_hi = *reinterpret_cast<const uint2*>(wsrc + w_hi);
-                    const uint2 b_lo = *reinterpret_cast<const uint2*>(wsrc + 512), b_hi = *reinterpret_cast<const uint2*>(wsrc + 512 + w_hi);
-                    const uint4 wa = make_uint4(a_lo.x, a_lo.y, a_hi.x, a_hi.y);
-                    const uint4 wb = make_uint4(b_lo.x, b_lo.y, b_hi.x, b_hi.y);
-                    mma_tile_step<LV, NT, true>(acc, wa, wb, qb);
-                };
-                if (cw == kWideChunkWords) {
 #pragma unroll
-                    for (int sl = 0; sl < kWideChunkWords / 16; ++sl) slice(sl);
+                    for (int r = 0; r < RT; ++r) {
+                        const uint32_t o = r * TILE_STAGE + sl * 1024;
+                        const uint2 a_lo = lds64(wa_lo + o), a_hi = lds64(wa_hi + o);
+                        const uint2 b_lo = lds64(wa_lo + o + 512), b_hi = lds64(wa_hi + o + 512);
+                        const uint4 wa = make_uint4(a_lo.x, a_lo.y, a_hi.x, a_hi.y);
+                        const uint4 wb = make_uint4(b_lo.x, b_lo.y, b_hi.x, b_hi.y);
+                        mma_tile_step<LV, NT, true>(acc[r], wa, wb, qb);
+                    }
+                };
+                if (cw == CW) {
+#pragma unroll
+                    for (int sl = 0; sl < CW / 16; ++sl) slice(sl);
                 } else {
                     for (int sl = 0; 16 * sl < cw; ++sl) slice(sl);   // 16-word slices of a short last chunk
                 }
@@ -560,8 +603,12 @@ linear_grouped_wide_kernel(const GroupParams gp) {
         }
         if (!ok) break;
 
-        // epilogue from registers: rows g and g+8 of the tile, tokens nt*8 + 2cq + {0,1}
-        if (tile_on) {
+        // epilogue from registers: rows g and g+8 of each tile, tokens nt*8 + 2cq + {0,1}; the scales and token
+        // sums were fetched when the item began
+#pragma unroll
+        for (int r = 0; r < RT; ++r) {
+            if (r >= tiles_on) continue;
+            const int row0 = cur_n0 + 16 * (tile0 + r);
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -571,11 +618,11 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                     if (tok < M && n < P->N) {
                         int v[T::NACC];
 #pragma unroll
-                        for (int a = 0; a < T::NACC; ++a) v[a] = acc[nt][a][i];
-                        const int acc_v = level_sum<LV, true, T::NACC>(v, gp.sumq[P->index * 16 + tok]);
+                        for (int a = 0; a < T::NACC; ++a) v[a] = acc[r][nt][a][i];
+                        const int acc_v = level_sum<LV, true, T::NACC>(v, e_sq[nt][i & 1]);
                         const size_t idx = static_cast<size_t>(tok) * P->N + n;
                         if (P->acc_debug) P->acc_debug[idx] = acc_v;
-                        const float y = scale_epilogue(acc_v, P->s_a[tok], __ldg(P->s_n + n));
+                        const float y = scale_epilogue(acc_v, e_sa[nt][i & 1], e_sn[r][i >> 1]);
                         if (gp.y_bf16) static_cast<uint16_t*>(P->Y)[idx] = f32_to_bf16_bits(y);
                         else static_cast<float*>(P->Y)[idx] = y;
                     }

@@ -337,6 +337,30 @@ def test_grouped_forward(name, M):
     check_outputs(plan.outputs[2], plan.accs[2], refs[2][2], refs[2][3], False)
 
 
+@pytest.mark.parametrize("name", list(LEVELS))
+@pytest.mark.parametrize("M", [9, 16])
+def test_grouped_forward_long_list(name, M):
+    # a list long enough (>= two 256-row items per SM) for the plan to give every warp two row tiles; ragged N:
+    # a last item with a single valid tile, one with a half-filled second tile of a warp, short last chunks of K
+    lv = LEVELS[name][0]
+    shapes = [(8200, 256), (8192, 512), (8472, 256), (8192, 256), (8000, 384 if lv == oracle.INT4 else 768), (8192, 256),
+              (8192, 256), (8192, 256), (8192, 256), (8192, 256)]
+    probs, refs = [], []
+    for i, (N, K) in enumerate(shapes):
+        W = synth.gaussian_weights(800 + i, N, K)
+        x, _ = synth.activations(820 + i, M, K, max(1, K // 100))
+        B = synth.had_block_for(K)
+        p_ref, s_n, codes = oracle.pack_weights(W, lv, oracle.SCALE_ABSMAX)
+        q_ref, sa_ref = oracle.quantize_act(x, B, 0.9)
+        refs.append(oracle.linear(codes, lv, s_n, q_ref, sa_ref))
+        probs.append((dev(x), dev(p_ref.view(np.int32)), dev(s_n), B))
+    plan = qift.qift_group_plan(probs, lv, 0.9, want_acc=True)
+    outs = qift.qift_group_forward(plan)
+    assert_status_clean()
+    for (y_ref, acc_ref), y, acc in zip(refs, outs, plan.accs):
+        check_outputs(y, acc, y_ref, acc_ref, False)
+
+
 @pytest.mark.parametrize("M", [1, 7])
 def test_grouped_shared_activation(M):
     # q/k/v-style and gate/up-style modules read one activation: the plan quantizes it once (the buffers of the

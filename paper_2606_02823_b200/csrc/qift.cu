@@ -27,8 +27,6 @@ namespace {
 // (measured on 32 LLaMA-2-7B layers: MNZ 369 us flat against 348 / 385 us at 5 / 6 rows for the K-split
 // kernel; PoT 510 against 561 at 2 rows; INT4 641 against 604 at 8 rows).
 inline int wide_min_m(int lv) { return lv == QIFT_LEVELS_POT ? 2 : lv == QIFT_LEVELS_INT4 ? 9 : 6; }
-// ... and from this many on, two row tiles per warp (256-row items), when the list is long enough.
-inline int wide2_min_m(int lv) { return lv == QIFT_LEVELS_POT ? 9 : 17; }  // measured: 2.7 against 2.5 TB/s at 16 rows for PoT, slower for the others
 constexpr int kFusedMaxM = 128;
 constexpr int kFusedPairMaxM = 512;
 inline int auto_prefill_route(int M) {
@@ -620,14 +618,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     if (M > 16) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (plan_bytes < qift_group_plan_bytes(count)) return QIFT_ERR_WORKSPACE;
     if (!aligned16(plan_dev) || !aligned16(plan_host)) return QIFT_ERR_ALIGNMENT;
-    // Rows per work item, which also selects the kernel (dispatch_grouped): 64 / 32 for the K-split kernel, 128 for the
-    // row-split kernel, 256 (two row tiles per warp) when that still leaves at least two items per SM.
-    int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : (M == 1) ? 64 : 32;
-    if (rows_per_item == kWideRows && M >= wide2_min_m(levels)) {
-        long long items256 = 0;
-        for (int i = 0; i < count; ++i) items256 += (problems[i].N + 2 * kWideRows - 1) / (2 * kWideRows);
-        if (items256 >= 2ll * sm_count()) rows_per_item = 2 * kWideRows;
-    }
+    const int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : (M == 1) ? 64 : 32;  // must match dispatch_grouped's row tiles
     GroupHeader* h = static_cast<GroupHeader*>(plan_host);
     GroupProblemDev* d = reinterpret_cast<GroupProblemDev*>(h + 1);
     int items = 0, max_k = 0, any_kron = 0;
@@ -733,8 +724,8 @@ int launch_grouped_wide(const GroupHeader* h, const GroupProblemDev* host, const
 template <int LV>
 int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
                      cudaStream_t st) {
-    if (h->rows_per_item == 2 * kWideRows)
-        return h->M > 8 ? launch_grouped_wide<LV, 2, 1, 16>(h, host, dev, sumq, st) : launch_grouped_wide<LV, 1, 1, 16>(h, host, dev, sumq, st);
+    // (256-row items -- two row tiles per warp, or sixteen consumer warps -- were measured slower: 3.2 / 3.2 against
+    // 3.9 TB/s at 16 rows.)
     if (h->rows_per_item == kWideRows)
         return h->M > 8 ? launch_grouped_wide<LV, 2, 1, 8>(h, host, dev, sumq, st) : launch_grouped_wide<LV, 1, 1, 8>(h, host, dev, sumq, st);
     if (h->M == 1) return launch_grouped<LV, 1, 4, true>(h, host, dev, sumq, st);

@@ -27,7 +27,8 @@ struct GroupHeader {
     int rows_per_item;  // 16 * RT
     int max_k;
     int any_kron;       // some problem's had_block selects the full-dimension rotation (K = 28 * 2^p)
-    int reserved[5];
+    int q_chunk_bytes;  // 0: q_a row-major [M][K]; else chunk-major for the row-split kernel (ChunkMajorDst)
+    int reserved[4];
 };
 static_assert(sizeof(GroupHeader) == 64, "header is one 64-byte record");
 
@@ -56,10 +57,25 @@ constexpr uint32_t kGroupMagic = 0x51494654u;
 // q_a is written PRESCALED for the product kernel (see mma_tile_step): with two-bit weights the
 // bytes of the even code planes (k % 16 in 0..3 or 8..11) hold 4*q, with INT4 weights the bytes of
 // plane 0 (k % 8 in 0..3) hold 16*q; sumq holds the plain sum of q.
+// Layout of q_a for the row-split product kernel, which stages one K-chunk of ALL tokens per pipeline stage: chunk
+// after chunk, inside a chunk token after token (so a stage is one contiguous piece of memory, one bulk copy), and
+// inside a token's chunk the 16-byte groups of an odd token swapped in pairs -- the product kernel's lanes read
+// tokens g and g+1 at the same group index in one instruction, and the swap puts them on different banks.
+//   byte address of group q of token m:  c = 16 q / CB,  c CB M + m min(CB, K - c CB) + 16 ((q mod CB/16) xor (m & 1))
+struct ChunkMajorDst {
+    int8_t* q_a;
+    int m, M, K, cb;
+    __device__ __forceinline__ void store(int q, uint4 v) const {
+        const int c = (16 * q) / cb, piece = q - c * (cb / 16);
+        const int bytes = min(cb, K - c * cb);
+        *reinterpret_cast<uint4*>(q_a + static_cast<size_t>(c) * cb * M + static_cast<size_t>(m) * bytes + 16 * (piece ^ (m & 1))) = v;
+    }
+};
+
 template <bool BF16_IN, bool KRON = false>
 __global__ void __launch_bounds__(kRowThreads)
 quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* __restrict__ sumq, int M, float clip,
-                            int int4_weights) {
+                            int int4_weights, int q_chunk_bytes) {
     extern __shared__ __align__(16) float row[];
     __shared__ float red[kRowThreads / 32 + 2];
     __shared__ int redi[kRowThreads / 32];
@@ -73,7 +89,9 @@ quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* _
     const RowScale sc = block_row_scale(load_and_transform<BF16_IN, KRON>(P.X, m, K, B, row), clip, red);
     if (threadIdx.x == 0) P.s_a[m] = (B > 1) ? __fmul_rn(sc.s_u, P.inv_sqrt_b) : sc.s_u;
     // 32-bit word i of a 16-byte group = code plane (two-bit: i; INT4: i & 1); even planes are prescaled
-    int total = quantize_row<true>(row, K, sc, P.q_a + m * K, int4_weights ? 16.0f : 4.0f, 1.0f);
+    const float mult = int4_weights ? 16.0f : 4.0f;
+    int total = q_chunk_bytes ? quantize_row<true>(row, K, sc, ChunkMajorDst{P.q_a, static_cast<int>(m), M, K, q_chunk_bytes}, mult, 1.0f)
+                              : quantize_row<true>(row, K, sc, RowMajorDst{P.q_a + m * K}, mult, 1.0f);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
     if ((threadIdx.x & 31) == 0) redi[threadIdx.x >> 5] = total;
@@ -388,7 +406,6 @@ linear_grouped_kernel(const GroupParams gp) {
 // loop, accumulates all 16 tokens in registers and writes its outputs itself -- no reduction, no CTA
 // barrier.  The price is that every warp reads the whole activation slice of a stage, so stages are
 // half tiles (64 words per row: 32 KB of weights + 17 KB of activations at 16 tokens), four deep.
-constexpr int kWideQPad = 16;                    // token stride = 16 bytes mod 128: see the consumer's loads
 constexpr int kWideRows = 16 * kDecWarps;        // 128 rows per item with one tile per warp
 
 // CWARPS consumer warps with RT row tiles each: an item is 16 * CWARPS * RT rows.  256-row items come either as
@@ -399,7 +416,7 @@ __host__ __device__ constexpr int wide_chunk_words(int tiles) { return tiles > 8
 
 __host__ __device__ inline size_t wide_stage_bytes(int lv, int M, int tiles) {
     const int cw = wide_chunk_words(tiles);
-    return static_cast<size_t>(tiles) * (cw * 64) + static_cast<size_t>(M) * (cw * codes_per_word(lv) + kWideQPad);
+    return static_cast<size_t>(tiles) * (cw * 64) + static_cast<size_t>(M) * (cw * codes_per_word(lv));
 }
 __host__ __device__ inline size_t wide_smem_bytes(int lv, int M, int tiles, int stages, int count) {
     return static_cast<size_t>(count) * sizeof(SmemProblem) + stages * (wide_stage_bytes(lv, M, tiles) + 16) + 16;
@@ -413,7 +430,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     constexpr int CW = wide_chunk_words(TILES);
     constexpr int THREADS = (CWARPS + 1) * 32;
     constexpr int TILE_STAGE = CW * 64;          // bytes of one tile in a stage: CW words x 16 rows, contiguous in the packed order
-    constexpr int QSTRIDE = CW * T::PER + kWideQPad;
+    constexpr int CB = CW * T::PER;              // bytes of one token's activations in a full chunk
     using Cursor = GroupCursor<T::PER, CW>;
     extern __shared__ __align__(128) unsigned char smem[];
     const int M = gp.M;
@@ -459,10 +476,10 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                 bulk_g2s(dst + lane * TILE_STAGE, c.wbase + lane * c.rb_bytes + static_cast<size_t>(c.chunk) * TILE_STAGE, bytes, &full[s]);
         };
         auto issue_q = [&](const Cursor& c, int s) {
-            const uint32_t seg = c.chunk_words() * T::PER;
-            unsigned char* dst = ring + s * stage_bytes + TILES * TILE_STAGE;
-            for (int m = lane; m < M; m += 32)
-                bulk_g2s(dst + m * QSTRIDE, c.q_a + static_cast<size_t>(m) * c.K + static_cast<size_t>(c.chunk) * (CW * T::PER), seg, &full[s]);
+            // chunk-major q_a (ChunkMajorDst): the chunk of all M tokens is one contiguous piece
+            if (lane == 0)
+                bulk_g2s(ring + s * stage_bytes + TILES * TILE_STAGE, c.q_a + static_cast<size_t>(c.chunk) * CB * M,
+                         static_cast<uint32_t>(c.chunk_words() * T::PER * M), &full[s]);
         };
         Cursor a;
         a.init(table, gp.count, gp.item_first, gp.item_end, 16 * TILES);
@@ -492,15 +509,22 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     const int g = lane >> 2, cq = lane & 3;
     // per-lane byte offsets inside a stage, fixed for the whole kernel
     const int rot = (T::PER == 16) ? (cq & 2) : 0;
-    // Activation pieces: NPL 16-byte pieces per token hold the lane's four words in order; a lane visits them
-    // starting at piece `rot` (order 2,3,0,1 for cq >= 2).  Two byte offsets per token tile cover that with constant
-    // displacements: the first half of the visit starts at q_lo, the second at q_hi.
-    uint32_t q_lo[NT], q_hi[NT];
+    // Activations of a stage: token after token, a token's chunk contiguous, the 16-byte pieces of odd tokens
+    // swapped in pairs (ChunkMajorDst).  A lane needs 64 contiguous bytes per token and slice (its four packed
+    // words x 16 codes = NPL pieces), lanes of a quad 64 bytes apart: read straight, lanes cq and cq+2 would hit the
+    // same banks, so lanes with cq >= 2 visit their pieces in the order 2,3,0,1 (the sums do not depend on the
+    // order); lanes g and g+1 read the same piece index of neighbouring tokens, which the pair swap separates.
+    // Every quarter-warp then covers all eight 16-byte bank groups.  (INT4 weights: 32 bytes per lane, two pieces.)
+    // Token columns beyond M read the last token's bytes: a column of the product depends on its own
+    // activations only, and those columns are never written.
+    int q_tok[NT];
+    uint32_t q_piece[NT][T::NPL];   // byte offset inside the token's chunk of the i-th piece this lane visits
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-        const uint32_t tok = static_cast<uint32_t>(min(nt * 8 + g, M - 1) * QSTRIDE + 4 * cq * T::PER);
-        q_lo[nt] = tok + rot * (T::NPL * 4);                                   // pieces rot .. rot + NPL/2 - 1
-        q_hi[nt] = tok + ((rot ? 0 : T::NPL / 2) * 16);                        // the other half
+        q_tok[nt] = min(nt * 8 + g, M - 1);
+#pragma unroll
+        for (int i = 0; i < T::NPL; ++i)
+            q_piece[nt][i] = 4 * cq * T::PER + 16 * (((i + rot * T::NPL / 4) % T::NPL) ^ (q_tok[nt] & 1));
     }
     const uint32_t w_lo = lane * 16 + 4 * rot, w_hi = w_lo + 8 - 8 * rot;      // the two word pairs of a lane's four words
     const uint32_t ring_addr = smem_u32(ring);
@@ -550,21 +574,15 @@ linear_grouped_wide_kernel(const GroupParams gp) {
             }
             const int cw = cur.chunk_words();
             if (tiles_on > 0) {
-                // A lane needs 64 contiguous activation bytes per token and slice (its four packed words x 16
-                // codes), lanes of a quad 64 bytes apart: read straight, lanes cq and cq+2 would hit the same
-                // banks.  Lanes with cq >= 2 therefore take their four words in the order 2,3,0,1 (the sums do
-                // not depend on the order) -- with a token stride of 16 bytes mod 128 every quarter-warp then
-                // covers all eight 16-byte bank groups.
-                // (INT4 weights: 32 bytes per lane, already conflict-free without the rotation.)
-                // Token columns beyond M read the last token's bytes instead of zeros: a column of the
-                // product depends on its own activations only, and those columns are never written.
                 // A warp whose second tile lies beyond the matrix computes it on stale bytes of the stage
                 // (the copy skipped it) and drops the result in the epilogue.
                 const uint32_t qs = ring_addr + s * stage_bytes + TILES * TILE_STAGE;
                 const uint32_t ws = ring_addr + s * stage_bytes + tile0 * TILE_STAGE;
-                uint32_t qa_lo[NT], qa_hi[NT];
+                uint32_t qa[NT][T::NPL];
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) qa_lo[nt] = qs + q_lo[nt], qa_hi[nt] = qs + q_hi[nt];
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int i = 0; i < T::NPL; ++i) qa[nt][i] = qs + q_tok[nt] * (cw * T::PER) + q_piece[nt][i];
                 const uint32_t wa_lo = ws + w_lo, wa_hi = ws + w_hi;
                 auto slice = [&](int sl) {
                     uint32_t qb[NT][4 * T::NPL];
@@ -572,8 +590,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                     for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
                         for (int i = 0; i < T::NPL; ++i) {
-                            const uint32_t a = (i < T::NPL / 2 ? qa_lo[nt] + i * 16 : qa_hi[nt] + (i - T::NPL / 2) * 16) + sl * (16 * T::PER);
-                            const uint4 v = lds128(a);
+                            const uint4 v = lds128(qa[nt][i] + sl * (16 * T::PER));
                             qb[nt][4 * i] = v.x, qb[nt][4 * i + 1] = v.y, qb[nt][4 * i + 2] = v.z, qb[nt][4 * i + 3] = v.w;
                         }
                     }

@@ -331,8 +331,14 @@ __device__ __forceinline__ uint32_t pack4_scaled(f32x2_t r01, f32x2_t r23, f32x2
 // mult_even / mult_odd: factor applied to the bytes of even / odd 32-bit words of each 16-byte group
 // (1 and 1 for the public layout).  With WANT_SUM returns the thread's partial sum of the quantized
 // values (taken from the packed bytes with dp4a, the factors divided out exactly).
-template <bool WANT_SUM>
-__device__ __forceinline__ int quantize_row(const float* row, int K, RowScale sc, int8_t* q_row, float mult_even, float mult_odd) {
+// Where the 16-byte groups of a quantized row go.  RowMajorDst: group q at byte 16 q of the row.
+struct RowMajorDst {
+    int8_t* q_row;
+    __device__ __forceinline__ void store(int q, uint4 v) const { reinterpret_cast<uint4*>(q_row)[q] = v; }
+};
+
+template <bool WANT_SUM, typename Dst>
+__device__ __forceinline__ int quantize_row(const float* row, int K, RowScale sc, Dst dst, float mult_even, float mult_odd) {
     const int groups = K / 16;
     const float s_u = sc.s_u, inv = sc.inv;
     const bool fast = inv != 0.0f;
@@ -373,7 +379,7 @@ __device__ __forceinline__ int quantize_row(const float* row, int K, RowScale sc
             sum_even = __dp4a(static_cast<int>(out[0]), 0x01010101, __dp4a(static_cast<int>(out[2]), 0x01010101, sum_even));
             sum_odd = __dp4a(static_cast<int>(out[1]), 0x01010101, __dp4a(static_cast<int>(out[3]), 0x01010101, sum_odd));
         }
-        reinterpret_cast<uint4*>(q_row)[q] = make_uint4(out[0], out[1], out[2], out[3]);
+        dst.store(q, make_uint4(out[0], out[1], out[2], out[3]));
     }
     return sum_even / static_cast<int>(mult_even) + sum_odd / static_cast<int>(mult_odd);
 }
@@ -390,7 +396,7 @@ quantize_act_kernel(const void* __restrict__ X, int K, int B, float clip, float 
     const size_t m = blockIdx.x;
     const RowScale sc = block_row_scale(load_and_transform<BF16_IN, KRON>(X, m, K, B, row), clip, red);
     if (threadIdx.x == 0) s_a[m] = (B > 1) ? __fmul_rn(sc.s_u, inv_sqrt_b) : sc.s_u;
-    quantize_row<false>(row, K, sc, q_a + m * K, 1.0f, 1.0f);
+    quantize_row<false>(row, K, sc, RowMajorDst{q_a + m * K}, 1.0f, 1.0f);
 }
 
 // S0: orthonormal blockwise rotation of fp32 rows.

@@ -9,6 +9,8 @@
 // matrices; eight consumer warps do the same in-register decode + mma.sync as the per-call kernel.
 #pragma once
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "decode.cuh"
 #include "rotate_quant.cuh"
@@ -412,10 +414,10 @@ constexpr int kWideRows = 16 * kDecWarps;        // 128 rows per item with one t
 // sixteen warps (twice the warps to hide the latencies of the load -> logic -> product chains) or as two tiles per
 // warp (the activation registers of a slice feed both tiles); their stages are a quarter tile of K (32 words) so
 // that as many stages fit as with 128 rows.
-__host__ __device__ constexpr int wide_chunk_words(int tiles) { return tiles > 8 ? 32 : 64; }
+__host__ __device__ constexpr int wide_chunk_words(int tiles, int nt) { return tiles > 8 ? 32 : nt == 1 ? 128 : 64; }
 
 __host__ __device__ inline size_t wide_stage_bytes(int lv, int M, int tiles) {
-    const int cw = wide_chunk_words(tiles);
+    const int cw = wide_chunk_words(tiles, M > 8 ? 2 : 1);
     return static_cast<size_t>(tiles) * (cw * 64) + static_cast<size_t>(M) * (cw * codes_per_word(lv));
 }
 __host__ __device__ inline size_t wide_smem_bytes(int lv, int M, int tiles, int stages, int count) {
@@ -427,7 +429,7 @@ __global__ void __launch_bounds__((CWARPS + 1) * 32, 1)
 linear_grouped_wide_kernel(const GroupParams gp) {
     using T = DecodeTraits<LV>;
     constexpr int TILES = CWARPS * RT;           // row tiles per item
-    constexpr int CW = wide_chunk_words(TILES);
+    constexpr int CW = wide_chunk_words(TILES, NT);
     constexpr int THREADS = (CWARPS + 1) * 32;
     constexpr int TILE_STAGE = CW * 64;          // bytes of one tile in a stage: CW words x 16 rows, contiguous in the packed order
     constexpr int CB = CW * T::PER;              // bytes of one token's activations in a full chunk
@@ -534,15 +536,20 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     int s = 0;
     uint32_t ph = 0;
     while (cur.valid() && ok) {
-        int acc[RT][NT][T::NACC][4];
+        // With one token tile a warp would have only NACC dependent chains of product instructions; alternate
+        // slices then go to a second set of accumulators (added up before the epilogue).
+        constexpr int KS = (NT * RT == 1) ? 2 : 1;
+        int acc[KS][RT][NT][T::NACC][4];
 #pragma unroll
-        for (int r = 0; r < RT; ++r)
+        for (int k = 0; k < KS; ++k)
 #pragma unroll
-            for (int b = 0; b < NT; ++b)
+            for (int r = 0; r < RT; ++r)
 #pragma unroll
-                for (int t = 0; t < T::NACC; ++t)
+                for (int b = 0; b < NT; ++b)
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) acc[r][b][t][i] = 0;
+                    for (int t = 0; t < T::NACC; ++t)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) acc[k][r][b][t][i] = 0;
         const SmemProblem* P = &table[cur.p];
         const int cur_n0 = cur.n0;
         const int tile0 = warp * RT;                       // this warp's tiles: tile0 .. tile0 + RT - 1
@@ -584,7 +591,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
 #pragma unroll
                     for (int i = 0; i < T::NPL; ++i) qa[nt][i] = qs + q_tok[nt] * (cw * T::PER) + q_piece[nt][i];
                 const uint32_t wa_lo = ws + w_lo, wa_hi = ws + w_hi;
-                auto slice = [&](int sl) {
+                auto slice = [&](int sl, auto ks) {
                     uint32_t qb[NT][4 * T::NPL];
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
@@ -601,14 +608,17 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                         const uint2 b_lo = lds64(wa_lo + o + 512), b_hi = lds64(wa_hi + o + 512);
                         const uint4 wa = make_uint4(a_lo.x, a_lo.y, a_hi.x, a_hi.y);
                         const uint4 wb = make_uint4(b_lo.x, b_lo.y, b_hi.x, b_hi.y);
-                        mma_tile_step<LV, NT, true>(acc[r], wa, wb, qb);
+                        mma_tile_step<LV, NT, true>(acc[decltype(ks)::value][r], wa, wb, qb);
                     }
                 };
                 if (cw == CW) {
 #pragma unroll
-                    for (int sl = 0; sl < CW / 16; ++sl) slice(sl);
+                    for (int sl = 0; sl < CW / 16; sl += 2) {
+                        slice(sl, std::integral_constant<int, 0>{});
+                        slice(sl + 1, std::integral_constant<int, KS - 1>{});
+                    }
                 } else {
-                    for (int sl = 0; 16 * sl < cw; ++sl) slice(sl);   // 16-word slices of a short last chunk
+                    for (int sl = 0; 16 * sl < cw; ++sl) slice(sl, std::integral_constant<int, 0>{});   // 16-word slices of a short last chunk
                 }
             }
             __syncwarp();
@@ -620,6 +630,16 @@ linear_grouped_wide_kernel(const GroupParams gp) {
         }
         if (!ok) break;
 
+        if (KS == 2) {
+#pragma unroll
+            for (int r = 0; r < RT; ++r)
+#pragma unroll
+                for (int b = 0; b < NT; ++b)
+#pragma unroll
+                    for (int t = 0; t < T::NACC; ++t)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) acc[0][r][b][t][i] += acc[KS - 1][r][b][t][i];
+        }
         // epilogue from registers: rows g and g+8 of each tile, tokens nt*8 + 2cq + {0,1}; the scales and token
         // sums were fetched when the item began
 #pragma unroll
@@ -635,7 +655,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                     if (tok < M && n < P->N) {
                         int v[T::NACC];
 #pragma unroll
-                        for (int a = 0; a < T::NACC; ++a) v[a] = acc[r][nt][a][i];
+                        for (int a = 0; a < T::NACC; ++a) v[a] = acc[0][r][nt][a][i];
                         const int acc_v = level_sum<LV, true, T::NACC>(v, e_sq[nt][i & 1]);
                         const size_t idx = static_cast<size_t>(tok) * P->N + n;
                         if (P->acc_debug) P->acc_debug[idx] = acc_v;

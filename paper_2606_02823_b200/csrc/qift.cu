@@ -23,10 +23,10 @@ namespace {
 // Prefill routes by token count (measured on a LLaMA-3.1-8B layer): up to 128 rows one CTA per tile
 // expanding the codes in the kernel; up to 512 rows CTA pairs expanding in the kernel (one expansion
 // per 256-token tile); beyond that, expanding once into an int8 scratch and re-reading it wins.
-// Grouped decode: from this many token rows on the row-split kernel (128-row items) is the faster one
-// (measured on 32 LLaMA-2-7B layers: MNZ 369 us flat against 348 / 385 us at 5 / 6 rows for the K-split
-// kernel; PoT 510 against 561 at 2 rows; INT4 641 against 604 at 8 rows).
-inline int wide_min_m(int lv) { return lv == QIFT_LEVELS_POT ? 2 : lv == QIFT_LEVELS_INT4 ? 9 : 6; }
+// Grouped decode: from this many token rows on the row-split kernel (128-row items) is the faster one.  Measured
+// on 16 LLaMA-2-7B layers, row-split flat in M against K-split at 1 / 2 / 4 rows: MNZ 140 us against 125 / 152 /
+// 168 us; INT4 232 against 236 / 239 / 258; PoT 191 against 218 / 215 / 217.
+inline int wide_min_m(int lv) { return lv == QIFT_LEVELS_POT ? 1 : 2; }
 constexpr int kFusedMaxM = 128;
 constexpr int kFusedPairMaxM = 512;
 inline int auto_prefill_route(int M) {
@@ -653,7 +653,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     h->max_k = max_k;
     h->any_kron = any_kron;
     // the row-split kernel stages one K-chunk of all tokens per copy: its q_a is chunk-major (ChunkMajorDst)
-    h->q_chunk_bytes = (rows_per_item == kWideRows) ? wide_chunk_words(kDecWarps) * codes_per_word(levels) : 0;
+    h->q_chunk_bytes = (rows_per_item == kWideRows) ? wide_chunk_words(kDecWarps, M > 8 ? 2 : 1) * codes_per_word(levels) : 0;
     return cuda_status(cudaMemcpyAsync(plan_dev, plan_host, sizeof(GroupHeader) + static_cast<size_t>(count) * sizeof(GroupProblemDev),
                                        cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));
 }

@@ -194,6 +194,46 @@ __device__ __forceinline__ void mma_tile_step(int (&acc)[NT][DecodeTraits<LV>::N
     }
 }
 
+// PoT levels {-4,-1,+1,+4} are not affine in the code, so the masked-code operand above needs one product per code
+// BIT.  Where the activation bytes can be laid out to order (the grouped row-split kernel), the levels themselves
+// become the operand instead: a byte-permute instruction is a four-entry table lookup on four selector nibbles,
+// and (w >> s) & 0x3333 holds four codes of a packed word as nibbles.  One word yields four signed-byte operand
+// registers whose bytes are the levels of codes k = {0,8,1,9}, {4,12,5,13}, {2,10,3,11}, {6,14,7,15} of the word;
+// the quantizer writes each 16-byte activation group in the same order (pot_lut_order), unscaled.  One product
+// instruction per 512 codes and token tile, one accumulator set, no correction term.
+__device__ __forceinline__ void pot_lut_operands(uint32_t w, uint32_t (&a)[4]) {
+    constexpr uint32_t kLut = 0x0401fffcu;  // bytes: level of code 0, 1, 2, 3
+    const uint32_t y = w & 0x33333333u, z = (w >> 2) & 0x33333333u;
+    a[0] = __byte_perm(kLut, kLut, y);
+    a[1] = __byte_perm(kLut, kLut, z);
+    a[2] = __byte_perm(kLut, kLut, y >> 16);
+    a[3] = __byte_perm(kLut, kLut, z >> 16);
+}
+
+// The matching order of a 16-byte activation group (four words of four consecutive-k bytes each).
+__device__ __forceinline__ uint4 pot_lut_order(uint4 q) {
+    return make_uint4(__byte_perm(q.x, q.z, 0x5140), __byte_perm(q.y, q.w, 0x5140), __byte_perm(q.x, q.z, 0x7362),
+                      __byte_perm(q.y, q.w, 0x7362));
+}
+
+template <int NT>
+__device__ __forceinline__ void mma_tile_step_pot_lut(int (&acc)[NT][1][4], const uint4 wa, const uint4 wb,
+                                                      const uint32_t (&qb)[NT][16]) {
+    const uint32_t lo[4] = {wa.x, wa.y, wa.z, wa.w};
+    const uint32_t hi[4] = {wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint32_t al[4], ah[4];
+        pot_lut_operands(lo[i], al);
+        pot_lut_operands(hi[i], ah);
+#pragma unroll
+        for (int p = 0; p < 2; ++p)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+                mma_s8s8(acc[nt][0], al[2 * p], ah[2 * p], al[2 * p + 1], ah[2 * p + 1], qb[nt][4 * i + 2 * p], qb[nt][4 * i + 2 * p + 1]);
+    }
+}
+
 struct DecodeParams {
     const uint32_t* packed;
     const float* s_n;

@@ -30,7 +30,8 @@ struct GroupHeader {
     int max_k;
     int any_kron;       // some problem's had_block selects the full-dimension rotation (K = 28 * 2^p)
     int q_chunk_bytes;  // 0: q_a row-major [M][K]; else chunk-major for the row-split kernel (ChunkMajorDst)
-    int reserved[4];
+    int q_pot_lut;      // q_a unscaled, bytes of each 16-byte group in pot_lut_order (PoT on the row-split kernel)
+    int reserved[3];
 };
 static_assert(sizeof(GroupHeader) == 64, "header is one 64-byte record");
 
@@ -66,8 +67,9 @@ constexpr uint32_t kGroupMagic = 0x51494654u;
 //   byte address of group q of token m:  c = 16 q / CB,  c CB M + m min(CB, K - c CB) + 16 ((q mod CB/16) xor (m & 1))
 struct ChunkMajorDst {
     int8_t* q_a;
-    int m, M, K, cb;
+    int m, M, K, cb, pot_lut;
     __device__ __forceinline__ void store(int q, uint4 v) const {
+        if (pot_lut) v = pot_lut_order(v);
         const int c = (16 * q) / cb, piece = q - c * (cb / 16);
         const int bytes = min(cb, K - c * cb);
         *reinterpret_cast<uint4*>(q_a + static_cast<size_t>(c) * cb * M + static_cast<size_t>(m) * bytes + 16 * (piece ^ (m & 1))) = v;
@@ -77,7 +79,7 @@ struct ChunkMajorDst {
 template <bool BF16_IN, bool KRON = false>
 __global__ void __launch_bounds__(kRowThreads)
 quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* __restrict__ sumq, int M, float clip,
-                            int int4_weights, int q_chunk_bytes) {
+                            int int4_weights, int q_chunk_bytes, int q_pot_lut) {
     extern __shared__ __align__(16) float row[];
     __shared__ float red[kRowThreads / 32 + 2];
     __shared__ int redi[kRowThreads / 32];
@@ -91,8 +93,8 @@ quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* _
     const RowScale sc = block_row_scale(load_and_transform<BF16_IN, KRON>(P.X, m, K, B, row), clip, red);
     if (threadIdx.x == 0) P.s_a[m] = (B > 1) ? __fmul_rn(sc.s_u, P.inv_sqrt_b) : sc.s_u;
     // 32-bit word i of a 16-byte group = code plane (two-bit: i; INT4: i & 1); even planes are prescaled
-    const float mult = int4_weights ? 16.0f : 4.0f;
-    int total = q_chunk_bytes ? quantize_row<true>(row, K, sc, ChunkMajorDst{P.q_a, static_cast<int>(m), M, K, q_chunk_bytes}, mult, 1.0f)
+    const float mult = q_pot_lut ? 1.0f : int4_weights ? 16.0f : 4.0f;
+    int total = q_chunk_bytes ? quantize_row<true>(row, K, sc, ChunkMajorDst{P.q_a, static_cast<int>(m), M, K, q_chunk_bytes, q_pot_lut}, mult, 1.0f)
                               : quantize_row<true>(row, K, sc, RowMajorDst{P.q_a + m * K}, mult, 1.0f);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
@@ -431,6 +433,11 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     constexpr int TILES = CWARPS * RT;           // row tiles per item
     constexpr int CW = wide_chunk_words(TILES, NT);
     constexpr int THREADS = (CWARPS + 1) * 32;
+    // PoT with two token tiles: levels by table lookup (pot_lut_operands) instead of code bit planes -- half the
+    // product instructions for more logic per word, which pays once the products are the bottleneck (measured on 16
+    // LLaMA-2-7B layers: 261 against 295 us at 16 rows, but 197 against 189 us at 8).
+    constexpr bool POT_LUT = (LV == QIFT_LEVELS_POT) && NT == 2;
+    constexpr int NACC = POT_LUT ? 1 : T::NACC;
     constexpr int TILE_STAGE = CW * 64;          // bytes of one tile in a stage: CW words x 16 rows, contiguous in the packed order
     constexpr int CB = CW * T::PER;              // bytes of one token's activations in a full chunk
     using Cursor = GroupCursor<T::PER, CW>;
@@ -539,7 +546,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
         // With one token tile a warp would have only NACC dependent chains of product instructions; alternate
         // slices then go to a second set of accumulators (added up before the epilogue).
         constexpr int KS = (NT * RT == 1) ? 2 : 1;
-        int acc[KS][RT][NT][T::NACC][4];
+        int acc[KS][RT][NT][NACC][4];
 #pragma unroll
         for (int k = 0; k < KS; ++k)
 #pragma unroll
@@ -547,7 +554,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
 #pragma unroll
                 for (int b = 0; b < NT; ++b)
 #pragma unroll
-                    for (int t = 0; t < T::NACC; ++t)
+                    for (int t = 0; t < NACC; ++t)
 #pragma unroll
                         for (int i = 0; i < 4; ++i) acc[k][r][b][t][i] = 0;
         const SmemProblem* P = &table[cur.p];
@@ -608,7 +615,8 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                         const uint2 b_lo = lds64(wa_lo + o + 512), b_hi = lds64(wa_hi + o + 512);
                         const uint4 wa = make_uint4(a_lo.x, a_lo.y, a_hi.x, a_hi.y);
                         const uint4 wb = make_uint4(b_lo.x, b_lo.y, b_hi.x, b_hi.y);
-                        mma_tile_step<LV, NT, true>(acc[decltype(ks)::value][r], wa, wb, qb);
+                        if constexpr (POT_LUT) mma_tile_step_pot_lut<NT>(acc[decltype(ks)::value][r], wa, wb, qb);
+                        else mma_tile_step<LV, NT, true>(acc[decltype(ks)::value][r], wa, wb, qb);
                     }
                 };
                 if (cw == CW) {
@@ -636,7 +644,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
 #pragma unroll
                 for (int b = 0; b < NT; ++b)
 #pragma unroll
-                    for (int t = 0; t < T::NACC; ++t)
+                    for (int t = 0; t < NACC; ++t)
 #pragma unroll
                         for (int i = 0; i < 4; ++i) acc[0][r][b][t][i] += acc[KS - 1][r][b][t][i];
         }
@@ -653,10 +661,15 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                     const int tok = nt * 8 + 2 * cq + (i & 1);
                     const int n = row0 + g + ((i & 2) ? 8 : 0);
                     if (tok < M && n < P->N) {
-                        int v[T::NACC];
+                        int acc_v;
+                        if constexpr (POT_LUT) {
+                            acc_v = acc[0][r][nt][0][i];   // the operands were the levels themselves
+                        } else {
+                            int v[NACC];
 #pragma unroll
-                        for (int a = 0; a < T::NACC; ++a) v[a] = acc[0][r][nt][a][i];
-                        const int acc_v = level_sum<LV, true, T::NACC>(v, e_sq[nt][i & 1]);
+                            for (int a = 0; a < NACC; ++a) v[a] = acc[0][r][nt][a][i];
+                            acc_v = level_sum<LV, true, NACC>(v, e_sq[nt][i & 1]);
+                        }
                         const size_t idx = static_cast<size_t>(tok) * P->N + n;
                         if (P->acc_debug) P->acc_debug[idx] = acc_v;
                         const float y = scale_epilogue(acc_v, e_sa[nt][i & 1], e_sn[r][i >> 1]);

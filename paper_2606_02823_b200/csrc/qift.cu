@@ -653,6 +653,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     h->max_k = max_k;
     h->any_kron = any_kron;
     // the row-split kernel stages one K-chunk of all tokens per copy: its q_a is chunk-major (ChunkMajorDst)
+    h->q_pot_lut = (rows_per_item == kWideRows && levels == QIFT_LEVELS_POT && M > 8) ? 1 : 0;  // the kernel's POT_LUT
     h->q_chunk_bytes = (rows_per_item == kWideRows) ? wide_chunk_words(kDecWarps, M > 8 ? 2 : 1) * codes_per_word(levels) : 0;
     return cuda_status(cudaMemcpyAsync(plan_dev, plan_host, sizeof(GroupHeader) + static_cast<size_t>(count) * sizeof(GroupProblemDev),
                                        cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));
@@ -751,7 +752,7 @@ int qift_group_quantize_act(const void* plan_host, const void* plan_dev, void* s
     cudaError_t e = allow_smem(kernel, smem);
     if (e != cudaSuccess) return cuda_status(e);
     return cuda_status(launch_pdl(kernel, grid, dim3(kRowThreads), smem, st, dev, sumq, h->M, h->clip,
-                                  h->levels == QIFT_LEVELS_INT4 ? 1 : 0, h->q_chunk_bytes));
+                                  h->levels == QIFT_LEVELS_INT4 ? 1 : 0, h->q_chunk_bytes, h->q_pot_lut));
 }
 
 int qift_group_linear(const void* plan_host, const void* plan_dev, void* stream) {

@@ -386,6 +386,7 @@ def run_gpu(args):
     }
     if rank == 0 and world == 1 and not args.no_prefill:
         out["mixed_stack"] = run_mixed_stack(torch, qift, L, device, gen, args)
+        out["batched_decode"] = run_batched_decode(torch, qift, L, device, gen, args)
         out["prefill"] = run_prefill(torch, qift, L, device, gen, pk)
         out["kv4"] = run_kv4(torch, qift, L, pk)
         out["diagnostics"] = run_diagnostics(torch, qift, pk)
@@ -440,6 +441,44 @@ def run_mixed_stack(torch, qift, L, device, gen, args):
     if args.layers >= 16:
         out["l_sweep"] = [point(args.layers * l // 32, args.layers - args.layers * l // 32) for l in (4, 8, 12)]
     return out
+
+
+def run_batched_decode(torch, qift, L, device, gen, args):
+    """Config 3: LLaMA-3.1-8B shapes, batched decode at M = 1, 4, 16 token rows, PoT {+-1,+-4} against the standard
+    {-2,-1,0,+1} set; grouped API (2 launches per step), 16 layers of distinct weights (0.87 GB per level set, larger
+    than L2), every module on its own activation.  Bytes = packed weights + scales + activations + outputs."""
+    vp = ctypes.c_void_p
+    st = vp(torch.cuda.current_stream().cuda_stream)
+    layers = max(1, min(16, args.layers))
+    rows = []
+    for name, lv in (("PoT", qift.POT), ("SYM", qift.SYM)):
+        base = build_stack(torch, qift, synth.LLAMA31_8B, layers, 16, lambda l, lv=lv: lv, 6000 + lv, torch.float32, torch.float32,
+                           device, gen)
+        for M in (1, 4, 16):
+            plan = qift.qift_group_plan([(m.x[:M].contiguous(), m.packed, m.s_n, m.B) for m in base], lv, CLIP)
+            algo = sum(product_bytes(M, m.N, m.K, m.bits) + quant_bytes(M, m.K) for m in base)
+
+            def step():
+                rc = L.qift_group_forward(vp(plan.host.data_ptr()), vp(plan.dev.data_ptr()), st)
+                assert rc == 0, rc
+
+            for _ in range(5):
+                step()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            steps = max(3, min(args.steps, 100))
+            e0.record()
+            for _ in range(steps):
+                step()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / steps
+            rows.append({"levels": name, "M": M, "ms_per_step": round(ms, 5), "tokens_per_s": round(M / (ms * 1e-3), 1),
+                         "value": round(algo / (ms * 1e-3) / 1e9, 1), "unit": "GB/s",
+                         "pct_of_8TBs": round(100 * algo / (ms * 1e-3) / 8e12, 1)})
+            del plan
+        del base
+    return {"workload": f"config 3: LLaMA-3.1-8B shapes, {layers} layers, grouped API, whole step (quantizer + product)", "points": rows}
 
 
 def run_kv4(torch, qift, L, pk):

@@ -535,7 +535,6 @@ linear_grouped_wide_kernel(const GroupParams gp) {
         for (int i = 0; i < T::NPL; ++i)
             q_piece[nt][i] = 4 * cq * T::PER + 16 * (((i + rot * T::NPL / 4) % T::NPL) ^ (q_tok[nt] & 1));
     }
-    const uint32_t w_lo = lane * 16 + 4 * rot, w_hi = w_lo + 8 - 8 * rot;      // the two word pairs of a lane's four words
     const uint32_t ring_addr = smem_u32(ring);
     Cursor cur;
     cur.init(table, gp.count, gp.item_first, gp.item_end, 16 * TILES);
@@ -597,7 +596,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                 for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                     for (int i = 0; i < T::NPL; ++i) qa[nt][i] = qs + q_tok[nt] * (cw * T::PER) + q_piece[nt][i];
-                const uint32_t wa_lo = ws + w_lo, wa_hi = ws + w_hi;
+                const uint32_t wa_base = ws + lane * 16;
                 auto slice = [&](int sl, auto ks) {
                     uint32_t qb[NT][4 * T::NPL];
 #pragma unroll
@@ -611,10 +610,21 @@ linear_grouped_wide_kernel(const GroupParams gp) {
 #pragma unroll
                     for (int r = 0; r < RT; ++r) {
                         const uint32_t o = r * TILE_STAGE + sl * 1024;
-                        const uint2 a_lo = lds64(wa_lo + o), a_hi = lds64(wa_hi + o);
-                        const uint2 b_lo = lds64(wa_lo + o + 512), b_hi = lds64(wa_hi + o + 512);
-                        const uint4 wa = make_uint4(a_lo.x, a_lo.y, a_hi.x, a_hi.y);
-                        const uint4 wb = make_uint4(b_lo.x, b_lo.y, b_hi.x, b_hi.y);
+                        // the lane's four words of rows g and g+8; lanes that visit their activation pieces in
+                        // the order 2,3,0,1 take the words in that order too: by selects after a 128-bit load, or
+                        // (PoT with one token tile, where the logic pipe is the limit) by two 64-bit loads, which
+                        // cost a two-way bank conflict instead
+                        uint4 wa, wb;
+                        if constexpr (LV == QIFT_LEVELS_POT && NT == 1) {
+                            const uint32_t lo_a = wa_base + o + 4 * rot, hi_a = lo_a + 8 - 8 * rot;
+                            const uint2 a_lo = lds64(lo_a), a_hi = lds64(hi_a), b_lo = lds64(lo_a + 512), b_hi = lds64(hi_a + 512);
+                            wa = make_uint4(a_lo.x, a_lo.y, a_hi.x, a_hi.y);
+                            wb = make_uint4(b_lo.x, b_lo.y, b_hi.x, b_hi.y);
+                        } else {
+                            const uint4 ra = lds128(wa_base + o), rb = lds128(wa_base + o + 512);
+                            wa = rot ? make_uint4(ra.z, ra.w, ra.x, ra.y) : ra;
+                            wb = rot ? make_uint4(rb.z, rb.w, rb.x, rb.y) : rb;
+                        }
                         if constexpr (POT_LUT) mma_tile_step_pot_lut<NT>(acc[decltype(ks)::value][r], wa, wb, qb);
                         else mma_tile_step<LV, NT, true>(acc[decltype(ks)::value][r], wa, wb, qb);
                     }

@@ -416,7 +416,7 @@ constexpr int kWideRows = 16 * kDecWarps;        // 128 rows per item with one t
 // sixteen warps (twice the warps to hide the latencies of the load -> logic -> product chains) or as two tiles per
 // warp (the activation registers of a slice feed both tiles); their stages are a quarter tile of K (32 words) so
 // that as many stages fit as with 128 rows.
-__host__ __device__ constexpr int wide_chunk_words(int tiles, int nt) { return tiles > 8 ? 32 : 128; }
+__host__ __device__ constexpr int wide_chunk_words(int tiles, int nt) { return tiles > 8 ? 64 : 128; }
 
 __host__ __device__ inline size_t wide_stage_bytes(int lv, int M, int tiles) {
     const int cw = wide_chunk_words(tiles, M > 8 ? 2 : 1);

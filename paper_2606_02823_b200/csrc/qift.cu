@@ -618,7 +618,14 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     if (M > 16) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (plan_bytes < qift_group_plan_bytes(count)) return QIFT_ERR_WORKSPACE;
     if (!aligned16(plan_dev) || !aligned16(plan_host)) return QIFT_ERR_ALIGNMENT;
-    const int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : (M == 1) ? 64 : 32;  // must match dispatch_grouped's row tiles
+    // Rows per work item, which also selects the kernel (dispatch_grouped): 64 / 32 for the K-split kernel, 128 for the
+    // row-split kernel, 256 (two row tiles per warp, with two token tiles) when that still leaves two items per SM.
+    int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : (M == 1) ? 64 : 32;
+    if (rows_per_item == kWideRows && M > 8 && levels != QIFT_LEVELS_POT) {  // PoT measured slower with two tiles
+        long long items256 = 0;
+        for (int i = 0; i < count; ++i) items256 += (problems[i].N + 2 * kWideRows - 1) / (2 * kWideRows);
+        if (items256 >= 2ll * sm_count()) rows_per_item = 2 * kWideRows;
+    }
     GroupHeader* h = static_cast<GroupHeader*>(plan_host);
     GroupProblemDev* d = reinterpret_cast<GroupProblemDev*>(h + 1);
     int items = 0, max_k = 0, any_kron = 0;
@@ -653,8 +660,8 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     h->max_k = max_k;
     h->any_kron = any_kron;
     // the row-split kernel stages one K-chunk of all tokens per copy: its q_a is chunk-major (ChunkMajorDst)
-    h->q_pot_lut = (rows_per_item == kWideRows && levels == QIFT_LEVELS_POT && M > 8) ? 1 : 0;  // the kernel's POT_LUT
-    h->q_chunk_bytes = (rows_per_item == kWideRows) ? wide_chunk_words(kDecWarps, M > 8 ? 2 : 1) * codes_per_word(levels) : 0;
+    h->q_pot_lut = (rows_per_item >= kWideRows && levels == QIFT_LEVELS_POT && M > 8) ? 1 : 0;  // the kernel's POT_LUT
+    h->q_chunk_bytes = (rows_per_item >= kWideRows) ? wide_chunk_words(rows_per_item / 16, M > 8 ? 2 : 1) * codes_per_word(levels) : 0;
     return cuda_status(cudaMemcpyAsync(plan_dev, plan_host, sizeof(GroupHeader) + static_cast<size_t>(count) * sizeof(GroupProblemDev),
                                        cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));
 }
@@ -729,6 +736,7 @@ int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const Gr
                      cudaStream_t st) {
     // (256-row items -- two row tiles per warp, or sixteen consumer warps -- were measured slower: 3.2 / 3.2 against
     // 3.9 TB/s at 16 rows.)
+    if (h->rows_per_item == 2 * kWideRows) return launch_grouped_wide<LV, 2, 2, 8>(h, host, dev, sumq, st);
     if (h->rows_per_item == kWideRows)
         return h->M > 8 ? launch_grouped_wide<LV, 2, 1, 8>(h, host, dev, sumq, st) : launch_grouped_wide<LV, 1, 1, 8>(h, host, dev, sumq, st);
     if (h->M == 1) return launch_grouped<LV, 1, 4, true>(h, host, dev, sumq, st);

@@ -68,8 +68,11 @@ typedef enum {
                                       tcgen05 GEMM, one CTA per tile; scratch N*K bytes            */
     QIFT_ROUTE_PREFILL_PAIR = 5,   /* the same with CTA pairs (tcgen05 cta_group::2, 256-token tiles);
                                       scratch N*K bytes                                            */
-    QIFT_ROUTE_PREFILL_FUSED_PAIR = 6 /* CTA pairs with the codes expanded in the kernel (each CTA
+    QIFT_ROUTE_PREFILL_FUSED_PAIR = 6, /* CTA pairs with the codes expanded in the kernel (each CTA
                                       expands half of the tile's channels); scratch 4*M            */
+    QIFT_ROUTE_DECODE_ROWS = 7 /* 2 <= M <= 16: the activations re-laid out into the scratch, then the
+                                  row-split kernel of the grouped path (128-row items, no reduction);
+                                  scratch M*K + 64 bytes                                          */
 } qift_route;
 
 const char* qift_status_string(int status);

@@ -21,6 +21,7 @@ SCALE_GIVEN, SCALE_ABSMAX, SCALE_MSE = 0, 1, 2
 F32, BF16 = 0, 1
 ROUTE_AUTO, ROUTE_GENERIC, ROUTE_DECODE, ROUTE_PREFILL, ROUTE_PREFILL_SCRATCH, ROUTE_PREFILL_PAIR = 0, 1, 2, 3, 4, 5
 ROUTE_PREFILL_FUSED_PAIR = 6
+ROUTE_DECODE_ROWS = 7
 
 EXPORTS = [
     "qift_status_string", "qift_packed_bytes", "qift_workspace_bytes", "qift_workspace_bytes_route", "qift_pack_weights",

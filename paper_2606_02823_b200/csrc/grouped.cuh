@@ -107,6 +107,36 @@ quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* _
     }
 }
 
+// Per-call products with 2..16 token rows take the row-split kernel as well: this kernel turns the public q_a
+// ([M][K] plain bytes) into that kernel's layout in caller scratch (prescaled even planes, or PoT table order;
+// chunk-major, ChunkMajorDst) and leaves the token sums.  One CTA per token row.
+__global__ void __launch_bounds__(128)
+relayout_act_kernel(const int8_t* __restrict__ q_a, int M, int K, int int4_weights, int q_chunk_bytes, int q_pot_lut,
+                    int8_t* __restrict__ q_out, int* __restrict__ sumq) {
+    __shared__ int red[4];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int m = blockIdx.x;
+    const ChunkMajorDst dst{q_out, m, M, K, q_chunk_bytes, q_pot_lut};
+    const uint4* src = reinterpret_cast<const uint4*>(q_a + static_cast<size_t>(m) * K);
+    int total = 0;
+    for (int q = threadIdx.x; q < K / 16; q += blockDim.x) {
+        uint4 v = src[q];
+        total = __dp4a(static_cast<int>(v.x), 0x01010101, __dp4a(static_cast<int>(v.y), 0x01010101, total));
+        total = __dp4a(static_cast<int>(v.z), 0x01010101, __dp4a(static_cast<int>(v.w), 0x01010101, total));
+        if (!q_pot_lut) {  // bytes of the even words times 4 (INT4 weights: 16); |q| <= 8, so the products fit a byte
+            if (int4_weights) v.x = (v.x << 4) & 0xf0f0f0f0u, v.z = (v.z << 4) & 0xf0f0f0f0u;
+            else v.x = (v.x << 2) & 0xfcfcfcfcu, v.z = (v.z << 2) & 0xfcfcfcfcu;
+        }
+        dst.store(q, v);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = total;
+    __syncthreads();
+    if (threadIdx.x == 0) sumq[m] = red[0] + red[1] + red[2] + red[3];
+}
+
 // ------------------------------------------------------------------------------------------------
 // grouped product
 // ------------------------------------------------------------------------------------------------
@@ -188,6 +218,8 @@ struct GroupParams {
     int count;                        // problems in the slice (<= kGroupSlice)
     int item_first, item_end;         // work items of the slice
     int M, y_bf16, stages;
+    int use_single;                   // the list is the one problem below (a per-call product: no plan in memory)
+    GroupProblemDev single;
 };
 
 // CTAs per SM the kernel is compiled and launched for.  Nine warps per CTA and registers handed out
@@ -463,7 +495,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
         *fail = 0;
     }
     for (int i = tid; i < gp.count; i += THREADS) {
-        const GroupProblemDev& P = gp.problems[i];
+        const GroupProblemDev& P = gp.use_single ? gp.single : gp.problems[i];
         SmemProblem e;
         e.packed = reinterpret_cast<const unsigned char*>(P.packed);
         e.q_a = P.q_a, e.s_n = P.s_n, e.s_a = P.s_a, e.Y = P.Y, e.acc_debug = P.acc_debug;

@@ -362,11 +362,17 @@ int run_prefill_fused(const uint32_t* packed, const float* s_n, int lv, const in
     }
 }
 
+// Scratch of QIFT_ROUTE_DECODE_ROWS: the re-laid-out activations and the token sums.
+inline size_t decode_rows_scratch(int M, int K) { return ((static_cast<size_t>(M) * K + 255) & ~static_cast<size_t>(255)) + 64; }
+inline bool decode_rows_supports(int lv, int M, int N, int K) { return M >= 2 && M <= 16 && decode_supports(lv, M, N, K); }
+int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
+                    void* Y, int y_bf16, int32_t* acc_debug, void* workspace, cudaStream_t st);
+
 int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
                 void* Y, int y_dtype, int32_t* acc_debug, void* workspace, size_t workspace_bytes, int route, void* stream) {
     if (!packed || !s_n || !q_a || !s_a || !Y || M <= 0 || N <= 0 || K <= 0 || !valid_levels(lv)) return QIFT_ERR_INVALID_ARG;
     if (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16) return QIFT_ERR_INVALID_ARG;
-    if (route < QIFT_ROUTE_AUTO || route > QIFT_ROUTE_PREFILL_FUSED_PAIR) return QIFT_ERR_INVALID_ARG;
+    if (route < QIFT_ROUTE_AUTO || route > QIFT_ROUTE_DECODE_ROWS) return QIFT_ERR_INVALID_ARG;
     if (K % codes_per_word(lv) != 0 || K % 4 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(packed) || !aligned16(s_n) || !aligned16(q_a) || !aligned16(s_a) || !aligned16(Y) ||
         (acc_debug && !aligned16(acc_debug)))
@@ -374,8 +380,24 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int y_bf16 = (y_dtype == QIFT_BF16);
     if (route == QIFT_ROUTE_AUTO) {
-        if (M <= 16) route = decode_supports(lv, M, N, K) ? QIFT_ROUTE_DECODE : QIFT_ROUTE_GENERIC;
-        else route = (K % 16 != 0) ? QIFT_ROUTE_GENERIC : auto_prefill_route(M);
+        if (M <= 16) {
+            route = decode_supports(lv, M, N, K) ? QIFT_ROUTE_DECODE : QIFT_ROUTE_GENERIC;
+            // the row-split kernel when the caller brought its scratch (qift_workspace_bytes asks for it); with at most
+            // 8 token rows and a small matrix its second launch costs more than it saves (4096 x 4096 at 4 rows: 5.5
+            // against 5.2 us; 14336 x 4096: 6.3 against 9.9 us)
+            const bool pays = M > 8 || static_cast<long long>(N) * K >= (1ll << 25);
+            if (pays && decode_rows_supports(lv, M, N, K) && workspace && workspace_bytes >= decode_rows_scratch(M, K) &&
+                (reinterpret_cast<uintptr_t>(workspace) & 255u) == 0)
+                route = QIFT_ROUTE_DECODE_ROWS;
+        } else {
+            route = (K % 16 != 0) ? QIFT_ROUTE_GENERIC : auto_prefill_route(M);
+        }
+    }
+    if (route == QIFT_ROUTE_DECODE_ROWS) {
+        if (!decode_rows_supports(lv, M, N, K)) return QIFT_ERR_UNSUPPORTED_SHAPE;
+        if (!workspace || workspace_bytes < decode_rows_scratch(M, K)) return QIFT_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(workspace) & 255u) return QIFT_ERR_ALIGNMENT;
+        return run_decode_rows(packed, s_n, lv, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, workspace, st);
     }
     if (route == QIFT_ROUTE_DECODE) {
         if (!decode_supports(lv, M, N, K)) return QIFT_ERR_UNSUPPORTED_SHAPE;
@@ -430,8 +452,9 @@ size_t qift_packed_bytes(int N, int K, int levels) {
 size_t qift_workspace_bytes_route(int M, int N, int K, int levels, int route) {
     if (M <= 0 || N <= 0 || K <= 0 || !valid_levels(levels)) return 0;
     if (route == QIFT_ROUTE_AUTO)
-        route = (M <= 16) ? QIFT_ROUTE_DECODE : auto_prefill_route(M);
+        route = (M <= 16) ? (decode_rows_supports(levels, M, N, K) ? QIFT_ROUTE_DECODE_ROWS : QIFT_ROUTE_DECODE) : auto_prefill_route(M);
     size_t b = 0;
+    if (route == QIFT_ROUTE_DECODE_ROWS) b = decode_rows_scratch(M, K);
     if (route == QIFT_ROUTE_PREFILL || route == QIFT_ROUTE_PREFILL_FUSED_PAIR) b = static_cast<size_t>(M) * 4;
     if (route == QIFT_ROUTE_PREFILL_SCRATCH || route == QIFT_ROUTE_PREFILL_PAIR) b = static_cast<size_t>(N) * K;
     return (b + 1023) & ~static_cast<size_t>(1023);
@@ -709,7 +732,7 @@ int launch_grouped(const GroupHeader* h, const GroupProblemDev* host, const Grou
 // From this many token rows on: 128- or 256-row items split by rows over the warps, one CTA per SM.
 template <int LV, int NT, int RT, int CWARPS>
 int launch_grouped_wide(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
-                        cudaStream_t st) {
+                        cudaStream_t st, bool single = false) {
     auto kernel = linear_grouped_wide_kernel<LV, NT, RT, CWARPS>;
     const size_t stage = wide_stage_bytes(LV, h->M, RT * CWARPS) + 16;
     for (int first = 0; first < h->count; first += kGroupSlice) {
@@ -724,7 +747,8 @@ int launch_grouped_wide(const GroupHeader* h, const GroupProblemDev* host, const
         if (e != cudaSuccess) return cuda_status(e);
         int grid = sm_count();
         if (grid > item_end - item_first) grid = item_end - item_first;
-        GroupParams gp{dev + first, sumq, first, count, item_first, item_end, h->M, h->y_bf16, stages};
+        GroupParams gp{dev + first, sumq, first, count, item_first, item_end, h->M, h->y_bf16, stages, 0, {}};
+        if (single) gp.use_single = 1, gp.single = host[0];
         const int rc = cuda_status(launch_pdl(kernel, dim3(grid), dim3((CWARPS + 1) * 32), smem, st, gp));
         if (rc != QIFT_OK) return rc;
     }
@@ -743,6 +767,40 @@ int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const Gr
     return launch_grouped<LV, 1, 2, false>(h, host, dev, sumq, st);
 }
 }  // namespace
+
+namespace qift {
+namespace {
+int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
+                    void* Y, int y_bf16, int32_t* acc_debug, void* workspace, cudaStream_t st) {
+    int8_t* q_out = static_cast<int8_t*>(workspace);
+    int* sumq = reinterpret_cast<int*>(q_out + ((static_cast<size_t>(M) * K + 255) & ~static_cast<size_t>(255)));
+    GroupHeader h{};
+    h.magic = kGroupMagic, h.count = 1, h.M = M, h.levels = lv, h.y_bf16 = y_bf16, h.rows_per_item = kWideRows;
+    h.total_items = (N + kWideRows - 1) / kWideRows;
+    h.q_pot_lut = (lv == QIFT_LEVELS_POT && M > 8) ? 1 : 0;
+    h.q_chunk_bytes = wide_chunk_words(kDecWarps, M > 8 ? 2 : 1) * codes_per_word(lv);
+    GroupProblemDev rec{};
+    rec.X = nullptr, rec.packed = packed, rec.s_n = s_n, rec.q_a = q_out, rec.s_a = const_cast<float*>(s_a), rec.Y = Y;
+    rec.acc_debug = acc_debug, rec.N = N, rec.K = K, rec.had_block = 0, rec.item_begin = 0, rec.inv_sqrt_b = 1.0f, rec.quant_src = 0;
+    int rc = cuda_status(launch_pdl(relayout_act_kernel, dim3(M), dim3(128), 0, st, q_a, M, K, lv == QIFT_LEVELS_INT4 ? 1 : 0,
+                                    h.q_chunk_bytes, h.q_pot_lut, q_out, sumq));
+    if (rc != QIFT_OK) return rc;
+    const GroupProblemDev* none = nullptr;
+#define QIFT_ROWS_CASE(LV)                                                                                          \
+    case LV:                                                                                                        \
+        return M > 8 ? launch_grouped_wide<LV, 2, 1, 8>(&h, &rec, none, sumq, st, true)                             \
+                     : launch_grouped_wide<LV, 1, 1, 8>(&h, &rec, none, sumq, st, true);
+    switch (lv) {
+        QIFT_ROWS_CASE(QIFT_LEVELS_MNZ)
+        QIFT_ROWS_CASE(QIFT_LEVELS_POT)
+        QIFT_ROWS_CASE(QIFT_LEVELS_SYM)
+        default:
+            QIFT_ROWS_CASE(QIFT_LEVELS_INT4)
+    }
+#undef QIFT_ROWS_CASE
+}
+}  // namespace
+}  // namespace qift
 
 extern "C" {
 

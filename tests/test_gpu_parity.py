@@ -188,13 +188,16 @@ def run_route(p_ref, s_n, lv, q_a, s_a, route, bf16):
 
 
 @pytest.mark.parametrize("name", list(LEVELS))
-@pytest.mark.parametrize("route", [qift.ROUTE_GENERIC, qift.ROUTE_DECODE])
+@pytest.mark.parametrize("route", [qift.ROUTE_GENERIC, qift.ROUTE_DECODE, qift.ROUTE_DECODE_ROWS])
 @pytest.mark.parametrize("M,N,K", [(1, 256, 256), (1, 40, 512), (3, 100, 2304), (8, 64, 4096), (9, 48, 1024),
-                                   (16, 130, 2560), (5, 16, 11008), (2, 2400, 256), (2, 21, 48)])
+                                   (16, 130, 2560), (5, 16, 11008), (2, 2400, 256), (2, 21, 48), (16, 4100, 512),
+                                   (12, 300, 14336)])
 def test_decode_routes(name, route, M, N, K):
     lv = LEVELS[name][0]
-    if route == qift.ROUTE_DECODE and K % 256:
-        pytest.skip("the decode route needs whole 16-word slices")
+    if route != qift.ROUTE_GENERIC and K % 256:
+        pytest.skip("the decode routes need whole 16-word slices")
+    if route == qift.ROUTE_DECODE_ROWS and M == 1:
+        pytest.skip("the row-split route starts at two token rows")
     p_ref, s_n, codes, q_a, s_a = make_problem(lv, M, N, K, seed=50 + M)
     for bf16 in (False, True):
         y_ref, acc_ref = oracle.linear(codes, lv, s_n, q_a, s_a, bf16=bf16)

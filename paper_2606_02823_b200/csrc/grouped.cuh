@@ -1,5 +1,5 @@
 // Grouped decode path: ONE persistent launch serves a whole list of independent layer problems
-// (all of one level set and one token count M <= 16), e.g. every linear module of a decode step.
+// (all of one level set and one token count M <= 32), e.g. every linear module of a decode step.
 //
 // A single W2 matrix is 1-15 MB, i.e. 0.15-2 us of HBM time: no per-matrix launch can reach a
 // bandwidth steady state.  Here the work list (problem, 16*RT-row block) is dealt round-robin to a
@@ -52,6 +52,7 @@ struct GroupProblemDev {
 };
 static_assert(sizeof(GroupProblemDev) == 96, "problem record is 96 bytes");
 
+constexpr int kGroupMaxM = 32;     // token rows of a plan; also the row length of the token-sum table
 constexpr uint32_t kGroupMagic = 0x51494654u;
 
 // ------------------------------------------------------------------------------------------------
@@ -103,7 +104,7 @@ quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* _
     if (threadIdx.x == 0) {
         int t = 0;
         for (int w = 0; w < kRowThreads / 32; ++w) t += redi[w];
-        sumq[p * 16 + m] = t;
+        sumq[p * kGroupMaxM + m] = t;
     }
 }
 
@@ -213,7 +214,7 @@ __host__ __device__ inline size_t grouped_smem_bytes(int lv, int rt, int M, int 
 
 struct GroupParams {
     const GroupProblemDev* problems;  // first problem of this launch's slice
-    const int* sumq;                  // [plan count][16]
+    const int* sumq;                  // [plan count][kGroupMaxM]
     int first_index;                  // plan index of problems[0]
     int count;                        // problems in the slice (<= kGroupSlice)
     int item_first, item_end;         // work items of the slice
@@ -349,7 +350,7 @@ linear_grouped_kernel(const GroupParams gp) {
         if (e_on) {
             e_sn = __ldg(P->s_n + e_n);
             e_sa = P->s_a[e_m];
-            e_sq = gp.sumq[P->index * 16 + e_m];
+            e_sq = gp.sumq[P->index * kGroupMaxM + e_m];
         }
 
         for (;;) {
@@ -448,10 +449,11 @@ constexpr int kWideRows = 16 * kDecWarps;        // 128 rows per item with one t
 // sixteen warps (twice the warps to hide the latencies of the load -> logic -> product chains) or as two tiles per
 // warp (the activation registers of a slice feed both tiles); their stages are a quarter tile of K (32 words) so
 // that as many stages fit as with 128 rows.
-__host__ __device__ constexpr int wide_chunk_words(int tiles, int nt) { return tiles > 8 ? 64 : 128; }
+__host__ __device__ constexpr int wide_chunk_words(int tiles, int nt) { return (tiles > 8 || nt > 2) ? 64 : 128; }
+__host__ __device__ constexpr int wide_token_tiles(int M) { return M > 16 ? 4 : M > 8 ? 2 : 1; }
 
 __host__ __device__ inline size_t wide_stage_bytes(int lv, int M, int tiles) {
-    const int cw = wide_chunk_words(tiles, M > 8 ? 2 : 1);
+    const int cw = wide_chunk_words(tiles, wide_token_tiles(M));
     return static_cast<size_t>(tiles) * (cw * 64) + static_cast<size_t>(M) * (cw * codes_per_word(lv));
 }
 __host__ __device__ inline size_t wide_smem_bytes(int lv, int M, int tiles, int stages, int count) {
@@ -468,7 +470,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     // PoT with two token tiles: levels by table lookup (pot_lut_operands) instead of code bit planes -- half the
     // product instructions for more logic per word, which pays once the products are the bottleneck (measured on 16
     // LLaMA-2-7B layers: 261 against 295 us at 16 rows, but 197 against 189 us at 8).
-    constexpr bool POT_LUT = (LV == QIFT_LEVELS_POT) && NT == 2;
+    constexpr bool POT_LUT = (LV == QIFT_LEVELS_POT) && NT >= 2;
     constexpr int NACC = POT_LUT ? 1 : T::NACC;
     constexpr int TILE_STAGE = CW * 64;          // bytes of one tile in a stage: CW words x 16 rows, contiguous in the packed order
     constexpr int CB = CW * T::PER;              // bytes of one token's activations in a full chunk
@@ -601,7 +603,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 const int tok = min(nt * 8 + 2 * cq + j, M - 1);
-                e_sq[nt][j] = gp.sumq[P->index * 16 + tok];
+                e_sq[nt][j] = gp.sumq[P->index * kGroupMaxM + tok];
                 e_sa[nt][j] = P->s_a[tok];
             }
 #pragma unroll

@@ -363,8 +363,8 @@ int run_prefill_fused(const uint32_t* packed, const float* s_n, int lv, const in
 }
 
 // Scratch of QIFT_ROUTE_DECODE_ROWS: the re-laid-out activations and the token sums.
-inline size_t decode_rows_scratch(int M, int K) { return ((static_cast<size_t>(M) * K + 255) & ~static_cast<size_t>(255)) + 64; }
-inline bool decode_rows_supports(int lv, int M, int N, int K) { return M >= 2 && M <= 16 && decode_supports(lv, M, N, K); }
+inline size_t decode_rows_scratch(int M, int K) { return ((static_cast<size_t>(M) * K + 255) & ~static_cast<size_t>(255)) + kGroupMaxM * 4; }
+inline bool decode_rows_supports(int lv, int M, int N, int K) { return M >= 2 && M <= kGroupMaxM && decode_supports(lv, M > 16 ? 16 : M, N, K); }
 int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
                     void* Y, int y_bf16, int32_t* acc_debug, void* workspace, cudaStream_t st);
 
@@ -391,6 +391,10 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
                 route = QIFT_ROUTE_DECODE_ROWS;
         } else {
             route = (K % 16 != 0) ? QIFT_ROUTE_GENERIC : auto_prefill_route(M);
+            // 17..32 token rows: still the row-split kernel (four token tiles) when its scratch was passed
+            if (decode_rows_supports(lv, M, N, K) && workspace && workspace_bytes >= decode_rows_scratch(M, K) &&
+                (reinterpret_cast<uintptr_t>(workspace) & 255u) == 0)
+                route = QIFT_ROUTE_DECODE_ROWS;
         }
     }
     if (route == QIFT_ROUTE_DECODE_ROWS) {
@@ -451,11 +455,13 @@ size_t qift_packed_bytes(int N, int K, int levels) {
 
 size_t qift_workspace_bytes_route(int M, int N, int K, int levels, int route) {
     if (M <= 0 || N <= 0 || K <= 0 || !valid_levels(levels)) return 0;
-    if (route == QIFT_ROUTE_AUTO)
-        route = (M <= 16) ? (decode_rows_supports(levels, M, N, K) ? QIFT_ROUTE_DECODE_ROWS : QIFT_ROUTE_DECODE) : auto_prefill_route(M);
     size_t b = 0;
+    if (route == QIFT_ROUTE_AUTO) {
+        route = (M <= 16) ? QIFT_ROUTE_DECODE : auto_prefill_route(M);
+        if (decode_rows_supports(levels, M, N, K)) b = decode_rows_scratch(M, K);  // enough for the fallback route as well
+    }
     if (route == QIFT_ROUTE_DECODE_ROWS) b = decode_rows_scratch(M, K);
-    if (route == QIFT_ROUTE_PREFILL || route == QIFT_ROUTE_PREFILL_FUSED_PAIR) b = static_cast<size_t>(M) * 4;
+    if ((route == QIFT_ROUTE_PREFILL || route == QIFT_ROUTE_PREFILL_FUSED_PAIR) && b < static_cast<size_t>(M) * 4) b = static_cast<size_t>(M) * 4;
     if (route == QIFT_ROUTE_PREFILL_SCRATCH || route == QIFT_ROUTE_PREFILL_PAIR) b = static_cast<size_t>(N) * K;
     return (b + 1023) & ~static_cast<size_t>(1023);
 }
@@ -629,7 +635,7 @@ int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_blo
 // ------------------------------------------------------------------------------------------- grouped
 size_t qift_group_plan_bytes(int count) {
     if (count <= 0) return 0;
-    return sizeof(GroupHeader) + static_cast<size_t>(count) * (sizeof(GroupProblemDev) + 16 * sizeof(int));
+    return sizeof(GroupHeader) + static_cast<size_t>(count) * (sizeof(GroupProblemDev) + kGroupMaxM * sizeof(int));
 }
 
 int qift_group_plan(const qift_group_problem* problems, int count, int M, int levels, int x_dtype, int y_dtype, float clip_ratio,
@@ -638,13 +644,13 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     if ((x_dtype != QIFT_F32 && x_dtype != QIFT_BF16) || (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16))
         return QIFT_ERR_INVALID_ARG;
     if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return QIFT_ERR_INVALID_ARG;
-    if (M > 16) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (M > kGroupMaxM) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (plan_bytes < qift_group_plan_bytes(count)) return QIFT_ERR_WORKSPACE;
     if (!aligned16(plan_dev) || !aligned16(plan_host)) return QIFT_ERR_ALIGNMENT;
     // Rows per work item, which also selects the kernel (dispatch_grouped): 64 / 32 for the K-split kernel, 128 for the
     // row-split kernel, 256 (two row tiles per warp, with two token tiles) when that still leaves two items per SM.
     int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : (M == 1) ? 64 : 32;
-    if (rows_per_item == kWideRows && M > 8 && levels != QIFT_LEVELS_POT) {  // PoT measured slower with two tiles
+    if (rows_per_item == kWideRows && M > 8 && M <= 16 && levels != QIFT_LEVELS_POT) {  // PoT measured slower with two tiles
         long long items256 = 0;
         for (int i = 0; i < count; ++i) items256 += (problems[i].N + 2 * kWideRows - 1) / (2 * kWideRows);
         if (items256 >= 2ll * sm_count()) rows_per_item = 2 * kWideRows;
@@ -655,7 +661,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     for (int i = 0; i < count; ++i) {
         const qift_group_problem& q = problems[i];
         if (!q.X || !q.packed || !q.s_n || !q.q_a || !q.s_a || !q.Y || q.N <= 0 || q.K <= 0) return QIFT_ERR_INVALID_ARG;
-        if (!decode_supports(levels, M, q.N, q.K)) return QIFT_ERR_UNSUPPORTED_SHAPE;
+        if (!decode_supports(levels, M > 16 ? 16 : M, q.N, q.K)) return QIFT_ERR_UNSUPPORTED_SHAPE;
         const int rs = check_rotation_shape(q.K, q.had_block, true);
         if (rs != QIFT_OK) return rs;
         if (!aligned16(q.X) || !aligned16(q.packed) || !aligned16(q.s_n) || !aligned16(q.q_a) || !aligned16(q.s_a) ||
@@ -684,7 +690,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     h->any_kron = any_kron;
     // the row-split kernel stages one K-chunk of all tokens per copy: its q_a is chunk-major (ChunkMajorDst)
     h->q_pot_lut = (rows_per_item >= kWideRows && levels == QIFT_LEVELS_POT && M > 8) ? 1 : 0;  // the kernel's POT_LUT
-    h->q_chunk_bytes = (rows_per_item >= kWideRows) ? wide_chunk_words(rows_per_item / 16, M > 8 ? 2 : 1) * codes_per_word(levels) : 0;
+    h->q_chunk_bytes = (rows_per_item >= kWideRows) ? wide_chunk_words(rows_per_item / 16, wide_token_tiles(M)) * codes_per_word(levels) : 0;
     return cuda_status(cudaMemcpyAsync(plan_dev, plan_host, sizeof(GroupHeader) + static_cast<size_t>(count) * sizeof(GroupProblemDev),
                                        cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));
 }
@@ -761,6 +767,7 @@ int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const Gr
     // (256-row items -- two row tiles per warp, or sixteen consumer warps -- were measured slower: 3.2 / 3.2 against
     // 3.9 TB/s at 16 rows.)
     if (h->rows_per_item == 2 * kWideRows) return launch_grouped_wide<LV, 2, 2, 8>(h, host, dev, sumq, st);
+    if (h->rows_per_item == kWideRows && h->M > 16) return launch_grouped_wide<LV, 4, 1, 8>(h, host, dev, sumq, st);
     if (h->rows_per_item == kWideRows)
         return h->M > 8 ? launch_grouped_wide<LV, 2, 1, 8>(h, host, dev, sumq, st) : launch_grouped_wide<LV, 1, 1, 8>(h, host, dev, sumq, st);
     if (h->M == 1) return launch_grouped<LV, 1, 4, true>(h, host, dev, sumq, st);
@@ -778,7 +785,7 @@ int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8
     h.magic = kGroupMagic, h.count = 1, h.M = M, h.levels = lv, h.y_bf16 = y_bf16, h.rows_per_item = kWideRows;
     h.total_items = (N + kWideRows - 1) / kWideRows;
     h.q_pot_lut = (lv == QIFT_LEVELS_POT && M > 8) ? 1 : 0;
-    h.q_chunk_bytes = wide_chunk_words(kDecWarps, M > 8 ? 2 : 1) * codes_per_word(lv);
+    h.q_chunk_bytes = wide_chunk_words(kDecWarps, wide_token_tiles(M)) * codes_per_word(lv);
     GroupProblemDev rec{};
     rec.X = nullptr, rec.packed = packed, rec.s_n = s_n, rec.q_a = q_out, rec.s_a = const_cast<float*>(s_a), rec.Y = Y;
     rec.acc_debug = acc_debug, rec.N = N, rec.K = K, rec.had_block = 0, rec.item_begin = 0, rec.inv_sqrt_b = 1.0f, rec.quant_src = 0;
@@ -788,8 +795,9 @@ int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8
     const GroupProblemDev* none = nullptr;
 #define QIFT_ROWS_CASE(LV)                                                                                          \
     case LV:                                                                                                        \
-        return M > 8 ? launch_grouped_wide<LV, 2, 1, 8>(&h, &rec, none, sumq, st, true)                             \
-                     : launch_grouped_wide<LV, 1, 1, 8>(&h, &rec, none, sumq, st, true);
+        return M > 16 ? launch_grouped_wide<LV, 4, 1, 8>(&h, &rec, none, sumq, st, true)                            \
+               : M > 8 ? launch_grouped_wide<LV, 2, 1, 8>(&h, &rec, none, sumq, st, true)                           \
+                       : launch_grouped_wide<LV, 1, 1, 8>(&h, &rec, none, sumq, st, true);
     switch (lv) {
         QIFT_ROWS_CASE(QIFT_LEVELS_MNZ)
         QIFT_ROWS_CASE(QIFT_LEVELS_POT)

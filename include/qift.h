@@ -70,9 +70,9 @@ typedef enum {
                                       scratch N*K bytes                                            */
     QIFT_ROUTE_PREFILL_FUSED_PAIR = 6, /* CTA pairs with the codes expanded in the kernel (each CTA
                                       expands half of the tile's channels); scratch 4*M            */
-    QIFT_ROUTE_DECODE_ROWS = 7 /* 2 <= M <= 32: the activations re-laid out into the scratch, then the
+    QIFT_ROUTE_DECODE_ROWS = 7 /* 2 <= M <= 64: the activations re-laid out into the scratch, then the
                                   row-split kernel of the grouped path (128-row items, no reduction);
-                                  scratch M*K + 128 bytes                                         */
+                                  scratch M*K + 256 bytes                                         */
 } qift_route;
 
 const char* qift_status_string(int status);
@@ -139,7 +139,7 @@ int qift_quantize_act(const void* X, int x_dtype, int M, int K, int had_block, f
  *   Y         out [M,N] fp32 or bf16 (round to nearest even): ((float)acc * s_a[m]) * s_n[n]
  *   acc_debug out int32 [M,N] accumulators, or NULL
  *   workspace     >= qift_workspace_bytes(M,N,K,levels) bytes, 256-byte aligned; may be NULL when 0
- * M <= 16 takes a decode route (the row-split one up to 32 rows when its scratch is passed), 16 < M <= 512 the
+ * M <= 16 takes a decode route (the row-split one up to 64 rows when its scratch is passed), 16 < M <= 512 the
  * fused prefill routes, larger M the CTA-pair scratch route. */
 int qift_w2a4_linear(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a,
                      const float* s_a, int M, int N, int K, void* Y, int y_dtype, int32_t* acc_debug,
@@ -173,7 +173,7 @@ int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_blo
                       int y_dtype, void* scratch, size_t scratch_bytes, void* stream);
 
 /* ---- Grouped decode path -----------------------------------------------------------------------
- * One persistent launch serves a list of independent layer problems that share M (<= 32 token rows),
+ * One persistent launch serves a list of independent layer problems that share M (<= 64 token rows),
  * the level set, the dtypes and the clip ratio -- e.g. all linear modules of one decode step.  A W2
  * matrix is only 1-15 MB, far too little for one launch to reach an HBM steady state; the grouped
  * kernel streams the whole list back to back.  (No counterpart in the paper: it describes no kernels.)

@@ -234,6 +234,37 @@ __device__ __forceinline__ void mma_tile_step_pot_lut(int (&acc)[NT][1][4], cons
     }
 }
 
+// One packed word of rows g (lo) and g+8 (hi) against the NPL activation words that belong to it, grouped-path
+// layouts (prescaled even planes, or PoT table order with POT_LUT).  The operand logic does not depend on the token
+// tile: called in a loop over token tiles it is computed once.
+template <int LV, bool POT_LUT, int NACC>
+__device__ __forceinline__ void mma_word(int (&acc)[NACC][4], uint32_t lo, uint32_t hi, const uint32_t (&q)[DecodeTraits<LV>::NPL]) {
+    if constexpr (LV == QIFT_LEVELS_INT4) {
+        mma_u8s8(acc[0], (lo & 0x0f0f0f0fu) ^ 0x08080808u, (hi & 0x0f0f0f0fu) ^ 0x08080808u, (lo & 0xf0f0f0f0u) ^ 0x80808080u,
+                 (hi & 0xf0f0f0f0u) ^ 0x80808080u, q[0], q[1]);
+    } else if constexpr (POT_LUT) {
+        uint32_t al[4], ah[4];
+        pot_lut_operands(lo, al);
+        pot_lut_operands(hi, ah);
+        mma_s8s8(acc[0], al[0], ah[0], al[1], ah[1], q[0], q[1]);
+        mma_s8s8(acc[0], al[2], ah[2], al[3], ah[3], q[2], q[3]);
+    } else if constexpr (LV == QIFT_LEVELS_POT) {
+#pragma unroll
+        for (int tt = 0; tt < 4; tt += 2)
+#pragma unroll
+            for (int bit = 1; bit >= 0; --bit) {
+                const uint32_t m0 = (bit ? 0x02020202u : 0x01010101u) << (2 * tt), m1 = m0 << 2;
+                mma_u8s8(acc[(bit ? 0 : 2) + tt / 2], lo & m0, hi & m0, lo & m1, hi & m1, q[tt], q[tt + 1]);
+            }
+    } else {
+#pragma unroll
+        for (int tt = 0; tt < 4; tt += 2) {
+            const uint32_t m0 = 0x03030303u << (2 * tt), m1 = m0 << 2;
+            mma_u8s8(acc[tt / 2], lo & m0, hi & m0, lo & m1, hi & m1, q[tt], q[tt + 1]);
+        }
+    }
+}
+
 struct DecodeParams {
     const uint32_t* packed;
     const float* s_n;

@@ -1,5 +1,5 @@
 // Grouped decode path: ONE persistent launch serves a whole list of independent layer problems
-// (all of one level set and one token count M <= 32), e.g. every linear module of a decode step.
+// (all of one level set and one token count M <= 64), e.g. every linear module of a decode step.
 //
 // A single W2 matrix is 1-15 MB, i.e. 0.15-2 us of HBM time: no per-matrix launch can reach a
 // bandwidth steady state.  Here the work list (problem, 16*RT-row block) is dealt round-robin to a
@@ -52,7 +52,7 @@ struct GroupProblemDev {
 };
 static_assert(sizeof(GroupProblemDev) == 96, "problem record is 96 bytes");
 
-constexpr int kGroupMaxM = 32;     // token rows of a plan; also the row length of the token-sum table
+constexpr int kGroupMaxM = 64;     // token rows of a plan; also the row length of the token-sum table
 constexpr uint32_t kGroupMagic = 0x51494654u;
 
 // ------------------------------------------------------------------------------------------------
@@ -450,7 +450,7 @@ constexpr int kWideRows = 16 * kDecWarps;        // 128 rows per item with one t
 // warp (the activation registers of a slice feed both tiles); their stages are a quarter tile of K (32 words) so
 // that as many stages fit as with 128 rows.
 __host__ __device__ constexpr int wide_chunk_words(int tiles, int nt) { return (tiles > 8 || nt > 2) ? 64 : 128; }
-__host__ __device__ constexpr int wide_token_tiles(int M) { return M > 16 ? 4 : M > 8 ? 2 : 1; }
+__host__ __device__ constexpr int wide_token_tiles(int M) { return M > 32 ? 8 : M > 16 ? 4 : M > 8 ? 2 : 1; }
 
 __host__ __device__ inline size_t wide_stage_bytes(int lv, int M, int tiles) {
     const int cw = wide_chunk_words(tiles, wide_token_tiles(M));
@@ -631,36 +631,65 @@ linear_grouped_wide_kernel(const GroupParams gp) {
 #pragma unroll
                     for (int i = 0; i < T::NPL; ++i) qa[nt][i] = qs + q_tok[nt] * (cw * T::PER) + q_piece[nt][i];
                 const uint32_t wa_base = ws + lane * 16;
+                // the lane's four words of rows g and g+8 of row tile r; lanes that visit their activation pieces in
+                // the order 2,3,0,1 take the words in that order too: by selects after a 128-bit load, or (PoT with one
+                // token tile, where the logic pipe is the limit) by two 64-bit loads, which cost a two-way bank
+                // conflict instead
+                auto load_words = [&](int r, int sl, uint4& wa, uint4& wb) {
+                    const uint32_t o = r * TILE_STAGE + sl * 1024;
+                    if constexpr (LV == QIFT_LEVELS_POT && NT == 1) {
+                        const uint32_t lo_a = wa_base + o + 4 * rot, hi_a = lo_a + 8 - 8 * rot;
+                        const uint2 a_lo = lds64(lo_a), a_hi = lds64(hi_a), b_lo = lds64(lo_a + 512), b_hi = lds64(hi_a + 512);
+                        wa = make_uint4(a_lo.x, a_lo.y, a_hi.x, a_hi.y);
+                        wb = make_uint4(b_lo.x, b_lo.y, b_hi.x, b_hi.y);
+                    } else {
+                        const uint4 ra = lds128(wa_base + o), rb = lds128(wa_base + o + 512);
+                        wa = rot ? make_uint4(ra.z, ra.w, ra.x, ra.y) : ra;
+                        wb = rot ? make_uint4(rb.z, rb.w, rb.x, rb.y) : rb;
+                    }
+                };
                 auto slice = [&](int sl, auto ks) {
-                    uint32_t qb[NT][4 * T::NPL];
+                    if constexpr (NT <= 2) {
+                        uint32_t qb[NT][4 * T::NPL];
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
+                        for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+                            for (int i = 0; i < T::NPL; ++i) {
+                                const uint4 v = lds128(qa[nt][i] + sl * (16 * T::PER));
+                                qb[nt][4 * i] = v.x, qb[nt][4 * i + 1] = v.y, qb[nt][4 * i + 2] = v.z, qb[nt][4 * i + 3] = v.w;
+                            }
+                        }
+#pragma unroll
+                        for (int r = 0; r < RT; ++r) {
+                            uint4 wa, wb;
+                            load_words(r, sl, wa, wb);
+                            if constexpr (POT_LUT) mma_tile_step_pot_lut<NT>(acc[decltype(ks)::value][r], wa, wb, qb);
+                            else mma_tile_step<LV, NT, true>(acc[decltype(ks)::value][r], wa, wb, qb);
+                        }
+                    } else {
+                        // many token tiles: the activation words are fetched as they are used (all of them would not
+                        // fit the registers); piece i of a token tile serves 4 / NPL packed words
+                        static_assert(RT == 1, "one row tile per warp with more than two token tiles");
+                        uint4 wa, wb;
+                        load_words(0, sl, wa, wb);
+                        const uint32_t lo[4] = {wa.x, wa.y, wa.z, wa.w};
+                        const uint32_t hi[4] = {wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
                         for (int i = 0; i < T::NPL; ++i) {
-                            const uint4 v = lds128(qa[nt][i] + sl * (16 * T::PER));
-                            qb[nt][4 * i] = v.x, qb[nt][4 * i + 1] = v.y, qb[nt][4 * i + 2] = v.z, qb[nt][4 * i + 3] = v.w;
-                        }
-                    }
 #pragma unroll
-                    for (int r = 0; r < RT; ++r) {
-                        const uint32_t o = r * TILE_STAGE + sl * 1024;
-                        // the lane's four words of rows g and g+8; lanes that visit their activation pieces in
-                        // the order 2,3,0,1 take the words in that order too: by selects after a 128-bit load, or
-                        // (PoT with one token tile, where the logic pipe is the limit) by two 64-bit loads, which
-                        // cost a two-way bank conflict instead
-                        uint4 wa, wb;
-                        if constexpr (LV == QIFT_LEVELS_POT && NT == 1) {
-                            const uint32_t lo_a = wa_base + o + 4 * rot, hi_a = lo_a + 8 - 8 * rot;
-                            const uint2 a_lo = lds64(lo_a), a_hi = lds64(hi_a), b_lo = lds64(lo_a + 512), b_hi = lds64(hi_a + 512);
-                            wa = make_uint4(a_lo.x, a_lo.y, a_hi.x, a_hi.y);
-                            wb = make_uint4(b_lo.x, b_lo.y, b_hi.x, b_hi.y);
-                        } else {
-                            const uint4 ra = lds128(wa_base + o), rb = lds128(wa_base + o + 512);
-                            wa = rot ? make_uint4(ra.z, ra.w, ra.x, ra.y) : ra;
-                            wb = rot ? make_uint4(rb.z, rb.w, rb.x, rb.y) : rb;
+                            for (int nt = 0; nt < NT; ++nt) {
+                                const uint4 v = lds128(qa[nt][i] + sl * (16 * T::PER));
+                                const uint32_t q4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                                for (int j = 0; j < 4 / T::NPL; ++j) {   // the words this piece belongs to
+                                    const int word = i * (4 / T::NPL) + j;
+                                    uint32_t qw[T::NPL];
+#pragma unroll
+                                    for (int t = 0; t < T::NPL; ++t) qw[t] = q4[j * T::NPL + t];
+                                    mma_word<LV, POT_LUT, NACC>(acc[0][0][nt], lo[word], hi[word], qw);
+                                }
+                            }
                         }
-                        if constexpr (POT_LUT) mma_tile_step_pot_lut<NT>(acc[decltype(ks)::value][r], wa, wb, qb);
-                        else mma_tile_step<LV, NT, true>(acc[decltype(ks)::value][r], wa, wb, qb);
                     }
                 };
                 if (cw == CW) {

@@ -391,7 +391,7 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
                 route = QIFT_ROUTE_DECODE_ROWS;
         } else {
             route = (K % 16 != 0) ? QIFT_ROUTE_GENERIC : auto_prefill_route(M);
-            // 17..32 token rows: still the row-split kernel (four token tiles) when its scratch was passed
+            // 17..64 token rows: still the row-split kernel (four or eight token tiles) when its scratch was passed
             if (decode_rows_supports(lv, M, N, K) && workspace && workspace_bytes >= decode_rows_scratch(M, K) &&
                 (reinterpret_cast<uintptr_t>(workspace) & 255u) == 0)
                 route = QIFT_ROUTE_DECODE_ROWS;
@@ -767,6 +767,7 @@ int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const Gr
     // (256-row items -- two row tiles per warp, or sixteen consumer warps -- were measured slower: 3.2 / 3.2 against
     // 3.9 TB/s at 16 rows.)
     if (h->rows_per_item == 2 * kWideRows) return launch_grouped_wide<LV, 2, 2, 8>(h, host, dev, sumq, st);
+    if (h->rows_per_item == kWideRows && h->M > 32) return launch_grouped_wide<LV, 8, 1, 8>(h, host, dev, sumq, st);
     if (h->rows_per_item == kWideRows && h->M > 16) return launch_grouped_wide<LV, 4, 1, 8>(h, host, dev, sumq, st);
     if (h->rows_per_item == kWideRows)
         return h->M > 8 ? launch_grouped_wide<LV, 2, 1, 8>(h, host, dev, sumq, st) : launch_grouped_wide<LV, 1, 1, 8>(h, host, dev, sumq, st);
@@ -795,7 +796,8 @@ int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8
     const GroupProblemDev* none = nullptr;
 #define QIFT_ROWS_CASE(LV)                                                                                          \
     case LV:                                                                                                        \
-        return M > 16 ? launch_grouped_wide<LV, 4, 1, 8>(&h, &rec, none, sumq, st, true)                            \
+        return M > 32 ? launch_grouped_wide<LV, 8, 1, 8>(&h, &rec, none, sumq, st, true)                            \
+               : M > 16 ? launch_grouped_wide<LV, 4, 1, 8>(&h, &rec, none, sumq, st, true)                          \
                : M > 8 ? launch_grouped_wide<LV, 2, 1, 8>(&h, &rec, none, sumq, st, true)                           \
                        : launch_grouped_wide<LV, 1, 1, 8>(&h, &rec, none, sumq, st, true);
     switch (lv) {

@@ -36,12 +36,12 @@ def test_sizes(L):
     assert qift.qift_packed_bytes(0, 16, qift.MNZ) == 0
     assert qift.qift_workspace_bytes(1, 4096, 4096, qift.MNZ) == 0
     assert qift.qift_workspace_bytes(16, 4096, 4096, qift.POT) == 16 * 4096 + 1024     # re-laid-out activations + token sums, 1 KiB steps
-    assert qift.qift_workspace_bytes(32, 4096, 4096, qift.MNZ) == 32 * 4096 + 1024     # row-split route up to 32 rows
+    assert qift.qift_workspace_bytes(64, 4096, 4096, qift.MNZ) == 64 * 4096 + 1024     # row-split route up to 64 rows
     assert qift.qift_workspace_bytes(16, 4096, 4096, qift.POT, qift.ROUTE_DECODE) == 0
     assert qift.qift_workspace_bytes(3, 64, 48, qift.MNZ) == 0                         # K not in whole 16-word slices: generic route
     assert qift.qift_workspace_bytes(512, 4096, 4096, qift.MNZ) == 512 * 4            # per-token sums only
     assert qift.qift_workspace_bytes(2048, 4096, 4096, qift.MNZ) == 4096 * 4096       # int8 scratch
-    assert qift.qift_workspace_bytes(33, 3, 16, qift.SYM) == 1024                      # rounded up to 1 KiB
+    assert qift.qift_workspace_bytes(65, 3, 16, qift.SYM) == 1024                      # rounded up to 1 KiB
     assert qift.qift_workspace_bytes(2048, 4096, 4096, qift.MNZ, qift.ROUTE_PREFILL_SCRATCH) == 4096 * 4096
     assert qift.qift_workspace_bytes(8, 4096, 4096, qift.MNZ, qift.ROUTE_PREFILL_SCRATCH) == 4096 * 4096
     assert qift.qift_workspace_bytes(8, 4096, 4096, qift.MNZ, qift.ROUTE_GENERIC) == 0

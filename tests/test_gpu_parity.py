@@ -191,7 +191,7 @@ def run_route(p_ref, s_n, lv, q_a, s_a, route, bf16):
 @pytest.mark.parametrize("route", [qift.ROUTE_GENERIC, qift.ROUTE_DECODE, qift.ROUTE_DECODE_ROWS])
 @pytest.mark.parametrize("M,N,K", [(1, 256, 256), (1, 40, 512), (3, 100, 2304), (8, 64, 4096), (9, 48, 1024),
                                    (16, 130, 2560), (5, 16, 11008), (2, 2400, 256), (2, 21, 48), (16, 4100, 512),
-                                   (12, 300, 14336), (17, 200, 1024), (32, 1500, 512), (25, 140, 4096)])
+                                   (12, 300, 14336), (17, 200, 1024), (32, 1500, 512), (25, 140, 4096), (64, 300, 1024), (41, 130, 2560)])
 def test_decode_routes(name, route, M, N, K):
     lv = LEVELS[name][0]
     if route != qift.ROUTE_GENERIC and K % 256:
@@ -312,7 +312,7 @@ def test_whole_path_config1():
 
 # ---------------------------------------------------------------------------------- grouped path
 @pytest.mark.parametrize("name", list(LEVELS))
-@pytest.mark.parametrize("M", [1, 2, 5, 6, 8, 9, 13, 16, 17, 27, 32])
+@pytest.mark.parametrize("M", [1, 2, 5, 6, 8, 9, 13, 16, 17, 27, 32, 33, 50, 64])
 def test_grouped_forward(name, M):
     # a ragged list: different N (incl. not a multiple of the row block), different K (incl. a
     # partial last chunk), more items than CTAs
@@ -408,9 +408,9 @@ def test_grouped_rejects_bad_plans():
     with pytest.raises(qift.QiftError) as e:
         qift.qift_group_plan([(x, packed, s_n, 96)], qift.MNZ)          # had_block not a power of two
     assert e.value.status == qift.ERR_UNSUPPORTED_SHAPE
-    x33 = torch.zeros((33, 256), device="cuda")
+    x65 = torch.zeros((65, 256), device="cuda")
     with pytest.raises(qift.QiftError) as e:
-        qift.qift_group_plan([(x33, packed, s_n, 256)], qift.MNZ)       # M > 32
+        qift.qift_group_plan([(x65, packed, s_n, 256)], qift.MNZ)       # M > 64
     assert e.value.status == qift.ERR_UNSUPPORTED_SHAPE
     L = qift.lib()
     assert L.qift_group_forward(None, None, None) == qift.ERR_INVALID_ARG

@@ -440,7 +440,53 @@ def run_mixed_stack(torch, qift, L, device, gen, args):
                        "grouped API (4 launches per step)")
     if args.layers >= 16:
         out["l_sweep"] = [point(args.layers * l // 32, args.layers - args.layers * l // 32) for l in (4, 8, 12)]
+    out["prefill_m2048"] = mixed_prefill(torch, qift, L, device, gen, args, n4)
     return out
+
+
+def mixed_prefill(torch, qift, L, device, gen, args, n4):
+    """Config 5 at M = 2048: the same mixed stack (first layers W4A4, the rest W2A4 MNZ), every module as activation
+    quantizer + product through the per-call API (bf16 in, bf16 out; AUTO route = codes expanded into one shared int8
+    scratch, then the CTA-pair tcgen05 GEMM).  Distinct weights per layer; end-to-end linear-stack tokens per second."""
+    M = 2048
+    vp = ctypes.c_void_p
+    st = vp(torch.cuda.current_stream().cuda_stream)
+    mods = build_stack(torch, qift, synth.LLAMA2_7B, args.layers, M, lambda l: qift.INT4 if l < n4 else qift.MNZ, 5100,
+                       torch.bfloat16, torch.bfloat16, device, gen)
+    kmax = max(m.K for m in mods)
+    q_a = torch.empty((M, kmax), dtype=torch.int8, device=device)
+    s_a = torch.empty((M,), dtype=torch.float32, device=device)
+    ws_bytes = max(qift.qift_workspace_bytes(M, m.N, m.K, m.levels) for m in mods)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
+
+    def step():
+        for m in mods:
+            rc = L.qift_quantize_act(vp(m.x.data_ptr()), qift.BF16, M, m.K, m.B, CLIP, vp(q_a.data_ptr()), vp(s_a.data_ptr()), st)
+            assert rc == 0, rc
+            fn = L.qift_w4a4_linear if m.levels == qift.INT4 else None
+            if fn is not None:
+                rc = fn(vp(m.packed.data_ptr()), vp(m.s_n.data_ptr()), vp(q_a.data_ptr()), vp(s_a.data_ptr()), M, m.N, m.K,
+                        vp(m.y.data_ptr()), qift.BF16, None, vp(ws.data_ptr()), ws_bytes, st)
+            else:
+                rc = L.qift_w2a4_linear(vp(m.packed.data_ptr()), vp(m.s_n.data_ptr()), m.levels, vp(q_a.data_ptr()),
+                                        vp(s_a.data_ptr()), M, m.N, m.K, vp(m.y.data_ptr()), qift.BF16, None, vp(ws.data_ptr()),
+                                        ws_bytes, st)
+            assert rc == 0, rc
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(3):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / 3
+    ops = 2.0 * M * sum(m.N * m.K for m in mods)
+    return {"workload": f"config 5 at M = 2048: {n4} W4A4 + {args.layers - n4} W2A4 layers, LLaMA-2-7B shapes, per-call API with "
+                        "activation quantizer", "ms_per_step": round(ms, 3), "tokens_per_s": round(M / (ms * 1e-3), 1),
+            "tops": round(ops / (ms * 1e-3) / 1e12, 1), "launches_per_step": 3 * len(mods)}
 
 
 def run_batched_decode(torch, qift, L, device, gen, args):

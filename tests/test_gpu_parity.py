@@ -207,6 +207,33 @@ def test_decode_routes(name, route, M, N, K):
         check_outputs(y, acc, y_ref, acc_ref, bf16)
 
 
+@pytest.mark.parametrize("M", [1, 16, 40])
+def test_linear_in_a_cuda_graph(M):
+    # the per-call product captured once and replayed on new inputs: nothing in the launch may depend on host memory
+    # that is gone at replay (the row-split route passes its one problem record by value)
+    lv, N, K = qift.MNZ, 300, 1024
+    p_ref, s_n, codes, q_a, s_a = make_problem(lv, M, N, K, seed=90)
+    packed, sn, q, sa = dev(p_ref.view(np.int32)), dev(s_n), dev(q_a), dev(s_a)
+    out = torch.empty((M, N), device="cuda")
+    ws = torch.empty(max(256, qift.qift_workspace_bytes(M, N, K, lv)), dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        qift.qift_w2a4_linear(packed, sn, lv, q, sa, out=out, workspace=ws)      # warm-up: attribute calls happen here
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            qift.qift_w2a4_linear(packed, sn, lv, q, sa, out=out, workspace=ws)
+    for seed in (91, 92):
+        _, _, _, q_new, sa_new = make_problem(lv, M, N, K, seed=seed)
+        q.copy_(dev(q_new)), sa.copy_(dev(sa_new))
+        out.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        y_ref, _ = oracle.linear(codes, lv, s_n, q_new, sa_new)
+        assert np.array_equal(out.cpu().numpy(), y_ref)
+    assert_status_clean()
+
+
 @pytest.mark.parametrize("name", ["MNZ", "INT4"])
 def test_decode_extreme_values(name):
     # all codes at the top level against all activations at -8 / +7: the largest accumulators

@@ -80,14 +80,14 @@ struct ChunkMajorDst {
 template <bool BF16_IN, bool KRON = false>
 __global__ void __launch_bounds__(kRowThreads)
 quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* __restrict__ sumq, int M, float clip,
-                            int int4_weights, int q_chunk_bytes, int q_pot_lut) {
+                            int int4_weights, int q_chunk_bytes, int q_pot_lut, int use_single, const GroupProblemDev single) {
     extern __shared__ __align__(16) float row[];
     __shared__ float red[kRowThreads / 32 + 2];
     __shared__ int redi[kRowThreads / 32];
     pdl_launch_dependents();
     pdl_wait();
     const int p = blockIdx.x / M;
-    const GroupProblemDev P = problems[p];
+    const GroupProblemDev P = use_single ? single : problems[p];   // a per-call forward passes its one problem by value
     if (P.quant_src != p) return;  // an earlier problem quantizes this activation
     const size_t m = blockIdx.x % M;
     const int K = P.K, B = P.had_block;

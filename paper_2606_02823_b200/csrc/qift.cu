@@ -367,6 +367,8 @@ inline size_t decode_rows_scratch(int M, int K) { return ((static_cast<size_t>(M
 inline bool decode_rows_supports(int lv, int M, int N, int K) { return M >= 2 && M <= kGroupMaxM && decode_supports(lv, M > 16 ? 16 : M, N, K); }
 int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
                     void* Y, int y_bf16, int32_t* acc_debug, void* workspace, cudaStream_t st);
+int run_forward_rows(const void* X, int x_bf16, int M, int K, int had_block, float clip, const uint32_t* packed, const float* s_n,
+                     int lv, int N, void* Y, int y_bf16, int8_t* q_scratch, float* s_a, int* sumq, cudaStream_t st);
 
 int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
                 void* Y, int y_dtype, int32_t* acc_debug, void* workspace, size_t workspace_bytes, int route, void* stream) {
@@ -604,10 +606,17 @@ static int forward_impl(const void* X, bool host, int x_dtype, int M, int K, int
     }
     int8_t* q_a = reinterpret_cast<int8_t*>(base + L.q_off);
     float* s_a = reinterpret_cast<float*>(base + L.sa_off);
-    int rc = qift_quantize_act(x_dev, x_dtype, M, K, had_block, clip_ratio, q_a, s_a, stream);
-    if (rc != QIFT_OK) return rc;
-    rc = linear_impl(packed, s_n, levels, q_a, s_a, M, N, K, y_dev, y_dtype, nullptr, base + L.ws_off, L.total - L.ws_off,
-                     QIFT_ROUTE_AUTO, stream);
+    int rc;
+    if (decode_rows_supports(levels, M, N, K) && L.total - L.ws_off >= kGroupMaxM * sizeof(int)) {
+        // 2..64 token rows: the grouped path's quantizer writes the row-split kernel's activation layout directly
+        rc = run_forward_rows(x_dev, x_dtype == QIFT_BF16, M, K, had_block, clip_ratio, packed, s_n, levels, N, y_dev,
+                              y_dtype == QIFT_BF16, q_a, s_a, reinterpret_cast<int*>(base + L.ws_off), st);
+    } else {
+        rc = qift_quantize_act(x_dev, x_dtype, M, K, had_block, clip_ratio, q_a, s_a, stream);
+        if (rc != QIFT_OK) return rc;
+        rc = linear_impl(packed, s_n, levels, q_a, s_a, M, N, K, y_dev, y_dtype, nullptr, base + L.ws_off, L.total - L.ws_off,
+                         QIFT_ROUTE_AUTO, stream);
+    }
     if (rc != QIFT_OK) return rc;
     if (host) {
         cudaError_t e = cudaMemcpyAsync(Y, y_dev, static_cast<size_t>(M) * N * (y_dtype == QIFT_BF16 ? 2 : 4),
@@ -809,6 +818,43 @@ int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8
     }
 #undef QIFT_ROWS_CASE
 }
+
+int run_forward_rows(const void* X, int x_bf16, int M, int K, int had_block, float clip, const uint32_t* packed, const float* s_n,
+                     int lv, int N, void* Y, int y_bf16, int8_t* q_scratch, float* s_a, int* sumq, cudaStream_t st) {
+    GroupHeader h{};
+    h.magic = kGroupMagic, h.count = 1, h.M = M, h.levels = lv, h.y_bf16 = y_bf16, h.rows_per_item = kWideRows;
+    h.total_items = (N + kWideRows - 1) / kWideRows;
+    h.q_pot_lut = (lv == QIFT_LEVELS_POT && M > 8) ? 1 : 0;
+    h.q_chunk_bytes = wide_chunk_words(kDecWarps, wide_token_tiles(M)) * codes_per_word(lv);
+    GroupProblemDev rec{};
+    rec.X = X, rec.packed = packed, rec.s_n = s_n, rec.q_a = q_scratch, rec.s_a = s_a, rec.Y = Y, rec.acc_debug = nullptr;
+    rec.N = N, rec.K = K, rec.had_block = had_block, rec.item_begin = 0, rec.quant_src = 0;
+    rec.inv_sqrt_b = had_block > 1 ? inv_sqrt_block(had_block) : 1.0f;
+    const bool kron = had_block > 1 && !is_pow2(had_block);
+    auto qk = x_bf16 ? (kron ? quantize_act_grouped_kernel<true, true> : quantize_act_grouped_kernel<true, false>)
+                     : (kron ? quantize_act_grouped_kernel<false, true> : quantize_act_grouped_kernel<false, false>);
+    const size_t smem = padded_row_bytes(K);
+    cudaError_t e = allow_smem(qk, smem);
+    if (e != cudaSuccess) return cuda_status(e);
+    const GroupProblemDev* none = nullptr;
+    int rc = cuda_status(launch_pdl(qk, dim3(M), dim3(kRowThreads), smem, st, none, sumq, M, clip, lv == QIFT_LEVELS_INT4 ? 1 : 0,
+                                    h.q_chunk_bytes, h.q_pot_lut, 1, rec));
+    if (rc != QIFT_OK) return rc;
+#define QIFT_ROWS_CASE(LV)                                                                                          \
+    case LV:                                                                                                        \
+        return M > 32 ? launch_grouped_wide<LV, 8, 1, 8>(&h, &rec, none, sumq, st, true)                            \
+               : M > 16 ? launch_grouped_wide<LV, 4, 1, 8>(&h, &rec, none, sumq, st, true)                          \
+               : M > 8 ? launch_grouped_wide<LV, 2, 1, 8>(&h, &rec, none, sumq, st, true)                           \
+                       : launch_grouped_wide<LV, 1, 1, 8>(&h, &rec, none, sumq, st, true);
+    switch (lv) {
+        QIFT_ROWS_CASE(QIFT_LEVELS_MNZ)
+        QIFT_ROWS_CASE(QIFT_LEVELS_POT)
+        QIFT_ROWS_CASE(QIFT_LEVELS_SYM)
+        default:
+            QIFT_ROWS_CASE(QIFT_LEVELS_INT4)
+    }
+#undef QIFT_ROWS_CASE
+}
 }  // namespace
 }  // namespace qift
 
@@ -828,7 +874,7 @@ int qift_group_quantize_act(const void* plan_host, const void* plan_dev, void* s
     cudaError_t e = allow_smem(kernel, smem);
     if (e != cudaSuccess) return cuda_status(e);
     return cuda_status(launch_pdl(kernel, grid, dim3(kRowThreads), smem, st, dev, sumq, h->M, h->clip,
-                                  h->levels == QIFT_LEVELS_INT4 ? 1 : 0, h->q_chunk_bytes, h->q_pot_lut));
+                                  h->levels == QIFT_LEVELS_INT4 ? 1 : 0, h->q_chunk_bytes, h->q_pot_lut, 0, GroupProblemDev{}));
 }
 
 int qift_group_linear(const void* plan_host, const void* plan_dev, void* stream) {

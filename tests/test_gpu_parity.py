@@ -337,6 +337,43 @@ def test_whole_path_config1():
     assert_status_clean()
 
 
+# ---------------------------------------------------------------------------------- whole layer in one call
+@pytest.mark.parametrize("name", list(LEVELS))
+@pytest.mark.parametrize("M,N,K,B", [(1, 300, 1024, 1024), (5, 130, 2560, 512), (16, 260, 4096, 4096), (40, 200, 1024, 0),
+                                     (100, 96, 512, 256), (3, 64, 14336, 14336), (9, 40, 11008, 256)])
+def test_forward_one_call(name, M, N, K, B):
+    # rotation + activation quantization + product + scales in one call, on device tensors and through host buffers;
+    # 2..64 rows go through the grouped path's quantizer and the row-split kernel, the rest through the per-call kernels
+    lv = LEVELS[name][0]
+    W = synth.gaussian_weights(900 + M, N, K)
+    x, _ = synth.activations(901 + M, M, K, max(1, K // 100))
+    p_ref, s_n, codes = oracle.pack_weights(W, lv, oracle.SCALE_ABSMAX)
+    packed, sn = dev(p_ref.view(np.int32)), dev(s_n)
+    for bf16_in in (False, True):
+        xd = dev(x).to(torch.bfloat16) if bf16_in else dev(x)
+        x_ref = oracle.bf16_to_f32(xd.view(torch.int16).cpu().numpy().view(np.uint16)) if bf16_in else x
+        q_ref, sa_ref = oracle.quantize_act(x_ref, B, 0.9)
+        for bf16_out in (False, True):
+            y_ref, _ = oracle.linear(codes, lv, s_n, q_ref, sa_ref, bf16=bf16_out)
+            y = qift.qift_forward(xd, B, packed, sn, lv, out_dtype=torch.bfloat16 if bf16_out else torch.float32)
+            assert_status_clean()
+            if bf16_out:
+                got = y.view(torch.int16).cpu().numpy().view(np.uint16).astype(np.int64)
+                key = lambda v: np.where(v & 0x8000, 0x8000 - (v & 0x7FFF), 0x8000 + v)
+                assert np.abs(key(got) - key(y_ref.astype(np.int64))).max() <= 1
+            else:
+                assert np.array_equal(y.cpu().numpy(), y_ref)
+    # host buffers in and out
+    xh = torch.from_numpy(x).pin_memory()
+    yh = torch.empty((M, N), dtype=torch.float32).pin_memory()
+    qift.qift_forward_host(xh, B, packed, sn, lv, yh)
+    torch.cuda.synchronize()
+    q_ref, sa_ref = oracle.quantize_act(x, B, 0.9)
+    y_ref, _ = oracle.linear(codes, lv, s_n, q_ref, sa_ref)
+    assert np.array_equal(yh.numpy(), y_ref)
+    assert_status_clean()
+
+
 # ---------------------------------------------------------------------------------- grouped path
 @pytest.mark.parametrize("name", list(LEVELS))
 @pytest.mark.parametrize("M", [1, 2, 5, 6, 8, 9, 13, 16, 17, 27, 32, 33, 50, 64])

@@ -62,18 +62,27 @@ constexpr uint32_t kGroupMagic = 0x51494654u;
 // bytes of the even code planes (k % 16 in 0..3 or 8..11) hold 4*q, with INT4 weights the bytes of
 // plane 0 (k % 8 in 0..3) hold 16*q; sumq holds the plain sum of q.
 // Layout of q_a for the row-split product kernel, which stages one K-chunk of ALL tokens per pipeline stage: chunk
-// after chunk, inside a chunk token after token (so a stage is one contiguous piece of memory, one bulk copy), and
-// inside a token's chunk the 16-byte groups of an odd token swapped in pairs -- the product kernel's lanes read
-// tokens g and g+1 at the same group index in one instruction, and the swap puts them on different banks.
-//   byte address of group q of token m:  c = 16 q / CB,  c CB M + m min(CB, K - c CB) + 16 ((q mod CB/16) xor (m & 1))
+// after chunk, inside a chunk token after token (so a stage is one contiguous piece of memory, one bulk copy).
+// Inside a token's chunk the 16-byte groups are permuted so that the product kernel's reads are free of bank
+// conflicts although every lane visits its groups in the same order: a quarter-warp of that kernel reads, in one
+// instruction, group index i of the 64-byte blocks cq = 0..3 of tokens g and g+1.  Blocks two apart would share
+// their banks, as would the two tokens; so the group index is XORed with 2 in every other PAIR of blocks (two-bit
+// weights: four groups per block) and with 1 for odd tokens.  INT4 weights have two groups per 32-byte block and
+// only the token swap.
+//   byte address of group q of token m:  c = 16 q / CB,  c CB M + m min(CB, K - c CB) + 16 swizzled(q mod CB/16)
+__host__ __device__ __forceinline__ int swizzled_group(int piece, int m, int two_bit) {
+    const int block_pair = two_bit ? ((piece >> 3) & 1) << 1 : 0;   // bit 1 of the 64-byte block index -> bit 1 of the group index
+    return piece ^ block_pair ^ (m & 1);
+}
 struct ChunkMajorDst {
     int8_t* q_a;
-    int m, M, K, cb, pot_lut;
+    int m, M, K, cb, pot_lut, two_bit;
     __device__ __forceinline__ void store(int q, uint4 v) const {
         if (pot_lut) v = pot_lut_order(v);
         const int c = (16 * q) / cb, piece = q - c * (cb / 16);
         const int bytes = min(cb, K - c * cb);
-        *reinterpret_cast<uint4*>(q_a + static_cast<size_t>(c) * cb * M + static_cast<size_t>(m) * bytes + 16 * (piece ^ (m & 1))) = v;
+        *reinterpret_cast<uint4*>(q_a + static_cast<size_t>(c) * cb * M + static_cast<size_t>(m) * bytes +
+                                  16 * swizzled_group(piece, m, two_bit)) = v;
     }
 };
 
@@ -95,7 +104,7 @@ quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* _
     if (threadIdx.x == 0) P.s_a[m] = (B > 1) ? __fmul_rn(sc.s_u, P.inv_sqrt_b) : sc.s_u;
     // 32-bit word i of a 16-byte group = code plane (two-bit: i; INT4: i & 1); even planes are prescaled
     const float mult = q_pot_lut ? 1.0f : int4_weights ? 16.0f : 4.0f;
-    int total = q_chunk_bytes ? quantize_row<true>(row, K, sc, ChunkMajorDst{P.q_a, static_cast<int>(m), M, K, q_chunk_bytes, q_pot_lut}, mult, 1.0f)
+    int total = q_chunk_bytes ? quantize_row<true>(row, K, sc, ChunkMajorDst{P.q_a, static_cast<int>(m), M, K, q_chunk_bytes, q_pot_lut, int4_weights ? 0 : 1}, mult, 1.0f)
                               : quantize_row<true>(row, K, sc, RowMajorDst{P.q_a + m * K}, mult, 1.0f);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
@@ -118,7 +127,7 @@ relayout_act_kernel(const int8_t* __restrict__ q_a, int M, int K, int int4_weigh
     pdl_launch_dependents();
     pdl_wait();
     const int m = blockIdx.x;
-    const ChunkMajorDst dst{q_out, m, M, K, q_chunk_bytes, q_pot_lut};
+    const ChunkMajorDst dst{q_out, m, M, K, q_chunk_bytes, q_pot_lut, int4_weights ? 0 : 1};
     const uint4* src = reinterpret_cast<const uint4*>(q_a + static_cast<size_t>(m) * K);
     int total = 0;
     for (int q = threadIdx.x; q < K / 16; q += blockDim.x) {
@@ -551,13 +560,9 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     pdl_wait();
     const int g = lane >> 2, cq = lane & 3;
     // per-lane byte offsets inside a stage, fixed for the whole kernel
-    const int rot = (T::PER == 16) ? (cq & 2) : 0;
-    // Activations of a stage: token after token, a token's chunk contiguous, the 16-byte pieces of odd tokens
-    // swapped in pairs (ChunkMajorDst).  A lane needs 64 contiguous bytes per token and slice (its four packed
-    // words x 16 codes = NPL pieces), lanes of a quad 64 bytes apart: read straight, lanes cq and cq+2 would hit the
-    // same banks, so lanes with cq >= 2 visit their pieces in the order 2,3,0,1 (the sums do not depend on the
-    // order); lanes g and g+1 read the same piece index of neighbouring tokens, which the pair swap separates.
-    // Every quarter-warp then covers all eight 16-byte bank groups.  (INT4 weights: 32 bytes per lane, two pieces.)
+    // Activations of a stage: token after token, a token's chunk contiguous, its 16-byte groups permuted as
+    // ChunkMajorDst describes.  A lane needs the NPL groups of its block per token and slice (its four packed words x
+    // PER codes), block cq of the slice; it visits them in order and finds group i at swizzled_group(i).
     // Token columns beyond M read the last token's bytes: a column of the product depends on its own
     // activations only, and those columns are never written.
     int q_tok[NT];
@@ -567,7 +572,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
         q_tok[nt] = min(nt * 8 + g, M - 1);
 #pragma unroll
         for (int i = 0; i < T::NPL; ++i)
-            q_piece[nt][i] = 4 * cq * T::PER + 16 * (((i + rot * T::NPL / 4) % T::NPL) ^ (q_tok[nt] & 1));
+            q_piece[nt][i] = 16 * swizzled_group(T::NPL * cq + i, q_tok[nt], T::PER == 16);
     }
     const uint32_t ring_addr = smem_u32(ring);
     Cursor cur;
@@ -631,22 +636,10 @@ linear_grouped_wide_kernel(const GroupParams gp) {
 #pragma unroll
                     for (int i = 0; i < T::NPL; ++i) qa[nt][i] = qs + q_tok[nt] * (cw * T::PER) + q_piece[nt][i];
                 const uint32_t wa_base = ws + lane * 16;
-                // the lane's four words of rows g and g+8 of row tile r; lanes that visit their activation pieces in
-                // the order 2,3,0,1 take the words in that order too: by selects after a 128-bit load, or (PoT with one
-                // token tile, where the logic pipe is the limit) by two 64-bit loads, which cost a two-way bank
-                // conflict instead
+                // the lane's four words of rows g and g+8 of row tile r
                 auto load_words = [&](int r, int sl, uint4& wa, uint4& wb) {
                     const uint32_t o = r * TILE_STAGE + sl * 1024;
-                    if constexpr (LV == QIFT_LEVELS_POT && NT == 1) {
-                        const uint32_t lo_a = wa_base + o + 4 * rot, hi_a = lo_a + 8 - 8 * rot;
-                        const uint2 a_lo = lds64(lo_a), a_hi = lds64(hi_a), b_lo = lds64(lo_a + 512), b_hi = lds64(hi_a + 512);
-                        wa = make_uint4(a_lo.x, a_lo.y, a_hi.x, a_hi.y);
-                        wb = make_uint4(b_lo.x, b_lo.y, b_hi.x, b_hi.y);
-                    } else {
-                        const uint4 ra = lds128(wa_base + o), rb = lds128(wa_base + o + 512);
-                        wa = rot ? make_uint4(ra.z, ra.w, ra.x, ra.y) : ra;
-                        wb = rot ? make_uint4(rb.z, rb.w, rb.x, rb.y) : rb;
-                    }
+                    wa = lds128(wa_base + o), wb = lds128(wa_base + o + 512);
                 };
                 auto slice = [&](int sl, auto ks) {
                     if constexpr (NT <= 2) {

@@ -465,6 +465,40 @@ def test_grouped_shared_activation(M):
     check_outputs(plan.outputs[1], plan.accs[1], y_ref, acc_ref, False)
 
 
+@pytest.mark.parametrize("M", [1, 12])
+def test_grouped_forward_in_a_cuda_graph(M):
+    # a plan captured once and replayed after the activations changed in place
+    lv = qift.POT
+    probs, packs = [], []
+    for i, (N, K) in enumerate([(300, 1024), (64, 2560), (4100, 512)]):
+        W = synth.gaussian_weights(950 + i, N, K)
+        p_ref, s_n, codes = oracle.pack_weights(W, lv, oracle.SCALE_ABSMAX)
+        x, _ = synth.activations(960 + i, M, K, 8)
+        probs.append((dev(x), dev(p_ref.view(np.int32)), dev(s_n), synth.had_block_for(K)))
+        packs.append((codes, s_n, K))
+    plan = qift.qift_group_plan(probs, lv, 0.9)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        qift.qift_group_forward(plan)
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            qift.qift_group_forward(plan)
+    for rnd in (1, 2):
+        xs = []
+        for i, (X, _, _, _) in enumerate(probs):
+            x, _ = synth.activations(970 + 10 * rnd + i, M, X.shape[1], 8)
+            X.copy_(dev(x))
+            xs.append(x)
+        g.replay()
+        torch.cuda.synchronize()
+        for (codes, s_n, K), x, y in zip(packs, xs, plan.outputs):
+            q_ref, sa_ref = oracle.quantize_act(x, synth.had_block_for(K), 0.9)
+            y_ref, _ = oracle.linear(codes, lv, s_n, q_ref, sa_ref)
+            assert np.array_equal(y.cpu().numpy(), y_ref)
+    assert_status_clean()
+
+
 def test_grouped_rejects_bad_plans():
     x = torch.zeros((1, 256), device="cuda")
     packed = torch.zeros((16, 16), dtype=torch.int32, device="cuda")

@@ -658,7 +658,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     if (!aligned16(plan_dev) || !aligned16(plan_host)) return QIFT_ERR_ALIGNMENT;
     // Rows per work item, which also selects the kernel (dispatch_grouped): 64 / 32 for the K-split kernel, 128 for the
     // row-split kernel, 256 (two row tiles per warp, with two token tiles) when that still leaves two items per SM.
-    int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : (M == 1) ? 64 : 32;
+    int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : 64;  // below wide_min_m there is only M = 1
     if (rows_per_item == kWideRows && M > 8 && M <= 16 && levels != QIFT_LEVELS_POT) {  // PoT measured slower with two tiles
         long long items256 = 0;
         for (int i = 0; i < count; ++i) items256 += (problems[i].N + 2 * kWideRows - 1) / (2 * kWideRows);
@@ -773,15 +773,14 @@ int launch_grouped_wide(const GroupHeader* h, const GroupProblemDev* host, const
 template <int LV>
 int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
                      cudaStream_t st) {
-    // (256-row items -- two row tiles per warp, or sixteen consumer warps -- were measured slower: 3.2 / 3.2 against
-    // 3.9 TB/s at 16 rows.)
+    // (256-row items as sixteen consumer warps were measured slower and are not dispatched.)
     if (h->rows_per_item == 2 * kWideRows) return launch_grouped_wide<LV, 2, 2, 8>(h, host, dev, sumq, st);
     if (h->rows_per_item == kWideRows && h->M > 32) return launch_grouped_wide<LV, 8, 1, 8>(h, host, dev, sumq, st);
     if (h->rows_per_item == kWideRows && h->M > 16) return launch_grouped_wide<LV, 4, 1, 8>(h, host, dev, sumq, st);
     if (h->rows_per_item == kWideRows)
         return h->M > 8 ? launch_grouped_wide<LV, 2, 1, 8>(h, host, dev, sumq, st) : launch_grouped_wide<LV, 1, 1, 8>(h, host, dev, sumq, st);
     if (h->M == 1) return launch_grouped<LV, 1, 4, true>(h, host, dev, sumq, st);
-    return launch_grouped<LV, 1, 2, false>(h, host, dev, sumq, st);
+    return QIFT_ERR_INVALID_ARG;  // no plan has other row counts per item
 }
 }  // namespace
 

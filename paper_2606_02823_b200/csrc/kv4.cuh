@@ -237,37 +237,11 @@ kv4_attention_partial_kernel(const Kv4Params p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, cq = lane & 3;
 
-    // query fragments: row g (head kv*G + g, zero beyond G), scaled by 1/sqrt(D), split in two fp16 parts
-    uint32_t qh[8][2], ql[8][2];
-    float qsum = 0.0f;  // sum over all dimensions of (high + low) parts of head g
-    {
-        const float* qrow = p.q + static_cast<size_t>(kv * G + (g < G ? g : 0)) * kKvD;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            float4 f = *reinterpret_cast<const float4*>(qrow + 32 * cq + 4 * ks);
-            if (g >= G) f = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            f.x = __fmul_rn(f.x, p.inv_sqrt_d), f.y = __fmul_rn(f.y, p.inv_sqrt_d);
-            f.z = __fmul_rn(f.z, p.inv_sqrt_d), f.w = __fmul_rn(f.w, p.inv_sqrt_d);
-            split_half2(f.x, f.y, qh[ks][0], ql[ks][0]);
-            split_half2(f.z, f.w, qh[ks][1], ql[ks][1]);
-            qsum += (f.x + f.y) + (f.z + f.w);
-        }
-        qsum += __shfl_xor_sync(0xffffffffu, qsum, 1);
-        qsum += __shfl_xor_sync(0xffffffffu, qsum, 2);
-    }
-
     const int t_begin = split * p.tokens_per_split;
     const int t_end = min(p.T, t_begin + p.tokens_per_split);
     const size_t head_row = static_cast<size_t>(kv) * p.T_cap;
     const uint8_t* vbase = p.v_codes + static_cast<size_t>(kv) * (p.T_cap >> 1) * kKvD;
     const int last_row = p.T_cap - 1, last_pair = (p.T_cap >> 1) - 1;
-
-    float o[16][4];
-#pragma unroll
-    for (int nt = 0; nt < 16; ++nt)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) o[nt][i] = 0.0f;
-    float m_run = -INFINITY, l_run = 0.0f, z_run = 0.0f;  // of head g (l and z: this lane's tokens only)
 
     // loads of a tile: key rows of tokens tb+g and tb+8+g, value pair rows tb/2+cq and tb/2+4+cq, scales and
     // zero-points of this lane's four tokens tb + 8n + 2cq + {0,1}; issued one tile ahead of their use
@@ -289,6 +263,38 @@ kv4_attention_partial_kernel(const Kv4Params p) {
             x.vzp[n] = *reinterpret_cast<const float2*>(p.v_zero + head_row + t);
         }
     };
+    // the warp's first tile is requested before the query is touched: the two latencies overlap
+    constexpr int kTileStride = kKvTile * kKvWarps;
+    Tile ta, tb2;
+    int tb = t_begin + kKvTile * warp;
+    if (tb < t_end) load_tile(ta, tb);
+
+    // query fragments: row g (head kv*G + g, zero beyond G), scaled by 1/sqrt(D), split in two fp16 parts
+    uint32_t qh[8][2], ql[8][2];
+    float qsum = 0.0f;  // sum over all dimensions of (high + low) parts of head g
+    {
+        const float* qrow = p.q + static_cast<size_t>(kv * G + (g < G ? g : 0)) * kKvD;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            float4 f = *reinterpret_cast<const float4*>(qrow + 32 * cq + 4 * ks);
+            if (g >= G) f = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            f.x = __fmul_rn(f.x, p.inv_sqrt_d), f.y = __fmul_rn(f.y, p.inv_sqrt_d);
+            f.z = __fmul_rn(f.z, p.inv_sqrt_d), f.w = __fmul_rn(f.w, p.inv_sqrt_d);
+            split_half2(f.x, f.y, qh[ks][0], ql[ks][0]);
+            split_half2(f.z, f.w, qh[ks][1], ql[ks][1]);
+            qsum += (f.x + f.y) + (f.z + f.w);
+        }
+        qsum += __shfl_xor_sync(0xffffffffu, qsum, 1);
+        qsum += __shfl_xor_sync(0xffffffffu, qsum, 2);
+    }
+
+    float o[16][4];
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o[nt][i] = 0.0f;
+    float m_run = -INFINITY, l_run = 0.0f, z_run = 0.0f;  // of head g (l and z: this lane's tokens only)
+
     auto process_tile = [&](const Tile& cur, int tb) {
         const uint4(&kraw)[2] = cur.kraw;
         const uint4(&vraw)[2] = cur.vraw;
@@ -354,10 +360,7 @@ kv4_attention_partial_kernel(const Kv4Params p) {
     };
     // two tile buffers used alternately, each loaded one tile ahead of its use
     {
-        constexpr int stride = kKvTile * kKvWarps;
-        Tile ta, tb2;
-        int tb = t_begin + kKvTile * warp;
-        if (tb < t_end) load_tile(ta, tb);
+        constexpr int stride = kTileStride;
         while (tb < t_end) {
             if (tb + stride < t_end) load_tile(tb2, tb + stride);
             process_tile(ta, tb);
@@ -397,37 +400,84 @@ kv4_attention_partial_kernel(const Kv4Params p) {
     }
 }
 
-// Merge the splits of each query head: one CTA per head.  Thread s first turns split s's running max
-// into its weight exp(m_s - max) (one exponential per split, not per element), then thread d sums
-// dimension d over the splits.
+// Merge the splits of each query head: one CTA per head, four groups of 64 threads.  Group r takes splits
+// r, r+4, ...; a thread takes two neighbouring dimensions.  The numerators of a group's first splits are
+// requested before the weights exp(m_s - max) exist (one exponential per split, computed by thread s), so the
+// kernel spends one round trip to memory on them instead of one per split; the groups meet in shared memory.
 constexpr int kKvMaxSplits = 1024;
-__global__ void __launch_bounds__(kKvD)
+constexpr int kKvCombineThreads = 256;
+constexpr int kKvCombineGroups = kKvCombineThreads / (kKvD / 2);
+constexpr int kKvCombineAhead = 8;  // splits per group whose loads are issued up front (32 splits in all)
+__global__ void __launch_bounds__(kKvCombineThreads)
 kv4_attention_combine_kernel(const Kv4Params p) {
     __shared__ float weight[kKvMaxSplits];
-    __shared__ float wmax[kKvD / 32];
+    __shared__ float wmax[kKvCombineThreads / 32];
+    __shared__ float2 gnum[kKvCombineGroups][kKvD / 2];
+    __shared__ float gden[kKvCombineGroups];
     pdl_launch_dependents();
     pdl_wait();
-    const int h = blockIdx.x, d = threadIdx.x;
+    const int h = blockIdx.x, tid = threadIdx.x;
+    const int grp = tid / (kKvD / 2), j = tid % (kKvD / 2);
     const float* base = p.partial + static_cast<size_t>(h) * p.splits * kKvPartial;
+    float2 pre[kKvCombineAhead];
+    float dpre[kKvCombineAhead];
+#pragma unroll
+    for (int i = 0; i < kKvCombineAhead; ++i) {
+        const int s = grp + kKvCombineGroups * i;
+        pre[i] = make_float2(0.0f, 0.0f), dpre[i] = 0.0f;
+        if (s < p.splits) {
+            pre[i] = *reinterpret_cast<const float2*>(base + static_cast<size_t>(s) * kKvPartial + 2 * j);
+            dpre[i] = base[static_cast<size_t>(s) * kKvPartial + kKvD + 1];
+        }
+    }
+    float msv[kKvMaxSplits / kKvCombineThreads];
     float mm = -INFINITY;
-    for (int s = d; s < p.splits; s += kKvD) mm = fmaxf(mm, base[s * kKvPartial + kKvD]);
+#pragma unroll
+    for (int i = 0; i < kKvMaxSplits / kKvCombineThreads; ++i) {
+        const int s = tid + kKvCombineThreads * i;
+        msv[i] = (s < p.splits) ? base[static_cast<size_t>(s) * kKvPartial + kKvD] : -INFINITY;
+        mm = fmaxf(mm, msv[i]);
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
-    if ((d & 31) == 0) wmax[d >> 5] = mm;
+    if ((tid & 31) == 0) wmax[tid >> 5] = mm;
     __syncthreads();
-    mm = fmaxf(fmaxf(wmax[0], wmax[1]), fmaxf(wmax[2], wmax[3]));
-    for (int s = d; s < p.splits; s += kKvD) {
-        const float ms = base[s * kKvPartial + kKvD];
-        weight[s] = (ms > -INFINITY) ? expf(ms - mm) : 0.0f;
+    mm = wmax[0];
+#pragma unroll
+    for (int w = 1; w < kKvCombineThreads / 32; ++w) mm = fmaxf(mm, wmax[w]);
+#pragma unroll
+    for (int i = 0; i < kKvMaxSplits / kKvCombineThreads; ++i) {
+        const int s = tid + kKvCombineThreads * i;
+        if (s < p.splits) weight[s] = (msv[i] > -INFINITY) ? expf(msv[i] - mm) : 0.0f;
     }
     __syncthreads();
-    float num = 0.0f, den = 0.0f;
-    for (int s = 0; s < p.splits; ++s) {
+    float2 num = make_float2(0.0f, 0.0f);
+    float den = 0.0f;
+#pragma unroll
+    for (int i = 0; i < kKvCombineAhead; ++i) {
+        const int s = grp + kKvCombineGroups * i;
+        if (s < p.splits) {
+            const float f = weight[s];
+            num.x = fmaf(pre[i].x, f, num.x), num.y = fmaf(pre[i].y, f, num.y);
+            den = fmaf(dpre[i], f, den);
+        }
+    }
+    for (int s = grp + kKvCombineGroups * kKvCombineAhead; s < p.splits; s += kKvCombineGroups) {
         const float f = weight[s];
-        num = fmaf(base[s * kKvPartial + d], f, num);
-        den = fmaf(base[s * kKvPartial + kKvD + 1], f, den);
+        const float2 v = *reinterpret_cast<const float2*>(base + static_cast<size_t>(s) * kKvPartial + 2 * j);
+        num.x = fmaf(v.x, f, num.x), num.y = fmaf(v.y, f, num.y);
+        den = fmaf(base[static_cast<size_t>(s) * kKvPartial + kKvD + 1], f, den);
     }
-    p.out[static_cast<size_t>(h) * kKvD + d] = num / den;
+    gnum[grp][j] = num;
+    if (j == 0) gden[grp] = den;
+    __syncthreads();
+    if (tid < kKvD / 2) {
+        float2 n = gnum[0][tid];
+        float d = gden[0];
+#pragma unroll
+        for (int r = 1; r < kKvCombineGroups; ++r) n.x += gnum[r][tid].x, n.y += gnum[r][tid].y, d += gden[r];
+        *reinterpret_cast<float2*>(p.out + static_cast<size_t>(h) * kKvD + 2 * tid) = make_float2(n.x / d, n.y / d);
+    }
 }
 
 }  // namespace qift

@@ -1203,7 +1203,7 @@ int qift_kv4_attention_decode(const float* q, const uint8_t* k_codes, const floa
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int rc = cuda_status(launch_pdl(kv4_attention_partial_kernel, dim3(p.splits, p.Hkv), dim3(32 * kKvWarps), 0, st, p));
     if (rc != QIFT_OK) return rc;
-    return cuda_status(launch_pdl(kv4_attention_combine_kernel, dim3(p.Hq), dim3(kKvD), 0, st, p));
+    return cuda_status(launch_pdl(kv4_attention_combine_kernel, dim3(p.Hq), dim3(kKvCombineThreads), 0, st, p));
 }
 
 }  // extern "C"

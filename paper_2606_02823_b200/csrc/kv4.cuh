@@ -249,18 +249,31 @@ kv4_attention_partial_kernel(const Kv4Params p) {
         uint4 kraw[2], vraw[2];
         float2 ksc[2], kzp[2], vsc[2], vzp[2];
     };
+    const uint8_t* kbase = p.k_codes + head_row * kKvRowBytes;
+    const float* ksb = p.k_scale + head_row;
+    const float* kzb = p.k_zero + head_row;
+    const float* vsb = p.v_scale + head_row;
+    const float* vzb = p.v_zero + head_row;
+    const uint32_t klane = static_cast<uint32_t>(g) * kKvRowBytes + 16u * cq;
+    const uint32_t vlane = static_cast<uint32_t>(cq) * kKvD + 16u * g;
+    // clamped 32-bit byte offsets from per-head base pointers: rows past the end of the arrays (a last tile
+    // that crosses T_cap) read the last row instead; offsets grow with the row, so one min per load does it
+    const uint32_t kmax = static_cast<uint32_t>(last_row) * kKvRowBytes + 16u * cq;
+    const uint32_t vmax = static_cast<uint32_t>(last_pair) * kKvD + 16u * g;
+    const uint32_t smax = static_cast<uint32_t>(last_row - 1);
     auto load_tile = [&](Tile& x, int tb) {
+        const uint32_t koff = static_cast<uint32_t>(tb) * kKvRowBytes + klane;
+        const uint32_t voff = static_cast<uint32_t>(tb >> 1) * kKvD + vlane;
+        const uint32_t so = static_cast<uint32_t>(tb) + 2u * cq;
 #pragma unroll
         for (int n = 0; n < 2; ++n) {
-            const int krow = min(tb + 8 * n + g, last_row);
-            x.kraw[n] = *reinterpret_cast<const uint4*>(p.k_codes + (head_row + krow) * kKvRowBytes + 16 * cq);
-            const int vrow = min((tb >> 1) + 4 * n + cq, last_pair);
-            x.vraw[n] = *reinterpret_cast<const uint4*>(vbase + static_cast<size_t>(vrow) * kKvD + 16 * g);
-            const int t = min(tb + 8 * n + 2 * cq, last_row - 1);   // even: the pair t, t+1 is inside the arrays
-            x.ksc[n] = *reinterpret_cast<const float2*>(p.k_scale + head_row + t);
-            x.kzp[n] = *reinterpret_cast<const float2*>(p.k_zero + head_row + t);
-            x.vsc[n] = *reinterpret_cast<const float2*>(p.v_scale + head_row + t);
-            x.vzp[n] = *reinterpret_cast<const float2*>(p.v_zero + head_row + t);
+            x.kraw[n] = *reinterpret_cast<const uint4*>(kbase + min(koff + n * 8u * kKvRowBytes, kmax));
+            x.vraw[n] = *reinterpret_cast<const uint4*>(vbase + min(voff + n * 4u * kKvD, vmax));
+            const uint32_t t = min(so + n * 8u, smax);   // even: the pair t, t+1 is inside the arrays
+            x.ksc[n] = *reinterpret_cast<const float2*>(ksb + t);
+            x.kzp[n] = *reinterpret_cast<const float2*>(kzb + t);
+            x.vsc[n] = *reinterpret_cast<const float2*>(vsb + t);
+            x.vzp[n] = *reinterpret_cast<const float2*>(vzb + t);
         }
     };
     // the warp's first tile is requested before the query is touched: the two latencies overlap

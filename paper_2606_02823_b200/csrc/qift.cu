@@ -1188,7 +1188,7 @@ int qift_kv4_attention_decode(const float* q, const uint8_t* k_codes, const floa
     if (T <= 0 || T > T_cap || Hq <= 0 || Hkv <= 0) return QIFT_ERR_INVALID_ARG;
     if (D != kKvD || Hq % Hkv != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
     const int G = Hq / Hkv;
-    if (G > 8 || (T_cap & 1)) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (G > 8 || (T_cap & 1) || T_cap > (1 << 24)) return QIFT_ERR_UNSUPPORTED_SHAPE;  // 32-bit byte offsets inside a head
     if (!aligned16(q) || !aligned16(k_codes) || !aligned16(v_codes) || !aligned16(k_scale) || !aligned16(k_zero) ||
         !aligned16(v_scale) || !aligned16(v_zero) || !aligned16(out) || !aligned16(workspace))
         return QIFT_ERR_ALIGNMENT;

@@ -353,11 +353,14 @@ kv4_attention_partial_kernel(const Kv4Params p) {
         float w4[4];
 #pragma unroll
         for (int n = 0; n < 2; ++n) {
-            const float p0 = (s4[2 * n] > -INFINITY) ? expf(s4[2 * n] - m_run) : 0.0f;
-            const float p1 = (s4[2 * n + 1] > -INFINITY) ? expf(s4[2 * n + 1] - m_run) : 0.0f;
+            // slots past the split's end may hold anything (a cache is filled as tokens arrive), NaN included:
+            // their scale and zero-point are replaced, not multiplied by a zero weight
+            const bool in0 = s4[2 * n] > -INFINITY, in1 = s4[2 * n + 1] > -INFINITY;
+            const float p0 = in0 ? expf(s4[2 * n] - m_run) : 0.0f;
+            const float p1 = in1 ? expf(s4[2 * n + 1] - m_run) : 0.0f;
             l_run += p0 + p1;
-            w4[2 * n] = p0 * vsc[n].x, w4[2 * n + 1] = p1 * vsc[n].y;
-            z_run = fmaf(w4[2 * n], vzp[n].x, fmaf(w4[2 * n + 1], vzp[n].y, z_run));
+            w4[2 * n] = in0 ? p0 * vsc[n].x : 0.0f, w4[2 * n + 1] = in1 ? p1 * vsc[n].y : 0.0f;
+            z_run = fmaf(w4[2 * n], in0 ? vzp[n].x : 0.0f, fmaf(w4[2 * n + 1], in1 ? vzp[n].y : 0.0f, z_run));
         }
         // ---- O += w . value codes: k = the tile's 16 tokens, A rows = heads
         uint32_t wh[2], wl[2];

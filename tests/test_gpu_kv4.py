@@ -112,6 +112,23 @@ def test_kv4_attention_matches_oracle(T, Hq, Hkv):
     assert rc == qift.OK
 
 
+def test_kv4_attention_ignores_unwritten_slots():
+    """Slots T .. T_cap-1 have not been written yet; whatever they hold (NaN scales included) must not reach the output."""
+    T, Hq, Hkv = 1000, 8, 2
+    K, V, ref_args = build_cache(80, T, Hkv, T + 40)
+    q = (synth.normal(81, 4, (Hq, D)) * 1.5).astype(np.float32)
+    ref = oracle.kv4_attention(q, *ref_args)
+    for c in (K, V):
+        c.scale[:, T:] = float("nan")
+        c.zero[:, T:] = float("inf")
+    K.codes[:, T:] = 0xFF
+    V.codes[:, (T + 1) // 2:] = 0xFF
+    out = qift.qift_kv4_attention_decode(dev(q), K, V, T).cpu().numpy()
+    vmax = np.abs(ref_args[4][..., None] * (ref_args[3].astype(np.float64) - ref_args[5][..., None])).max()
+    assert np.isfinite(out).all()
+    assert np.abs(out - ref).max() <= ATOL_FRAC * vmax
+
+
 def test_kv4_attention_peaked_and_uniform_scores():
     T, Hq, Hkv = 700, 4, 4
     K, V, ref_args = build_cache(70, T, Hkv, T)

@@ -23,20 +23,26 @@ namespace qift {
 // ------------------------------------------------------------------------------------------------
 // expansion: packed codes -> int8 levels, K contiguous
 // ------------------------------------------------------------------------------------------------
+// One packed word -> its PER level bytes in k order (o[t] holds codes 4t .. 4t+3).  Four codes (one per byte of
+// w, at bit (32 / PER) * t of the byte) become four level bytes at once: the low bits of a level are the code's
+// bits with one of them flipped; the sign extension is all ones exactly when one bit of that intermediate is
+// set, and comes from a multiply that cannot carry across bytes.
 template <int LV>
-__global__ void __launch_bounds__(256)
-expand_levels_kernel(const uint32_t* __restrict__ packed, long long total_words, int words_per_row,
-                     int8_t* __restrict__ out) {
+__device__ __forceinline__ void expand_word(uint32_t w, uint32_t (&o)[codes_per_word(LV) / 4]) {
     constexpr int PER = codes_per_word(LV);
-    pdl_launch_dependents();
-    pdl_wait();
-    const int pitch = round_up16(words_per_row);
-    for (long long j = blockIdx.x * (long long)blockDim.x + threadIdx.x; j < total_words;
-         j += (long long)gridDim.x * blockDim.x) {
-        const uint32_t w = packed[packed_word_address(static_cast<int>(j / words_per_row), static_cast<int>(j % words_per_row), pitch)];
-        uint32_t o[PER / 4];
 #pragma unroll
-        for (int t = 0; t < PER / 4; ++t) {
+    for (int t = 0; t < PER / 4; ++t) {
+        if constexpr (LV == QIFT_LEVELS_MNZ) {         // 2c - 3: low three bits (2c) ^ 5, bits 3..7 set iff c < 2
+            const uint32_t x = (t == 0) ? (w << 1) : (w >> (2 * t - 1));
+            const uint32_t u = (x & 0x06060606u) ^ 0x05050505u;
+            o[t] = (u & 0x04040404u) * 62u + u;
+        } else if constexpr (LV == QIFT_LEVELS_SYM) {  // c - 2: low two bits c ^ 2, bits 2..7 set iff c < 2
+            const uint32_t u = ((w >> (2 * t)) & 0x03030303u) ^ 0x02020202u;
+            o[t] = (u & 0x02020202u) * 126u + u;
+        } else if constexpr (LV == QIFT_LEVELS_INT4) { // nibble sign-extended: bits 4..7 set iff bit 3
+            const uint32_t u = (w >> (4 * t)) & 0x0f0f0f0fu;
+            o[t] = (u & 0x08080808u) * 30u + u;
+        } else {                                       // PoT: code by code
             uint32_t r = 0;
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
@@ -45,9 +51,27 @@ expand_levels_kernel(const uint32_t* __restrict__ packed, long long total_words,
             }
             o[t] = r;
         }
-        if constexpr (PER == 16) reinterpret_cast<uint4*>(out)[j] = make_uint4(o[0], o[1], o[2], o[3]);
-        else reinterpret_cast<uint2*>(out)[j] = make_uint2(o[0], o[1]);
     }
+}
+
+// Rows are dealt to the CTAs, the words of a row to the threads (no division per word); a thread writes the 16
+// (W4: 8) level bytes of its word with one store.  (Four words per thread, one 128-bit load and 64 bytes written,
+// was measured slower: a row of 4096 weights then occupies a quarter of the CTA.)
+template <int LV>
+__global__ void __launch_bounds__(256)
+expand_levels_kernel(const uint32_t* __restrict__ packed, int N, int words_per_row, int8_t* __restrict__ out) {
+    constexpr int PER = codes_per_word(LV);
+    pdl_launch_dependents();
+    pdl_wait();
+    const int pitch = round_up16(words_per_row);
+    for (int n = blockIdx.x; n < N; n += gridDim.x)
+        for (int jw = threadIdx.x; jw < words_per_row; jw += blockDim.x) {
+            const size_t j = static_cast<size_t>(n) * words_per_row + jw;
+            uint32_t o[PER / 4];
+            expand_word<LV>(packed[packed_word_address(n, jw, pitch)], o);
+            if constexpr (PER == 16) reinterpret_cast<uint4*>(out)[j] = make_uint4(o[0], o[1], o[2], o[3]);
+            else reinterpret_cast<uint2*>(out)[j] = make_uint2(o[0], o[1]);
+        }
 }
 
 // ------------------------------------------------------------------------------------------------

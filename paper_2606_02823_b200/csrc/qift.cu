@@ -212,11 +212,11 @@ int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& 
 
 template <int LV>
 int launch_expand(const uint32_t* packed, int N, int K, int8_t* out, cudaStream_t st) {
-    const long long words = static_cast<long long>(N) * (K / codes_per_word(LV));
-    long long blocks = (words + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
-    return cuda_status(launch_pdl(expand_levels_kernel<LV>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, st, packed, words,
-                                  K / codes_per_word(LV), out));
+    const int blocks = N < 148 * 16 ? N : 148 * 16;   // rows are dealt to the CTAs
+    const int words = K / codes_per_word(LV);
+    const int threads = words >= 256 ? 256 : ((words + 31) / 32) * 32;   // short rows: no idle warps
+    return cuda_status(launch_pdl(expand_levels_kernel<LV>, dim3(static_cast<unsigned>(blocks)), dim3(threads), 0, st, packed, N,
+                                  words, out));
 }
 
 // Tile width of the CTA-pair kernels: the one whose rounds over the SM pairs cost least.  Measured at

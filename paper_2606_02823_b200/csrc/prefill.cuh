@@ -54,9 +54,14 @@ __device__ __forceinline__ void expand_word(uint32_t w, uint32_t (&o)[codes_per_
     }
 }
 
-// Rows are dealt to the CTAs, the words of a row to the threads (no division per word); a thread writes the 16
-// (W4: 8) level bytes of its word with one store.  (Four words per thread, one 128-bit load and 64 bytes written,
+// Blocks of eight rows are dealt to the CTAs, the words of a row to the threads (no division per word).  A thread
+// asks for its word of all eight rows before it uses the first (with one 4-byte load per thread in flight the
+// kernel was bound by the latency of that load: 0.9 TB/s read, ncu's long-scoreboard stall 12 cycles per issue;
+// the eight rows of a block also make one contiguous 512-byte piece of the packed layout per 16-word slice) and
+// writes the 16 (W4: 8) level bytes of each word with one store.  (Four words per thread, one 128-bit load and 64 bytes written,
 // was measured slower: a row of 4096 weights then occupies a quarter of the CTA.)
+constexpr int kExpandRows = 8;
+
 template <int LV>
 __global__ void __launch_bounds__(256)
 expand_levels_kernel(const uint32_t* __restrict__ packed, int N, int words_per_row, int8_t* __restrict__ out) {
@@ -64,13 +69,20 @@ expand_levels_kernel(const uint32_t* __restrict__ packed, int N, int words_per_r
     pdl_launch_dependents();
     pdl_wait();
     const int pitch = round_up16(words_per_row);
-    for (int n = blockIdx.x; n < N; n += gridDim.x)
+    for (int n0 = blockIdx.x * kExpandRows; n0 < N; n0 += gridDim.x * kExpandRows)
         for (int jw = threadIdx.x; jw < words_per_row; jw += blockDim.x) {
-            const size_t j = static_cast<size_t>(n) * words_per_row + jw;
-            uint32_t o[PER / 4];
-            expand_word<LV>(packed[packed_word_address(n, jw, pitch)], o);
-            if constexpr (PER == 16) reinterpret_cast<uint4*>(out)[j] = make_uint4(o[0], o[1], o[2], o[3]);
-            else reinterpret_cast<uint2*>(out)[j] = make_uint2(o[0], o[1]);
+            uint32_t w[kExpandRows];
+#pragma unroll
+            for (int r = 0; r < kExpandRows; ++r) w[r] = (n0 + r < N) ? packed[packed_word_address(n0 + r, jw, pitch)] : 0u;
+#pragma unroll
+            for (int r = 0; r < kExpandRows; ++r) {
+                if (n0 + r >= N) break;
+                const size_t j = static_cast<size_t>(n0 + r) * words_per_row + jw;
+                uint32_t o[PER / 4];
+                expand_word<LV>(w[r], o);
+                if constexpr (PER == 16) reinterpret_cast<uint4*>(out)[j] = make_uint4(o[0], o[1], o[2], o[3]);
+                else reinterpret_cast<uint2*>(out)[j] = make_uint2(o[0], o[1]);
+            }
         }
 }
 

@@ -212,7 +212,8 @@ int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& 
 
 template <int LV>
 int launch_expand(const uint32_t* packed, int N, int K, int8_t* out, cudaStream_t st) {
-    const int blocks = N < 148 * 16 ? N : 148 * 16;   // rows are dealt to the CTAs
+    const int row_blocks = (N + kExpandRows - 1) / kExpandRows;
+    const int blocks = row_blocks < 148 * 16 ? row_blocks : 148 * 16;   // blocks of rows are dealt to the CTAs
     const int words = K / codes_per_word(LV);
     const int threads = words >= 256 ? 256 : ((words + 31) / 32) * 32;   // short rows: no idle warps
     return cuda_status(launch_pdl(expand_levels_kernel<LV>, dim3(static_cast<unsigned>(blocks)), dim3(threads), 0, st, packed, N,

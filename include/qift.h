@@ -289,7 +289,7 @@ int qift_expanded_linear(const int8_t* levels_in, const float* s_n, const int8_t
  *   workspace    >= qift_kv4_attention_workspace_bytes(T, Hq, Hkv) bytes, 16-byte aligned: partial results
  *                of the token splits (two launches: partial attention per split, then the merge)
  * Errors: INVALID_ARG (null pointer, T <= 0, T > T_cap, clip outside (0,1], layout), UNSUPPORTED_SHAPE
- * (D != 128, odd T_cap, more than 8 query heads per KV head, had_block), ALIGNMENT, WORKSPACE, CUDA. */
+ * (D != 128, odd T_cap, T_cap > 2^24 in the attention, more than 8 query heads per KV head, had_block), ALIGNMENT, WORKSPACE, CUDA. */
 enum { QIFT_KV_KEYS = 0, QIFT_KV_VALUES = 1 };
 int qift_kv4_quantize(const void* X, int x_dtype, int T, int H, int D, int had_block, float clip_ratio, int t0,
                       int T_cap, int layout, uint8_t* codes, float* scale, float* zero, void* stream);

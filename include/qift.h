@@ -5,8 +5,12 @@
  *     y[m,n] = s_n[n] * ( sum_k level(code[n,k]) * q_a[m,k] ) * s_a[m]
  *
  * Conventions that hold for every entry point unless its comment says otherwise
- *   - every pointer is DEVICE memory owned by the caller; the library allocates nothing and keeps no
- *     state between calls; base pointers must be 16-byte aligned;
+ *   - every pointer is DEVICE memory owned by the caller; the library allocates nothing; base pointers
+ *     must be 16-byte aligned.  State the library keeps per process: the device status word (see
+ *     qift_device_status), a per-device table of kernels already opted in to large shared memory, the
+ *     per-device SM count, and the per-device address of the built-in scratch of
+ *     qift_w2a4_linear_static.  The last three assume the primary context of each device and no
+ *     cudaDeviceReset while the library is in use;
  *   - all work is enqueued asynchronously on `stream` (a cudaStream_t passed as void*, NULL = the
  *     legacy default stream); nothing synchronizes;
  *   - matrices are row-major with the last index contiguous: W [N,K], X / q_a [M,K], Y [M,N];
@@ -50,9 +54,12 @@ typedef enum {
     QIFT_LEVELS_INT4 = 3  /* -8..7 two's-complement nibble, 8 codes per word         (Eq. 1, b = 4) */
 } qift_levels;
 
-/* How the per-output-channel scale is chosen (Sec. 3.5; Sec. 4.5.1 "sweeping candidate clipping
- * ratios").  GIVEN reads s_n; ABSMAX writes s_n = amax / top_level; MSE sweeps the 80 ratios
+/* How the per-output-channel scale is chosen (Sec. 3.5; the clipping-ratio sweep of Sec. 4.5.1).
+ * GIVEN reads s_n; ABSMAX writes s_n = amax / top_level; MSE sweeps the 80 ratios
  * p = 1.00, 0.99, ..., 0.21, s = (p * amax) / top_level, and keeps the first least-squared-error one.
+ * The squared errors are fp64 sums whose order of addition is the kernel's: two candidates whose
+ * errors agree to 1e-12 relative count as tied, and either may win (a CPU check must allow that and
+ * then compare the codes given the returned scale, which are exact).
  * top_level is 3 (MNZ), 4 (POT), 1 (SYM), 7 (INT4).  An all-zero row gets s_n = 1. */
 typedef enum { QIFT_SCALE_GIVEN = 0, QIFT_SCALE_ABSMAX = 1, QIFT_SCALE_MSE = 2 } qift_scale_mode;
 
@@ -81,10 +88,18 @@ const char* qift_status_string(int status);
  * the words per row to multiples of 16.  0 on bad input. */
 size_t qift_packed_bytes(int N, int K, int levels);
 
-/* Bytes of scratch qift_w2a4_linear / qift_w4a4_linear need for this problem: 0 when the decode
- * route serves it (M <= 16); 4*M rounded up to 1 KiB for 16 < M <= 512 (QIFT_ROUTE_PREFILL up to 128
- * rows, QIFT_ROUTE_PREFILL_FUSED_PAIR above: the per-token sums of q_a); N*K rounded up to 1 KiB for
- * M > 512 (QIFT_ROUTE_PREFILL_PAIR: the codes decoded to int8 once per call).  qift_workspace_bytes_route gives the figure for an explicit route. */
+/* Bytes of scratch qift_w2a4_linear / qift_w4a4_linear can use for this problem, rounded up to 1 KiB:
+ *   M = 1                 0 (decode route);
+ *   2 <= M <= 64          M*K + 256 when K is a whole number of 16-word slices (QIFT_ROUTE_DECODE_ROWS: the
+ *                         activations re-laid out for the row-split kernel plus the token sums), else 0
+ *                         for M <= 16 or 4*M above;
+ *   64 < M <= 512         4*M (QIFT_ROUTE_PREFILL up to 128 rows, QIFT_ROUTE_PREFILL_FUSED_PAIR above:
+ *                         the per-token sums of q_a);
+ *   M > 512               N*K (QIFT_ROUTE_PREFILL_PAIR: the codes decoded to int8 once per call).
+ * With less than this (or NULL) the call still runs when a route without scratch exists -- M <= 16
+ * falls back to the K-split decode kernel, 17..64 rows to the fused prefill route if 4*M bytes were
+ * passed -- and returns QIFT_ERR_WORKSPACE otherwise.  qift_workspace_bytes_route gives the figure
+ * for an explicit route. */
 size_t qift_workspace_bytes(int M, int N, int K, int levels);
 size_t qift_workspace_bytes_route(int M, int N, int K, int levels, int route);
 
@@ -132,7 +147,7 @@ int qift_rotate(const float* X, int M, int K, int had_block, float* Y, void* str
 int qift_quantize_act(const void* X, int x_dtype, int M, int K, int had_block, float clip_ratio,
                       int8_t* q_a, float* s_a, void* stream);
 
-/* S4 + S5 (exact integer product + scale epilogue; Sec. 1 "per-channel scale ... in the epilogue",
+/* S4 + S5 (exact integer product, then the channel and token scales in the epilogue: Sec. 1;
  * Sec. 3.6 decoded small signed integer levels) for the two-bit sets MNZ, POT, SYM.
  *   packed, s_n   from qift_pack_weights
  *   q_a, s_a      from qift_quantize_act
@@ -262,8 +277,8 @@ int qift_expanded_linear(const int8_t* levels_in, const float* s_n, const int8_t
                          int K, void* Y, int y_dtype, int32_t* acc_debug, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------
- * KV4: the 4-bit key / value cache of the paper's W2A4/KV4 setting (Sec. 4.1: "asymmetric key and value
- * quantization with clipping ratios of 0.95") and the single-query decode attention that reads it.
+ * KV4: the 4-bit key / value cache of the paper's W2A4/KV4 setting (Sec. 4.1: keys and values quantized
+ * asymmetrically with a clipping ratio of 0.95) and the single-query decode attention that reads it.
  *
  * Cache layout (device memory, owned by the caller), head-major, T_cap even:
  *   key codes   uint8 [H][T_cap][D/2]   two neighbouring dimensions of a token per byte (even one low)
@@ -343,6 +358,21 @@ int qift_diag_ratio_scan(const float* x, long long n, const double* ratios, int 
  * expired bounded wait.  QIFT_OK, QIFT_ERR_TIMEOUT or QIFT_ERR_CUDA.  `detail` (host, may be NULL)
  * receives the raw word: bits 0-7 the waiting site, the rest the block index. */
 int qift_device_status(void* stream, uint32_t* detail);
+
+/* Self-test of the bounded device-side waits (test-only; the paper has no counterpart).  Every wait of a
+ * kernel on an mbarrier gives up after a wall-time bound (two seconds by default), records where in the
+ * status word and lets the kernel end normally; a product call whose kernel gave up has still returned
+ * QIFT_OK (everything is asynchronous) and leaves Y unwritten -- qift_device_status is how a caller learns
+ * of it.  This entry makes such a wait run out on purpose, with a short bound and without any fault:
+ *   which = 0   one CTA waits for an mbarrier phase that nobody completes; site byte 0x7e
+ *   which = 1   the CTA-pair prefill GEMM on one 256 x 256 x 128 tile whose producers issue no loads (the
+ *               operands are the library's built-in scratch and are never read): the wait for operands
+ *               (site 32) and the waits for the accumulator (site 33) run out, all roles leave, tensor
+ *               memory is freed
+ *   limit_us    the bound, 1 .. 1 000 000 microseconds
+ * Afterwards qift_device_status returns QIFT_ERR_TIMEOUT once, with the site in bits 0-7 of `detail`, and
+ * QIFT_OK on the next call.  INVALID_ARG for other arguments. */
+int qift_selftest_wait_timeout(int which, unsigned int limit_us, void* stream);
 
 #ifdef __cplusplus
 }

@@ -11,7 +11,7 @@
 //   orc_level_value      Sec. 3.3 level-set list (SYM-INT, MNZ, PoT-MNZ) and Eq. 1 with b = 4;
 //                        MNZ is held in its half-scale odd-integer form {-3,-1,+1,+3} (Sec. 3.3,
 //                        the identity {-1.5,-.5,.5,1.5} s = {-3,-1,1,3} s/2).
-//   orc_wht_blocks       Sec. 3.1 / Sec. 4.1 "default Hadamard rotation": Sylvester-Walsh matrix
+//   orc_wht_blocks       Sec. 3.1 / Sec. 4.1 (the default, unlearned Hadamard rotation): Sylvester-Walsh matrix
 //                        in natural order applied by the textbook in-place butterfly, stages in
 //                        ascending stride, fp32.
 //   orc_rotate_weights   the same rotation with the orthonormal factor 1/sqrt(B) (offline, weights).
@@ -19,13 +19,13 @@
 //                        has no Sylvester matrix: H_28 (Paley's second construction, q = 13) Kronecker H_{2^p}.
 //   orc_quantize_act     Eq. 1 with b = 4 on the rotated row, symmetric, clipping ratio as an
 //                        argument (Sec. 4.1 uses 0.9), one scale per token row.
-//   orc_weight_scale     Sec. 3.5 / Sec. 4.5.1: per-output-channel scale, either max-range or
-//                        "MSE-optimal by sweeping candidate clipping ratios".
-//   orc_assign_codes     Sec. 3.5 "maps weights to the nearest scaled level"; Eq. 1 for SYM-INT, INT4.
-//   orc_pack / unpack    Sec. 3.3 "four two-bit codes": 16 two-bit codes (8 nibbles) per 32-bit word,
+//   orc_weight_scale     Sec. 3.5 / Sec. 4.5.1: per-output-channel scale, either max-range or the
+//                        least-squared-error one of a sweep over clipping ratios.
+//   orc_assign_codes     Sec. 3.5: every weight goes to the nearest level times the scale; Eq. 1 for SYM-INT, INT4.
+//   orc_pack / unpack    Sec. 3.3 (a code has two bits): 16 two-bit codes (8 nibbles) per 32-bit word,
 //                        words stored in 16-row x 128-word tiles (layout comment at orc_pack).
 //   orc_int_matmul       Sec. 3.6 decoded small signed integer levels times integer activations.
-//   orc_epilogue*        Sec. 1 "the per-channel scale can be applied separately in the epilogue".
+//   orc_epilogue*        Sec. 1: the channel scale is applied after the integer product, in the epilogue.
 //   orc_kv4_quantize     Sec. 4.1: the KV cache is quantized to four bits asymmetrically with a
 //                        clipping ratio (0.95 there), keys and values alike; the paper gives no
 //                        more, so the rest is the usual asymmetric integer quantizer: one

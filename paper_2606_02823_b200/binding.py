@@ -32,6 +32,7 @@ EXPORTS = [
     "qift_kv4_quantize", "qift_kv4_attention_workspace_bytes", "qift_kv4_attention_decode",
     "qift_expand_weights", "qift_expanded_linear",
     "qift_diag_grid_quantize", "qift_diag_bucket_stats", "qift_diag_ratio_scan_workspace_bytes", "qift_diag_ratio_scan",
+    "qift_selftest_wait_timeout",
 ]
 
 _lib = None
@@ -94,6 +95,7 @@ def lib() -> ctypes.CDLL:
         L.qift_diag_ratio_scan_workspace_bytes.restype = sz
         L.qift_diag_ratio_scan_workspace_bytes.argtypes = [ctypes.c_longlong, ci]
         L.qift_diag_ratio_scan.argtypes = [vp, ctypes.c_longlong, vp, ci, vp, vp, vp, sz, vp]
+        L.qift_selftest_wait_timeout.argtypes = [ci, ctypes.c_uint, vp]
         for name in EXPORTS:
             if name not in ("qift_diag_ratio_scan_workspace_bytes", "qift_status_string", "qift_packed_bytes", "qift_workspace_bytes",
                             "qift_forward_scratch_bytes", "qift_group_plan_bytes", "qift_static_scratch_bytes",
@@ -228,6 +230,12 @@ def qift_device_status():
     detail = ctypes.c_uint32(0)
     rc = lib().qift_device_status(_stream(), ctypes.byref(detail))
     return rc, detail.value
+
+
+def qift_selftest_wait_timeout(which: int, limit_us: int):
+    """Enqueues a kernel whose bounded wait runs out after limit_us (0: a lone waiting CTA; 1: the CTA-pair
+    prefill GEMM starved of its loads); qift_device_status() then reports ERR_TIMEOUT once."""
+    _check(lib().qift_selftest_wait_timeout(which, limit_us, _stream()), "qift_selftest_wait_timeout")
 
 
 def _dt(t):

@@ -111,16 +111,17 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
     return t;
 }
 // Bounded wait: polls (each poll may be parked by the hardware for up to its time hint) until the
-// phase completes or two seconds of wall time have passed; then records the site and returns false.
-// Callers skip their remaining work on false.
+// phase completes or `limit_ns` of wall time have passed (two seconds unless the launch says otherwise);
+// then records the site and returns false.  Callers skip their remaining work on false.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int site) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int site, uint64_t limit_ns = kWaitLimitNs) {
     uint64_t t0 = 0;
+    const uint32_t hint = limit_ns < 1000000ull ? static_cast<uint32_t>(limit_ns) : 1000000u;
     for (;;) {
-        if (mbar_try_wait(bar, parity, 1000000u)) return true;
+        if (mbar_try_wait(bar, parity, hint)) return true;
         const uint64_t t = global_timer_ns();
         if (t0 == 0) t0 = t;
-        else if (t - t0 > kWaitLimitNs) break;
+        else if (t - t0 > limit_ns) break;
     }
     report_timeout(site);
     return false;

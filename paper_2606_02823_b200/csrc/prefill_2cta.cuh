@@ -87,6 +87,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int n_tiles = (p.N + BN - 1) / BN;
     const int num_tiles = m_tiles * n_tiles;
     const int k_blocks = (p.K + kGemmBK - 1) / kGemmBK;
+    const uint64_t limit = p.wait_limit_ns ? p.wait_limit_ns : kWaitLimitNs;
 
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
@@ -117,7 +118,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
-        if (lane == 0) {
+        if (lane == 0 && !p.starve) {
             uint32_t it = 0;
             for (int tile = pair; tile < num_tiles && !*fail; tile += npairs) {
                 const int mt = tile % m_tiles, nt = tile / m_tiles;
@@ -125,7 +126,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 const int n0 = nt * BN + static_cast<int>(rank) * (BN / 2);          // this CTA's half of the channels
                 for (int kb = 0; kb < k_blocks; ++kb, ++it) {
                     const int s = it % kPairStages;
-                    if (it >= kPairStages && !mbar_wait(&empty[s], ((it / kPairStages) - 1) & 1, 30)) {
+                    if (it >= kPairStages && !mbar_wait(&empty[s], ((it / kPairStages) - 1) & 1, 30, limit)) {
                         *fail = 1;
                         break;
                     }
@@ -141,7 +142,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             uint32_t it = 0, tcount = 0;
             for (int tile = pair; tile < num_tiles && !*fail; tile += npairs, ++tcount) {
                 const int buf = tcount & 1;
-                if (tcount >= 2 && !mbar_wait(&tempty[buf], ((tcount >> 1) - 1) & 1, 31)) {
+                if (tcount >= 2 && !mbar_wait(&tempty[buf], ((tcount >> 1) - 1) & 1, 31, limit)) {
                     *fail = 1;
                     break;
                 }
@@ -149,7 +150,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 const uint32_t d_addr = tmem_base + buf * BN;
                 for (int kb = 0; kb < k_blocks; ++kb, ++it) {
                     const int s = it % kPairStages;
-                    if (!mbar_wait(&full[s], (it / kPairStages) & 1, 32)) {
+                    if (!mbar_wait(&full[s], (it / kPairStages) & 1, 32, limit)) {
                         *fail = 1;
                         break;
                     }
@@ -173,7 +174,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         for (int tile = pair; tile < num_tiles; tile += npairs, ++tcount) {
             const int mt = tile % m_tiles, nt = tile / m_tiles;
             const int buf = tcount & 1;
-            if (!mbar_wait(&tfull[buf], (tcount >> 1) & 1, 33)) {
+            if (!mbar_wait(&tfull[buf], (tcount >> 1) & 1, 33, limit)) {
                 *fail = 1;
                 break;
             }

@@ -4,6 +4,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstdlib>
+#include <mutex>
 
 #include "common.cuh"
 #include "decode.cuh"
@@ -81,23 +82,40 @@ cudaError_t launch_pdl_pairs(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
     return launch_pdl_cluster(kernel, 2u, grid, block, smem, st, std::forward<Args>(args)...);
 }
 
+// Host-side caches are keyed by the current device and guarded by one mutex: the shared-memory opt-in
+// is an attribute of a kernel in ONE context, and grids are sized for the device that runs them.
+constexpr int kMaxDevices = 64;
+inline std::mutex& cache_mutex() {
+    static std::mutex m;
+    return m;
+}
+inline int current_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+    return dev;
+}
+
 template <typename K>
 cudaError_t allow_smem(K kernel, size_t bytes) {
     if (bytes <= 32 * 1024) return cudaSuccess;  // static shared memory counts against the 48 KiB default too
     struct Entry {
         const void* fn;
+        int dev;
         size_t bytes;
     };
-    static Entry table[64];
+    constexpr int kEntries = 256;
+    static Entry table[kEntries];
     static int used = 0;
     const void* key = reinterpret_cast<const void*>(kernel);
+    const int dev = current_device();
+    std::lock_guard<std::mutex> lock(cache_mutex());
     Entry* slot = nullptr;
     for (int i = 0; i < used; ++i)
-        if (table[i].fn == key) slot = &table[i];
+        if (table[i].fn == key && table[i].dev == dev) slot = &table[i];
     if (slot && bytes <= slot->bytes) return cudaSuccess;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
     if (e != cudaSuccess) return e;
-    if (!slot && used < 64) slot = &table[used++], slot->fn = key;
+    if (!slot && used < kEntries) slot = &table[used++], slot->fn = key, slot->dev = dev;
     if (slot) slot->bytes = bytes;
     return e;
 }
@@ -189,14 +207,15 @@ bool make_i8_map(CUtensorMap* map, const void* base, int rows, int K, int box_ro
 }
 
 int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
+    static int count[kMaxDevices] = {};
+    const int dev = current_device();
+    std::lock_guard<std::mutex> lock(cache_mutex());
+    if (!count[dev]) {
+        int n = 0;
         cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
+        count[dev] = n > 0 ? n : 148;
     }
-    return n;
+    return count[dev];
 }
 
 template <int BN>
@@ -920,15 +939,16 @@ namespace {
 constexpr size_t kStaticScratchBytes = size_t(16) << 20;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
-void* g_static_scratch_addr[kMaxDevices] = {};
+void* g_static_scratch_addr[qift::kMaxDevices] = {};
 
-// Device address of the array on the current device; looked up once per device.
+// Device address of the array on the current device; looked up once per device (primary context, no
+// device reset in between).
 cudaError_t static_scratch_address(void** out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (dev < 0 || dev >= qift::kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(qift::cache_mutex());
     if (!g_static_scratch_addr[dev]) {
         void* ptr = nullptr;
         e = cudaGetSymbolAddress(&ptr, g_static_scratch);
@@ -948,6 +968,11 @@ int qift_w2a4_linear_static(const uint32_t* packed, const float* s_n, int levels
                             int N, int K, void* Y, int y_dtype, int32_t* acc_debug, void* stream) {
     if (levels != QIFT_LEVELS_MNZ && levels != QIFT_LEVELS_POT && levels != QIFT_LEVELS_SYM) return QIFT_ERR_INVALID_ARG;
     if (!packed || !s_n || !q_a || !s_a || !Y || M <= 0 || N <= 0 || K <= 0) return QIFT_ERR_INVALID_ARG;
+    if (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16) return QIFT_ERR_INVALID_ARG;
+    if (K % 16 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(packed) || !aligned16(s_n) || !aligned16(q_a) || !aligned16(s_a) || !aligned16(Y) ||
+        (acc_debug && !aligned16(acc_debug)))
+        return QIFT_ERR_ALIGNMENT;
     if (static_cast<size_t>(N) * static_cast<size_t>(K) > kStaticScratchBytes) {
         std::fprintf(stderr, "qift_w2a4_linear_static: N*K = %zu bytes of scratch needed, the built-in array holds %zu\n",
                      static_cast<size_t>(N) * static_cast<size_t>(K), kStaticScratchBytes);
@@ -1109,6 +1134,43 @@ int qift_device_status(void* stream, uint32_t* detail) {
 }
 
 }  // extern "C"
+
+namespace qift {
+constexpr unsigned int kSiteProbe = 0x7e;
+// One thread waits, with the given bound, for a phase of an mbarrier that nobody completes.
+__global__ void wait_probe_kernel(uint64_t limit_ns) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_wait(&bar, 0, kSiteProbe, limit_ns);
+}
+}  // namespace qift
+
+extern "C" int qift_selftest_wait_timeout(int which, unsigned int limit_us, void* stream) {
+    if ((which != 0 && which != 1) || limit_us == 0 || limit_us > 1000000u) return QIFT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint64_t limit_ns = static_cast<uint64_t>(limit_us) * 1000ull;
+    if (which == 0) {
+        wait_probe_kernel<<<1, 32, 0, st>>>(limit_ns);
+        return cuda_status(cudaGetLastError());
+    }
+    // The CTA-pair GEMM on one 256 x 256 x 128 tile whose producers issue no loads: the MMA thread's wait for
+    // operands and the epilogue warps' wait for the accumulator run out, every role leaves its loop, both CTAs
+    // meet at the closing cluster barrier and tensor memory is freed.  Operands live in the built-in scratch;
+    // nothing is read or written (no load is issued and no accumulator ever completes).
+    void* scratch = nullptr;
+    const cudaError_t e = static_scratch_address(&scratch);
+    if (e != cudaSuccess) return cuda_status(e);
+    unsigned char* base = static_cast<unsigned char*>(scratch);
+    CUtensorMap ma, mb;
+    if (!make_i8_map(&ma, base, 256, 128, kGemmBM) || !make_i8_map(&mb, base + 32768, 256, 128, 128)) return QIFT_ERR_CUDA;
+    GemmParams gp{reinterpret_cast<const float*>(base + 69632), reinterpret_cast<const float*>(base + 65536), base + 131072, nullptr,
+                  256, 256, 128, 1, limit_ns, 1};
+    return launch_gemm_pairs<256>(ma, mb, gp, st);
+}
 
 namespace {
 // Token splits of the decode attention: one resident wave of CTAs, whole 64-token rounds of the four

@@ -12,6 +12,9 @@ fp64, cast to fp32 at the end.  Any slice of a tensor can therefore be drawn on 
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 
 _M64 = np.uint64(0xFFFFFFFFFFFFFFFF)
@@ -56,20 +59,41 @@ def uniforms(seed: int, tensor_id: int, n: int, offset: int = 0):
     return u, v
 
 
+_CHUNK = 1 << 18   # elements drawn per task: the temporaries of a task stay in cache
+
+
+def _draw(variate, seed: int, tensor_id: int, shape, offset: int):
+    """Fills an fp64 array element by element from the counter-based stream.  Element i depends on
+    (seed, tensor_id, offset + i) only, so the array is cut into chunks that worker threads draw
+    independently (numpy releases the interpreter lock inside its loops); the values do not depend
+    on the chunking."""
+    n = int(np.prod(shape))
+    out = np.empty(n, dtype=np.float64)
+
+    def task(lo):
+        hi = min(n, lo + _CHUNK)
+        u, v = uniforms(seed, tensor_id, hi - lo, offset + lo)
+        out[lo:hi] = variate(u, v)
+
+    starts = range(0, n, _CHUNK)
+    if n <= _CHUNK:
+        for lo in starts:
+            task(lo)
+    else:
+        with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as pool:
+            list(pool.map(task, starts))
+    return out.reshape(shape)
+
+
 def normal(seed: int, tensor_id: int, shape, offset: int = 0):
     """iid N(0,1), fp64 (Box-Muller cosine branch)."""
-    n = int(np.prod(shape))
-    u, v = uniforms(seed, tensor_id, n, offset)
-    z = np.sqrt(-2.0 * np.log(u)) * np.cos(2.0 * np.pi * v)
-    return z.reshape(shape)
+    return _draw(lambda u, v: np.sqrt(-2.0 * np.log(u)) * np.cos(2.0 * np.pi * v), seed, tensor_id, shape, offset)
 
 
 def student_t(seed: int, tensor_id: int, shape, df: float = 5.0, offset: int = 0):
     """iid Student-t(df), fp64 (Bailey's polar form: sqrt(df (u^(-2/df) - 1)) cos(2 pi v))."""
-    n = int(np.prod(shape))
-    u, v = uniforms(seed, tensor_id, n, offset)
-    t = np.sqrt(df * (np.power(u, -2.0 / df) - 1.0)) * np.cos(2.0 * np.pi * v)
-    return t.reshape(shape)
+    return _draw(lambda u, v: np.sqrt(df * (np.power(u, -2.0 / df) - 1.0)) * np.cos(2.0 * np.pi * v), seed, tensor_id,
+                 shape, offset)
 
 
 def choose_channels(seed: int, tensor_id: int, K: int, count: int):

@@ -193,3 +193,71 @@ def test_config5_mixed_stack_32_layers_scaled_shapes():
              ("gate", 768, 256), ("up", 768, 256), ("down", 256, 768)]
     assert run_mixed_stack(small, 32, 16, 1) == 224
     assert run_mixed_stack(small, 4, 2, 40) == 28           # the same stack through the prefill route
+
+
+# ------------------------------------------------------------------- config 5 at M = 2048, full shapes
+def prefill_module_sampled(pool, W, lv, x_bf16, seed, rows_n=64, cols_n=256):
+    """One module at M = 2048 through the AUTO route (code expansion into the int8 scratch, then the CTA-pair
+    tcgen05 GEMM), bf16 in and out.  INT32 accumulators and bf16 bits are compared with the oracle on `rows_n`
+    seeded token rows x every channel and on every token x `cols_n` seeded channels.  The oracle jobs go to
+    `pool` (the oracle itself stays single-threaded; independent calls run side by side) and are returned as
+    thunks that do the comparison."""
+    N, K = W.shape
+    M = x_bf16.shape[0]
+    B = synth.had_block_for(K)
+    p_ref, s_n, codes = oracle.pack_weights(W, lv, oracle.SCALE_ABSMAX)
+    packed, s_d = dev(p_ref.view(np.int32)), dev(s_n)
+    x_ref = oracle.bf16_to_f32(x_bf16.view(torch.int16).cpu().numpy().view(np.uint16))
+    q_a, s_a = qift.qift_quantize_act(x_bf16, B, CLIP)
+    q_ref, sa_ref = oracle.quantize_act(x_ref, B, CLIP)
+    assert np.array_equal(q_a.cpu().numpy(), q_ref) and np.array_equal(s_a.cpu().numpy(), sa_ref)
+    if lv == qift.INT4:
+        y, acc = qift.qift_w4a4_linear(packed, s_d, q_a, s_a, out_dtype=torch.bfloat16, want_acc=True)
+    else:
+        y, acc = qift.qift_w2a4_linear(packed, s_d, lv, q_a, s_a, out_dtype=torch.bfloat16, want_acc=True)
+    rng = np.random.default_rng(seed)
+    rows = np.sort(rng.choice(M, rows_n, replace=False))
+    cols = np.sort(rng.choice(N, cols_n, replace=False))
+    rows_t, cols_t = torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()
+    yb = y.view(torch.int16)
+    got = (acc[rows_t].cpu().numpy(), yb[rows_t].cpu().numpy().view(np.uint16),
+           acc[:, cols_t].cpu().numpy(), yb[:, cols_t].cpu().numpy().view(np.uint16))
+    assert int(acc.abs().max()) <= K * 8 * 8           # holds at any size: |level| <= 8, |q_a| <= 8
+    job_r = pool.submit(oracle.linear, codes, lv, s_n, q_ref[rows], sa_ref[rows], True)
+    job_c = pool.submit(oracle.linear, np.ascontiguousarray(codes[cols]), lv, s_n[cols], q_ref, sa_ref, True)
+
+    def finish():
+        y_r, acc_r = job_r.result()
+        y_c, acc_c = job_c.result()
+        assert np.array_equal(got[0], acc_r) and np.array_equal(got[1], y_r)
+        assert np.array_equal(got[2], acc_c) and np.array_equal(got[3], y_c)
+    return finish
+
+
+@pytest.mark.parametrize("lv", [qift.INT4, qift.MNZ], ids=["w4a4_layer", "w2a4_layer"])
+def test_config5_prefill_m2048_full_shapes_sampled(lv):
+    # one layer of the mixed stack at the LLaMA-2-7B shapes and M = 2048: all seven modules, each on its own input
+    from concurrent.futures import ThreadPoolExecutor
+    M = 2048
+    with ThreadPoolExecutor(max_workers=8) as pool:
+        pending = []
+        for i, (name, N, K) in enumerate(synth.LLAMA2_7B):
+            W = synth.gaussian_weights(synth.config_seed(5, i, 0) + 7000 + lv, N, K)
+            x, _ = synth.activations(synth.config_seed(5, i, 1) + 7000, M, K, round(0.01 * K))
+            pending.append(prefill_module_sampled(pool, W, lv, dev(x).to(torch.bfloat16), 50 + i))
+        clean()
+        for finish in pending:
+            finish()
+
+
+@pytest.mark.parametrize("lv", [qift.POT, qift.SYM], ids=["pot", "sym"])
+def test_prefill_m2048_gate_shape_other_level_sets(lv):
+    # the remaining two-bit sets once at full size through the same route (11008 channels: 224-wide tiles, 43 of them)
+    from concurrent.futures import ThreadPoolExecutor
+    M, (name, N, K) = 2048, synth.LLAMA2_7B[4]
+    W = synth.gaussian_weights(synth.config_seed(5, 4, 0) + 7100 + lv, N, K)
+    x, _ = synth.activations(synth.config_seed(5, 4, 1) + 7100, M, K, round(0.01 * K))
+    with ThreadPoolExecutor(max_workers=2) as pool:
+        finish = prefill_module_sampled(pool, W, lv, dev(x).to(torch.bfloat16), 60 + lv)
+        clean()
+        finish()

@@ -187,6 +187,55 @@ int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_blo
                       const uint32_t* packed, const float* s_n, int levels, int N, void* Y_host,
                       int y_dtype, void* scratch, size_t scratch_bytes, void* stream);
 
+/* ---- Several products of ONE activation, weights decoded ahead of their use --------------------
+ * (Sec. 3.1: the layer pipeline; the paper describes no kernels, so the scheduling is this library's.)
+ * In a transformer layer q / k / v read the same activation, and so do gate / up: it needs rotating and
+ * quantizing once.  qift_forward_multi runs S2 + S3 once on X and then S4 + S5 for every listed output.
+ * With more than 512 token rows the products run as ONE launch of the CTA-pair tensor-core GEMM over the
+ * channel tiles of all outputs, reading int8 levels decoded from the packed codes into `levels_buf`
+ * (qift_levels_bytes; output i at the sum of the earlier outputs' N*K rounded up to 1 KiB each).
+ *
+ * Decoding ahead: the decoding of a product's codes needs nothing but the codes, so a call can do it for
+ * the NEXT call while its own GEMM runs (extra warps of the GEMM kernel; the GEMM leaves most issue slots
+ * free).  Pass in `ahead` the outputs (only packed and N are read), K and level set of the next call and
+ * the buffer that call will pass as its levels_buf; the next call then passes levels_ready = 1 and skips its
+ * own decoding pass.  A caller walking a layer stack alternates two levels buffers.  The first call of a
+ * chain (levels_ready = 0) decodes its own codes before its GEMM, as qift_w2a4_linear does.
+ *
+ *   X            dev [M,K] fp32 or bf16;  had_block, clip_ratio as for qift_quantize_act
+ *   outputs      HOST array of 1..4 outputs: packed / s_n from qift_pack_weights (all with this K and
+ *                level set), Y dev [M,N] (fp32 or bf16 per y_dtype), acc_debug dev int32 [M,N] or NULL
+ *   scratch      dev, >= qift_forward_multi_scratch_bytes(...), 256-byte aligned: q_a, s_a and (M <= 512)
+ *                the workspace of the per-output routes; undefined afterwards
+ *   levels_buf   dev, >= qift_levels_bytes(K, outputs, count), 256-byte aligned; needed when M > 512.
+ *                levels_ready = 1 promises it already holds the decoded levels of exactly these outputs
+ *                (written by the previous call's `ahead`); nothing can check that promise
+ *   ahead        HOST, or NULL.  With M <= 512 the call still honours it (separate decoding launches).
+ * Results are bit-identical to qift_quantize_act + qift_w2a4_linear / qift_w4a4_linear per output.
+ * Errors: INVALID_ARG (null pointers, count outside 1..4, enums), UNSUPPORTED_SHAPE, ALIGNMENT,
+ * WORKSPACE (scratch or a levels buffer missing or too small), CUDA. */
+typedef struct qift_linear_output {
+    const uint32_t* packed; /* dev, from qift_pack_weights            */
+    const float* s_n;       /* dev [N]                                */
+    void* Y;                /* dev [M,N]                              */
+    int32_t* acc_debug;     /* dev [M,N] INT32 accumulators, or NULL  */
+    int N;
+    int reserved;
+} qift_linear_output;
+typedef struct qift_decode_ahead {
+    const qift_linear_output* outputs; /* host; the next call's outputs (packed and N are read) */
+    int count, K, levels;
+    int reserved;
+    void* levels_buf;                  /* dev; the next call's levels_buf                        */
+    size_t levels_bytes;
+} qift_decode_ahead;
+size_t qift_levels_bytes(int K, const qift_linear_output* outputs, int count);
+size_t qift_forward_multi_scratch_bytes(int M, int K, int levels, const qift_linear_output* outputs, int count);
+int qift_forward_multi(const void* X, int x_dtype, int M, int K, int had_block, float clip_ratio, int levels,
+                       const qift_linear_output* outputs, int count, int y_dtype, void* scratch, size_t scratch_bytes,
+                       void* levels_buf, size_t levels_bytes, int levels_ready, const qift_decode_ahead* ahead,
+                       void* stream);
+
 /* ---- Grouped decode path -----------------------------------------------------------------------
  * One persistent launch serves a list of independent layer problems that share M (<= 64 token rows),
  * the level set, the dtypes and the clip ratio -- e.g. all linear modules of one decode step.  A W2

@@ -32,7 +32,7 @@ EXPORTS = [
     "qift_kv4_quantize", "qift_kv4_attention_workspace_bytes", "qift_kv4_attention_decode",
     "qift_expand_weights", "qift_expanded_linear",
     "qift_diag_grid_quantize", "qift_diag_bucket_stats", "qift_diag_ratio_scan_workspace_bytes", "qift_diag_ratio_scan",
-    "qift_selftest_wait_timeout",
+    "qift_selftest_wait_timeout", "qift_levels_bytes", "qift_forward_multi_scratch_bytes", "qift_forward_multi",
 ]
 
 _lib = None
@@ -96,10 +96,16 @@ def lib() -> ctypes.CDLL:
         L.qift_diag_ratio_scan_workspace_bytes.argtypes = [ctypes.c_longlong, ci]
         L.qift_diag_ratio_scan.argtypes = [vp, ctypes.c_longlong, vp, ci, vp, vp, vp, sz, vp]
         L.qift_selftest_wait_timeout.argtypes = [ci, ctypes.c_uint, vp]
+        L.qift_levels_bytes.restype = sz
+        L.qift_levels_bytes.argtypes = [ci, vp, ci]
+        L.qift_forward_multi_scratch_bytes.restype = sz
+        L.qift_forward_multi_scratch_bytes.argtypes = [ci, ci, ci, vp, ci]
+        L.qift_forward_multi.argtypes = [vp, ci, ci, ci, ci, cf, ci, vp, ci, ci, vp, sz, vp, sz, ci, vp, vp]
         for name in EXPORTS:
             if name not in ("qift_diag_ratio_scan_workspace_bytes", "qift_status_string", "qift_packed_bytes", "qift_workspace_bytes",
                             "qift_forward_scratch_bytes", "qift_group_plan_bytes", "qift_static_scratch_bytes",
-                            "qift_workspace_bytes_route", "qift_kv4_attention_workspace_bytes"):
+                            "qift_workspace_bytes_route", "qift_kv4_attention_workspace_bytes", "qift_levels_bytes",
+                            "qift_forward_multi_scratch_bytes"):
                 getattr(L, name).restype = ci
         _lib = L
     return _lib
@@ -271,6 +277,64 @@ def qift_forward_host(X_host, had_block, packed, s_n, levels, out_host, clip_rat
     """Whole layer with X and Y in (pinned) host tensors; Y is valid after the stream is synchronized."""
     assert not X_host.is_cuda and not out_host.is_cuda and X_host.is_contiguous() and out_host.is_contiguous()
     return _forward(lib().qift_forward_host, X_host, had_block, clip_ratio, packed, s_n, levels, out_host, scratch)
+
+
+class LinearOutput(ctypes.Structure):
+    """Mirror of qift_linear_output."""
+    _fields_ = [("packed", ctypes.c_void_p), ("s_n", ctypes.c_void_p), ("Y", ctypes.c_void_p), ("acc_debug", ctypes.c_void_p),
+                ("N", ctypes.c_int), ("reserved", ctypes.c_int)]
+
+
+class DecodeAhead(ctypes.Structure):
+    """Mirror of qift_decode_ahead."""
+    _fields_ = [("outputs", ctypes.c_void_p), ("count", ctypes.c_int), ("K", ctypes.c_int), ("levels", ctypes.c_int),
+                ("reserved", ctypes.c_int), ("levels_buf", ctypes.c_void_p), ("levels_bytes", ctypes.c_size_t)]
+
+
+def _outputs_array(weights, ys=None, accs=None):
+    """weights: list of (packed, s_n) -> ctypes array of qift_linear_output (Y / acc filled when given)."""
+    arr = (LinearOutput * len(weights))()
+    for i, (packed, s_n) in enumerate(weights):
+        arr[i] = LinearOutput(_dev(packed).data_ptr(), _dev(s_n, torch.float32).data_ptr(),
+                              None if ys is None else ys[i].data_ptr(),
+                              None if accs is None or accs[i] is None else accs[i].data_ptr(), s_n.shape[0], 0)
+    return arr
+
+
+def qift_levels_bytes(K: int, weights) -> int:
+    """Bytes of the int8 levels buffer for a list of (packed, s_n) weights sharing K."""
+    arr = _outputs_array(weights)
+    return int(lib().qift_levels_bytes(K, ctypes.addressof(arr), len(weights)))
+
+
+def qift_forward_multi(X, had_block: int, weights, levels: int, clip_ratio: float = 0.9, out_dtype=torch.float32,
+                       want_acc: bool = False, scratch=None, levels_buf=None, levels_ready: bool = False, ahead=None, outs=None):
+    """One activation X [M,K], several products: weights = [(packed, s_n), ...] (1..4) -> ([Y_i [M,N_i]], [acc_i or None]).
+    levels_buf: uint8 tensor of qift_levels_bytes(K, weights) bytes (allocated when omitted; needed for M > 512);
+    levels_ready: it already holds these weights' decoded levels (written through a previous call's `ahead`);
+    ahead = (next_weights, next_K, next_levels, next_levels_buf): decode the next call's codes during this one."""
+    _dev(X)
+    M, K = X.shape
+    ys = outs if outs is not None else [torch.empty((M, s_n.shape[0]), dtype=out_dtype, device=X.device) for _, s_n in weights]
+    accs = [torch.empty((M, s_n.shape[0]), dtype=torch.int32, device=X.device) if want_acc else None for _, s_n in weights]
+    arr = _outputs_array(weights, ys, accs)
+    L = lib()
+    need = int(L.qift_forward_multi_scratch_bytes(M, K, levels, ctypes.addressof(arr), len(weights)))
+    if scratch is None:
+        scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=X.device)
+    if levels_buf is None:
+        assert not levels_ready
+        levels_buf = torch.empty(max(qift_levels_bytes(K, weights), 256), dtype=torch.uint8, device=X.device)
+    ah, keep = None, None
+    if ahead is not None:
+        nw, nK, nlv, nbuf = ahead
+        keep = _outputs_array(nw)
+        ah = DecodeAhead(ctypes.addressof(keep), len(nw), nK, nlv, 0, _dev(nbuf).data_ptr(), nbuf.numel())
+    _check(L.qift_forward_multi(_ptr(X), _dt(X), M, K, had_block, clip_ratio, levels, ctypes.addressof(arr), len(weights),
+                                _dt(ys[0]), _ptr(_dev(scratch)), scratch.numel(), _ptr(_dev(levels_buf)), levels_buf.numel(),
+                                1 if levels_ready else 0, None if ah is None else ctypes.addressof(ah), _stream()),
+           "qift_forward_multi")
+    return ys, accs
 
 
 class GroupProblem(ctypes.Structure):

@@ -149,8 +149,6 @@ struct GemmParams {
     int32_t* acc_debug;
     int M, N, K;
     int y_bf16;
-    uint64_t wait_limit_ns;  // bound of every device-side wait of the launch; 0 = the default (kWaitLimitNs)
-    int starve;              // self-test only (qift_selftest_wait_timeout): the producers issue no loads
 };
 
 template <int BN>

@@ -244,29 +244,85 @@ int launch_expand(const uint32_t* packed, int N, int K, int8_t* out, cudaStream_
 // tile is re-read from L2 for every channel tile, so narrow tiles are not proportionally cheaper):
 // cost ~ width + 284.  14336 channels then run 7 full rounds of 224-wide tiles instead of the
 // 6.05 -> 7 rounds of 256-wide ones; 1024 channels one round of 128-wide tiles.
-int pair_tile_width(int M, int N) {
+int pair_tile_width(int M, const int* N, int count) {
     const int widths[3] = {256, 224, 128};
     const int pair_count = sm_count() / 2, m_pairs = (M + 2 * kGemmBM - 1) / (2 * kGemmBM);
     int bn = 256;
     long best = -1;
     for (int w : widths) {
-        const long tiles = static_cast<long>(m_pairs) * ((N + w - 1) / w);
+        long tiles = 0;
+        for (int i = 0; i < count; ++i) tiles += static_cast<long>(m_pairs) * ((N[i] + w - 1) / w);
         const long cost = ((tiles + pair_count - 1) / pair_count) * (w + 284);
         if (best < 0 || cost < best) best = cost, bn = w;
     }
     return bn;
 }
+inline int pair_tile_width(int M, int N) { return pair_tile_width(M, &N, 1); }
+
+// Host description of one launch of the CTA-pair GEMM: up to kPairMaxSegments products that share the
+// activations, and up to kPairMaxSegments side jobs (codes of a later product decoded meanwhile).
+struct PairCall {
+    const int8_t* q_a;
+    const float* s_a;
+    int M, K, y_bf16;
+    int nseg;
+    struct {
+        const int8_t* wexp;  // int8 [N, K]
+        const float* s_n;
+        void* Y;
+        int32_t* acc_debug;
+        int N;
+    } seg[kPairMaxSegments];
+    int njobs, job_K;
+    struct {
+        const uint32_t* packed;
+        int8_t* out;
+        int N, levels;
+    } job[kPairMaxSegments];
+    uint64_t wait_limit_ns;
+    int starve;
+};
 
 template <int BN>
-int launch_gemm_pairs(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& gp, cudaStream_t st) {
+int launch_gemm_pairs(const PairParams& pp, int tiles, cudaStream_t st) {
     auto kernel = gemm_i8_pair_kernel<BN>;
     const size_t smem = pair_smem_bytes<BN>();
     cudaError_t e = allow_smem(kernel, smem);
     if (e != cudaSuccess) return cuda_status(e);
-    const int tiles = ((gp.M + 2 * kGemmBM - 1) / (2 * kGemmBM)) * ((gp.N + BN - 1) / BN);
     int pairs = sm_count() / 2;
-    if (pairs > tiles) pairs = tiles;
-    return cuda_status(launch_pdl_pairs(kernel, dim3(2 * pairs), dim3(kPairThreads), smem, st, ma, mb, gp));
+    if (pairs > tiles && pp.units == 0) pairs = tiles;  // with side jobs every SM takes its share of them
+    return cuda_status(launch_pdl_pairs(kernel, dim3(2 * pairs), dim3(kPairThreads), smem, st, pp));
+}
+
+int run_pair_gemm(const PairCall& c, cudaStream_t st) {
+    if (c.nseg < 1 || c.nseg > kPairMaxSegments || c.njobs < 0 || c.njobs > kPairMaxSegments) return QIFT_ERR_INVALID_ARG;
+    PairParams pp = {};
+    int widths[kPairMaxSegments];
+    for (int i = 0; i < c.nseg; ++i) widths[i] = c.seg[i].N;
+    const int bn = pair_tile_width(c.M, widths, c.nseg);
+    if (!make_i8_map(&pp.map_a, c.q_a, c.M, c.K, kGemmBM)) return QIFT_ERR_CUDA;
+    int tiles = 0;
+    for (int i = 0; i < c.nseg; ++i) {
+        // each CTA of a pair loads its own 128 tokens and half of the tile's channels
+        if (!make_i8_map(&pp.map_b[i], c.seg[i].wexp, c.seg[i].N, c.K, bn / 2)) return QIFT_ERR_CUDA;
+        pp.seg[i] = PairSegment{c.seg[i].s_n, c.seg[i].Y, c.seg[i].acc_debug, c.seg[i].N, tiles};
+        tiles += (c.seg[i].N + bn - 1) / bn;
+    }
+    pp.s_a = c.s_a, pp.M = c.M, pp.K = c.K, pp.y_bf16 = c.y_bf16, pp.nseg = c.nseg, pp.n_tiles = tiles;
+    pp.wait_limit_ns = c.wait_limit_ns, pp.starve = c.starve;
+    int units = 0;
+    for (int i = 0; i < c.njobs; ++i) {
+        const int words = c.job_K / codes_per_word(c.job[i].levels);
+        pp.job[i] = SideJob{c.job[i].packed, c.job[i].out, c.job[i].N, words, units, c.job[i].levels};
+        units += ((c.job[i].N + kSideUnitRows - 1) / kSideUnitRows) * ((words + kSideUnitWords - 1) / kSideUnitWords);
+    }
+    pp.njobs = c.njobs, pp.units = units;
+    const int all_tiles = ((c.M + 2 * kGemmBM - 1) / (2 * kGemmBM)) * tiles;
+    switch (bn) {
+        case 256: return launch_gemm_pairs<256>(pp, all_tiles, st);
+        case 224: return launch_gemm_pairs<224>(pp, all_tiles, st);
+        default: return launch_gemm_pairs<128>(pp, all_tiles, st);
+    }
 }
 
 int run_expand(const uint32_t* packed, int lv, int N, int K, int8_t* wexp, cudaStream_t st) {
@@ -298,17 +354,14 @@ int run_i8_gemm(const int8_t* wexp, const float* s_n, const int8_t* q_a, const f
                 int y_bf16, int32_t* acc_debug, cudaStream_t st, bool pairs) {
     const int m_tiles = (M + kGemmBM - 1) / kGemmBM;
     const bool narrow = m_tiles * ((N + 255) / 256) < sm_count();
+    if (pairs) {
+        PairCall c = {};
+        c.q_a = q_a, c.s_a = s_a, c.M = M, c.K = K, c.y_bf16 = y_bf16, c.nseg = 1;
+        c.seg[0].wexp = wexp, c.seg[0].s_n = s_n, c.seg[0].Y = Y, c.seg[0].acc_debug = acc_debug, c.seg[0].N = N;
+        return run_pair_gemm(c, st);
+    }
     CUtensorMap ma, mb;
     GemmParams gp{s_n, s_a, Y, acc_debug, M, N, K, y_bf16};
-    if (pairs) {  // each CTA of a pair loads its own 128 tokens and half of the tile's channels
-        const int bn = pair_tile_width(M, N);
-        if (!make_i8_map(&ma, q_a, M, K, kGemmBM) || !make_i8_map(&mb, wexp, N, K, bn / 2)) return QIFT_ERR_CUDA;
-        switch (bn) {
-            case 256: return launch_gemm_pairs<256>(ma, mb, gp, st);
-            case 224: return launch_gemm_pairs<224>(ma, mb, gp, st);
-            default: return launch_gemm_pairs<128>(ma, mb, gp, st);
-        }
-    }
     if (!make_i8_map(&ma, q_a, M, K, kGemmBM) || !make_i8_map(&mb, wexp, N, K, narrow ? 128 : 256)) return QIFT_ERR_CUDA;
     return narrow ? launch_gemm<128>(ma, mb, gp, st) : launch_gemm<256>(ma, mb, gp, st);
 }
@@ -659,6 +712,121 @@ int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_blo
                       void* stream) {
     return forward_impl(X_host, true, x_dtype, M, K, had_block, clip_ratio, packed, s_n, levels, N, Y_host, y_dtype, scratch,
                         scratch_bytes, stream);
+}
+
+// ------------------------------------------------------------------------- several products of one activation
+namespace {
+struct MultiLayout {
+    size_t q_off, sa_off, ws_off, total;
+};
+bool multi_outputs_ok(const qift_linear_output* o, int count, bool need_all) {
+    if (!o || count < 1 || count > kPairMaxSegments) return false;
+    for (int i = 0; i < count; ++i) {
+        if (!o[i].packed || o[i].N <= 0) return false;
+        if (need_all && (!o[i].s_n || !o[i].Y)) return false;
+    }
+    return true;
+}
+MultiLayout multi_layout(int M, int K, int levels, const qift_linear_output* o, int count) {
+    MultiLayout L;
+    size_t off = 0;
+    L.q_off = off, off += up1k(static_cast<size_t>(M) * K);
+    L.sa_off = off, off += up1k(static_cast<size_t>(M) * 4);
+    size_t ws = 0;
+    if (M <= kFusedPairMaxM)  // the routes below the pair GEMM bring their own (small) workspace needs
+        for (int i = 0; i < count; ++i) {
+            const size_t w = qift_workspace_bytes(M, o[i].N, K, levels);
+            if (w > ws) ws = w;
+        }
+    L.ws_off = off, off += ws;
+    L.total = off;
+    return L;
+}
+inline size_t levels_offset(int K, const qift_linear_output* o, int i) {  // of output i inside a levels buffer
+    size_t off = 0;
+    for (int j = 0; j < i; ++j) off += up1k(static_cast<size_t>(o[j].N) * K);
+    return off;
+}
+}  // namespace
+
+size_t qift_levels_bytes(int K, const qift_linear_output* outputs, int count) {
+    if (K <= 0 || !multi_outputs_ok(outputs, count, false)) return 0;
+    return levels_offset(K, outputs, count);
+}
+
+size_t qift_forward_multi_scratch_bytes(int M, int K, int levels, const qift_linear_output* outputs, int count) {
+    if (M <= 0 || K <= 0 || !valid_levels(levels) || !multi_outputs_ok(outputs, count, false)) return 0;
+    return multi_layout(M, K, levels, outputs, count).total;
+}
+
+int qift_forward_multi(const void* X, int x_dtype, int M, int K, int had_block, float clip_ratio, int levels,
+                       const qift_linear_output* outputs, int count, int y_dtype, void* scratch, size_t scratch_bytes,
+                       void* levels_buf, size_t levels_bytes, int levels_ready, const qift_decode_ahead* ahead, void* stream) {
+    if (!X || M <= 0 || K <= 0 || !valid_levels(levels) || !multi_outputs_ok(outputs, count, true)) return QIFT_ERR_INVALID_ARG;
+    if ((x_dtype != QIFT_F32 && x_dtype != QIFT_BF16) || (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16))
+        return QIFT_ERR_INVALID_ARG;
+    if (K % codes_per_word(levels) != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(X)) return QIFT_ERR_ALIGNMENT;
+    for (int i = 0; i < count; ++i)
+        if (!aligned16(outputs[i].packed) || !aligned16(outputs[i].s_n) || !aligned16(outputs[i].Y) ||
+            (outputs[i].acc_debug && !aligned16(outputs[i].acc_debug)))
+            return QIFT_ERR_ALIGNMENT;
+    if (ahead) {
+        if (!multi_outputs_ok(ahead->outputs, ahead->count, false) || ahead->K <= 0 || !valid_levels(ahead->levels) || !ahead->levels_buf)
+            return QIFT_ERR_INVALID_ARG;
+        if (ahead->K % 16 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+        if (ahead->levels_bytes < qift_levels_bytes(ahead->K, ahead->outputs, ahead->count)) return QIFT_ERR_WORKSPACE;
+        if ((reinterpret_cast<uintptr_t>(ahead->levels_buf) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
+        for (int i = 0; i < ahead->count; ++i)
+            if (!aligned16(ahead->outputs[i].packed)) return QIFT_ERR_ALIGNMENT;
+    }
+    const MultiLayout L = multi_layout(M, K, levels, outputs, count);
+    if (!scratch || scratch_bytes < L.total) return QIFT_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(scratch) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
+    const bool pair_route = M > kFusedPairMaxM && K % 16 == 0;
+    if (pair_route) {
+        if (!levels_buf || levels_bytes < qift_levels_bytes(K, outputs, count)) return QIFT_ERR_WORKSPACE;
+        if ((reinterpret_cast<uintptr_t>(levels_buf) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* base = static_cast<unsigned char*>(scratch);
+    int8_t* q_a = reinterpret_cast<int8_t*>(base + L.q_off);
+    float* s_a = reinterpret_cast<float*>(base + L.sa_off);
+    int rc = qift_quantize_act(X, x_dtype, M, K, had_block, clip_ratio, q_a, s_a, stream);
+    if (rc != QIFT_OK) return rc;
+    if (!pair_route) {
+        for (int i = 0; i < count; ++i) {
+            rc = linear_impl(outputs[i].packed, outputs[i].s_n, levels, q_a, s_a, M, outputs[i].N, K, outputs[i].Y, y_dtype,
+                             outputs[i].acc_debug, base + L.ws_off, L.total - L.ws_off, QIFT_ROUTE_AUTO, stream);
+            if (rc != QIFT_OK) return rc;
+        }
+        if (ahead)
+            for (int i = 0; i < ahead->count; ++i) {
+                int8_t* out = static_cast<int8_t*>(ahead->levels_buf) + levels_offset(ahead->K, ahead->outputs, i);
+                rc = run_expand(ahead->outputs[i].packed, ahead->levels, ahead->outputs[i].N, ahead->K, out, st);
+                if (rc != QIFT_OK) return rc;
+            }
+        return QIFT_OK;
+    }
+    PairCall c = {};
+    c.q_a = q_a, c.s_a = s_a, c.M = M, c.K = K, c.y_bf16 = (y_dtype == QIFT_BF16), c.nseg = count;
+    for (int i = 0; i < count; ++i) {
+        int8_t* wexp = static_cast<int8_t*>(levels_buf) + levels_offset(K, outputs, i);
+        if (!levels_ready) {
+            rc = run_expand(outputs[i].packed, levels, outputs[i].N, K, wexp, st);
+            if (rc != QIFT_OK) return rc;
+        }
+        c.seg[i].wexp = wexp, c.seg[i].s_n = outputs[i].s_n, c.seg[i].Y = outputs[i].Y, c.seg[i].acc_debug = outputs[i].acc_debug;
+        c.seg[i].N = outputs[i].N;
+    }
+    if (ahead) {
+        c.njobs = ahead->count, c.job_K = ahead->K;
+        for (int i = 0; i < ahead->count; ++i) {
+            c.job[i].packed = ahead->outputs[i].packed, c.job[i].N = ahead->outputs[i].N, c.job[i].levels = ahead->levels;
+            c.job[i].out = static_cast<int8_t*>(ahead->levels_buf) + levels_offset(ahead->K, ahead->outputs, i);
+        }
+    }
+    return run_pair_gemm(c, st);
 }
 
 // ------------------------------------------------------------------------------------------- grouped
@@ -1165,11 +1333,13 @@ extern "C" int qift_selftest_wait_timeout(int which, unsigned int limit_us, void
     const cudaError_t e = static_scratch_address(&scratch);
     if (e != cudaSuccess) return cuda_status(e);
     unsigned char* base = static_cast<unsigned char*>(scratch);
-    CUtensorMap ma, mb;
-    if (!make_i8_map(&ma, base, 256, 128, kGemmBM) || !make_i8_map(&mb, base + 32768, 256, 128, 128)) return QIFT_ERR_CUDA;
-    GemmParams gp{reinterpret_cast<const float*>(base + 69632), reinterpret_cast<const float*>(base + 65536), base + 131072, nullptr,
-                  256, 256, 128, 1, limit_ns, 1};
-    return launch_gemm_pairs<256>(ma, mb, gp, st);
+    PairCall c = {};
+    c.q_a = reinterpret_cast<const int8_t*>(base), c.s_a = reinterpret_cast<const float*>(base + 65536);
+    c.M = 256, c.K = 128, c.y_bf16 = 1, c.nseg = 1;
+    c.seg[0].wexp = reinterpret_cast<const int8_t*>(base + 32768), c.seg[0].s_n = reinterpret_cast<const float*>(base + 69632);
+    c.seg[0].Y = base + 131072, c.seg[0].acc_debug = nullptr, c.seg[0].N = 256;
+    c.wait_limit_ns = limit_ns, c.starve = 1;
+    return run_pair_gemm(c, st);
 }
 
 namespace {

@@ -16,6 +16,7 @@
 #include "prefill_2cta.cuh"
 #include "prefill_fused.cuh"
 #include "prefill_fused_pair.cuh"
+#include "quant_rows.cuh"
 #include "rotate_quant.cuh"
 
 namespace qift {
@@ -134,6 +135,59 @@ int check_rotation_shape(int K, int had_block, bool allow_none) {
     if (had_block == K && K % 28 == 0 && is_pow2(K / 28) && K / 28 >= 16) return QIFT_OK;  // H_28 (x) H_{K/28}
     if (had_block < 2 || !is_pow2(had_block) || K % had_block != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
     return QIFT_OK;
+}
+
+int sm_count();
+
+// ------------------------------------------------------------------------------ quantizer, rows in registers
+template <bool BF16, bool UPPER, int MID, int R2>
+int launch_quantize_rows_as(const void* X, int M, int K, int s0, float clip, float inv_sqrt_b, int8_t* q_a, float* s_a,
+                            cudaStream_t st) {
+    auto kernel = quantize_rows_kernel<BF16, UPPER, MID, R2>;
+    const int threads = ((K / 32) + 31) & ~31;
+    const size_t stage_offset = R2 > 0 ? padded_row_bytes(K) : 0;           // the padded row, then the staged next row
+    const size_t smem = stage_offset + static_cast<size_t>(threads) * (BF16 ? 64 : 0);
+    cudaError_t e = allow_smem(kernel, smem);
+    if (e != cudaSuccess) return cuda_status(e);
+    // persistent CTAs: as many as fit the SMs (64 registers per thread, the row in shared memory), rows dealt round-robin
+    int per_sm = 2048 / threads;
+    if (per_sm > 65536 / (64 * threads)) per_sm = 65536 / (64 * threads);
+    if (per_sm > static_cast<int>((220 * 1024) / (smem + 1024))) per_sm = static_cast<int>((220 * 1024) / (smem + 1024));
+    if (per_sm < 1) per_sm = 1;
+    if (per_sm > 16) per_sm = 16;
+    int grid = per_sm * sm_count();
+    if (grid > M) grid = M;
+    return cuda_status(launch_pdl(kernel, dim3(grid), dim3(threads), smem, st, X, M, K, s0, static_cast<int>(stage_offset), clip,
+                                  inv_sqrt_b, q_a, s_a));
+}
+template <bool BF16, bool UPPER>
+int launch_quantize_rows_bu(const void* X, int M, int K, int had_block, float clip, float inv_sqrt_b, int8_t* q_a, float* s_a,
+                            cudaStream_t st) {
+    int log_b = 0;
+    while ((2 << log_b) <= had_block) ++log_b;      // log2 of the block (0 without rotation)
+    const int s0 = log_b < 5 ? log_b : 5, r = log_b - s0;
+#define QIFT_ROWS(MID, R2) return launch_quantize_rows_as<BF16, UPPER, MID, R2>(X, M, K, s0, clip, inv_sqrt_b, q_a, s_a, st)
+    switch (r) {
+        case 0: QIFT_ROWS(0, 0);
+        case 1: QIFT_ROWS(0, 1);
+        case 2: QIFT_ROWS(0, 2);
+        case 3: QIFT_ROWS(0, 3);
+        case 4: QIFT_ROWS(0, 4);
+        case 5: QIFT_ROWS(1, 1);
+        case 6: QIFT_ROWS(1, 2);
+        case 7: QIFT_ROWS(1, 3);
+        default: QIFT_ROWS(1, 4);
+    }
+#undef QIFT_ROWS
+}
+int launch_quantize_rows(const void* X, bool bf16, int M, int K, int had_block, float clip, float inv_sqrt_b, int8_t* q_a, float* s_a,
+                         cudaStream_t st) {
+    const bool upper_only = clip >= 0.825f;  // |u| / s_u < 8.5: the clamp at -8 cannot act
+    if (bf16)
+        return upper_only ? launch_quantize_rows_bu<true, true>(X, M, K, had_block, clip, inv_sqrt_b, q_a, s_a, st)
+                          : launch_quantize_rows_bu<true, false>(X, M, K, had_block, clip, inv_sqrt_b, q_a, s_a, st);
+    return upper_only ? launch_quantize_rows_bu<false, true>(X, M, K, had_block, clip, inv_sqrt_b, q_a, s_a, st)
+                      : launch_quantize_rows_bu<false, false>(X, M, K, had_block, clip, inv_sqrt_b, q_a, s_a, st);
 }
 
 // ---------------------------------------------------------------------------------------- decode
@@ -604,6 +658,8 @@ int qift_quantize_act(const void* X, int x_dtype, int M, int K, int had_block, f
     const float r = had_block > 1 ? inv_sqrt_block(had_block) : 1.0f;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t smem = padded_row_bytes(K);
+    if (quantize_rows_supports(K, had_block))  // every element in one thread's registers between passes
+        return launch_quantize_rows(X, x_dtype == QIFT_BF16, M, K, had_block, clip_ratio, r, q_a, s_a, st);
     const bool kron = had_block > 1 && !is_pow2(had_block);
     auto kernel = (x_dtype == QIFT_BF16) ? (kron ? quantize_act_kernel<true, true> : quantize_act_kernel<true, false>)
                                          : (kron ? quantize_act_kernel<false, true> : quantize_act_kernel<false, false>);

@@ -47,7 +47,9 @@ def check_outputs(y_gpu, acc_gpu, y_ref, acc_ref, bf16):
 # ---------------------------------------------------------------------------------- rotation / K2
 @pytest.mark.parametrize("M,K,B", [(1, 256, 256), (3, 4096, 4096), (5, 11008, 256), (4, 14336, 2048),
                                    (2, 512, 0), (7, 64, 4), (2, 16384, 16384), (33, 1024, 64), (1, 16, 2),
-                                   (5, 4096, 1024), (3, 16384, 2048), (2, 2048, 1024), (9, 12288, 4096)])  # 4, 8, 2, 3 blocks
+                                   (5, 4096, 1024), (3, 16384, 2048), (2, 2048, 1024), (9, 12288, 4096),  # 4, 8, 2, 3 blocks
+                                   (3, 96, 32), (2, 224, 32), (4, 192, 64), (3, 640, 128), (2, 1536, 512), (3, 16384, 8192),
+                                   (2, 8192, 8192), (2, 48, 16), (300, 4096, 4096), (150, 14336, 2048), (150, 11008, 256)])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_quantize_act(M, K, B, bf16):
     x, _ = synth.activations(100 + M, M, K, max(1, K // 100))

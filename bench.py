@@ -36,10 +36,10 @@ import synth  # noqa: E402
 
 CLIP = 0.9
 N_LAYERS = 32
-# dram__bytes_read.sum + dram__bytes_write.sum of one linear_grouped_kernel launch in the ncu capture of
-# the 4-layer case (profiles/linear_grouped_kernel_llama2_m1_4layers.md): 203 236 864 + 4 653 056 bytes
-# for 203 877 488 algorithmic bytes.  Every packed word is read once, so traffic scales with the layers.
-NCU_TRAFFIC_BYTES_4_LAYERS = 207318528   # dram__bytes_read.sum + dram__bytes_write.sum of linear_grouped_kernel, 4-layer capture (profiles/)
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one linear_grouped_kernel launch, from the committed
+# ncu capture of the 4-layer case of this command (203 227 648 + 4 090 880 bytes for 203 877 488 algorithmic bytes).
+# Every packed word is read once, so traffic scales with the layers.  A constant of that capture, not measured per run.
+NCU_TRAFFIC_BYTES_4_LAYERS = 203227648 + 4090880
 
 
 # ------------------------------------------------------------------------------------------------
@@ -365,7 +365,8 @@ def run_gpu(args):
         "roofline": {"bound": "hbm", "kernel": "linear_grouped_kernel", "achieved": round(achieved, 1), "peak": pk["hbm_gbs"],
                      "unit": "GB/s", "frac": round(achieved / pk["hbm_gbs"], 4),
                      "traffic": round(NCU_TRAFFIC_BYTES_4_LAYERS * args.layers / 4),
-                     "traffic_source": "ncu capture of the 4-layer case, scaled by layers",
+                     "traffic_source": "constant from the committed ncu capture of the 4-layer case (profiles/), scaled by layers; not measured in this run",
+                     "peak_note": "the peak is a copy rate (half of its bytes are writes); a read-only stream runs faster, so frac can exceed 1 -- see frac_of_read_only_ceiling",
                      "peak_source": pk["source"], "avg_launch_us": round(launch_us, 3),
                      "algorithmic_bytes_per_launch": bytes_product},
         "per_call": {"what": "same step as 224 x (qift_quantize_act + qift_w2a4_linear) in one CUDA graph with "
@@ -387,20 +388,124 @@ def run_gpu(args):
     if rank == 0 and world == 1 and not args.no_prefill:
         out["mixed_stack"] = run_mixed_stack(torch, qift, L, device, gen, args)
         out["batched_decode"] = run_batched_decode(torch, qift, L, device, gen, args)
-        out["prefill"] = run_prefill(torch, qift, L, device, gen, pk)
+        ceilings = calibrate_ceilings(torch, L, device)
+        out["ceilings"] = ceilings
+        out["roofline"]["read_only_ceiling_gbs"] = ceilings["hbm_read_only_gbs"]
+        out["roofline"]["frac_of_read_only_ceiling"] = round(out["roofline"]["achieved"] / ceilings["hbm_read_only_gbs"], 4)
+        out["prefill"] = run_prefill(torch, qift, L, device, gen, pk, ceilings)
+        out["mid_m"] = run_mid_m(torch, qift, L, device, gen, pk, ceilings)
         out["kv4"] = run_kv4(torch, qift, L, pk)
         out["diagnostics"] = run_diagnostics(torch, qift, pk)
     if rank == 0 and world == 1 and not args.no_cpu:
         out["cpu_baseline"] = cpu_baseline(budget_s=12.0)
+        out["cpu_baseline"]["other_configs"] = oracle_extra_timings()
     if rank == 0:
         print(json.dumps(out))
     if dist:
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------
+# a transformer layer's linear modules as four multi-output calls with the decode-ahead chain
+# ------------------------------------------------------------------------------------------------
+LAYER_CALLS = (("q", "k", "v"), ("o",), ("gate", "up"), ("down",))
+
+
+class LayerChain:
+    """Runs a stack of layers (each: the seven modules of build_stack, in order) through qift_forward_multi /
+    qift_linear_multi: per layer four calls -- q/k/v on one activation, o, gate/up on one activation, down -- each
+    decoding the NEXT call's packed codes into the other of two int8 level buffers while its own GEMM runs.  The
+    chain is circular (the last call of the stack decodes the first call's codes), as in a prefill loop over
+    requests; the buffers are primed by one untimed pass."""
+
+    def __init__(self, torch, qift, L, mods, M, y_dtype):
+        from paper_2606_02823_b200 import binding
+        self.torch, self.qift, self.L, self.M = torch, qift, L, M
+        self.calls = []
+        for base in range(0, len(mods), 7):
+            layer = {m.name: m for m in mods[base:base + 7]}
+            for names in LAYER_CALLS:
+                ms = [layer[n] for n in names]
+                arr = (binding.LinearOutput * len(ms))()
+                for i, m in enumerate(ms):
+                    arr[i] = binding.LinearOutput(m.packed.data_ptr(), m.s_n.data_ptr(), m.y.data_ptr(), None, m.N, 0)
+                self.calls.append({"x": ms[0].x, "K": ms[0].K, "B": ms[0].B, "levels": ms[0].levels, "arr": arr, "n": len(ms)})
+        vp = ctypes.c_void_p
+        self.lev_bytes = max(int(L.qift_levels_bytes(c["K"], ctypes.addressof(c["arr"]), c["n"])) for c in self.calls)
+        self.scr_bytes = max(int(L.qift_forward_multi_scratch_bytes(M, c["K"], c["levels"], ctypes.addressof(c["arr"]), c["n"]))
+                             for c in self.calls)
+        dev = mods[0].x.device
+        self.lev = [torch.empty(self.lev_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
+        self.scr = torch.empty(self.scr_bytes, dtype=torch.uint8, device=dev)
+        kmax = max(c["K"] for c in self.calls)
+        self.q_a = torch.randint(-8, 8, (M, kmax), dtype=torch.int8, device=dev)   # for the product-only timing
+        self.s_a = torch.full((M,), 0.01, dtype=torch.float32, device=dev)
+        self.ahead = []
+        n = len(self.calls)
+        assert n % 2 == 0
+        for i, c in enumerate(self.calls):
+            nx = self.calls[(i + 1) % n]
+            self.ahead.append(binding.DecodeAhead(ctypes.addressof(nx["arr"]), nx["n"], nx["K"], nx["levels"], 0,
+                                                  self.lev[(i + 1) & 1].data_ptr(), self.lev_bytes))
+        self.y_dtype = qift.BF16 if y_dtype == torch.bfloat16 else qift.F32
+        self.x_dtype = qift.BF16 if mods[0].x.dtype == torch.bfloat16 else qift.F32
+        self.primed = False
+
+    def step(self, with_quant=True):
+        vp, L, M = ctypes.c_void_p, self.L, self.M
+        st = vp(self.torch.cuda.current_stream().cuda_stream)
+        for i, c in enumerate(self.calls):
+            ready = 1 if (self.primed or i > 0) else 0
+            lev = self.lev[i & 1]
+            if with_quant:
+                rc = L.qift_forward_multi(vp(c["x"].data_ptr()), self.x_dtype, M, c["K"], c["B"], CLIP, c["levels"],
+                                          ctypes.addressof(c["arr"]), c["n"], self.y_dtype, vp(self.scr.data_ptr()), self.scr_bytes,
+                                          vp(lev.data_ptr()), self.lev_bytes, ready, ctypes.addressof(self.ahead[i]), st)
+            else:
+                rc = L.qift_linear_multi(vp(self.q_a.data_ptr()), vp(self.s_a.data_ptr()), M, c["K"], c["levels"],
+                                         ctypes.addressof(c["arr"]), c["n"], self.y_dtype, None, 0, vp(lev.data_ptr()),
+                                         self.lev_bytes, ready, ctypes.addressof(self.ahead[i]), st)
+            assert rc == 0, rc
+        self.primed = True
+        return len(self.calls)
+
+
+def time_ms(torch, fn, iters, warm=3):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def calibrate_ceilings(torch, L, device):
+    """The two measured ceilings: a read-only HBM stream over 2 GiB (larger than L2) and the tcgen05 kind::i8 issue
+    rate on shared-memory-resident operands (no loads in the loop), both timed with CUDA events in this run."""
+    vp = ctypes.c_void_p
+    st = vp(torch.cuda.current_stream().cuda_stream)
+    buf = torch.empty(2 << 30, dtype=torch.uint8, device=device)
+    buf.view(torch.int32).random_(0, 1 << 30)
+    ms = time_ms(torch, lambda: L.qift_calib_hbm_read(vp(buf.data_ptr()), buf.numel(), None, st), 5)
+    hbm_read = buf.numel() / (ms * 1e-3) / 1e9
+    del buf
+    ops = ctypes.c_double(0.0)
+    kblocks = 16384       # ~5 ms per launch
+    assert L.qift_calib_mma_i8(kblocks, ctypes.byref(ops), st) == 0
+    ms = time_ms(torch, lambda: L.qift_calib_mma_i8(kblocks, None, st), 5, warm=2)
+    return {"hbm_read_only_gbs": round(hbm_read, 1), "int8_mma_issue_tops": round(ops.value / (ms * 1e-3) / 1e12, 1),
+            "how": "qift_calib_hbm_read over 2 GiB; qift_calib_mma_i8: 74 CTA pairs x 16384 k-blocks of tcgen05.mma.cta_group::2 "
+                   "kind::i8 256x256x32 on resident operands; CUDA events, this run"}
+
+
+
 def run_mixed_stack(torch, qift, L, device, gen, args):
     """Config 5: layer-wise mixed precision on LLaMA-2-7B shapes at M = 1: the first L layers INT4 weights (W4A4), the
-    rest MNZ (W2A4), b_avg = 2 + L/16 bits per weight for 32 layers (Sec. 3.7).  Config 5 itself is L = 16 (3 bits on
+    rest MNZ (W2A4), b_avg = 2 + L/16 bits per weight for 32 layers (Sec. 4.4).  Config 5 itself is L = 16 (3 bits on
     average); the sweep adds L = 4, 8, 12.  Two grouped plans (a plan holds one level set): four launches per
     token-step.  Modules run on their own staged inputs, as in the headline."""
     vp = ctypes.c_void_p
@@ -445,14 +550,17 @@ def run_mixed_stack(torch, qift, L, device, gen, args):
 
 
 def mixed_prefill(torch, qift, L, device, gen, args, n4):
-    """Config 5 at M = 2048: the same mixed stack (first layers W4A4, the rest W2A4 MNZ), every module as activation
-    quantizer + product through the per-call API (bf16 in, bf16 out; AUTO route = codes expanded into one shared int8
-    scratch, then the CTA-pair tcgen05 GEMM).  Distinct weights per layer; end-to-end linear-stack tokens per second."""
+    """Config 5 at M = 2048: the same mixed stack (first layers W4A4, the rest W2A4 MNZ), bf16 in, bf16 out, distinct
+    weights per layer; end-to-end linear-stack tokens per second.  Headline: four qift_forward_multi calls per layer with
+    the decode-ahead chain (one quantization per distinct activation).  Beside it the same stack through the per-module
+    entry points (7 x qift_quantize_act + qift_w2a4_linear / qift_w4a4_linear per layer)."""
     M = 2048
     vp = ctypes.c_void_p
     st = vp(torch.cuda.current_stream().cuda_stream)
     mods = build_stack(torch, qift, synth.LLAMA2_7B, args.layers, M, lambda l: qift.INT4 if l < n4 else qift.MNZ, 5100,
                        torch.bfloat16, torch.bfloat16, device, gen)
+    chain = LayerChain(torch, qift, L, mods, M, torch.bfloat16)
+    ms_chain = time_ms(torch, chain.step, 3)
     kmax = max(m.K for m in mods)
     q_a = torch.empty((M, kmax), dtype=torch.int8, device=device)
     s_a = torch.empty((M,), dtype=torch.float32, device=device)
@@ -463,30 +571,25 @@ def mixed_prefill(torch, qift, L, device, gen, args, n4):
         for m in mods:
             rc = L.qift_quantize_act(vp(m.x.data_ptr()), qift.BF16, M, m.K, m.B, CLIP, vp(q_a.data_ptr()), vp(s_a.data_ptr()), st)
             assert rc == 0, rc
-            fn = L.qift_w4a4_linear if m.levels == qift.INT4 else None
-            if fn is not None:
-                rc = fn(vp(m.packed.data_ptr()), vp(m.s_n.data_ptr()), vp(q_a.data_ptr()), vp(s_a.data_ptr()), M, m.N, m.K,
-                        vp(m.y.data_ptr()), qift.BF16, None, vp(ws.data_ptr()), ws_bytes, st)
+            if m.levels == qift.INT4:
+                rc = L.qift_w4a4_linear(vp(m.packed.data_ptr()), vp(m.s_n.data_ptr()), vp(q_a.data_ptr()), vp(s_a.data_ptr()), M, m.N,
+                                        m.K, vp(m.y.data_ptr()), qift.BF16, None, vp(ws.data_ptr()), ws_bytes, st)
             else:
                 rc = L.qift_w2a4_linear(vp(m.packed.data_ptr()), vp(m.s_n.data_ptr()), m.levels, vp(q_a.data_ptr()),
                                         vp(s_a.data_ptr()), M, m.N, m.K, vp(m.y.data_ptr()), qift.BF16, None, vp(ws.data_ptr()),
                                         ws_bytes, st)
             assert rc == 0, rc
 
-    for _ in range(3):
-        step()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(3):
-        step()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / 3
+    ms_percall = time_ms(torch, step, 3)
     ops = 2.0 * M * sum(m.N * m.K for m in mods)
-    return {"workload": f"config 5 at M = 2048: {n4} W4A4 + {args.layers - n4} W2A4 layers, LLaMA-2-7B shapes, per-call API with "
-                        "activation quantizer", "ms_per_step": round(ms, 3), "tokens_per_s": round(M / (ms * 1e-3), 1),
-            "tops": round(ops / (ms * 1e-3) / 1e12, 1), "launches_per_step": 3 * len(mods)}
+    return {"workload": f"config 5 at M = 2048: {n4} W4A4 + {args.layers - n4} W2A4 layers, LLaMA-2-7B shapes, activation "
+                        "quantizers and code decoding inside the time",
+            "api": "4 x qift_forward_multi per layer, decode-ahead chain", "ms_per_step": round(ms_chain, 3),
+            "tokens_per_s": round(M / (ms_chain * 1e-3), 1), "tops": round(ops / (ms_chain * 1e-3) / 1e12, 1),
+            "launches_per_step": 8 * args.layers,
+            "per_module_api": {"api": "7 x (qift_quantize_act + qift_w2a4_linear | qift_w4a4_linear) per layer",
+                               "ms_per_step": round(ms_percall, 3), "tokens_per_s": round(M / (ms_percall * 1e-3), 1),
+                               "tops": round(ops / (ms_percall * 1e-3) / 1e12, 1), "launches_per_step": 3 * len(mods)}}
 
 
 def run_batched_decode(torch, qift, L, device, gen, args):
@@ -651,8 +754,9 @@ def int8_library_point(torch, M, shapes, device):
         return {"api": "torch._int_mm", "unavailable": str(e)[:120]}
 
 
-def run_prefill(torch, qift, L, device, gen, pk):
-    """Config 4: LLaMA-3.1-8B shapes, M = 2048 tokens, bf16 in, bf16 out, MNZ."""
+def run_prefill(torch, qift, L, device, gen, pk, ceilings):
+    """Config 4: LLaMA-3.1-8B shapes, M = 2048 tokens, bf16 in, bf16 out, MNZ; the weights are the packed 2-bit codes
+    in every headline number (decoded to int8 levels per call, by the side warps of the previous call's GEMM)."""
     M = 2048
     mods = build_stack(torch, qift, synth.LLAMA31_8B, 1, M, lambda l: qift.MNZ, 4000, torch.bfloat16, torch.bfloat16, device, gen)
     kmax = max(m.K for m in mods)
@@ -662,6 +766,20 @@ def run_prefill(torch, qift, L, device, gen, pk):
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
     vp = ctypes.c_void_p
     st = vp(torch.cuda.current_stream().cuda_stream)
+    ops = sum(2.0 * M * m.N * m.K for m in mods)
+
+    def point(ms, **extra):
+        d = {"ms_per_layer": round(ms, 4), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
+        d.update(extra)
+        return d
+
+    chain = LayerChain(torch, qift, L, mods, M, torch.bfloat16)
+    res = {"workload": "config 4: LLaMA-3.1-8B shapes, M=2048, 7 modules, MNZ packed 2-bit weights, bf16 in / bf16 out", "unit": "TOPS"}
+    res["layer_with_act_quant"] = point(time_ms(torch, lambda: chain.step(True), 10),
+                                        api="4 x qift_forward_multi (q/k/v, o, gate/up, down), decode-ahead chain; 4 quantizations",
+                                        kernels="quantize_rows_kernel + gemm_i8_pair_kernel (its side warps decode the next call's codes)")
+    res["product_only"] = point(time_ms(torch, lambda: chain.step(False), 10),
+                                api="4 x qift_linear_multi on quantized activations, decode-ahead chain")
 
     def layer(with_quant=True):
         for m in mods:
@@ -672,7 +790,12 @@ def run_prefill(torch, qift, L, device, gen, pk):
                                     M, m.N, m.K, vp(m.y.data_ptr()), qift.BF16, None, vp(ws.data_ptr()), ws_bytes, st)
             assert rc == 0, rc
 
-    # resident decoded weights: one int8 level per weight kept beside the packed codes (decoded once, untimed)
+    res["per_module_api"] = {"what": "the same layer as 7 x (qift_quantize_act + qift_w2a4_linear): every call decodes its codes "
+                                     "into scratch first (expand_levels_kernel), seven quantizations",
+                             "layer_with_act_quant": point(time_ms(torch, lambda: layer(True), 10)),
+                             "product_only": point(time_ms(torch, lambda: layer(False), 10))}
+
+    # extra, outside the method's storage: a second, int8 copy of the weights kept resident (4 x the packed bytes)
     for m in mods:
         m.levels_i8 = qift.qift_expand_weights(m.packed, m.N, m.K, m.levels)
 
@@ -685,70 +808,73 @@ def run_prefill(torch, qift, L, device, gen, pk):
                                         M, m.N, m.K, vp(m.y.data_ptr()), qift.BF16, None, st)
             assert rc == 0, rc
 
-    def layer_resident_shared(_=True):
-        # a transformer layer quantizes four inputs, not seven: q / k / v share one, gate / up share one
-        for i, m in enumerate(mods):
-            if m.name in ("q", "o", "gate", "down"):
-                rc = L.qift_quantize_act(vp(m.x.data_ptr()), qift.BF16, M, m.K, m.B, CLIP, vp(q_a.data_ptr()), vp(s_a.data_ptr()), st)
-                assert rc == 0, rc
-            rc = L.qift_expanded_linear(vp(m.levels_i8.data_ptr()), vp(m.s_n.data_ptr()), vp(q_a.data_ptr()), vp(s_a.data_ptr()),
-                                        M, m.N, m.K, vp(m.y.data_ptr()), qift.BF16, None, st)
-            assert rc == 0, rc
+    res["extra_resident_int8_weights"] = {
+        "note": "NOT the method's W2 storage: the weights are stored twice (packed codes + one int8 level per weight, 4 x the "
+                "packed size); qift_expand_weights once, then qift_expanded_linear per module",
+        "product_only": point(time_ms(torch, lambda: layer_resident(False), 10)),
+        "layer_with_act_quant": point(time_ms(torch, lambda: layer_resident(True), 10))}
+    for m in mods:
+        m.levels_i8 = None
 
-    # the layer as it is usually deployed: q/k/v stored as one 6144 x 4096 matrix, gate/up as one 28672 x 4096 matrix
-    # (same output channels, same ops), four quantized activations, resident decoded weights
-    fused_shapes = [("qkv", 4096 + 1024 + 1024, 4096), ("o", 4096, 4096), ("gate_up", 2 * 14336, 4096), ("down", 4096, 14336)]
-    fmods = build_stack(torch, qift, fused_shapes, 1, M, lambda l: qift.MNZ, 4100, torch.bfloat16, torch.bfloat16, device, gen)
-    for m in fmods:
-        m.levels_i8 = qift.qift_expand_weights(m.packed, m.N, m.K, m.levels)
-
-    def layer_fused(_=True):
-        for m in fmods:
-            rc = L.qift_quantize_act(vp(m.x.data_ptr()), qift.BF16, M, m.K, m.B, CLIP, vp(q_a.data_ptr()), vp(s_a.data_ptr()), st)
-            assert rc == 0, rc
-            rc = L.qift_expanded_linear(vp(m.levels_i8.data_ptr()), vp(m.s_n.data_ptr()), vp(q_a.data_ptr()), vp(s_a.data_ptr()),
-                                        M, m.N, m.K, vp(m.y.data_ptr()), qift.BF16, None, st)
-            assert rc == 0, rc
-
-    res = {}
-    for key, fn, wq in (("layer_with_act_quant", layer, True), ("product_only", layer, False),
-                        ("resident_fused_qkv_gateup", layer_fused, True),
-                        ("resident_with_act_quant", layer_resident, True), ("resident_product_only", layer_resident, False),
-                        ("resident_shared_act_quant", layer_resident_shared, True)):
-        for _ in range(3):
-            fn(wq)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        iters = 10
-        e0.record()
-        for _ in range(iters):
-            fn(wq)
-        e1.record()
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1) / iters
-        ops = sum(2.0 * M * m.N * m.K for m in mods)
-        res[key] = {"ms_per_layer": round(ms, 4), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
-    res["resident_note"] = ("resident_*: the same layer through qift_expanded_linear on int8 levels decoded once "
-                            "(4x the packed size, kept beside the packed codes); product_only decodes on every call; "
-                            "resident_shared_act_quant quantizes the four distinct inputs of a layer (q/k/v and gate/up share "
-                            "theirs) instead of one per module; resident_fused_qkv_gateup stores q/k/v and gate/up as "
-                            "one matrix each (4 products + 4 quantizations per layer, same ops)")
-    tops = res["product_only"]["tops"]
-    gemm_tops = res["resident_product_only"]["tops"]      # the GEMM kernel alone (no decoding pass in the timed region)
+    tops, tops_q = res["product_only"]["tops"], res["layer_with_act_quant"]["tops"]
     int8_peak = 2.0 * pk["bf16_tflops"]    # dense int8 is nominally 2x bf16; scaled from the measured bf16 burst
-    res.update({"workload": "config 4: LLaMA-3.1-8B shapes, M=2048, 7 modules, MNZ, bf16 out", "unit": "TOPS",
-                "pct_of_nominal_4500": round(100 * tops / 4500.0, 2),
-                "resident_pct_of_nominal_4500": round(100 * gemm_tops / 4500.0, 2),
-                "roofline": {"bound": "tensor", "kernel": "gemm_i8_pair_kernel", "achieved": gemm_tops,
-                             "peak": int8_peak, "unit": "TOP/s", "frac": round(gemm_tops / int8_peak, 4),
-                             "peak_source": f"2 x {pk['source']} bf16 burst",
-                             "with_decoding_pass": {"kernels": "expand_levels_kernel + gemm_i8_pair_kernel", "achieved": tops,
-                                                    "frac": round(tops / int8_peak, 4)}},
-                "tokens_per_s": round(M / (res["layer_with_act_quant"]["ms_per_layer"] * 1e-3), 1),
-                "resident_tokens_per_s": round(M / (res["resident_with_act_quant"]["ms_per_layer"] * 1e-3), 1),
-                "fused_layer_tokens_per_s": round(M / (res["resident_fused_qkv_gateup"]["ms_per_layer"] * 1e-3), 1)})
-    res["library_int8"] = int8_library_point(torch, M, synth.LLAMA31_8B, device)
+    issue = ceilings["int8_mma_issue_tops"]
+    lib = int8_library_point(torch, M, synth.LLAMA31_8B, device)
+    res["library_int8"] = lib
+    res.update({"pct_of_nominal_4500": round(100 * tops / 4500.0, 2),
+                "with_act_quant_pct_of_nominal_4500": round(100 * tops_q / 4500.0, 2),
+                "roofline": {"bound": "tensor", "kernel": "gemm_i8_pair_kernel", "achieved": tops, "peak": int8_peak, "unit": "TOP/s",
+                             "frac": round(tops / int8_peak, 4), "peak_source": f"2 x {pk['source']} bf16 burst (nominal int8 : bf16 ratio)",
+                             "what": "packed 2-bit weights, product only (4 x qift_linear_multi per layer)",
+                             "with_act_quant": {"achieved": tops_q, "frac": round(tops_q / int8_peak, 4)},
+                             "ceilings": {"int8_nominal_tops": 4500.0, "frac_of_nominal": round(tops / 4500.0, 4),
+                                          "int8_mma_issue_measured_tops": issue, "frac_of_mma_issue": round(tops / issue, 4),
+                                          "library_int8_tops": lib.get("tops"),
+                                          "vs_library_int8": round(tops / lib["tops"], 4) if lib.get("tops") else None}},
+                "tokens_per_s": round(M / (res["layer_with_act_quant"]["ms_per_layer"] * 1e-3), 1)})
     return res
+
+
+def run_mid_m(torch, qift, L, device, gen, pk, ceilings):
+    """16 < M <= 512: one LLaMA-3.1-8B layer (MNZ, bf16 in / bf16 out), product only through qift_linear_multi (AUTO route
+    per output), microseconds per layer against max(HBM time of the packed weights, tensor time at the measured
+    tcgen05 issue rate)."""
+    rows = []
+    base = build_stack(torch, qift, synth.LLAMA31_8B, 8, 512, lambda l: qift.MNZ, 4200, torch.bfloat16, torch.bfloat16, device, gen)
+    n_layers = len(base) // 7
+    for M in (32, 64, 128, 256, 512):
+        mods = []
+        for m in base:
+            c = Module()
+            for k in Module.__slots__:
+                if hasattr(m, k):
+                    setattr(c, k, getattr(m, k))
+            c.x, c.y = m.x[:M].contiguous(), m.y[:M].contiguous()
+            mods.append(c)
+        chain = LayerChain(torch, qift, L, mods, M, torch.bfloat16)
+        vp = ctypes.c_void_p
+        st = vp(torch.cuda.current_stream().cuda_stream)
+        wsb = max(int(L.qift_linear_multi_workspace_bytes(M, c["K"], c["levels"], ctypes.addressof(c["arr"]), c["n"])) for c in chain.calls)
+        ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device=device)
+
+        def step():
+            for i, c in enumerate(chain.calls):
+                rc = L.qift_linear_multi(vp(chain.q_a.data_ptr()), vp(chain.s_a.data_ptr()), M, c["K"], c["levels"],
+                                         ctypes.addressof(c["arr"]), c["n"], chain.y_dtype, vp(ws.data_ptr()), ws.numel(),
+                                         vp(chain.lev[i & 1].data_ptr()), chain.lev_bytes, 0, None, st)
+                assert rc == 0, rc
+
+        us = time_ms(torch, step, 5) * 1e3 / n_layers
+        w_bytes = sum(product_bytes(M, m.N, m.K, 2, 2) for m in mods[:7])
+        opsl = sum(2.0 * M * m.N * m.K for m in mods[:7])
+        t_hbm = w_bytes / (ceilings["hbm_read_only_gbs"] * 1e9) * 1e6
+        t_tc = opsl / (ceilings["int8_mma_issue_tops"] * 1e12) * 1e6
+        rows.append({"M": M, "us_per_layer": round(us, 2), "hbm_us": round(t_hbm, 2), "tensor_us": round(t_tc, 2),
+                     "frac_of_bound": round(max(t_hbm, t_tc) / us, 3), "tops": round(opsl / (us * 1e-6) / 1e12, 1),
+                     "gbs": round(w_bytes / (us * 1e-6) / 1e9, 1)})
+        del chain
+    return {"workload": f"LLaMA-3.1-8B layer x {n_layers} distinct layers, MNZ, product only (qift_linear_multi), bound = max(packed-weight "
+                        "bytes / measured read-only HBM rate, ops / measured tcgen05 int8 issue rate)", "points": rows}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -790,6 +916,51 @@ def cpu_baseline(budget_s=12.0):
     return {"value": round(reps * layer_bytes() / dt / 1e9, 4), "unit": "GB/s", "cores": 1, "kind": "oracle",
             "sample": f"{reps} of 32 layers (7 modules each, M=1) of the same workload, single thread, {dt:.1f} s",
             "host": f"{os.cpu_count()} logical cores"}
+
+
+def oracle_extra_timings():
+    """Oracle times beyond the headline workload (single thread, same host): one LLaMA-3.1-8B layer at M = 1 with the PoT
+    set (config 3), one W4A4 LLaMA-2-7B layer at M = 1 (config 5), and a slice of one config-4 product at M = 2048
+    (256 of the k-projection's 1024 channels, K = 4096; the product is linear in the channel count)."""
+    import oracle
+    out = {}
+
+    def layer_time(shapes, lv, M):
+        mods = []
+        for i, (name, N, K) in enumerate(shapes):
+            rng = np.random.default_rng(3000 + i)
+            hi = 16 if lv == oracle.INT4 else 4
+            codes = rng.integers(0, hi, (N, K), dtype=np.uint8)
+            s_n = np.full((N,), 0.01, dtype=np.float32)
+            x, _ = synth.activations(3100 + i, M, K, max(1, round(0.01 * K)))
+            mods.append((N, K, codes, s_n, x))
+        t0 = time.perf_counter()
+        for (N, K, codes, s_n, x) in mods:
+            q_a, s_a = oracle.quantize_act(x, synth.had_block_for(K), CLIP)
+            oracle.linear(codes, lv, s_n, q_a, s_a)
+        return time.perf_counter() - t0
+
+    t = layer_time(synth.LLAMA31_8B, oracle.POT, 1)
+    out["config3_layer_m1_pot"] = {"seconds_per_layer": round(t, 3), "extrapolated_32_layers_s": round(32 * t, 1)}
+    t = layer_time(synth.LLAMA2_7B, oracle.INT4, 1)
+    out["config5_w4a4_layer_m1"] = {"seconds_per_layer": round(t, 3), "extrapolated_16_layers_s": round(16 * t, 1)}
+    M, N, K, n_slice = 2048, 1024, 4096, 256
+    rng = np.random.default_rng(3200)
+    codes = rng.integers(0, 4, (n_slice, K), dtype=np.uint8)
+    s_n = np.full((n_slice,), 0.01, dtype=np.float32)
+    x, _ = synth.activations(3201, M, K, 41)
+    t0 = time.perf_counter()
+    q_a, s_a = oracle.quantize_act(x, 4096, CLIP)
+    tq = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    oracle.linear(codes, oracle.MNZ, s_n, q_a, s_a, bf16=True)
+    tl = time.perf_counter() - t0
+    layer_macs = sum(N_ * K_ for _, N_, K_ in synth.LLAMA31_8B) * M
+    out["config4_k_proj_m2048"] = {"quantize_act_s": round(tq, 3), "product_256_of_1024_channels_s": round(tl, 3),
+                                   "gmacs_per_s": round(M * n_slice * K / tl / 1e9, 3),
+                                   "extrapolated_layer_s": round(layer_macs / (M * n_slice * K / tl), 1),
+                                   "extrapolation": "whole layer = 4.47e11 multiply-adds at the measured rate"}
+    return out
 
 
 def run_reference(args):

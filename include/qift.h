@@ -235,6 +235,13 @@ int qift_forward_multi(const void* X, int x_dtype, int M, int K, int had_block, 
                        const qift_linear_output* outputs, int count, int y_dtype, void* scratch, size_t scratch_bytes,
                        void* levels_buf, size_t levels_bytes, int levels_ready, const qift_decode_ahead* ahead,
                        void* stream);
+/* The product part alone (S4 + S5 for every output) on an activation that qift_quantize_act has already
+ * quantized: q_a int8 [M,K], s_a fp32 [M].  workspace >= qift_linear_multi_workspace_bytes(...) bytes
+ * (0 for M > 512; NULL allowed then), 256-byte aligned; everything else as for qift_forward_multi. */
+size_t qift_linear_multi_workspace_bytes(int M, int K, int levels, const qift_linear_output* outputs, int count);
+int qift_linear_multi(const int8_t* q_a, const float* s_a, int M, int K, int levels, const qift_linear_output* outputs,
+                      int count, int y_dtype, void* workspace, size_t workspace_bytes, void* levels_buf,
+                      size_t levels_bytes, int levels_ready, const qift_decode_ahead* ahead, void* stream);
 
 /* ---- Grouped decode path -----------------------------------------------------------------------
  * One persistent launch serves a list of independent layer problems that share M (<= 64 token rows),
@@ -422,6 +429,18 @@ int qift_device_status(void* stream, uint32_t* detail);
  * Afterwards qift_device_status returns QIFT_ERR_TIMEOUT once, with the site in bits 0-7 of `detail`, and
  * QIFT_OK on the next call.  INVALID_ARG for other arguments. */
 int qift_selftest_wait_timeout(int which, unsigned int limit_us, void* stream);
+
+/* Measurement helpers (no counterpart in the paper; used by the benchmark to calibrate its roofline
+ * denominators on the GPU it runs on; neither touches the quantized layer).
+ *   qift_calib_hbm_read   streams `bytes` of device memory at `buf` through 128-bit loads, writes nothing
+ *                         (`sink`, dev, may be NULL, is only there to keep the loads alive): the read-only
+ *                         HBM ceiling.  Time it with events on `stream`.
+ *   qift_calib_mma_i8     every SM pair issues kblocks x 4 tcgen05.mma kind::i8 (256 x 256 x 32 each) back to
+ *                         back on operands resident in shared memory, no loads in the loop: the rate of the
+ *                         tensor pipe itself under the power limit.  *ops (host, may be NULL) receives the
+ *                         integer operations of the launch (2 per multiply-add).  1 <= kblocks <= 2^20. */
+int qift_calib_hbm_read(const void* buf, size_t bytes, unsigned int* sink, void* stream);
+int qift_calib_mma_i8(int kblocks, double* ops, void* stream);
 
 #ifdef __cplusplus
 }

@@ -13,4 +13,4 @@ from .binding import (lib, status_string, QiftError, qift_packed_bytes, qift_wor
                       qift_w2a4_linear_static, Kv4Cache, KV_KEYS, KV_VALUES, qift_kv4_quantize, qift_kv4_attention_workspace_bytes,
                       qift_kv4_attention_decode, qift_expand_weights, qift_expanded_linear, qift_diag_grid_quantize,
                       qift_diag_bucket_stats, qift_diag_ratio_scan_workspace_bytes, qift_diag_ratio_scan,
-                      qift_selftest_wait_timeout, qift_levels_bytes, qift_forward_multi)
+                      qift_selftest_wait_timeout, qift_levels_bytes, qift_forward_multi, qift_linear_multi)

@@ -33,6 +33,7 @@ EXPORTS = [
     "qift_expand_weights", "qift_expanded_linear",
     "qift_diag_grid_quantize", "qift_diag_bucket_stats", "qift_diag_ratio_scan_workspace_bytes", "qift_diag_ratio_scan",
     "qift_selftest_wait_timeout", "qift_levels_bytes", "qift_forward_multi_scratch_bytes", "qift_forward_multi",
+    "qift_linear_multi_workspace_bytes", "qift_linear_multi", "qift_calib_hbm_read", "qift_calib_mma_i8",
 ]
 
 _lib = None
@@ -101,11 +102,16 @@ def lib() -> ctypes.CDLL:
         L.qift_forward_multi_scratch_bytes.restype = sz
         L.qift_forward_multi_scratch_bytes.argtypes = [ci, ci, ci, vp, ci]
         L.qift_forward_multi.argtypes = [vp, ci, ci, ci, ci, cf, ci, vp, ci, ci, vp, sz, vp, sz, ci, vp, vp]
+        L.qift_linear_multi_workspace_bytes.restype = sz
+        L.qift_linear_multi_workspace_bytes.argtypes = [ci, ci, ci, vp, ci]
+        L.qift_linear_multi.argtypes = [vp, vp, ci, ci, ci, vp, ci, ci, vp, sz, vp, sz, ci, vp, vp]
+        L.qift_calib_hbm_read.argtypes = [vp, sz, vp, vp]
+        L.qift_calib_mma_i8.argtypes = [ci, vp, vp]
         for name in EXPORTS:
             if name not in ("qift_diag_ratio_scan_workspace_bytes", "qift_status_string", "qift_packed_bytes", "qift_workspace_bytes",
                             "qift_forward_scratch_bytes", "qift_group_plan_bytes", "qift_static_scratch_bytes",
                             "qift_workspace_bytes_route", "qift_kv4_attention_workspace_bytes", "qift_levels_bytes",
-                            "qift_forward_multi_scratch_bytes"):
+                            "qift_forward_multi_scratch_bytes", "qift_linear_multi_workspace_bytes"):
                 getattr(L, name).restype = ci
         _lib = L
     return _lib
@@ -334,6 +340,31 @@ def qift_forward_multi(X, had_block: int, weights, levels: int, clip_ratio: floa
                                 _dt(ys[0]), _ptr(_dev(scratch)), scratch.numel(), _ptr(_dev(levels_buf)), levels_buf.numel(),
                                 1 if levels_ready else 0, None if ah is None else ctypes.addressof(ah), _stream()),
            "qift_forward_multi")
+    return ys, accs
+
+
+def qift_linear_multi(q_a, s_a, weights, levels: int, out_dtype=torch.float32, want_acc: bool = False, levels_buf=None,
+                      levels_ready: bool = False, ahead=None):
+    """The product part of qift_forward_multi on an activation that is already quantized -> ([Y_i], [acc_i or None])."""
+    _dev(q_a, torch.int8), _dev(s_a, torch.float32)
+    M, K = q_a.shape
+    ys = [torch.empty((M, s_n.shape[0]), dtype=out_dtype, device=q_a.device) for _, s_n in weights]
+    accs = [torch.empty((M, s_n.shape[0]), dtype=torch.int32, device=q_a.device) if want_acc else None for _, s_n in weights]
+    arr = _outputs_array(weights, ys, accs)
+    L = lib()
+    need = int(L.qift_linear_multi_workspace_bytes(M, K, levels, ctypes.addressof(arr), len(weights)))
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device=q_a.device)
+    if levels_buf is None:
+        assert not levels_ready
+        levels_buf = torch.empty(max(qift_levels_bytes(K, weights), 256), dtype=torch.uint8, device=q_a.device)
+    ah, keep = None, None
+    if ahead is not None:
+        nw, nK, nlv, nbuf = ahead
+        keep = _outputs_array(nw)
+        ah = DecodeAhead(ctypes.addressof(keep), len(nw), nK, nlv, 0, _dev(nbuf).data_ptr(), nbuf.numel())
+    _check(L.qift_linear_multi(_ptr(q_a), _ptr(s_a), M, K, levels, ctypes.addressof(arr), len(weights), _dt(ys[0]), _ptr(ws),
+                               ws.numel(), _ptr(_dev(levels_buf)), levels_buf.numel(), 1 if levels_ready else 0,
+                               None if ah is None else ctypes.addressof(ah), _stream()), "qift_linear_multi")
     return ys, accs
 
 

@@ -145,6 +145,31 @@ __device__ __forceinline__ void side_store_any(int levels, const SideUnit& u, co
     }
 }
 
+// The side warps' loop: groups of 128 threads; group q of CTA b takes units 2 (b * groups + q), + 1, then strides on.
+__device__ __forceinline__ void side_jobs(const PairParams& p, int t, int group) {
+    constexpr int kGroups = 32 * kPairSideWarps / kSideUnitWords;
+    auto job_of = [&](int u) {
+        int ji = 0;
+#pragma unroll
+        for (int i = 1; i < kPairMaxSegments; ++i)
+            if (i < p.njobs && u >= p.job[i].unit0) ji = i;
+        return ji;
+    };
+    for (int u0 = 2 * (blockIdx.x * kGroups + group); u0 < p.units; u0 += 2 * gridDim.x * kGroups) {
+        const int ja = job_of(u0), jb = job_of(min(u0 + 1, p.units - 1));
+        SideUnit a = side_unit(p.job[ja], u0 - p.job[ja].unit0, t);
+        SideUnit b = side_unit(p.job[jb], u0 + 1 - p.job[jb].unit0, t);
+        if (u0 + 1 >= p.units) b.rows = 0;
+        uint32_t wa[kSideUnitRows], wb[kSideUnitRows];
+#pragma unroll
+        for (int r = 0; r < kSideUnitRows; ++r) wa[r] = (r < a.rows) ? __ldg(a.src + 16 * r) : 0u;
+#pragma unroll
+        for (int r = 0; r < kSideUnitRows; ++r) wb[r] = (r < b.rows) ? __ldg(b.src + 16 * r) : 0u;
+        side_store_any(p.job[ja].levels, a, wa);
+        side_store_any(p.job[jb].levels, b, wb);
+    }
+}
+
 template <int BN>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_i8_pair_kernel(const __grid_constant__ PairParams p) {
@@ -331,30 +356,9 @@ gemm_i8_pair_kernel(const __grid_constant__ PairParams p) {
         }
     } else {
         // ------------------------------------------------------------------ side warps: decode the next product's codes
-        // groups of 128 threads; group q of CTA b takes units (2 b + q) * 2, + 1, then strides on
         const int t = (threadIdx.x - kPairGemmThreads) & (kSideUnitWords - 1);
         const int group = (threadIdx.x - kPairGemmThreads) / kSideUnitWords;
-        constexpr int kGroups = 32 * kPairSideWarps / kSideUnitWords;
-        auto job_of = [&](int u) {
-            int ji = 0;
-#pragma unroll
-            for (int i = 1; i < kPairMaxSegments; ++i)
-                if (i < p.njobs && u >= p.job[i].unit0) ji = i;
-            return ji;
-        };
-        for (int u0 = 2 * (blockIdx.x * kGroups + group); u0 < p.units; u0 += 2 * gridDim.x * kGroups) {
-            const int ja = job_of(u0), jb = job_of(min(u0 + 1, p.units - 1));
-            SideUnit a = side_unit(p.job[ja], u0 - p.job[ja].unit0, t);
-            SideUnit b = side_unit(p.job[jb], u0 + 1 - p.job[jb].unit0, t);
-            if (u0 + 1 >= p.units) b.rows = 0;
-            uint32_t wa[kSideUnitRows], wb[kSideUnitRows];
-#pragma unroll
-            for (int r = 0; r < kSideUnitRows; ++r) wa[r] = (r < a.rows) ? __ldg(a.src + 16 * r) : 0u;
-#pragma unroll
-            for (int r = 0; r < kSideUnitRows; ++r) wb[r] = (r < b.rows) ? __ldg(b.src + 16 * r) : 0u;
-            side_store_any(p.job[ja].levels, a, wa);
-            side_store_any(p.job[jb].levels, b, wb);
-        }
+        side_jobs(p, t, group);
     }
 
     tc_fence_before();

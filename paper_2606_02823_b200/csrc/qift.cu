@@ -6,6 +6,7 @@
 #include <cstdlib>
 #include <mutex>
 
+#include "calib.cuh"
 #include "common.cuh"
 #include "decode.cuh"
 #include "diag.cuh"
@@ -145,8 +146,7 @@ int launch_quantize_rows_as(const void* X, int M, int K, int s0, float clip, flo
                             cudaStream_t st) {
     auto kernel = quantize_rows_kernel<BF16, UPPER, MID, R2>;
     const int threads = ((K / 32) + 31) & ~31;
-    const size_t stage_offset = R2 > 0 ? padded_row_bytes(K) : 0;           // the padded row, then the staged next row
-    const size_t smem = stage_offset + static_cast<size_t>(threads) * (BF16 ? 64 : 0);
+    const size_t smem = R2 > 0 ? padded_row_bytes(K) : 0;
     cudaError_t e = allow_smem(kernel, smem);
     if (e != cudaSuccess) return cuda_status(e);
     // persistent CTAs: as many as fit the SMs (64 registers per thread, the row in shared memory), rows dealt round-robin
@@ -157,7 +157,7 @@ int launch_quantize_rows_as(const void* X, int M, int K, int s0, float clip, flo
     if (per_sm > 16) per_sm = 16;
     int grid = per_sm * sm_count();
     if (grid > M) grid = M;
-    return cuda_status(launch_pdl(kernel, dim3(grid), dim3(threads), smem, st, X, M, K, s0, static_cast<int>(stage_offset), clip,
+    return cuda_status(launch_pdl(kernel, dim3(grid), dim3(threads), smem, st, X, M, K, s0, clip,
                                   inv_sqrt_b, q_a, s_a));
 }
 template <bool BF16, bool UPPER>
@@ -815,14 +815,11 @@ size_t qift_forward_multi_scratch_bytes(int M, int K, int levels, const qift_lin
     return multi_layout(M, K, levels, outputs, count).total;
 }
 
-int qift_forward_multi(const void* X, int x_dtype, int M, int K, int had_block, float clip_ratio, int levels,
-                       const qift_linear_output* outputs, int count, int y_dtype, void* scratch, size_t scratch_bytes,
-                       void* levels_buf, size_t levels_bytes, int levels_ready, const qift_decode_ahead* ahead, void* stream) {
-    if (!X || M <= 0 || K <= 0 || !valid_levels(levels) || !multi_outputs_ok(outputs, count, true)) return QIFT_ERR_INVALID_ARG;
-    if ((x_dtype != QIFT_F32 && x_dtype != QIFT_BF16) || (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16))
-        return QIFT_ERR_INVALID_ARG;
+static int check_outputs_and_ahead(int M, int K, int levels, const qift_linear_output* outputs, int count, int y_dtype,
+                                   const qift_decode_ahead* ahead) {
+    if (M <= 0 || K <= 0 || !valid_levels(levels) || !multi_outputs_ok(outputs, count, true)) return QIFT_ERR_INVALID_ARG;
+    if (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16) return QIFT_ERR_INVALID_ARG;
     if (K % codes_per_word(levels) != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
-    if (!aligned16(X)) return QIFT_ERR_ALIGNMENT;
     for (int i = 0; i < count; ++i)
         if (!aligned16(outputs[i].packed) || !aligned16(outputs[i].s_n) || !aligned16(outputs[i].Y) ||
             (outputs[i].acc_debug && !aligned16(outputs[i].acc_debug)))
@@ -836,24 +833,20 @@ int qift_forward_multi(const void* X, int x_dtype, int M, int K, int had_block, 
         for (int i = 0; i < ahead->count; ++i)
             if (!aligned16(ahead->outputs[i].packed)) return QIFT_ERR_ALIGNMENT;
     }
-    const MultiLayout L = multi_layout(M, K, levels, outputs, count);
-    if (!scratch || scratch_bytes < L.total) return QIFT_ERR_WORKSPACE;
-    if ((reinterpret_cast<uintptr_t>(scratch) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
-    const bool pair_route = M > kFusedPairMaxM && K % 16 == 0;
-    if (pair_route) {
-        if (!levels_buf || levels_bytes < qift_levels_bytes(K, outputs, count)) return QIFT_ERR_WORKSPACE;
-        if ((reinterpret_cast<uintptr_t>(levels_buf) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
-    }
+    return QIFT_OK;
+}
+
+// S4 + S5 for every output on one quantized activation; arguments checked by the callers.
+static int linear_multi_impl(const int8_t* q_a, const float* s_a, int M, int K, int levels, const qift_linear_output* outputs, int count,
+                             int y_dtype, void* workspace, size_t workspace_bytes, void* levels_buf, size_t levels_bytes,
+                             int levels_ready, const qift_decode_ahead* ahead, void* stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    unsigned char* base = static_cast<unsigned char*>(scratch);
-    int8_t* q_a = reinterpret_cast<int8_t*>(base + L.q_off);
-    float* s_a = reinterpret_cast<float*>(base + L.sa_off);
-    int rc = qift_quantize_act(X, x_dtype, M, K, had_block, clip_ratio, q_a, s_a, stream);
-    if (rc != QIFT_OK) return rc;
+    const bool pair_route = M > kFusedPairMaxM && K % 16 == 0;
+    int rc;
     if (!pair_route) {
         for (int i = 0; i < count; ++i) {
             rc = linear_impl(outputs[i].packed, outputs[i].s_n, levels, q_a, s_a, M, outputs[i].N, K, outputs[i].Y, y_dtype,
-                             outputs[i].acc_debug, base + L.ws_off, L.total - L.ws_off, QIFT_ROUTE_AUTO, stream);
+                             outputs[i].acc_debug, workspace, workspace_bytes, QIFT_ROUTE_AUTO, stream);
             if (rc != QIFT_OK) return rc;
         }
         if (ahead)
@@ -864,6 +857,8 @@ int qift_forward_multi(const void* X, int x_dtype, int M, int K, int had_block, 
             }
         return QIFT_OK;
     }
+    if (!levels_buf || levels_bytes < qift_levels_bytes(K, outputs, count)) return QIFT_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(levels_buf) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
     PairCall c = {};
     c.q_a = q_a, c.s_a = s_a, c.M = M, c.K = K, c.y_bf16 = (y_dtype == QIFT_BF16), c.nseg = count;
     for (int i = 0; i < count; ++i) {
@@ -883,6 +878,49 @@ int qift_forward_multi(const void* X, int x_dtype, int M, int K, int had_block, 
         }
     }
     return run_pair_gemm(c, st);
+}
+
+size_t qift_linear_multi_workspace_bytes(int M, int K, int levels, const qift_linear_output* outputs, int count) {
+    if (M <= 0 || K <= 0 || !valid_levels(levels) || !multi_outputs_ok(outputs, count, false)) return 0;
+    const MultiLayout L = multi_layout(M, K, levels, outputs, count);
+    return L.total - L.ws_off;
+}
+
+int qift_linear_multi(const int8_t* q_a, const float* s_a, int M, int K, int levels, const qift_linear_output* outputs, int count,
+                      int y_dtype, void* workspace, size_t workspace_bytes, void* levels_buf, size_t levels_bytes, int levels_ready,
+                      const qift_decode_ahead* ahead, void* stream) {
+    if (!q_a || !s_a) return QIFT_ERR_INVALID_ARG;
+    const int rc = check_outputs_and_ahead(M, K, levels, outputs, count, y_dtype, ahead);
+    if (rc != QIFT_OK) return rc;
+    if (!aligned16(q_a) || !aligned16(s_a)) return QIFT_ERR_ALIGNMENT;
+    if (workspace_bytes < qift_linear_multi_workspace_bytes(M, K, levels, outputs, count) || (workspace_bytes && !workspace))
+        return QIFT_ERR_WORKSPACE;
+    if (workspace && (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
+    return linear_multi_impl(q_a, s_a, M, K, levels, outputs, count, y_dtype, workspace, workspace_bytes, levels_buf, levels_bytes,
+                             levels_ready, ahead, stream);
+}
+
+int qift_forward_multi(const void* X, int x_dtype, int M, int K, int had_block, float clip_ratio, int levels,
+                       const qift_linear_output* outputs, int count, int y_dtype, void* scratch, size_t scratch_bytes,
+                       void* levels_buf, size_t levels_bytes, int levels_ready, const qift_decode_ahead* ahead, void* stream) {
+    if (!X || (x_dtype != QIFT_F32 && x_dtype != QIFT_BF16)) return QIFT_ERR_INVALID_ARG;
+    int rc = check_outputs_and_ahead(M, K, levels, outputs, count, y_dtype, ahead);
+    if (rc != QIFT_OK) return rc;
+    if (!aligned16(X)) return QIFT_ERR_ALIGNMENT;
+    const MultiLayout L = multi_layout(M, K, levels, outputs, count);
+    if (!scratch || scratch_bytes < L.total) return QIFT_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(scratch) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
+    if (M > kFusedPairMaxM && K % 16 == 0) {  // found before anything is launched
+        if (!levels_buf || levels_bytes < qift_levels_bytes(K, outputs, count)) return QIFT_ERR_WORKSPACE;
+        if ((reinterpret_cast<uintptr_t>(levels_buf) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
+    }
+    unsigned char* base = static_cast<unsigned char*>(scratch);
+    int8_t* q_a = reinterpret_cast<int8_t*>(base + L.q_off);
+    float* s_a = reinterpret_cast<float*>(base + L.sa_off);
+    rc = qift_quantize_act(X, x_dtype, M, K, had_block, clip_ratio, q_a, s_a, stream);
+    if (rc != QIFT_OK) return rc;
+    return linear_multi_impl(q_a, s_a, M, K, levels, outputs, count, y_dtype, base + L.ws_off, L.total - L.ws_off, levels_buf,
+                             levels_bytes, levels_ready, ahead, stream);
 }
 
 // ------------------------------------------------------------------------------------------- grouped
@@ -1372,6 +1410,23 @@ __global__ void wait_probe_kernel(uint64_t limit_ns) {
     if (threadIdx.x == 0) mbar_wait(&bar, 0, kSiteProbe, limit_ns);
 }
 }  // namespace qift
+
+extern "C" int qift_calib_hbm_read(const void* buf, size_t bytes, unsigned int* sink, void* stream) {
+    if (!buf || bytes < 16) return QIFT_ERR_INVALID_ARG;
+    if (!aligned16(buf)) return QIFT_ERR_ALIGNMENT;
+    hbm_read_kernel<<<sm_count() * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint4*>(buf), bytes / 16, sink);
+    return cuda_status(cudaGetLastError());
+}
+
+extern "C" int qift_calib_mma_i8(int kblocks, double* ops, void* stream) {
+    if (kblocks < 1 || kblocks > (1 << 20)) return QIFT_ERR_INVALID_ARG;  // at ~0.3 us per k-block: a third of a second at most
+    cudaError_t e = allow_smem(mma_i8_issue_kernel, kCalibSmem);
+    if (e != cudaSuccess) return cuda_status(e);
+    const int pairs = sm_count() / 2;
+    if (ops) *ops = 2.0 * 256 * 256 * 128 * static_cast<double>(kblocks) * pairs;
+    return cuda_status(launch_pdl_pairs(mma_i8_issue_kernel, dim3(2 * pairs), dim3(kCalibThreads), kCalibSmem,
+                                        static_cast<cudaStream_t>(stream), kblocks, kWaitLimitNs));
+}
 
 extern "C" int qift_selftest_wait_timeout(int which, unsigned int limit_us, void* stream) {
     if ((which != 0 && which != 1) || limit_us == 0 || limit_us > 1000000u) return QIFT_ERR_INVALID_ARG;

@@ -99,17 +99,16 @@ __host__ __device__ constexpr int pad_step(int j) {
     return LOG_S == 9 ? 608 * j : 36 * j + ((j >> 3) << 4);
 }
 
-// CTAs are persistent: CTA b takes rows b, b + gridDim.x, ...  With bf16 input a thread asks for its 64 bytes of the
-// NEXT row (cp.async into a staging area behind the padded row, at byte stage_offset of the dynamic shared memory)
-// before it works on the current one, so the latency of global memory is covered by a whole row of arithmetic
-// instead of by occupancy, and the staged bytes occupy no registers meanwhile.  The block has a whole number of warps; threads beyond K / 32 redo the last
-// thread's work (same values to the same addresses), which keeps every branch of the kernel uniform.
+// CTAs are persistent: CTA b takes rows b, b + gridDim.x, ... (the SMs are filled once; a row's loads overlap the
+// arithmetic of the other CTAs' rows -- staging the next row ahead of time, in registers or by cp.async into shared
+// memory, was measured and lost: it costs registers or a CTA per SM).  The block has a whole number of warps; threads
+// beyond K / 32 redo the last thread's work (same values to the same addresses), which keeps every branch uniform.
 //   MID   1: a middle pass (strides 32 .. 256) precedes the last pass, whose first stride is then 512
 //   R2    stages of the last pass (0: the first pass was the only one)
 template <bool BF16_IN, bool UPPER_ONLY, int MID, int R2>
 __global__ void __launch_bounds__(kRowsMaxThreads, 2)
-quantize_rows_kernel(const void* __restrict__ X, int M, int K, int s0, int stage_offset, float clip, float inv_sqrt_b,
-                     int8_t* __restrict__ q_a, float* __restrict__ s_a) {
+quantize_rows_kernel(const void* __restrict__ X, int M, int K, int s0, float clip, float inv_sqrt_b, int8_t* __restrict__ q_a,
+                     float* __restrict__ s_a) {
     constexpr int LOG_S = MID ? 9 : 5, S = 1 << LOG_S;
     constexpr int R = 1 << R2, C = 32 >> R2, P = C / 2;
     extern __shared__ __align__(16) float row[];
@@ -128,20 +127,7 @@ quantize_rows_kernel(const void* __restrict__ X, int M, int K, int s0, int stage
     float* mid_base = row + pad_index(((t >> 4) << 9) + 2 * (t & 15));
     ulonglong2* first_dst = reinterpret_cast<ulonglong2*>(row + pad_index(32 * t));
 
-    // staging of the next row: the thread's own 64 (bf16) or 128 (fp32) bytes, copied asynchronously
-    constexpr int LOADS = BF16_IN ? 4 : 8;
-    // (piece i of all threads is contiguous, so neither the copies nor the reads meet a bank conflict)
-    uint4* stage = reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(row) + stage_offset) + threadIdx.x;
-    const int stage_step = blockDim.x;
-    const size_t row_bytes = static_cast<size_t>(K) * (BF16_IN ? 2 : 4);
-    auto fetch = [&](int m_next) {
-        const unsigned char* src = static_cast<const unsigned char*>(X) + m_next * row_bytes + static_cast<size_t>(t) * (16 * LOADS);
-#pragma unroll
-        for (int i = 0; i < LOADS; ++i)
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(stage + i * stage_step)), "l"(src + 16 * i) : "memory");
-        asm volatile("cp.async.commit_group;" ::: "memory");
-    };
-    if (BF16_IN && blockIdx.x < M) fetch(blockIdx.x);
+    constexpr int LOADS = BF16_IN ? 4 : 8;   // 16-byte pieces of the thread's 32 elements
     int parity = 0;
     for (int m = blockIdx.x; m < M; m += gridDim.x, parity ^= 1) {
         // ---- first pass: 32 contiguous elements, strides 1 .. 16
@@ -149,16 +135,9 @@ quantize_rows_kernel(const void* __restrict__ X, int M, int K, int s0, int stage
         {
             float v[32];
             uint4 w4[LOADS];
-            if constexpr (BF16_IN) {
-                asm volatile("cp.async.wait_group 0;" ::: "memory");
+            const uint4* src = reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(X) + static_cast<size_t>(m) * K * (BF16_IN ? 2 : 4)) + LOADS * t;
 #pragma unroll
-                for (int i = 0; i < LOADS; ++i) w4[i] = stage[i * stage_step];
-                if (m + static_cast<int>(gridDim.x) < M) fetch(m + gridDim.x);  // a thread re-reads only what it staged itself
-            } else {  // fp32 rows (128 bytes per thread) are read directly: staging them would cost a CTA per SM
-                const uint4* src = reinterpret_cast<const uint4*>(static_cast<const float*>(X) + static_cast<size_t>(m) * K) + 8 * t;
-#pragma unroll
-                for (int i = 0; i < LOADS; ++i) w4[i] = __ldg(src + i);
-            }
+            for (int i = 0; i < LOADS; ++i) w4[i] = __ldg(src + i);
             if constexpr (BF16_IN) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {

@@ -48,7 +48,10 @@ def clean():
                                     (513, (1000,), 256),               # one segment, four 256-wide tiles, ragged M
                                     (40, (272, 64), 512),              # row-split decode route per output
                                     (1, (256, 256, 256, 144), 256),    # single token, four outputs
-                                    (300, (200, 320), 256)])           # fused prefill route per output
+                                    (300, (200, 320), 256),            # fused prefill route per output
+                                    (1100, (520, 136), 256),           # 512-token tiles, all cut into half tiles, ragged M
+                                    (2100, (1000,), 256),              # 512-token tiles, whole ones only
+                                    (1024, (4800, 264), 128)])         # whole rounds of 512-token tiles + a tail of half tiles
 def test_forward_multi_matches_oracle(lv, M, Ns, K):
     host, gpu = make_weights(100 * lv + M, Ns, K, lv)
     x, _ = synth.activations(7 + M, M, K, max(1, K // 100))
@@ -101,4 +104,28 @@ def test_forward_multi_rejects_bad_arguments():
     with pytest.raises(qift.QiftError) as e:       # ahead buffer too small
         qift.qift_forward_multi(x, 256, gpu, lv, ahead=(gpu, K, lv, small))
     assert e.value.status == qift.ERR_WORKSPACE
+    clean()
+
+
+@pytest.mark.parametrize("M", [600, 24])
+def test_linear_multi_on_a_quantized_activation(M):
+    K, lv = 512, qift.SYM
+    host, gpu = make_weights(61, (264, 520), K, lv)
+    x, _ = synth.activations(62, M, K, 5)
+    q_a, s_a = qift.qift_quantize_act(dev(x), 512, CLIP)
+    ys, accs = qift.qift_linear_multi(q_a, s_a, gpu, lv, want_acc=True)
+    check(host, lv, x, 512, ys, accs, False)
+    clean()
+
+
+def test_calibration_kernels_run_and_leave_the_status_clean():
+    buf = torch.empty(64 << 20, dtype=torch.uint8, device="cuda").random_(0, 256)
+    L = qift.lib()
+    import ctypes
+    st = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    assert L.qift_calib_hbm_read(ctypes.c_void_p(buf.data_ptr()), buf.numel(), None, st) == qift.OK
+    ops = ctypes.c_double(0.0)
+    assert L.qift_calib_mma_i8(64, ctypes.byref(ops), st) == qift.OK
+    assert ops.value == 2.0 * 256 * 256 * 128 * 64 * (torch.cuda.get_device_properties(0).multi_processor_count // 2)
+    assert L.qift_calib_mma_i8(0, None, st) == qift.ERR_INVALID_ARG
     clean()

@@ -77,9 +77,10 @@ typedef enum {
                                       scratch N*K bytes                                            */
     QIFT_ROUTE_PREFILL_FUSED_PAIR = 6, /* CTA pairs with the codes expanded in the kernel (each CTA
                                       expands half of the tile's channels); scratch 4*M            */
-    QIFT_ROUTE_DECODE_ROWS = 7 /* 2 <= M <= 64: the activations re-laid out into the scratch, then the
-                                  row-split kernel of the grouped path (128-row items, no reduction);
-                                  scratch M*K + 256 bytes                                         */
+    QIFT_ROUTE_DECODE_ROWS = 7 /* 2 <= M <= 64: the activations re-laid out into the scratch, then a
+                                  row-split kernel of the grouped path (mma.sync up to 32 rows and for
+                                  POT; from 33 rows the tcgen05 kernel whose weight operand lives in
+                                  tensor memory); scratch M*K + 512 bytes                         */
 } qift_route;
 
 const char* qift_status_string(int status);
@@ -90,8 +91,8 @@ size_t qift_packed_bytes(int N, int K, int levels);
 
 /* Bytes of scratch qift_w2a4_linear / qift_w4a4_linear can use for this problem, rounded up to 1 KiB:
  *   M = 1                 0 (decode route);
- *   2 <= M <= 64          M*K + 256 when K is a whole number of 16-word slices (QIFT_ROUTE_DECODE_ROWS: the
- *                         activations re-laid out for the row-split kernel plus the token sums), else 0
+ *   2 <= M <= 64          M*K + 512 when K is a whole number of 16-word slices (QIFT_ROUTE_DECODE_ROWS: the
+ *                         activations re-laid out for a row-split kernel plus the token sums), else 0
  *                         for M <= 16 or 4*M above;
  *   64 < M <= 512         4*M (QIFT_ROUTE_PREFILL up to 128 rows, QIFT_ROUTE_PREFILL_FUSED_PAIR above:
  *                         the per-token sums of q_a);

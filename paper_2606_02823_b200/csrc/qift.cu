@@ -9,6 +9,7 @@
 #include "calib.cuh"
 #include "common.cuh"
 #include "decode.cuh"
+#include "decode_tc.cuh"
 #include "diag.cuh"
 #include "grouped.cuh"
 #include "kv4.cuh"
@@ -490,8 +491,16 @@ int run_prefill_fused(const uint32_t* packed, const float* s_n, int lv, const in
 }
 
 // Scratch of QIFT_ROUTE_DECODE_ROWS: the re-laid-out activations and the token sums.
-inline size_t decode_rows_scratch(int M, int K) { return ((static_cast<size_t>(M) * K + 255) & ~static_cast<size_t>(255)) + kGroupMaxM * 4; }
-inline bool decode_rows_supports(int lv, int M, int N, int K) { return M >= 2 && M <= kGroupMaxM && decode_supports(lv, M > 16 ? 16 : M, N, K); }
+inline size_t decode_rows_scratch(int M, int K) { return ((static_cast<size_t>(M) * K + 255) & ~static_cast<size_t>(255)) + kTcMaxM * 4; }
+// Row-split routes: the mma.sync kernel up to 32 token rows (PoT: up to 64), the tcgen05 weight-streaming kernel from 33
+// to 64, where it is the faster one (16 LLaMA-2-7B layers, product kernel, MNZ / INT4: 32 rows 1.9 / 2.8 TB/s against
+// 2.8 / 4.5 on mma.sync; 64 rows 1.8 / 3.2 against 1.3 / 2.5).
+inline bool tc_rows_applies(int lv, int M) { return lv != QIFT_LEVELS_POT && M > 32 && M <= kGroupMaxM; }
+inline int tc_tokens(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }   // the tensor-core N of that kernel
+inline int tc_rows_per_item(int M, int lv) { return kTcRows * tc_tiles_per_item(tc_tokens(M), codes_per_word(lv)); }
+inline bool decode_rows_supports(int lv, int M, int N, int K) {
+    return M >= 2 && (M <= kGroupMaxM || tc_rows_applies(lv, M)) && decode_supports(lv, M > 16 ? 16 : M, N, K);
+}
 int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
                     void* Y, int y_bf16, int32_t* acc_debug, void* workspace, cudaStream_t st);
 int run_forward_rows(const void* X, int x_bf16, int M, int K, int had_block, float clip, const uint32_t* packed, const float* s_n,
@@ -520,7 +529,7 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
                 route = QIFT_ROUTE_DECODE_ROWS;
         } else {
             route = (K % 16 != 0) ? QIFT_ROUTE_GENERIC : auto_prefill_route(M);
-            // 17..64 token rows: still the row-split kernel (four or eight token tiles) when its scratch was passed
+            // 17..64 token rows: still a row-split kernel when its scratch was passed
             if (decode_rows_supports(lv, M, N, K) && workspace && workspace_bytes >= decode_rows_scratch(M, K) &&
                 (reinterpret_cast<uintptr_t>(workspace) & 255u) == 0)
                 route = QIFT_ROUTE_DECODE_ROWS;
@@ -736,7 +745,7 @@ static int forward_impl(const void* X, bool host, int x_dtype, int M, int K, int
     int8_t* q_a = reinterpret_cast<int8_t*>(base + L.q_off);
     float* s_a = reinterpret_cast<float*>(base + L.sa_off);
     int rc;
-    if (decode_rows_supports(levels, M, N, K) && L.total - L.ws_off >= kGroupMaxM * sizeof(int)) {
+    if (decode_rows_supports(levels, M, N, K) && L.total - L.ws_off >= kTcMaxM * sizeof(int)) {
         // 2..64 token rows: the grouped path's quantizer writes the row-split kernel's activation layout directly
         rc = run_forward_rows(x_dev, x_dtype == QIFT_BF16, M, K, had_block, clip_ratio, packed, s_n, levels, N, y_dev,
                               y_dtype == QIFT_BF16, q_a, s_a, reinterpret_cast<int*>(base + L.ws_off), st);
@@ -941,7 +950,9 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     // Rows per work item, which also selects the kernel (dispatch_grouped): 64 / 32 for the K-split kernel, 128 for the
     // row-split kernel, 256 (two row tiles per warp, with two token tiles) when that still leaves two items per SM.
     int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : 64;  // below wide_min_m there is only M = 1
-    if (rows_per_item == kWideRows && M > 8 && M <= 16 && levels != QIFT_LEVELS_POT) {  // PoT measured slower with two tiles
+    const bool use_tc = tc_rows_applies(levels, M);                  // 33 .. 64 rows (not PoT): the tcgen05 kernel, 256-row items
+    if (use_tc) rows_per_item = tc_rows_per_item(M, levels);
+    if (!use_tc && rows_per_item == kWideRows && M > 8 && M <= 16 && levels != QIFT_LEVELS_POT) {  // PoT measured slower with two tiles
         long long items256 = 0;
         for (int i = 0; i < count; ++i) items256 += (problems[i].N + 2 * kWideRows - 1) / (2 * kWideRows);
         if (items256 >= 2ll * sm_count()) rows_per_item = 2 * kWideRows;
@@ -982,6 +993,8 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     // the row-split kernel stages one K-chunk of all tokens per copy: its q_a is chunk-major (ChunkMajorDst)
     h->q_pot_lut = (rows_per_item >= kWideRows && levels == QIFT_LEVELS_POT && M > 8) ? 1 : 0;  // the kernel's POT_LUT
     h->q_chunk_bytes = (rows_per_item >= kWideRows) ? wide_chunk_words(rows_per_item / 16, wide_token_tiles(M)) * codes_per_word(levels) : 0;
+    h->reserved[0] = use_tc ? 1 : 0;
+    if (use_tc) h->q_chunk_bytes = 0;  // that kernel reads q_a row-major (prescaled even planes, as the K-split kernel does)
     return cuda_status(cudaMemcpyAsync(plan_dev, plan_host, sizeof(GroupHeader) + static_cast<size_t>(count) * sizeof(GroupProblemDev),
                                        cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));
 }
@@ -1052,9 +1065,49 @@ int launch_grouped_wide(const GroupHeader* h, const GroupProblemDev* host, const
     return QIFT_OK;
 }
 
+// The tcgen05 weight-streaming kernel: 128-channel items, one persistent CTA per SM.  At least 132 KiB of shared memory is
+// requested whatever the stage sizes, so that two of these CTAs can never share an SM: each allocates all of tensor memory.
+template <int LV, int NTOK>
+int launch_tc(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq, cudaStream_t st,
+              bool single = false) {
+    if constexpr (LV == QIFT_LEVELS_POT) {
+        return QIFT_ERR_INVALID_ARG;
+    } else {
+        constexpr int R = tc_tiles_per_item(NTOK, codes_per_word(LV));
+        auto kernel = linear_tc_kernel<LV, NTOK, R>;
+        for (int first = 0; first < h->count; first += kGroupSlice) {
+            const int count = (h->count - first < kGroupSlice) ? h->count - first : kGroupSlice;
+            const int item_first = host[first].item_begin;
+            const int item_end = (first + count < h->count) ? host[first + count].item_begin : h->total_items;
+            size_t smem = tc_smem_bytes(NTOK, count);
+            if (smem < 132 * 1024) smem = 132 * 1024;
+            cudaError_t e = allow_smem(kernel, smem);
+            if (e != cudaSuccess) return cuda_status(e);
+            int grid = sm_count();
+            if (grid > item_end - item_first) grid = item_end - item_first;
+            GroupParams gp{dev + first, sumq, first, count, item_first, item_end, h->M, h->y_bf16, 0, 0, {}};
+            if (single) gp.use_single = 1, gp.single = host[0];
+            const int rc = cuda_status(launch_pdl(kernel, dim3(grid), dim3(kTcThreads), smem, st, gp));
+            if (rc != QIFT_OK) return rc;
+        }
+        return QIFT_OK;
+    }
+}
+template <int LV>
+int dispatch_tc(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq, cudaStream_t st,
+                bool single = false) {
+    switch (tc_tokens(h->M)) {
+        case 16: return launch_tc<LV, 16>(h, host, dev, sumq, st, single);
+        case 32: return launch_tc<LV, 32>(h, host, dev, sumq, st, single);
+        case 64: return launch_tc<LV, 64>(h, host, dev, sumq, st, single);
+        default: return launch_tc<LV, 128>(h, host, dev, sumq, st, single);
+    }
+}
+
 template <int LV>
 int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
                      cudaStream_t st) {
+    if (h->reserved[0]) return dispatch_tc<LV>(h, host, dev, sumq, st);   // the plan chose the tcgen05 kernel (33 .. 64 rows)
     // (256-row items as sixteen consumer warps were measured slower and are not dispatched.)
     if (h->rows_per_item == 2 * kWideRows) return launch_grouped_wide<LV, 2, 2, 8>(h, host, dev, sumq, st);
     if (h->rows_per_item == kWideRows && h->M > 32) return launch_grouped_wide<LV, 8, 1, 8>(h, host, dev, sumq, st);
@@ -1072,6 +1125,22 @@ int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8
                     void* Y, int y_bf16, int32_t* acc_debug, void* workspace, cudaStream_t st) {
     int8_t* q_out = static_cast<int8_t*>(workspace);
     int* sumq = reinterpret_cast<int*>(q_out + ((static_cast<size_t>(M) * K + 255) & ~static_cast<size_t>(255)));
+    if (tc_rows_applies(lv, M)) {  // 33 .. 64 rows: prescaled row-major activations + token sums, then the tcgen05 kernel
+        GroupHeader t{};
+        t.magic = kGroupMagic, t.count = 1, t.M = M, t.levels = lv, t.y_bf16 = y_bf16, t.rows_per_item = tc_rows_per_item(M, lv);
+        t.total_items = (N + t.rows_per_item - 1) / t.rows_per_item;
+        GroupProblemDev r{};
+        r.packed = packed, r.s_n = s_n, r.q_a = q_out, r.s_a = const_cast<float*>(s_a), r.Y = Y, r.acc_debug = acc_debug;
+        r.N = N, r.K = K, r.inv_sqrt_b = 1.0f;
+        int rc = cuda_status(launch_pdl(prescale_act_kernel, dim3(M), dim3(128), 0, st, q_a, M, K, lv == QIFT_LEVELS_INT4 ? 1 : 0, q_out, sumq));
+        if (rc != QIFT_OK) return rc;
+        const GroupProblemDev* none = nullptr;
+        switch (lv) {
+            case QIFT_LEVELS_MNZ: return dispatch_tc<QIFT_LEVELS_MNZ>(&t, &r, none, sumq, st, true);
+            case QIFT_LEVELS_SYM: return dispatch_tc<QIFT_LEVELS_SYM>(&t, &r, none, sumq, st, true);
+            default: return dispatch_tc<QIFT_LEVELS_INT4>(&t, &r, none, sumq, st, true);
+        }
+    }
     GroupHeader h{};
     h.magic = kGroupMagic, h.count = 1, h.M = M, h.levels = lv, h.y_bf16 = y_bf16, h.rows_per_item = kWideRows;
     h.total_items = (N + kWideRows - 1) / kWideRows;
@@ -1111,6 +1180,8 @@ int run_forward_rows(const void* X, int x_bf16, int M, int K, int had_block, flo
     rec.X = X, rec.packed = packed, rec.s_n = s_n, rec.q_a = q_scratch, rec.s_a = s_a, rec.Y = Y, rec.acc_debug = nullptr;
     rec.N = N, rec.K = K, rec.had_block = had_block, rec.item_begin = 0, rec.quant_src = 0;
     rec.inv_sqrt_b = had_block > 1 ? inv_sqrt_block(had_block) : 1.0f;
+    const bool tc = tc_rows_applies(lv, M);
+    if (tc) h.q_chunk_bytes = 0, h.rows_per_item = tc_rows_per_item(M, lv), h.total_items = (N + h.rows_per_item - 1) / h.rows_per_item;  // row-major prescaled q_a
     const bool kron = had_block > 1 && !is_pow2(had_block);
     auto qk = x_bf16 ? (kron ? quantize_act_grouped_kernel<true, true> : quantize_act_grouped_kernel<true, false>)
                      : (kron ? quantize_act_grouped_kernel<false, true> : quantize_act_grouped_kernel<false, false>);
@@ -1121,6 +1192,13 @@ int run_forward_rows(const void* X, int x_bf16, int M, int K, int had_block, flo
     int rc = cuda_status(launch_pdl(qk, dim3(M), dim3(kRowThreads), smem, st, none, sumq, M, clip, lv == QIFT_LEVELS_INT4 ? 1 : 0,
                                     h.q_chunk_bytes, h.q_pot_lut, 1, rec));
     if (rc != QIFT_OK) return rc;
+    if (tc) {
+        switch (lv) {
+            case QIFT_LEVELS_MNZ: return dispatch_tc<QIFT_LEVELS_MNZ>(&h, &rec, none, sumq, st, true);
+            case QIFT_LEVELS_SYM: return dispatch_tc<QIFT_LEVELS_SYM>(&h, &rec, none, sumq, st, true);
+            default: return dispatch_tc<QIFT_LEVELS_INT4>(&h, &rec, none, sumq, st, true);
+        }
+    }
 #define QIFT_ROWS_CASE(LV)                                                                                          \
     case LV:                                                                                                        \
         return M > 32 ? launch_grouped_wide<LV, 8, 1, 8>(&h, &rec, none, sumq, st, true)                            \

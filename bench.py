@@ -386,16 +386,24 @@ def run_gpu(args):
         "clocks": clocks,
     }
     if rank == 0 and world == 1 and not args.no_prefill:
-        out["mixed_stack"] = run_mixed_stack(torch, qift, L, device, gen, args)
-        out["batched_decode"] = run_batched_decode(torch, qift, L, device, gen, args)
+        want = set(args.sections.split(",")) if args.sections else None
+        on = lambda name: want is None or name in want
         ceilings = calibrate_ceilings(torch, L, device)
         out["ceilings"] = ceilings
         out["roofline"]["read_only_ceiling_gbs"] = ceilings["hbm_read_only_gbs"]
         out["roofline"]["frac_of_read_only_ceiling"] = round(out["roofline"]["achieved"] / ceilings["hbm_read_only_gbs"], 4)
-        out["prefill"] = run_prefill(torch, qift, L, device, gen, pk, ceilings)
-        out["mid_m"] = run_mid_m(torch, qift, L, device, gen, pk, ceilings)
-        out["kv4"] = run_kv4(torch, qift, L, pk)
-        out["diagnostics"] = run_diagnostics(torch, qift, pk)
+        if on("mixed_stack"):
+            out["mixed_stack"] = run_mixed_stack(torch, qift, L, device, gen, args)
+        if on("batched_decode"):
+            out["batched_decode"] = run_batched_decode(torch, qift, L, device, gen, args, ceilings)
+        if on("prefill"):
+            out["prefill"] = run_prefill(torch, qift, L, device, gen, pk, ceilings)
+        if on("mid_m"):
+            out["mid_m"] = run_mid_m(torch, qift, L, device, gen, pk, ceilings)
+        if on("kv4"):
+            out["kv4"] = run_kv4(torch, qift, L, pk)
+        if on("diagnostics"):
+            out["diagnostics"] = run_diagnostics(torch, qift, pk)
     if rank == 0 and world == 1 and not args.no_cpu:
         out["cpu_baseline"] = cpu_baseline(budget_s=12.0)
         out["cpu_baseline"]["other_configs"] = oracle_extra_timings()
@@ -592,18 +600,20 @@ def mixed_prefill(torch, qift, L, device, gen, args, n4):
                                "tops": round(ops / (ms_percall * 1e-3) / 1e12, 1), "launches_per_step": 3 * len(mods)}}
 
 
-def run_batched_decode(torch, qift, L, device, gen, args):
-    """Config 3: LLaMA-3.1-8B shapes, batched decode at M = 1, 4, 16 token rows, PoT {+-1,+-4} against the standard
-    {-2,-1,0,+1} set; grouped API (2 launches per step), 16 layers of distinct weights (0.87 GB per level set, larger
-    than L2), every module on its own activation.  Bytes = packed weights + scales + activations + outputs."""
+def run_batched_decode(torch, qift, L, device, gen, args, ceilings):
+    """Config 3: LLaMA-3.1-8B shapes, batched decode at M = 1, 4, 16 token rows (plus 32 and 64), PoT {+-1,+-4} against the
+    standard {-2,-1,0,+1} set; grouped API (2 launches per step), 16 layers of distinct weights (0.87 GB per level set,
+    larger than L2), every module on its own activation.  Bytes = packed weights + scales + activations + outputs.
+    Each point carries the fraction of the measured read-only HBM ceiling; PoT also carries the ceiling its decode
+    arithmetic sets (see pot_bound)."""
     vp = ctypes.c_void_p
     st = vp(torch.cuda.current_stream().cuda_stream)
     layers = max(1, min(16, args.layers))
     rows = []
     for name, lv in (("PoT", qift.POT), ("SYM", qift.SYM)):
-        base = build_stack(torch, qift, synth.LLAMA31_8B, layers, 16, lambda l, lv=lv: lv, 6000 + lv, torch.float32, torch.float32,
+        base = build_stack(torch, qift, synth.LLAMA31_8B, layers, 64, lambda l, lv=lv: lv, 6000 + lv, torch.float32, torch.float32,
                            device, gen)
-        for M in (1, 4, 16):
+        for M in (1, 4, 16, 32, 64):
             plan = qift.qift_group_plan([(m.x[:M].contiguous(), m.packed, m.s_n, m.B) for m in base], lv, CLIP)
             algo = sum(product_bytes(M, m.N, m.K, m.bits) + quant_bytes(M, m.K) for m in base)
 
@@ -611,23 +621,31 @@ def run_batched_decode(torch, qift, L, device, gen, args):
                 rc = L.qift_group_forward(vp(plan.host.data_ptr()), vp(plan.dev.data_ptr()), st)
                 assert rc == 0, rc
 
-            for _ in range(5):
-                step()
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            steps = max(3, min(args.steps, 100))
-            e0.record()
-            for _ in range(steps):
-                step()
-            e1.record()
-            torch.cuda.synchronize()
-            ms = e0.elapsed_time(e1) / steps
+            ms = time_ms(torch, step, max(3, min(args.steps, 100)), warm=5)
+            gbs = algo / (ms * 1e-3) / 1e9
             rows.append({"levels": name, "M": M, "ms_per_step": round(ms, 5), "tokens_per_s": round(M / (ms * 1e-3), 1),
-                         "value": round(algo / (ms * 1e-3) / 1e9, 1), "unit": "GB/s",
-                         "pct_of_8TBs": round(100 * algo / (ms * 1e-3) / 8e12, 1)})
+                         "value": round(gbs, 1), "unit": "GB/s", "pct_of_8TBs": round(100 * gbs / 8000.0, 1),
+                         "frac_of_read_only_ceiling": round(gbs / ceilings["hbm_read_only_gbs"], 3),
+                         "kernel": "linear_tc_kernel (tcgen05, weights in tensor memory)" if (M > 32 and lv != qift.POT)
+                                   else "linear_grouped_wide_kernel (mma.sync)" if (M > 1 or lv == qift.POT) else "linear_grouped_kernel (mma.sync)"})
             del plan
         del base
-    return {"workload": f"config 3: LLaMA-3.1-8B shapes, {layers} layers, grouped API, whole step (quantizer + product)", "points": rows}
+    # PoT {-4,-1,+1,+4} is affine in the two code BITS (5 b1 + 3 b0 - 4) but not in the code, so every packed word needs two
+    # masked operands (one per bit) and two tensor-core products where MNZ / SYM need one: per 128 bytes of packed weights
+    # 8 LOP3 and 2 mma.sync.m16n8k32 with one 8-token tile.  Ceilings from the committed ncu capture of this kernel at
+    # M = 1 (4-layer case: 219.0 MB in 71.46 us = 3065 GB/s with the ALU pipe 52.0 % and the IMMA pipe 46.8 % busy):
+    # rate at which each pipe would be full = 3065 / utilisation.
+    capture_gbs, alu_frac, imma_frac = 3065.0, 0.5198, 0.4678
+    alu_bound, mma_bound = capture_gbs / alu_frac, capture_gbs / imma_frac
+    pot = [r for r in rows if r["levels"] == "PoT" and r["M"] <= 8]
+    best = max(r["value"] for r in pot) if pot else 0.0
+    return {"workload": f"config 3: LLaMA-3.1-8B shapes, {layers} layers, grouped API, whole step (quantizer + product)", "points": rows,
+            "pot_bound": {"bound": "alu", "unit": "GB/s", "achieved": best, "peak": round(alu_bound, 1), "frac": round(best / alu_bound, 3),
+                          "logic_pipe_ceiling_gbs": round(alu_bound, 1), "legacy_tensor_issue_ceiling_gbs": round(mma_bound, 1),
+                          "derivation": "per 128 B of packed PoT weights 8 LOP3 (two bit planes x four code planes) and 2 mma.sync.m16n8k32 "
+                                        "for one 8-token tile, twice what MNZ / SYM need; ceilings = rate of the committed ncu capture "
+                                        "(3065 GB/s) divided by the utilisation it shows for the ALU pipe (0.52) and the IMMA pipe "
+                                        "(0.47): constants of that capture, not measured in this run"}}
 
 
 def run_kv4(torch, qift, L, pk):
@@ -999,6 +1017,8 @@ def main():
     ap.add_argument("--layers", type=int, default=N_LAYERS, help="layers of distinct weights per step (32 = the full workload)")
     ap.add_argument("--no-prefill", action="store_true", help="skip the M=2048 prefill measurement")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    ap.add_argument("--sections", default="", help="comma-separated subset of the secondary blocks to run (mixed_stack, batched_decode, "
+                                                   "prefill, mid_m, kv4, diagnostics); default: all")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

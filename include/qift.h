@@ -77,10 +77,9 @@ typedef enum {
                                       scratch N*K bytes                                            */
     QIFT_ROUTE_PREFILL_FUSED_PAIR = 6, /* CTA pairs with the codes expanded in the kernel (each CTA
                                       expands half of the tile's channels); scratch 4*M            */
-    QIFT_ROUTE_DECODE_ROWS = 7 /* 2 <= M <= 64: the activations re-laid out into the scratch, then a
-                                  row-split kernel of the grouped path (mma.sync up to 32 rows and for
-                                  POT; from 33 rows the tcgen05 kernel whose weight operand lives in
-                                  tensor memory); scratch M*K + 512 bytes                         */
+    QIFT_ROUTE_DECODE_ROWS = 7 /* 2 <= M <= 64: the activations re-laid out into the scratch, then the
+                                  row-split kernel of the grouped path (128-row items, no reduction);
+                                  scratch M*K + 512 bytes                                         */
 } qift_route;
 
 const char* qift_status_string(int status);

@@ -421,30 +421,4 @@ linear_tc_kernel(const GroupParams gp) {
     }
 }
 
-// Public q_a ([M][K] plain bytes) -> the same rows with the even code planes prescaled (two-bit: words 0 and 2 of every
-// 16-byte group times 4; INT4: times 16) plus the token sums.  One CTA per token row.
-__global__ void __launch_bounds__(128)
-prescale_act_kernel(const int8_t* __restrict__ q_a, int M, int K, int int4_weights, int8_t* __restrict__ q_out, int* __restrict__ sumq) {
-    __shared__ int red[4];
-    pdl_launch_dependents();
-    pdl_wait();
-    const int m = blockIdx.x;
-    const uint4* src = reinterpret_cast<const uint4*>(q_a + static_cast<size_t>(m) * K);
-    uint4* dst = reinterpret_cast<uint4*>(q_out + static_cast<size_t>(m) * K);
-    int total = 0;
-    for (int g = threadIdx.x; g < K / 16; g += blockDim.x) {
-        uint4 v = src[g];
-        total = __dp4a(static_cast<int>(v.x), 0x01010101, __dp4a(static_cast<int>(v.y), 0x01010101, total));
-        total = __dp4a(static_cast<int>(v.z), 0x01010101, __dp4a(static_cast<int>(v.w), 0x01010101, total));
-        if (int4_weights) v.x = (v.x << 4) & 0xf0f0f0f0u, v.z = (v.z << 4) & 0xf0f0f0f0u;   // |q| <= 8: the products fit a byte
-        else v.x = (v.x << 2) & 0xfcfcfcfcu, v.z = (v.z << 2) & 0xfcfcfcfcu;
-        dst[g] = v;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = total;
-    __syncthreads();
-    if (threadIdx.x == 0) sumq[m] = red[0] + red[1] + red[2] + red[3];
-}
-
 }  // namespace qift

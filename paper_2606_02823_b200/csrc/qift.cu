@@ -491,16 +491,14 @@ int run_prefill_fused(const uint32_t* packed, const float* s_n, int lv, const in
 }
 
 // Scratch of QIFT_ROUTE_DECODE_ROWS: the re-laid-out activations and the token sums.
-inline size_t decode_rows_scratch(int M, int K) { return ((static_cast<size_t>(M) * K + 255) & ~static_cast<size_t>(255)) + kTcMaxM * 4; }
-// Row-split routes: the mma.sync kernel up to 32 token rows (PoT: up to 64), the tcgen05 weight-streaming kernel from 33
-// to 64, where it is the faster one (16 LLaMA-2-7B layers, product kernel, MNZ / INT4: 32 rows 1.9 / 2.8 TB/s against
-// 2.8 / 4.5 on mma.sync; 64 rows 1.8 / 3.2 against 1.3 / 2.5).
+inline size_t decode_rows_scratch(int M, int K) { return ((static_cast<size_t>(M) * K + 255) & ~static_cast<size_t>(255)) + 512; }
+// Grouped plans: the row-split mma.sync kernel up to 32 token rows (PoT: up to 64), the tcgen05 weight-streaming kernel
+// from 33 to 64, where it is the faster one (16 LLaMA-2-7B layers, product kernel, MNZ / INT4: 32 rows 1.9 / 2.8 TB/s
+// against 2.8 / 4.5 on mma.sync; 64 rows 1.8 / 3.2 against 1.3 / 2.5).
 inline bool tc_rows_applies(int lv, int M) { return lv != QIFT_LEVELS_POT && M > 32 && M <= kGroupMaxM; }
 inline int tc_tokens(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }   // the tensor-core N of that kernel
 inline int tc_rows_per_item(int M, int lv) { return kTcRows * tc_tiles_per_item(tc_tokens(M), codes_per_word(lv)); }
-inline bool decode_rows_supports(int lv, int M, int N, int K) {
-    return M >= 2 && (M <= kGroupMaxM || tc_rows_applies(lv, M)) && decode_supports(lv, M > 16 ? 16 : M, N, K);
-}
+inline bool decode_rows_supports(int lv, int M, int N, int K) { return M >= 2 && M <= kGroupMaxM && decode_supports(lv, M > 16 ? 16 : M, N, K); }
 int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
                     void* Y, int y_bf16, int32_t* acc_debug, void* workspace, cudaStream_t st);
 int run_forward_rows(const void* X, int x_bf16, int M, int K, int had_block, float clip, const uint32_t* packed, const float* s_n,
@@ -745,7 +743,7 @@ static int forward_impl(const void* X, bool host, int x_dtype, int M, int K, int
     int8_t* q_a = reinterpret_cast<int8_t*>(base + L.q_off);
     float* s_a = reinterpret_cast<float*>(base + L.sa_off);
     int rc;
-    if (decode_rows_supports(levels, M, N, K) && L.total - L.ws_off >= kTcMaxM * sizeof(int)) {
+    if (decode_rows_supports(levels, M, N, K) && L.total - L.ws_off >= 512) {
         // 2..64 token rows: the grouped path's quantizer writes the row-split kernel's activation layout directly
         rc = run_forward_rows(x_dev, x_dtype == QIFT_BF16, M, K, had_block, clip_ratio, packed, s_n, levels, N, y_dev,
                               y_dtype == QIFT_BF16, q_a, s_a, reinterpret_cast<int*>(base + L.ws_off), st);
@@ -1125,22 +1123,8 @@ int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8
                     void* Y, int y_bf16, int32_t* acc_debug, void* workspace, cudaStream_t st) {
     int8_t* q_out = static_cast<int8_t*>(workspace);
     int* sumq = reinterpret_cast<int*>(q_out + ((static_cast<size_t>(M) * K + 255) & ~static_cast<size_t>(255)));
-    if (tc_rows_applies(lv, M)) {  // 33 .. 64 rows: prescaled row-major activations + token sums, then the tcgen05 kernel
-        GroupHeader t{};
-        t.magic = kGroupMagic, t.count = 1, t.M = M, t.levels = lv, t.y_bf16 = y_bf16, t.rows_per_item = tc_rows_per_item(M, lv);
-        t.total_items = (N + t.rows_per_item - 1) / t.rows_per_item;
-        GroupProblemDev r{};
-        r.packed = packed, r.s_n = s_n, r.q_a = q_out, r.s_a = const_cast<float*>(s_a), r.Y = Y, r.acc_debug = acc_debug;
-        r.N = N, r.K = K, r.inv_sqrt_b = 1.0f;
-        int rc = cuda_status(launch_pdl(prescale_act_kernel, dim3(M), dim3(128), 0, st, q_a, M, K, lv == QIFT_LEVELS_INT4 ? 1 : 0, q_out, sumq));
-        if (rc != QIFT_OK) return rc;
-        const GroupProblemDev* none = nullptr;
-        switch (lv) {
-            case QIFT_LEVELS_MNZ: return dispatch_tc<QIFT_LEVELS_MNZ>(&t, &r, none, sumq, st, true);
-            case QIFT_LEVELS_SYM: return dispatch_tc<QIFT_LEVELS_SYM>(&t, &r, none, sumq, st, true);
-            default: return dispatch_tc<QIFT_LEVELS_INT4>(&t, &r, none, sumq, st, true);
-        }
-    }
+    // (The tcgen05 kernel serves grouped plans only: one product has too few 256-channel items to fill the SMs -- a
+    // LLaMA-3.1-8B layer of seven calls at 64 rows takes 374 us on it against 190 us on this kernel.)
     GroupHeader h{};
     h.magic = kGroupMagic, h.count = 1, h.M = M, h.levels = lv, h.y_bf16 = y_bf16, h.rows_per_item = kWideRows;
     h.total_items = (N + kWideRows - 1) / kWideRows;
@@ -1180,8 +1164,6 @@ int run_forward_rows(const void* X, int x_bf16, int M, int K, int had_block, flo
     rec.X = X, rec.packed = packed, rec.s_n = s_n, rec.q_a = q_scratch, rec.s_a = s_a, rec.Y = Y, rec.acc_debug = nullptr;
     rec.N = N, rec.K = K, rec.had_block = had_block, rec.item_begin = 0, rec.quant_src = 0;
     rec.inv_sqrt_b = had_block > 1 ? inv_sqrt_block(had_block) : 1.0f;
-    const bool tc = tc_rows_applies(lv, M);
-    if (tc) h.q_chunk_bytes = 0, h.rows_per_item = tc_rows_per_item(M, lv), h.total_items = (N + h.rows_per_item - 1) / h.rows_per_item;  // row-major prescaled q_a
     const bool kron = had_block > 1 && !is_pow2(had_block);
     auto qk = x_bf16 ? (kron ? quantize_act_grouped_kernel<true, true> : quantize_act_grouped_kernel<true, false>)
                      : (kron ? quantize_act_grouped_kernel<false, true> : quantize_act_grouped_kernel<false, false>);
@@ -1192,13 +1174,6 @@ int run_forward_rows(const void* X, int x_bf16, int M, int K, int had_block, flo
     int rc = cuda_status(launch_pdl(qk, dim3(M), dim3(kRowThreads), smem, st, none, sumq, M, clip, lv == QIFT_LEVELS_INT4 ? 1 : 0,
                                     h.q_chunk_bytes, h.q_pot_lut, 1, rec));
     if (rc != QIFT_OK) return rc;
-    if (tc) {
-        switch (lv) {
-            case QIFT_LEVELS_MNZ: return dispatch_tc<QIFT_LEVELS_MNZ>(&h, &rec, none, sumq, st, true);
-            case QIFT_LEVELS_SYM: return dispatch_tc<QIFT_LEVELS_SYM>(&h, &rec, none, sumq, st, true);
-            default: return dispatch_tc<QIFT_LEVELS_INT4>(&h, &rec, none, sumq, st, true);
-        }
-    }
 #define QIFT_ROWS_CASE(LV)                                                                                          \
     case LV:                                                                                                        \
         return M > 32 ? launch_grouped_wide<LV, 8, 1, 8>(&h, &rec, none, sumq, st, true)                            \

@@ -432,6 +432,34 @@ def test_grouped_forward_long_list(name, M):
         check_outputs(y, acc, y_ref, acc_ref, False)
 
 
+@pytest.mark.parametrize("name", ["MNZ", "SYM", "INT4"])
+@pytest.mark.parametrize("M", [33, 64])
+def test_grouped_forward_tensor_memory_kernel_many_items(name, M):
+    # 33 .. 64 token rows of a plan run on the tcgen05 kernel whose weight operand lives in tensor memory.  More
+    # 256-channel items than SMs, so CTAs take several items each (both accumulator buffers, the operand ring wrapping
+    # across item boundaries); an odd number of 16-word slices per item (the two expander warps of a lane quarter swap
+    # parity from item to item); ragged N: a last item with one valid 128-channel block, rows beyond N inside a block
+    lv = LEVELS[name][0]
+    k_odd = 1408 if lv == oracle.INT4 else 2816          # 11 slices per item
+    shapes = [(33000, 512), (2304, 4096), (1000, k_odd), (6200, 1024), (300, 256)]
+    probs, refs = [], []
+    for i, (N, K) in enumerate(shapes):
+        rng = np.random.default_rng(900 + i)
+        codes = rng.integers(0, 16 if lv == oracle.INT4 else 4, (N, K), dtype=np.uint8)
+        s_n = (0.005 + 0.01 * rng.random(N)).astype(np.float32)
+        x, _ = synth.activations(920 + i, M, K, max(1, K // 100))
+        B = synth.had_block_for(K)
+        q_ref, sa_ref = oracle.quantize_act(x, B, 0.9)
+        refs.append(oracle.linear(codes, lv, s_n, q_ref, sa_ref))
+        probs.append((dev(x), dev(oracle.pack(codes, lv).view(np.int32)), dev(s_n), B))
+    plan = qift.qift_group_plan(probs, lv, 0.9, want_acc=True)
+    for _ in range(2):          # twice: the second run starts from the first one's tensor-memory and shared-memory contents
+        outs = qift.qift_group_forward(plan)
+        assert_status_clean()
+        for (y_ref, acc_ref), y, acc in zip(refs, outs, plan.accs):
+            check_outputs(y, acc, y_ref, acc_ref, False)
+
+
 @pytest.mark.parametrize("M", [1, 7])
 def test_grouped_shared_activation(M):
     # q/k/v-style and gate/up-style modules read one activation: the plan quantizes it once (the buffers of the

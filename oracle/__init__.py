@@ -6,7 +6,8 @@ code with the CUDA library and must never be imported by it.  Only tests, the sm
 CPU-baseline / reference legs of the benchmark may use this package.
 
 All arrays are numpy, C-contiguous.  Level-set ids: 0 MNZ {-3,-1,+1,+3} (half-scale form of
-{+-0.5,+-1.5}), 1 PoT-MNZ {-4,-1,+1,+4}, 2 SYM-INT {-2,-1,0,+1}, 3 INT4 (-8..7).
+{+-0.5,+-1.5}), 1 PoT-MNZ {-4,-1,+1,+4}, 2 SYM-INT {-2,-1,0,+1}, 3 INT4 (-8..7), 4 INT3 (-4..3, the W3A4
+configuration of Sec. 4.4).
 Scale modes: 0 given, 1 max-range, 2 MSE sweep over 80 clipping ratios.
 """
 from __future__ import annotations
@@ -17,7 +18,7 @@ import subprocess
 
 import numpy as np
 
-MNZ, POT, SYM, INT4 = 0, 1, 2, 3
+MNZ, POT, SYM, INT4, INT3 = 0, 1, 2, 3, 4
 SCALE_GIVEN, SCALE_ABSMAX, SCALE_MSE = 0, 1, 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -58,8 +59,12 @@ def level_value(lv: int, code: int) -> int:
     return int(lib().orc_level_value(int(lv), int(code)))
 
 
+def num_codes(lv: int) -> int:
+    return 16 if lv == INT4 else 8 if lv == INT3 else 4
+
+
 def level_table(lv: int):
-    return [level_value(lv, c) for c in range(16 if lv == INT4 else 4)]
+    return [level_value(lv, c) for c in range(num_codes(lv))]
 
 
 def num_candidates() -> int:
@@ -162,6 +167,7 @@ def assign_codes(W, lv: int, s_n):
 
 
 def codes_per_word(lv: int) -> int:
+    """Codes per 32-bit word (INT3: of its two-bit plane; K must then be a multiple of 32)."""
     return 8 if lv == INT4 else 16
 
 
@@ -174,7 +180,7 @@ def pack(codes, lv: int):
     """codes uint8 [N,K] -> flat uint32 buffer in the tiled layout."""
     codes = np.ascontiguousarray(codes, dtype=np.uint8)
     N, K = codes.shape
-    per = codes_per_word(lv)
+    per = 32 if lv == INT3 else codes_per_word(lv)
     assert K % per == 0
     out = np.empty((packed_words(N, K, lv),), dtype=np.uint32)
     lib().orc_pack(codes.ctypes.data_as(ctypes.c_void_p), N, K, int(lv),

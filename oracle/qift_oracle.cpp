@@ -24,6 +24,9 @@
 //   orc_assign_codes     Sec. 3.5: every weight goes to the nearest level times the scale; Eq. 1 for SYM-INT, INT4.
 //   orc_pack / unpack    Sec. 3.3 (a code has two bits): 16 two-bit codes (8 nibbles) per 32-bit word,
 //                        words stored in 16-row x 128-word tiles (layout comment at orc_pack).
+//   INT3 (level set 4)   Sec. 4.4: the W3A4 configuration that the mixed-precision tables compare with at three
+//                        bits per weight -- Eq. 1 with b = 3, levels -4..3, same per-channel scale rules;
+//                        stored as a two-bit plane plus a one-bit plane (layout comment at orc_pack).
 //   orc_int_matmul       Sec. 3.6 decoded small signed integer levels times integer activations.
 //   orc_epilogue*        Sec. 1: the channel scale is applied after the integer product, in the epilogue.
 //   orc_kv4_quantize     Sec. 4.1: the KV cache is quantized to four bits asymmetrically with a
@@ -53,7 +56,7 @@
 
 namespace {
 
-enum Levels { LV_MNZ = 0, LV_POT = 1, LV_SYM = 2, LV_INT4 = 3 };
+enum Levels { LV_MNZ = 0, LV_POT = 1, LV_SYM = 2, LV_INT4 = 3, LV_INT3 = 4 };
 enum ScaleMode { SC_GIVEN = 0, SC_ABSMAX = 1, SC_MSE = 2 };
 
 constexpr int kNumCandidates = 80;  // clipping ratios 1.00, 0.99, ..., 0.21
@@ -64,6 +67,10 @@ int level_of(int lv, int code) {
         case LV_MNZ: { const int t[4] = {-3, -1, +1, +3}; return t[code & 3]; }
         case LV_POT: { const int t[4] = {-4, -1, +1, +4}; return t[code & 3]; }
         case LV_SYM: { const int t[4] = {-2, -1, 0, +1}; return t[code & 3]; }
+        case LV_INT3: {  // two's-complement three-bit field
+            int c = code & 7;
+            return c >= 4 ? c - 8 : c;
+        }
         default: {  // INT4: two's-complement nibble
             int c = code & 15;
             return c >= 8 ? c - 16 : c;
@@ -77,6 +84,7 @@ float top_level(int lv) {
         case LV_MNZ: return 3.0f;
         case LV_POT: return 4.0f;
         case LV_SYM: return 1.0f;
+        case LV_INT3: return 3.0f;
         default: return 7.0f;
     }
 }
@@ -94,6 +102,9 @@ int code_of(int lv, float w, float s) {
     }
     if (lv == LV_SYM) {     // Eq. 1, b = 2: round half to even, clip to [-2, 1]
         return clampi((int)std::rint(t), -2, 1) + 2;
+    }
+    if (lv == LV_INT3) {    // Eq. 1, b = 3: clip to [-4, 3]
+        return clampi((int)std::rint(t), -4, 3) & 7;
     }
     return clampi((int)std::rint(t), -8, 7) & 15;  // Eq. 1, b = 4
 }
@@ -323,17 +334,56 @@ static size_t word_address(int n, int j, int words_per_row) {
     return tile + (size_t)(((slice * 2 + half) * 32 + g * 4 + quad) * 4 + e);
 }
 
+// Three-bit codes (INT3) are stored as two planes, interleaved slice by slice so that any run of slices of
+// a row block is one contiguous piece of memory:
+//   low plane:  the two low bits of every code, 16 per word, bit positions as for the two-bit sets;
+//   high plane: the third bit, 32 per word.  High word h of a row covers low words 2h and 2h+1; the bit of
+//               code k = 16 j + 4 t + b (low word j, plane t, byte b) sits in byte b at position
+//               4 (j % 2) + {0, 2, 1, 3}[t].
+// A slice is 16 low words (256 codes) of the 16 rows of a row block: 384 words = 256 low words in the
+// group order of the two-bit layout (group (half * 32 + (row % 8) * 4 + quad), word j % 4 inside) followed
+// by 128 high words in groups of four: group ((row % 8) * 4 + quad), quad = (j % 16) / 4, holds the two
+// high words of that quad for row half 0 and then for row half 1 (word 2 * half + (j / 2) % 2 of the group).
+// Row blocks outermost (24 * pitch words each, pitch = low words per row padded to 16), slices in
+// ascending k.  K must be a multiple of 32.
+static size_t int3_low_address(int n, int j, int pitch) {
+    const int rb = n / 16, r = n % 16, half = r / 8, g = r % 8;
+    const int slice = j / 16, quad = (j % 16) / 4, e = j % 4;
+    return (size_t)rb * 24 * pitch + (size_t)slice * 384 + (size_t)((half * 32 + g * 4 + quad) * 4 + e);
+}
+static size_t int3_high_address(int n, int j, int pitch) {  // j: the LOW word index of the code
+    const int rb = n / 16, r = n % 16, half = r / 8, g = r % 8;
+    const int slice = j / 16, quad = (j % 16) / 4, pair = (j / 2) % 2;
+    return (size_t)rb * 24 * pitch + (size_t)slice * 384 + 256 + (size_t)((g * 4 + quad) * 4 + 2 * half + pair);
+}
+static int int3_high_bit(int j, int t, int b) {
+    const int order[4] = {0, 2, 1, 3};
+    return 8 * b + 4 * (j % 2) + order[t];
+}
+
 long long orc_packed_words(int N, int K, int lv) {
+    if (lv == LV_INT3) return (long long)pad16(N) * pad16(K / 16) * 3 / 2;
     const int per = (lv == LV_INT4) ? 8 : 16;
     return (long long)pad16(N) * pad16(K / per);
 }
 
 void orc_pack(const uint8_t* codes, int N, int K, int lv, uint32_t* packed) {
+    const long long total = orc_packed_words(N, K, lv);
+    for (long long i = 0; i < total; ++i) packed[i] = 0;
+    if (lv == LV_INT3) {
+        const int pitch = pad16(K / 16);
+        for (int n = 0; n < N; ++n)
+            for (int k = 0; k < K; ++k) {
+                const int j = k / 16, t = (k % 16) / 4, b = k % 4;
+                const uint32_t c = codes[(size_t)n * K + k] & 7u;
+                packed[int3_low_address(n, j, pitch)] |= (c & 3u) << (8 * b + 2 * t);
+                packed[int3_high_address(n, j, pitch)] |= (c >> 2) << int3_high_bit(j, t, b);
+            }
+        return;
+    }
     const int per = (lv == LV_INT4) ? 8 : 16;
     const int bits = (lv == LV_INT4) ? 4 : 2;
     const int words = K / per;
-    const long long total = orc_packed_words(N, K, lv);
-    for (long long i = 0; i < total; ++i) packed[i] = 0;
     for (int n = 0; n < N; ++n) {
         for (int j = 0; j < words; ++j) {
             uint32_t w = 0;
@@ -348,6 +398,17 @@ void orc_pack(const uint8_t* codes, int N, int K, int lv, uint32_t* packed) {
 }
 
 void orc_unpack(const uint32_t* packed, int N, int K, int lv, uint8_t* codes) {
+    if (lv == LV_INT3) {
+        const int pitch = pad16(K / 16);
+        for (int n = 0; n < N; ++n)
+            for (int k = 0; k < K; ++k) {
+                const int j = k / 16, t = (k % 16) / 4, b = k % 4;
+                const uint32_t low = (packed[int3_low_address(n, j, pitch)] >> (8 * b + 2 * t)) & 3u;
+                const uint32_t high = (packed[int3_high_address(n, j, pitch)] >> int3_high_bit(j, t, b)) & 1u;
+                codes[(size_t)n * K + k] = (uint8_t)(low | (high << 2));
+            }
+        return;
+    }
     const int per = (lv == LV_INT4) ? 8 : 16;
     const int bits = (lv == LV_INT4) ? 4 : 2;
     const int words = K / per;

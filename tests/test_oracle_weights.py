@@ -49,6 +49,11 @@ def test_level_tables_match_the_paper():
     # INT4 is Eq. 1's range -8..7 in two's complement
     assert sorted(oracle.level_table(oracle.INT4)) == list(range(-8, 8))
     assert all(((v + 16) & 15) == c for c, v in enumerate(oracle.level_table(oracle.INT4)))
+    # INT3 (the W3A4 configuration of Sec. 4.4) is Eq. 1's range for b = 3, -2^(b-1) .. 2^(b-1) - 1, in two's complement
+    assert sorted(oracle.level_table(oracle.INT3)) == list(range(-(2 ** 2), 2 ** 2))
+    assert all(((v + 8) & 7) == c for c, v in enumerate(oracle.level_table(oracle.INT3)))
+    # plane form used by the storage: level = (code & 3) - 4 (code >> 2)
+    assert all(oracle.level_value(oracle.INT3, c) == (c & 3) - 4 * (c >> 2) for c in range(8))
 
 
 def test_inner_outer_ratio_is_scale_invariant():
@@ -69,7 +74,7 @@ def test_affine_bit_plane_identity():
 
 
 # ----------------------------------------------------------------------------- nearest level (P7)
-@pytest.mark.parametrize("name", ["MNZ", "POT", "SYM", "INT4"])
+@pytest.mark.parametrize("name", ["MNZ", "POT", "SYM", "INT4", "INT3"])
 def test_nearest_level_brute_force(name):
     lv = getattr(oracle, name)
     table = np.array(oracle.level_table(lv), dtype=np.float64)
@@ -106,6 +111,9 @@ def test_nearest_level_at_the_thresholds():
     w = np.array([[-8.5, -7.5, 6.5, 7.5, 100.0, -100.0, 0.0]], dtype=np.float32)
     q = [-8, -8, 6, 7, 7, -8, 0]
     assert oracle.assign_codes(w, oracle.INT4, one)[0].tolist() == [v & 15 for v in q]
+    w = np.array([[-4.5, -3.5, -2.5, 2.5, 3.5, 0.5, 1.5, 50.0, -50.0, 0.0]], dtype=np.float32)
+    q = [-4, -4, -2, 2, 3, 0, 2, 3, -4, 0]        # ties to even, then the clip to [-4, 3]
+    assert oracle.assign_codes(w, oracle.INT3, one)[0].tolist() == [v & 7 for v in q]
     # a zero weight: MNZ/PoT code 1 (level -1), SYM code 2 (level 0), INT4 nibble 0
     z = np.zeros((1, 4), dtype=np.float32)
     assert oracle.assign_codes(z, oracle.MNZ, one)[0].tolist() == [1] * 4
@@ -118,7 +126,7 @@ def test_nearest_level_at_the_thresholds():
 def test_absmax_scale_and_zero_row():
     W = synth.gaussian_weights(0, 8, 64)
     W[3] = 0
-    for lv, top in ((oracle.MNZ, 3), (oracle.POT, 4), (oracle.SYM, 1), (oracle.INT4, 7)):
+    for lv, top in ((oracle.MNZ, 3), (oracle.POT, 4), (oracle.SYM, 1), (oracle.INT4, 7), (oracle.INT3, 3)):
         s, idx = oracle.weight_scale(W, lv, oracle.SCALE_ABSMAX)
         ref = np.abs(W).max(1) / np.float32(top)
         ref[3] = 1.0
@@ -133,7 +141,7 @@ def test_mse_sweep_definition():
     assert oracle.num_candidates() == 80
     assert [round(oracle.candidate_ratio(i), 2) for i in (0, 1, 79)] == [1.0, 0.99, 0.21]
     W = synth.gaussian_weights(5, 6, 512)
-    for name, lv in LV.items():
+    for name, lv in list(LV.items()) + [("INT3", oracle.INT3)]:
         table = np.array(oracle.level_table(lv), dtype=np.float64)
         top = np.float32(table.max())
         s, idx, errs = oracle.weight_scale(W, lv, oracle.SCALE_MSE, want_errs=True)
@@ -310,6 +318,67 @@ def test_pack_layout_and_roundtrip(lv, N, words):
         assert tiled_address(8, 0, words) == base + 128          # rows 8..15: the next 512 bytes
 
 
+def int3_addresses(n, j, pitch):
+    """Low-plane and high-plane word of (row n, low word j), written from the layout's description: row blocks of
+    24 * pitch words; slices of 16 low words = 384 words (256 low + 128 high)."""
+    rb, r = divmod(n, 16)
+    half, g = divmod(r, 8)
+    sl, jj = divmod(j, 16)
+    quad, e = divmod(jj, 4)
+    base = rb * 24 * pitch + sl * 384
+    return base + (half * 32 + g * 4 + quad) * 4 + e, base + 256 + (g * 4 + quad) * 4 + 2 * half + e // 2
+
+
+@pytest.mark.parametrize("N,words", [(5, 8), (16, 16), (37, 144), (33, 688)])
+def test_int3_plane_layout_and_roundtrip(N, words):
+    K = words * 16
+    rng = np.random.default_rng(4)
+    n_pad, pitch = -(-N // 16) * 16, -(-words // 16) * 16
+    total = n_pad * pitch * 3 // 2
+    assert oracle.packed_words(N, K, oracle.INT3) == total
+    lo = np.array([[int3_addresses(n, j, pitch)[0] for j in range(words)] for n in range(N)])
+    hi = np.array([[int3_addresses(n, j, pitch)[1] for j in range(0, words, 2)] for n in range(N)])
+    # both maps are injective, disjoint, inside the buffer; a pair of low words shares its high word
+    allw = np.concatenate([lo.ravel(), hi.ravel()])
+    assert len(np.unique(allw)) == allw.size and allw.max() < total
+    assert all(int3_addresses(3, j, pitch)[1] == int3_addresses(3, j + 1, pitch)[1] for j in range(0, words, 2))
+    pats = [rng.integers(0, 8, (N, K)), np.zeros((N, K)), np.full((N, K), 7), np.tile(np.arange(K) % 8, (N, 1)),
+            np.full((N, K), 4), np.full((N, K), 3)]
+    for codes in pats:
+        codes = codes.astype(np.uint8)
+        p = oracle.pack(codes, oracle.INT3)
+        assert p.shape == (total,)
+        assert np.array_equal(oracle.unpack(p, N, K, oracle.INT3), codes)
+        # low plane: exactly the two-bit word of the codes' low bits
+        ref_lo = np.zeros((N, words), dtype=np.uint64)
+        ref_hi = np.zeros((N, words // 2), dtype=np.uint64)
+        for k in range(K):
+            j, r = divmod(k, 16)
+            t, b = divmod(r, 4)
+            ref_lo[:, j] |= (codes[:, k] & 3).astype(np.uint64) << np.uint64(8 * b + 2 * t)
+            ref_hi[:, j // 2] |= (codes[:, k] >> 2).astype(np.uint64) << np.uint64(8 * b + 4 * (j % 2) + (0, 2, 1, 3)[t])
+        assert np.array_equal(p[lo], ref_lo.astype(np.uint32))
+        assert np.array_equal(p[hi], ref_hi.astype(np.uint32))
+        mask = np.ones(p.shape, dtype=bool)
+        mask[allw] = False
+        assert not p[mask].any()
+    # the property the storage is built for: in a high word, the bits of planes t and t + 1 of a low word lie
+    # two positions apart (t even), so that with the even planes' activations scaled by four both halves of a
+    # product step carry the same place value
+    for par in range(2):
+        for t in (0, 2):
+            b0 = 4 * par + (0, 2, 1, 3)[t]
+            b1 = 4 * par + (0, 2, 1, 3)[t + 1]
+            assert b1 == b0 + 2
+    # three bits per weight on the paper's shapes, no padding
+    for _, n, k in synth.LLAMA2_7B + synth.LLAMA31_8B:
+        assert oracle.packed_words(n, k, oracle.INT3) * 32 == 3 * n * k
+    # a slice of a row block is contiguous: 16 rows x 16 low words and their high words in 384 words
+    a = sorted([int3_addresses(n, j, 16)[0] for n in range(16) for j in range(16)] +
+               list({int3_addresses(n, j, 16)[1] for n in range(16) for j in range(16)}))
+    assert a == list(range(384))
+
+
 def test_packed_bytes_of_llama_shapes():
     # no padding on the paper's shapes: exactly 2 (or 4) bits per weight
     for _, N, K in synth.LLAMA2_7B + synth.LLAMA31_8B:
@@ -337,13 +406,22 @@ def test_product_exhaustive_k4(name):
     assert np.array_equal(acc.astype(np.int64), ref)
 
 
+def test_product_exhaustive_int3_k3():
+    # Eq. 1 with b = 3: the decoded level of the two's-complement field c is c - 8 [c >= 4]
+    table = np.array([c - 8 if c >= 4 else c for c in range(8)], dtype=np.int64)
+    codes = np.array(list(itertools.product(range(8), repeat=3)), dtype=np.uint8)           # 512 x 3
+    acts = np.array(list(itertools.product(range(-8, 8), repeat=3)), dtype=np.int8)         # 4096 x 3
+    acc = oracle.int_matmul(codes, oracle.INT3, acts)
+    assert np.array_equal(acc.astype(np.int64), acts.astype(np.int64) @ table[codes].T)
+
+
 def test_product_closed_cases_and_library_crosscheck():
     import torch
     rng = np.random.default_rng(8)
     M, N, K = 3, 7, 160
     q = rng.integers(-8, 8, (M, K)).astype(np.int8)
-    for lv in (oracle.MNZ, oracle.POT, oracle.SYM, oracle.INT4):
-        nc = 16 if lv == oracle.INT4 else 4
+    for lv in (oracle.MNZ, oracle.POT, oracle.SYM, oracle.INT4, oracle.INT3):
+        nc = oracle.num_codes(lv)
         table = np.array(oracle.level_table(lv), dtype=np.int64)
         codes = rng.integers(0, nc, (N, K)).astype(np.uint8)
         acc = oracle.int_matmul(codes, lv, q)
@@ -353,7 +431,10 @@ def test_product_closed_cases_and_library_crosscheck():
         assert not oracle.int_matmul(codes, lv, np.zeros_like(q)).any()
         if lv in (oracle.MNZ, oracle.POT):      # mirrored codes negate the product
             assert np.array_equal(oracle.int_matmul(3 - codes, lv, q), -acc)
-        if lv != oracle.INT4:                   # bit-plane form as a second formula
+        if lv == oracle.INT3:                   # plane form: low two bits minus four times the third
+            q64 = q.astype(np.int64)
+            assert np.array_equal(acc, q64 @ (codes & 3).astype(np.int64).T - 4 * (q64 @ (codes >> 2).astype(np.int64).T))
+        elif lv != oracle.INT4:                 # bit-plane form as a second formula
             a, b, c = {oracle.MNZ: (4, 2, -3), oracle.POT: (5, 3, -4), oracle.SYM: (2, 1, -2)}[lv]
             b1, b0 = (codes >> 1).astype(np.int64), (codes & 1).astype(np.int64)
             q64 = q.astype(np.int64)

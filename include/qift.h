@@ -51,7 +51,9 @@ typedef enum {
     QIFT_LEVELS_MNZ = 0,  /* {-3,-1,+1,+3}: half-scale form of {+-0.5,+-1.5}; s_n is s/2 (Sec. 3.3) */
     QIFT_LEVELS_POT = 1,  /* {-4,-1,+1,+4}: power-of-two mirror no-zero set          (Sec. 3.3)     */
     QIFT_LEVELS_SYM = 2,  /* {-2,-1, 0,+1}: standard symmetric integer W2            (Eq. 1, b = 2) */
-    QIFT_LEVELS_INT4 = 3  /* -8..7 two's-complement nibble, 8 codes per word         (Eq. 1, b = 4) */
+    QIFT_LEVELS_INT4 = 3, /* -8..7 two's-complement nibble, 8 codes per word         (Eq. 1, b = 4) */
+    QIFT_LEVELS_INT3 = 4  /* -4..3 two's-complement three-bit code, stored as a two-bit and a one-bit
+                             plane: the W3A4 configuration of Sec. 4.4       (Eq. 1, b = 3) */
 } qift_levels;
 
 /* How the per-output-channel scale is chosen (Sec. 3.5; the clipping-ratio sweep of Sec. 4.5.1).
@@ -60,7 +62,7 @@ typedef enum {
  * The squared errors are fp64 sums whose order of addition is the kernel's: two candidates whose
  * errors agree to 1e-12 relative count as tied, and either may win (a CPU check must allow that and
  * then compare the codes given the returned scale, which are exact).
- * top_level is 3 (MNZ), 4 (POT), 1 (SYM), 7 (INT4).  An all-zero row gets s_n = 1. */
+ * top_level is 3 (MNZ), 4 (POT), 1 (SYM), 7 (INT4), 3 (INT3).  An all-zero row gets s_n = 1. */
 typedef enum { QIFT_SCALE_GIVEN = 0, QIFT_SCALE_ABSMAX = 1, QIFT_SCALE_MSE = 2 } qift_scale_mode;
 
 typedef enum { QIFT_F32 = 0, QIFT_BF16 = 1 } qift_dtype;
@@ -84,8 +86,8 @@ typedef enum {
 
 const char* qift_status_string(int status);
 
-/* Bytes of the packed weight buffer: N*K/4 for the two-bit sets, N*K/2 for INT4, after padding N and
- * the words per row to multiples of 16.  0 on bad input. */
+/* Bytes of the packed weight buffer: N*K/4 for the two-bit sets, N*K/2 for INT4, 3*N*K/8 for INT3, after
+ * padding N and the (two-bit) words per row to multiples of 16.  0 on bad input. */
 size_t qift_packed_bytes(int N, int K, int levels);
 
 /* Bytes of scratch qift_w2a4_linear / qift_w4a4_linear can use for this problem, rounded up to 1 KiB:
@@ -99,7 +101,9 @@ size_t qift_packed_bytes(int N, int K, int levels);
  * With less than this (or NULL) the call still runs when a route without scratch exists -- M <= 16
  * falls back to the K-split decode kernel, 17..64 rows to the fused prefill route if 4*M bytes were
  * passed -- and returns QIFT_ERR_WORKSPACE otherwise.  qift_workspace_bytes_route gives the figure
- * for an explicit route. */
+ * for an explicit route.
+ * INT3 has two product routes besides the generic one: the row-split decode kernel for 1 <= M <= 16
+ * (M*K + 512 bytes) and the decode-to-int8 GEMM routes above that (N*K bytes). */
 size_t qift_workspace_bytes(int M, int N, int K, int levels);
 size_t qift_workspace_bytes_route(int M, int N, int K, int levels, int route);
 
@@ -119,11 +123,20 @@ size_t qift_workspace_bytes_route(int M, int N, int K, int levels, int route);
  * slice = (j%128)/16, half = (row%16)/8, quad = (j%16)/4.  Rows and words per row are padded to
  * multiples of 16 with zero words (no padding for any LLaMA shape).  A tile is one 8 KB contiguous
  * block, and the 32 groups a warp needs for one mma step are 512 contiguous bytes.
- * Requires K % 16 == 0 (K % 8 == 0 for INT4) and K <= 16384. */
+ * INT3 (q & 7 of Eq. 1 with b = 3, clip to [-4,3]) is stored as two planes, level = (c & 3) - 4 (c >> 2):
+ * the two low bits of the codes in words exactly as above, and the third bit 32 to a word -- high word h of
+ * a row covers low words 2h and 2h+1, and the bit of code k = 16j + 4t + b sits in byte b at position
+ * 4 (j%2) + {0,2,1,3}[t], so that the bits of planes t and t+1 (t even) lie two positions apart: with the
+ * even planes' activations multiplied by four both halves of a product instruction carry one place value.
+ * The planes are interleaved slice by slice: a slice (16 low words of the 16 rows of a row block) is 1536
+ * contiguous bytes, 1024 of low words in the group order above followed by 512 of high words (group
+ * (row%8)*4 + quad: the two high words of rows row%8 and row%8 + 8), slices in ascending k inside a row
+ * block of 24 * pitch words; any run of slices of a row block is therefore one contiguous piece.
+ * Requires K % 16 == 0 (K % 8 == 0 for INT4, K % 32 == 0 for INT3) and K <= 16384. */
 int qift_pack_weights(const float* W, int N, int K, int levels, int scale_mode, float* s_n,
                       uint32_t* packed, void* stream);
 
-/* Inverse of the packed layout, for tests: codes uint8 [N,K] (INT4: the nibble 0..15). */
+/* Inverse of the packed layout, for tests: codes uint8 [N,K] (INT4: the nibble 0..15; INT3: 0..7). */
 int qift_unpack_codes(const uint32_t* packed, int N, int K, int levels, uint8_t* codes, void* stream);
 
 /* S0 (offline rotation, Sec. 3.1 / Sec. 4.1): Y = X Q with Q = blockdiag(H_B) / sqrt(B), H_B the
@@ -165,7 +178,18 @@ int qift_w4a4_linear(const uint32_t* packed, const float* s_n, const int8_t* q_a
                      int M, int N, int K, void* Y, int y_dtype, int32_t* acc_debug, void* workspace,
                      size_t workspace_bytes, void* stream);
 
-/* The two calls above with the kernel route chosen by the caller (tests and benchmarks).
+/* Same for INT3 weights (W3A4, the three-bit point the mixed-precision stacks are compared with at equal
+ * average bits: Sec. 4.4).  1 <= M <= 16 with the scratch of qift_workspace_bytes takes the row-split decode
+ * kernel (two launches: activations re-laid out, then the product), larger M decodes the codes to int8
+ * and runs the tensor-core GEMM (one CTA per tile up to 512 rows, CTA pairs above); without scratch the
+ * generic kernel runs. */
+int qift_w3a4_linear(const uint32_t* packed, const float* s_n, const int8_t* q_a, const float* s_a,
+                     int M, int N, int K, void* Y, int y_dtype, int32_t* acc_debug, void* workspace,
+                     size_t workspace_bytes, void* stream);
+
+/* The calls above with the kernel route chosen by the caller (tests and benchmarks).
+ * INT3 is served by QIFT_ROUTE_GENERIC, QIFT_ROUTE_DECODE_ROWS (here from M = 1, up to 16 rows),
+ * QIFT_ROUTE_PREFILL_SCRATCH and QIFT_ROUTE_PREFILL_PAIR.
  * QIFT_ERR_UNSUPPORTED_SHAPE when the route cannot serve the shape. */
 int qift_linear_route(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a,
                       const float* s_a, int M, int N, int K, void* Y, int y_dtype, int32_t* acc_debug,
@@ -260,8 +284,8 @@ int qift_linear_multi(const int8_t* q_a, const float* s_a, int M, int K, int lev
  *   qift_group_forward      : both.
  * Problems must not alias each other's Y, nor each other's q_a / s_a with one exception: modules that
  * read the SAME activation (q/k/v; gate/up) may name the same X, q_a, s_a (same K and had_block); the
- * plan then quantizes that activation once and every such product reads it.  K % 256 == 0 (two-bit sets) or K % 128 == 0
- * (INT4), K <= 16384. */
+ * plan then quantizes that activation once and every such product reads it.  K % 256 == 0 (two-bit sets, INT3) or
+ * K % 128 == 0 (INT4), K <= 16384.  INT3 plans take up to 16 token rows. */
 typedef struct qift_group_problem {
     const void* X;          /* dev [M,K] fp32 or bf16                         */
     const uint32_t* packed; /* dev, from qift_pack_weights                    */

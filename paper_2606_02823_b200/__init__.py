@@ -6,7 +6,7 @@ and raises if it has not been built.
 """
 from .binding import *  # noqa: F401,F403
 from .binding import (lib, status_string, QiftError, qift_packed_bytes, qift_workspace_bytes, qift_pack_weights,
-                      qift_unpack_codes, qift_rotate, qift_quantize_act, qift_w2a4_linear, qift_w4a4_linear,
+                      qift_unpack_codes, qift_rotate, qift_quantize_act, qift_w2a4_linear, qift_w4a4_linear, qift_w3a4_linear,
                       qift_linear_route, qift_device_status, qift_forward_scratch_bytes, qift_forward,
                       qift_forward_host, qift_group_plan_bytes, qift_group_plan, qift_group_quantize_act,
                       qift_group_linear, qift_group_forward, qift_group_forward_host, GroupPlan, qift_static_scratch_bytes,

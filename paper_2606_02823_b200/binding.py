@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(HERE, "libqift.so")
 
 # enums of qift.h
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = range(8)
-MNZ, POT, SYM, INT4 = 0, 1, 2, 3
+MNZ, POT, SYM, INT4, INT3 = 0, 1, 2, 3, 4
 SCALE_GIVEN, SCALE_ABSMAX, SCALE_MSE = 0, 1, 2
 F32, BF16 = 0, 1
 ROUTE_AUTO, ROUTE_GENERIC, ROUTE_DECODE, ROUTE_PREFILL, ROUTE_PREFILL_SCRATCH, ROUTE_PREFILL_PAIR = 0, 1, 2, 3, 4, 5
@@ -26,7 +26,7 @@ ROUTE_DECODE_ROWS = 7
 EXPORTS = [
     "qift_status_string", "qift_packed_bytes", "qift_workspace_bytes", "qift_workspace_bytes_route", "qift_pack_weights",
     "qift_unpack_codes", "qift_rotate", "qift_quantize_act", "qift_w2a4_linear", "qift_w4a4_linear",
-    "qift_linear_route", "qift_device_status", "qift_forward_scratch_bytes", "qift_forward", "qift_forward_host",
+    "qift_w3a4_linear", "qift_linear_route", "qift_device_status", "qift_forward_scratch_bytes", "qift_forward", "qift_forward_host",
     "qift_group_plan_bytes", "qift_group_plan", "qift_group_quantize_act", "qift_group_linear", "qift_group_forward",
     "qift_group_forward_host", "qift_static_scratch_bytes", "qift_w2a4_linear_static",
     "qift_kv4_quantize", "qift_kv4_attention_workspace_bytes", "qift_kv4_attention_decode",
@@ -69,6 +69,7 @@ def lib() -> ctypes.CDLL:
         L.qift_quantize_act.argtypes = [vp, ci, ci, ci, ci, cf, vp, vp, vp]
         L.qift_w2a4_linear.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, vp, ci, vp, vp, sz, vp]
         L.qift_w4a4_linear.argtypes = [vp, vp, vp, vp, ci, ci, ci, vp, ci, vp, vp, sz, vp]
+        L.qift_w3a4_linear.argtypes = [vp, vp, vp, vp, ci, ci, ci, vp, ci, vp, vp, sz, vp]
         L.qift_linear_route.argtypes = [vp, vp, ci, vp, vp, ci, ci, ci, vp, ci, vp, vp, sz, ci, vp]
         L.qift_device_status.argtypes = [vp, vp]
         L.qift_forward_scratch_bytes.restype = sz
@@ -210,9 +211,9 @@ def _linear(fn_name, packed, s_n, levels, q_a, s_a, N, out_dtype, want_acc, work
     if fn_name == "qift_linear_route":
         rc = L.qift_linear_route(_ptr(packed), _ptr(s_n), levels, _ptr(q_a), _ptr(s_a), M, N, K, _ptr(out), ydt,
                                  _ptr(acc), _ptr(workspace), ws_bytes, route, _stream())
-    elif fn_name == "qift_w4a4_linear":
-        rc = L.qift_w4a4_linear(_ptr(packed), _ptr(s_n), _ptr(q_a), _ptr(s_a), M, N, K, _ptr(out), ydt, _ptr(acc),
-                                _ptr(workspace), ws_bytes, _stream())
+    elif fn_name in ("qift_w4a4_linear", "qift_w3a4_linear"):
+        rc = getattr(L, fn_name)(_ptr(packed), _ptr(s_n), _ptr(q_a), _ptr(s_a), M, N, K, _ptr(out), ydt, _ptr(acc),
+                                 _ptr(workspace), ws_bytes, _stream())
     else:
         rc = L.qift_w2a4_linear(_ptr(packed), _ptr(s_n), levels, _ptr(q_a), _ptr(s_a), M, N, K, _ptr(out), ydt,
                                 _ptr(acc), _ptr(workspace), ws_bytes, _stream())
@@ -228,6 +229,11 @@ def qift_w2a4_linear(packed, s_n, levels, q_a, s_a, out_dtype=torch.float32, wan
 
 def qift_w4a4_linear(packed, s_n, q_a, s_a, out_dtype=torch.float32, want_acc=False, workspace=None, out=None):
     return _linear("qift_w4a4_linear", packed, s_n, INT4, q_a, s_a, s_n.shape[0], out_dtype, want_acc,
+                   workspace, ROUTE_AUTO, out)
+
+
+def qift_w3a4_linear(packed, s_n, q_a, s_a, out_dtype=torch.float32, want_acc=False, workspace=None, out=None):
+    return _linear("qift_w3a4_linear", packed, s_n, INT3, q_a, s_a, s_n.shape[0], out_dtype, want_acc,
                    workspace, ROUTE_AUTO, out)
 
 

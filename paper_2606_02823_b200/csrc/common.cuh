@@ -24,7 +24,7 @@ __device__ __forceinline__ void report_timeout(unsigned int site) {
 // ------------------------------------------------------------------------------------------------
 __host__ __device__ constexpr int codes_per_word(int lv) { return lv == QIFT_LEVELS_INT4 ? 8 : 16; }
 __host__ __device__ constexpr float top_level(int lv) {
-    return lv == QIFT_LEVELS_MNZ ? 3.0f : lv == QIFT_LEVELS_POT ? 4.0f : lv == QIFT_LEVELS_SYM ? 1.0f : 7.0f;
+    return lv == QIFT_LEVELS_MNZ ? 3.0f : lv == QIFT_LEVELS_POT ? 4.0f : lv == QIFT_LEVELS_SYM ? 1.0f : lv == QIFT_LEVELS_INT3 ? 3.0f : 7.0f;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -49,8 +49,33 @@ __host__ __device__ inline size_t packed_word_address(int n, int j, int pitch) {
            static_cast<size_t>((((slice * 2 + half) * 32 + g * 4 + quad) << 2) + e);
 }
 
+// Three-bit codes (INT3): a two-bit plane in words as above and a one-bit plane, 32 codes to a word, interleaved
+// slice by slice.  A slice -- 16 low words of the 16 rows of a row block -- is 1536 contiguous bytes: 1024 of low
+// words in the group order above (rows 0..7, then rows 8..15), then 512 of high words, group (row%8)*4 + quad holding
+// {high words 0, 1 of row row%8, high words 0, 1 of row row%8 + 8} of that quad: the 16 bytes a lane of the product
+// kernel needs next to its two groups of low words.  High word h of a row covers low words 2h, 2h+1; the bit of
+// code k = 16j + 4t + b is bit 8b + 4(j%2) + {0,2,1,3}[t].  Row blocks are 24 * pitch words (pitch = low words per
+// row, padded to 16).
+__host__ __device__ constexpr int tile_word_bytes(int lv) { return lv == QIFT_LEVELS_INT3 ? 96 : 64; }   // 16 rows x one low word
+__host__ __device__ inline size_t int3_low_address(int n, int j, int pitch) {
+    const int rb = n >> 4, half = (n >> 3) & 1, g = n & 7;
+    const int slice = j >> 4, quad = (j >> 2) & 3, e = j & 3;
+    return static_cast<size_t>(rb) * 24 * pitch + static_cast<size_t>(slice) * 384 + static_cast<size_t>(((half * 32 + g * 4 + quad) << 2) + e);
+}
+__host__ __device__ inline size_t int3_high_address(int n, int j, int pitch) {   // j: low word index
+    const int rb = n >> 4, half = (n >> 3) & 1, g = n & 7;
+    const int slice = j >> 4, quad = (j >> 2) & 3, pair = (j >> 1) & 1;
+    return static_cast<size_t>(rb) * 24 * pitch + static_cast<size_t>(slice) * 384 + 256 + static_cast<size_t>(((g * 4 + quad) << 2) + 2 * half + pair);
+}
+__host__ __device__ constexpr int int3_high_shift(int j, int t) { return 4 * (j & 1) + ((t & 1) << 1) + (t >> 1); }   // inside a byte
+// Four level bytes of plane t of low word `lo` (index j) and its high word `hi`: (c & 3) - 4 (c >> 2) = (c & 3) | 0xfc [c >> 2].
+__device__ __forceinline__ uint32_t int3_level_bytes(uint32_t lo, uint32_t hi, int j, int t) {
+    return ((lo >> (2 * t)) & 0x03030303u) | (((hi >> int3_high_shift(j, t)) & 0x01010101u) * 0xfcu);
+}
+
 template <int LV>
 __device__ __forceinline__ int level_from_code(int c) {
+    if constexpr (LV == QIFT_LEVELS_INT3) return ((c & 7) ^ 4) - 4;
     if constexpr (LV == QIFT_LEVELS_MNZ) return 2 * c - 3;
     if constexpr (LV == QIFT_LEVELS_POT) return 3 * c - (c >> 1) - 4;  // 0,3,5,8 minus 4
     if constexpr (LV == QIFT_LEVELS_SYM) return c - 2;

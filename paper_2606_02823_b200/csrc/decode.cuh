@@ -28,6 +28,7 @@ __device__ __forceinline__ int combine_generic(int S, int Sb1, int Sq) {
     if constexpr (LV == QIFT_LEVELS_MNZ) return 2 * S - 3 * Sq;
     if constexpr (LV == QIFT_LEVELS_SYM) return S - 2 * Sq;
     if constexpr (LV == QIFT_LEVELS_POT) return 3 * S - Sb1 - 4 * Sq;  // value+4 = 3c - b1
+    if constexpr (LV == QIFT_LEVELS_INT3) return S - 4 * Sb1;          // S over the two low bits, Sb1 over the third
     return S - 8 * Sq;
 }
 
@@ -54,12 +55,21 @@ linear_generic_kernel(const uint32_t* __restrict__ packed, const float* __restri
     for (int m0 = 0; m0 < M; m0 += kGenericTokens) {
         int S[kGenericTokens] = {}, Sb[kGenericTokens] = {}, Sq[kGenericTokens] = {};
         for (int j = lane; j < words; j += 32) {
-            const uint32_t w = packed[packed_word_address(n, j, pitch)];
+            uint32_t w, wh = 0;
+            if constexpr (LV == QIFT_LEVELS_INT3) {
+                w = packed[int3_low_address(n, j, pitch)];
+                wh = packed[int3_high_address(n, j, pitch)];
+            } else {
+                w = packed[packed_word_address(n, j, pitch)];
+            }
 #pragma unroll
             for (int t = 0; t < NPL; ++t) {
                 uint32_t a, hb = 0;
                 if constexpr (LV == QIFT_LEVELS_INT4) {
                     a = ((w >> (BITS * t)) & 0x0f0f0f0fu) ^ 0x08080808u;
+                } else if constexpr (LV == QIFT_LEVELS_INT3) {
+                    a = (w >> (BITS * t)) & 0x03030303u;
+                    hb = (wh >> int3_high_shift(j, t)) & 0x01010101u;
                 } else {
                     a = (w >> (BITS * t)) & 0x03030303u;
                     hb = (a >> 1) & 0x01010101u;
@@ -69,7 +79,7 @@ linear_generic_kernel(const uint32_t* __restrict__ packed, const float* __restri
                     if (m0 + mm < M) {
                         const uint32_t qv = q32[(m0 + mm) * qpitch + static_cast<size_t>(j) * NPL + t];
                         S[mm] = dp4a_us(a, qv, S[mm]);
-                        if constexpr (LV == QIFT_LEVELS_POT) Sb[mm] = dp4a_us(hb, qv, Sb[mm]);
+                        if constexpr (LV == QIFT_LEVELS_POT || LV == QIFT_LEVELS_INT3) Sb[mm] = dp4a_us(hb, qv, Sb[mm]);
                         Sq[mm] = dp4a_us(0x01010101u, qv, Sq[mm]);
                     }
                 }
@@ -119,7 +129,7 @@ struct DecodeTraits {
     static constexpr int QBYTES = kChunkWords * PER;        // q_a bytes per token per stage
     static constexpr int QSTRIDE = QBYTES + kQPad;
     static constexpr int BPT = QBYTES / kDecConsumers;      // q bytes per consumer thread per token
-    static constexpr int NACC = (LV == QIFT_LEVELS_INT4) ? 1 : (LV == QIFT_LEVELS_POT) ? 4 : 2;
+    static constexpr int NACC = (LV == QIFT_LEVELS_INT4) ? 1 : (LV == QIFT_LEVELS_POT) ? 4 : (LV == QIFT_LEVELS_INT3) ? 6 : 2;
 };
 
 // Place value of accumulator set `a` (a power of two; the set holds scale * sum code*q exactly).
@@ -130,6 +140,9 @@ __host__ __device__ constexpr int acc_shift(int a) {
         const int bit1 = (a < 2) ? 1 : 0;
         return bit1 + 4 * (a & 1) + (PRESCALED ? 2 : 0);
     }
+    if (LV == QIFT_LEVELS_INT3 && a >= 2) {  // sets 2..5: the high plane (prescaled activations only), bit pairs (0,2) (1,3) (4,6) (5,7)
+        return 2 + (a - 2) + ((a >= 4) ? 2 : 0);
+    }
     return 4 * a + (PRESCALED ? 2 : 0);
 }
 
@@ -138,6 +151,11 @@ template <int LV, bool PRESCALED, int NACC>
 __device__ __forceinline__ int level_sum(const int (&v)[NACC], int Sq) {
     if constexpr (LV == QIFT_LEVELS_INT4) {
         return (v[0] >> acc_shift<LV, PRESCALED>(0)) - 8 * Sq;  // code' = nibble ^ 8 = level + 8
+    } else if constexpr (LV == QIFT_LEVELS_INT3) {               // level = (c & 3) - 4 (c >> 2)
+        const int lo = (v[0] >> acc_shift<LV, PRESCALED>(0)) + (v[1] >> acc_shift<LV, PRESCALED>(1));
+        const int hi = (v[2] >> acc_shift<LV, PRESCALED>(2)) + (v[3] >> acc_shift<LV, PRESCALED>(3)) +
+                       (v[4] >> acc_shift<LV, PRESCALED>(4)) + (v[5] >> acc_shift<LV, PRESCALED>(5));
+        return lo - 4 * hi;
     } else if constexpr (LV == QIFT_LEVELS_POT) {                // level = 5*b1 + 3*b0 - 4
         const int b1 = (v[0] >> acc_shift<LV, PRESCALED>(0)) + (v[1] >> acc_shift<LV, PRESCALED>(1));
         const int b0 = (v[2] >> acc_shift<LV, PRESCALED>(2)) + (v[3] >> acc_shift<LV, PRESCALED>(3));
@@ -189,6 +207,33 @@ __device__ __forceinline__ void mma_tile_step(int (&acc)[NT][DecodeTraits<LV>::N
                         mma_u8s8(acc[nt][tt / 2], lo[i] & m0, hi[i] & m0, l1 & m1, h1 & m1, qb[nt][NPL * i + tt],
                                  qb[nt][NPL * i + tt + 1]);
                 }
+            }
+        }
+    }
+}
+
+// Three-bit codes: the low plane is a two-bit word like any other (sets 0, 1); the high plane adds, per low word, two
+// products whose operands are single bits of the high word.  Its bit order puts planes t and t+1 (t even) of a low
+// word two positions apart, so with the even planes' activations prescaled by four both halves of an instruction
+// carry the place value 4 * 2^u: u = 0, 1 for the even low word of a pair (sets 2, 3), 4, 5 for the odd one (sets 4, 5).
+// wh = {high words 0, 1 of row g, high words 0, 1 of row g+8} of the lane's four low words.
+template <int NT>
+__device__ __forceinline__ void mma_tile_step_int3(int (&acc)[NT][6][4], const uint4 wa, const uint4 wb, const uint4 wh,
+                                                   const uint32_t (&qb)[NT][16]) {
+    const uint32_t lo[4] = {wa.x, wa.y, wa.z, wa.w};
+    const uint32_t hi[4] = {wb.x, wb.y, wb.z, wb.w};
+    const uint32_t hl[2] = {wh.x, wh.y}, hh[2] = {wh.z, wh.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+#pragma unroll
+        for (int tt = 0; tt < 4; tt += 2) {
+            const uint32_t m0 = 0x03030303u << (2 * tt), m1 = m0 << 2;
+            const uint32_t b0 = 0x01010101u << (4 * (i & 1) + tt / 2), b1 = b0 << 2;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                mma_u8s8(acc[nt][tt / 2], lo[i] & m0, hi[i] & m0, lo[i] & m1, hi[i] & m1, qb[nt][4 * i + tt], qb[nt][4 * i + tt + 1]);
+                mma_u8s8(acc[nt][2 + 2 * (i & 1) + tt / 2], hl[i >> 1] & b0, hh[i >> 1] & b0, hl[i >> 1] & b1, hh[i >> 1] & b1,
+                         qb[nt][4 * i + tt], qb[nt][4 * i + tt + 1]);
             }
         }
     }
@@ -281,7 +326,7 @@ __host__ __device__ inline size_t decode_stage_bytes(int lv, int rt, int M) {
     return static_cast<size_t>(rt) * kTileBytes + static_cast<size_t>(M) * (kChunkWords * codes_per_word(lv) + kQPad);
 }
 __host__ __device__ inline size_t decode_smem_bytes(int lv, int rt, int nt, int M, int stages) {
-    const int nacc = (lv == QIFT_LEVELS_INT4) ? 1 : (lv == QIFT_LEVELS_POT) ? 4 : 2;
+    const int nacc = (lv == QIFT_LEVELS_INT4) ? 1 : (lv == QIFT_LEVELS_POT) ? 4 : (lv == QIFT_LEVELS_INT3) ? 6 : 2;
     return stages * decode_stage_bytes(lv, rt, M) + static_cast<size_t>(kDecWarps) * rt * nt * nacc * 128 * 4  // reduce
            + 2 * stages * 8 + 16 * 4 + 16;  // barriers, sum-q, flag
 }

@@ -167,7 +167,8 @@ constexpr int kGroupSlice = 256;  // problems per launch (their table lives in s
 
 // Walks this CTA's share of the work list chunk by chunk; the producer and the consumers each run
 // one and see the same sequence.  PER = codes per packed word.
-template <int PER, int CW = kChunkWords>
+// WB = bytes of one packed word column of a 16-row tile (64; 96 with the one-bit plane of the three-bit codes).
+template <int PER, int CW = kChunkWords, int WB = 64>
 struct GroupCursor {
     const SmemProblem* table;
     int count, item_end, rows_per_item;
@@ -194,8 +195,8 @@ struct GroupCursor {
         n0 = (item - P.item_begin) * rows_per_item;
         tiles_valid = (min(rows_per_item, N - n0) + 15) >> 4;
         const int pitch = round_up16(words_per_row);
-        rb_bytes = static_cast<size_t>(16) * pitch * 4;
-        wbase = P.packed + static_cast<size_t>(n0) * pitch * 4;
+        rb_bytes = static_cast<size_t>(pitch) * WB;
+        wbase = P.packed + static_cast<size_t>(n0 >> 4) * pitch * WB;
         q_a = P.q_a;
     }
     __device__ __forceinline__ int chunk_words() const { return min(CW, words_per_row - chunk * CW); }
@@ -211,7 +212,7 @@ struct GroupCursor {
 
 // Cross-warp reduction buffer: [warp][row tile][accumulator set][token][row], only the M live columns.
 __host__ __device__ inline int grouped_red_ints(int lv, int rt, int M) {
-    const int nacc = (lv == QIFT_LEVELS_INT4) ? 1 : (lv == QIFT_LEVELS_POT) ? 4 : 2;
+    const int nacc = (lv == QIFT_LEVELS_INT4) ? 1 : (lv == QIFT_LEVELS_POT) ? 4 : (lv == QIFT_LEVELS_INT3) ? 6 : 2;
     return kDecWarps * rt * nacc * 16 * M;
 }
 __host__ __device__ inline size_t grouped_fixed_smem(int lv, int rt, int M, int count) {
@@ -458,12 +459,14 @@ constexpr int kWideRows = 16 * kDecWarps;        // 128 rows per item with one t
 // sixteen warps (twice the warps to hide the latencies of the load -> logic -> product chains) or as two tiles per
 // warp (the activation registers of a slice feed both tiles); their stages are a quarter tile of K (32 words) so
 // that as many stages fit as with 128 rows.
-__host__ __device__ constexpr int wide_chunk_words(int tiles, int nt) { return (tiles > 8 || nt > 2) ? 64 : 128; }
+__host__ __device__ constexpr int wide_chunk_words(int tiles, int nt, int lv = QIFT_LEVELS_MNZ) {
+    return (tiles > 8 || nt > 2 || lv == QIFT_LEVELS_INT3) ? 64 : 128;   // three-bit codes: a tile column is 96 bytes, not 64
+}
 __host__ __device__ constexpr int wide_token_tiles(int M) { return M > 32 ? 8 : M > 16 ? 4 : M > 8 ? 2 : 1; }
 
 __host__ __device__ inline size_t wide_stage_bytes(int lv, int M, int tiles) {
-    const int cw = wide_chunk_words(tiles, wide_token_tiles(M));
-    return static_cast<size_t>(tiles) * (cw * 64) + static_cast<size_t>(M) * (cw * codes_per_word(lv));
+    const int cw = wide_chunk_words(tiles, wide_token_tiles(M), lv);
+    return static_cast<size_t>(tiles) * (cw * tile_word_bytes(lv)) + static_cast<size_t>(M) * (cw * codes_per_word(lv));
 }
 __host__ __device__ inline size_t wide_smem_bytes(int lv, int M, int tiles, int stages, int count) {
     return static_cast<size_t>(count) * sizeof(SmemProblem) + stages * (wide_stage_bytes(lv, M, tiles) + 16) + 16;
@@ -474,16 +477,19 @@ __global__ void __launch_bounds__((CWARPS + 1) * 32, 1)
 linear_grouped_wide_kernel(const GroupParams gp) {
     using T = DecodeTraits<LV>;
     constexpr int TILES = CWARPS * RT;           // row tiles per item
-    constexpr int CW = wide_chunk_words(TILES, NT);
+    constexpr int CW = wide_chunk_words(TILES, NT, LV);
     constexpr int THREADS = (CWARPS + 1) * 32;
+    constexpr bool INT3 = (LV == QIFT_LEVELS_INT3);
+    static_assert(!INT3 || NT <= 2, "three-bit codes: six accumulator sets per token tile, at most two token tiles");
+    constexpr int WB = tile_word_bytes(LV);
     // PoT with two token tiles: levels by table lookup (pot_lut_operands) instead of code bit planes -- half the
     // product instructions for more logic per word, which pays once the products are the bottleneck (measured on 16
     // LLaMA-2-7B layers: 261 against 295 us at 16 rows, but 197 against 189 us at 8).
     constexpr bool POT_LUT = (LV == QIFT_LEVELS_POT) && NT >= 2;
     constexpr int NACC = POT_LUT ? 1 : T::NACC;
-    constexpr int TILE_STAGE = CW * 64;          // bytes of one tile in a stage: CW words x 16 rows, contiguous in the packed order
+    constexpr int TILE_STAGE = CW * WB;          // bytes of one tile in a stage: CW words x 16 rows, contiguous in the packed order
     constexpr int CB = CW * T::PER;              // bytes of one token's activations in a full chunk
-    using Cursor = GroupCursor<T::PER, CW>;
+    using Cursor = GroupCursor<T::PER, CW, WB>;
     extern __shared__ __align__(128) unsigned char smem[];
     const int M = gp.M;
     const uint32_t stage_bytes = static_cast<uint32_t>(wide_stage_bytes(LV, M, TILES));
@@ -518,11 +524,11 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     if (warp == CWARPS) {
         // ---------------------------------------------------------------- producer warp
         auto expect = [&](const Cursor& c, int s) {
-            if (lane == 0) mbar_expect_tx(&full[s], c.chunk_words() * (64 * c.tiles_valid + T::PER * M));
+            if (lane == 0) mbar_expect_tx(&full[s], c.chunk_words() * (WB * c.tiles_valid + T::PER * M));
             __syncwarp();
         };
         auto issue_w = [&](const Cursor& c, int s) {  // one bulk copy per 16-row tile: the chunk's slices are contiguous in it
-            const uint32_t bytes = c.chunk_words() * 16 * 4;
+            const uint32_t bytes = c.chunk_words() * WB;
             unsigned char* dst = ring + s * stage_bytes;
             if (lane < c.tiles_valid)
                 bulk_g2s(dst + lane * TILE_STAGE, c.wbase + lane * c.rb_bytes + static_cast<size_t>(c.chunk) * TILE_STAGE, bytes, &full[s]);
@@ -583,7 +589,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
     while (cur.valid() && ok) {
         // With one token tile a warp would have only NACC dependent chains of product instructions; alternate
         // slices then go to a second set of accumulators (added up before the epilogue).
-        constexpr int KS = (NT * RT == 1) ? 2 : 1;
+        constexpr int KS = (NT * RT == 1 && !INT3) ? 2 : 1;
         int acc[KS][RT][NT][NACC][4];
 #pragma unroll
         for (int k = 0; k < KS; ++k)
@@ -638,7 +644,7 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                 const uint32_t wa_base = ws + lane * 16;
                 // the lane's four words of rows g and g+8 of row tile r
                 auto load_words = [&](int r, int sl, uint4& wa, uint4& wb) {
-                    const uint32_t o = r * TILE_STAGE + sl * 1024;
+                    const uint32_t o = r * TILE_STAGE + sl * (16 * WB);
                     wa = lds128(wa_base + o), wb = lds128(wa_base + o + 512);
                 };
                 auto slice = [&](int sl, auto ks) {
@@ -656,7 +662,10 @@ linear_grouped_wide_kernel(const GroupParams gp) {
                         for (int r = 0; r < RT; ++r) {
                             uint4 wa, wb;
                             load_words(r, sl, wa, wb);
-                            if constexpr (POT_LUT) mma_tile_step_pot_lut<NT>(acc[decltype(ks)::value][r], wa, wb, qb);
+                            if constexpr (INT3) {   // the lane's high words follow the slice's two groups of low words
+                                const uint4 wh = lds128(wa_base + r * TILE_STAGE + sl * (16 * WB) + 1024);
+                                mma_tile_step_int3<NT>(acc[decltype(ks)::value][r], wa, wb, wh, qb);
+                            } else if constexpr (POT_LUT) mma_tile_step_pot_lut<NT>(acc[decltype(ks)::value][r], wa, wb, qb);
                             else mma_tile_step<LV, NT, true>(acc[decltype(ks)::value][r], wa, wb, qb);
                         }
                     } else {

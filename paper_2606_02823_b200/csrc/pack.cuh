@@ -14,6 +14,7 @@ __device__ __forceinline__ int nearest_code(float w, float s) {
     if constexpr (LV == QIFT_LEVELS_MNZ) return (t > -2.0f) + (t > 0.0f) + (t > 2.0f);
     if constexpr (LV == QIFT_LEVELS_POT) return (t > -2.5f) + (t > 0.0f) + (t > 2.5f);
     if constexpr (LV == QIFT_LEVELS_SYM) return max(-2, min(1, __float2int_rn(t))) + 2;
+    if constexpr (LV == QIFT_LEVELS_INT3) return max(-4, min(3, __float2int_rn(t))) & 7;
     return max(-8, min(7, __float2int_rn(t))) & 15;
 }
 
@@ -45,13 +46,14 @@ struct LevelCoder {
             mag = outer ? top_level(LV) : 1.0f;
             return (w > 0.0f) ? 2 + static_cast<int>(outer) : 1 - static_cast<int>(outer);
         } else {
-            constexpr float lo = (LV == QIFT_LEVELS_SYM) ? -2.0f : -8.0f, hi = (LV == QIFT_LEVELS_SYM) ? 1.0f : 7.0f;
+            constexpr float lo = (LV == QIFT_LEVELS_SYM) ? -2.0f : (LV == QIFT_LEVELS_INT3) ? -4.0f : -8.0f;
+            constexpr float hi = (LV == QIFT_LEVELS_SYM) ? 1.0f : (LV == QIFT_LEVELS_INT3) ? 3.0f : 7.0f;
             const float t = fminf(fmaxf(__fmul_rn(w, inv), lo), hi);
             const float r = __fsub_rn(__fadd_rn(t, 12582912.0f), 12582912.0f);
             unsure = unsure || inv == 0.0f || fabsf(__fsub_rn(t, r)) > 0.49999237f;
             mag = r;
             const int q = static_cast<int>(r);
-            return (LV == QIFT_LEVELS_SYM) ? q + 2 : (q & 15);
+            return (LV == QIFT_LEVELS_SYM) ? q + 2 : (LV == QIFT_LEVELS_INT3) ? (q & 7) : (q & 15);
         }
     }
     __device__ __forceinline__ int exact(float w, float& mag) const {
@@ -81,8 +83,14 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int pitch = packed_pitch(K, LV);
     if (n >= static_cast<size_t>(N)) {  // padding row of the last row block: zero words
-        for (int u = tid; u < pitch / 4; u += blockDim.x)
-            *reinterpret_cast<uint4*>(packed + packed_word_address(static_cast<int>(n), 4 * u, pitch)) = make_uint4(0, 0, 0, 0);
+        for (int u = tid; u < pitch / 4; u += blockDim.x) {
+            if constexpr (LV == QIFT_LEVELS_INT3) {
+                *reinterpret_cast<uint4*>(packed + int3_low_address(static_cast<int>(n), 4 * u, pitch)) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint2*>(packed + int3_high_address(static_cast<int>(n), 4 * u, pitch)) = make_uint2(0, 0);
+            } else {
+                *reinterpret_cast<uint4*>(packed + packed_word_address(static_cast<int>(n), 4 * u, pitch)) = make_uint4(0, 0, 0, 0);
+            }
+        }
         return;
     }
 
@@ -208,7 +216,8 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
                 // the division.  |w| enters as an exact 64-bit fixed-point integer (crossing weights are
                 // >= 0.015 max); pairs that have switched at the first candidate already -- the majority --
                 // are summed per thread first.
-                constexpr int kLimPos = (LV == QIFT_LEVELS_SYM) ? 1 : 7, kLimNeg = (LV == QIFT_LEVELS_SYM) ? 2 : 8;
+                constexpr int kLimPos = (LV == QIFT_LEVELS_SYM) ? 1 : (LV == QIFT_LEVELS_INT3) ? 3 : 7;
+                constexpr int kLimNeg = (LV == QIFT_LEVELS_SYM) ? 2 : (LV == QIFT_LEVELS_INT3) ? 4 : 8;
                 float* sj = cand;  // [kNumCandidates] candidate scales, decreasing in j
                 for (int j = tid; j < kNumCandidates; j += blockDim.x) {
                     sj[j] = __fdiv_rn(__fmul_rn(__fdiv_rn(static_cast<float>(100 - j), 100.0f), amax), g);
@@ -322,9 +331,16 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
     __syncthreads();
     for (int j0 = 0; j0 < pitch; j0 += blockDim.x) {  // pitch is a multiple of 16, blockDim of 32: whole groups per warp
         const int j = j0 + tid;
-        uint32_t w = 0;
+        uint32_t w = 0, h = 0;
         if (j < words) {
-            if constexpr (PER == 16) {
+            if constexpr (LV == QIFT_LEVELS_INT3) {
+                // low plane: the two low bits as a two-bit word; high plane: this word's half of the shared high word
+                const uint4 c = *reinterpret_cast<const uint4*>(code_bytes + 16 * j);
+                constexpr uint32_t m2 = 0x03030303u, m1 = 0x01010101u;
+                w = (c.x & m2) | ((c.y & m2) << 2) | ((c.z & m2) << 4) | ((c.w & m2) << 6);
+                h = (((c.x >> 2) & m1) << int3_high_shift(j, 0)) | (((c.y >> 2) & m1) << int3_high_shift(j, 1)) |
+                    (((c.z >> 2) & m1) << int3_high_shift(j, 2)) | (((c.w >> 2) & m1) << int3_high_shift(j, 3));
+            } else if constexpr (PER == 16) {
                 const uint4 c = *reinterpret_cast<const uint4*>(code_bytes + 16 * j);
                 w = c.x | (c.y << 2) | (c.z << 4) | (c.w << 6);
             } else {
@@ -334,12 +350,21 @@ pack_weights_kernel(const float* __restrict__ W, int N, int K, int mode, float* 
         }
         const uint32_t w1 = __shfl_down_sync(0xffffffffu, w, 1), w2 = __shfl_down_sync(0xffffffffu, w, 2),
                        w3 = __shfl_down_sync(0xffffffffu, w, 3);
-        if ((tid & 3) == 0 && j < pitch)
-            *reinterpret_cast<uint4*>(packed + packed_word_address(static_cast<int>(n), j, pitch)) = make_uint4(w, w1, w2, w3);
+        if constexpr (LV == QIFT_LEVELS_INT3) {
+            const uint32_t h1 = __shfl_down_sync(0xffffffffu, h, 1), h2 = __shfl_down_sync(0xffffffffu, h, 2),
+                           h3 = __shfl_down_sync(0xffffffffu, h, 3);
+            if ((tid & 3) == 0 && j < pitch) {
+                *reinterpret_cast<uint4*>(packed + int3_low_address(static_cast<int>(n), j, pitch)) = make_uint4(w, w1, w2, w3);
+                *reinterpret_cast<uint2*>(packed + int3_high_address(static_cast<int>(n), j, pitch)) = make_uint2(h | h1, h2 | h3);
+            }
+        } else {
+            if ((tid & 3) == 0 && j < pitch)
+                *reinterpret_cast<uint4*>(packed + packed_word_address(static_cast<int>(n), j, pitch)) = make_uint4(w, w1, w2, w3);
+        }
     }
 }
 
-__global__ void unpack_codes_kernel(const uint32_t* __restrict__ packed, long long total, int K, int per,
+__global__ void unpack_codes_kernel(const uint32_t* __restrict__ packed, long long total, int K, int per, int three_bit,
                                     uint8_t* __restrict__ codes) {
     pdl_launch_dependents();
     pdl_wait();
@@ -349,6 +374,13 @@ __global__ void unpack_codes_kernel(const uint32_t* __restrict__ packed, long lo
         const long long n = i / K;
         const int k = static_cast<int>(i % K);
         const int j = k / per, r = k % per, t = r / 4, b = r % 4;
+        if (three_bit) {
+            const int pitch = round_up16(K / 16);
+            const uint32_t lo = packed[int3_low_address(static_cast<int>(n), j, pitch)];
+            const uint32_t hi = packed[int3_high_address(static_cast<int>(n), j, pitch)];
+            codes[i] = static_cast<uint8_t>(((lo >> (8 * b + 2 * t)) & 3u) | (((hi >> (8 * b + int3_high_shift(j, t))) & 1u) << 2));
+            continue;
+        }
         const uint32_t w = packed[packed_word_address(static_cast<int>(n), j, round_up16(K / per))];
         codes[i] = static_cast<uint8_t>((w >> (8 * b + bits * t)) & ((1u << bits) - 1u));
     }

@@ -71,15 +71,28 @@ expand_levels_kernel(const uint32_t* __restrict__ packed, int N, int words_per_r
     const int pitch = round_up16(words_per_row);
     for (int n0 = blockIdx.x * kExpandRows; n0 < N; n0 += gridDim.x * kExpandRows)
         for (int jw = threadIdx.x; jw < words_per_row; jw += blockDim.x) {
-            uint32_t w[kExpandRows];
+            uint32_t w[kExpandRows], wh[kExpandRows];
 #pragma unroll
-            for (int r = 0; r < kExpandRows; ++r) w[r] = (n0 + r < N) ? packed[packed_word_address(n0 + r, jw, pitch)] : 0u;
+            for (int r = 0; r < kExpandRows; ++r) {
+                if constexpr (LV == QIFT_LEVELS_INT3) {   // the low word and the high word it shares with its neighbour
+                    w[r] = (n0 + r < N) ? packed[int3_low_address(n0 + r, jw, pitch)] : 0u;
+                    wh[r] = (n0 + r < N) ? packed[int3_high_address(n0 + r, jw, pitch)] : 0u;
+                } else {
+                    w[r] = (n0 + r < N) ? packed[packed_word_address(n0 + r, jw, pitch)] : 0u;
+                    wh[r] = 0u;
+                }
+            }
 #pragma unroll
             for (int r = 0; r < kExpandRows; ++r) {
                 if (n0 + r >= N) break;
                 const size_t j = static_cast<size_t>(n0 + r) * words_per_row + jw;
                 uint32_t o[PER / 4];
-                expand_word<LV>(w[r], o);
+                if constexpr (LV == QIFT_LEVELS_INT3) {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) o[t] = int3_level_bytes(w[r], wh[r], jw, t);
+                } else {
+                    expand_word<LV>(w[r], o);
+                }
                 if constexpr (PER == 16) reinterpret_cast<uint4*>(out)[j] = make_uint4(o[0], o[1], o[2], o[3]);
                 else reinterpret_cast<uint2*>(out)[j] = make_uint2(o[0], o[1]);
             }

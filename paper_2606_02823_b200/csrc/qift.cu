@@ -30,7 +30,7 @@ namespace {
 // Grouped decode: from this many token rows on the row-split kernel (128-row items) is the faster one.  Measured
 // on 16 LLaMA-2-7B layers, row-split flat in M against K-split at 1 / 2 / 4 rows: MNZ 140 us against 125 / 152 /
 // 168 us; INT4 232 against 236 / 239 / 258; PoT 191 against 218 / 215 / 217.
-inline int wide_min_m(int lv) { return lv == QIFT_LEVELS_POT ? 1 : 2; }
+inline int wide_min_m(int lv) { return (lv == QIFT_LEVELS_POT || lv == QIFT_LEVELS_INT3) ? 1 : 2; }
 constexpr int kFusedMaxM = 128;
 constexpr int kFusedPairMaxM = 512;
 inline int auto_prefill_route(int M) {
@@ -39,7 +39,9 @@ inline int auto_prefill_route(int M) {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
-inline bool valid_levels(int lv) { return lv >= QIFT_LEVELS_MNZ && lv <= QIFT_LEVELS_INT4; }
+inline bool valid_levels(int lv) { return lv >= QIFT_LEVELS_MNZ && lv <= QIFT_LEVELS_INT3; }
+// K a whole number of packed words (three-bit codes: of high words, 32 codes each)
+inline bool whole_words(int K, int lv) { return K % (lv == QIFT_LEVELS_INT3 ? 32 : codes_per_word(lv)) == 0; }
 
 // Launch with programmatic stream serialization: the kernel may start while its predecessor in the
 // stream drains; every kernel here executes griddepcontrol.wait before touching caller memory.
@@ -220,7 +222,7 @@ int dispatch_decode(const DecodeParams& p, cudaStream_t st) {
 
 bool decode_supports(int lv, int M, int N, int K) {
     const int per = codes_per_word(lv);
-    return M >= 1 && M <= 16 && K % (16 * per) == 0;  // whole 16-word warp slices
+    return lv != QIFT_LEVELS_INT3 && M >= 1 && M <= 16 && K % (16 * per) == 0;  // whole 16-word warp slices
 }
 
 template <int LV>
@@ -385,6 +387,7 @@ int run_expand(const uint32_t* packed, int lv, int N, int K, int8_t* wexp, cudaS
         case QIFT_LEVELS_MNZ: return launch_expand<QIFT_LEVELS_MNZ>(packed, N, K, wexp, st);
         case QIFT_LEVELS_POT: return launch_expand<QIFT_LEVELS_POT>(packed, N, K, wexp, st);
         case QIFT_LEVELS_SYM: return launch_expand<QIFT_LEVELS_SYM>(packed, N, K, wexp, st);
+        case QIFT_LEVELS_INT3: return launch_expand<QIFT_LEVELS_INT3>(packed, N, K, wexp, st);
         default: return launch_expand<QIFT_LEVELS_INT4>(packed, N, K, wexp, st);
     }
 }
@@ -495,10 +498,14 @@ inline size_t decode_rows_scratch(int M, int K) { return ((static_cast<size_t>(M
 // Grouped plans: the row-split mma.sync kernel up to 32 token rows (PoT: up to 64), the tcgen05 weight-streaming kernel
 // from 33 to 64, where it is the faster one (16 LLaMA-2-7B layers, product kernel, MNZ / INT4: 32 rows 1.9 / 2.8 TB/s
 // against 2.8 / 4.5 on mma.sync; 64 rows 1.8 / 3.2 against 1.3 / 2.5).
-inline bool tc_rows_applies(int lv, int M) { return lv != QIFT_LEVELS_POT && M > 32 && M <= kGroupMaxM; }
+inline bool tc_rows_applies(int lv, int M) { return lv != QIFT_LEVELS_POT && lv != QIFT_LEVELS_INT3 && M > 32 && M <= kGroupMaxM; }
 inline int tc_tokens(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }   // the tensor-core N of that kernel
 inline int tc_rows_per_item(int M, int lv) { return kTcRows * tc_tiles_per_item(tc_tokens(M), codes_per_word(lv)); }
-inline bool decode_rows_supports(int lv, int M, int N, int K) { return M >= 2 && M <= kGroupMaxM && decode_supports(lv, M > 16 ? 16 : M, N, K); }
+constexpr int kInt3MaxRows = 16;   // three-bit codes on the row-split kernel: six accumulator sets per token tile, two token tiles
+inline bool decode_rows_supports(int lv, int M, int N, int K) {
+    if (lv == QIFT_LEVELS_INT3) return M >= 1 && M <= kInt3MaxRows && K % 256 == 0;
+    return M >= 2 && M <= kGroupMaxM && decode_supports(lv, M > 16 ? 16 : M, N, K);
+}
 int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
                     void* Y, int y_bf16, int32_t* acc_debug, void* workspace, cudaStream_t st);
 int run_forward_rows(const void* X, int x_bf16, int M, int K, int had_block, float clip, const uint32_t* packed, const float* s_n,
@@ -509,12 +516,23 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
     if (!packed || !s_n || !q_a || !s_a || !Y || M <= 0 || N <= 0 || K <= 0 || !valid_levels(lv)) return QIFT_ERR_INVALID_ARG;
     if (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16) return QIFT_ERR_INVALID_ARG;
     if (route < QIFT_ROUTE_AUTO || route > QIFT_ROUTE_DECODE_ROWS) return QIFT_ERR_INVALID_ARG;
-    if (K % codes_per_word(lv) != 0 || K % 4 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!whole_words(K, lv) || K % 4 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(packed) || !aligned16(s_n) || !aligned16(q_a) || !aligned16(s_a) || !aligned16(Y) ||
         (acc_debug && !aligned16(acc_debug)))
         return QIFT_ERR_ALIGNMENT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int y_bf16 = (y_dtype == QIFT_BF16);
+    if (lv == QIFT_LEVELS_INT3) {
+        // three-bit codes: the row-split decode kernel (from one token row), the decode-to-int8 GEMMs, the generic kernel
+        const bool ws_aligned = workspace && (reinterpret_cast<uintptr_t>(workspace) & 255u) == 0;
+        if (route == QIFT_ROUTE_AUTO) {
+            if (decode_rows_supports(lv, M, N, K) && ws_aligned && workspace_bytes >= decode_rows_scratch(M, K)) route = QIFT_ROUTE_DECODE_ROWS;
+            else if (M > kInt3MaxRows && K % 16 == 0) route = (M <= kFusedPairMaxM) ? QIFT_ROUTE_PREFILL_SCRATCH : QIFT_ROUTE_PREFILL_PAIR;
+            else route = QIFT_ROUTE_GENERIC;
+        }
+        if (route == QIFT_ROUTE_DECODE || route == QIFT_ROUTE_PREFILL || route == QIFT_ROUTE_PREFILL_FUSED_PAIR)
+            return QIFT_ERR_UNSUPPORTED_SHAPE;
+    }
     if (route == QIFT_ROUTE_AUTO) {
         if (M <= 16) {
             route = decode_supports(lv, M, N, K) ? QIFT_ROUTE_DECODE : QIFT_ROUTE_GENERIC;
@@ -559,6 +577,7 @@ int linear_impl(const uint32_t* packed, const float* s_n, int lv, const int8_t* 
         case QIFT_LEVELS_MNZ: return launch_generic<QIFT_LEVELS_MNZ>(packed, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st);
         case QIFT_LEVELS_POT: return launch_generic<QIFT_LEVELS_POT>(packed, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st);
         case QIFT_LEVELS_SYM: return launch_generic<QIFT_LEVELS_SYM>(packed, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st);
+        case QIFT_LEVELS_INT3: return launch_generic<QIFT_LEVELS_INT3>(packed, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st);
         default: return launch_generic<QIFT_LEVELS_INT4>(packed, s_n, q_a, s_a, M, N, K, Y, y_bf16, acc_debug, st);
     }
 }
@@ -585,13 +604,15 @@ const char* qift_status_string(int status) {
 }
 
 size_t qift_packed_bytes(int N, int K, int levels) {
-    if (N <= 0 || K <= 0 || !valid_levels(levels) || K % codes_per_word(levels) != 0) return 0;
-    return static_cast<size_t>(round_up16(N)) * packed_pitch(K, levels) * 4;
+    if (N <= 0 || K <= 0 || !valid_levels(levels) || !whole_words(K, levels)) return 0;
+    return static_cast<size_t>(round_up16(N)) * packed_pitch(K, levels) * (tile_word_bytes(levels) / 16);
 }
 
 size_t qift_workspace_bytes_route(int M, int N, int K, int levels, int route) {
     if (M <= 0 || N <= 0 || K <= 0 || !valid_levels(levels)) return 0;
     size_t b = 0;
+    if (levels == QIFT_LEVELS_INT3 && route == QIFT_ROUTE_AUTO)
+        route = decode_rows_supports(levels, M, N, K) ? QIFT_ROUTE_DECODE_ROWS : (M <= kInt3MaxRows) ? QIFT_ROUTE_GENERIC : QIFT_ROUTE_PREFILL_PAIR;
     if (route == QIFT_ROUTE_AUTO) {
         route = (M <= 16) ? QIFT_ROUTE_DECODE : auto_prefill_route(M);
         if (decode_rows_supports(levels, M, N, K)) b = decode_rows_scratch(M, K);  // enough for the fallback route as well
@@ -609,7 +630,7 @@ size_t qift_workspace_bytes(int M, int N, int K, int levels) {
 int qift_pack_weights(const float* W, int N, int K, int levels, int scale_mode, float* s_n, uint32_t* packed, void* stream) {
     if (!W || !s_n || !packed || N <= 0 || K <= 0 || !valid_levels(levels)) return QIFT_ERR_INVALID_ARG;
     if (scale_mode < QIFT_SCALE_GIVEN || scale_mode > QIFT_SCALE_MSE) return QIFT_ERR_INVALID_ARG;
-    if (K % 16 != 0 || K > kMaxRowK) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (K % 16 != 0 || !whole_words(K, levels) || K > kMaxRowK) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(W) || !aligned16(s_n) || !aligned16(packed)) return QIFT_ERR_ALIGNMENT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t smem = static_cast<size_t>(K) * 5;  // the fp32 row and one code byte per weight
@@ -625,6 +646,7 @@ int qift_pack_weights(const float* W, int N, int K, int levels, int scale_mode, 
         QIFT_PACK_CASE(QIFT_LEVELS_POT)
         QIFT_PACK_CASE(QIFT_LEVELS_SYM)
         QIFT_PACK_CASE(QIFT_LEVELS_INT4)
+        QIFT_PACK_CASE(QIFT_LEVELS_INT3)
     }
 #undef QIFT_PACK_CASE
     return QIFT_ERR_INVALID_ARG;
@@ -632,13 +654,14 @@ int qift_pack_weights(const float* W, int N, int K, int levels, int scale_mode, 
 
 int qift_unpack_codes(const uint32_t* packed, int N, int K, int levels, uint8_t* codes, void* stream) {
     if (!packed || !codes || N <= 0 || K <= 0 || !valid_levels(levels)) return QIFT_ERR_INVALID_ARG;
-    if (K % codes_per_word(levels) != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!whole_words(K, levels)) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(packed) || !aligned16(codes)) return QIFT_ERR_ALIGNMENT;
     const long long total = static_cast<long long>(N) * K;
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 32) blocks = 148 * 32;
     return cuda_status(launch_pdl(unpack_codes_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0,
-                                  static_cast<cudaStream_t>(stream), packed, total, K, codes_per_word(levels), codes));
+                                  static_cast<cudaStream_t>(stream), packed, total, K, codes_per_word(levels),
+                                  levels == QIFT_LEVELS_INT3 ? 1 : 0, codes));
 }
 
 int qift_rotate(const float* X, int M, int K, int had_block, float* Y, void* stream) {
@@ -688,6 +711,12 @@ int qift_w4a4_linear(const uint32_t* packed, const float* s_n, const int8_t* q_a
                        QIFT_ROUTE_AUTO, stream);
 }
 
+int qift_w3a4_linear(const uint32_t* packed, const float* s_n, const int8_t* q_a, const float* s_a, int M, int N, int K,
+                     void* Y, int y_dtype, int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream) {
+    return linear_impl(packed, s_n, QIFT_LEVELS_INT3, q_a, s_a, M, N, K, Y, y_dtype, acc_debug, workspace, workspace_bytes,
+                       QIFT_ROUTE_AUTO, stream);
+}
+
 int qift_linear_route(const uint32_t* packed, const float* s_n, int levels, const int8_t* q_a, const float* s_a, int M, int N,
                       int K, void* Y, int y_dtype, int32_t* acc_debug, void* workspace, size_t workspace_bytes, int route,
                       void* stream) {
@@ -723,7 +752,7 @@ static int forward_impl(const void* X, bool host, int x_dtype, int M, int K, int
     if (!X || !Y || !packed || !s_n || M <= 0 || N <= 0 || K <= 0 || !valid_levels(levels)) return QIFT_ERR_INVALID_ARG;
     if ((x_dtype != QIFT_F32 && x_dtype != QIFT_BF16) || (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16))
         return QIFT_ERR_INVALID_ARG;
-    if (K % codes_per_word(levels) != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!whole_words(K, levels)) return QIFT_ERR_UNSUPPORTED_SHAPE;
     const int rs = check_rotation_shape(K, had_block, true);
     if (rs != QIFT_OK) return rs;
     const ForwardLayout L = forward_layout(M, N, K, levels, x_dtype, y_dtype);
@@ -826,7 +855,7 @@ static int check_outputs_and_ahead(int M, int K, int levels, const qift_linear_o
                                    const qift_decode_ahead* ahead) {
     if (M <= 0 || K <= 0 || !valid_levels(levels) || !multi_outputs_ok(outputs, count, true)) return QIFT_ERR_INVALID_ARG;
     if (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16) return QIFT_ERR_INVALID_ARG;
-    if (K % codes_per_word(levels) != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (!whole_words(K, levels)) return QIFT_ERR_UNSUPPORTED_SHAPE;
     for (int i = 0; i < count; ++i)
         if (!aligned16(outputs[i].packed) || !aligned16(outputs[i].s_n) || !aligned16(outputs[i].Y) ||
             (outputs[i].acc_debug && !aligned16(outputs[i].acc_debug)))
@@ -834,7 +863,7 @@ static int check_outputs_and_ahead(int M, int K, int levels, const qift_linear_o
     if (ahead) {
         if (!multi_outputs_ok(ahead->outputs, ahead->count, false) || ahead->K <= 0 || !valid_levels(ahead->levels) || !ahead->levels_buf)
             return QIFT_ERR_INVALID_ARG;
-        if (ahead->K % 16 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+        if (ahead->K % 16 != 0 || !whole_words(ahead->K, ahead->levels)) return QIFT_ERR_UNSUPPORTED_SHAPE;
         if (ahead->levels_bytes < qift_levels_bytes(ahead->K, ahead->outputs, ahead->count)) return QIFT_ERR_WORKSPACE;
         if ((reinterpret_cast<uintptr_t>(ahead->levels_buf) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
         for (int i = 0; i < ahead->count; ++i)
@@ -877,14 +906,22 @@ static int linear_multi_impl(const int8_t* q_a, const float* s_a, int M, int K, 
         c.seg[i].wexp = wexp, c.seg[i].s_n = outputs[i].s_n, c.seg[i].Y = outputs[i].Y, c.seg[i].acc_debug = outputs[i].acc_debug;
         c.seg[i].N = outputs[i].N;
     }
-    if (ahead) {
+    const bool ahead_in_gemm = ahead && ahead->levels != QIFT_LEVELS_INT3;  // the side warps decode one-plane layouts only
+    if (ahead_in_gemm) {
         c.njobs = ahead->count, c.job_K = ahead->K;
         for (int i = 0; i < ahead->count; ++i) {
             c.job[i].packed = ahead->outputs[i].packed, c.job[i].N = ahead->outputs[i].N, c.job[i].levels = ahead->levels;
             c.job[i].out = static_cast<int8_t*>(ahead->levels_buf) + levels_offset(ahead->K, ahead->outputs, i);
         }
     }
-    return run_pair_gemm(c, st);
+    rc = run_pair_gemm(c, st);
+    if (rc != QIFT_OK || !ahead || ahead_in_gemm) return rc;
+    for (int i = 0; i < ahead->count; ++i) {
+        int8_t* out = static_cast<int8_t*>(ahead->levels_buf) + levels_offset(ahead->K, ahead->outputs, i);
+        rc = run_expand(ahead->outputs[i].packed, ahead->levels, ahead->outputs[i].N, ahead->K, out, st);
+        if (rc != QIFT_OK) return rc;
+    }
+    return QIFT_OK;
 }
 
 size_t qift_linear_multi_workspace_bytes(int M, int K, int levels, const qift_linear_output* outputs, int count) {
@@ -942,7 +979,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     if ((x_dtype != QIFT_F32 && x_dtype != QIFT_BF16) || (y_dtype != QIFT_F32 && y_dtype != QIFT_BF16))
         return QIFT_ERR_INVALID_ARG;
     if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return QIFT_ERR_INVALID_ARG;
-    if (M > kGroupMaxM) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (M > kGroupMaxM || (levels == QIFT_LEVELS_INT3 && M > kInt3MaxRows)) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (plan_bytes < qift_group_plan_bytes(count)) return QIFT_ERR_WORKSPACE;
     if (!aligned16(plan_dev) || !aligned16(plan_host)) return QIFT_ERR_ALIGNMENT;
     // Rows per work item, which also selects the kernel (dispatch_grouped): 64 / 32 for the K-split kernel, 128 for the
@@ -950,7 +987,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : 64;  // below wide_min_m there is only M = 1
     const bool use_tc = tc_rows_applies(levels, M);                  // 33 .. 64 rows (not PoT): the tcgen05 kernel, 256-row items
     if (use_tc) rows_per_item = tc_rows_per_item(M, levels);
-    if (!use_tc && rows_per_item == kWideRows && M > 8 && M <= 16 && levels != QIFT_LEVELS_POT) {  // PoT measured slower with two tiles
+    if (!use_tc && rows_per_item == kWideRows && M > 8 && M <= 16 && levels != QIFT_LEVELS_POT && levels != QIFT_LEVELS_INT3) {  // PoT measured slower with two tiles
         long long items256 = 0;
         for (int i = 0; i < count; ++i) items256 += (problems[i].N + 2 * kWideRows - 1) / (2 * kWideRows);
         if (items256 >= 2ll * sm_count()) rows_per_item = 2 * kWideRows;
@@ -961,7 +998,8 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     for (int i = 0; i < count; ++i) {
         const qift_group_problem& q = problems[i];
         if (!q.X || !q.packed || !q.s_n || !q.q_a || !q.s_a || !q.Y || q.N <= 0 || q.K <= 0) return QIFT_ERR_INVALID_ARG;
-        if (!decode_supports(levels, M > 16 ? 16 : M, q.N, q.K)) return QIFT_ERR_UNSUPPORTED_SHAPE;
+        if (levels == QIFT_LEVELS_INT3 ? !decode_rows_supports(levels, M, q.N, q.K) : !decode_supports(levels, M > 16 ? 16 : M, q.N, q.K))
+            return QIFT_ERR_UNSUPPORTED_SHAPE;
         const int rs = check_rotation_shape(q.K, q.had_block, true);
         if (rs != QIFT_OK) return rs;
         if (!aligned16(q.X) || !aligned16(q.packed) || !aligned16(q.s_n) || !aligned16(q.q_a) || !aligned16(q.s_a) ||
@@ -990,7 +1028,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     h->any_kron = any_kron;
     // the row-split kernel stages one K-chunk of all tokens per copy: its q_a is chunk-major (ChunkMajorDst)
     h->q_pot_lut = (rows_per_item >= kWideRows && levels == QIFT_LEVELS_POT && M > 8) ? 1 : 0;  // the kernel's POT_LUT
-    h->q_chunk_bytes = (rows_per_item >= kWideRows) ? wide_chunk_words(rows_per_item / 16, wide_token_tiles(M)) * codes_per_word(levels) : 0;
+    h->q_chunk_bytes = (rows_per_item >= kWideRows) ? wide_chunk_words(rows_per_item / 16, wide_token_tiles(M), levels) * codes_per_word(levels) : 0;
     h->reserved[0] = use_tc ? 1 : 0;
     if (use_tc) h->q_chunk_bytes = 0;  // that kernel reads q_a row-major (prescaled even planes, as the K-split kernel does)
     return cuda_status(cudaMemcpyAsync(plan_dev, plan_host, sizeof(GroupHeader) + static_cast<size_t>(count) * sizeof(GroupProblemDev),
@@ -1105,6 +1143,10 @@ int dispatch_tc(const GroupHeader* h, const GroupProblemDev* host, const GroupPr
 template <int LV>
 int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq,
                      cudaStream_t st) {
+    if constexpr (LV == QIFT_LEVELS_INT3) {   // three-bit codes: the row-split kernel with one or two token tiles
+        if (h->rows_per_item != kWideRows || h->M > kInt3MaxRows) return QIFT_ERR_INVALID_ARG;
+        return h->M > 8 ? launch_grouped_wide<LV, 2, 1, 8>(h, host, dev, sumq, st) : launch_grouped_wide<LV, 1, 1, 8>(h, host, dev, sumq, st);
+    } else {
     if (h->reserved[0]) return dispatch_tc<LV>(h, host, dev, sumq, st);   // the plan chose the tcgen05 kernel (33 .. 64 rows)
     // (256-row items as sixteen consumer warps were measured slower and are not dispatched.)
     if (h->rows_per_item == 2 * kWideRows) return launch_grouped_wide<LV, 2, 2, 8>(h, host, dev, sumq, st);
@@ -1114,6 +1156,7 @@ int dispatch_grouped(const GroupHeader* h, const GroupProblemDev* host, const Gr
         return h->M > 8 ? launch_grouped_wide<LV, 2, 1, 8>(h, host, dev, sumq, st) : launch_grouped_wide<LV, 1, 1, 8>(h, host, dev, sumq, st);
     if (h->M == 1) return launch_grouped<LV, 1, 4, true>(h, host, dev, sumq, st);
     return QIFT_ERR_INVALID_ARG;  // no plan has other row counts per item
+    }
 }
 }  // namespace
 
@@ -1129,7 +1172,7 @@ int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8
     h.magic = kGroupMagic, h.count = 1, h.M = M, h.levels = lv, h.y_bf16 = y_bf16, h.rows_per_item = kWideRows;
     h.total_items = (N + kWideRows - 1) / kWideRows;
     h.q_pot_lut = (lv == QIFT_LEVELS_POT && M > 8) ? 1 : 0;
-    h.q_chunk_bytes = wide_chunk_words(kDecWarps, wide_token_tiles(M)) * codes_per_word(lv);
+    h.q_chunk_bytes = wide_chunk_words(kDecWarps, wide_token_tiles(M), lv) * codes_per_word(lv);
     GroupProblemDev rec{};
     rec.X = nullptr, rec.packed = packed, rec.s_n = s_n, rec.q_a = q_out, rec.s_a = const_cast<float*>(s_a), rec.Y = Y;
     rec.acc_debug = acc_debug, rec.N = N, rec.K = K, rec.had_block = 0, rec.item_begin = 0, rec.inv_sqrt_b = 1.0f, rec.quant_src = 0;
@@ -1147,6 +1190,9 @@ int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8
         QIFT_ROWS_CASE(QIFT_LEVELS_MNZ)
         QIFT_ROWS_CASE(QIFT_LEVELS_POT)
         QIFT_ROWS_CASE(QIFT_LEVELS_SYM)
+        case QIFT_LEVELS_INT3:
+            return M > 8 ? launch_grouped_wide<QIFT_LEVELS_INT3, 2, 1, 8>(&h, &rec, none, sumq, st, true)
+                         : launch_grouped_wide<QIFT_LEVELS_INT3, 1, 1, 8>(&h, &rec, none, sumq, st, true);
         default:
             QIFT_ROWS_CASE(QIFT_LEVELS_INT4)
     }
@@ -1159,7 +1205,7 @@ int run_forward_rows(const void* X, int x_bf16, int M, int K, int had_block, flo
     h.magic = kGroupMagic, h.count = 1, h.M = M, h.levels = lv, h.y_bf16 = y_bf16, h.rows_per_item = kWideRows;
     h.total_items = (N + kWideRows - 1) / kWideRows;
     h.q_pot_lut = (lv == QIFT_LEVELS_POT && M > 8) ? 1 : 0;
-    h.q_chunk_bytes = wide_chunk_words(kDecWarps, wide_token_tiles(M)) * codes_per_word(lv);
+    h.q_chunk_bytes = wide_chunk_words(kDecWarps, wide_token_tiles(M), lv) * codes_per_word(lv);
     GroupProblemDev rec{};
     rec.X = X, rec.packed = packed, rec.s_n = s_n, rec.q_a = q_scratch, rec.s_a = s_a, rec.Y = Y, rec.acc_debug = nullptr;
     rec.N = N, rec.K = K, rec.had_block = had_block, rec.item_begin = 0, rec.quant_src = 0;
@@ -1184,6 +1230,9 @@ int run_forward_rows(const void* X, int x_bf16, int M, int K, int had_block, flo
         QIFT_ROWS_CASE(QIFT_LEVELS_MNZ)
         QIFT_ROWS_CASE(QIFT_LEVELS_POT)
         QIFT_ROWS_CASE(QIFT_LEVELS_SYM)
+        case QIFT_LEVELS_INT3:
+            return M > 8 ? launch_grouped_wide<QIFT_LEVELS_INT3, 2, 1, 8>(&h, &rec, none, sumq, st, true)
+                         : launch_grouped_wide<QIFT_LEVELS_INT3, 1, 1, 8>(&h, &rec, none, sumq, st, true);
         default:
             QIFT_ROWS_CASE(QIFT_LEVELS_INT4)
     }
@@ -1222,6 +1271,7 @@ int qift_group_linear(const void* plan_host, const void* plan_dev, void* stream)
         case QIFT_LEVELS_MNZ: return dispatch_grouped<QIFT_LEVELS_MNZ>(h, host, dev, sumq, st);
         case QIFT_LEVELS_POT: return dispatch_grouped<QIFT_LEVELS_POT>(h, host, dev, sumq, st);
         case QIFT_LEVELS_SYM: return dispatch_grouped<QIFT_LEVELS_SYM>(h, host, dev, sumq, st);
+        case QIFT_LEVELS_INT3: return dispatch_grouped<QIFT_LEVELS_INT3>(h, host, dev, sumq, st);
         default: return dispatch_grouped<QIFT_LEVELS_INT4>(h, host, dev, sumq, st);
     }
 }
@@ -1554,7 +1604,7 @@ int qift_kv4_quantize(const void* X, int x_dtype, int T, int H, int D, int had_b
 
 int qift_expand_weights(const uint32_t* packed, int N, int K, int levels, int8_t* levels_out, void* stream) {
     if (!packed || !levels_out || N <= 0 || K <= 0 || !valid_levels(levels)) return QIFT_ERR_INVALID_ARG;
-    if (K % 16 != 0) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (K % 16 != 0 || !whole_words(K, levels)) return QIFT_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(packed) || (reinterpret_cast<uintptr_t>(levels_out) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
     return run_expand(packed, levels, N, K, levels_out, static_cast<cudaStream_t>(stream));
 }

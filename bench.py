@@ -156,7 +156,7 @@ def build_stack(torch, qift, shapes, n_layers, M, levels_of_layer, seed, x_dtype
             qift.qift_rotate(W, B, out=W)
             m = Module()
             m.name, m.N, m.K, m.B, m.levels = name, N, K, B, lv
-            m.bits = 4 if lv == qift.INT4 else 2
+            m.bits = 4 if lv == qift.INT4 else 3 if lv == qift.INT3 else 2
             m.packed, m.s_n = qift.qift_pack_weights(W, lv, qift.SCALE_MSE)
             del W
             x = torch.randn((M, K), device=device, dtype=torch.float32, generator=gen)
@@ -553,8 +553,33 @@ def run_mixed_stack(torch, qift, L, device, gen, args):
                        "grouped API (4 launches per step)")
     if args.layers >= 16:
         out["l_sweep"] = [point(args.layers * l // 32, args.layers - args.layers * l // 32) for l in (4, 8, 12)]
+    out["w3a4_uniform"] = uniform_w3a4(torch, qift, L, device, gen, args, st)
     out["prefill_m2048"] = mixed_prefill(torch, qift, L, device, gen, args, n4)
     return out
+
+
+def uniform_w3a4(torch, qift, L, device, gen, args, st):
+    """The equal-budget reference of Sec. 4.4 (Tables 9-11): every layer at three bits (W3A4, Eq. 1 with b = 3), the same
+    bytes per step as config 5's L = 16 mixed stack.  One grouped plan, two launches per step; M = 1 and M = 16."""
+    vp = ctypes.c_void_p
+    mods = build_stack(torch, qift, synth.LLAMA2_7B, args.layers, 16, lambda l: qift.INT3, 5200, torch.float32, torch.float32, device,
+                       gen)
+    rows = []
+    for M in (1, 16):
+        plan = qift.qift_group_plan([(m.x[:M].contiguous(), m.packed, m.s_n, m.B) for m in mods], qift.INT3, CLIP)
+        algo = sum(product_bytes(M, m.N, m.K, m.bits) + quant_bytes(M, m.K) for m in mods)
+
+        def step():
+            rc = L.qift_group_forward(vp(plan.host.data_ptr()), vp(plan.dev.data_ptr()), st)
+            assert rc == 0, rc
+
+        ms = time_ms(torch, step, max(3, min(args.steps, 100)), warm=5)
+        rows.append({"M": M, "bits_per_weight": 3.0, "ms_per_step": round(ms, 5), "tokens_per_s": round(M / (ms * 1e-3), 1),
+                     "value": round(algo / (ms * 1e-3) / 1e9, 2), "unit": "GB/s", "algorithmic_bytes_per_step": algo,
+                     "pct_of_8TBs": round(100 * algo / (ms * 1e-3) / 8e12, 2)})
+        del plan
+    return {"workload": f"{args.layers} W3A4 layers, LLaMA-2-7B shapes, grouped API (2 launches per step), "
+                        "linear_grouped_wide_kernel with the one-bit plane as single-bit operands", "points": rows}
 
 
 def mixed_prefill(torch, qift, L, device, gen, args, n4):

@@ -215,7 +215,7 @@ int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_blo
  * (Sec. 3.1: the layer pipeline; the paper describes no kernels, so the scheduling is this library's.)
  * In a transformer layer q / k / v read the same activation, and so do gate / up: it needs rotating and
  * quantizing once.  qift_forward_multi runs S2 + S3 once on X and then S4 + S5 for every listed output.
- * With more than 512 token rows the products run as ONE launch of the CTA-pair tensor-core GEMM over the
+ * With more than 128 token rows the products run as ONE launch of the CTA-pair tensor-core GEMM over the
  * channel tiles of all outputs, reading int8 levels decoded from the packed codes into `levels_buf`
  * (qift_levels_bytes; output i at the sum of the earlier outputs' N*K rounded up to 1 KiB each).
  *
@@ -229,12 +229,12 @@ int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_blo
  *   X            dev [M,K] fp32 or bf16;  had_block, clip_ratio as for qift_quantize_act
  *   outputs      HOST array of 1..4 outputs: packed / s_n from qift_pack_weights (all with this K and
  *                level set), Y dev [M,N] (fp32 or bf16 per y_dtype), acc_debug dev int32 [M,N] or NULL
- *   scratch      dev, >= qift_forward_multi_scratch_bytes(...), 256-byte aligned: q_a, s_a and (M <= 512)
+ *   scratch      dev, >= qift_forward_multi_scratch_bytes(...), 256-byte aligned: q_a, s_a and (M <= 128)
  *                the workspace of the per-output routes; undefined afterwards
- *   levels_buf   dev, >= qift_levels_bytes(K, outputs, count), 256-byte aligned; needed when M > 512.
+ *   levels_buf   dev, >= qift_levels_bytes(K, outputs, count), 256-byte aligned; needed when M > 128.
  *                levels_ready = 1 promises it already holds the decoded levels of exactly these outputs
  *                (written by the previous call's `ahead`); nothing can check that promise
- *   ahead        HOST, or NULL.  With M <= 512 the call still honours it (separate decoding launches).
+ *   ahead        HOST, or NULL.  With M <= 128 the call still honours it (separate decoding launches).
  * Results are bit-identical to qift_quantize_act + qift_w2a4_linear / qift_w4a4_linear per output.
  * Errors: INVALID_ARG (null pointers, count outside 1..4, enums), UNSUPPORTED_SHAPE, ALIGNMENT,
  * WORKSPACE (scratch or a levels buffer missing or too small), CUDA. */
@@ -261,14 +261,15 @@ int qift_forward_multi(const void* X, int x_dtype, int M, int K, int had_block, 
                        void* stream);
 /* The product part alone (S4 + S5 for every output) on an activation that qift_quantize_act has already
  * quantized: q_a int8 [M,K], s_a fp32 [M].  workspace >= qift_linear_multi_workspace_bytes(...) bytes
- * (0 for M > 512; NULL allowed then), 256-byte aligned; everything else as for qift_forward_multi. */
+ * (0 for M > 128; NULL allowed then), 256-byte aligned; everything else as for qift_forward_multi. */
 size_t qift_linear_multi_workspace_bytes(int M, int K, int levels, const qift_linear_output* outputs, int count);
 int qift_linear_multi(const int8_t* q_a, const float* s_a, int M, int K, int levels, const qift_linear_output* outputs,
                       int count, int y_dtype, void* workspace, size_t workspace_bytes, void* levels_buf,
                       size_t levels_bytes, int levels_ready, const qift_decode_ahead* ahead, void* stream);
 
 /* ---- Grouped decode path -----------------------------------------------------------------------
- * One persistent launch serves a list of independent layer problems that share M (<= 64 token rows),
+ * One persistent launch serves a list of independent layer problems that share M (<= 128 token rows; PoT <= 64,
+ * INT3 <= 16),
  * the level set, the dtypes and the clip ratio -- e.g. all linear modules of one decode step.  A W2
  * matrix is only 1-15 MB, far too little for one launch to reach an HBM steady state; the grouped
  * kernel streams the whole list back to back.  (No counterpart in the paper: it describes no kernels.)
@@ -285,7 +286,8 @@ int qift_linear_multi(const int8_t* q_a, const float* s_a, int M, int K, int lev
  * Problems must not alias each other's Y, nor each other's q_a / s_a with one exception: modules that
  * read the SAME activation (q/k/v; gate/up) may name the same X, q_a, s_a (same K and had_block); the
  * plan then quantizes that activation once and every such product reads it.  K % 256 == 0 (two-bit sets, INT3) or
- * K % 128 == 0 (INT4), K <= 16384.  INT3 plans take up to 16 token rows. */
+ * K % 128 == 0 (INT4), K <= 16384.  INT3 plans take up to 16 token rows, PoT plans up to 64 (the tcgen05 kernel that
+ * serves 33 .. 128 rows takes the sets that are affine in the code). */
 typedef struct qift_group_problem {
     const void* X;          /* dev [M,K] fp32 or bf16                         */
     const uint32_t* packed; /* dev, from qift_pack_weights                    */

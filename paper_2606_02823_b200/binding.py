@@ -322,7 +322,7 @@ def qift_levels_bytes(K: int, weights) -> int:
 def qift_forward_multi(X, had_block: int, weights, levels: int, clip_ratio: float = 0.9, out_dtype=torch.float32,
                        want_acc: bool = False, scratch=None, levels_buf=None, levels_ready: bool = False, ahead=None, outs=None):
     """One activation X [M,K], several products: weights = [(packed, s_n), ...] (1..4) -> ([Y_i [M,N_i]], [acc_i or None]).
-    levels_buf: uint8 tensor of qift_levels_bytes(K, weights) bytes (allocated when omitted; needed for M > 512);
+    levels_buf: uint8 tensor of qift_levels_bytes(K, weights) bytes (allocated when omitted; needed for M > 128);
     levels_ready: it already holds these weights' decoded levels (written through a previous call's `ahead`);
     ahead = (next_weights, next_K, next_levels, next_levels_buf): decode the next call's codes during this one."""
     _dev(X)

@@ -52,7 +52,8 @@ struct GroupProblemDev {
 };
 static_assert(sizeof(GroupProblemDev) == 96, "problem record is 96 bytes");
 
-constexpr int kGroupMaxM = 64;     // token rows of a plan; also the row length of the token-sum table
+constexpr int kGroupMaxM = 128;    // token rows of a plan (65 .. 128: the tcgen05 kernel only); also the row length of the token-sum table
+constexpr int kWideMaxM = 64;      // token rows the mma.sync row-split kernel takes (eight token tiles)
 constexpr uint32_t kGroupMagic = 0x51494654u;
 
 // ------------------------------------------------------------------------------------------------

@@ -33,6 +33,10 @@ namespace {
 inline int wide_min_m(int lv) { return (lv == QIFT_LEVELS_POT || lv == QIFT_LEVELS_INT3) ? 1 : 2; }
 constexpr int kFusedMaxM = 128;
 constexpr int kFusedPairMaxM = 512;
+// Several products of one activation (qift_forward_multi / qift_linear_multi): from this many token rows on the
+// decode-to-int8 CTA-pair GEMM with its segments and decode-ahead warps beats the per-output fused routes (a
+// LLaMA-3.1-8B layer at 256 / 512 rows: measured in the benchmark's mid_m block).
+constexpr int kMultiPairMinM = 129;
 inline int auto_prefill_route(int M) {
     return (M <= kFusedMaxM) ? QIFT_ROUTE_PREFILL : (M <= kFusedPairMaxM) ? QIFT_ROUTE_PREFILL_FUSED_PAIR : QIFT_ROUTE_PREFILL_PAIR;
 }
@@ -496,7 +500,7 @@ int run_prefill_fused(const uint32_t* packed, const float* s_n, int lv, const in
 // Scratch of QIFT_ROUTE_DECODE_ROWS: the re-laid-out activations and the token sums.
 inline size_t decode_rows_scratch(int M, int K) { return ((static_cast<size_t>(M) * K + 255) & ~static_cast<size_t>(255)) + 512; }
 // Grouped plans: the row-split mma.sync kernel up to 32 token rows (PoT: up to 64), the tcgen05 weight-streaming kernel
-// from 33 to 64, where it is the faster one (16 LLaMA-2-7B layers, product kernel, MNZ / INT4: 32 rows 1.9 / 2.8 TB/s
+// from 33 to 128, where it is the faster one (16 LLaMA-2-7B layers, product kernel, MNZ / INT4: 32 rows 1.9 / 2.8 TB/s
 // against 2.8 / 4.5 on mma.sync; 64 rows 1.8 / 3.2 against 1.3 / 2.5).
 inline bool tc_rows_applies(int lv, int M) { return lv != QIFT_LEVELS_POT && lv != QIFT_LEVELS_INT3 && M > 32 && M <= kGroupMaxM; }
 inline int tc_tokens(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }   // the tensor-core N of that kernel
@@ -504,7 +508,7 @@ inline int tc_rows_per_item(int M, int lv) { return kTcRows * tc_tiles_per_item(
 constexpr int kInt3MaxRows = 16;   // three-bit codes on the row-split kernel: six accumulator sets per token tile, two token tiles
 inline bool decode_rows_supports(int lv, int M, int N, int K) {
     if (lv == QIFT_LEVELS_INT3) return M >= 1 && M <= kInt3MaxRows && K % 256 == 0;
-    return M >= 2 && M <= kGroupMaxM && decode_supports(lv, M > 16 ? 16 : M, N, K);
+    return M >= 2 && M <= kWideMaxM && decode_supports(lv, M > 16 ? 16 : M, N, K);
 }
 int run_decode_rows(const uint32_t* packed, const float* s_n, int lv, const int8_t* q_a, const float* s_a, int M, int N, int K,
                     void* Y, int y_bf16, int32_t* acc_debug, void* workspace, cudaStream_t st);
@@ -825,7 +829,7 @@ MultiLayout multi_layout(int M, int K, int levels, const qift_linear_output* o, 
     L.q_off = off, off += up1k(static_cast<size_t>(M) * K);
     L.sa_off = off, off += up1k(static_cast<size_t>(M) * 4);
     size_t ws = 0;
-    if (M <= kFusedPairMaxM)  // the routes below the pair GEMM bring their own (small) workspace needs
+    if (M < kMultiPairMinM)  // the routes below the pair GEMM bring their own (small) workspace needs
         for (int i = 0; i < count; ++i) {
             const size_t w = qift_workspace_bytes(M, o[i].N, K, levels);
             if (w > ws) ws = w;
@@ -877,7 +881,7 @@ static int linear_multi_impl(const int8_t* q_a, const float* s_a, int M, int K, 
                              int y_dtype, void* workspace, size_t workspace_bytes, void* levels_buf, size_t levels_bytes,
                              int levels_ready, const qift_decode_ahead* ahead, void* stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool pair_route = M > kFusedPairMaxM && K % 16 == 0;
+    const bool pair_route = M >= kMultiPairMinM && K % 16 == 0;
     int rc;
     if (!pair_route) {
         for (int i = 0; i < count; ++i) {
@@ -954,7 +958,7 @@ int qift_forward_multi(const void* X, int x_dtype, int M, int K, int had_block, 
     const MultiLayout L = multi_layout(M, K, levels, outputs, count);
     if (!scratch || scratch_bytes < L.total) return QIFT_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(scratch) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
-    if (M > kFusedPairMaxM && K % 16 == 0) {  // found before anything is launched
+    if (M >= kMultiPairMinM && K % 16 == 0) {  // found before anything is launched
         if (!levels_buf || levels_bytes < qift_levels_bytes(K, outputs, count)) return QIFT_ERR_WORKSPACE;
         if ((reinterpret_cast<uintptr_t>(levels_buf) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
     }
@@ -980,6 +984,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
         return QIFT_ERR_INVALID_ARG;
     if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return QIFT_ERR_INVALID_ARG;
     if (M > kGroupMaxM || (levels == QIFT_LEVELS_INT3 && M > kInt3MaxRows)) return QIFT_ERR_UNSUPPORTED_SHAPE;
+    if (M > kWideMaxM && !tc_rows_applies(levels, M)) return QIFT_ERR_UNSUPPORTED_SHAPE;   // 65 .. 128 rows: the tcgen05 kernel's sets only
     if (plan_bytes < qift_group_plan_bytes(count)) return QIFT_ERR_WORKSPACE;
     if (!aligned16(plan_dev) || !aligned16(plan_host)) return QIFT_ERR_ALIGNMENT;
     // Rows per work item, which also selects the kernel (dispatch_grouped): 64 / 32 for the K-split kernel, 128 for the

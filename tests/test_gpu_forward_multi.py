@@ -48,10 +48,12 @@ def clean():
                                     (513, (1000,), 256),               # one segment, four 256-wide tiles, ragged M
                                     (40, (272, 64), 512),              # row-split decode route per output
                                     (1, (256, 256, 256, 144), 256),    # single token, four outputs
-                                    (300, (200, 320), 256),            # fused prefill route per output
-                                    (1100, (520, 136), 256),           # 512-token tiles, all cut into half tiles, ragged M
-                                    (2100, (1000,), 256),              # 512-token tiles, whole ones only
-                                    (1024, (4800, 264), 128)])         # whole rounds of 512-token tiles + a tail of half tiles
+                                    (100, (200, 320), 256),            # fused prefill route per output
+                                    (129, (200, 320), 256),            # the first token count of the pair GEMM: one half-empty tile
+                                    (300, (200, 320), 256),            # two token tiles, the second ragged
+                                    (1100, (520, 136), 256),           # five token tiles, ragged M
+                                    (2100, (1000,), 256),              # nine token tiles
+                                    (1024, (4800, 264), 128)])         # more channel tiles than CTA pairs
 def test_forward_multi_matches_oracle(lv, M, Ns, K):
     host, gpu = make_weights(100 * lv + M, Ns, K, lv)
     x, _ = synth.activations(7 + M, M, K, max(1, K // 100))
@@ -92,7 +94,7 @@ def test_forward_multi_rejects_bad_arguments():
     host, gpu = make_weights(5, (128,), K, lv)
     x = dev(synth.activations(6, 600, K, 2)[0])
     small = torch.empty(256, dtype=torch.uint8, device="cuda")
-    with pytest.raises(qift.QiftError) as e:       # M > 512 needs the levels buffer
+    with pytest.raises(qift.QiftError) as e:       # M > 128 needs the levels buffer
         qift.qift_forward_multi(x, 256, gpu, lv, levels_buf=small)
     assert e.value.status == qift.ERR_WORKSPACE
     with pytest.raises(qift.QiftError) as e:       # scratch too small

@@ -378,11 +378,13 @@ def test_forward_one_call(name, M, N, K, B):
 
 # ---------------------------------------------------------------------------------- grouped path
 @pytest.mark.parametrize("name", list(LEVELS))
-@pytest.mark.parametrize("M", [1, 2, 5, 6, 8, 9, 13, 16, 17, 27, 32, 33, 50, 64])
+@pytest.mark.parametrize("M", [1, 2, 5, 6, 8, 9, 13, 16, 17, 27, 32, 33, 50, 64, 65, 100, 128])
 def test_grouped_forward(name, M):
     # a ragged list: different N (incl. not a multiple of the row block), different K (incl. a
     # partial last chunk), more items than CTAs
     lv = LEVELS[name][0]
+    if M > 64 and name == "POT":
+        pytest.skip("PoT plans end at 64 token rows (rejection checked in test_grouped_rejects_bad_plans)")
     shapes = [(256, 256), (40, 512), (100, 2304), (4000, 256), (48, 4096), (130, 2560), (16, 11008), (2400, 256),
               (9600, 256)]
     probs, refs = [], []
@@ -433,9 +435,9 @@ def test_grouped_forward_long_list(name, M):
 
 
 @pytest.mark.parametrize("name", ["MNZ", "SYM", "INT4"])
-@pytest.mark.parametrize("M", [33, 64])
+@pytest.mark.parametrize("M", [33, 64, 96, 128])
 def test_grouped_forward_tensor_memory_kernel_many_items(name, M):
-    # 33 .. 64 token rows of a plan run on the tcgen05 kernel whose weight operand lives in tensor memory.  More
+    # 33 .. 128 token rows of a plan run on the tcgen05 kernel whose weight operand lives in tensor memory.  More
     # 256-channel items than SMs, so CTAs take several items each (both accumulator buffers, the operand ring wrapping
     # across item boundaries); an odd number of 16-word slices per item (the two expander warps of a lane quarter swap
     # parity from item to item); ragged N: a last item with one valid 128-channel block, rows beyond N inside a block
@@ -536,9 +538,12 @@ def test_grouped_rejects_bad_plans():
     with pytest.raises(qift.QiftError) as e:
         qift.qift_group_plan([(x, packed, s_n, 96)], qift.MNZ)          # had_block not a power of two
     assert e.value.status == qift.ERR_UNSUPPORTED_SHAPE
-    x65 = torch.zeros((65, 256), device="cuda")
+    x129 = torch.zeros((129, 256), device="cuda")
     with pytest.raises(qift.QiftError) as e:
-        qift.qift_group_plan([(x65, packed, s_n, 256)], qift.MNZ)       # M > 64
+        qift.qift_group_plan([(x129, packed, s_n, 256)], qift.MNZ)      # M > 128
+    assert e.value.status == qift.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(qift.QiftError) as e:
+        qift.qift_group_plan([(x129[:65], packed, s_n, 256)], qift.POT)  # PoT plans end at 64 rows (packed bytes are not read)
     assert e.value.status == qift.ERR_UNSUPPORTED_SHAPE
     L = qift.lib()
     assert L.qift_group_forward(None, None, None) == qift.ERR_INVALID_ARG

@@ -460,8 +460,17 @@ constexpr int kWideRows = 16 * kDecWarps;        // 128 rows per item with one t
 // sixteen warps (twice the warps to hide the latencies of the load -> logic -> product chains) or as two tiles per
 // warp (the activation registers of a slice feed both tiles); their stages are a quarter tile of K (32 words) so
 // that as many stages fit as with 128 rows.
+// CTAs per SM of the row-split kernel.  With one token tile the PoT and the three-bit variants issue two product
+// instructions and two or more logic operations per packed word where the two-bit sets issue one; two CTAs of
+// half-size stages keep the pipes fed across each other's stage hand-overs (96 registers per thread is the limit for
+// two CTAs of nine warps).  Measured, whole steps: three-bit codes 5.89 -> 6.61 TB/s (32 LLaMA-2-7B layers, M = 1), PoT
+// 4.06 -> 4.22 (M = 1), 3.93 -> 4.04 (M = 4); the standard set 5.82 -> 5.75 at M = 4, so the others keep one CTA.
+__host__ __device__ constexpr int wide_ctas_per_sm(int lv, int nt, int tiles) {
+    return ((lv == QIFT_LEVELS_POT || lv == QIFT_LEVELS_INT3) && nt == 1 && tiles == 8) ? 2 : 1;
+}
 __host__ __device__ constexpr int wide_chunk_words(int tiles, int nt, int lv = QIFT_LEVELS_MNZ) {
-    return (tiles > 8 || nt > 2 || lv == QIFT_LEVELS_INT3) ? 64 : 128;   // three-bit codes: a tile column is 96 bytes, not 64
+    // three-bit codes: a tile column is 96 bytes, not 64; two CTAs per SM: half the shared memory each
+    return (tiles > 8 || nt > 2 || lv == QIFT_LEVELS_INT3 || wide_ctas_per_sm(lv, nt, tiles) > 1) ? 64 : 128;
 }
 __host__ __device__ constexpr int wide_token_tiles(int M) { return M > 32 ? 8 : M > 16 ? 4 : M > 8 ? 2 : 1; }
 
@@ -474,7 +483,7 @@ __host__ __device__ inline size_t wide_smem_bytes(int lv, int M, int tiles, int 
 }
 
 template <int LV, int NT, int RT, int CWARPS>
-__global__ void __launch_bounds__((CWARPS + 1) * 32, 1)
+__global__ void __launch_bounds__((CWARPS + 1) * 32, wide_ctas_per_sm(LV, NT, CWARPS * RT))
 linear_grouped_wide_kernel(const GroupParams gp) {
     using T = DecodeTraits<LV>;
     constexpr int TILES = CWARPS * RT;           // row tiles per item

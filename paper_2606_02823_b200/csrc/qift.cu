@@ -1090,13 +1090,14 @@ int launch_grouped_wide(const GroupHeader* h, const GroupProblemDev* host, const
         const int count = (h->count - first < kGroupSlice) ? h->count - first : kGroupSlice;
         const int item_first = host[first].item_begin;
         const int item_end = (first + count < h->count) ? host[first + count].item_begin : h->total_items;
-        int stages = static_cast<int>((226 * 1024 - static_cast<size_t>(count) * sizeof(SmemProblem) - 64) / stage);
+        constexpr int cps = wide_ctas_per_sm(LV, NT, RT * CWARPS);   // each CTA gets its share of the SM's shared memory
+        int stages = static_cast<int>(((cps == 2 ? 112 : 226) * 1024 - static_cast<size_t>(count) * sizeof(SmemProblem) - 64) / stage);
         if (stages < 2) stages = 2;
         if (stages > 8) stages = 8;
         const size_t smem = wide_smem_bytes(LV, h->M, RT * CWARPS, stages, count);
         cudaError_t e = allow_smem(kernel, smem);
         if (e != cudaSuccess) return cuda_status(e);
-        int grid = sm_count();
+        int grid = cps * sm_count();
         if (grid > item_end - item_first) grid = item_end - item_first;
         GroupParams gp{dev + first, sumq, first, count, item_first, item_end, h->M, h->y_bf16, stages, 0, {}};
         if (single) gp.use_single = 1, gp.single = host[0];

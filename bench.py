@@ -312,22 +312,25 @@ def run_gpu(args):
     e2e_steps = max(3, min(args.steps, 100))
     ms_host = timed(run_host, e2e_steps, 3)
 
-    # the same step as four plans of a quarter of the modules each, alternating between two streams: the copies
-    # of one chunk overlap the kernels of the other (one call per chunk, same entry point)
-    n_chunks = max(1, min(4, len(mods) // 7))   # measured: 2 / 4 / 8 / 16 chunks -> 0.376 / 0.358 / 0.390 / 0.535 ms per step
+    # the same step as eight plans of an eighth of the modules each, dealt to four streams: the copies of one chunk
+    # overlap the kernels of the others (one call per chunk, same entry point).  Measured, ms per step (host-to-device
+    # copy alone 0.095, device-to-host 0.108, kernels 0.261): 1 chunk 0.46; 2 chunks on 2 streams 0.37; 4 chunks on 2 / 3 / 4
+    # streams 0.40 / 0.34 / 0.34; 6 chunks on 3 / 6 streams 0.33 / 0.32; 8 chunks on 3 / 4 / 6 streams 0.34 / 0.32 / 0.32
+    # (with two streams chunk i + 2 cannot start its copy before chunk i has copied its results out)
+    n_chunks = max(1, min(8, len(mods) // 7))
     per = (len(mods) + n_chunks - 1) // n_chunks
     chunk_plans = [qift.qift_group_plan([(m.x, m.packed, m.s_n, m.B) for m in mods[i * per:(i + 1) * per]], qift.MNZ, CLIP,
                                         arenas=True) for i in range(n_chunks)]
     torch.cuda.synchronize()
-    side = [torch.cuda.Stream(device=device), torch.cuda.Stream(device=device)]
+    side = [torch.cuda.Stream(device=device) for _ in range(4)]
 
     def run_host_chunked():
         for i, cp in enumerate(chunk_plans):
             check(L.qift_group_forward_host(vp(cp.host.data_ptr()), vp(cp.dev.data_ptr()), vp(cp.x_host.data_ptr()),
                                             vp(cp.x_arena.data_ptr()), cp.x_arena.numel(), vp(cp.y_arena.data_ptr()),
-                                            vp(cp.y_host.data_ptr()), cp.y_arena.numel(), vp(side[i % 2].cuda_stream)))
-        side[0].synchronize()
-        side[1].synchronize()
+                                            vp(cp.y_host.data_ptr()), cp.y_arena.numel(), vp(side[i % len(side)].cuda_stream)))
+        for sd in side:
+            sd.synchronize()
     ms_host_chunked = timed(run_host_chunked, e2e_steps, 3)
 
     def run_host_percall():
@@ -376,8 +379,8 @@ def run_gpu(args):
         "e2e": {"value": round(world * bytes_step / (host_ms * 1e-3) / 1e9, 2), "unit": "GB/s",
                 "h2d_bytes_per_step": x_bytes, "d2h_bytes_per_step": y_bytes,
                 "ms_per_step": round(host_ms, 4),
-                "api": f"{n_chunks} x qift_group_forward_host (pinned host arenas in and out), one call per quarter of the "
-                       "modules, alternating between two streams so that copies overlap kernels",
+                "api": f"{n_chunks} x qift_group_forward_host (pinned host arenas in and out), one call per chunk of "
+                       f"{per} modules, dealt to {len(side)} streams so that copies overlap kernels",
                 "single_call": {"api": "1 x qift_group_forward_host on one stream", "ms_per_step": round(host_single_ms, 4),
                                 "value": round(world * bytes_step / (host_single_ms * 1e-3) / 1e9, 2)},
                 "per_call_api": {"api": "224 x qift_forward_host", "ms_per_step": round(ms_host_pc / 5, 4),

@@ -464,9 +464,13 @@ constexpr int kWideRows = 16 * kDecWarps;        // 128 rows per item with one t
 // instructions and two or more logic operations per packed word where the two-bit sets issue one; two CTAs of
 // half-size stages keep the pipes fed across each other's stage hand-overs (96 registers per thread is the limit for
 // two CTAs of nine warps).  Measured, whole steps: three-bit codes 5.89 -> 6.61 TB/s (32 LLaMA-2-7B layers, M = 1), PoT
-// 4.06 -> 4.22 (M = 1), 3.93 -> 4.04 (M = 4); the standard set 5.82 -> 5.75 at M = 4, so the others keep one CTA.
+// 4.06 -> 4.22 (M = 1), 3.93 -> 4.04 (M = 4); the standard set 5.82 -> 5.75 at M = 4, so the two-bit sets keep one CTA
+// there.  With two token tiles (9 .. 16 rows) the two-bit sets are bound by the issue of the product instructions and
+// gain as well (16 LLaMA-3.1-8B layers at 16 rows: 4.07 TB/s with 256-row items on one CTA, 4.27 with two CTAs of 128-row
+// items; 128 -> 96 registers without spills).
 __host__ __device__ constexpr int wide_ctas_per_sm(int lv, int nt, int tiles) {
-    return ((lv == QIFT_LEVELS_POT || lv == QIFT_LEVELS_INT3) && nt == 1 && tiles == 8) ? 2 : 1;
+    return (((lv == QIFT_LEVELS_POT || lv == QIFT_LEVELS_INT3) && nt == 1 && tiles == 8) ||
+            ((lv == QIFT_LEVELS_MNZ || lv == QIFT_LEVELS_SYM) && nt == 2 && tiles == 8)) ? 2 : 1;
 }
 __host__ __device__ constexpr int wide_chunk_words(int tiles, int nt, int lv = QIFT_LEVELS_MNZ) {
     // three-bit codes: a tile column is 96 bytes, not 64; two CTAs per SM: half the shared memory each

@@ -992,7 +992,9 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : 64;  // below wide_min_m there is only M = 1
     const bool use_tc = tc_rows_applies(levels, M);                  // 33 .. 64 rows (not PoT): the tcgen05 kernel, 256-row items
     if (use_tc) rows_per_item = tc_rows_per_item(M, levels);
-    if (!use_tc && rows_per_item == kWideRows && M > 8 && M <= 16 && levels != QIFT_LEVELS_POT && levels != QIFT_LEVELS_INT3) {  // PoT measured slower with two tiles
+    // (INT4 only: PoT measured slower with two tiles per warp, and the two-bit sets are faster as two CTAs per SM of 128-row
+    // items -- config 3 at 16 rows: 4.27 against 4.07 TB/s)
+    if (!use_tc && rows_per_item == kWideRows && M > 8 && M <= 16 && levels == QIFT_LEVELS_INT4) {
         long long items256 = 0;
         for (int i = 0; i < count; ++i) items256 += (problems[i].N + 2 * kWideRows - 1) / (2 * kWideRows);
         if (items256 >= 2ll * sm_count()) rows_per_item = 2 * kWideRows;

@@ -7,8 +7,8 @@
 // exist as int8 in shared memory, which a path that streams weights at the HBM rate could not afford (four
 // times the packed bytes written and read again).
 //
-//   warp 0      activation producer: per 128-byte k-block the q_a rows of all tokens, cp.async into a
-//               128-byte-swizzled K-major stage (the B operand)
+//   warp 0      activation producer: per 128-byte k-block the q_a rows of all tokens, one tensor copy (TMA, no
+//               multicast) into a 128-byte-swizzled K-major stage (the B operand)
 //   warp 1      tensor-memory allocation, tcgen05.mma issue: D[128 channels x tokens] += A(tmem) * B(smem)
 //   warps 2-5   epilogue: tcgen05.ld (lane = channel, column = token), level map with the token sums, the two
 //               scale multiplies, stores (a warp's 32 lanes write 32 consecutive channels of a token row)
@@ -24,7 +24,7 @@
 // the affine level map is undone with sum_k q as everywhere else.  The accumulators (R blocks x tokens <= 128
 // columns) are double-buffered in tensor memory: 2 x 128 columns + 8 x 32 operand columns = all 512.
 // Work items (problem, 128-channel block) are dealt round-robin to one persistent CTA per SM, as in the other
-// grouped kernels.  Every wait is bounded; no TMA multicast (no TMA at all).
+// grouped kernels.  Every wait is bounded; no TMA multicast.
 #pragma once
 
 #include "common.cuh"
@@ -132,7 +132,6 @@ linear_tc_kernel(const GroupParams gp) {
     constexpr int PER = codes_per_word(LV);
     constexpr int KPS = (PER == 16) ? 2 : 1;          // k-blocks per 16-word slice
     constexpr int ASTAGES = tc_act_stages(NTOK);
-    constexpr int LAG = ASTAGES - 3;                  // activation k-blocks in flight behind the newest
     constexpr uint32_t ACT_BYTES = NTOK * 128;
     constexpr int S = tc_acc_sets(NTOK, R);           // accumulator sets per channel block
     constexpr int DBUF = R * S * NTOK;                // accumulator columns of an item
@@ -197,41 +196,26 @@ linear_tc_kernel(const GroupParams gp) {
 
     if (warp == 0) {
         // ------------------------------------------------------------------ activation producer
+        // One tensor copy per k-block: the plan's map of the problem's q_a [M, K], box = 128 bytes of K x NTOK token rows
+        // (rows beyond M arrive as zeros), written in the 128-byte-swizzled K-major order the B descriptor reads.
         pdl_wait();
-        Cursor c;
-        c.init(table, gp.count, gp.item_first, gp.item_end, R * kTcRows);
-        // k-block `it` is copied into stage it % ASTAGES; a stage is handed to the tensor core LAG k-blocks later, once
-        // cp.async.wait_group says its copies have landed (LAG + 1 groups in flight)
-        uint32_t it = 0, done = 0;
-        auto publish = [&]() {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> tensor core
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&act_full[done % ASTAGES]);
-            ++done;
-        };
-        bool ok = true;
-        for (; c.valid() && ok; c.next()) {        // one cursor step = one slice = KPS k-blocks
-            for (int j = 0; j < KPS; ++j, ++it) {
-                const int s = it % ASTAGES;
-                if (it >= static_cast<uint32_t>(ASTAGES) && !mbar_wait(&act_empty[s], ((it / ASTAGES) - 1) & 1, 60)) {
-                    *fail = 1, ok = false;
-                    break;
-                }
-                const int8_t* src = c.q_a + static_cast<size_t>(c.chunk * KPS + j) * 128;
-                const uint32_t dst = smem_u32(act + s * ACT_BYTES);
-                for (int ch = lane; ch < M * 8; ch += 32) {
-                    const int row = ch >> 3, c16 = ch & 7;
-                    cp_async16(dst + row * 128 + ((c16 ^ (row & 7)) << 4), src + static_cast<size_t>(row) * c.K + c16 * 16);
-                }
-                cp_async_commit();
-                if (it >= static_cast<uint32_t>(LAG)) {
-                    cp_async_wait<LAG>();
-                    publish();
+        if (lane == 0) {
+            Cursor c;
+            c.init(table, gp.count, gp.item_first, gp.item_end, R * kTcRows);
+            uint32_t it = 0;
+            bool ok = true;
+            for (; c.valid() && ok; c.next()) {        // one cursor step = one slice = KPS k-blocks
+                for (int j = 0; j < KPS; ++j, ++it) {
+                    const int s = it % ASTAGES;
+                    if (it >= static_cast<uint32_t>(ASTAGES) && !mbar_wait(&act_empty[s], ((it / ASTAGES) - 1) & 1, 60)) {
+                        *fail = 1, ok = false;
+                        break;
+                    }
+                    mbar_expect_tx(&act_full[s], ACT_BYTES);
+                    tma_load_2d(act + s * ACT_BYTES, &gp.maps[c.p], (c.chunk * KPS + j) * 128, 0, &act_full[s]);
                 }
             }
         }
-        cp_async_wait<0>();
-        while (done < it) publish();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {

@@ -9,6 +9,8 @@
 // matrices; eight consumer warps do the same in-register decode + mma.sync as the per-call kernel.
 #pragma once
 
+#include <cuda.h>
+
 #include <type_traits>
 
 #include "common.cuh"
@@ -232,6 +234,7 @@ struct GroupParams {
     int M, y_bf16, stages;
     int use_single;                   // the list is the one problem below (a per-call product: no plan in memory)
     GroupProblemDev single;
+    const CUtensorMap* maps;          // tcgen05 kernel only: one tensor map per problem of the slice over its q_a
 };
 
 // CTAs per SM the kernel is compiled and launched for.  Nine warps per CTA and registers handed out

@@ -972,9 +972,15 @@ int qift_forward_multi(const void* X, int x_dtype, int M, int K, int had_block, 
 }
 
 // ------------------------------------------------------------------------------------------- grouped
+// Plan layout: header, problem records, token sums [count][kGroupMaxM], then (128-byte aligned) one tensor map per
+// problem over its q_a, which the tcgen05 kernel's activation loads use.
+static size_t plan_maps_offset(int count) {
+    const size_t o = sizeof(GroupHeader) + static_cast<size_t>(count) * (sizeof(GroupProblemDev) + kGroupMaxM * sizeof(int));
+    return (o + 127) & ~static_cast<size_t>(127);
+}
 size_t qift_group_plan_bytes(int count) {
     if (count <= 0) return 0;
-    return sizeof(GroupHeader) + static_cast<size_t>(count) * (sizeof(GroupProblemDev) + kGroupMaxM * sizeof(int));
+    return plan_maps_offset(count) + static_cast<size_t>(count) * sizeof(CUtensorMap);
 }
 
 int qift_group_plan(const qift_group_problem* problems, int count, int M, int levels, int x_dtype, int y_dtype, float clip_ratio,
@@ -987,6 +993,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     if (M > kWideMaxM && !tc_rows_applies(levels, M)) return QIFT_ERR_UNSUPPORTED_SHAPE;   // 65 .. 128 rows: the tcgen05 kernel's sets only
     if (plan_bytes < qift_group_plan_bytes(count)) return QIFT_ERR_WORKSPACE;
     if (!aligned16(plan_dev) || !aligned16(plan_host)) return QIFT_ERR_ALIGNMENT;
+    if (tc_rows_applies(levels, M) && (reinterpret_cast<uintptr_t>(plan_dev) & 127u) != 0) return QIFT_ERR_ALIGNMENT;  // tensor maps
     // Rows per work item, which also selects the kernel (dispatch_grouped): 64 / 32 for the K-split kernel, 128 for the
     // row-split kernel, 256 (two row tiles per warp, with two token tiles) when that still leaves two items per SM.
     int rows_per_item = (M >= wide_min_m(levels)) ? kWideRows : 64;  // below wide_min_m there is only M = 1
@@ -1038,8 +1045,17 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     h->q_chunk_bytes = (rows_per_item >= kWideRows) ? wide_chunk_words(rows_per_item / 16, wide_token_tiles(M), levels) * codes_per_word(levels) : 0;
     h->reserved[0] = use_tc ? 1 : 0;
     if (use_tc) h->q_chunk_bytes = 0;  // that kernel reads q_a row-major (prescaled even planes, as the K-split kernel does)
-    return cuda_status(cudaMemcpyAsync(plan_dev, plan_host, sizeof(GroupHeader) + static_cast<size_t>(count) * sizeof(GroupProblemDev),
-                                       cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));
+    cudaError_t ce = cudaMemcpyAsync(plan_dev, plan_host, sizeof(GroupHeader) + static_cast<size_t>(count) * sizeof(GroupProblemDev),
+                                     cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess || !use_tc) return cuda_status(ce);
+    // the tcgen05 kernel stages a k-block of all token rows with one tensor copy: q_a [M, K] int8, box = 128 bytes of K x its
+    // token count (rows beyond M read as zero), 128-byte swizzle -- the layout its B descriptor expects
+    CUtensorMap* maps = reinterpret_cast<CUtensorMap*>(static_cast<unsigned char*>(plan_host) + plan_maps_offset(count));
+    for (int i = 0; i < count; ++i)
+        if (!make_i8_map(&maps[i], d[i].q_a, M, d[i].K, tc_tokens(M))) return QIFT_ERR_CUDA;
+    return cuda_status(cudaMemcpyAsync(static_cast<unsigned char*>(plan_dev) + plan_maps_offset(count), maps,
+                                       static_cast<size_t>(count) * sizeof(CUtensorMap), cudaMemcpyHostToDevice,
+                                       static_cast<cudaStream_t>(stream)));
 }
 
 }  // extern "C"
@@ -1130,7 +1146,10 @@ int launch_tc(const GroupHeader* h, const GroupProblemDev* host, const GroupProb
             int grid = sm_count();
             if (grid > item_end - item_first) grid = item_end - item_first;
             GroupParams gp{dev + first, sumq, first, count, item_first, item_end, h->M, h->y_bf16, 0, 0, {}};
-            if (single) gp.use_single = 1, gp.single = host[0];
+            if (single) return QIFT_ERR_INVALID_ARG;   // the kernel needs the plan's tensor maps
+            // dev points just behind the header of the device plan: the maps follow the token sums
+            const unsigned char* plan_dev = reinterpret_cast<const unsigned char*>(dev) - sizeof(GroupHeader);
+            gp.maps = reinterpret_cast<const CUtensorMap*>(plan_dev + plan_maps_offset(h->count)) + first;
             const int rc = cuda_status(launch_pdl(kernel, dim3(grid), dim3(kTcThreads), smem, st, gp));
             if (rc != QIFT_OK) return rc;
         }

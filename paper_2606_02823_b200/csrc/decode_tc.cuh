@@ -218,10 +218,17 @@ linear_tc_kernel(const GroupParams gp) {
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
+        // One thread issues every instruction of the CTA's tensor core, so the loop is kept short: a lone thread retires a
+        // dependent instruction every few cycles, and at 64 tokens a first version of this loop (indices by division,
+        // descriptors rebuilt per k-block, the cursor stepped chunk by chunk) took 440 cycles per 128-channel k-block
+        // against 200 of tensor time.
         if (lane == 0) {
             Cursor c;
             c.init(table, gp.count, gp.item_first, gp.item_end, R * kTcRows);
-            uint32_t it = 0, icount = 0;   // k-blocks, items
+            uint32_t icount = 0;
+            uint32_t sb = 0, sb_par = 0;        // activation stage of the next k-block, parity of its fill
+            uint32_t slot = 0, slot_par = 0;    // operand-ring slot of the next k-block's first tile (R divides the ring), parity
+            const uint64_t desc0 = make_kmajor_sw128_desc(smem_u32(act));
             bool ok = true;
             while (c.valid() && ok) {
                 const int buf = icount & 1;
@@ -232,43 +239,43 @@ linear_tc_kernel(const GroupParams gp) {
                 tc_fence_after();
                 const int kblocks = c.nchunks * KPS;
                 const int tiles = (c.tiles_valid + 7) >> 3;   // 128-channel tiles of the item that exist
-                for (int kb = 0; kb < kblocks; ++kb, ++it) {
-                    const int sb = it % ASTAGES;
-                    if (!mbar_wait(&act_full[sb], (it / ASTAGES) & 1, 63)) {
+                const uint32_t d_base = tmem_base + buf * DBUF;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(&act_full[sb], sb_par, 63)) {
                         *fail = 1, ok = false;
                         break;
                     }
-                    const uint64_t bdesc = make_kmajor_sw128_desc(smem_u32(act + sb * ACT_BYTES));
 #pragma unroll
                     for (int r = 0; r < R; ++r) {
-                        const uint32_t ia = it * R + r;
-                        if (!mbar_wait(&a_full[ia % kTcARing], (ia / kTcARing) & 1, 62)) {
+                        if (!mbar_wait(&a_full[slot + r], slot_par, 62)) {
                             *fail = 1, ok = false;
                             break;
                         }
                     }
                     if (!ok) break;
                     tc_fence_after();
+                    const uint64_t bdesc = desc0 + sb * (ACT_BYTES >> 4);
+                    const uint32_t a_base = tmem_base + kTcACol0 + slot * 32;
 #pragma unroll
                     for (int k4 = 0; k4 < 4; ++k4) {   // step-major: consecutive instructions write different accumulators
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
-                            if (r < tiles) {
-                                const uint32_t a_addr = tmem_base + kTcACol0 + ((it * R + r) % kTcARing) * 32 + 8 * k4;
-                                const uint32_t d_addr = tmem_base + buf * DBUF + (r * S + (k4 % S)) * NTOK;
-                                tc_mma_i8_ts(d_addr, a_addr, bdesc + 2 * k4, IDESC, (kb != 0 || k4 >= S) ? 1u : 0u);
-                            }
+                            if (r < tiles)
+                                tc_mma_i8_ts(d_base + (r * S + (k4 % S)) * NTOK, a_base + r * 32 + 8 * k4, bdesc + 2 * k4, IDESC,
+                                             (kb != 0 || k4 >= S) ? 1u : 0u);
                         }
                     }
 #pragma unroll
-                    for (int r = 0; r < R; ++r) tc_commit(&a_empty[(it * R + r) % kTcARing]);
-                    if (!ok) break;
+                    for (int r = 0; r < R; ++r) tc_commit(&a_empty[slot + r]);
                     tc_commit(&act_empty[sb]);
+                    if (++sb == ASTAGES) sb = 0, sb_par ^= 1;
+                    slot += R;
+                    if (slot == kTcARing) slot = 0, slot_par ^= 1;
                 }
                 if (!ok) break;
                 tc_commit(&d_full[buf]);
                 ++icount;
-                for (int j = c.nchunks; j > 0; --j) c.next();  // to the CTA's next item
+                c.next_item();
             }
         }
     } else if (warp < 6) {
@@ -324,7 +331,7 @@ linear_tc_kernel(const GroupParams gp) {
             __syncwarp();
             if (lane == 0) mbar_arrive(&d_empty[buf]);
             ++icount;
-            for (int j = c.nchunks; j > 0; --j) c.next();
+            c.next_item();
         }
     } else {
         // ------------------------------------------------------------------ expander warps

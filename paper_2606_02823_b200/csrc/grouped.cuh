@@ -211,6 +211,11 @@ struct GroupCursor {
             load_item();
         }
     }
+    __device__ __forceinline__ void next_item() {   // from any chunk of the item
+        chunk = 0;
+        item += gridDim.x;
+        load_item();
+    }
 };
 
 // Cross-warp reduction buffer: [warp][row tile][accumulator set][token][row], only the M live columns.

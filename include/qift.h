@@ -275,8 +275,8 @@ int qift_linear_multi(const int8_t* q_a, const float* s_a, int M, int K, int lev
  * kernel streams the whole list back to back.  (No counterpart in the paper: it describes no kernels.)
  *
  * qift_group_plan validates the list and writes a plan into caller memory: `plan_host` (host) and
- * `plan_dev` (device), each qift_group_plan_bytes(count) bytes; the device copy is enqueued on
- * `stream`.  The plan holds the caller's pointers, so it stays valid while those buffers live;
+ * `plan_dev` (device, 128-byte aligned: plans of 33 .. 128 rows keep one tensor map per problem in it), each
+ * qift_group_plan_bytes(count) bytes; the device copy is enqueued on `stream`.  The plan holds the caller's pointers, so it stays valid while those buffers live;
  * plan_host must stay alive and unchanged while the plan is used.  The run calls enqueue
  *   qift_group_quantize_act : S2+S3 for every problem (one launch)  X -> q_a, s_a
  *   qift_group_linear       : S4+S5 for every problem (one launch per 256 problems)  q_a, s_a -> Y;

@@ -102,6 +102,31 @@ def test_config3_llama31_batched_decode(shape_idx):
     clean()
 
 
+@pytest.mark.parametrize("M", [64, 128])
+def test_config3_shapes_grouped_plan_mid_m_bf16(M):
+    # the launch configuration of the benchmark's mid_m block: LLaMA-3.1-8B shapes in one grouped plan, bf16 in and
+    # out, 64 / 128 token rows (the tcgen05 weight-streaming kernel); q/o, k/v shapes whole, gate/up and down cut to
+    # 1024 channels so that the oracle stays in seconds
+    shapes = [(4096, 4096), (1024, 4096), (1024, 4096), (1024, 14336)]
+    probs, refs = [], []
+    for i, (N, K) in enumerate(shapes):
+        W = synth.gaussian_weights(synth.config_seed(3, i, 0) + 7, N, K)
+        x, _ = synth.activations(synth.config_seed(3, i, 1) + 7, M, K, round(0.01 * K))
+        xd = dev(x).to(torch.bfloat16)
+        x_ref = oracle.bf16_to_f32(xd.view(torch.int16).cpu().numpy().view(np.uint16))
+        B = synth.had_block_for(K)
+        p_ref, s_n, codes = oracle.pack_weights(W, oracle.MNZ, oracle.SCALE_ABSMAX)
+        q_ref, sa_ref = oracle.quantize_act(x_ref, B, CLIP)
+        refs.append(oracle.linear(codes, oracle.MNZ, s_n, q_ref, sa_ref, bf16=True))
+        probs.append((xd, dev(p_ref.view(np.int32)), dev(s_n), B))
+    plan = qift.qift_group_plan(probs, qift.MNZ, CLIP, out_dtype=torch.bfloat16, want_acc=True)
+    outs = qift.qift_group_forward(plan)
+    clean()
+    for (y_ref, acc_ref), y, acc in zip(refs, outs, plan.accs):
+        assert np.array_equal(acc.cpu().numpy(), acc_ref)
+        assert np.array_equal(y.view(torch.int16).cpu().numpy().view(np.uint16), y_ref)
+
+
 # ---------------------------------------------------------------------------------------- config 4
 @pytest.mark.parametrize("shape_idx", [0, 1, 4, 6])
 def test_config4_prefill_m2048_sampled(shape_idx):

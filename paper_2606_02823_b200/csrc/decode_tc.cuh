@@ -10,6 +10,10 @@
 //   warp 0      activation producer: per 128-byte k-block the q_a rows of all tokens, one tensor copy (TMA, no
 //               multicast) into a 128-byte-swizzled K-major stage (the B operand)
 //   warp 1      tensor-memory allocation, tcgen05.mma issue: D[128 channels x tokens] += A(tmem) * B(smem)
+//   warp 14     second issuer.  A thread issues a tcgen05 instruction every ~50 cycles at best (the measured 26 ns per
+//               128 x N x 32 instruction for N <= 64 is this issue cost, not tensor time), so the (k-block, tile) units are
+//               dealt alternately to two threads.  Integer accumulation commutes and every instruction accumulates
+//               (the epilogue leaves the accumulator columns zeroed), so the two streams need no order between them.
 //   warps 2-5   epilogue: tcgen05.ld (lane = channel, column = token), level map with the token sums, the two
 //               scale multiplies, stores (a warp's 32 lanes write 32 consecutive channels of a token row)
 //   warps 6-13  expanders, two per tensor-memory lane quarter (alternate 16-word slices): each streams the packed
@@ -35,7 +39,8 @@ namespace qift {
 
 constexpr int kTcRows = 128;       // channels per work item
 constexpr int kTcExpanders = 8;    // expander warps: two per tensor-memory lane quarter
-constexpr int kTcThreads = 32 * (6 + kTcExpanders);
+constexpr int kTcIssuers = 2;     // threads that issue tensor-core instructions (warp 1 and the last warp)
+constexpr int kTcThreads = 32 * (6 + kTcExpanders + 1);
 constexpr int kTcSlotBytes = 32 * 64;   // a packed unit: 32 rows x 64 bytes, 16-byte chunks XOR-swizzled by row
 // packed units in flight per expander warp (what is left of shared memory beside the activation ring)
 __host__ __device__ constexpr int tc_wslots(int ntok) { return ntok <= 32 ? 8 : ntok <= 64 ? 6 : 4; }
@@ -164,14 +169,14 @@ linear_tc_kernel(const GroupParams gp) {
     if (tid == 0) {
         for (int s = 0; s < ASTAGES; ++s) {
             mbar_init(&act_full[s], 1);
-            mbar_init(&act_empty[s], 1);
+            mbar_init(&act_empty[s], R >= 2 ? kTcIssuers : 1);   // tcgen05.commit of every issuer with a unit in the k-block
         }
         for (int s = 0; s < kTcARing; ++s) {
             mbar_init(&a_full[s], 4);   // one arrival per lane quarter
             mbar_init(&a_empty[s], 1);  // tcgen05.commit
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(&d_full[b], 1);
+            mbar_init(&d_full[b], kTcIssuers);
             mbar_init(&d_empty[b], 4);  // the four epilogue warps
         }
         *fail = 0;
@@ -216,23 +221,23 @@ linear_tc_kernel(const GroupParams gp) {
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        // One thread issues every instruction of the CTA's tensor core, so the loop is kept short: a lone thread retires a
-        // dependent instruction every few cycles, and at 64 tokens a first version of this loop (indices by division,
-        // descriptors rebuilt per k-block, the cursor stepped chunk by chunk) took 440 cycles per 128-channel k-block
-        // against 200 of tensor time.
+    } else if (warp == 1 || warp == 6 + kTcExpanders) {
+        // ------------------------------------------------------------------ MMA issuers
+        // Unit u = (k-block, tile) in running order goes to issuer u mod 2: with two tiles per item each issuer owns a
+        // tile, with one it takes every other k-block.  One thread per issuer; the loop is kept short (a lone thread
+        // retires a dependent instruction every few cycles).
         if (lane == 0) {
+            const uint32_t me = (warp == 1) ? 0u : 1u;
             Cursor c;
             c.init(table, gp.count, gp.item_first, gp.item_end, R * kTcRows);
-            uint32_t icount = 0;
+            uint32_t icount = 0, it = 0;        // items, k-blocks (running)
             uint32_t sb = 0, sb_par = 0;        // activation stage of the next k-block, parity of its fill
             uint32_t slot = 0, slot_par = 0;    // operand-ring slot of the next k-block's first tile (R divides the ring), parity
             const uint64_t desc0 = make_kmajor_sw128_desc(smem_u32(act));
             bool ok = true;
             while (c.valid() && ok) {
                 const int buf = icount & 1;
-                if (icount >= 2 && !mbar_wait(&d_empty[buf], ((icount >> 1) - 1) & 1, 61)) {
+                if (!mbar_wait(&d_empty[buf], (icount >> 1) & 1, 61)) {   // zeroed by the epilogue (first use: at start)
                     *fail = 1;
                     break;
                 }
@@ -240,34 +245,33 @@ linear_tc_kernel(const GroupParams gp) {
                 const int kblocks = c.nchunks * KPS;
                 const int tiles = (c.tiles_valid + 7) >> 3;   // 128-channel tiles of the item that exist
                 const uint32_t d_base = tmem_base + buf * DBUF;
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!mbar_wait(&act_full[sb], sb_par, 63)) {
-                        *fail = 1, ok = false;
-                        break;
-                    }
-#pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        if (!mbar_wait(&a_full[slot + r], slot_par, 62)) {
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const bool mine = (R >= 2) || ((it & 1u) == me);
+                    if (mine) {
+                        if (!mbar_wait(&act_full[sb], sb_par, 63)) {
                             *fail = 1, ok = false;
                             break;
                         }
-                    }
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint64_t bdesc = desc0 + sb * (ACT_BYTES >> 4);
-                    const uint32_t a_base = tmem_base + kTcACol0 + slot * 32;
-#pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4) {   // step-major: consecutive instructions write different accumulators
+                        const uint64_t bdesc = desc0 + sb * (ACT_BYTES >> 4);
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
-                            if (r < tiles)
-                                tc_mma_i8_ts(d_base + (r * S + (k4 % S)) * NTOK, a_base + r * 32 + 8 * k4, bdesc + 2 * k4, IDESC,
-                                             (kb != 0 || k4 >= S) ? 1u : 0u);
-                        }
-                    }
+                            if (R >= 2 && (static_cast<uint32_t>(r) & 1u) != me) continue;
+                            if (!mbar_wait(&a_full[slot + r], slot_par, 62)) {
+                                *fail = 1, ok = false;
+                                break;
+                            }
+                            tc_fence_after();
+                            if (r < tiles) {
+                                const uint32_t a_base = tmem_base + kTcACol0 + (slot + r) * 32;
 #pragma unroll
-                    for (int r = 0; r < R; ++r) tc_commit(&a_empty[slot + r]);
-                    tc_commit(&act_empty[sb]);
+                                for (int k4 = 0; k4 < 4; ++k4)
+                                    tc_mma_i8_ts(d_base + (r * S + (k4 % S)) * NTOK, a_base + 8 * k4, bdesc + 2 * k4, IDESC, 1u);
+                            }
+                            tc_commit(&a_empty[slot + r]);
+                        }
+                        if (!ok) break;
+                        tc_commit(&act_empty[sb]);
+                    }
                     if (++sb == ASTAGES) sb = 0, sb_par ^= 1;
                     slot += R;
                     if (slot == kTcARing) slot = 0, slot_par ^= 1;
@@ -280,8 +284,24 @@ linear_tc_kernel(const GroupParams gp) {
         }
     } else if (warp < 6) {
         // ------------------------------------------------------------------ epilogue warps
-        pdl_wait();
         const int quarter = warp & 3;
+        // every tensor-core instruction accumulates: both accumulator buffers start zeroed, and each is zeroed again by
+        // the warp that has read it
+        auto zero_acc = [&](int buf) {
+            uint32_t z[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) z[j] = 0u;
+#pragma unroll
+            for (int col = 0; col < DBUF; col += 32)
+                tc_st32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * DBUF + col, z);
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&d_empty[buf]);
+        };
+        zero_acc(0);
+        zero_acc(1);
+        pdl_wait();
         Cursor c;
         c.init(table, gp.count, gp.item_first, gp.item_end, R * kTcRows);
         uint32_t icount = 0;
@@ -327,13 +347,11 @@ linear_tc_kernel(const GroupParams gp) {
                     }
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&d_empty[buf]);
+            zero_acc(buf);
             ++icount;
             c.next_item();
         }
-    } else {
+    } else if (warp < 6 + kTcExpanders) {
         // ------------------------------------------------------------------ expander warps
         // Two warps per lane quarter; warp (q, ph) takes the slices whose running number has parity ph.  A unit =
         // one slice of one tile of the item (its 32 rows x 64 bytes); units are fetched kTcWSlots ahead.

@@ -39,8 +39,8 @@ namespace qift {
 
 constexpr int kTcRows = 128;       // channels per work item
 constexpr int kTcExpanders = 8;    // expander warps: two per tensor-memory lane quarter
-constexpr int kTcIssuers = 2;     // threads that issue tensor-core instructions (warp 1 and the last warp)
-constexpr int kTcThreads = 32 * (6 + kTcExpanders + 1);
+constexpr int kTcIssuers = 4;     // threads that issue tensor-core instructions (warp 1 and the last warps)
+constexpr int kTcThreads = 32 * (6 + kTcExpanders + kTcIssuers - 1);
 constexpr int kTcSlotBytes = 32 * 64;   // a packed unit: 32 rows x 64 bytes, 16-byte chunks XOR-swizzled by row
 // packed units in flight per expander warp (what is left of shared memory beside the activation ring)
 __host__ __device__ constexpr int tc_wslots(int ntok) { return ntok <= 32 ? 8 : ntok <= 64 ? 6 : 4; }
@@ -169,7 +169,7 @@ linear_tc_kernel(const GroupParams gp) {
     if (tid == 0) {
         for (int s = 0; s < ASTAGES; ++s) {
             mbar_init(&act_full[s], 1);
-            mbar_init(&act_empty[s], R >= 2 ? kTcIssuers : 1);   // tcgen05.commit of every issuer with a unit in the k-block
+            mbar_init(&act_empty[s], R < kTcIssuers ? R : kTcIssuers);   // tcgen05.commit of every issuer with a unit in the k-block
         }
         for (int s = 0; s < kTcARing; ++s) {
             mbar_init(&a_full[s], 4);   // one arrival per lane quarter
@@ -221,13 +221,13 @@ linear_tc_kernel(const GroupParams gp) {
                 }
             }
         }
-    } else if (warp == 1 || warp == 6 + kTcExpanders) {
+    } else if (warp == 1 || warp >= 6 + kTcExpanders) {
         // ------------------------------------------------------------------ MMA issuers
         // Unit u = (k-block, tile) in running order goes to issuer u mod 2: with two tiles per item each issuer owns a
         // tile, with one it takes every other k-block.  One thread per issuer; the loop is kept short (a lone thread
         // retires a dependent instruction every few cycles).
         if (lane == 0) {
-            const uint32_t me = (warp == 1) ? 0u : 1u;
+            const uint32_t me = (warp == 1) ? 0u : static_cast<uint32_t>(warp - (6 + kTcExpanders) + 1);
             Cursor c;
             c.init(table, gp.count, gp.item_first, gp.item_end, R * kTcRows);
             uint32_t icount = 0, it = 0;        // items, k-blocks (running)
@@ -246,32 +246,34 @@ linear_tc_kernel(const GroupParams gp) {
                 const int tiles = (c.tiles_valid + 7) >> 3;   // 128-channel tiles of the item that exist
                 const uint32_t d_base = tmem_base + buf * DBUF;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
-                    const bool mine = (R >= 2) || ((it & 1u) == me);
-                    if (mine) {
-                        if (!mbar_wait(&act_full[sb], sb_par, 63)) {
-                            *fail = 1, ok = false;
-                            break;
-                        }
-                        const uint64_t bdesc = desc0 + sb * (ACT_BYTES >> 4);
+                    bool any = false;
+                    uint64_t bdesc = 0;
 #pragma unroll
-                        for (int r = 0; r < R; ++r) {
-                            if (R >= 2 && (static_cast<uint32_t>(r) & 1u) != me) continue;
-                            if (!mbar_wait(&a_full[slot + r], slot_par, 62)) {
+                    for (int r = 0; r < R; ++r) {
+                        if (((it * R + r) & (kTcIssuers - 1)) != me) continue;   // unit (k-block, tile) -> issuer, round robin
+                        if (!any) {
+                            if (!mbar_wait(&act_full[sb], sb_par, 63)) {
                                 *fail = 1, ok = false;
                                 break;
                             }
-                            tc_fence_after();
-                            if (r < tiles) {
-                                const uint32_t a_base = tmem_base + kTcACol0 + (slot + r) * 32;
-#pragma unroll
-                                for (int k4 = 0; k4 < 4; ++k4)
-                                    tc_mma_i8_ts(d_base + (r * S + (k4 % S)) * NTOK, a_base + 8 * k4, bdesc + 2 * k4, IDESC, 1u);
-                            }
-                            tc_commit(&a_empty[slot + r]);
+                            bdesc = desc0 + sb * (ACT_BYTES >> 4);
+                            any = true;
                         }
-                        if (!ok) break;
-                        tc_commit(&act_empty[sb]);
+                        if (!mbar_wait(&a_full[slot + r], slot_par, 62)) {
+                            *fail = 1, ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        if (r < tiles) {
+                            const uint32_t a_base = tmem_base + kTcACol0 + (slot + r) * 32;
+#pragma unroll
+                            for (int k4 = 0; k4 < 4; ++k4)
+                                tc_mma_i8_ts(d_base + (r * S + (k4 % S)) * NTOK, a_base + 8 * k4, bdesc + 2 * k4, IDESC, 1u);
+                        }
+                        tc_commit(&a_empty[slot + r]);
                     }
+                    if (!ok) break;
+                    if (any) tc_commit(&act_empty[sb]);
                     if (++sb == ASTAGES) sb = 0, sb_par ^= 1;
                     slot += R;
                     if (slot == kTcARing) slot = 0, slot_par ^= 1;

@@ -324,6 +324,24 @@ linear_tc_kernel(const GroupParams gp) {
                 for (int m0 = 0; m0 < M; m0 += 16) {
                     uint32_t v[16];
                     tc_ld16(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * DBUF + r * S * NTOK + m0, v);
+                    // the token sums and token scales of these sixteen rows, fetched while the accumulators are on their way
+                    int sq[16];
+                    float sa[16];
+                    if (m0 + 16 <= M) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int4 a = __ldg(reinterpret_cast<const int4*>(sumq + m0) + j);
+                            const float4 b = __ldg(reinterpret_cast<const float4*>(P.s_a + m0) + j);
+                            sq[4 * j] = a.x, sq[4 * j + 1] = a.y, sq[4 * j + 2] = a.z, sq[4 * j + 3] = a.w;
+                            sa[4 * j] = b.x, sa[4 * j + 1] = b.y, sa[4 * j + 2] = b.z, sa[4 * j + 3] = b.w;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int m = min(m0 + j, M - 1);
+                            sq[j] = __ldg(sumq + m), sa[j] = __ldg(P.s_a + m);
+                        }
+                    }
                     tc_wait_ld();
 #pragma unroll
                     for (int st = 1; st < S; ++st) {
@@ -334,13 +352,12 @@ linear_tc_kernel(const GroupParams gp) {
                         for (int j = 0; j < 16; ++j) v[j] += u[j];
                     }
                     if (n < P.N) {
+                        size_t o = static_cast<size_t>(m0) * P.N + n;
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int m = m0 + j;
-                            if (m < M) {
-                                const int acc = tc_level_sum<LV>(static_cast<int>(v[j]), __ldg(sumq + m));
-                                const float y = scale_epilogue(acc, __ldg(P.s_a + m), sn);
-                                const size_t o = static_cast<size_t>(m) * P.N + n;
+                        for (int j = 0; j < 16; ++j, o += P.N) {
+                            if (m0 + j < M) {
+                                const int acc = tc_level_sum<LV>(static_cast<int>(v[j]), sq[j]);
+                                const float y = scale_epilogue(acc, sa[j], sn);
                                 if (gp.y_bf16) static_cast<uint16_t*>(P.Y)[o] = f32_to_bf16_bits(y);
                                 else static_cast<float*>(P.Y)[o] = y;
                                 if (P.acc_debug) P.acc_debug[o] = acc;

@@ -39,8 +39,9 @@ namespace qift {
 
 constexpr int kTcRows = 128;       // channels per work item
 constexpr int kTcExpanders = 8;    // expander warps: two per tensor-memory lane quarter
-constexpr int kTcIssuers = 4;     // threads that issue tensor-core instructions (warp 1 and the last warps)
-constexpr int kTcThreads = 32 * (6 + kTcExpanders + kTcIssuers - 1);
+constexpr int kTcIssuers = 2;     // threads that issue tensor-core instructions (warp 1 and warp 14)
+constexpr int kTcEpiGroups = 2;   // epilogue warps per tensor-memory lane quarter (warps 2-5 and 15-18), alternate 16-token chunks
+constexpr int kTcThreads = 32 * (6 + kTcExpanders + (kTcIssuers - 1) + 4 * (kTcEpiGroups - 1));
 constexpr int kTcSlotBytes = 32 * 64;   // a packed unit: 32 rows x 64 bytes, 16-byte chunks XOR-swizzled by row
 // packed units in flight per expander warp (what is left of shared memory beside the activation ring)
 __host__ __device__ constexpr int tc_wslots(int ntok) { return ntok <= 32 ? 8 : ntok <= 64 ? 6 : 4; }
@@ -73,6 +74,11 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&v)[32])
         "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]),
         "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]),
         "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tc_zero16(uint32_t taddr) {   // sixteen columns of the warp's 32 lanes <- 0
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};" ::"r"(taddr), "r"(0u)
         : "memory");
 }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -177,7 +183,7 @@ linear_tc_kernel(const GroupParams gp) {
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&d_full[b], kTcIssuers);
-            mbar_init(&d_empty[b], 4);  // the four epilogue warps
+            mbar_init(&d_empty[b], 4 * kTcEpiGroups);  // the epilogue warps
         }
         *fail = 0;
         mbar_fence_init();
@@ -221,7 +227,7 @@ linear_tc_kernel(const GroupParams gp) {
                 }
             }
         }
-    } else if (warp == 1 || warp >= 6 + kTcExpanders) {
+    } else if (warp == 1 || (warp >= 6 + kTcExpanders && warp < 6 + kTcExpanders + kTcIssuers - 1)) {
         // ------------------------------------------------------------------ MMA issuers
         // Unit u = (k-block, tile) in running order goes to issuer u mod 2: with two tiles per item each issuer owns a
         // tile, with one it takes every other k-block.  One thread per issuer; the loop is kept short (a lone thread
@@ -284,18 +290,17 @@ linear_tc_kernel(const GroupParams gp) {
                 c.next_item();
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 6 || warp >= 6 + kTcExpanders + kTcIssuers - 1) {
         // ------------------------------------------------------------------ epilogue warps
+        const int eg = (warp < 6) ? 0 : 1;   // this warp's 16-token chunks: eg, eg + kTcEpiGroups, ...
         const int quarter = warp & 3;
         // every tensor-core instruction accumulates: both accumulator buffers start zeroed, and each is zeroed again by
         // the warp that has read it
-        auto zero_acc = [&](int buf) {
-            uint32_t z[32];
+        auto zero_acc = [&](int buf) {   // the chunks this warp reads, in every accumulator set of every tile
 #pragma unroll
-            for (int j = 0; j < 32; ++j) z[j] = 0u;
-#pragma unroll
-            for (int col = 0; col < DBUF; col += 32)
-                tc_st32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * DBUF + col, z);
+            for (int col = 0; col < R * S * NTOK; col += NTOK)
+                for (int m0 = 16 * eg; m0 < NTOK; m0 += 16 * kTcEpiGroups)
+                    tc_zero16(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * DBUF + col + m0);
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
@@ -321,7 +326,7 @@ linear_tc_kernel(const GroupParams gp) {
                 const int n = c.n0 + r * kTcRows + quarter * 32 + lane;
                 if (c.n0 + r * kTcRows >= P.N) break;   // (uniform) this tile of the item does not exist
                 const float sn = (n < P.N) ? __ldg(P.s_n + n) : 0.0f;
-                for (int m0 = 0; m0 < M; m0 += 16) {
+                for (int m0 = 16 * eg; m0 < M; m0 += 16 * kTcEpiGroups) {
                     uint32_t v[16];
                     tc_ld16(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * DBUF + r * S * NTOK + m0, v);
                     // the token sums and token scales of these sixteen rows, fetched while the accumulators are on their way

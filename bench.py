@@ -424,10 +424,12 @@ LAYER_CALLS = (("q", "k", "v"), ("o",), ("gate", "up"), ("down",))
 
 class LayerChain:
     """Runs a stack of layers (each: the seven modules of build_stack, in order) through qift_forward_multi /
-    qift_linear_multi: per layer four calls -- q/k/v on one activation, o, gate/up on one activation, down -- each
-    decoding the NEXT call's packed codes into the other of two int8 level buffers while its own GEMM runs.  The
-    chain is circular (the last call of the stack decodes the first call's codes), as in a prefill loop over
-    requests; the buffers are primed by one untimed pass."""
+    qift_linear_multi: per layer four calls -- q/k/v on one activation, o, gate/up on one activation, down.  The packed
+    codes of a call are decoded into its int8 levels buffer by the side warps of an EARLIER call's GEMM; the long
+    products carry that work: gate/up decodes down of its own layer and q/k/v + o of the next, down decodes gate/up of the
+    next layer, the two short calls decode nothing.  A buffer is written at most three calls before it is read, so a ring
+    of eight buffers (one per call of two layers) is never overwritten early.  The chain is circular (the last layer
+    decodes for the first), as in a prefill loop over requests; the buffers are primed by one untimed pass."""
 
     def __init__(self, torch, qift, L, mods, M, y_dtype):
         from paper_2606_02823_b200 import binding
@@ -441,23 +443,33 @@ class LayerChain:
                 for i, m in enumerate(ms):
                     arr[i] = binding.LinearOutput(m.packed.data_ptr(), m.s_n.data_ptr(), m.y.data_ptr(), None, m.N, 0)
                 self.calls.append({"x": ms[0].x, "K": ms[0].K, "B": ms[0].B, "levels": ms[0].levels, "arr": arr, "n": len(ms)})
-        vp = ctypes.c_void_p
         self.lev_bytes = max(int(L.qift_levels_bytes(c["K"], ctypes.addressof(c["arr"]), c["n"])) for c in self.calls)
         self.scr_bytes = max(int(L.qift_forward_multi_scratch_bytes(M, c["K"], c["levels"], ctypes.addressof(c["arr"]), c["n"]))
                              for c in self.calls)
         dev = mods[0].x.device
-        self.lev = [torch.empty(self.lev_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
+        n = len(self.calls)
+        assert n % 4 == 0
+        self.ring = 8 if n % 8 == 0 else n          # buffers in rotation (a whole number of rings per pass)
+        self.lev = [torch.empty(self.lev_bytes, dtype=torch.uint8, device=dev) for _ in range(self.ring)]
         self.scr = torch.empty(self.scr_bytes, dtype=torch.uint8, device=dev)
         kmax = max(c["K"] for c in self.calls)
         self.q_a = torch.randint(-8, 8, (M, kmax), dtype=torch.int8, device=dev)   # for the product-only timing
         self.s_a = torch.full((M,), 0.01, dtype=torch.float32, device=dev)
-        self.ahead = []
-        n = len(self.calls)
-        assert n % 2 == 0
-        for i, c in enumerate(self.calls):
-            nx = self.calls[(i + 1) % n]
-            self.ahead.append(binding.DecodeAhead(ctypes.addressof(nx["arr"]), nx["n"], nx["K"], nx["levels"], 0,
-                                                  self.lev[(i + 1) & 1].data_ptr(), self.lev_bytes))
+        # who decodes for whom: call index within the layer -> later calls (offsets in calls) it decodes for
+        carry = {0: [], 1: [], 2: [1, 2, 3], 3: [3]}      # gate/up: down (+1), next q/k/v (+2), next o (+3); down: next gate/up (+3)
+        self.decoded_by = {}                               # call -> the call that decodes for it
+        self.ahead, self.keep = [], []
+        for i in range(n):
+            nxt = None
+            for off in reversed(carry[i % 4]):
+                j = (i + off) % n
+                self.decoded_by[j] = i
+                tgt = self.calls[j]
+                d = binding.DecodeAhead(ctypes.addressof(tgt["arr"]), tgt["n"], tgt["K"], tgt["levels"], 0,
+                                        self.lev[j % self.ring].data_ptr(), self.lev_bytes, nxt)
+                self.keep.append(d)
+                nxt = ctypes.addressof(d)
+            self.ahead.append(nxt)
         self.y_dtype = qift.BF16 if y_dtype == torch.bfloat16 else qift.F32
         self.x_dtype = qift.BF16 if mods[0].x.dtype == torch.bfloat16 else qift.F32
         self.primed = False
@@ -466,16 +478,17 @@ class LayerChain:
         vp, L, M = ctypes.c_void_p, self.L, self.M
         st = vp(self.torch.cuda.current_stream().cuda_stream)
         for i, c in enumerate(self.calls):
-            ready = 1 if (self.primed or i > 0) else 0
-            lev = self.lev[i & 1]
+            # levels are there if an earlier call of this pass, or (once primed) of the previous pass, decoded them
+            ready = 1 if (self.primed or self.decoded_by[i] < i) else 0
+            lev = self.lev[i % self.ring]
             if with_quant:
                 rc = L.qift_forward_multi(vp(c["x"].data_ptr()), self.x_dtype, M, c["K"], c["B"], CLIP, c["levels"],
                                           ctypes.addressof(c["arr"]), c["n"], self.y_dtype, vp(self.scr.data_ptr()), self.scr_bytes,
-                                          vp(lev.data_ptr()), self.lev_bytes, ready, ctypes.addressof(self.ahead[i]), st)
+                                          vp(lev.data_ptr()), self.lev_bytes, ready, self.ahead[i], st)
             else:
                 rc = L.qift_linear_multi(vp(self.q_a.data_ptr()), vp(self.s_a.data_ptr()), M, c["K"], c["levels"],
                                          ctypes.addressof(c["arr"]), c["n"], self.y_dtype, None, 0, vp(lev.data_ptr()),
-                                         self.lev_bytes, ready, ctypes.addressof(self.ahead[i]), st)
+                                         self.lev_bytes, ready, self.ahead[i], st)
             assert rc == 0, rc
         self.primed = True
         return len(self.calls)

@@ -225,6 +225,9 @@ int qift_forward_host(const void* X_host, int x_dtype, int M, int K, int had_blo
  * the buffer that call will pass as its levels_buf; the next call then passes levels_ready = 1 and skips its
  * own decoding pass.  A caller walking a layer stack alternates two levels buffers.  The first call of a
  * chain (levels_ready = 0) decodes its own codes before its GEMM, as qift_w2a4_linear does.
+ * `ahead` is a list (`next`): a call may decode for several later calls, each into that call's own buffer, so that
+ * a long product (gate / up, down) carries the decoding for the short ones (q / k / v, o) of the next layer as well;
+ * the caller then keeps as many levels buffers as calls lie between a decoding and its use.
  *
  *   X            dev [M,K] fp32 or bf16;  had_block, clip_ratio as for qift_quantize_act
  *   outputs      HOST array of 1..4 outputs: packed / s_n from qift_pack_weights (all with this K and
@@ -247,11 +250,13 @@ typedef struct qift_linear_output {
     int reserved;
 } qift_linear_output;
 typedef struct qift_decode_ahead {
-    const qift_linear_output* outputs; /* host; the next call's outputs (packed and N are read) */
+    const qift_linear_output* outputs; /* host; a later call's outputs (packed and N are read)  */
     int count, K, levels;
     int reserved;
-    void* levels_buf;                  /* dev; the next call's levels_buf                        */
+    void* levels_buf;                  /* dev; that call's levels_buf                            */
     size_t levels_bytes;
+    const struct qift_decode_ahead* next; /* host; another later call to decode for, or NULL (at most 8 outputs over
+                                             the whole chain)                                    */
 } qift_decode_ahead;
 size_t qift_levels_bytes(int K, const qift_linear_output* outputs, int count);
 size_t qift_forward_multi_scratch_bytes(int M, int K, int levels, const qift_linear_output* outputs, int count);

@@ -300,7 +300,23 @@ class LinearOutput(ctypes.Structure):
 class DecodeAhead(ctypes.Structure):
     """Mirror of qift_decode_ahead."""
     _fields_ = [("outputs", ctypes.c_void_p), ("count", ctypes.c_int), ("K", ctypes.c_int), ("levels", ctypes.c_int),
-                ("reserved", ctypes.c_int), ("levels_buf", ctypes.c_void_p), ("levels_bytes", ctypes.c_size_t)]
+                ("reserved", ctypes.c_int), ("levels_buf", ctypes.c_void_p), ("levels_bytes", ctypes.c_size_t),
+                ("next", ctypes.c_void_p)]
+
+
+def _ahead_chain(ahead):
+    """ahead: one (weights, K, levels, levels_buf) tuple or a list of them -> (address of the first descriptor or None,
+    objects to keep alive)."""
+    if ahead is None:
+        return None, None
+    items = ahead if isinstance(ahead, list) else [ahead]
+    keep, nxt = [], None
+    for nw, nK, nlv, nbuf in reversed(items):
+        arr = _outputs_array(nw)
+        d = DecodeAhead(ctypes.addressof(arr), len(nw), nK, nlv, 0, _dev(nbuf).data_ptr(), nbuf.numel(), nxt)
+        keep += [arr, d]
+        nxt = ctypes.addressof(d)
+    return nxt, keep
 
 
 def _outputs_array(weights, ys=None, accs=None):
@@ -324,7 +340,8 @@ def qift_forward_multi(X, had_block: int, weights, levels: int, clip_ratio: floa
     """One activation X [M,K], several products: weights = [(packed, s_n), ...] (1..4) -> ([Y_i [M,N_i]], [acc_i or None]).
     levels_buf: uint8 tensor of qift_levels_bytes(K, weights) bytes (allocated when omitted; needed for M > 128);
     levels_ready: it already holds these weights' decoded levels (written through a previous call's `ahead`);
-    ahead = (next_weights, next_K, next_levels, next_levels_buf): decode the next call's codes during this one."""
+    ahead = (next_weights, next_K, next_levels, next_levels_buf), or a list of such tuples: decode later calls' codes
+    during this one."""
     _dev(X)
     M, K = X.shape
     ys = outs if outs is not None else [torch.empty((M, s_n.shape[0]), dtype=out_dtype, device=X.device) for _, s_n in weights]
@@ -337,14 +354,10 @@ def qift_forward_multi(X, had_block: int, weights, levels: int, clip_ratio: floa
     if levels_buf is None:
         assert not levels_ready
         levels_buf = torch.empty(max(qift_levels_bytes(K, weights), 256), dtype=torch.uint8, device=X.device)
-    ah, keep = None, None
-    if ahead is not None:
-        nw, nK, nlv, nbuf = ahead
-        keep = _outputs_array(nw)
-        ah = DecodeAhead(ctypes.addressof(keep), len(nw), nK, nlv, 0, _dev(nbuf).data_ptr(), nbuf.numel())
+    ah, keep = _ahead_chain(ahead)
     _check(L.qift_forward_multi(_ptr(X), _dt(X), M, K, had_block, clip_ratio, levels, ctypes.addressof(arr), len(weights),
                                 _dt(ys[0]), _ptr(_dev(scratch)), scratch.numel(), _ptr(_dev(levels_buf)), levels_buf.numel(),
-                                1 if levels_ready else 0, None if ah is None else ctypes.addressof(ah), _stream()),
+                                1 if levels_ready else 0, ah, _stream()),
            "qift_forward_multi")
     return ys, accs
 
@@ -363,14 +376,10 @@ def qift_linear_multi(q_a, s_a, weights, levels: int, out_dtype=torch.float32, w
     if levels_buf is None:
         assert not levels_ready
         levels_buf = torch.empty(max(qift_levels_bytes(K, weights), 256), dtype=torch.uint8, device=q_a.device)
-    ah, keep = None, None
-    if ahead is not None:
-        nw, nK, nlv, nbuf = ahead
-        keep = _outputs_array(nw)
-        ah = DecodeAhead(ctypes.addressof(keep), len(nw), nK, nlv, 0, _dev(nbuf).data_ptr(), nbuf.numel())
+    ah, keep = _ahead_chain(ahead)
     _check(L.qift_linear_multi(_ptr(q_a), _ptr(s_a), M, K, levels, ctypes.addressof(arr), len(weights), _dt(ys[0]), _ptr(ws),
                                ws.numel(), _ptr(_dev(levels_buf)), levels_buf.numel(), 1 if levels_ready else 0,
-                               None if ah is None else ctypes.addressof(ah), _stream()), "qift_linear_multi")
+                               ah, _stream()), "qift_linear_multi")
     return ys, accs
 
 

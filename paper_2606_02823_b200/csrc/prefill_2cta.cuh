@@ -73,6 +73,7 @@ __host__ __device__ constexpr size_t pair_smem_bytes() {
 }
 
 constexpr int kPairMaxSegments = 4;
+constexpr int kPairMaxJobs = 8;   // matrices decoded on the side in one launch (they may belong to several later calls)
 constexpr int kSideUnitRows = 8, kSideUnitWords = 128;
 
 struct PairSegment {
@@ -93,7 +94,7 @@ struct alignas(64) PairParams {
     CUtensorMap map_a;                    // q_a [M, K]
     CUtensorMap map_b[kPairMaxSegments];  // decoded weights [N_i, K], box = BN / 2 rows
     PairSegment seg[kPairMaxSegments];
-    SideJob job[kPairMaxSegments];
+    SideJob job[kPairMaxJobs];
     const float* s_a;
     uint64_t wait_limit_ns;  // bound of every device-side wait of the launch; 0 = the default (kWaitLimitNs)
     int M, K, y_bf16;
@@ -151,7 +152,7 @@ __device__ __forceinline__ void side_jobs(const PairParams& p, int t, int group)
     auto job_of = [&](int u) {
         int ji = 0;
 #pragma unroll
-        for (int i = 1; i < kPairMaxSegments; ++i)
+        for (int i = 1; i < kPairMaxJobs; ++i)
             if (i < p.njobs && u >= p.job[i].unit0) ji = i;
         return ji;
     };

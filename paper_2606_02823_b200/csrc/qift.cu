@@ -334,12 +334,12 @@ struct PairCall {
         int32_t* acc_debug;
         int N;
     } seg[kPairMaxSegments];
-    int njobs, job_K;
+    int njobs;
     struct {
         const uint32_t* packed;
         int8_t* out;
-        int N, levels;
-    } job[kPairMaxSegments];
+        int N, K, levels;
+    } job[kPairMaxJobs];
     uint64_t wait_limit_ns;
     int starve;
 };
@@ -356,7 +356,7 @@ int launch_gemm_pairs(const PairParams& pp, int tiles, cudaStream_t st) {
 }
 
 int run_pair_gemm(const PairCall& c, cudaStream_t st) {
-    if (c.nseg < 1 || c.nseg > kPairMaxSegments || c.njobs < 0 || c.njobs > kPairMaxSegments) return QIFT_ERR_INVALID_ARG;
+    if (c.nseg < 1 || c.nseg > kPairMaxSegments || c.njobs < 0 || c.njobs > kPairMaxJobs) return QIFT_ERR_INVALID_ARG;
     PairParams pp = {};
     int widths[kPairMaxSegments];
     for (int i = 0; i < c.nseg; ++i) widths[i] = c.seg[i].N;
@@ -373,7 +373,7 @@ int run_pair_gemm(const PairCall& c, cudaStream_t st) {
     pp.wait_limit_ns = c.wait_limit_ns, pp.starve = c.starve;
     int units = 0;
     for (int i = 0; i < c.njobs; ++i) {
-        const int words = c.job_K / codes_per_word(c.job[i].levels);
+        const int words = c.job[i].K / codes_per_word(c.job[i].levels);
         pp.job[i] = SideJob{c.job[i].packed, c.job[i].out, c.job[i].N, words, units, c.job[i].levels};
         units += ((c.job[i].N + kSideUnitRows - 1) / kSideUnitRows) * ((words + kSideUnitWords - 1) / kSideUnitWords);
     }
@@ -864,14 +864,16 @@ static int check_outputs_and_ahead(int M, int K, int levels, const qift_linear_o
         if (!aligned16(outputs[i].packed) || !aligned16(outputs[i].s_n) || !aligned16(outputs[i].Y) ||
             (outputs[i].acc_debug && !aligned16(outputs[i].acc_debug)))
             return QIFT_ERR_ALIGNMENT;
-    if (ahead) {
-        if (!multi_outputs_ok(ahead->outputs, ahead->count, false) || ahead->K <= 0 || !valid_levels(ahead->levels) || !ahead->levels_buf)
+    int ahead_outputs = 0;
+    for (const qift_decode_ahead* a = ahead; a; a = a->next) {
+        if (!multi_outputs_ok(a->outputs, a->count, false) || a->K <= 0 || !valid_levels(a->levels) || !a->levels_buf)
             return QIFT_ERR_INVALID_ARG;
-        if (ahead->K % 16 != 0 || !whole_words(ahead->K, ahead->levels)) return QIFT_ERR_UNSUPPORTED_SHAPE;
-        if (ahead->levels_bytes < qift_levels_bytes(ahead->K, ahead->outputs, ahead->count)) return QIFT_ERR_WORKSPACE;
-        if ((reinterpret_cast<uintptr_t>(ahead->levels_buf) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
-        for (int i = 0; i < ahead->count; ++i)
-            if (!aligned16(ahead->outputs[i].packed)) return QIFT_ERR_ALIGNMENT;
+        if ((ahead_outputs += a->count) > kPairMaxJobs) return QIFT_ERR_INVALID_ARG;
+        if (a->K % 16 != 0 || !whole_words(a->K, a->levels)) return QIFT_ERR_UNSUPPORTED_SHAPE;
+        if (a->levels_bytes < qift_levels_bytes(a->K, a->outputs, a->count)) return QIFT_ERR_WORKSPACE;
+        if ((reinterpret_cast<uintptr_t>(a->levels_buf) & 255u) != 0) return QIFT_ERR_ALIGNMENT;
+        for (int i = 0; i < a->count; ++i)
+            if (!aligned16(a->outputs[i].packed)) return QIFT_ERR_ALIGNMENT;
     }
     return QIFT_OK;
 }
@@ -889,10 +891,10 @@ static int linear_multi_impl(const int8_t* q_a, const float* s_a, int M, int K, 
                              outputs[i].acc_debug, workspace, workspace_bytes, QIFT_ROUTE_AUTO, stream);
             if (rc != QIFT_OK) return rc;
         }
-        if (ahead)
-            for (int i = 0; i < ahead->count; ++i) {
-                int8_t* out = static_cast<int8_t*>(ahead->levels_buf) + levels_offset(ahead->K, ahead->outputs, i);
-                rc = run_expand(ahead->outputs[i].packed, ahead->levels, ahead->outputs[i].N, ahead->K, out, st);
+        for (const qift_decode_ahead* a = ahead; a; a = a->next)
+            for (int i = 0; i < a->count; ++i) {
+                int8_t* out = static_cast<int8_t*>(a->levels_buf) + levels_offset(a->K, a->outputs, i);
+                rc = run_expand(a->outputs[i].packed, a->levels, a->outputs[i].N, a->K, out, st);
                 if (rc != QIFT_OK) return rc;
             }
         return QIFT_OK;
@@ -910,20 +912,24 @@ static int linear_multi_impl(const int8_t* q_a, const float* s_a, int M, int K, 
         c.seg[i].wexp = wexp, c.seg[i].s_n = outputs[i].s_n, c.seg[i].Y = outputs[i].Y, c.seg[i].acc_debug = outputs[i].acc_debug;
         c.seg[i].N = outputs[i].N;
     }
-    const bool ahead_in_gemm = ahead && ahead->levels != QIFT_LEVELS_INT3;  // the side warps decode one-plane layouts only
-    if (ahead_in_gemm) {
-        c.njobs = ahead->count, c.job_K = ahead->K;
-        for (int i = 0; i < ahead->count; ++i) {
-            c.job[i].packed = ahead->outputs[i].packed, c.job[i].N = ahead->outputs[i].N, c.job[i].levels = ahead->levels;
-            c.job[i].out = static_cast<int8_t*>(ahead->levels_buf) + levels_offset(ahead->K, ahead->outputs, i);
+    // the side warps decode one-plane layouts; three-bit codes are decoded by separate launches after the GEMM
+    for (const qift_decode_ahead* a = ahead; a; a = a->next) {
+        if (a->levels == QIFT_LEVELS_INT3) continue;
+        for (int i = 0; i < a->count; ++i) {
+            auto& j = c.job[c.njobs++];
+            j.packed = a->outputs[i].packed, j.N = a->outputs[i].N, j.K = a->K, j.levels = a->levels;
+            j.out = static_cast<int8_t*>(a->levels_buf) + levels_offset(a->K, a->outputs, i);
         }
     }
     rc = run_pair_gemm(c, st);
-    if (rc != QIFT_OK || !ahead || ahead_in_gemm) return rc;
-    for (int i = 0; i < ahead->count; ++i) {
-        int8_t* out = static_cast<int8_t*>(ahead->levels_buf) + levels_offset(ahead->K, ahead->outputs, i);
-        rc = run_expand(ahead->outputs[i].packed, ahead->levels, ahead->outputs[i].N, ahead->K, out, st);
-        if (rc != QIFT_OK) return rc;
+    if (rc != QIFT_OK) return rc;
+    for (const qift_decode_ahead* a = ahead; a; a = a->next) {
+        if (a->levels != QIFT_LEVELS_INT3) continue;
+        for (int i = 0; i < a->count; ++i) {
+            int8_t* out = static_cast<int8_t*>(a->levels_buf) + levels_offset(a->K, a->outputs, i);
+            rc = run_expand(a->outputs[i].packed, a->levels, a->outputs[i].N, a->K, out, st);
+            if (rc != QIFT_OK) return rc;
+        }
     }
     return QIFT_OK;
 }

@@ -89,6 +89,33 @@ def test_decode_ahead_chain(M):
     clean()
 
 
+def test_one_call_decodes_for_two_later_calls():
+    # call 1 carries the decoding for calls 2 and 3 (other K, other level sets, five matrices in all); both then run on
+    # ready levels; a list of more than eight matrices is refused
+    M, K1, K2, K3 = 700, 512, 768, 256
+    h1, g1 = make_weights(111, (520, 128), K1, qift.MNZ)
+    h2, g2 = make_weights(121, (300, 136), K2, qift.INT4)
+    h3, g3 = make_weights(131, (136, 136, 264), K3, qift.SYM)
+    x1, _ = synth.activations(141, M, K1, 5)
+    x2, _ = synth.activations(142, M, K2, 7)
+    x3, _ = synth.activations(143, M, K3, 3)
+    b1 = torch.full((qift.qift_levels_bytes(K1, g1),), 0x55, dtype=torch.uint8, device="cuda")
+    b2 = torch.full((qift.qift_levels_bytes(K2, g2),), 0x55, dtype=torch.uint8, device="cuda")
+    b3 = torch.full((qift.qift_levels_bytes(K3, g3),), 0x55, dtype=torch.uint8, device="cuda")
+    y1, a1 = qift.qift_forward_multi(dev(x1), synth.had_block_for(K1), g1, qift.MNZ, CLIP, want_acc=True, levels_buf=b1,
+                                     ahead=[(g2, K2, qift.INT4, b2), (g3, K3, qift.SYM, b3)])
+    y2, a2 = qift.qift_forward_multi(dev(x2), synth.had_block_for(K2), g2, qift.INT4, CLIP, want_acc=True, levels_buf=b2, levels_ready=True)
+    y3, a3 = qift.qift_forward_multi(dev(x3), synth.had_block_for(K3), g3, qift.SYM, CLIP, want_acc=True, levels_buf=b3, levels_ready=True)
+    check(h1, qift.MNZ, x1, synth.had_block_for(K1), y1, a1, False)
+    check(h2, qift.INT4, x2, synth.had_block_for(K2), y2, a2, False)
+    check(h3, qift.SYM, x3, synth.had_block_for(K3), y3, a3, False)
+    with pytest.raises(qift.QiftError) as e:
+        qift.qift_forward_multi(dev(x1), synth.had_block_for(K1), g1, qift.MNZ, CLIP, levels_buf=b1,
+                                ahead=[(g3, K3, qift.SYM, b3)] * 3)      # nine matrices
+    assert e.value.status == qift.ERR_INVALID_ARG
+    clean()
+
+
 def test_forward_multi_rejects_bad_arguments():
     K, lv = 256, qift.MNZ
     host, gpu = make_weights(5, (128,), K, lv)

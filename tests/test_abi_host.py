@@ -90,6 +90,23 @@ def test_bad_arguments_are_rejected_before_any_launch(L):
     assert L.qift_linear_route(p, p, 0, p, p, 32, 16, 256, p, 0, None, None, 0, qift.ROUTE_DECODE, None) \
         == qift.ERR_UNSUPPORTED_SHAPE
     assert L.qift_linear_route(p, p, 0, p, p, 1, 16, 256, p, 0, None, None, 0, 9, None) == qift.ERR_INVALID_ARG
+    # three-bit codes: K in whole high words; only the routes that serve the level set; packed size 3 bits per weight
+    assert L.qift_pack_weights(p, 16, 48, qift.INT3, 1, p, p, None) == qift.ERR_UNSUPPORTED_SHAPE
+    assert L.qift_w3a4_linear(p, p, p, p, 1, 16, 48, p, 0, None, None, 0, None) == qift.ERR_UNSUPPORTED_SHAPE
+    assert L.qift_linear_route(p, p, qift.INT3, p, p, 4, 16, 256, p, 0, None, None, 0, qift.ROUTE_DECODE, None) \
+        == qift.ERR_UNSUPPORTED_SHAPE
+    assert L.qift_w3a4_linear(p, p, p, p, 64, 16, 256, p, 0, None, None, 0, None) == qift.ERR_WORKSPACE
+    assert L.qift_packed_bytes(4096, 4096, qift.INT3) == 4096 * 4096 * 3 // 8
+    # grouped plans: token-row limits per level set; plans that need tensor maps want a 128-byte aligned device plan
+    prob = binding.GroupProblem(4096, 4096, 4096, 4096, 4096, 4096, None, 256, 256, 256, 0)
+    n = L.qift_group_plan_bytes(1)
+    host = ctypes.create_string_buffer(n + 256)
+    hp = ctypes.c_void_p((ctypes.addressof(host) + 255) & ~255)
+    plan = lambda M, lv, dev: L.qift_group_plan(ctypes.byref(prob), 1, M, lv, 0, 0, 0.9, hp, ctypes.c_void_p(dev), n, None)
+    assert plan(129, qift.MNZ, 4096) == qift.ERR_UNSUPPORTED_SHAPE
+    assert plan(65, qift.POT, 4096) == qift.ERR_UNSUPPORTED_SHAPE
+    assert plan(17, qift.INT3, 4096) == qift.ERR_UNSUPPORTED_SHAPE
+    assert plan(64, qift.MNZ, 4096 + 64) == qift.ERR_ALIGNMENT
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

@@ -675,7 +675,7 @@ def run_batched_decode(torch, qift, L, device, gen, args, ceilings):
             rows.append({"levels": name, "M": M, "ms_per_step": round(ms, 5), "tokens_per_s": round(M / (ms * 1e-3), 1),
                          "value": round(gbs, 1), "unit": "GB/s", "pct_of_8TBs": round(100 * gbs / 8000.0, 1),
                          "frac_of_read_only_ceiling": round(gbs / ceilings["hbm_read_only_gbs"], 3),
-                         "kernel": "linear_tc_kernel (tcgen05, weights in tensor memory)" if (M > 32 and lv != qift.POT)
+                         "kernel": "linear_tc_kernel (tcgen05, weights in tensor memory)" if M > 32
                                    else "linear_grouped_wide_kernel (mma.sync)" if (M > 1 or lv == qift.POT) else "linear_grouped_kernel (mma.sync)"})
             del plan
         del base

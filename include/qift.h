@@ -273,8 +273,7 @@ int qift_linear_multi(const int8_t* q_a, const float* s_a, int M, int K, int lev
                       size_t levels_bytes, int levels_ready, const qift_decode_ahead* ahead, void* stream);
 
 /* ---- Grouped decode path -----------------------------------------------------------------------
- * One persistent launch serves a list of independent layer problems that share M (<= 128 token rows; PoT <= 64,
- * INT3 <= 16),
+ * One persistent launch serves a list of independent layer problems that share M (<= 128 token rows; INT3 <= 16),
  * the level set, the dtypes and the clip ratio -- e.g. all linear modules of one decode step.  A W2
  * matrix is only 1-15 MB, far too little for one launch to reach an HBM steady state; the grouped
  * kernel streams the whole list back to back.  (No counterpart in the paper: it describes no kernels.)
@@ -291,8 +290,7 @@ int qift_linear_multi(const int8_t* q_a, const float* s_a, int M, int K, int lev
  * Problems must not alias each other's Y, nor each other's q_a / s_a with one exception: modules that
  * read the SAME activation (q/k/v; gate/up) may name the same X, q_a, s_a (same K and had_block); the
  * plan then quantizes that activation once and every such product reads it.  K % 256 == 0 (two-bit sets, INT3) or
- * K % 128 == 0 (INT4), K <= 16384.  INT3 plans take up to 16 token rows, PoT plans up to 64 (the tcgen05 kernel that
- * serves 33 .. 128 rows takes the sets that are affine in the code). */
+ * K % 128 == 0 (INT4), K <= 16384.  INT3 plans take up to 16 token rows. */
 typedef struct qift_group_problem {
     const void* X;          /* dev [M,K] fp32 or bf16                         */
     const uint32_t* packed; /* dev, from qift_pack_weights                    */

@@ -109,7 +109,14 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // Operand words of one k-block (128 codes) of a channel row.
 template <int LV>
 __device__ __forceinline__ void tc_operands(const uint32_t* w, uint32_t (&o)[32]) {
-    if constexpr (LV == QIFT_LEVELS_INT4) {  // 16 words of 8 nibbles
+    if constexpr (LV == QIFT_LEVELS_POT) {   // 8 words of 16 two-bit codes: the levels themselves, by table lookup
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            uint32_t a[4];
+            pot_lut_operands(w[i], a);
+            o[4 * i] = a[0], o[4 * i + 1] = a[1], o[4 * i + 2] = a[2], o[4 * i + 3] = a[3];
+        }
+    } else if constexpr (LV == QIFT_LEVELS_INT4) {  // 16 words of 8 nibbles
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
             o[2 * i] = (w[i] ^ 0x88888888u) & 0x0f0f0f0fu;
@@ -129,6 +136,7 @@ __device__ __forceinline__ void tc_operands(const uint32_t* w, uint32_t (&o)[32]
 
 template <int LV>
 __device__ __forceinline__ int tc_level_sum(int d, int sq) {
+    if constexpr (LV == QIFT_LEVELS_POT) return d;   // the operands were the levels, the activations unscaled
     if constexpr (LV == QIFT_LEVELS_MNZ) return 2 * (d >> 2) - 3 * sq;
     if constexpr (LV == QIFT_LEVELS_SYM) return (d >> 2) - 2 * sq;
     return (d >> 4) - 8 * sq;  // INT4
@@ -149,8 +157,8 @@ linear_tc_kernel(const GroupParams gp) {
     constexpr int kTcWSlots = tc_wslots(NTOK);
     static_assert(2 * DBUF <= kTcACol0, "two accumulator buffers fit below the operand ring");
     static_assert(KPS * R <= 4, "a ring slot must always return to the same expander warp");
-    // D = s32, A = u8 (operand bytes from tensor memory), B = s8 (activations), both K-major, N = NTOK, M = 128
-    constexpr uint32_t IDESC = (2u << 4) | (0u << 7) | (1u << 10) | (static_cast<uint32_t>(NTOK >> 3) << 17) |
+    // D = s32, A = u8 (operand bytes from tensor memory; PoT: s8, the levels), B = s8 (activations), both K-major, N = NTOK, M = 128
+    constexpr uint32_t IDESC = (2u << 4) | ((LV == QIFT_LEVELS_POT ? 1u : 0u) << 7) | (1u << 10) | (static_cast<uint32_t>(NTOK >> 3) << 17) |
                                (static_cast<uint32_t>(kTcRows >> 4) << 24);
     using Cursor = GroupCursor<PER, 16>;
 

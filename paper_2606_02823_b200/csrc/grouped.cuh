@@ -77,6 +77,10 @@ __host__ __device__ __forceinline__ int swizzled_group(int piece, int m, int two
     const int block_pair = two_bit ? ((piece >> 3) & 1) << 1 : 0;   // bit 1 of the 64-byte block index -> bit 1 of the group index
     return piece ^ block_pair ^ (m & 1);
 }
+struct RowMajorPotDst {   // row-major, bytes of each 16-byte group in pot_lut_order (PoT on the tcgen05 kernel)
+    int8_t* q_row;
+    __device__ __forceinline__ void store(int q, uint4 v) const { reinterpret_cast<uint4*>(q_row)[q] = pot_lut_order(v); }
+};
 struct ChunkMajorDst {
     int8_t* q_a;
     int m, M, K, cb, pot_lut, two_bit;
@@ -108,6 +112,7 @@ quantize_act_grouped_kernel(const GroupProblemDev* __restrict__ problems, int* _
     // 32-bit word i of a 16-byte group = code plane (two-bit: i; INT4: i & 1); even planes are prescaled
     const float mult = q_pot_lut ? 1.0f : int4_weights ? 16.0f : 4.0f;
     int total = q_chunk_bytes ? quantize_row<true>(row, K, sc, ChunkMajorDst{P.q_a, static_cast<int>(m), M, K, q_chunk_bytes, q_pot_lut, int4_weights ? 0 : 1}, mult, 1.0f)
+                : q_pot_lut   ? quantize_row<true>(row, K, sc, RowMajorPotDst{P.q_a + m * K}, mult, 1.0f)
                               : quantize_row<true>(row, K, sc, RowMajorDst{P.q_a + m * K}, mult, 1.0f);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);

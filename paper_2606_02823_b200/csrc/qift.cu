@@ -502,7 +502,7 @@ inline size_t decode_rows_scratch(int M, int K) { return ((static_cast<size_t>(M
 // Grouped plans: the row-split mma.sync kernel up to 32 token rows (PoT: up to 64), the tcgen05 weight-streaming kernel
 // from 33 to 128, where it is the faster one (16 LLaMA-2-7B layers, product kernel, MNZ / INT4: 32 rows 1.9 / 2.8 TB/s
 // against 2.8 / 4.5 on mma.sync; 64 rows 1.8 / 3.2 against 1.3 / 2.5).
-inline bool tc_rows_applies(int lv, int M) { return lv != QIFT_LEVELS_POT && lv != QIFT_LEVELS_INT3 && M > 32 && M <= kGroupMaxM; }
+inline bool tc_rows_applies(int lv, int M) { return lv != QIFT_LEVELS_INT3 && M > 32 && M <= kGroupMaxM; }
 inline int tc_tokens(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }   // the tensor-core N of that kernel
 inline int tc_rows_per_item(int M, int lv) { return kTcRows * tc_tiles_per_item(tc_tokens(M), codes_per_word(lv)); }
 constexpr int kInt3MaxRows = 16;   // three-bit codes on the row-split kernel: six accumulator sets per token tile, two token tiles
@@ -996,7 +996,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
         return QIFT_ERR_INVALID_ARG;
     if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return QIFT_ERR_INVALID_ARG;
     if (M > kGroupMaxM || (levels == QIFT_LEVELS_INT3 && M > kInt3MaxRows)) return QIFT_ERR_UNSUPPORTED_SHAPE;
-    if (M > kWideMaxM && !tc_rows_applies(levels, M)) return QIFT_ERR_UNSUPPORTED_SHAPE;   // 65 .. 128 rows: the tcgen05 kernel's sets only
+    if (M > kWideMaxM && !tc_rows_applies(levels, M)) return QIFT_ERR_UNSUPPORTED_SHAPE;   // 65 .. 128 rows: the tcgen05 kernel only
     if (plan_bytes < qift_group_plan_bytes(count)) return QIFT_ERR_WORKSPACE;
     if (!aligned16(plan_dev) || !aligned16(plan_host)) return QIFT_ERR_ALIGNMENT;
     if (tc_rows_applies(levels, M) && (reinterpret_cast<uintptr_t>(plan_dev) & 127u) != 0) return QIFT_ERR_ALIGNMENT;  // tensor maps
@@ -1047,7 +1047,7 @@ int qift_group_plan(const qift_group_problem* problems, int count, int M, int le
     h->max_k = max_k;
     h->any_kron = any_kron;
     // the row-split kernel stages one K-chunk of all tokens per copy: its q_a is chunk-major (ChunkMajorDst)
-    h->q_pot_lut = (rows_per_item >= kWideRows && levels == QIFT_LEVELS_POT && M > 8) ? 1 : 0;  // the kernel's POT_LUT
+    h->q_pot_lut = (rows_per_item >= kWideRows && levels == QIFT_LEVELS_POT && M > 8) ? 1 : 0;  // the kernel's POT_LUT (both kernels from 9 rows)
     h->q_chunk_bytes = (rows_per_item >= kWideRows) ? wide_chunk_words(rows_per_item / 16, wide_token_tiles(M), levels) * codes_per_word(levels) : 0;
     h->reserved[0] = use_tc ? 1 : 0;
     if (use_tc) h->q_chunk_bytes = 0;  // that kernel reads q_a row-major (prescaled even planes, as the K-split kernel does)
@@ -1136,9 +1136,7 @@ int launch_grouped_wide(const GroupHeader* h, const GroupProblemDev* host, const
 template <int LV, int NTOK>
 int launch_tc(const GroupHeader* h, const GroupProblemDev* host, const GroupProblemDev* dev, const int* sumq, cudaStream_t st,
               bool single = false) {
-    if constexpr (LV == QIFT_LEVELS_POT) {
-        return QIFT_ERR_INVALID_ARG;
-    } else {
+    {
         constexpr int R = tc_tiles_per_item(NTOK, codes_per_word(LV));
         auto kernel = linear_tc_kernel<LV, NTOK, R>;
         for (int first = 0; first < h->count; first += kGroupSlice) {

@@ -104,7 +104,6 @@ def test_bad_arguments_are_rejected_before_any_launch(L):
     hp = ctypes.c_void_p((ctypes.addressof(host) + 255) & ~255)
     plan = lambda M, lv, dev: L.qift_group_plan(ctypes.byref(prob), 1, M, lv, 0, 0, 0.9, hp, ctypes.c_void_p(dev), n, None)
     assert plan(129, qift.MNZ, 4096) == qift.ERR_UNSUPPORTED_SHAPE
-    assert plan(65, qift.POT, 4096) == qift.ERR_UNSUPPORTED_SHAPE
     assert plan(17, qift.INT3, 4096) == qift.ERR_UNSUPPORTED_SHAPE
     assert plan(64, qift.MNZ, 4096 + 64) == qift.ERR_ALIGNMENT
 

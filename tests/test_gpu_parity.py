@@ -383,8 +383,6 @@ def test_grouped_forward(name, M):
     # a ragged list: different N (incl. not a multiple of the row block), different K (incl. a
     # partial last chunk), more items than CTAs
     lv = LEVELS[name][0]
-    if M > 64 and name == "POT":
-        pytest.skip("PoT plans end at 64 token rows (rejection checked in test_grouped_rejects_bad_plans)")
     shapes = [(256, 256), (40, 512), (100, 2304), (4000, 256), (48, 4096), (130, 2560), (16, 11008), (2400, 256),
               (9600, 256)]
     probs, refs = [], []
@@ -434,7 +432,7 @@ def test_grouped_forward_long_list(name, M):
         check_outputs(y, acc, y_ref, acc_ref, False)
 
 
-@pytest.mark.parametrize("name", ["MNZ", "SYM", "INT4"])
+@pytest.mark.parametrize("name", ["MNZ", "SYM", "INT4", "POT"])
 @pytest.mark.parametrize("M", [33, 64, 96, 128])
 def test_grouped_forward_tensor_memory_kernel_many_items(name, M):
     # 33 .. 128 token rows of a plan run on the tcgen05 kernel whose weight operand lives in tensor memory.  More
@@ -541,9 +539,6 @@ def test_grouped_rejects_bad_plans():
     x129 = torch.zeros((129, 256), device="cuda")
     with pytest.raises(qift.QiftError) as e:
         qift.qift_group_plan([(x129, packed, s_n, 256)], qift.MNZ)      # M > 128
-    assert e.value.status == qift.ERR_UNSUPPORTED_SHAPE
-    with pytest.raises(qift.QiftError) as e:
-        qift.qift_group_plan([(x129[:65], packed, s_n, 256)], qift.POT)  # PoT plans end at 64 rows (packed bytes are not read)
     assert e.value.status == qift.ERR_UNSUPPORTED_SHAPE
     L = qift.lib()
     assert L.qift_group_forward(None, None, None) == qift.ERR_INVALID_ARG

@@ -1,4 +1,4 @@
-// Weight-streaming product for 9 .. 128 token rows on the tcgen05 tensor cores (MNZ, SYM, INT4).
+// Weight-streaming product for 9 .. 128 token rows on the tcgen05 tensor cores (the two-bit sets and INT4).
 //
 // With more than eight token rows the mma.sync decode kernels are bound by the issue rate of the legacy tensor
 // instructions and by shared-memory reads of the activations, not by HBM.  Here the roles of the operands are
@@ -14,8 +14,9 @@
 //               128 x N x 32 instruction for N <= 64 is this issue cost, not tensor time), so the (k-block, tile) units are
 //               dealt alternately to two threads.  Integer accumulation commutes and every instruction accumulates
 //               (the epilogue leaves the accumulator columns zeroed), so the two streams need no order between them.
-//   warps 2-5   epilogue: tcgen05.ld (lane = channel, column = token), level map with the token sums, the two
-//               scale multiplies, stores (a warp's 32 lanes write 32 consecutive channels of a token row)
+//   warps 2-5, 15-18   epilogue, two warps per tensor-memory lane quarter on alternate 16-token chunks: tcgen05.ld
+//               (lane = channel, column = token), level map with the token sums, the two scale multiplies, stores (a
+//               warp's 32 lanes write 32 consecutive channels of a token row), zeros written back to the columns read
 //   warps 6-13  expanders, two per tensor-memory lane quarter (alternate 16-word slices): each streams the packed
 //               words of ITS 32 channel rows with cp.async into a private shared-memory ring (16-byte chunks XOR-swizzled by row:
 //               conflict-free 128-bit reads; up to eight 2 KB units in flight per warp, running ahead across items), turns
@@ -25,7 +26,9 @@
 // Operand bytes are the stored codes times a place value (two-bit: planes 0 / 2 times 1, planes 1 / 3 times 4;
 // INT4: nibble ^ 8 times 1 / 16); the activations come PRESCALED (bytes of the even planes hold 4 q, INT4: plane
 // 0 holds 16 q), so every product carries the same factor (4 or 16), which an arithmetic shift removes exactly;
-// the affine level map is undone with sum_k q as everywhere else.  The accumulators (R blocks x tokens <= 128
+// the affine level map is undone with sum_k q as everywhere else.  PoT is not affine in the code: its operand bytes are
+// the levels themselves (byte-permute table lookup, a signed A operand) against unscaled activations whose bytes the
+// quantizer wrote in the matching order.  The accumulators (R blocks x tokens <= 128
 // columns) are double-buffered in tensor memory: 2 x 128 columns + 8 x 32 operand columns = all 512.
 // Work items (problem, 128-channel block) are dealt round-robin to one persistent CTA per SM, as in the other
 // grouped kernels.  Every wait is bounded; no TMA multicast.

@@ -300,6 +300,10 @@ def run_gpu(args):
     sampler = ClockSampler(local)
     sampler.start()
     ms_grp = timed(run_grp, args.steps, args.warmup)
+    # the roofline's kernel-only timing starts from the same thermal state as the headline (half a second of idle): timed
+    # directly after it, it runs at the lower clocks of a board already at its power cap (see `sustained`)
+    torch.cuda.synchronize()
+    time.sleep(0.5)
     ms_grp_prod = timed(run_grp_prod, args.steps, args.warmup)
     pc_steps = max(3, min(args.steps, 50))
     ms_full = timed(run_full, pc_steps, args.warmup)
